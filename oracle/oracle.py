@@ -1,0 +1,294 @@
+"""ctypes front end of the CPU oracle (``hann_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: the plain, slow RNS-CKKS reference that the CUDA library is checked
+against.  Nothing here is imported by the product package; it imports nothing from it either.
+
+Every polynomial crossing this interface is in the canonical exchange layout: coefficient
+domain, natural order, residues in [0, q_i), ``uint64``, index order ``[poly][limb][coeff]``.
+CRT reconstruction (Sec. 2, "The round trip": the client decrypts the scores) is done here with
+python integers, the most obviously exact arithmetic available.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "hann_oracle.c")
+_LIB = os.path.join(_HERE, "libhann_oracle.so")
+
+u64p = C.POINTER(C.c_uint64)
+i64p = C.POINTER(C.c_int64)
+i8p = C.POINTER(C.c_int8)
+f32p = C.POINTER(C.c_float)
+f64p = C.POINTER(C.c_double)
+i32p = C.POINTER(C.c_int)
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (no FMA contraction: the encode order of operations is pinned)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".%d.tmp" % os.getpid()
+        subprocess.check_call(
+            ["gcc", "-O2", "-ffp-contract=off", "-fopenmp", "-shared", "-fPIC", "-o", tmp, _SRC, "-lquadmath", "-lm"]
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.orc_create.restype = C.c_void_p
+        _lib.orc_create.argtypes = [C.c_int, C.c_int, u64p, C.c_int, C.c_int, C.c_int]
+        _lib.orc_destroy.argtypes = [C.c_void_p]
+        _lib.orc_get_psi.restype = C.c_uint64
+        _lib.orc_get_psi.argtypes = [C.c_void_p, C.c_int]
+        _lib.orc_galois.restype = C.c_long
+        _lib.orc_galois.argtypes = [C.c_void_p, C.c_int]
+        _lib.orc_is_prime.argtypes = [C.c_uint64]
+        _lib.orc_find_primes.argtypes = [C.c_int, C.c_int, C.c_int, u64p]
+        _lib.orc_automorphism.argtypes = [C.c_void_p, C.c_int, C.c_long, u64p, u64p]
+        _lib.orc_automorphism_ntt.argtypes = [C.c_void_p, C.c_long, u64p, u64p]
+        _lib.orc_decode.argtypes = [C.c_void_p, f64p, C.c_double, f64p, f64p]
+    return _lib
+
+
+def _p(a, typ):
+    return a.ctypes.data_as(typ)
+
+
+def _u64(a):
+    a = np.ascontiguousarray(a, dtype=np.uint64)
+    return a
+
+
+def find_primes(bits: int, logstep: int, count: int):
+    out = np.zeros(count, dtype=np.uint64)
+    k = lib().orc_find_primes(bits, logstep, count, _p(out, u64p))
+    return [int(x) for x in out[:k]]
+
+
+def is_prime(x: int) -> bool:
+    return bool(lib().orc_is_prime(C.c_uint64(x)))
+
+
+class Oracle:
+    """One parameter set: ring 2^logN, ciphertext primes q (list), special prime p, scale 2^log_scale,
+    padded dimension R, baby-step count B (G = R/B giant steps)."""
+
+    def __init__(self, logN, q, p, log_scale, R, B):
+        self.logN, self.N, self.n = logN, 1 << logN, 1 << (logN - 1)
+        self.L = len(q)
+        self.q = [int(x) for x in q]
+        self.p = int(p)
+        self.mods = self.q + [self.p]
+        self.log_scale, self.R, self.B, self.G = log_scale, R, B, R // B
+        m = np.array(self.mods, dtype=np.uint64)
+        self._h = lib().orc_create(logN, self.L, _p(m, u64p), log_scale, R, B)
+        if not self._h:
+            raise ValueError("invalid oracle parameters")
+        self.Q = 1
+        for x in self.q:
+            self.Q *= x
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            lib().orc_destroy(C.c_void_p(self._h))
+            self._h = None
+
+    @property
+    def h(self):
+        return C.c_void_p(self._h)
+
+    # ---- tables and index maps
+    def tables(self):
+        n = self.n
+        nh = max(n // 2, 1)
+        Tr, Ti = np.zeros(nh), np.zeros(nh)
+        Ur, Ui = np.zeros(n), np.zeros(n)
+        g5, u = np.zeros(n, dtype=np.int32), np.zeros(n, dtype=np.int32)
+        lib().orc_get_tables(self.h, _p(Tr, f64p), _p(Ti, f64p), _p(Ur, f64p), _p(Ui, f64p), _p(g5, i32p), _p(u, i32p))
+        return dict(T_re=Tr, T_im=Ti, U_re=Ur, U_im=Ui, g5=g5, uidx=u)
+
+    def psi(self, limb):
+        return int(lib().orc_get_psi(self.h, limb))
+
+    def galois(self, r):
+        return int(lib().orc_galois(self.h, r))
+
+    # ---- transforms (one limb)
+    def ntt(self, limb, a):
+        a = _u64(a).copy()
+        lib().orc_ntt(self.h, C.c_int(limb), _p(a, u64p))
+        return a
+
+    def intt(self, limb, a):
+        a = _u64(a).copy()
+        lib().orc_intt(self.h, C.c_int(limb), _p(a, u64p))
+        return a
+
+    def negacyclic_mul(self, limb, a, b):
+        a, b = _u64(a), _u64(b)
+        out = np.zeros(self.N, dtype=np.uint64)
+        lib().orc_negacyclic_mul(self.h, C.c_int(limb), _p(a, u64p), _p(b, u64p), _p(out, u64p))
+        return out
+
+    def automorphism(self, limb, k, a):
+        a = _u64(a)
+        out = np.zeros(self.N, dtype=np.uint64)
+        lib().orc_automorphism(self.h, limb, C.c_long(k), _p(a, u64p), _p(out, u64p))
+        return out
+
+    def automorphism_ntt(self, k, a):
+        a = _u64(a)
+        out = np.zeros(self.N, dtype=np.uint64)
+        lib().orc_automorphism_ntt(self.h, C.c_long(k), _p(a, u64p), _p(out, u64p))
+        return out
+
+    # ---- encode / decode
+    def encode(self, z, log_scale=None):
+        z = np.ascontiguousarray(z, dtype=np.float64)
+        assert z.shape == (self.n,)
+        m = np.zeros(self.N, dtype=np.int64)
+        lib().orc_encode(self.h, _p(z, f64p), C.c_int(self.log_scale if log_scale is None else log_scale), _p(m, i64p))
+        return m
+
+    def decode(self, mu, scale):
+        """mu: float64[N] real coefficients -> complex slots[n] (z_j = mu(omega^{g_j}) / scale)."""
+        mu = np.ascontiguousarray(mu, dtype=np.float64)
+        zr, zi = np.zeros(self.n), np.zeros(self.n)
+        lib().orc_decode(self.h, _p(mu, f64p), C.c_double(scale), _p(zr, f64p), _p(zi, f64p))
+        return zr + 1j * zi
+
+    def reduce(self, m, nlimbs=None):
+        """integer polynomial (python ints / int64) -> residues [nlimbs][N]"""
+        nl = self.L if nlimbs is None else nlimbs
+        mo = np.array([int(x) for x in m], dtype=object)
+        return np.stack([np.array([int(v) for v in (mo % self.mods[l])], dtype=np.uint64) for l in range(nl)])
+
+    def crt_centred(self, res):
+        """residues [L][N] -> list-like object array of centred python integers in (-Q/2, Q/2]."""
+        res = np.asarray(res)
+        L, Q = self.L, self.Q
+        acc = np.zeros(res.shape[1], dtype=object)
+        for l in range(L):
+            Qh = Q // self.q[l]
+            w = Qh * pow(Qh % self.q[l], -1, self.q[l])
+            acc = acc + res[l].astype(object) * w
+        acc = acc % Q
+        half = Q // 2
+        return np.array([int(v) - Q if int(v) > half else int(v) for v in acc], dtype=object)
+
+    # ---- encryption
+    def encrypt(self, s, m, a, e):
+        s = np.ascontiguousarray(s, dtype=np.int8)
+        m = np.ascontiguousarray(m, dtype=np.int64)
+        a = _u64(a)
+        e = np.ascontiguousarray(e, dtype=np.int8)
+        assert a.shape == (self.L, self.N)
+        ct = np.zeros((2, self.L, self.N), dtype=np.uint64)
+        lib().orc_encrypt(self.h, _p(s, i8p), _p(m, i64p), _p(a, u64p), _p(e, i8p), _p(ct, u64p))
+        return ct
+
+    def encrypt_query(self, s, qvec, a, e):
+        """E3: slot vector z[i] = q[i mod R] (query tiled n/R times), encoded at Delta, encrypted."""
+        qv = np.zeros(self.R, dtype=np.float32)
+        qv[: len(qvec)] = np.asarray(qvec, dtype=np.float32)
+        z = np.tile(qv.astype(np.float64), self.n // self.R)
+        return self.encrypt(s, self.encode(z), a, e)
+
+    def decrypt_residues(self, s, ct):
+        s = np.ascontiguousarray(s, dtype=np.int8)
+        ct = _u64(ct)
+        mu = np.zeros((self.L, self.N), dtype=np.uint64)
+        lib().orc_decrypt_residues(self.h, _p(s, i8p), _p(ct, u64p), _p(mu, u64p))
+        return mu
+
+    def decrypt_int(self, s, ct):
+        return self.crt_centred(self.decrypt_residues(s, ct))
+
+    def decrypt_slots(self, s, ct, log_scale_out):
+        mu = self.decrypt_int(s, ct)
+        muf = np.array([float(v) for v in mu], dtype=np.float64)
+        return self.decode(muf, float(2.0 ** log_scale_out))
+
+    # ---- keys, key switching, rotation
+    def evk_gen(self, s, r, a, e):
+        s = np.ascontiguousarray(s, dtype=np.int8)
+        a = _u64(a)
+        e = np.ascontiguousarray(e, dtype=np.int8)
+        L = self.L
+        assert a.shape == (L, L + 1, self.N) and e.shape == (L, self.N)
+        evk = np.zeros((L, 2, L + 1, self.N), dtype=np.uint64)
+        lib().orc_evk_gen(self.h, _p(s, i8p), C.c_int(r), _p(a, u64p), _p(e, i8p), _p(evk, u64p))
+        return evk
+
+    def moddown(self, u):
+        u = _u64(u)
+        out = np.zeros((self.L, self.N), dtype=np.uint64)
+        lib().orc_moddown(self.h, _p(u, u64p), _p(out, u64p))
+        return out
+
+    def keyswitch(self, d, evk):
+        d, evk = _u64(d), _u64(evk)
+        ks0 = np.zeros((self.L, self.N), dtype=np.uint64)
+        ks1 = np.zeros((self.L, self.N), dtype=np.uint64)
+        lib().orc_keyswitch(self.h, _p(d, u64p), _p(evk, u64p), _p(ks0, u64p), _p(ks1, u64p))
+        return ks0, ks1
+
+    def rotate(self, ct, r, evk_r, hoisted=False):
+        ct, evk_r = _u64(ct), _u64(evk_r)
+        out = np.zeros((2, self.L, self.N), dtype=np.uint64)
+        f = lib().orc_rotate_hoisted if hoisted else lib().orc_rotate
+        f(self.h, _p(ct, u64p), C.c_int(r), _p(evk_r, u64p), _p(out, u64p))
+        return out
+
+    def baby_set(self, ct, evk):
+        """evk[r-1] is the key of rotation r, r = 1..B-1 (more keys may follow; they are ignored)."""
+        ct, evk = _u64(ct), _u64(evk)
+        baby = np.zeros((self.B, 2, self.L, self.N), dtype=np.uint64)
+        lib().orc_baby_set(self.h, _p(ct, u64p), _p(evk, u64p), _p(baby, u64p))
+        return baby
+
+    # ---- block scoring
+    def encode_block(self, rows):
+        rows = np.ascontiguousarray(rows, dtype=np.float32)
+        assert rows.ndim == 2 and rows.shape[1] == self.R and rows.shape[0] <= self.n
+        pt = np.zeros((self.G, self.B, self.L, self.N), dtype=np.uint64)
+        lib().orc_encode_block(self.h, _p(rows, f32p), C.c_int(rows.shape[0]), _p(pt, u64p))
+        return pt
+
+    def mac(self, pt, baby):
+        pt, baby = _u64(pt), _u64(baby)
+        inner = np.zeros((self.G, 2, self.L, self.N), dtype=np.uint64)
+        lib().orc_mac(self.h, _p(pt, u64p), _p(baby, u64p), _p(inner, u64p))
+        return inner
+
+    def rotate_sum(self, inner, evk_B):
+        inner, evk_B = _u64(inner), _u64(evk_B)
+        out = np.zeros((2, self.L, self.N), dtype=np.uint64)
+        lib().orc_rotate_sum(self.h, _p(inner, u64p), _p(evk_B, u64p), _p(out, u64p))
+        return out
+
+    def score_block(self, rows, baby, evk_B, want_pt=False, want_inner=False):
+        rows = np.ascontiguousarray(rows, dtype=np.float32)
+        baby, evk_B = _u64(baby), _u64(evk_B)
+        out = np.zeros((2, self.L, self.N), dtype=np.uint64)
+        pt = np.zeros((self.G, self.B, self.L, self.N), dtype=np.uint64) if want_pt else None
+        inner = np.zeros((self.G, 2, self.L, self.N), dtype=np.uint64) if want_inner else None
+        lib().orc_score_block(
+            self.h, _p(rows, f32p), C.c_int(rows.shape[0]), _p(baby, u64p), _p(evk_B, u64p), _p(out, u64p),
+            _p(pt, u64p) if want_pt else None, _p(inner, u64p) if want_inner else None,
+        )
+        return out, pt, inner
+
+    @staticmethod
+    def num_threads():
+        return int(lib().orc_num_threads())

@@ -1,0 +1,412 @@
+"""Pins of the CPU oracle against what the scheme and the mathematics fix, none of them the oracle itself:
+python-integer schoolbook products, direct polynomial evaluation, multi-precision cosine sums, explicit slot
+permutations, the known error arrays, the analytic key-switch noise bound, plain float64 matrix-vector products.
+"""
+import math
+
+import mpmath
+import numpy as np
+import pytest
+import sympy
+
+from oracle.oracle import Oracle, find_primes, is_prime
+from paper_2608_21131_b200 import synth
+
+
+def make(ps):
+    return Oracle(ps.logN, ps.q, ps.p, ps.log_scale, ps.R, ps.B)
+
+
+def schoolbook_negacyclic(a, b, q):
+    N = len(a)
+    out = [0] * N
+    for i in range(N):
+        for j in range(N):
+            k = i + j
+            v = int(a[i]) * int(b[j])
+            if k < N:
+                out[k] = (out[k] + v) % q
+            else:
+                out[k - N] = (out[k - N] - v) % q
+    return out
+
+
+def rand_poly(rng, N, q):
+    return np.array([int(rng.integers(0, q)) for _ in range(N)], dtype=np.uint64)
+
+
+# ------------------------------------------------------------------ primes
+
+
+def test_primes_are_the_largest_below_the_bound():
+    for bits, logstep, want in ((50, 17, synth.Q50), (60, 17, (synth.P60,)), (30, 13, synth.Q30), (31, 13, (synth.P31,))):
+        got = find_primes(bits, logstep, len(want))
+        assert tuple(got) == tuple(want)
+        step = 1 << logstep
+        # brute recomputation with an independent primality test: every skipped candidate is composite
+        c = (1 << bits) - step + 1
+        found = []
+        while len(found) < len(want):
+            if sympy.isprime(c):
+                found.append(c)
+            c -= step
+        assert tuple(found) == tuple(want)
+
+
+def test_miller_rabin_agrees_with_sympy():
+    rng = np.random.default_rng(0)
+    for x in [0, 1, 2, 3, 4, 561, 2147377153, 2147377155, 3215031751, 2 ** 61 - 1, 2 ** 61 + 1]:
+        assert is_prime(x) == sympy.isprime(x)
+    for x in rng.integers(2, 2 ** 62, size=300):
+        assert is_prime(int(x) | 1) == sympy.isprime(int(x) | 1)
+
+
+# ------------------------------------------------------------------ NTT
+
+
+@pytest.mark.parametrize("logN,big", [(4, False), (6, False), (8, False), (8, True)])
+def test_ntt_roundtrip_definition_and_schoolbook(logN, big):
+    ps = synth.small_params(logN, 4, 2, big=big)
+    o = make(ps)
+    rng = np.random.default_rng(logN)
+    N = ps.N
+    for limb in range(ps.L + 1):
+        q = o.mods[limb]
+        a, b = rand_poly(rng, N, q), rand_poly(rng, N, q)
+        assert np.array_equal(o.intt(limb, o.ntt(limb, a)), a)
+        # definition: a_hat[t] = a(psi^(2t+1))
+        psi = o.psi(limb)
+        assert pow(psi, N, q) == q - 1
+        ah = o.ntt(limb, a)
+        for t in (0, 1, N // 2, N - 1):
+            x = pow(psi, 2 * t + 1, q)
+            assert int(ah[t]) == sum(int(a[i]) * pow(x, i, q) for i in range(N)) % q
+        # product through the transform == schoolbook product in Z_q[X]/(X^N+1)
+        got = o.negacyclic_mul(limb, a, b)
+        assert [int(v) for v in got] == schoolbook_negacyclic(a, b, q)
+
+
+def test_crt_roundtrip():
+    o = make(synth.small_params(4, 4, 2, L=4, big=True))
+    rng = np.random.default_rng(1)
+    vals = [int(rng.integers(-2 ** 62, 2 ** 62)) * int(rng.integers(1, 2 ** 62)) * int(rng.integers(1, 2 ** 62)) for _ in range(14)]
+    vals += [o.Q // 2, -(o.Q // 2)]
+    assert all(abs(v) <= o.Q // 2 for v in vals)
+    res = o.reduce(vals)
+    back = o.crt_centred(res)
+    assert [int(v) for v in back] == vals
+
+
+# ------------------------------------------------------------------ encode / decode
+
+
+def exact_encode(z, N, log_scale):
+    """m_k = rint((Delta/n) sum_j z_j cos(pi g_j k / N)) in 200-bit arithmetic; also returns the distance of the
+    exact value from the nearest half-integer (a near-tie may legitimately round either way in binary64)."""
+    mpmath.mp.prec = 200
+    n = N // 2
+    g = [pow(5, j, 2 * N) for j in range(n)]
+    zs = [mpmath.mpf(float(v)) for v in z]
+    out, margin = [], []
+    for k in range(N):
+        acc = mpmath.mpf(0)
+        for j in range(n):
+            acc += zs[j] * mpmath.cos(mpmath.pi * ((g[j] * k) % (2 * N)) / N)
+        val = acc * mpmath.mpf(2) ** log_scale / n
+        out.append(int(mpmath.nint(val)))
+        margin.append(float(abs(abs(val - mpmath.floor(val)) - mpmath.mpf(0.5))))
+    return out, margin
+
+
+@pytest.mark.parametrize("logN", [3, 4, 6, 8])
+def test_encode_equals_exact_cosine_sum(logN):
+    ps = synth.small_params(logN, 1, 1)
+    o = make(ps)
+    z = synth.gaussian(9, logN, np.arange(ps.n))
+    m = o.encode(z, 25)
+    want, margin = exact_encode(z, ps.N, 25)
+    for k in range(ps.N):
+        assert int(m[k]) == want[k] or (abs(int(m[k]) - want[k]) == 1 and margin[k] < 1e-6)
+    assert sum(int(m[k]) != want[k] for k in range(ps.N)) == 0
+
+
+def test_encode_known_answer_n8():
+    # N = 8, Delta = 2^10, z = (1/4, 1/2, 3/4, 1): m_0 = (Delta/n) * sum z = 256 * 2.5 = 640; the other
+    # coefficients are (Delta/n) sum_j z_j cos(pi g_j k/8) with g = (1, 5, 9, 13), e.g.
+    # m_4 = 256 * (cos(pi/2))*(...) = 0 and m_k = -m_{8-k} for odd symmetry of the cosine sum.
+    o = Oracle(3, synth.Q30, synth.P31, 10, 1, 1)
+    m = o.encode(np.array([0.25, 0.5, 0.75, 1.0]), 10)
+    assert m.tolist() == [640, -69, -91, -167, 0, 167, 91, 69]
+    # rotation by one slot is X -> X^5 on the coefficients
+    res = o.reduce(m, 1)[0]
+    rot = o.automorphism(0, 5, res)
+    cent = [int(v) if int(v) < o.mods[0] // 2 else int(v) - o.mods[0] for v in rot]
+    assert cent == [640, -167, 91, 69, 0, -69, -91, 167]
+    assert cent == o.encode(np.array([0.5, 0.75, 1.0, 0.25]), 10).tolist()
+
+
+def test_index_tables():
+    t = Oracle(3, synth.Q30, synth.P31, 10, 1, 1).tables()
+    assert t["g5"].tolist() == [1, 5, 9, 13] and t["uidx"].tolist() == [0, 1, 2, 3]
+    t = Oracle(5, synth.Q30, synth.P31, 10, 1, 1).tables()
+    assert t["uidx"].tolist() == [0, 1, 6, 15, 12, 13, 2, 11, 8, 9, 14, 7, 4, 5, 10, 3]
+    assert t["g5"].tolist() == [pow(5, j, 64) for j in range(16)]
+    assert sorted(t["uidx"].tolist()) == list(range(16))
+
+
+@pytest.mark.parametrize("logN,stride", [(10, 1), (12, 1), (16, 37)])
+def test_unit_root_tables_are_correctly_rounded(logN, stride):
+    mpmath.mp.prec = 200
+    o = Oracle(logN, synth.Q50[:1], synth.P60, 40, 1, 1)
+    t = o.tables()
+    n, N = o.n, o.N
+    assert t["T_re"][0] == 1.0 and t["T_im"][0] == 0.0
+    assert t["T_re"][n // 4] == 0.0 and t["T_im"][n // 4] == -1.0
+    assert t["U_re"][0] == 1.0 and t["U_im"][0] == 0.0
+    assert t["U_re"][n // 2] == -t["U_im"][n // 2]
+    for k in list(range(0, n // 2, stride)) + [n // 2 - 1]:
+        x = mpmath.mpf(2 * k) / n  # angle / pi, exact
+        assert t["T_re"][k] == float(mpmath.cospi(x)) and t["T_im"][k] == float(-mpmath.sinpi(x))
+    for k in list(range(0, n, stride)) + [n - 1]:
+        x = mpmath.mpf(k) / N
+        assert t["U_re"][k] == float(mpmath.cospi(x)) and t["U_im"][k] == float(-mpmath.sinpi(x))
+
+
+def test_encode_special_cases_and_decode_roundtrip():
+    ps = synth.small_params(10, 1, 1)
+    o = make(ps)
+    assert not o.encode(np.zeros(ps.n)).any()
+    m = o.encode(np.full(ps.n, 0.3125))
+    assert m[0] == round(0.3125 * 2 ** 25) and not m[1:].any()
+    z = synth.uniform(4, 0, np.arange(ps.n)) * 2 - 1
+    m = o.encode(z)
+    back = o.decode(m.astype(np.float64), 2.0 ** 25)
+    err = np.abs(back - z)
+    # coefficient rounding error is uniform(-1/2,1/2) per coefficient: slot error std sqrt(N/12)/Delta
+    std = math.sqrt(ps.N / 12) / 2 ** 25
+    assert err.max() < 6 * std and err.max() > 0.2 * std
+
+
+@pytest.mark.parametrize("r", [1, 3, 7])
+def test_automorphism_is_slot_rotation_and_ntt_gather(r):
+    ps = synth.small_params(8, 1, 1)
+    o = make(ps)
+    z = synth.uniform(5, r, np.arange(ps.n))
+    m = o.encode(z)
+    k = o.galois(r)
+    assert k == pow(5, r, 2 * ps.N)
+    res = o.reduce(m, 1)[0]
+    rot = o.automorphism(0, k, res)
+    q = o.mods[0]
+    cent = np.array([int(v) if int(v) <= q // 2 else int(v) - q for v in rot], dtype=np.float64)
+    back = o.decode(cent, 2.0 ** 25).real
+    assert np.abs(back - np.roll(z, -r)).max() < 1e-5  # left rotation: out[i] = z[i + r]
+    # bit-exact form of the same statement: phi_k(encode(z)) == encode(roll(z)) up to rounding ties only
+    assert np.abs(cent - o.encode(np.roll(z, -r))).max() <= 1
+    # transform-domain gather == transform of the coefficient-domain map
+    assert np.array_equal(o.automorphism_ntt(k, o.ntt(0, res)), o.ntt(0, rot))
+
+
+# ------------------------------------------------------------------ encryption
+
+
+def test_decrypt_of_encrypt_returns_message_plus_the_error_array():
+    ps = synth.small_params(8, 4, 2, L=2)
+    o = make(ps)
+    km = synth.key_material(ps, 11)
+    m = (synth.gaussian(1, 0, np.arange(ps.N)) * 1e6).astype(np.int64)
+    ct = o.encrypt(km.s, m, km.ct_a, km.ct_e)
+    assert np.array_equal(ct[1], km.ct_a)
+    mu = o.decrypt_int(km.s, ct)
+    assert [int(v) for v in mu] == [int(a) + int(b) for a, b in zip(m, km.ct_e)]
+
+
+# ------------------------------------------------------------------ key switching
+
+
+def centred_product_mod_Q(o, d_res, s2):
+    """d * s2 mod Q as centred python integers, by schoolbook over the integers (N small)."""
+    d = o.crt_centred(d_res)
+    N = o.N
+    out = [0] * N
+    for i in range(N):
+        if s2[i] == 0:
+            continue
+        for j in range(N):
+            k = i + j
+            v = int(s2[i]) * int(d[j])
+            if k < N:
+                out[k] += v
+            else:
+                out[k - N] -= v
+    Q = o.Q
+    return [((v + Q // 2) % Q) - Q // 2 for v in out]
+
+
+def signed_automorphism(s, k, N):
+    out = np.zeros(N, dtype=np.int64)
+    for i in range(N):
+        e = (i * k) % (2 * N)
+        if e < N:
+            out[e] = s[i]
+        else:
+            out[e - N] = -s[i]
+    return out
+
+
+@pytest.mark.parametrize("big", [False, True])
+def test_keyswitch_error_within_analytic_bound(big):
+    ps = synth.small_params(8, 8, 4, L=2, big=big)
+    o = make(ps)
+    km = synth.key_material(ps, 21)
+    rng = np.random.default_rng(2)
+    r = 3
+    evk = o.evk_gen(km.s, r, km.evk_a[r - 1], km.evk_e[r - 1])
+    d = np.stack([rand_poly(rng, ps.N, q) for q in ps.q])
+    ks0, ks1 = o.keyswitch(d, evk)
+    s2 = signed_automorphism(km.s, o.galois(r), ps.N)
+    want = centred_product_mod_Q(o, d, s2)
+    # ks0 + ks1*s as centred integers
+    ct = np.stack([ks0, ks1])
+    got = o.decrypt_int(km.s, ct)
+    Q = o.Q
+    err = np.array([float(((int(g) - int(w) + Q // 2) % Q) - Q // 2) for g, w in zip(got, want)])
+    qmean = float(np.mean([float(x) for x in ps.q]))
+    std = math.sqrt(ps.L * ps.N * 3.2 ** 2 * qmean ** 2 / (12 * float(ps.p) ** 2) + ps.N / 18.0)
+    assert abs(err.mean()) < 0.5 * std
+    assert 0.7 * std < err.std() < 1.3 * std
+    assert np.abs(err).max() < 6 * std
+
+
+def test_moddown_of_multiple_of_p_is_exact():
+    ps = synth.small_params(6, 4, 2, L=2, big=True)
+    o = make(ps)
+    rng = np.random.default_rng(3)
+    x = [int(rng.integers(-2 ** 40, 2 ** 40)) for _ in range(ps.N)]
+    px = [v * ps.p for v in x]
+    u = o.reduce(px, ps.L + 1)
+    out = o.moddown(u)
+    assert [int(v) for v in o.crt_centred(out)] == x
+    # and rounds to nearest otherwise
+    px1 = [v * ps.p + ps.p // 2 - 3 for v in x]
+    assert [int(v) for v in o.crt_centred(o.moddown(o.reduce(px1, ps.L + 1)))] == x
+
+
+def test_rotate_decrypts_to_left_rotation_and_hoisting_is_bit_identical():
+    ps = synth.small_params(8, 8, 4, L=2)
+    o = make(ps)
+    km = synth.key_material(ps, 31)
+    z = synth.uniform(6, 0, np.arange(ps.n)) - 0.5
+    ct = o.encrypt(km.s, o.encode(z), km.ct_a, km.ct_e)
+    for r in (1, 4):
+        evk = o.evk_gen(km.s, r, km.evk_a[r - 1], km.evk_e[r - 1])
+        rot = o.rotate(ct, r, evk)
+        back = o.decrypt_slots(km.s, rot, ps.log_scale).real
+        assert np.abs(back - np.roll(z, -r)).max() < 2e-4
+        assert np.array_equal(rot, o.rotate(ct, r, evk, hoisted=True))
+
+
+# ------------------------------------------------------------------ diagonal / BSGS scoring
+
+
+def all_keys(o, km):
+    return np.stack([o.evk_gen(km.s, r, km.evk_a[i], km.evk_e[i]) for i, r in enumerate(km.rots)])
+
+
+@pytest.mark.parametrize("logN,R,B", [(4, 4, 2), (5, 4, 2), (6, 8, 2), (6, 4, 4), (6, 4, 1)])
+def test_bsgs_without_noise_equals_plain_matvec(logN, R, B):
+    ps = synth.small_params(logN, R, B, L=2)
+    o = make(ps)
+    km = synth.key_material(ps, 41, zero_noise=True)
+    rows = synth.toy_corpus(3, rows=ps.n - 3, dim=R)  # ragged block: last 3 rows missing
+    qv = synth.toy_query(4, dim=R)
+    ct = o.encrypt_query(km.s, qv, km.ct_a, km.ct_e)
+    evk = all_keys(o, km)
+    baby = o.baby_set(ct, evk)
+    score, pt, inner = o.score_block(rows, baby, evk[B - 1], True, True)
+    got = o.decrypt_slots(km.s, score, 2 * ps.log_scale)
+    want = np.zeros(ps.n)
+    want[: ps.n - 3] = rows.astype(np.float64) @ qv.astype(np.float64)
+    # only encode rounding and key-switch rounding remain
+    assert np.abs(got.real - want).max() < 2e-5 and np.abs(got.imag).max() < 2e-5
+    # each plaintext decodes to the pre-rotated diagonal it was built from
+    M = np.zeros((ps.n, R))
+    M[: ps.n - 3] = rows
+    for g in range(ps.G):
+        for b in range(B):
+            cent = [int(v) if int(v) <= ps.q[0] // 2 else int(v) - ps.q[0] for v in pt[g, b, 0]]
+            z = o.decode(np.array(cent, dtype=np.float64), 2.0 ** ps.log_scale).real
+            i = np.arange(ps.n)
+            assert np.abs(z - M[(i - g * B) % ps.n, (i + b) % R]).max() < 1e-5
+    # Horner equals the sum of separately rotated partial sums (after decryption)
+    total = np.zeros(ps.n, dtype=complex)
+    for g in range(ps.G):
+        total += np.roll(o.decrypt_slots(km.s, inner[g], 2 * ps.log_scale), -g * B)
+    assert np.abs(total - got).max() < 2e-5
+
+
+def test_zero_padding_96_to_128_is_exact():
+    # Sec. 4 (datasets): zero-padding 96 -> 128 dimensions changes no dot product
+    x = synth.toy_corpus(8, rows=50, dim=96).astype(np.float64)
+    qv = synth.toy_query(9, dim=96).astype(np.float64)
+    xp = np.zeros((50, 128)); xp[:, :96] = x
+    qp = np.zeros(128); qp[:96] = qv
+    a = np.array([sum(x[i, d] * qv[d] for d in range(96)) for i in range(50)])
+    b = np.array([sum(xp[i, d] * qp[d] for d in range(128)) for i in range(50)])
+    assert np.array_equal(a, b)
+    # the padded coordinates occupy exact zeros in the slot vectors that get encoded: a block whose rows are all
+    # zero beyond dimension 96 has, on diagonal b, zero slots wherever (i + b) mod 128 >= 96
+    ps = synth.small_params(9, 128, 32, L=2)
+    o = make(ps)
+    pt = o.encode_block(synth.project_rows(x.astype(np.float32), None, 128))
+    q0 = ps.q[0]
+    for b in (0, 31):
+        cent = np.array([int(v) if int(v) <= q0 // 2 else int(v) - q0 for v in pt[0, b, 0]], dtype=np.float64)
+        z = o.decode(cent, 2.0 ** ps.log_scale).real
+        i = np.arange(ps.n)
+        assert np.abs(z[(i + b) % 128 >= 96]).max() < 1e-5
+
+
+def test_toy_configuration_scores_within_tolerance():
+    """Toy configuration: N = 2^12, two ~30-bit primes + one ~31-bit special prime, scale 2^25, 4,096 unit-norm
+    rows of dimension 64 -> two blocks; decrypted scores within 2^-10 of the float64 dot products."""
+    ps = synth.TOY
+    o = make(ps)
+    km = synth.key_material(ps, 3)
+    rows = synth.toy_corpus(1)
+    qv = synth.toy_query(2)
+    ct = o.encrypt_query(km.s, qv, km.ct_a, km.ct_e)
+    evk = all_keys(o, km)
+    baby = o.baby_set(ct, evk)
+    worst = 0.0
+    for blk in range(2):
+        sc, _, _ = o.score_block(rows[blk * ps.n:(blk + 1) * ps.n], baby, evk[ps.B - 1])
+        got = o.decrypt_slots(km.s, sc, 2 * ps.log_scale)
+        want = rows[blk * ps.n:(blk + 1) * ps.n].astype(np.float64) @ qv.astype(np.float64)
+        worst = max(worst, np.abs(got.real - want).max())
+        assert np.abs(got.imag).max() < 2.0 ** ps.tol_log2
+    assert worst < 2.0 ** ps.tol_log2
+    assert worst < 4 * 2.0 ** -12.2  # regression alarm: observed error level of this parameter set
+    # baby rotations taken directly from the query: each decrypts to the rotated tiled query
+    z = np.tile(np.pad(qv, (0, ps.R - len(qv))).astype(np.float64), ps.n // ps.R)
+    for r in (1, ps.B - 1):
+        back = o.decrypt_slots(km.s, baby[r], ps.log_scale).real
+        assert np.abs(back - np.roll(z, -r)).max() < 1e-3
+
+
+def test_full_size_primes_scores_within_tolerance_small_ring():
+    """The production primes (4 x ~50 bit + ~60 bit, scale 2^40) on a reduced ring: tolerance 2^-18."""
+    ps = synth.ParamSet("n11", 11, synth.Q50, synth.P60, 40, 128, 32, -18)
+    o = make(ps)
+    km = synth.key_material(ps, 5)
+    rows = synth.project_rows(synth.toy_corpus(1, rows=ps.n - 100, dim=96).astype(np.float64), None, 128)
+    qv = np.zeros(128, dtype=np.float32); qv[:96] = synth.toy_query(2, dim=96)
+    ct = o.encrypt_query(km.s, qv, km.ct_a, km.ct_e)
+    evk = all_keys(o, km)
+    baby = o.baby_set(ct, evk)
+    sc, _, _ = o.score_block(rows, baby, evk[ps.B - 1])
+    got = o.decrypt_slots(km.s, sc, 2 * ps.log_scale)
+    want = np.zeros(ps.n); want[: ps.n - 100] = rows.astype(np.float64) @ qv.astype(np.float64)
+    assert np.abs(got.real - want).max() < 2.0 ** -18
+    assert np.abs(got.real - want).max() < 2.0 ** -24
+    assert np.abs(got.imag).max() < 2.0 ** -18

@@ -1,0 +1,79 @@
+"""Seeded input generators: fixed check values, basic statistics, parameter sets."""
+import numpy as np
+import sympy
+
+from paper_2608_21131_b200 import synth
+
+
+def test_hash_check_values():
+    got = [int(x) for x in synth.hash64(1, 0, np.arange(4))]
+    assert got == [0xCE6D52A9E69DA903, 0x3C904E4F0D0C01AF, 0x6E6AE58702F2C840, 0xD254BD0790389C63]
+
+
+def test_uniform_and_gaussian_statistics():
+    u = synth.uniform(5, 0, np.arange(200_000))
+    assert 0.0 <= u.min() and u.max() < 1.0
+    assert abs(u.mean() - 0.5) < 5e-3 and abs(u.var() - 1 / 12) < 2e-3
+    g = synth.gaussian(5, 1, np.arange(200_000))
+    assert abs(g.mean()) < 1e-2 and abs(g.std() - 1.0) < 1e-2
+    assert abs((g ** 4).mean() - 3.0) < 0.1
+
+
+def test_key_material_distributions():
+    ps = synth.TOY
+    km = synth.key_material(ps, 3)
+    assert set(np.unique(km.s)) == {-1, 0, 1}
+    assert abs(km.evk_e.astype(float).std() - 3.2) < 0.1
+    mods = list(ps.q) + [ps.p]
+    for i, m in enumerate(mods):
+        assert int(km.evk_a[:, :, i].max()) < m
+    assert km.evk_a.shape == (ps.B, ps.L, ps.L + 1, ps.N)
+    # different seeds give different material; same seed reproduces
+    km2 = synth.key_material(ps, 3)
+    assert np.array_equal(km.evk_a, km2.evk_a) and np.array_equal(km.s, km2.s)
+    assert not np.array_equal(km.s, synth.key_material(ps, 4).s)
+
+
+def test_parameter_sets_are_ntt_friendly_primes():
+    for ps in (synth.TOY, synth.FULL15, synth.FULL16):
+        for m in list(ps.q) + [ps.p]:
+            assert sympy.isprime(m)
+            assert (m - 1) % (2 * ps.N) == 0
+        assert ps.R % ps.B == 0 and ps.n % ps.R == 0
+
+
+def test_corpora_unit_norm_and_reproducible():
+    x = synth.toy_corpus(1, rows=64, dim=64)
+    assert x.dtype == np.float32 and np.allclose(np.linalg.norm(x, axis=1), 1.0, atol=1e-6)
+    fm = synth.FlatMixture(rows=1000, dim=64, k=16)
+    ids = np.array([5, 17, 999, 5])
+    v = fm.vectors(ids)
+    assert np.allclose(np.linalg.norm(v, axis=1), 1.0)
+    assert np.array_equal(v[0], v[3])  # pure function of the id
+    h = synth.Hierarchy(dim=32, n_coarse=8, fan=4, leaf=5)
+    r = h.rows(np.array([0, 1, 159]))
+    assert r.shape == (3, 32) and np.allclose(np.linalg.norm(r, axis=1), 1.0)
+    # rows of one fine cell are closer to their fine mean than to another coarse cell's mean
+    f0 = h.fine(np.array([0]))[0]
+    assert r[0] @ f0 > r[0] @ h.coarse(np.array([5]))[0]
+    # a planted query's nearest row is the planted row
+    qv = h.query_near(7, 1001)
+    allrows = h.rows(np.arange(h.n_rows))
+    assert int(np.argmax(allrows @ qv)) == 7
+
+
+def test_projection_is_orthonormal():
+    W = synth.projection_matrix(21131, 64, 16)
+    assert np.allclose(W.T @ W, np.eye(16), atol=1e-12)
+
+
+def test_padding_groups_partition_and_inflate():
+    pi = synth.padding_groups(7, 1000, 4)
+    assert sorted(pi.tolist()) == list(range(1000))
+    wanted = np.array([3, 500, 999])
+    fetched = synth.padded_fetch(pi, wanted, 4)
+    assert set(wanted.tolist()) <= set(fetched.tolist())
+    assert len(fetched) == 12 and np.all(np.diff(fetched) > 0)
+    # fixed groups: the same cell always brings the same decoys
+    again = synth.padded_fetch(pi, np.array([500]), 4)
+    assert set(again.tolist()) <= set(fetched.tolist()) and len(again) == 4

@@ -1,0 +1,192 @@
+/*
+ * hann.h -- C ABI of the B200 encrypted nearest-neighbour scoring library.
+ *
+ * The library implements the server-side hot path of hierarchical encrypted ANN search with RNS-CKKS:
+ * one encrypted, rank-reduced query is scored against fetched batches of plaintext candidate rows at
+ * each routing level (Sec. 2 "The round trip": coarse -> fine -> rerank; Sec. 3.2 "How": every level
+ * is one call to the same stateless scorer), using the diagonal matrix-vector method with baby-step /
+ * giant-step rotations (Sec. 3.1 "How" and Detail) and plaintext pre-rotation of the database diagonals
+ * (Sec. 3.1 Detail).  The client half (key generation, query encryption, score decryption; Sec. 2,
+ * steps 1, 3, 5, 7 of the round trip) is here too so that a user needs nothing else.
+ *
+ * Conventions
+ *   - Every function returns HANN_OK (0) or a negative HANN_E* code; nothing throws or aborts across the
+ *     boundary.  `hann_last_error` gives a one-line description of the last failure of a context.
+ *     On error the outputs are unspecified but no buffer is freed or re-owned.
+ *   - "host" pointers are ordinary CPU memory; "device" pointers are CUDA global memory on the context's
+ *     device.  Device work is enqueued on the context's stream and is asynchronous; host-pointer
+ *     functions synchronise that stream before they return.
+ *   - The caller owns every buffer it passes.  The library owns the context, its tables and the keys
+ *     uploaded with `hann_load_keys`; these live until `hann_ctx_destroy`.
+ *   - Server-side calls (`hann_query_prepare`, `hann_encode_candidates`, `hann_score_level`,
+ *     `hann_rotate_sum`, `hann_keyswitch`) allocate nothing: all temporaries live in the caller's
+ *     workspace `ws` (256-byte aligned device memory, `ws_bytes` long; `hann_workspace_bytes` says how
+ *     much is enough; HANN_EWORKSPACE if it is too short) -- the counterpart of the paper's single
+ *     pre-allocated arena, Sec. 3.4.  One workspace serves one call at a time.
+ *   - Canonical exchange layout (the only layout with a meaning outside the library): coefficient
+ *     domain, natural coefficient order, residues in [0, q_i), uint64, index order [poly][limb][coeff];
+ *     a ciphertext is 2 polynomials (c0, c1) of L limbs.  The internal device layout (transform domain,
+ *     element order) is private; `hann_import` / `hann_export` convert.
+ *   - Ring degree N = 2^logN, n = N/2 slots; L ciphertext primes q_0..q_{L-1} and one special prime p,
+ *     each prime, below 2^62 and congruent to 1 mod 2N; R = padded vector dimension (R divides n);
+ *     B = baby-step count (B divides R), G = R/B giant steps.
+ *   - Row <-> slot mapping: row blk*n + i of a level's candidate list is slot i of score ciphertext blk;
+ *     the last block is zero-padded.
+ */
+#ifndef HANN_H
+#define HANN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HANN_OK 0
+#define HANN_EINVAL (-1)     /* bad parameter value or null pointer                        */
+#define HANN_ESHAPE (-2)     /* sizes inconsistent with the context (dim, counts, rotation) */
+#define HANN_ENOKEY (-3)     /* a needed evaluation key has not been loaded                 */
+#define HANN_EWORKSPACE (-4) /* workspace missing or misaligned                             */
+#define HANN_ECUDA (-5)      /* a CUDA runtime call or kernel launch failed                 */
+#define HANN_ENOMEM (-6)     /* host or device allocation failed (set-up calls only)        */
+
+#define HANN_MAX_PRIMES 8
+
+typedef struct hann_ctx hann_ctx; /* opaque */
+
+typedef struct {
+    int32_t logN;                /* 4..16                                                   */
+    int32_t L;                   /* number of ciphertext primes, 1..HANN_MAX_PRIMES         */
+    uint64_t q[HANN_MAX_PRIMES]; /* q_0..q_{L-1}                                            */
+    uint64_t p;                  /* special prime of hybrid key switching                   */
+    int32_t log_scale;           /* Delta = 2^log_scale for queries and candidates          */
+    int32_t R;                   /* padded dimension                                        */
+    int32_t B;                   /* baby-step count                                         */
+    int32_t device;              /* CUDA device ordinal                                     */
+    void *stream;                /* cudaStream_t the context enqueues on (NULL = default)   */
+} hann_params;
+
+/* what `hann_sizeof` can be asked */
+enum {
+    HANN_SIZE_POLY = 1,     /* one polynomial of L limbs: L*N*8                                          */
+    HANN_SIZE_CT = 2,       /* one ciphertext: 2*L*N*8                                                    */
+    HANN_SIZE_BABY = 3,     /* the B rotated query ciphertexts                                            */
+    HANN_SIZE_PT_BLOCK = 4, /* encoded candidates of one block of n rows: R*L*N*8 (= 16*L*R bytes a row) */
+    HANN_SIZE_INNER = 5,    /* the G partial-sum ciphertexts of one block                                 */
+    HANN_SIZE_EVK = 6,      /* one evaluation key in canonical layout: L*2*(L+1)*N*8                      */
+    HANN_SIZE_ROWS_PER_BLOCK = 7 /* n                                                                     */
+};
+
+/* element kinds of `hann_import` / `hann_export` */
+enum { HANN_KIND_POLY = 1, HANN_KIND_CT = 2, HANN_KIND_PT = 3 };
+
+typedef struct {
+    uint64_t launches;         /* kernels launched by this context since creation                      */
+    float ms_query_prepare;    /* device time of the last call of each kind, milliseconds; valid after */
+    float ms_encode;           /* hann_sync (0 if never called or timing disabled)                     */
+    float ms_score_level;
+    float ms_rotate_sum;
+    float ms_keyswitch;
+} hann_stats;
+
+/* ---- context ------------------------------------------------------------------------------------------- */
+
+/* Create a context: validates the parameters (HANN_EINVAL: not prime, not 1 mod 2N, out of range, B does not
+ * divide R, R does not divide n), builds the transform and encode tables on the device.  *out is set only on
+ * success and must be released with hann_ctx_destroy. */
+int hann_ctx_create(const hann_params *params, hann_ctx **out);
+void hann_ctx_destroy(hann_ctx *ctx);
+
+/* Byte sizes of the private device layouts (see the enum); negative on a bad argument. */
+int64_t hann_sizeof(const hann_ctx *ctx, int what);
+
+/* Bytes of workspace the server-side calls need when at most `max_blocks` blocks are processed per call. */
+int64_t hann_workspace_bytes(const hann_ctx *ctx, int64_t max_blocks);
+
+/* Block until everything enqueued on the context's stream has finished; reports asynchronous CUDA errors. */
+int hann_sync(hann_ctx *ctx);
+const char *hann_last_error(const hann_ctx *ctx);
+/* Enable (1) or disable (0) per-call CUDA-event timing; disabled by default. */
+int hann_set_timing(hann_ctx *ctx, int enable);
+int hann_get_stats(hann_ctx *ctx, hann_stats *out);
+
+/* ---- client side (host memory in and out; Sec. 2, The round trip, client steps) -------------------------- */
+
+/* Evaluation keys for the left slot rotations rot[0..n_rot) from caller-drawn randomness (hybrid key switching,
+ * one special prime, one digit per ciphertext prime).  For rotation r (Galois element k = 5^r mod 2N,
+ * s' = s(X^k)) and digit j: b_j = -a_j*s + e_j + F_j*s' over the L+1 moduli, F_j = p mod q_j on limb j and
+ * 0 elsewhere.
+ *   s   [N]                      ternary secret, int8 in {-1,0,1}
+ *   a   [n_rot][L][L+1][N]       uniform residues (limb order q_0..q_{L-1}, p), canonical
+ *   e   [n_rot][L][N]            small errors, int8
+ *   evk_out [n_rot][L][2][L+1][N]  canonical; [..][j][0] = b_j, [..][j][1] = a_j */
+int hann_keygen_from_samples(hann_ctx *ctx, const int8_t *s, int n_rot, const int32_t *rot, const uint64_t *a,
+                             const int8_t *e, uint64_t *evk_out);
+
+/* Symmetric encryption of a query: the slot vector holds q[i mod R] (q zero-padded from `dim` to R and tiled
+ * n/R times), encoded at scale Delta by the canonical encoder, then ct = (-a*s + e + m, a).
+ *   q [dim] float32, dim <= R;  a [L][N] uniform residues;  e [N] int8;  ct_out [2][L][N] canonical. */
+int hann_encrypt_query(hann_ctx *ctx, const int8_t *s, const float *q, int dim, const uint64_t *a, const int8_t *e,
+                       uint64_t *ct_out);
+
+/* Decrypt `count` score ciphertexts ct [count][2][L][N] (canonical) whose plaintext scale is 2^log_scale_out
+ * (2*log_scale straight after scoring) into real parts scores [count][n]; imag_or_null, if given, receives the
+ * imaginary parts [count][n] (pure noise for a correct computation). */
+int hann_decrypt_scores(hann_ctx *ctx, const int8_t *s, const uint64_t *ct, int64_t count, int log_scale_out,
+                        double *scores, double *imag_or_null);
+
+/* ---- server side ------------------------------------------------------------------------------------------ */
+
+/* Upload evaluation keys (canonical layout as produced by hann_keygen_from_samples; `evk` may be a host or a
+ * device pointer) into the context, replacing keys with the same rotation.  Allocates device memory owned by the
+ * context.  Needed later: rotations 1..B-1 for hann_query_prepare, rotation B for hann_rotate_sum. */
+int hann_load_keys(hann_ctx *ctx, const uint64_t *evk, int n_rot, const int32_t *rot);
+
+/* Once per query: the B rotated copies rot_r(ct), r = 0..B-1, each taken directly from the input ciphertext
+ * (key switch of the automorphed c1; the digit decomposition is shared by all rotations).
+ *   ct_dev   one ciphertext, internal layout (device)
+ *   baby_dev HANN_SIZE_BABY bytes (device), internal layout [B][2][L][N] */
+int hann_query_prepare(hann_ctx *ctx, const void *ct_dev, void *baby_dev, void *ws, size_t ws_bytes);
+
+/* Encode candidate rows into plaintext blocks.  rows_dev [n_rows][dim] float32 row-major (device), dim <= R
+ * (rows are zero-padded to R).  Block blk holds rows blk*n .. blk*n+n-1 (missing rows are zero).  For g < G,
+ * b < B plaintext (g,b) of a block encodes the slot vector z[i] = M[(i - g*B) mod n][(i + b) mod R] at scale
+ * Delta, reduced into every ciphertext prime and transformed.
+ *   pt_dev  ceil(n_rows/n) * HANN_SIZE_PT_BLOCK bytes (device), internal layout [blk][G][B][L][N] */
+int hann_encode_candidates(hann_ctx *ctx, const float *rows_dev, int64_t n_rows, int dim, void *pt_dev, void *ws, size_t ws_bytes);
+
+/* Multiply-accumulate of one level: inner[blk][g] = sum_b pt[blk][g][b] * baby[b] (both ciphertext components,
+ * every limb).   inner_dev n_blocks * HANN_SIZE_INNER bytes (device), internal layout [blk][G][2][L][N]. */
+int hann_score_level(hann_ctx *ctx, const void *baby_dev, const void *pt_dev, int64_t n_blocks, void *inner_dev,
+                     void *ws, size_t ws_bytes);
+
+/* Rotate-and-sum: score_ct[blk] = sum_g rot_{g*B}(inner[blk][g]), evaluated by Horner with the single key of
+ * rotation B: acc = inner[G-1]; for g = G-2..0: acc = rot_B(acc) + inner[g].
+ *   score_ct_dev n_blocks * HANN_SIZE_CT bytes (device), internal layout. */
+int hann_rotate_sum(hann_ctx *ctx, const void *inner_dev, int64_t n_blocks, void *score_ct_dev, void *ws, size_t ws_bytes);
+
+/* Hybrid key switch of one polynomial d (internal layout, L limbs) with the loaded key of rotation `rot`, WITHOUT
+ * applying the automorphism to d: outputs (ks0, ks1), L limbs each, with ks0 + ks1*s ~ d*s(X^k).
+ * Steps: digits [d]_{q_j} (inverse transform), centred lift into all L+1 moduli, transform, inner product with
+ * the key, ModDown: out_i = (u_i - centred([u]_p)) * p^{-1} mod q_i. */
+int hann_keyswitch(hann_ctx *ctx, int rot, const void *poly_dev, void *ks0_dev, void *ks1_dev, void *ws, size_t ws_bytes);
+
+/* Convert `count` elements between the canonical layout (host or device pointer) and the internal device layout.
+ * kind POLY / PT: one polynomial of L limbs per element; CT: two. */
+int hann_import(hann_ctx *ctx, int kind, const uint64_t *canonical, int64_t count, void *internal_dev);
+int hann_export(hann_ctx *ctx, int kind, const void *internal_dev, int64_t count, uint64_t *canonical_out);
+
+/* One level end to end from HOST buffers (copies included): import the canonical query ciphertext, prepare the baby
+ * set, copy the rows to the device, encode, multiply-accumulate, rotate-and-sum, export the score ciphertexts to the
+ * host in canonical layout.  Device buffers for the intermediates are carved from `ws_dev`, which must hold
+ * hann_level_host_bytes(ctx, n_rows) bytes.
+ *   ct_host [2][L][N];  rows_host [n_rows][dim] float32;  score_ct_host [ceil(n_rows/n)][2][L][N]. */
+int64_t hann_level_host_bytes(const hann_ctx *ctx, int64_t n_rows);
+int hann_score_level_host(hann_ctx *ctx, const uint64_t *ct_host, const float *rows_host, int64_t n_rows, int dim,
+                          uint64_t *score_ct_host, void *ws_dev, size_t ws_bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HANN_H */

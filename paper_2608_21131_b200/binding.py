@@ -1,0 +1,267 @@
+"""Thin ctypes binding of the C-ABI CUDA library (``include/hann.h``): argument marshalling only.
+
+Every function has the name of the C entry point it wraps (without the ``hann_`` prefix) and every step of
+the scoring path runs in the library's CUDA kernels.  PyTorch is used for device memory and streams; host
+arrays are numpy.  There is no CPU fallback: creating a `Context` raises if the library is not built or no
+CUDA device is present.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libhann.so")
+
+HANN_MAX_PRIMES = 8
+OK, EINVAL, ESHAPE, ENOKEY, EWORKSPACE, ECUDA, ENOMEM = 0, -1, -2, -3, -4, -5, -6
+SIZE_POLY, SIZE_CT, SIZE_BABY, SIZE_PT_BLOCK, SIZE_INNER, SIZE_EVK, SIZE_ROWS_PER_BLOCK = 1, 2, 3, 4, 5, 6, 7
+KIND_POLY, KIND_CT, KIND_PT = 1, 2, 3
+
+
+class HannError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__("hann error %d: %s" % (code, msg))
+        self.code = code
+
+
+class Params(C.Structure):
+    _fields_ = [
+        ("logN", C.c_int32), ("L", C.c_int32), ("q", C.c_uint64 * HANN_MAX_PRIMES), ("p", C.c_uint64),
+        ("log_scale", C.c_int32), ("R", C.c_int32), ("B", C.c_int32), ("device", C.c_int32), ("stream", C.c_void_p),
+    ]
+
+
+class Stats(C.Structure):
+    _fields_ = [
+        ("launches", C.c_uint64), ("ms_query_prepare", C.c_float), ("ms_encode", C.c_float),
+        ("ms_score_level", C.c_float), ("ms_rotate_sum", C.c_float), ("ms_keyswitch", C.c_float),
+    ]
+
+
+_lib = None
+
+
+def load_library():
+    """Load ``libhann.so``; raises (never falls back) when it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            "the CUDA library %s is missing: build it with `python -m paper_2608_21131_b200.build`" % LIB_PATH
+        )
+    lib = C.CDLL(LIB_PATH)
+    vp, i64, sz = C.c_void_p, C.c_int64, C.c_size_t
+    sig = {
+        "hann_ctx_create": (C.c_int, [C.POINTER(Params), C.POINTER(vp)]),
+        "hann_ctx_destroy": (None, [vp]),
+        "hann_sizeof": (i64, [vp, C.c_int]),
+        "hann_workspace_bytes": (i64, [vp, i64]),
+        "hann_sync": (C.c_int, [vp]),
+        "hann_last_error": (C.c_char_p, [vp]),
+        "hann_set_timing": (C.c_int, [vp, C.c_int]),
+        "hann_get_stats": (C.c_int, [vp, C.POINTER(Stats)]),
+        "hann_keygen_from_samples": (C.c_int, [vp, vp, C.c_int, vp, vp, vp, vp]),
+        "hann_encrypt_query": (C.c_int, [vp, vp, vp, C.c_int, vp, vp, vp]),
+        "hann_decrypt_scores": (C.c_int, [vp, vp, vp, i64, C.c_int, vp, vp]),
+        "hann_load_keys": (C.c_int, [vp, vp, C.c_int, vp]),
+        "hann_query_prepare": (C.c_int, [vp, vp, vp, vp, sz]),
+        "hann_encode_candidates": (C.c_int, [vp, vp, i64, C.c_int, vp, vp, sz]),
+        "hann_score_level": (C.c_int, [vp, vp, vp, i64, vp, vp, sz]),
+        "hann_rotate_sum": (C.c_int, [vp, vp, i64, vp, vp, sz]),
+        "hann_keyswitch": (C.c_int, [vp, C.c_int, vp, vp, vp, vp, sz]),
+        "hann_import": (C.c_int, [vp, C.c_int, vp, i64, vp]),
+        "hann_export": (C.c_int, [vp, C.c_int, vp, i64, vp]),
+        "hann_level_host_bytes": (i64, [vp, i64]),
+        "hann_score_level_host": (C.c_int, [vp, vp, vp, i64, C.c_int, vp, vp, sz]),
+    }
+    for name, (res, args) in sig.items():
+        f = getattr(lib, name)
+        f.restype = res
+        f.argtypes = args
+    _lib = lib
+    return lib
+
+
+def _np(a, dtype):
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def _ptr(a):
+    """address of a numpy array or a torch tensor (host or device)"""
+    if a is None:
+        return None
+    if isinstance(a, np.ndarray):
+        return a.ctypes.data
+    return a.data_ptr()
+
+
+class Context:
+    """One parameter set bound to one CUDA device and stream.  `ps` needs the attributes logN, q, p, log_scale,
+    R, B."""
+
+    def __init__(self, ps, device: int = 0, stream=None):
+        import torch
+
+        if not torch.cuda.is_available():
+            raise RuntimeError("no CUDA device: the scoring path has no CPU fallback")
+        self.torch = torch
+        self.lib = load_library()
+        self.device = torch.device("cuda", device)
+        self.logN, self.N, self.n = ps.logN, 1 << ps.logN, 1 << (ps.logN - 1)
+        self.L, self.R, self.B, self.G = len(ps.q), ps.R, ps.B, ps.R // ps.B
+        self.log_scale = ps.log_scale
+        prm = Params()
+        prm.logN, prm.L, prm.p, prm.log_scale, prm.R, prm.B, prm.device = ps.logN, len(ps.q), ps.p, ps.log_scale, ps.R, ps.B, device
+        for i, q in enumerate(ps.q):
+            prm.q[i] = q
+        if stream is None:
+            stream = torch.cuda.current_stream(self.device)
+        self.stream = stream
+        prm.stream = stream.cuda_stream
+        h = C.c_void_p()
+        rc = self.lib.hann_ctx_create(C.byref(prm), C.byref(h))
+        if rc != OK:
+            raise HannError(rc, "hann_ctx_create failed (invalid parameters or CUDA error)")
+        self.h = h
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.lib.hann_ctx_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _ck(self, rc):
+        if rc != OK:
+            raise HannError(rc, self.lib.hann_last_error(self.h).decode())
+
+    # ---- sizes and buffers
+    def sizeof(self, what):
+        return int(self.lib.hann_sizeof(self.h, what))
+
+    def workspace_bytes(self, max_blocks):
+        return int(self.lib.hann_workspace_bytes(self.h, max_blocks))
+
+    def alloc(self, nbytes):
+        """uint64 device tensor of at least nbytes (torch allocations are 512-byte aligned)"""
+        return self.torch.empty((int(nbytes) + 7) // 8, dtype=self.torch.int64, device=self.device)
+
+    def workspace(self, max_blocks):
+        return self.alloc(self.workspace_bytes(max_blocks))
+
+    def sync(self):
+        self._ck(self.lib.hann_sync(self.h))
+
+    def set_timing(self, on):
+        self._ck(self.lib.hann_set_timing(self.h, 1 if on else 0))
+
+    def get_stats(self):
+        st = Stats()
+        self._ck(self.lib.hann_get_stats(self.h, C.byref(st)))
+        return {k: getattr(st, k) for k, _ in Stats._fields_}
+
+    # ---- client side
+    def keygen_from_samples(self, s, rots, a, e):
+        s, a, e = _np(s, np.int8), _np(a, np.uint64), _np(e, np.int8)
+        rots = _np(rots, np.int32)
+        L, N = self.L, self.N
+        assert a.shape == (len(rots), L, L + 1, N) and e.shape == (len(rots), L, N) and s.shape == (N,)
+        evk = np.empty((len(rots), L, 2, L + 1, N), dtype=np.uint64)
+        self._ck(self.lib.hann_keygen_from_samples(self.h, _ptr(s), len(rots), _ptr(rots), _ptr(a), _ptr(e), _ptr(evk)))
+        return evk
+
+    def encrypt_query(self, s, q, a, e):
+        s, q, a, e = _np(s, np.int8), _np(q, np.float32), _np(a, np.uint64), _np(e, np.int8)
+        assert a.shape == (self.L, self.N) and e.shape == (self.N,)
+        ct = np.empty((2, self.L, self.N), dtype=np.uint64)
+        self._ck(self.lib.hann_encrypt_query(self.h, _ptr(s), _ptr(q), len(q), _ptr(a), _ptr(e), _ptr(ct)))
+        return ct
+
+    def decrypt_scores(self, s, ct, log_scale_out=None, want_imag=False):
+        s, ct = _np(s, np.int8), _np(ct, np.uint64)
+        ct = ct.reshape(-1, 2, self.L, self.N)
+        count = ct.shape[0]
+        scores = np.empty((count, self.n), dtype=np.float64)
+        imag = np.empty((count, self.n), dtype=np.float64) if want_imag else None
+        ls = 2 * self.log_scale if log_scale_out is None else log_scale_out
+        self._ck(self.lib.hann_decrypt_scores(self.h, _ptr(s), _ptr(ct), count, ls, _ptr(scores), _ptr(imag)))
+        return (scores, imag) if want_imag else scores
+
+    # ---- server side
+    def load_keys(self, evk, rots):
+        rots = _np(rots, np.int32)
+        if isinstance(evk, np.ndarray):
+            evk = _np(evk, np.uint64)
+        self._ck(self.lib.hann_load_keys(self.h, _ptr(evk), len(rots), _ptr(rots)))
+
+    def import_(self, kind, canonical, count):
+        if isinstance(canonical, np.ndarray):
+            canonical = _np(canonical, np.uint64)
+        per = self.sizeof(SIZE_CT if kind == KIND_CT else SIZE_POLY)
+        out = self.alloc(per * count)
+        self._ck(self.lib.hann_import(self.h, kind, _ptr(canonical), count, _ptr(out)))
+        return out
+
+    def export(self, kind, internal, count, offset_bytes=0):
+        polys = 2 if kind == KIND_CT else 1
+        out = np.empty((count, polys, self.L, self.N), dtype=np.uint64)
+        self._ck(self.lib.hann_export(self.h, kind, _ptr(internal) + offset_bytes, count, _ptr(out)))
+        return out
+
+    def query_prepare(self, ct_dev, ws, baby=None):
+        if baby is None:
+            baby = self.alloc(self.sizeof(SIZE_BABY))
+        self._ck(self.lib.hann_query_prepare(self.h, _ptr(ct_dev), _ptr(baby), _ptr(ws), ws.numel() * 8))
+        return baby
+
+    def n_blocks(self, n_rows):
+        return (n_rows + self.n - 1) // self.n
+
+    def encode_candidates(self, rows_dev, ws, pt=None):
+        n_rows, dim = rows_dev.shape
+        assert rows_dev.dtype == self.torch.float32 and rows_dev.is_contiguous()
+        if pt is None:
+            pt = self.alloc(self.n_blocks(n_rows) * self.sizeof(SIZE_PT_BLOCK))
+        self._ck(self.lib.hann_encode_candidates(self.h, _ptr(rows_dev), n_rows, dim, _ptr(pt), _ptr(ws), ws.numel() * 8))
+        return pt
+
+    def score_level(self, baby, pt, n_blocks, ws=None, inner=None):
+        if inner is None:
+            inner = self.alloc(n_blocks * self.sizeof(SIZE_INNER))
+        self._ck(self.lib.hann_score_level(self.h, _ptr(baby), _ptr(pt), n_blocks, _ptr(inner), _ptr(ws),
+                                           ws.numel() * 8 if ws is not None else 0))
+        return inner
+
+    def rotate_sum(self, inner, n_blocks, ws, score=None):
+        if score is None:
+            score = self.alloc(n_blocks * self.sizeof(SIZE_CT))
+        self._ck(self.lib.hann_rotate_sum(self.h, _ptr(inner), n_blocks, _ptr(score), _ptr(ws), ws.numel() * 8))
+        return score
+
+    def keyswitch(self, rot, poly, ws):
+        ks0 = self.alloc(self.sizeof(SIZE_POLY))
+        ks1 = self.alloc(self.sizeof(SIZE_POLY))
+        self._ck(self.lib.hann_keyswitch(self.h, rot, _ptr(poly), _ptr(ks0), _ptr(ks1), _ptr(ws), ws.numel() * 8))
+        return ks0, ks1
+
+    def level_host_bytes(self, n_rows):
+        return int(self.lib.hann_level_host_bytes(self.h, n_rows))
+
+    def score_level_host(self, ct_host, rows_host, ws_dev, out=None):
+        """ct_host: uint64 [2][L][N] (numpy or pinned torch), rows_host: float32 [n_rows][dim]; returns the score
+        ciphertexts [n_blocks][2][L][N] in host memory."""
+        n_rows, dim = rows_host.shape
+        nb = self.n_blocks(n_rows)
+        if out is None:
+            out = np.empty((nb, 2, self.L, self.N), dtype=np.uint64)
+        self._ck(self.lib.hann_score_level_host(self.h, _ptr(ct_host), _ptr(rows_host), n_rows, dim, _ptr(out), _ptr(ws_dev),
+                                                ws_dev.numel() * 8))
+        return out

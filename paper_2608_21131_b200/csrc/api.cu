@@ -1,0 +1,719 @@
+// C-ABI entry points (see include/hann.h): context set-up, the client half, and the server-side scoring calls,
+// each of which is a fixed sequence of kernel launches on the context's stream.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "internal.h"
+
+#define CK(call)                                                                   \
+    do {                                                                           \
+        cudaError_t e_ = (call);                                                   \
+        if (e_ != cudaSuccess) {                                                   \
+            c->err = std::string(#call) + ": " + cudaGetErrorString(e_);           \
+            return HANN_ECUDA;                                                     \
+        }                                                                          \
+    } while (0)
+
+#define RET(call)                      \
+    do {                               \
+        int r_ = (call);               \
+        if (r_ != HANN_OK) return r_;  \
+    } while (0)
+
+namespace {
+
+int fail(hann_ctx* c, int code, const char* msg) {
+    if (c) c->err = msg;
+    return code;
+}
+
+inline int64_t align256(int64_t x) { return (x + 255) & ~(int64_t)255; }
+
+// bump allocator over a caller-provided workspace
+struct Arena {
+    char* base;
+    int64_t off, cap;
+    template <typename T>
+    T* take(int64_t count) {
+        int64_t bytes = align256(count * (int64_t)sizeof(T));
+        if (off + bytes > cap) return nullptr;
+        T* p = (T*)(base + off);
+        off += bytes;
+        return p;
+    }
+};
+
+struct DeviceGuard {
+    int prev;
+    bool ok;
+    explicit DeviceGuard(int dev) {
+        ok = cudaGetDevice(&prev) == cudaSuccess && cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() {
+        if (ok) cudaSetDevice(prev);
+    }
+};
+
+int ensure_scratch(hann_ctx* c, int64_t bytes) {
+    if (bytes <= c->scratch_bytes) return HANN_OK;
+    CK(cudaStreamSynchronize(c->stream));
+    if (c->scratch) cudaFree(c->scratch);
+    c->scratch = nullptr;
+    c->scratch_bytes = 0;
+    if (cudaMalloc(&c->scratch, (size_t)bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(c, HANN_ENOMEM, "device allocation of the exchange scratch failed");
+    }
+    c->scratch_bytes = bytes;
+    return HANN_OK;
+}
+
+// per-call timing with CUDA events on the context's stream
+struct Timer {
+    hann_ctx* c;
+    int kind;
+    Timer(hann_ctx* c_, int kind_) : c(c_), kind(kind_) {
+        if (c->timing) cudaEventRecord(c->ev[kind][0], c->stream);
+    }
+    ~Timer() {
+        if (c->timing) {
+            cudaEventRecord(c->ev[kind][1], c->stream);
+            c->ev_pending[kind] = 1;
+        }
+    }
+};
+
+int64_t ks_item_words(const hann_ctx* c) {
+    // per item: c1 coefficients, digits, u, lifted, one temporary ciphertext
+    const int64_t L = c->L, N = c->N;
+    return L * N + L * (L + 1) * N + 2 * (L + 1) * N + 2 * L * N + 2 * L * N;
+}
+
+int64_t prepare_words(const hann_ctx* c) {
+    const int64_t L = c->L, N = c->N, nb = std::max(c->B - 1, 1);
+    return L * N + L * (L + 1) * N + nb * (2 * (L + 1) * N + 2 * L * N);
+}
+
+constexpr int64_t kSlack = 16 * 256;  // room for the alignment of a dozen sub-buffers
+
+// canonical (host or device) -> internal: copy, forward transform of count polynomials of L limbs
+int import_polys(hann_ctx* c, const u64* canonical, int64_t npolyL, u64* dst) {
+    const int64_t words = npolyL * c->L * c->N;
+    CK(cudaMemcpyAsync(dst, canonical, words * 8, cudaMemcpyDefault, c->stream));
+    return launch_ntt_fwd(c, dst, npolyL * c->L, c->N, limbmap_q(c));
+}
+
+// internal -> canonical through a device staging buffer
+int export_polys(hann_ctx* c, const u64* src, int64_t npolyL, u64* staging, u64* canonical_out) {
+    const int64_t words = npolyL * c->L * c->N;
+    CK(cudaMemcpyAsync(staging, src, words * 8, cudaMemcpyDeviceToDevice, c->stream));
+    RET(launch_ntt_inv(c, staging, npolyL * c->L, c->N, limbmap_q(c)));
+    CK(cudaMemcpyAsync(canonical_out, staging, words * 8, cudaMemcpyDefault, c->stream));
+    return HANN_OK;
+}
+
+int polys_of_kind(int kind) {
+    switch (kind) {
+        case HANN_KIND_POLY:
+        case HANN_KIND_PT: return 1;
+        case HANN_KIND_CT: return 2;
+        default: return 0;
+    }
+}
+
+// secret key residues in the transform domain for limbs 0..nlimbs-1, into dst[nlimbs][N]; s8 is device scratch [N]
+int upload_secret(hann_ctx* c, const int8_t* s_host, int nlimbs, int8_t* s8, u64* dst) {
+    CK(cudaMemcpyAsync(s8, s_host, c->N, cudaMemcpyHostToDevice, c->stream));
+    RET(launch_lift_i8(c, s8, nlimbs, dst));
+    LimbMap lm = nlimbs == c->L + 1 ? limbmap_qp(c) : limbmap_q(c);
+    return launch_ntt_fwd(c, dst, nlimbs, c->N, lm);
+}
+
+// ---- one key switch round on `items` polynomials already in coefficient form ------------------------------
+// c1c[items][L][N] (coefficients of the polynomials to switch, item stride L*N) -> u, lifted; combine is left to
+// the caller because its sources and targets differ between the callers.
+int ks_digits_to_lifted(hann_ctx* c, u64* c1c, int64_t items, u64* digits, int64_t digit_stride, int rot0, int rot_inc,
+                        int64_t u_items, u64* u, u64* lifted) {
+    const int L = c->L, N = c->N;
+    RET(launch_lift_digits(c, c1c, (int64_t)L * N, items, digits));
+    RET(launch_ntt_fwd(c, digits, items * L * (L + 1), N, limbmap_qp(c)));
+    RET(launch_ks_inner(c, digits, digit_stride, rot0, rot_inc, u_items, u));
+    // special-prime limbs of u back to coefficients (in place), lift, transform
+    RET(launch_ntt_inv(c, u + (int64_t)L * N, u_items * 2, (int64_t)(L + 1) * N, limbmap_single(L)));
+    RET(launch_moddown_lift(c, u, u_items * 2, lifted));
+    RET(launch_ntt_fwd(c, lifted, u_items * 2 * L, N, limbmap_q(c)));
+    return HANN_OK;
+}
+
+}  // namespace
+
+int ntt_configure(hann_ctx* c);
+
+// ================================================================================================ context
+
+extern "C" int hann_ctx_create(const hann_params* prm, hann_ctx** out) {
+    if (!prm || !out) return HANN_EINVAL;
+    if (prm->logN < 4 || prm->logN > 16 || prm->L < 1 || prm->L > HANN_MAX_PRIMES) return HANN_EINVAL;
+    const int N = 1 << prm->logN, n = N / 2, L = prm->L;
+    if (prm->R < 1 || prm->B < 1 || prm->R % prm->B || n % prm->R) return HANN_EINVAL;
+    if (prm->log_scale < 1 || prm->log_scale > 60) return HANN_EINVAL;
+    u64 mods[HANN_MAXL1];
+    for (int i = 0; i < L; i++) mods[i] = prm->q[i];
+    mods[L] = prm->p;
+    for (int i = 0; i <= L; i++) {
+        if (mods[i] >= (1ULL << 62) || mods[i] < 3 || (mods[i] - 1) % (2 * (u64)N) || !hm::is_prime(mods[i])) return HANN_EINVAL;
+        for (int k = 0; k < i; k++)
+            if (mods[k] == mods[i]) return HANN_EINVAL;
+    }
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || prm->device < 0 || prm->device >= ndev) {
+        cudaGetLastError();
+        return HANN_ECUDA;
+    }
+    hann_ctx* c = new (std::nothrow) hann_ctx();
+    if (!c) return HANN_ENOMEM;
+    c->prm = *prm;
+    c->logN = prm->logN; c->N = N; c->n = n; c->L = L; c->R = prm->R; c->B = prm->B; c->G = prm->R / prm->B;
+    c->device = prm->device;
+    c->stream = (cudaStream_t)prm->stream;
+    DeviceGuard dg(c->device);
+    if (!dg.ok) { delete c; return HANN_ECUDA; }
+
+    // per-limb constants and transform tables
+    std::vector<u64> twf((size_t)(L + 1) * N), twfs((size_t)(L + 1) * N), twi((size_t)(L + 1) * N), twis((size_t)(L + 1) * N);
+    std::vector<u64> pw(N), ipw(N);
+    for (int i = 0; i <= L; i++) {
+        const u64 q = mods[i];
+        c->mod[i] = q;
+        LimbConst& lc = c->lt.c[i];
+        lc.q = q;
+        lc.mu = (u64)((((unsigned __int128)1) << 64) / q);
+        lc.c64 = (u64)((((unsigned __int128)1) << 64) % q);
+        lc.c64s = hm::shoup(lc.c64, q);
+        lc.ninv = hm::invmod((u64)N % q, q);
+        lc.ninv_s = hm::shoup(lc.ninv, q);
+        lc.half = q / 2;
+        if (i < L) {
+            lc.pmod = prm->p % q;
+            lc.pinv = hm::invmod(lc.pmod, q);
+            lc.pinv_s = hm::shoup(lc.pinv, q);
+        } else {
+            lc.pmod = 0; lc.pinv = 0; lc.pinv_s = 0;
+        }
+        const u64 psi = hm::find_psi(q, N), ipsi = hm::invmod(psi, q);
+        pw[0] = ipw[0] = 1;
+        for (int k = 1; k < N; k++) {
+            pw[k] = hm::mulmod(pw[k - 1], psi, q);
+            ipw[k] = hm::mulmod(ipw[k - 1], ipsi, q);
+        }
+        for (int k = 0; k < N; k++) {
+            const int br = hm::bitrev(k, c->logN);
+            const size_t o = (size_t)i * N + k;
+            twf[o] = pw[br];  twfs[o] = hm::shoup(pw[br], q);
+            twi[o] = ipw[br]; twis[o] = hm::shoup(ipw[br], q);
+        }
+    }
+    // encode tables
+    const int nh = std::max(n / 2, 1);
+    std::vector<double2> T(nh), U(n);
+    c->hU_re.resize(n); c->hU_im.resize(n); c->h_uidx.resize(n);
+    for (int t = 0; t < nh; t++) { double cs, sn; hm::unit_root(t, n, &cs, &sn); T[t] = make_double2(cs, -sn + 0.0); }
+    for (int k = 0; k < n; k++) {
+        double cs, sn; hm::unit_root(k, 2L * N, &cs, &sn);
+        U[k] = make_double2(cs, -sn + 0.0);
+        c->hU_re[k] = U[k].x; c->hU_im[k] = U[k].y;
+    }
+    std::vector<int32_t> jinv(n);
+    std::vector<unsigned> gal(n);
+    {
+        long g = 1;
+        for (int j = 0; j < n; j++) {
+            gal[j] = (unsigned)g;
+            c->h_uidx[j] = (int32_t)((g - 1) / 4);
+            jinv[(g - 1) / 4] = j;
+            g = (g * 5) % (2L * N);
+        }
+    }
+    const size_t twb = (size_t)(L + 1) * N * 8;
+    bool ok = cudaMalloc(&c->tw_fwd, twb) == cudaSuccess && cudaMalloc(&c->tw_fwd_s, twb) == cudaSuccess &&
+              cudaMalloc(&c->tw_inv, twb) == cudaSuccess && cudaMalloc(&c->tw_inv_s, twb) == cudaSuccess &&
+              cudaMalloc(&c->fft_T, nh * sizeof(double2)) == cudaSuccess && cudaMalloc(&c->fft_U, n * sizeof(double2)) == cudaSuccess &&
+              cudaMalloc(&c->jinv, n * sizeof(int32_t)) == cudaSuccess && cudaMalloc(&c->galois_dev, n * sizeof(unsigned)) == cudaSuccess &&
+              cudaMalloc(&c->keytab_dev, n * sizeof(u64*)) == cudaSuccess;
+    if (ok) {
+        ok = cudaMemcpy(c->tw_fwd, twf.data(), twb, cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(c->tw_fwd_s, twfs.data(), twb, cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(c->tw_inv, twi.data(), twb, cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(c->tw_inv_s, twis.data(), twb, cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(c->fft_T, T.data(), nh * sizeof(double2), cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(c->fft_U, U.data(), n * sizeof(double2), cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(c->jinv, jinv.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(c->galois_dev, gal.data(), n * sizeof(unsigned), cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemset(c->keytab_dev, 0, n * sizeof(u64*)) == cudaSuccess;
+    }
+    c->h_galois = gal;
+    c->keytab_host.assign(n, nullptr);
+    for (int k = 0; k < HANN_NKINDS && ok; k++)
+        ok = cudaEventCreate(&c->ev[k][0]) == cudaSuccess && cudaEventCreate(&c->ev[k][1]) == cudaSuccess;
+    if (ok) ok = ntt_configure(c) == HANN_OK;
+    if (!ok) {
+        cudaGetLastError();
+        hann_ctx_destroy(c);
+        return HANN_ECUDA;
+    }
+    *out = c;
+    return HANN_OK;
+}
+
+extern "C" void hann_ctx_destroy(hann_ctx* c) {
+    if (!c) return;
+    DeviceGuard dg(c->device);
+    cudaStreamSynchronize(c->stream);
+    for (u64* k : c->keytab_host)
+        if (k) cudaFree(k);
+    cudaFree(c->tw_fwd); cudaFree(c->tw_fwd_s); cudaFree(c->tw_inv); cudaFree(c->tw_inv_s);
+    cudaFree(c->fft_T); cudaFree(c->fft_U); cudaFree(c->jinv); cudaFree(c->galois_dev); cudaFree(c->keytab_dev);
+    if (c->scratch) cudaFree(c->scratch);
+    for (int k = 0; k < HANN_NKINDS; k++) {
+        if (c->ev[k][0]) cudaEventDestroy(c->ev[k][0]);
+        if (c->ev[k][1]) cudaEventDestroy(c->ev[k][1]);
+    }
+    cudaGetLastError();
+    delete c;
+}
+
+extern "C" int64_t hann_sizeof(const hann_ctx* c, int what) {
+    if (!c) return HANN_EINVAL;
+    const int64_t L = c->L, N = c->N;
+    switch (what) {
+        case HANN_SIZE_POLY: return L * N * 8;
+        case HANN_SIZE_CT: return 2 * L * N * 8;
+        case HANN_SIZE_BABY: return (int64_t)c->B * 2 * L * N * 8;
+        case HANN_SIZE_PT_BLOCK: return (int64_t)c->R * L * N * 8;
+        case HANN_SIZE_INNER: return (int64_t)c->G * 2 * L * N * 8;
+        case HANN_SIZE_EVK: return L * 2 * (L + 1) * N * 8;
+        case HANN_SIZE_ROWS_PER_BLOCK: return c->n;
+        default: return HANN_EINVAL;
+    }
+}
+
+extern "C" int64_t hann_workspace_bytes(const hann_ctx* c, int64_t max_blocks) {
+    if (!c || max_blocks < 0) return HANN_EINVAL;
+    const int64_t items = std::max<int64_t>(1, std::min<int64_t>(max_blocks, 8));
+    int64_t w = std::max(ks_item_words(c) * items, prepare_words(c)) * 8;
+    w = std::max(w, (ks_item_words(c) + (int64_t)c->L * c->N) * 8);  // hann_keyswitch permutes its input first
+    w = std::max(w, encode_ws_bytes(c));
+    return w + kSlack;
+}
+
+extern "C" int hann_sync(hann_ctx* c) {
+    if (!c) return HANN_EINVAL;
+    DeviceGuard dg(c->device);
+    CK(cudaStreamSynchronize(c->stream));
+    return HANN_OK;
+}
+
+extern "C" const char* hann_last_error(const hann_ctx* c) { return c ? c->err.c_str() : "null context"; }
+
+extern "C" int hann_set_timing(hann_ctx* c, int enable) {
+    if (!c) return HANN_EINVAL;
+    c->timing = enable ? 1 : 0;
+    return HANN_OK;
+}
+
+extern "C" int hann_get_stats(hann_ctx* c, hann_stats* out) {
+    if (!c || !out) return HANN_EINVAL;
+    DeviceGuard dg(c->device);
+    float* field[HANN_NKINDS] = {&c->stats.ms_query_prepare, &c->stats.ms_encode, &c->stats.ms_score_level,
+                                 &c->stats.ms_rotate_sum, &c->stats.ms_keyswitch};
+    for (int k = 0; k < HANN_NKINDS; k++)
+        if (c->ev_pending[k]) {
+            CK(cudaEventSynchronize(c->ev[k][1]));
+            CK(cudaEventElapsedTime(field[k], c->ev[k][0], c->ev[k][1]));
+            c->ev_pending[k] = 0;
+        }
+    *out = c->stats;
+    return HANN_OK;
+}
+
+// ================================================================================================ exchange
+
+extern "C" int hann_import(hann_ctx* c, int kind, const uint64_t* canonical, int64_t count, void* internal_dev) {
+    if (!c) return HANN_EINVAL;
+    const int pk = polys_of_kind(kind);
+    if (!pk || !canonical || !internal_dev || count < 0) return fail(c, HANN_EINVAL, "hann_import: bad argument");
+    DeviceGuard dg(c->device);
+    RET(import_polys(c, canonical, count * pk, (u64*)internal_dev));
+    CK(cudaStreamSynchronize(c->stream));
+    return HANN_OK;
+}
+
+extern "C" int hann_export(hann_ctx* c, int kind, const void* internal_dev, int64_t count, uint64_t* canonical_out) {
+    if (!c) return HANN_EINVAL;
+    const int pk = polys_of_kind(kind);
+    if (!pk || !canonical_out || !internal_dev || count < 0) return fail(c, HANN_EINVAL, "hann_export: bad argument");
+    DeviceGuard dg(c->device);
+    // staged in pieces of at most 64 polynomials so that the scratch stays small
+    const int64_t total = count * pk, piece = 64;
+    RET(ensure_scratch(c, piece * c->L * c->N * 8));
+    for (int64_t p0 = 0; p0 < total; p0 += piece) {
+        const int64_t np = std::min(piece, total - p0);
+        RET(export_polys(c, (const u64*)internal_dev + p0 * c->L * c->N, np, (u64*)c->scratch, canonical_out + p0 * c->L * c->N));
+    }
+    CK(cudaStreamSynchronize(c->stream));
+    return HANN_OK;
+}
+
+// ================================================================================================ client side
+
+extern "C" int hann_keygen_from_samples(hann_ctx* c, const int8_t* s, int n_rot, const int32_t* rot, const uint64_t* a,
+                                        const int8_t* e, uint64_t* evk_out) {
+    if (!c) return HANN_EINVAL;
+    if (!s || !rot || !a || !e || !evk_out || n_rot < 0) return fail(c, HANN_EINVAL, "hann_keygen_from_samples: bad argument");
+    const int L = c->L, N = c->N;
+    for (int i = 0; i < n_rot; i++)
+        if (rot[i] < 1 || rot[i] >= c->n) return fail(c, HANN_ESHAPE, "hann_keygen_from_samples: rotation out of range");
+    DeviceGuard dg(c->device);
+    const int64_t W = (int64_t)N, keyw = (int64_t)L * (L + 1) * W;
+    // scratch: s_hat[L+1][N], A[L][L+1][N], AS[L][L+1][N], int8: s, s', e[L][N]
+    const int64_t words = (L + 1) * W + 2 * keyw;
+    RET(ensure_scratch(c, words * 8 + align256(N) * 2 + align256((int64_t)L * N) + kSlack));
+    Arena ar{(char*)c->scratch, 0, c->scratch_bytes};
+    u64* shat = ar.take<u64>((L + 1) * W);
+    u64* A = ar.take<u64>(keyw);
+    u64* AS = ar.take<u64>(keyw);
+    int8_t* s8 = ar.take<int8_t>(N);
+    int8_t* sp8 = ar.take<int8_t>(N);
+    int8_t* e8 = ar.take<int8_t>((int64_t)L * N);
+    RET(upload_secret(c, s, L + 1, s8, shat));
+    std::vector<int8_t> sprime(N);
+    for (int r = 0; r < n_rot; r++) {
+        const unsigned k = c->h_galois[rot[r]];
+        for (long i = 0; i < N; i++) {  // s'(X) = s(X^k)
+            long ex = (i * (long)k) % (2L * N);
+            if (ex < N) sprime[ex] = s[i];
+            else sprime[ex - N] = (int8_t)(-s[i]);
+        }
+        const u64* a_r = a + (int64_t)r * keyw;
+        CK(cudaMemcpyAsync(A, a_r, keyw * 8, cudaMemcpyHostToDevice, c->stream));
+        CK(cudaMemcpyAsync(sp8, sprime.data(), N, cudaMemcpyHostToDevice, c->stream));
+        CK(cudaMemcpyAsync(e8, e + (int64_t)r * L * N, (size_t)L * N, cudaMemcpyHostToDevice, c->stream));
+        RET(launch_ntt_fwd(c, A, (int64_t)L * (L + 1), N, limbmap_qp(c)));
+        RET(launch_mul(c, A, shat, L + 1, AS, (int64_t)L * (L + 1), limbmap_qp(c)));
+        RET(launch_ntt_inv(c, AS, (int64_t)L * (L + 1), N, limbmap_qp(c)));
+        RET(launch_evk_finish(c, AS, e8, sp8, AS));
+        u64* out_r = evk_out + (int64_t)r * 2 * keyw;
+        for (int j = 0; j < L; j++) {
+            CK(cudaMemcpyAsync(out_r + ((int64_t)j * 2 + 0) * (L + 1) * W, AS + (int64_t)j * (L + 1) * W, (size_t)(L + 1) * W * 8,
+                               cudaMemcpyDeviceToHost, c->stream));
+            memcpy(out_r + ((int64_t)j * 2 + 1) * (L + 1) * W, a_r + (int64_t)j * (L + 1) * W, (size_t)(L + 1) * W * 8);
+        }
+        CK(cudaStreamSynchronize(c->stream));  // sprime (host) is reused by the next rotation
+    }
+    return HANN_OK;
+}
+
+extern "C" int hann_encrypt_query(hann_ctx* c, const int8_t* s, const float* q, int dim, const uint64_t* a, const int8_t* e,
+                                  uint64_t* ct_out) {
+    if (!c) return HANN_EINVAL;
+    if (!s || !q || !a || !e || !ct_out) return fail(c, HANN_EINVAL, "hann_encrypt_query: null pointer");
+    if (dim < 1 || dim > c->R) return fail(c, HANN_ESHAPE, "hann_encrypt_query: dim must be in 1..R");
+    const int L = c->L, N = c->N, n = c->n;
+    DeviceGuard dg(c->device);
+    const int64_t LN = (int64_t)L * N;
+    RET(ensure_scratch(c, (4 * LN) * 8 + n * 8 + n * 16 + 2 * align256(N) + kSlack));
+    Arena ar{(char*)c->scratch, 0, c->scratch_bytes};
+    u64* shat = ar.take<u64>(LN);
+    u64* A = ar.take<u64>(LN);
+    u64* AS = ar.take<u64>(LN);
+    u64* M = ar.take<u64>(LN);
+    double* z = ar.take<double>(n);
+    double2* fbuf = ar.take<double2>(n);
+    int8_t* s8 = ar.take<int8_t>(N);
+    int8_t* e8 = ar.take<int8_t>(N);
+    std::vector<double> zh(n);
+    for (int i = 0; i < n; i++) {
+        int d = i % c->R;
+        zh[i] = d < dim ? (double)q[d] : 0.0;
+    }
+    CK(cudaMemcpyAsync(z, zh.data(), n * 8, cudaMemcpyHostToDevice, c->stream));
+    CK(cudaMemcpyAsync(A, a, LN * 8, cudaMemcpyHostToDevice, c->stream));
+    CK(cudaMemcpyAsync(e8, e, N, cudaMemcpyHostToDevice, c->stream));
+    RET(upload_secret(c, s, L, s8, shat));
+    RET(launch_encode_slots(c, z, M, fbuf));
+    RET(launch_ntt_fwd(c, A, L, N, limbmap_q(c)));
+    RET(launch_mul(c, A, shat, L, AS, L, limbmap_q(c)));
+    RET(launch_ntt_inv(c, AS, L, N, limbmap_q(c)));
+    RET(launch_encrypt_finish(c, AS, e8, M, AS));
+    CK(cudaMemcpyAsync(ct_out, AS, LN * 8, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    memcpy(ct_out + LN, a, LN * 8);
+    return HANN_OK;
+}
+
+extern "C" int hann_decrypt_scores(hann_ctx* c, const int8_t* s, const uint64_t* ct, int64_t count, int log_scale_out,
+                                   double* scores, double* imag_or_null) {
+    if (!c) return HANN_EINVAL;
+    if (!s || !ct || !scores || count < 0) return fail(c, HANN_EINVAL, "hann_decrypt_scores: bad argument");
+    const int L = c->L, N = c->N, n = c->n;
+    DeviceGuard dg(c->device);
+    const int64_t LN = (int64_t)L * N;
+    RET(ensure_scratch(c, 4 * LN * 8 + align256(N) + kSlack));
+    Arena ar{(char*)c->scratch, 0, c->scratch_bytes};
+    u64* shat = ar.take<u64>(LN);
+    u64* CT = ar.take<u64>(2 * LN);
+    u64* MU = ar.take<u64>(LN);
+    int8_t* s8 = ar.take<int8_t>(N);
+    RET(upload_secret(c, s, L, s8, shat));
+    std::vector<u64> mu(LN);
+    std::vector<long double> real(N);
+    std::vector<double> re(n), im(n);
+    const long double inv_scale = ldexpl(1.0L, -log_scale_out);
+    for (int64_t i = 0; i < count; i++) {
+        RET(import_polys(c, ct + i * 2 * LN, 2, CT));
+        RET(launch_mul(c, CT + LN, shat, L, MU, L, limbmap_q(c)));   // c1 * s
+        RET(launch_add(c, MU, CT, MU, L, limbmap_q(c)));             // + c0
+        RET(launch_ntt_inv(c, MU, L, N, limbmap_q(c)));
+        CK(cudaMemcpyAsync(mu.data(), MU, LN * 8, cudaMemcpyDeviceToHost, c->stream));
+        CK(cudaStreamSynchronize(c->stream));
+        hm::crt_to_real(mu.data(), L, N, c->mod, real.data());
+        // slots: a_k = (mu_k + i mu_{k+n}) conj(U[k]);  z_j * scale = sum_k a_k exp(+2 pi i u_j k / n)
+        for (int k = 0; k < n; k++) {
+            const double mr = (double)(real[k] * inv_scale), mi = (double)(real[k + n] * inv_scale);
+            const double ur = c->hU_re[k], ui = -c->hU_im[k];
+            re[k] = mr * ur - mi * ui;
+            im[k] = mr * ui + mi * ur;
+        }
+        hm::fft_inplace(re.data(), im.data(), n, c->logN - 1, +1);
+        for (int j = 0; j < n; j++) {
+            scores[i * n + j] = re[c->h_uidx[j]];
+            if (imag_or_null) imag_or_null[i * n + j] = im[c->h_uidx[j]];
+        }
+    }
+    return HANN_OK;
+}
+
+// ================================================================================================ server side
+
+extern "C" int hann_load_keys(hann_ctx* c, const uint64_t* evk, int n_rot, const int32_t* rot) {
+    if (!c) return HANN_EINVAL;
+    if (!evk || !rot || n_rot < 0) return fail(c, HANN_EINVAL, "hann_load_keys: bad argument");
+    const int L = c->L, N = c->N;
+    for (int i = 0; i < n_rot; i++)
+        if (rot[i] < 1 || rot[i] >= c->n) return fail(c, HANN_ESHAPE, "hann_load_keys: rotation out of range");
+    DeviceGuard dg(c->device);
+    const int64_t keyw = (int64_t)L * 2 * (L + 1) * N;
+    RET(ensure_scratch(c, keyw * 8));
+    for (int i = 0; i < n_rot; i++) {
+        const int r = rot[i];
+        if (!c->keytab_host[r]) {
+            u64* buf = nullptr;
+            if (cudaMalloc(&buf, keyw * 8) != cudaSuccess) {
+                cudaGetLastError();
+                return fail(c, HANN_ENOMEM, "hann_load_keys: device allocation failed");
+            }
+            c->keytab_host[r] = buf;
+        }
+        u64* tmp = (u64*)c->scratch;
+        CK(cudaMemcpyAsync(tmp, evk + (int64_t)i * keyw, keyw * 8, cudaMemcpyDefault, c->stream));
+        RET(launch_ntt_fwd(c, tmp, (int64_t)L * 2 * (L + 1), N, limbmap_qp(c)));
+        // store phi_k^{-1}(key): the inner product then runs on unpermuted digits and the automorphism is applied
+        // once, to its much smaller result
+        const unsigned k = c->h_galois[r];
+        const unsigned kinv = c->h_galois[(c->n - r) % c->n];  // 5^{-r} = 5^{n-r} (5 has order n modulo 2N)
+        (void)k;
+        RET(launch_permute(c, tmp, c->keytab_host[r], (int64_t)L * 2 * (L + 1), kinv));
+        CK(cudaStreamSynchronize(c->stream));
+    }
+    CK(cudaMemcpy(c->keytab_dev, c->keytab_host.data(), c->keytab_host.size() * sizeof(u64*), cudaMemcpyHostToDevice));
+    return HANN_OK;
+}
+
+extern "C" int hann_query_prepare(hann_ctx* c, const void* ct_dev, void* baby_dev, void* ws, size_t ws_bytes) {
+    if (!c) return HANN_EINVAL;
+    if (!ct_dev || !baby_dev) return fail(c, HANN_EINVAL, "hann_query_prepare: null pointer");
+    const int L = c->L, N = c->N, B = c->B;
+    const int64_t LN = (int64_t)L * N, L1N = (int64_t)(L + 1) * N, ctw = 2 * LN;
+    for (int r = 1; r < B; r++)
+        if (!c->keytab_host[r]) return fail(c, HANN_ENOKEY, "hann_query_prepare: a baby-step rotation key is not loaded");
+    DeviceGuard dg(c->device);
+    Timer tm(c, 0);
+    const u64* ct = (const u64*)ct_dev;
+    u64* baby = (u64*)baby_dev;
+    CK(cudaMemcpyAsync(baby, ct, ctw * 8, cudaMemcpyDeviceToDevice, c->stream));  // rotation 0
+    if (B == 1) return HANN_OK;
+    if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_query_prepare: workspace missing or not 256-byte aligned");
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
+    u64* c1c = ar.take<u64>(LN);
+    u64* digits = ar.take<u64>(L * L1N);
+    u64* u = ar.take<u64>((int64_t)(B - 1) * 2 * L1N);
+    u64* lifted = ar.take<u64>((int64_t)(B - 1) * 2 * LN);
+    if (!c1c || !digits || !u || !lifted) return fail(c, HANN_EWORKSPACE, "hann_query_prepare: workspace too small");
+    CK(cudaMemcpyAsync(c1c, ct + LN, LN * 8, cudaMemcpyDeviceToDevice, c->stream));
+    RET(launch_ntt_inv(c, c1c, L, N, limbmap_q(c)));
+    // one digit set, B-1 keys: item i uses rotation 1 + i
+    RET(ks_digits_to_lifted(c, c1c, 1, digits, 0, 1, 1, B - 1, u, lifted));
+    RET(launch_moddown_combine(c, u, lifted, B - 1, 1, 1, ct, 0, nullptr, 0, baby + ctw, baby + ctw + LN, ctw));
+    return HANN_OK;
+}
+
+extern "C" int hann_encode_candidates(hann_ctx* c, const float* rows_dev, int64_t n_rows, int dim, void* pt_dev, void* ws,
+                                      size_t ws_bytes) {
+    if (!c) return HANN_EINVAL;
+    if (n_rows < 0 || (n_rows > 0 && (!rows_dev || !pt_dev))) return fail(c, HANN_EINVAL, "hann_encode_candidates: bad argument");
+    if (dim < 1 || dim > c->R) return fail(c, HANN_ESHAPE, "hann_encode_candidates: dim must be in 1..R");
+    if (n_rows == 0) return HANN_OK;
+    if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_encode_candidates: workspace missing or not 256-byte aligned");
+    if ((int64_t)ws_bytes < encode_ws_bytes(c)) return fail(c, HANN_EWORKSPACE, "hann_encode_candidates: workspace too small");
+    DeviceGuard dg(c->device);
+    Timer tm(c, 1);
+    const int64_t n = c->n, nblk = (n_rows + n - 1) / n, ptw = (int64_t)c->R * c->L * c->N;
+    for (int64_t blk = 0; blk < nblk; blk++) {
+        const int64_t rows_here = std::min(n, n_rows - blk * n);
+        u64* pt = (u64*)pt_dev + blk * ptw;
+        RET(launch_encode_rows(c, rows_dev + blk * n * dim, rows_here, dim, pt, ws));
+        RET(launch_ntt_fwd(c, pt, (int64_t)c->R * c->L, c->N, limbmap_q(c)));
+    }
+    return HANN_OK;
+}
+
+extern "C" int hann_score_level(hann_ctx* c, const void* baby_dev, const void* pt_dev, int64_t n_blocks, void* inner_dev,
+                                void* ws, size_t ws_bytes) {
+    (void)ws; (void)ws_bytes;  // the multiply-accumulate needs no scratch
+    if (!c) return HANN_EINVAL;
+    if (n_blocks < 0 || (n_blocks > 0 && (!baby_dev || !pt_dev || !inner_dev))) return fail(c, HANN_EINVAL, "hann_score_level: bad argument");
+    DeviceGuard dg(c->device);
+    Timer tm(c, 2);
+    return launch_mac(c, (const u64*)baby_dev, (const u64*)pt_dev, n_blocks, (u64*)inner_dev);
+}
+
+extern "C" int hann_rotate_sum(hann_ctx* c, const void* inner_dev, int64_t n_blocks, void* score_ct_dev, void* ws, size_t ws_bytes) {
+    if (!c) return HANN_EINVAL;
+    if (n_blocks < 0 || (n_blocks > 0 && (!inner_dev || !score_ct_dev))) return fail(c, HANN_EINVAL, "hann_rotate_sum: bad argument");
+    if (n_blocks == 0) return HANN_OK;
+    const int L = c->L, N = c->N, G = c->G, B = c->B;
+    const int64_t LN = (int64_t)L * N, L1N = (int64_t)(L + 1) * N, ctw = 2 * LN;
+    const u64* inner = (const u64*)inner_dev;
+    u64* score = (u64*)score_ct_dev;
+    DeviceGuard dg(c->device);
+    Timer tm(c, 3);
+    if (G == 1) {
+        CK(cudaMemcpyAsync(score, inner, n_blocks * ctw * 8, cudaMemcpyDeviceToDevice, c->stream));
+        return HANN_OK;
+    }
+    if (!c->keytab_host[B]) return fail(c, HANN_ENOKEY, "hann_rotate_sum: the key of rotation B is not loaded");
+    if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_rotate_sum: workspace missing or not 256-byte aligned");
+    // as many blocks per round as the workspace holds
+    int64_t ch = ((int64_t)ws_bytes - kSlack) / (ks_item_words(c) * 8);
+    if (ch < 1) return fail(c, HANN_EWORKSPACE, "hann_rotate_sum: workspace too small");
+    ch = std::min<int64_t>(std::min<int64_t>(ch, n_blocks), 8);
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
+    u64* c1c = ar.take<u64>(ch * LN);
+    u64* digits = ar.take<u64>(ch * L * L1N);
+    u64* u = ar.take<u64>(ch * 2 * L1N);
+    u64* lifted = ar.take<u64>(ch * 2 * LN);
+    u64* tmp = ar.take<u64>(ch * ctw);
+    if (!c1c || !digits || !u || !lifted || !tmp) return fail(c, HANN_EWORKSPACE, "hann_rotate_sum: workspace too small");
+    for (int64_t b0 = 0; b0 < n_blocks; b0 += ch) {
+        const int64_t nb = std::min(ch, n_blocks - b0);
+        const u64* old = inner + (b0 * G + (G - 1)) * ctw;  // acc = inner[G-1]
+        int64_t old_stride = (int64_t)G * ctw;
+        for (int g = G - 2; g >= 0; g--) {
+            u64* out = (g % 2 == 0) ? score + b0 * ctw : tmp;
+            // c1 of every accumulator -> coefficients
+            CK(cudaMemcpy2DAsync(c1c, LN * 8, old + LN, old_stride * 8, LN * 8, nb, cudaMemcpyDeviceToDevice, c->stream));
+            RET(launch_ntt_inv(c, c1c, nb * L, N, limbmap_q(c)));
+            RET(ks_digits_to_lifted(c, c1c, nb, digits, (int64_t)L * L1N, B, 0, nb, u, lifted));
+            RET(launch_moddown_combine(c, u, lifted, nb, B, 0, old, old_stride, inner + (b0 * G + g) * ctw, (int64_t)G * ctw, out,
+                                       out + LN, ctw));
+            old = out;
+            old_stride = ctw;
+        }
+    }
+    return HANN_OK;
+}
+
+extern "C" int hann_keyswitch(hann_ctx* c, int rot, const void* poly_dev, void* ks0_dev, void* ks1_dev, void* ws, size_t ws_bytes) {
+    if (!c) return HANN_EINVAL;
+    if (!poly_dev || !ks0_dev || !ks1_dev) return fail(c, HANN_EINVAL, "hann_keyswitch: null pointer");
+    if (rot < 1 || rot >= c->n) return fail(c, HANN_ESHAPE, "hann_keyswitch: rotation out of range");
+    if (!c->keytab_host[rot]) return fail(c, HANN_ENOKEY, "hann_keyswitch: key not loaded");
+    if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_keyswitch: workspace missing or not 256-byte aligned");
+    const int L = c->L, N = c->N;
+    const int64_t LN = (int64_t)L * N, L1N = (int64_t)(L + 1) * N;
+    DeviceGuard dg(c->device);
+    Timer tm(c, 4);
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
+    u64* c1c = ar.take<u64>(LN);
+    u64* digits = ar.take<u64>(L * L1N);
+    u64* u = ar.take<u64>(2 * L1N);
+    u64* lifted = ar.take<u64>(2 * LN);
+    if (!c1c || !digits || !u || !lifted) return fail(c, HANN_EWORKSPACE, "hann_keyswitch: workspace too small");
+    // the stored key is phi_k^{-1}(evk): switch phi_k^{-1}(d) and apply phi_k to the result
+    const unsigned kinv = c->h_galois[(c->n - rot) % c->n];
+    RET(launch_permute(c, (const u64*)poly_dev, c1c, L, kinv));
+    RET(launch_ntt_inv(c, c1c, L, N, limbmap_q(c)));
+    RET(ks_digits_to_lifted(c, c1c, 1, digits, 0, rot, 0, 1, u, lifted));
+    RET(launch_moddown_combine(c, u, lifted, 1, rot, 0, nullptr, 0, nullptr, 0, (u64*)ks0_dev, (u64*)ks1_dev, 0));
+    return HANN_OK;
+}
+
+// ================================================================================================ host-buffer level
+
+namespace {
+struct LevelPlan {
+    int64_t nblk, ct, baby, rows, pt, inner, score, stage, ws, total;
+};
+LevelPlan plan_level(const hann_ctx* c, int64_t n_rows, int dim) {
+    LevelPlan p;
+    const int64_t ctb = hann_sizeof(c, HANN_SIZE_CT);
+    p.nblk = (n_rows + c->n - 1) / c->n;
+    p.ct = align256(ctb);
+    p.baby = align256(hann_sizeof(c, HANN_SIZE_BABY));
+    p.rows = align256(n_rows * (int64_t)dim * 4);
+    p.pt = align256(p.nblk * hann_sizeof(c, HANN_SIZE_PT_BLOCK));
+    p.inner = align256(p.nblk * hann_sizeof(c, HANN_SIZE_INNER));
+    p.score = align256(p.nblk * ctb);
+    p.stage = align256(p.nblk * ctb);
+    p.ws = align256(hann_workspace_bytes(c, p.nblk));
+    p.total = p.ct + p.baby + p.rows + p.pt + p.inner + p.score + p.stage + p.ws;
+    return p;
+}
+}  // namespace
+
+extern "C" int64_t hann_level_host_bytes(const hann_ctx* c, int64_t n_rows) {
+    if (!c || n_rows < 0) return HANN_EINVAL;
+    return plan_level(c, n_rows, c->R).total;
+}
+
+extern "C" int hann_score_level_host(hann_ctx* c, const uint64_t* ct_host, const float* rows_host, int64_t n_rows, int dim,
+                                     uint64_t* score_ct_host, void* ws_dev, size_t ws_bytes) {
+    if (!c) return HANN_EINVAL;
+    if (!ct_host || !rows_host || !score_ct_host || n_rows < 1) return fail(c, HANN_EINVAL, "hann_score_level_host: bad argument");
+    if (dim < 1 || dim > c->R) return fail(c, HANN_ESHAPE, "hann_score_level_host: dim must be in 1..R");
+    if (!ws_dev || ((uintptr_t)ws_dev & 255)) return fail(c, HANN_EWORKSPACE, "hann_score_level_host: workspace missing or not 256-byte aligned");
+    const LevelPlan p = plan_level(c, n_rows, dim);
+    if ((int64_t)ws_bytes < p.total) return fail(c, HANN_EWORKSPACE, "hann_score_level_host: workspace too small");
+    DeviceGuard dg(c->device);
+    char* b = (char*)ws_dev;
+    u64* ct = (u64*)b; b += p.ct;
+    u64* baby = (u64*)b; b += p.baby;
+    float* rows = (float*)b; b += p.rows;
+    u64* pt = (u64*)b; b += p.pt;
+    u64* inner = (u64*)b; b += p.inner;
+    u64* score = (u64*)b; b += p.score;
+    u64* stage = (u64*)b; b += p.stage;
+    void* ws = b;
+    CK(cudaMemcpyAsync(rows, rows_host, (size_t)n_rows * dim * 4, cudaMemcpyHostToDevice, c->stream));
+    RET(import_polys(c, ct_host, 2, ct));
+    RET(hann_query_prepare(c, ct, baby, ws, (size_t)p.ws));
+    RET(hann_encode_candidates(c, rows, n_rows, dim, pt, ws, (size_t)p.ws));
+    RET(hann_score_level(c, baby, pt, p.nblk, inner, ws, (size_t)p.ws));
+    RET(hann_rotate_sum(c, inner, p.nblk, score, ws, (size_t)p.ws));
+    RET(export_polys(c, score, p.nblk * 2, stage, score_ct_host));
+    CK(cudaStreamSynchronize(c->stream));
+    return HANN_OK;
+}

@@ -1,0 +1,93 @@
+// Private declarations shared by the translation units of the library.
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "../../include/hann.h"
+#include "modarith.cuh"
+
+#define HANN_NKINDS 5  // timed call kinds: query_prepare, encode, score_level, rotate_sum, keyswitch
+
+struct hann_ctx {
+    hann_params prm;
+    int logN = 0, N = 0, n = 0, L = 0, R = 0, B = 0, G = 0;
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    u64 mod[HANN_MAXL1] = {};  // q_0..q_{L-1}, p
+    LimbTable lt = {};
+    // transform tables on the device, [L+1][N] each: psi^brev(k) and psi^-brev(k) with their Shoup companions
+    u64 *tw_fwd = nullptr, *tw_fwd_s = nullptr, *tw_inv = nullptr, *tw_inv_s = nullptr;
+    // encode tables on the device
+    double2* fft_T = nullptr;  // [n/2] exp(-2 pi i t / n)
+    double2* fft_U = nullptr;  // [n]   exp(-i pi k / N)
+    int32_t* jinv = nullptr;   // [n]   jinv[u_j] = j with u_j = (5^j mod 2N - 1)/4
+    unsigned* galois_dev = nullptr;  // [n] 5^r mod 2N
+    std::vector<unsigned> h_galois;
+    // host copies used by decode
+    std::vector<double> hU_re, hU_im;
+    std::vector<int32_t> h_uidx;
+    // evaluation keys by rotation: device buffers [L][2][L+1][N], transformed and permuted by the inverse
+    // automorphism so that the key-switch inner product reads keys and digits contiguously
+    std::vector<u64*> keytab_host;
+    u64** keytab_dev = nullptr;  // [n] device copy of keytab_host
+    // growable device scratch of the exchange and client calls (never used by the server-side scoring calls)
+    void* scratch = nullptr;
+    int64_t scratch_bytes = 0;
+    // statistics
+    hann_stats stats = {};
+    int timing = 0;
+    cudaEvent_t ev[HANN_NKINDS][2] = {};
+    int ev_pending[HANN_NKINDS] = {};
+    std::string err;
+};
+
+// ---- host mathematics (hostmath.cpp)
+namespace hm {
+u64 mulmod(u64 a, u64 b, u64 q);
+u64 powmod(u64 a, u64 e, u64 q);
+u64 invmod(u64 a, u64 q);
+bool is_prime(u64 n);
+u64 find_psi(u64 q, int N);
+u64 shoup(u64 w, u64 q);  // floor(w * 2^64 / q)
+int bitrev(int x, int bits);
+void unit_root(long t, long den, double* c, double* s);  // exp(2 pi i t/den), correctly rounded
+// residues [L][N] -> centred integers in (-Q/2, Q/2] as long double
+void crt_to_real(const u64* res, int L, int N, const u64* q, long double* out);
+void fft_inplace(double* re, double* im, int n, int logn, int sign);
+}  // namespace hm
+
+// ---- launchers: each enqueues on ctx->stream, counts its launches and returns HANN_OK or HANN_ECUDA
+int check_launch(hann_ctx* c, const char* what);
+
+// transforms of npoly polynomials; polynomial p starts at data + p*stride and uses modulus lm.limb[p % lm.period]
+int launch_ntt_fwd(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
+int launch_ntt_inv(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
+LimbMap limbmap_q(const hann_ctx* c);   // period L: limbs 0..L-1
+LimbMap limbmap_qp(const hann_ctx* c);  // period L+1: limbs 0..L
+LimbMap limbmap_single(int limb);
+
+// encode (coefficient-domain residues out; the caller transforms)
+int launch_encode_rows(hann_ctx* c, const float* rows, int64_t rows_in_block, int dim, u64* pt_block, void* ws);
+int launch_encode_slots(hann_ctx* c, const double* z_dev, u64* poly_out, void* ws);
+int64_t encode_ws_bytes(const hann_ctx* c);
+
+// scoring
+int launch_mac(hann_ctx* c, const u64* baby, const u64* pt, int64_t n_blocks, u64* inner);
+
+// key switching pieces
+int launch_lift_digits(hann_ctx* c, const u64* src, int64_t src_stride, int64_t nitems, u64* digits);
+int launch_ks_inner(hann_ctx* c, const u64* digits, int64_t digit_stride, int rot0, int rot_inc, int64_t nitems, u64* u);
+int launch_moddown_lift(hann_ctx* c, const u64* u, int64_t npoly, u64* lifted);
+int launch_moddown_combine(hann_ctx* c, const u64* u, const u64* lifted, int64_t nitems, int rot0, int rot_inc, const u64* c0,
+                           int64_t c0_stride, const u64* addend, int64_t addend_stride, u64* out0, u64* out1,
+                           int64_t out_stride);
+int launch_permute(hann_ctx* c, const u64* src, u64* dst, int64_t npoly, unsigned k);
+
+// helpers of the client half
+int launch_lift_i8(hann_ctx* c, const int8_t* v, int nlimbs, u64* out);
+int launch_mul(hann_ctx* c, const u64* a, const u64* b, int bperiod, u64* out, int64_t npoly, const LimbMap& lm);
+int launch_add(hann_ctx* c, const u64* a, const u64* b, u64* out, int64_t npoly, const LimbMap& lm);
+int launch_evk_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const int8_t* sprime, u64* b_out);
+int launch_encrypt_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const u64* m, u64* c0_out);

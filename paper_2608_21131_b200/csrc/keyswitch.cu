@@ -1,0 +1,313 @@
+// Element-wise kernels of the scoring path: ciphertext x plaintext multiply-accumulate, the pieces of hybrid key
+// switching (digit lift, inner product with the evaluation key, ModDown), the automorphism gather, and the small
+// helpers of the client half.  All polynomials are [.][limb][N] arrays of 64-bit residues in [0, q).
+#include "internal.h"
+
+namespace {
+
+constexpr int kThreads = 256;
+
+inline int grid_for(int64_t work, int per_block = kThreads, int cap = 148 * 16) {
+    int64_t g = (work + per_block - 1) / per_block;
+    if (g > cap) g = cap;
+    if (g < 1) g = 1;
+    return (int)g;
+}
+
+// ------------------------------------------------------------------------------------------ multiply-accumulate
+
+// inner[blk][g][comp][l][x] = sum_b pt[blk][g][b][l][x] * baby[b][comp][l][x] mod q_l.
+// One thread owns one (l, x) position for a range of (blk, g) pairs; products are accumulated in 128 bits and
+// reduced once per output.
+__global__ void __launch_bounds__(kThreads) k_mac(const u64* __restrict__ baby, const u64* __restrict__ pt,
+                                                  u64* __restrict__ inner, int N, int L, int B, int G,
+                                                  long long n_bg, LimbTable lt) {
+    const long long LN = (long long)L * N;
+    for (long long pos = (long long)blockIdx.x * kThreads + threadIdx.x; pos < LN; pos += (long long)gridDim.x * kThreads) {
+        const int l = (int)(pos / N);
+        const LimbConst& lc = lt.c[l];
+        for (long long bg = blockIdx.y; bg < n_bg; bg += gridDim.y) {
+            const u64* p = pt + bg * B * LN + pos;
+            u64 h0 = 0, l0 = 0, h1 = 0, l1 = 0;
+            for (int b = 0; b < B; b++) {
+                u64 v = __ldcs(p + (long long)b * LN);
+                mac128(h0, l0, v, baby[((long long)b * 2 + 0) * LN + pos]);
+                mac128(h1, l1, v, baby[((long long)b * 2 + 1) * LN + pos]);
+            }
+            u64* o = inner + bg * 2 * LN + pos;
+            o[0] = reduce128(h0, l0, lc);
+            o[LN] = reduce128(h1, l1, lc);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------ key switching
+
+// digits[item][j][i][x] = centred lift of src[item][j][x] (a residue mod q_j, coefficient domain) reduced mod
+// modulus i, for j < L, i <= L.
+__global__ void __launch_bounds__(kThreads) k_lift_digits(const u64* __restrict__ src, long long src_stride,
+                                                          u64* __restrict__ digits, int N, int L, long long nitems,
+                                                          LimbTable lt) {
+    const long long total = nitems * L * N;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const int x = (int)(idx % N);
+        const int j = (int)((idx / N) % L);
+        const long long item = idx / ((long long)N * L);
+        const u64 v = src[item * src_stride + (long long)j * N + x];
+        const u64 qj = lt.c[j].q;
+        const bool neg = v > lt.c[j].half;
+        const u64 mag = neg ? qj - v : v;
+        u64* d = digits + ((item * L + j) * (L + 1)) * N + x;
+        for (int i = 0; i <= L; i++) {
+            u64 r = barrett64(mag, lt.c[i]);
+            d[(long long)i * N] = (neg && r) ? lt.c[i].q - r : r;
+        }
+    }
+}
+
+// u[item][comp][i][x] = sum_j digits[item_d][j][i][x] * key[j][comp][i][x] mod modulus i.
+// digit_stride = 0 shares one digit set among all items (hoisted rotations of one ciphertext); the key of item
+// `it` is keytab[rot0 + it*rot_inc].
+__global__ void __launch_bounds__(kThreads) k_ks_inner(const u64* __restrict__ digits, long long digit_stride,
+                                                       const u64* const* __restrict__ keytab, int rot0, int rot_inc,
+                                                       u64* __restrict__ u, int N, int L, long long nitems,
+                                                       LimbTable lt) {
+    const long long L1N = (long long)(L + 1) * N;
+    const long long total = nitems * L1N;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const long long item = idx / L1N;
+        const long long pos = idx % L1N;  // i*N + x
+        const int i = (int)(pos / N);
+        const u64* key = keytab[rot0 + (int)item * rot_inc];
+        const u64* d = digits + item * digit_stride + pos;
+        u64 h0 = 0, l0 = 0, h1 = 0, l1 = 0;
+        for (int j = 0; j < L; j++) {
+            u64 dv = d[(long long)j * L1N];
+            mac128(h0, l0, dv, __ldcs(key + ((long long)j * 2 + 0) * L1N + pos));
+            mac128(h1, l1, dv, __ldcs(key + ((long long)j * 2 + 1) * L1N + pos));
+        }
+        u64* o = u + item * 2 * L1N + pos;
+        o[0] = reduce128(h0, l0, lt.c[i]);
+        o[L1N] = reduce128(h1, l1, lt.c[i]);
+    }
+}
+
+// lifted[poly][i][x] = centred lift of up[poly][x] (residue mod p, coefficient domain) reduced mod q_i.
+// up is the special-prime limb inside u: poly = item*2 + comp lives at u + poly*(L+1)*N + L*N.
+__global__ void __launch_bounds__(kThreads) k_moddown_lift(const u64* __restrict__ u, u64* __restrict__ lifted, int N,
+                                                           int L, long long npoly, LimbTable lt) {
+    const long long total = npoly * N;
+    const u64 p = lt.c[L].q, half = lt.c[L].half;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const long long poly = idx / N;
+        const int x = (int)(idx % N);
+        const u64 v = u[poly * (L + 1) * N + (long long)L * N + x];
+        const bool neg = v > half;
+        const u64 mag = neg ? p - v : v;
+        for (int i = 0; i < L; i++) {
+            u64 r = barrett64(mag, lt.c[i]);
+            lifted[(poly * L + i) * N + x] = (neg && r) ? lt.c[i].q - r : r;
+        }
+    }
+}
+
+// out[item][comp][i][t] = (u[item][comp][i][s] - lifted[item][comp][i][s]) * p^{-1}
+//                         + (comp == 0 ? c0[item][i][s] : 0) + addend[item][comp][i][t],   s = galois source of t
+// for the Galois element of rotation rot0 + item*rot_inc (rotation 0 = identity).  All arrays in the transform domain.
+__global__ void __launch_bounds__(kThreads) k_moddown_combine(
+    const u64* __restrict__ u, const u64* __restrict__ lifted, long long nitems, const unsigned* __restrict__ galois,
+    int rot0, int rot_inc, const u64* __restrict__ c0, long long c0_stride, const u64* __restrict__ addend,
+    long long addend_stride, u64* __restrict__ out0, u64* __restrict__ out1, long long out_stride, int N, int logN, int L,
+    LimbTable lt) {
+    const long long LN = (long long)L * N, L1N = (long long)(L + 1) * N;
+    const long long total = nitems * 2 * LN;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const int t = (int)(idx % N);
+        const int i = (int)((idx / N) % L);
+        const int comp = (int)((idx / LN) % 2);
+        const long long item = idx / (2 * LN);
+        const unsigned k = galois[rot0 + (int)item * rot_inc];
+        const int s = (k == 1u) ? t : galois_src(t, k, logN);
+        const LimbConst& lc = lt.c[i];
+        u64 a = u[(item * 2 + comp) * L1N + (long long)i * N + s];
+        u64 b = lifted[((item * 2 + comp) * L + i) * N + s];
+        u64 v = csub(shoup_mul(submod(a, b, lc.q), lc.pinv, lc.pinv_s, lc.q), lc.q);
+        if (comp == 0 && c0) v = addmod(v, c0[item * c0_stride + (long long)i * N + s], lc.q);
+        if (addend) v = addmod(v, addend[item * addend_stride + (long long)comp * LN + (long long)i * N + t], lc.q);
+        u64* o = (comp == 0 ? out0 : out1) + item * out_stride + (long long)i * N + t;
+        *o = v;
+    }
+}
+
+// dst[poly][t] = src[poly][galois source of t]   (transform domain automorphism X -> X^k)
+__global__ void __launch_bounds__(kThreads) k_permute(const u64* __restrict__ src, u64* __restrict__ dst, long long npoly,
+                                                      unsigned k, int N, int logN) {
+    const long long total = npoly * N;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const long long poly = idx / N;
+        const int t = (int)(idx % N);
+        dst[idx] = src[poly * N + galois_src(t, k, logN)];
+    }
+}
+
+// ------------------------------------------------------------------------------------------ client-side helpers
+
+// out[l][x] = residue of the small signed coefficient v[x] modulo limb first + l
+__global__ void __launch_bounds__(kThreads) k_lift_i8(const int8_t* __restrict__ v, u64* __restrict__ out, int N,
+                                                      int nlimbs, LimbTable lt) {
+    const long long total = (long long)nlimbs * N;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const int l = (int)(idx / N), x = (int)(idx % N);
+        int s = v[x];
+        out[idx] = s >= 0 ? (u64)s : lt.c[l].q - (u64)(-s);
+    }
+}
+
+// out[p][x] = a[p][x] * b[(p % bperiod)][x] mod limb(p)
+__global__ void __launch_bounds__(kThreads) k_mul(const u64* __restrict__ a, const u64* __restrict__ b, int bperiod,
+                                                  u64* __restrict__ out, long long npoly, int N, LimbMap lm, LimbTable lt) {
+    const long long total = npoly * N;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const long long p = idx / N;
+        const int x = (int)(idx % N);
+        const LimbConst& lc = lt.c[lm.limb[p % lm.period]];
+        out[idx] = mulmod(a[idx], b[(p % bperiod) * N + x], lc);
+    }
+}
+
+// out[p][x] = a[p][x] + b[p][x] mod limb(p)
+__global__ void __launch_bounds__(kThreads) k_add(const u64* __restrict__ a, const u64* __restrict__ b,
+                                                  u64* __restrict__ out, long long npoly, int N, LimbMap lm, LimbTable lt) {
+    const long long total = npoly * N;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const long long p = idx / N;
+        out[idx] = addmod(a[idx], b[idx], lt.c[lm.limb[p % lm.period]].q);
+    }
+}
+
+// evaluation key finish, coefficient domain: b[j][i][x] = -as[j][i][x] + e[j][x] + (i == j ? (p mod q_j) * s'[x] : 0)
+__global__ void __launch_bounds__(kThreads) k_evk_finish(const u64* __restrict__ as, const int8_t* __restrict__ e,
+                                                         const int8_t* __restrict__ sprime, u64* __restrict__ b_out,
+                                                         int N, int L, LimbTable lt) {
+    const long long total = (long long)L * (L + 1) * N;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const int x = (int)(idx % N);
+        const int i = (int)((idx / N) % (L + 1));
+        const int j = (int)(idx / ((long long)N * (L + 1)));
+        const LimbConst& lc = lt.c[i];
+        u64 v = as[idx] ? lc.q - as[idx] : 0;
+        v = addmod(v, reduce_signed((i64)e[(long long)j * N + x], lc), lc.q);
+        if (i == j) {
+            int sp = sprime[x];
+            u64 f = lc.pmod;  // p mod q_j
+            if (sp > 0) v = addmod(v, f, lc.q);
+            else if (sp < 0) v = submod(v, f, lc.q);
+        }
+        b_out[idx] = v;
+    }
+}
+
+// symmetric encryption finish, coefficient domain: c0[l][x] = -as[l][x] + e[x] + m[l][x]
+__global__ void __launch_bounds__(kThreads) k_encrypt_finish(const u64* __restrict__ as, const int8_t* __restrict__ e,
+                                                             const u64* __restrict__ m, u64* __restrict__ c0, int N, int L,
+                                                             LimbTable lt) {
+    const long long total = (long long)L * N;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const int x = (int)(idx % N);
+        const int l = (int)(idx / N);
+        const LimbConst& lc = lt.c[l];
+        u64 v = as[idx] ? lc.q - as[idx] : 0;
+        v = addmod(v, reduce_signed((i64)e[x], lc), lc.q);
+        c0[idx] = addmod(v, m[idx], lc.q);
+    }
+}
+
+}  // namespace
+
+int check_launch(hann_ctx* c, const char* what) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        c->err = std::string(what) + ": " + cudaGetErrorString(e);
+        return HANN_ECUDA;
+    }
+    return HANN_OK;
+}
+
+int launch_mac(hann_ctx* c, const u64* baby, const u64* pt, int64_t n_blocks, u64* inner) {
+    if (n_blocks <= 0) return HANN_OK;
+    const long long LN = (long long)c->L * c->N;
+    const long long n_bg = n_blocks * c->G;
+    int gx = (int)((LN + kThreads - 1) / kThreads);
+    int gy = 1;
+    // enough CTAs to fill the machine even for a single small block
+    while ((long long)gx * gy < 148 * 8 && gy < n_bg) gy *= 2;
+    if (gy > n_bg) gy = (int)n_bg;
+    k_mac<<<dim3(gx, gy), kThreads, 0, c->stream>>>(baby, pt, inner, c->N, c->L, c->B, c->G, n_bg, c->lt);
+    c->stats.launches++;
+    return check_launch(c, "mac");
+}
+
+int launch_lift_digits(hann_ctx* c, const u64* src, int64_t src_stride, int64_t nitems, u64* digits) {
+    k_lift_digits<<<grid_for(nitems * c->L * c->N), kThreads, 0, c->stream>>>(src, src_stride, digits, c->N, c->L, nitems, c->lt);
+    c->stats.launches++;
+    return check_launch(c, "lift_digits");
+}
+
+int launch_ks_inner(hann_ctx* c, const u64* digits, int64_t digit_stride, int rot0, int rot_inc, int64_t nitems, u64* u) {
+    k_ks_inner<<<grid_for(nitems * (c->L + 1) * c->N), kThreads, 0, c->stream>>>(digits, digit_stride, c->keytab_dev, rot0, rot_inc, u,
+                                                                               c->N, c->L, nitems, c->lt);
+    c->stats.launches++;
+    return check_launch(c, "ks_inner");
+}
+
+int launch_moddown_lift(hann_ctx* c, const u64* u, int64_t npoly, u64* lifted) {
+    k_moddown_lift<<<grid_for(npoly * c->N), kThreads, 0, c->stream>>>(u, lifted, c->N, c->L, npoly, c->lt);
+    c->stats.launches++;
+    return check_launch(c, "moddown_lift");
+}
+
+int launch_moddown_combine(hann_ctx* c, const u64* u, const u64* lifted, int64_t nitems, int rot0, int rot_inc, const u64* c0,
+                           int64_t c0_stride, const u64* addend, int64_t addend_stride, u64* out0, u64* out1,
+                           int64_t out_stride) {
+    k_moddown_combine<<<grid_for(nitems * 2 * c->L * c->N), kThreads, 0, c->stream>>>(
+        u, lifted, nitems, c->galois_dev, rot0, rot_inc, c0, c0_stride, addend, addend_stride, out0, out1, out_stride, c->N,
+        c->logN, c->L, c->lt);
+    c->stats.launches++;
+    return check_launch(c, "moddown_combine");
+}
+
+int launch_permute(hann_ctx* c, const u64* src, u64* dst, int64_t npoly, unsigned k) {
+    k_permute<<<grid_for(npoly * c->N), kThreads, 0, c->stream>>>(src, dst, npoly, k, c->N, c->logN);
+    c->stats.launches++;
+    return check_launch(c, "permute");
+}
+
+int launch_lift_i8(hann_ctx* c, const int8_t* v, int nlimbs, u64* out) {
+    k_lift_i8<<<grid_for((int64_t)nlimbs * c->N), kThreads, 0, c->stream>>>(v, out, c->N, nlimbs, c->lt);
+    c->stats.launches++;
+    return check_launch(c, "lift_i8");
+}
+
+int launch_mul(hann_ctx* c, const u64* a, const u64* b, int bperiod, u64* out, int64_t npoly, const LimbMap& lm) {
+    k_mul<<<grid_for(npoly * c->N), kThreads, 0, c->stream>>>(a, b, bperiod, out, npoly, c->N, lm, c->lt);
+    c->stats.launches++;
+    return check_launch(c, "mul");
+}
+
+int launch_add(hann_ctx* c, const u64* a, const u64* b, u64* out, int64_t npoly, const LimbMap& lm) {
+    k_add<<<grid_for(npoly * c->N), kThreads, 0, c->stream>>>(a, b, out, npoly, c->N, lm, c->lt);
+    c->stats.launches++;
+    return check_launch(c, "add");
+}
+
+int launch_evk_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const int8_t* sprime, u64* b_out) {
+    k_evk_finish<<<grid_for((int64_t)c->L * (c->L + 1) * c->N), kThreads, 0, c->stream>>>(as_coeff, e, sprime, b_out, c->N, c->L, c->lt);
+    c->stats.launches++;
+    return check_launch(c, "evk_finish");
+}
+
+int launch_encrypt_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const u64* m, u64* c0_out) {
+    k_encrypt_finish<<<grid_for((int64_t)c->L * c->N), kThreads, 0, c->stream>>>(as_coeff, e, m, c0_out, c->N, c->L, c->lt);
+    c->stats.launches++;
+    return check_launch(c, "encrypt_finish");
+}

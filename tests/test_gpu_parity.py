@@ -1,0 +1,190 @@
+"""CUDA path vs CPU oracle, element by element, through the C ABI.  Ciphertext residues must be bit-identical in
+the canonical layout at the five conformance points (encoded plaintexts, baby ciphertexts, partial sums, score
+ciphertexts, key-switch outputs); decrypted scores must be within 2^-10 (toy scale 2^25) / 2^-18 (scale 2^40) of
+the float64 dot products."""
+import numpy as np
+import pytest
+
+from paper_2608_21131_b200 import synth
+from tests.helpers import Pair
+
+pytestmark = pytest.mark.gpu
+
+
+def torch_rows(p, rows):
+    import torch
+
+    return torch.from_numpy(np.ascontiguousarray(rows)).to(p.g.device)
+
+
+def run_level(p, rows, qv, check=True):
+    """score one level on both sides; returns decrypted GPU scores [n_rows]"""
+    ps, g, o, b = p.ps, p.g, p.o, p.b
+    ct_o, ct_g = p.query(qv)
+    assert np.array_equal(ct_o, ct_g)
+    ct_dev = g.import_(b.KIND_CT, ct_g, 1)
+    baby = g.query_prepare(ct_dev, p.ws)
+    baby_o = o.baby_set(ct_o, p.evk_o)
+    baby_g = g.export(b.KIND_CT, baby, ps.B)
+    assert np.array_equal(baby_g, baby_o)                                       # C2
+    n_rows = rows.shape[0]
+    nb = g.n_blocks(n_rows)
+    pt = g.encode_candidates(torch_rows(p, rows), p.ws)
+    inner = g.score_level(baby, pt, nb, p.ws)
+    score = g.rotate_sum(inner, nb, p.ws)
+    g.sync()
+    score_g = g.export(b.KIND_CT, score, nb)
+    if check:
+        pt_g = g.export(b.KIND_PT, pt, nb * ps.R).reshape(nb, ps.G, ps.B, ps.L, ps.N)
+        inner_g = g.export(b.KIND_CT, inner, nb * ps.G).reshape(nb, ps.G, 2, ps.L, ps.N)
+        Rr = np.zeros((n_rows, ps.R), dtype=np.float32)
+        Rr[:, : rows.shape[1]] = rows
+        for blk in range(nb):
+            sc_o, pt_o, in_o = o.score_block(Rr[blk * ps.n:(blk + 1) * ps.n], baby_o, p.evk_o[ps.B - 1], True, True)
+            assert np.array_equal(pt_g[blk], pt_o)                              # C1
+            assert np.array_equal(inner_g[blk], in_o)                           # C3
+            assert np.array_equal(score_g[blk], sc_o)                           # C4
+    got = g.decrypt_scores(p.km.s, score_g).reshape(-1)[:n_rows]
+    want = rows.astype(np.float64) @ qv.astype(np.float64)[: rows.shape[1]]
+    assert np.abs(got - want).max() < 2.0 ** ps.tol_log2
+    return got, score_g
+
+
+@pytest.mark.parametrize("logN", [4, 5, 8, 9, 10, 12])
+def test_import_export_roundtrip_and_transform(logN):
+    from paper_2608_21131_b200 import binding as b
+
+    ps = synth.small_params(logN, 4, 2, L=2)
+    g = b.Context(ps)
+    rng = np.random.default_rng(logN)
+    polys = np.stack([np.stack([rng.integers(0, q, size=ps.N, dtype=np.uint64) for q in ps.q]) for _ in range(3)])
+    dev = g.import_(b.KIND_POLY, polys, 3)
+    back = g.export(b.KIND_POLY, dev, 3).reshape(3, ps.L, ps.N)
+    assert np.array_equal(back, polys)
+    # the private layout is the negacyclic transform in bit-reversed order: position k holds a(psi^(2 brev(k)+1)),
+    # whatever psi the library picked; check the multiset-free consequence a(psi^...)=const for a constant poly
+    const = np.zeros((1, ps.L, ps.N), dtype=np.uint64)
+    const[0, :, 0] = 7
+    dev = g.import_(b.KIND_POLY, const, 1)
+    assert (dev.cpu().numpy().view(np.uint64)[: ps.L * ps.N] == 7).all()
+
+
+@pytest.mark.parametrize("logN,R,B,L,big", [(4, 4, 2, 2, False), (8, 8, 4, 2, False), (9, 16, 4, 3, True), (11, 64, 8, 2, False)])
+def test_client_half_matches_oracle(logN, R, B, L, big):
+    ps = synth.small_params(logN, R, B, L=L, big=big)
+    p = Pair(ps, key_seed=5)
+    assert np.array_equal(p.evk_g, p.evk_o)                 # keygen from the same samples
+    qv = synth.toy_query(2, dim=R)
+    ct_o, ct_g = p.query(qv)
+    assert np.array_equal(ct_o, ct_g)                       # canonical encode + symmetric encryption
+    # decrypt of the fresh query gives the tiled query back
+    z = p.g.decrypt_scores(p.km.s, ct_g, log_scale_out=ps.log_scale)[0]
+    assert np.abs(z - np.tile(qv.astype(np.float64), ps.n // R)).max() < 1e-3
+    zo = p.o.decrypt_slots(p.km.s, ct_o, ps.log_scale).real
+    assert np.abs(z - zo).max() < 1e-9
+
+
+@pytest.mark.parametrize("logN,L,big,rot", [(4, 2, False, 1), (8, 2, False, 3), (10, 2, False, 2), (10, 4, True, 4), (12, 2, False, 8)])
+def test_keyswitch_matches_oracle(logN, L, big, rot):
+    ps = synth.small_params(logN, 8, 8 if logN > 4 else 4, L=L, big=big)
+    p = Pair(ps, key_seed=7)
+    rng = np.random.default_rng(rot)
+    d = np.stack([rng.integers(0, q, size=ps.N, dtype=np.uint64) for q in ps.q])
+    ks0_o, ks1_o = p.o.keyswitch(d, p.evk_o[rot - 1])
+    dev = p.g.import_(p.b.KIND_POLY, d[None], 1)
+    ks0, ks1 = p.g.keyswitch(rot, dev, p.ws)
+    assert np.array_equal(p.g.export(p.b.KIND_POLY, ks0, 1)[0, 0], ks0_o)     # C5
+    assert np.array_equal(p.g.export(p.b.KIND_POLY, ks1, 1)[0, 0], ks1_o)
+
+
+@pytest.mark.parametrize(
+    "logN,R,B,L,big,n_rows,dim",
+    [
+        (4, 4, 2, 2, False, 8, 4),        # one full block, tiny ring
+        (5, 4, 4, 2, False, 13, 3),       # G = 1 (no rotate-and-sum), ragged, dim < R
+        (6, 8, 1, 2, False, 40, 8),       # B = 1 (no baby rotations), two blocks, ragged
+        (8, 16, 4, 2, False, 300, 16),    # single-pass transform, three blocks
+        (9, 32, 8, 3, True, 256, 24),     # two-pass transform, 50-bit primes, zero-padded dimension
+        (10, 64, 8, 2, False, 1500, 64),  # three blocks, last ragged
+    ],
+)
+def test_level_bit_exact_small(logN, R, B, L, big, n_rows, dim):
+    ps = synth.small_params(logN, R, B, L=L, big=big)
+    if big:
+        ps = ps.with_(log_scale=40)
+    p = Pair(ps, key_seed=logN)
+    rows = synth.toy_corpus(logN, rows=n_rows, dim=dim)
+    qv = np.zeros(R, dtype=np.float32)
+    qv[:dim] = synth.toy_query(logN + 1, dim=dim)
+    run_level(p, rows, qv)
+
+
+def test_toy_configuration_full():
+    """Toy configuration: 4,096 unit-norm rows of dimension 64, N = 2^12, scale 2^25 -> two blocks; every conformance
+    point bit-exact, every score within 2^-10; repeated with three seed triples."""
+    ps = synth.TOY
+    for cs, qs, ks in ((1, 2, 3), (11, 12, 13), (21, 22, 23)):
+        p = Pair(ps, key_seed=ks)
+        got, _ = run_level(p, synth.toy_corpus(cs), synth.toy_query(qs), check=(cs == 1))
+        assert got.shape == (4096,)
+
+
+def test_toy_other_baby_step_counts():
+    for B in (4, 32):
+        ps = synth.TOY.with_(B=B)
+        p = Pair(ps, key_seed=3)
+        run_level(p, synth.toy_corpus(1, rows=2048 + 77), synth.toy_query(2))
+
+
+def test_host_buffer_level_matches_device_path():
+    ps = synth.TOY
+    p = Pair(ps, key_seed=3)
+    rows = synth.toy_corpus(1, rows=3000)
+    qv = synth.toy_query(2)
+    _, score_dev = run_level(p, rows, qv, check=False)
+    ct_o, ct_g = p.query(qv)
+    ws = p.g.alloc(p.g.level_host_bytes(rows.shape[0]))
+    out = p.g.score_level_host(ct_g, rows, ws)
+    assert np.array_equal(out, score_dev)
+
+
+def test_full_ring_one_block():
+    """N = 2^16, 4 x ~50-bit primes + ~60-bit special prime, scale 2^40, R = 128, B = 32: one ragged block checked at
+    every conformance point, scores within 2^-18."""
+    ps = synth.FULL16
+    p = Pair(ps, key_seed=1)
+    rows = synth.project_rows(synth.toy_corpus(5, rows=ps.n - 1234, dim=96).astype(np.float64), None, 128)
+    qv = np.zeros(128, dtype=np.float32)
+    qv[:96] = synth.toy_query(6, dim=96)
+    got, _ = run_level(p, rows, qv)
+    want = rows.astype(np.float64) @ qv.astype(np.float64)
+    assert np.abs(got - want).max() < 2.0 ** -22  # observed error level, regression alarm
+
+
+def test_error_codes():
+    from paper_2608_21131_b200 import binding as b
+    import torch
+
+    ps = synth.small_params(8, 8, 4, L=2)
+    with pytest.raises(b.HannError):
+        b.Context(ps.with_(q=(ps.q[0], ps.q[0] + 2)))  # not prime
+    with pytest.raises(b.HannError):
+        b.Context(ps.with_(B=3))
+    g = b.Context(ps)
+    ws = g.workspace(1)
+    ct = g.alloc(g.sizeof(b.SIZE_CT))
+    with pytest.raises(b.HannError) as ei:
+        g.query_prepare(ct, ws)
+    assert ei.value.code == b.ENOKEY
+    km = synth.key_material(ps, 1)
+    g.load_keys(g.keygen_from_samples(km.s, km.rots, km.evk_a, km.evk_e), km.rots)
+    with pytest.raises(b.HannError) as ei:
+        g.query_prepare(ct, ws[:16])
+    assert ei.value.code == b.EWORKSPACE
+    rows = torch.zeros((4, 9), dtype=torch.float32, device=g.device)
+    with pytest.raises(b.HannError) as ei:
+        g.encode_candidates(rows, ws)
+    assert ei.value.code == b.ESHAPE
+    # the context stays usable after errors
+    g.query_prepare(ct, ws)
+    g.sync()

@@ -1,0 +1,384 @@
+#!/usr/bin/env python
+"""Benchmark of the encrypted scoring hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 0..4]
+
+One "step" is one pass of the whole server-side path for one encrypted query over one routing level:
+query_prepare (hoisted baby rotations) + encode_candidates + score_level (ct x pt multiply-accumulate) +
+rotate_sum (Horner with hybrid key switching).  The default workload is the face-corpus-like single level
+(222,049 rows, 512 -> 128 dims, N = 2^16, 4 x ~50-bit + ~60-bit primes, scale 2^40), all inputs synthetic.
+Prints ONE JSON line on rank 0.  With N > 1 every rank runs an independent replica of the workload on its own
+GPU (the path has no exchange step); the value is the sum over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "encrypted candidates scored/sec"
+UNIT = "candidates/s"
+SM_COUNT = 148
+IMAD_LANES_PER_SM = 64  # 32-bit integer multiply-add lanes per SM per clock
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), float(d.get("sm_max_mhz", 1965.0)), "measured"
+    return 6650.0, 1965.0, "fallback"
+
+
+class ClockSampler:
+    """samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs"""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for ln in self.proc.stdout:
+            self.lines.append(ln)
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); smax.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def build_workload(config, rows_override=None):
+    from paper_2608_21131_b200 import workloads as wl, synth
+
+    if config == 0:
+        ps, rows, q = wl.toy()
+        return ps, rows, q, "toy: 4,096 rows, dim 64, N=2^12, scale 2^25"
+    if config == 1:
+        n = rows_override or 222_049
+        ps, lvl, q, _ = wl.face_level(rows=n)
+        return ps, lvl.rows, q, "face-like flat level: %d rows, dim 512->128, N=2^16, 4x50b+60b primes, scale 2^40" % n
+    if config == 4:
+        base = rows_override or (1 << 18)
+        ps, lvl = wl.sweep_level(base)
+        q = synth.toy_query(wl.query_seed(0), dim=ps.R)
+        return ps, lvl.rows, q, "sweep: %d wanted rows inflated x4 to %d scored rows, dim 128, N=2^16" % (base, lvl.rows.shape[0])
+    raise SystemExit("bench.py times configs 0, 1 and 4; the hierarchy configs are exercised by the tests")
+
+
+def algorithmic_work(ctx, n_blocks, n_rows):
+    """algorithmic bytes (HBM-bound kernels) or 32-bit multiplies (ALU-bound kernels) of ONE step, per kernel class.
+    A 64-bit Shoup butterfly costs 10 32x32-bit multiplies: 4 for hi64(a*w'), 3 for lo64(a*w), 3 for lo64(t*q)."""
+    L, N, B, G, R = ctx.L, ctx.N, ctx.B, ctx.G, ctx.R
+    logN = ctx.logN
+    b = min(logN, 8)
+    a = logN - b
+    W = 8 * N
+    fwd_polys = n_blocks * R * L + (L * (L + 1) + (B - 1) * 2 * L) + (G - 1) * n_blocks * (L * (L + 1) + 2 * L)
+    inv_polys = (L + (B - 1) * 2) + (G - 1) * n_blocks * (L + 2)
+    return {
+        "mac": ("hbm", n_blocks * R * L * W + B * 2 * L * W + n_blocks * G * 2 * L * W),
+        "ks_inner": ("hbm", (B - 1) * (L * 2 * (L + 1) * W + 2 * (L + 1) * W) + L * (L + 1) * W
+                     + (G - 1) * (L * 2 * (L + 1) * W + n_blocks * (L * (L + 1) * W + 2 * (L + 1) * W))),
+        "ntt_fwd_a": ("alu", fwd_polys * (N // 2) * a * 10),
+        "ntt_fwd_b": ("alu", fwd_polys * (N // 2) * b * 10),
+        "ntt_inv_a": ("alu", inv_polys * (N // 2) * a * 10),
+        "ntt_inv_b": ("alu", inv_polys * (N // 2) * b * 10),
+        "fft_a": ("hbm", n_blocks * R * (ctx.n * 16) + n_rows * R * 4),
+        "fft_b": ("hbm", n_blocks * R * (ctx.n * 16 + L * W)),
+    }
+
+
+def run_ours(args):
+    import torch
+    from paper_2608_21131_b200 import binding, synth, workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the scoring path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    ps, rows_np, qR, wname = build_workload(args.config, args.rows)
+    n_rows = rows_np.shape[0]
+    ctx = binding.Context(ps, device=local)
+    km = synth.key_material(ps, wl.KEY_SEED)
+    evk = ctx.keygen_from_samples(km.s, km.rots, km.evk_a, km.evk_e)
+    ctx.load_keys(evk, km.rots)
+    ct_host = ctx.encrypt_query(km.s, qR, km.ct_a, km.ct_e)
+    ct_dev = ctx.import_(binding.KIND_CT, ct_host, 1)
+    rows_dev = torch.from_numpy(rows_np).to(ctx.device)
+    nb = ctx.n_blocks(n_rows)
+    ws = ctx.workspace(nb)
+    baby = ctx.alloc(ctx.sizeof(binding.SIZE_BABY))
+    pt = ctx.alloc(nb * ctx.sizeof(binding.SIZE_PT_BLOCK))
+    inner = ctx.alloc(nb * ctx.sizeof(binding.SIZE_INNER))
+    score = ctx.alloc(nb * ctx.sizeof(binding.SIZE_CT))
+
+    def step():
+        ctx.query_prepare(ct_dev, ws, baby)
+        ctx.encode_candidates(rows_dev, ws, pt)
+        ctx.score_level(baby, pt, nb, ws, inner)
+        ctx.rotate_sum(inner, nb, ws, score)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    if args.lean:
+        # profiling aid (ncu launch lists and captures): W warm-up steps, K steps, nothing else, no JSON line
+        for _ in range(args.warmup + args.steps):
+            step()
+        torch.cuda.synchronize()
+        print("lean run: %d steps, %d kernel launches" % (args.warmup + args.steps, ctx.get_stats()["launches"]))
+        return 0
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    l0 = ctx.get_stats()["launches"]
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = e0.elapsed_time(e1)
+    launches = ctx.get_stats()["launches"] - l0
+    t = torch.tensor([ms_total], dtype=torch.float64, device=ctx.device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+    value = world * n_rows / (ms_step * 1e-3)
+
+    # correctness of what was timed: decrypted scores against float64 dot products
+    score_host = ctx.export(binding.KIND_CT, score, nb)
+    got = ctx.decrypt_scores(km.s, score_host).reshape(-1)[:n_rows]
+    want = rows_np.astype(np.float64) @ qR.astype(np.float64)
+    max_err = float(np.abs(got - want).max())
+    check_ok = bool(max_err < 2.0 ** ps.tol_log2)
+
+    # per-stage device time (library event timers), median of the timed steps
+    ctx.set_timing(True)
+    stage = {k: [] for k in ("ms_query_prepare", "ms_encode", "ms_score_level", "ms_rotate_sum")}
+    for _ in range(args.steps):
+        step()
+        st = ctx.get_stats()
+        for k in stage:
+            stage[k].append(st[k])
+    ctx.set_timing(False)
+    stage_ms = {k[3:]: float(np.median(v)) for k, v in stage.items()}
+
+    # per-kernel device time, live, with an event pair around every launch of the same steps
+    ctx.kernel_profile(True)
+    for _ in range(args.steps):
+        step()
+    kt = ctx.kernel_times()
+    ctx.kernel_profile(False)
+    total_k = sum(v[0] for v in kt.values()) or 1.0
+    kernels = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps, "share": v[0] / total_k}
+               for k, v in kt.items() if v[1]}
+    hbm_peak, sm_max_mhz, peak_src = read_peaks()
+    work = algorithmic_work(ctx, nb, n_rows)
+    dom = max((k for k in kernels if k in work), key=lambda k: kernels[k]["ms_per_step"])
+    bound, amount = work[dom]
+    dom_s = kernels[dom]["ms_per_step"] * 1e-3
+    if bound == "hbm":
+        achieved, peak, runit = amount / dom_s / 1e9, hbm_peak, "GB/s"
+    else:
+        achieved, peak, runit = amount / dom_s / 1e12, SM_COUNT * IMAD_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12, "Tmul32/s"
+    roofline = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,
+                "peak_source": peak_src + (" copy bandwidth" if bound == "hbm" else
+                                           ": %d SMs x %d int32 multiply-add lanes x %.0f MHz" % (SM_COUNT, IMAD_LANES_PER_SM, sm_max_mhz)),
+                "traffic": None, "launches_per_step": kernels[dom]["launches_per_step"],
+                "avg_launch_ms": kernels[dom]["ms_per_step"] / max(kernels[dom]["launches_per_step"], 1)}
+    hbm_kernels = {}
+    for k in ("mac", "ks_inner"):
+        if k in kernels:
+            hbm_kernels[k] = {"GB/s": work[k][1] / (kernels[k]["ms_per_step"] * 1e-3) / 1e9,
+                              "frac_of_measured_copy": work[k][1] / (kernels[k]["ms_per_step"] * 1e-3) / 1e9 / hbm_peak}
+
+    # end to end through the host-buffer entry point: pinned host inputs, copies inside the timed region
+    rows_pin = torch.from_numpy(rows_np).pin_memory()
+    ct_pin = torch.from_numpy(ct_host.view(np.int64)).pin_memory()
+    out_pin = torch.empty((nb, 2, ctx.L, ctx.N), dtype=torch.int64).pin_memory()
+    del pt, inner, score, baby, ws
+    torch.cuda.empty_cache()
+    ws_host = ctx.alloc(ctx.level_host_bytes(n_rows))
+
+    def e2e_step():
+        ctx.lib.hann_score_level_host(ctx.h, ct_pin.data_ptr(), rows_pin.data_ptr(), n_rows, rows_np.shape[1], out_pin.data_ptr(),
+                                      ws_host.data_ptr(), ws_host.numel() * 8)
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        e2e_step()
+    torch.cuda.synchronize()
+    t_e2e = torch.tensor([time.perf_counter() - t0], dtype=torch.float64, device=ctx.device)
+    if dist is not None:
+        dist.all_reduce(t_e2e, op=dist.ReduceOp.MAX)
+    e2e_value = world * n_rows * args.steps / float(t_e2e.item())
+    e2e_same = bool(np.array_equal(out_pin.numpy().view(np.uint64), score_host))
+    e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(rows_np.nbytes + ct_host.nbytes),
+           "d2h_bytes_per_step": int(out_pin.numel() * 8), "matches_device_path": e2e_same}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cpu = cpu_baseline(ps, rows_np, qR, km, n_rows)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64",
+            "data": "synthetic",
+            "config": {"workload": wname, "rows": n_rows, "blocks": nb, "R": ps.R, "B": ps.B, "G": ps.G, "logN": ps.logN, "L": ps.L,
+                       "l2": "working set per step (%.1f GB of encoded plaintexts) exceeds L2; no flush" %
+                             (nb * ctx.sizeof(binding.SIZE_PT_BLOCK) / 1e9),
+                       "replicas": "each rank scores the whole level on its own GPU" if world > 1 else "single GPU"},
+            "ms_per_query_level": ms_step, "stage_ms": stage_ms,
+            "warm_value": world * n_rows / ((ms_step - stage_ms["encode"]) * 1e-3) if ms_step > stage_ms["encode"] else None,
+            "kernels": kernels, "hbm_kernels": hbm_kernels, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
+            "gpu_launches": int(launches), "clocks": clocks,
+            "check": {"max_abs_score_error": max_err, "tolerance": 2.0 ** ps.tol_log2, "ok": check_ok},
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0 if check_ok else 1
+
+
+def oracle_setup(ps, qR, km):
+    from oracle.oracle import Oracle
+
+    o = Oracle(ps.logN, ps.q, ps.p, ps.log_scale, ps.R, ps.B)
+    ct = o.encrypt_query(km.s, qR, km.ct_a, km.ct_e)
+    evk = np.stack([o.evk_gen(km.s, r, km.evk_a[i], km.evk_e[i]) for i, r in enumerate(km.rots)])
+    return o, ct, evk
+
+
+def cpu_baseline(ps, rows_np, qR, km, n_rows):
+    """the oracle as it stands on the host cores: one query_prepare + one block, scaled to the level by block count"""
+    o, ct, evk = oracle_setup(ps, qR, km)
+    t0 = time.perf_counter()
+    baby = o.baby_set(ct, evk)
+    t_prep = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    o.score_block(rows_np[: ps.n], baby, evk[ps.B - 1])
+    t_blk = time.perf_counter() - t0
+    nb = (n_rows + ps.n - 1) // ps.n
+    return {"value": n_rows / (t_prep + nb * t_blk), "unit": UNIT, "cores": o.num_threads(), "kind": "oracle",
+            "sample": "query_prepare once (%.1f s) + block 0 of %d (%d rows, %.1f s) timed; level time = prepare + blocks x "
+                      "block time (per-block work is constant)" % (t_prep, nb, min(ps.n, n_rows), t_blk)}
+
+
+def run_reference(args):
+    """reference arm: the CPU oracle, unmodified, on the host cores; a step is query_prepare + one block"""
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank != 0:
+        return 0
+    from paper_2608_21131_b200 import synth, workloads as wl
+
+    ps, rows_np, qR, wname = build_workload(args.config, args.rows)
+    n_rows = rows_np.shape[0]
+    km = synth.key_material(ps, wl.KEY_SEED)
+    o, ct, evk = oracle_setup(ps, qR, km)
+    sample_rows = min(ps.n, n_rows)
+
+    def step():
+        baby = o.baby_set(ct, evk)
+        o.score_block(rows_np[:sample_rows], baby, evk[ps.B - 1])
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    value = sample_rows / dt
+    sample = "each step = query_prepare + encode/MAC/rotate-sum of block 0 (%d of %d rows)" % (sample_rows, n_rows)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u64", "data": "synthetic", "config": {"workload": wname, "rows": n_rows, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": o.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1)
+    ap.add_argument("--rows", type=int, default=None, help="override the row count (debugging, ncu captures)")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--lean", action="store_true", help="only run warm-up + steps (for ncu); prints no JSON line")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 2 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        return run_reference(args)
+    args.steps = 10 if args.steps is None else args.steps
+    args.warmup = 3 if args.warmup is None else args.warmup
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

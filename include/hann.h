@@ -111,6 +111,15 @@ const char *hann_last_error(const hann_ctx *ctx);
 int hann_set_timing(hann_ctx *ctx, int enable);
 int hann_get_stats(hann_ctx *ctx, hann_stats *out);
 
+/* Per-launch profile: while enabled every kernel launch of the context is bracketed by a CUDA event pair (this
+ * serialises nothing but adds two event records per launch).  hann_kernel_times synchronises, writes the summed
+ * device milliseconds and launch counts per kernel class (arrays of hann_kernel_classes() entries, class names from
+ * hann_kernel_name) accumulated since the previous call, and clears them. */
+int hann_kernel_classes(void);
+const char *hann_kernel_name(int cls);
+int hann_kernel_profile(hann_ctx *ctx, int enable);
+int hann_kernel_times(hann_ctx *ctx, double *ms, uint64_t *launches);
+
 /* ---- client side (host memory in and out; Sec. 2, The round trip, client steps) -------------------------- */
 
 /* Evaluation keys for the left slot rotations rot[0..n_rot) from caller-drawn randomness (hybrid key switching,

@@ -64,6 +64,10 @@ def load_library():
         "hann_last_error": (C.c_char_p, [vp]),
         "hann_set_timing": (C.c_int, [vp, C.c_int]),
         "hann_get_stats": (C.c_int, [vp, C.POINTER(Stats)]),
+        "hann_kernel_classes": (C.c_int, []),
+        "hann_kernel_name": (C.c_char_p, [C.c_int]),
+        "hann_kernel_profile": (C.c_int, [vp, C.c_int]),
+        "hann_kernel_times": (C.c_int, [vp, vp, vp]),
         "hann_keygen_from_samples": (C.c_int, [vp, vp, C.c_int, vp, vp, vp, vp]),
         "hann_encrypt_query": (C.c_int, [vp, vp, vp, C.c_int, vp, vp, vp]),
         "hann_decrypt_scores": (C.c_int, [vp, vp, vp, i64, C.c_int, vp, vp]),
@@ -167,6 +171,17 @@ class Context:
         st = Stats()
         self._ck(self.lib.hann_get_stats(self.h, C.byref(st)))
         return {k: getattr(st, k) for k, _ in Stats._fields_}
+
+    def kernel_profile(self, on):
+        self._ck(self.lib.hann_kernel_profile(self.h, 1 if on else 0))
+
+    def kernel_times(self):
+        """{kernel class: (summed device ms, launches)} since the previous call"""
+        k = self.lib.hann_kernel_classes()
+        ms = np.zeros(k, dtype=np.float64)
+        cnt = np.zeros(k, dtype=np.uint64)
+        self._ck(self.lib.hann_kernel_times(self.h, _ptr(ms), _ptr(cnt)))
+        return {self.lib.hann_kernel_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(k)}
 
     # ---- client side
     def keygen_from_samples(self, s, rots, a, e):

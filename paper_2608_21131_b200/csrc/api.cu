@@ -277,6 +277,10 @@ extern "C" void hann_ctx_destroy(hann_ctx* c) {
     cudaFree(c->tw_fwd); cudaFree(c->tw_fwd_s); cudaFree(c->tw_inv); cudaFree(c->tw_inv_s);
     cudaFree(c->fft_T); cudaFree(c->fft_U); cudaFree(c->jinv); cudaFree(c->galois_dev); cudaFree(c->keytab_dev);
     if (c->scratch) cudaFree(c->scratch);
+    for (auto& r : c->krec) {
+        if (r.a) cudaEventDestroy(r.a);
+        if (r.b) cudaEventDestroy(r.b);
+    }
     for (int k = 0; k < HANN_NKINDS; k++) {
         if (c->ev[k][0]) cudaEventDestroy(c->ev[k][0]);
         if (c->ev[k][1]) cudaEventDestroy(c->ev[k][1]);
@@ -336,6 +340,36 @@ extern "C" int hann_get_stats(hann_ctx* c, hann_stats* out) {
             c->ev_pending[k] = 0;
         }
     *out = c->stats;
+    return HANN_OK;
+}
+
+static const char* kKernelNames[KC_COUNT] = {"ntt_fwd_a", "ntt_fwd_b", "ntt_inv_b", "ntt_inv_a", "fft_a", "fft_b", "mac",
+                                             "lift_digits", "ks_inner", "moddown_lift", "moddown_combine", "permute", "other"};
+
+extern "C" int hann_kernel_classes(void) { return KC_COUNT; }
+extern "C" const char* hann_kernel_name(int cls) { return cls >= 0 && cls < KC_COUNT ? kKernelNames[cls] : ""; }
+
+extern "C" int hann_kernel_profile(hann_ctx* c, int enable) {
+    if (!c) return HANN_EINVAL;
+    DeviceGuard dg(c->device);
+    CK(cudaStreamSynchronize(c->stream));
+    c->kprof = enable ? 1 : 0;
+    c->krec_used = 0;
+    return HANN_OK;
+}
+
+extern "C" int hann_kernel_times(hann_ctx* c, double* ms, uint64_t* launches) {
+    if (!c || !ms || !launches) return HANN_EINVAL;
+    DeviceGuard dg(c->device);
+    CK(cudaStreamSynchronize(c->stream));
+    for (int k = 0; k < KC_COUNT; k++) { ms[k] = 0; launches[k] = 0; }
+    for (size_t i = 0; i < c->krec_used; i++) {
+        float t = 0;
+        CK(cudaEventElapsedTime(&t, c->krec[i].a, c->krec[i].b));
+        ms[c->krec[i].cls] += t;
+        launches[c->krec[i].cls]++;
+    }
+    c->krec_used = 0;
     return HANN_OK;
 }
 

@@ -128,10 +128,14 @@ int run_encode(hann_ctx* c, EncArgs& A, int P) {
     A.L = c->L;
     A.R = c->R;
     A.B = c->B;
-    k_fft_a<<<dim3(chunks / A.K1, P), kThreads, (size_t)A.K1 * S1 * sizeof(double2), c->stream>>>(A);
-    c->stats.launches++;
-    k_fft_b<<<dim3(S1 / A.C1, P), kThreads, (size_t)(n >> A.b1) * A.C1 * sizeof(double2), c->stream>>>(A, c->lt);
-    c->stats.launches++;
+    {
+        KProf kp(c, KC_FFT_A);
+        k_fft_a<<<dim3(chunks / A.K1, P), kThreads, (size_t)A.K1 * S1 * sizeof(double2), c->stream>>>(A);
+    }
+    {
+        KProf kp(c, KC_FFT_B);
+        k_fft_b<<<dim3(S1 / A.C1, P), kThreads, (size_t)(n >> A.b1) * A.C1 * sizeof(double2), c->stream>>>(A, c->lt);
+    }
     return check_launch(c, "encode");
 }
 

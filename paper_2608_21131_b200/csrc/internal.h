@@ -10,6 +10,12 @@
 
 #define HANN_NKINDS 5  // timed call kinds: query_prepare, encode, score_level, rotate_sum, keyswitch
 
+// kernel classes of the per-launch profile (hann_kernel_profile / hann_kernel_times)
+enum {
+    KC_NTT_FWD_A = 0, KC_NTT_FWD_B, KC_NTT_INV_B, KC_NTT_INV_A, KC_FFT_A, KC_FFT_B, KC_MAC, KC_LIFT_DIGITS, KC_KS_INNER,
+    KC_MODDOWN_LIFT, KC_MODDOWN_COMBINE, KC_PERMUTE, KC_OTHER, KC_COUNT
+};
+
 struct hann_ctx {
     hann_params prm;
     int logN = 0, N = 0, n = 0, L = 0, R = 0, B = 0, G = 0;
@@ -40,7 +46,34 @@ struct hann_ctx {
     int timing = 0;
     cudaEvent_t ev[HANN_NKINDS][2] = {};
     int ev_pending[HANN_NKINDS] = {};
+    // per-launch profile: one event pair per launch while enabled
+    int kprof = 0;
+    struct KRec { int cls; cudaEvent_t a, b; };
+    std::vector<KRec> krec;
+    size_t krec_used = 0;
     std::string err;
+};
+
+// brackets one kernel launch with events when the per-launch profile is on
+struct KProf {
+    hann_ctx* c;
+    cudaEvent_t b = nullptr;
+    KProf(hann_ctx* c_, int cls) : c(c_) {
+        c->stats.launches++;
+        if (!c->kprof) return;
+        if (c->krec_used == c->krec.size()) {
+            hann_ctx::KRec r{cls, nullptr, nullptr};
+            if (cudaEventCreate(&r.a) != cudaSuccess || cudaEventCreate(&r.b) != cudaSuccess) return;
+            c->krec.push_back(r);
+        }
+        hann_ctx::KRec& r = c->krec[c->krec_used++];
+        r.cls = cls;
+        cudaEventRecord(r.a, c->stream);
+        b = r.b;
+    }
+    ~KProf() {
+        if (b) cudaEventRecord(b, c->stream);
+    }
 };
 
 // ---- host mathematics (hostmath.cpp)

@@ -242,72 +242,94 @@ int launch_mac(hann_ctx* c, const u64* baby, const u64* pt, int64_t n_blocks, u6
     // enough CTAs to fill the machine even for a single small block
     while ((long long)gx * gy < 148 * 8 && gy < n_bg) gy *= 2;
     if (gy > n_bg) gy = (int)n_bg;
-    k_mac<<<dim3(gx, gy), kThreads, 0, c->stream>>>(baby, pt, inner, c->N, c->L, c->B, c->G, n_bg, c->lt);
-    c->stats.launches++;
+    {
+        KProf kp(c, KC_MAC);
+        k_mac<<<dim3(gx, gy), kThreads, 0, c->stream>>>(baby, pt, inner, c->N, c->L, c->B, c->G, n_bg, c->lt);
+    }
     return check_launch(c, "mac");
 }
 
 int launch_lift_digits(hann_ctx* c, const u64* src, int64_t src_stride, int64_t nitems, u64* digits) {
-    k_lift_digits<<<grid_for(nitems * c->L * c->N), kThreads, 0, c->stream>>>(src, src_stride, digits, c->N, c->L, nitems, c->lt);
-    c->stats.launches++;
+    {
+        KProf kp(c, KC_LIFT_DIGITS);
+        k_lift_digits<<<grid_for(nitems * c->L * c->N), kThreads, 0, c->stream>>>(src, src_stride, digits, c->N, c->L, nitems, c->lt);
+    }
     return check_launch(c, "lift_digits");
 }
 
 int launch_ks_inner(hann_ctx* c, const u64* digits, int64_t digit_stride, int rot0, int rot_inc, int64_t nitems, u64* u) {
-    k_ks_inner<<<grid_for(nitems * (c->L + 1) * c->N), kThreads, 0, c->stream>>>(digits, digit_stride, c->keytab_dev, rot0, rot_inc, u,
-                                                                               c->N, c->L, nitems, c->lt);
-    c->stats.launches++;
+    {
+        KProf kp(c, KC_KS_INNER);
+        k_ks_inner<<<grid_for(nitems * (c->L + 1) * c->N), kThreads, 0, c->stream>>>(digits, digit_stride, c->keytab_dev, rot0, rot_inc, u,
+                                                                                   c->N, c->L, nitems, c->lt);
+    }
     return check_launch(c, "ks_inner");
 }
 
 int launch_moddown_lift(hann_ctx* c, const u64* u, int64_t npoly, u64* lifted) {
-    k_moddown_lift<<<grid_for(npoly * c->N), kThreads, 0, c->stream>>>(u, lifted, c->N, c->L, npoly, c->lt);
-    c->stats.launches++;
+    {
+        KProf kp(c, KC_MODDOWN_LIFT);
+        k_moddown_lift<<<grid_for(npoly * c->N), kThreads, 0, c->stream>>>(u, lifted, c->N, c->L, npoly, c->lt);
+    }
     return check_launch(c, "moddown_lift");
 }
 
 int launch_moddown_combine(hann_ctx* c, const u64* u, const u64* lifted, int64_t nitems, int rot0, int rot_inc, const u64* c0,
                            int64_t c0_stride, const u64* addend, int64_t addend_stride, u64* out0, u64* out1,
                            int64_t out_stride) {
-    k_moddown_combine<<<grid_for(nitems * 2 * c->L * c->N), kThreads, 0, c->stream>>>(
-        u, lifted, nitems, c->galois_dev, rot0, rot_inc, c0, c0_stride, addend, addend_stride, out0, out1, out_stride, c->N,
-        c->logN, c->L, c->lt);
-    c->stats.launches++;
+    {
+        KProf kp(c, KC_MODDOWN_COMBINE);
+        k_moddown_combine<<<grid_for(nitems * 2 * c->L * c->N), kThreads, 0, c->stream>>>(
+            u, lifted, nitems, c->galois_dev, rot0, rot_inc, c0, c0_stride, addend, addend_stride, out0, out1, out_stride, c->N,
+            c->logN, c->L, c->lt);
+    }
     return check_launch(c, "moddown_combine");
 }
 
 int launch_permute(hann_ctx* c, const u64* src, u64* dst, int64_t npoly, unsigned k) {
-    k_permute<<<grid_for(npoly * c->N), kThreads, 0, c->stream>>>(src, dst, npoly, k, c->N, c->logN);
-    c->stats.launches++;
+    {
+        KProf kp(c, KC_PERMUTE);
+        k_permute<<<grid_for(npoly * c->N), kThreads, 0, c->stream>>>(src, dst, npoly, k, c->N, c->logN);
+    }
     return check_launch(c, "permute");
 }
 
 int launch_lift_i8(hann_ctx* c, const int8_t* v, int nlimbs, u64* out) {
-    k_lift_i8<<<grid_for((int64_t)nlimbs * c->N), kThreads, 0, c->stream>>>(v, out, c->N, nlimbs, c->lt);
-    c->stats.launches++;
+    {
+        KProf kp(c, KC_OTHER);
+        k_lift_i8<<<grid_for((int64_t)nlimbs * c->N), kThreads, 0, c->stream>>>(v, out, c->N, nlimbs, c->lt);
+    }
     return check_launch(c, "lift_i8");
 }
 
 int launch_mul(hann_ctx* c, const u64* a, const u64* b, int bperiod, u64* out, int64_t npoly, const LimbMap& lm) {
-    k_mul<<<grid_for(npoly * c->N), kThreads, 0, c->stream>>>(a, b, bperiod, out, npoly, c->N, lm, c->lt);
-    c->stats.launches++;
+    {
+        KProf kp(c, KC_OTHER);
+        k_mul<<<grid_for(npoly * c->N), kThreads, 0, c->stream>>>(a, b, bperiod, out, npoly, c->N, lm, c->lt);
+    }
     return check_launch(c, "mul");
 }
 
 int launch_add(hann_ctx* c, const u64* a, const u64* b, u64* out, int64_t npoly, const LimbMap& lm) {
-    k_add<<<grid_for(npoly * c->N), kThreads, 0, c->stream>>>(a, b, out, npoly, c->N, lm, c->lt);
-    c->stats.launches++;
+    {
+        KProf kp(c, KC_OTHER);
+        k_add<<<grid_for(npoly * c->N), kThreads, 0, c->stream>>>(a, b, out, npoly, c->N, lm, c->lt);
+    }
     return check_launch(c, "add");
 }
 
 int launch_evk_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const int8_t* sprime, u64* b_out) {
-    k_evk_finish<<<grid_for((int64_t)c->L * (c->L + 1) * c->N), kThreads, 0, c->stream>>>(as_coeff, e, sprime, b_out, c->N, c->L, c->lt);
-    c->stats.launches++;
+    {
+        KProf kp(c, KC_OTHER);
+        k_evk_finish<<<grid_for((int64_t)c->L * (c->L + 1) * c->N), kThreads, 0, c->stream>>>(as_coeff, e, sprime, b_out, c->N, c->L, c->lt);
+    }
     return check_launch(c, "evk_finish");
 }
 
 int launch_encrypt_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const u64* m, u64* c0_out) {
-    k_encrypt_finish<<<grid_for((int64_t)c->L * c->N), kThreads, 0, c->stream>>>(as_coeff, e, m, c0_out, c->N, c->L, c->lt);
-    c->stats.launches++;
+    {
+        KProf kp(c, KC_OTHER);
+        k_encrypt_finish<<<grid_for((int64_t)c->L * c->N), kThreads, 0, c->stream>>>(as_coeff, e, m, c0_out, c->N, c->L, c->lt);
+    }
     return check_launch(c, "encrypt_finish");
 }

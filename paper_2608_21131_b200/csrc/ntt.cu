@@ -202,13 +202,13 @@ int launch_ntt_fwd(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const 
         if (A.a > 0) {
             dim3 grid(S / A.C, np);
             size_t smem = (size_t)(1 << A.a) * A.C * sizeof(u64);
+            KProf kp(c, KC_NTT_FWD_A);
             k_ntt_fwd_a<<<grid, kThreads, smem, c->stream>>>(Ap, c->lt);
-            c->stats.launches++;
         }
         dim3 grid((c->N >> A.b) / A.K, np);
         size_t smem = (size_t)A.K * S * sizeof(u64);
+        KProf kp(c, KC_NTT_FWD_B);
         k_ntt_fwd_b<<<grid, kThreads, smem, c->stream>>>(Ap, c->lt);
-        c->stats.launches++;
     }
     return check_launch(c, "ntt_fwd");
 }
@@ -224,13 +224,15 @@ int launch_ntt_inv(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const 
         for (int i = 0; i < lm.period; i++) Ap.lm.limb[i] = lm.limb[(p0 + i) % lm.period];
         dim3 grid((c->N >> A.b) / A.K, np);
         size_t smem = (size_t)A.K * S * sizeof(u64);
-        k_ntt_inv_b<<<grid, kThreads, smem, c->stream>>>(Ap, c->lt, A.a == 0 ? 1 : 0);
-        c->stats.launches++;
+        {
+            KProf kp(c, KC_NTT_INV_B);
+            k_ntt_inv_b<<<grid, kThreads, smem, c->stream>>>(Ap, c->lt, A.a == 0 ? 1 : 0);
+        }
         if (A.a > 0) {
             dim3 grid2(S / A.C, np);
             size_t smem2 = (size_t)(1 << A.a) * A.C * sizeof(u64);
+            KProf kp(c, KC_NTT_INV_A);
             k_ntt_inv_a<<<grid2, kThreads, smem2, c->stream>>>(Ap, c->lt);
-            c->stats.launches++;
         }
     }
     return check_launch(c, "ntt_inv");

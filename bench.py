@@ -88,6 +88,21 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(x, dist, device):
+    """the slowest rank's value of a per-rank scalar (identity without a process group)"""
+    import torch
+
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(units_per_rank, world, seconds_slowest):
+    """whole-job throughput of `world` independent replicas: all units divided by the slowest rank's time"""
+    return world * units_per_rank / seconds_slowest
+
+
 def build_workload(config, rows_override=None):
     from paper_2608_21131_b200 import workloads as wl, synth
 
@@ -195,11 +210,8 @@ def run_ours(args):
     clocks = sampler.stop()
     ms_total = e0.elapsed_time(e1)
     launches = ctx.get_stats()["launches"] - l0
-    t = torch.tensor([ms_total], dtype=torch.float64, device=ctx.device)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
-    value = world * n_rows / (ms_step * 1e-3)
+    ms_step = max_over_ranks(ms_total, dist, ctx.device) / args.steps
+    value = replica_throughput(n_rows, world, ms_step * 1e-3)
 
     # correctness of what was timed: decrypted scores against float64 dot products
     score_host = ctx.export(binding.KIND_CT, score, nb)
@@ -267,10 +279,8 @@ def run_ours(args):
     for _ in range(args.steps):
         e2e_step()
     torch.cuda.synchronize()
-    t_e2e = torch.tensor([time.perf_counter() - t0], dtype=torch.float64, device=ctx.device)
-    if dist is not None:
-        dist.all_reduce(t_e2e, op=dist.ReduceOp.MAX)
-    e2e_value = world * n_rows * args.steps / float(t_e2e.item())
+    t_e2e = max_over_ranks(time.perf_counter() - t0, dist, ctx.device)
+    e2e_value = replica_throughput(n_rows * args.steps, world, t_e2e)
     e2e_same = bool(np.array_equal(out_pin.numpy().view(np.uint64), score_host))
     e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(rows_np.nbytes + ct_host.nbytes),
            "d2h_bytes_per_step": int(out_pin.numel() * 8), "matches_device_path": e2e_same}

@@ -1,0 +1,72 @@
+"""The C-ABI library: it loads, exports every function the header declares, the binding covers them, and argument
+validation that needs no GPU returns the documented codes.  No compute call is made here."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2608_21131_b200 import binding, build, synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.load_library()
+
+
+def declared_functions():
+    src = open(os.path.join(ROOT, "include", "hann.h")).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(hann_[a-z0-9_]+)\s*\(", src)))
+
+
+def test_every_declared_symbol_is_exported_and_bound(lib):
+    names = declared_functions()
+    assert len(names) >= 20 and "hann_score_level" in names and "hann_keyswitch" in names
+    for n in names:
+        f = getattr(lib, n)  # raises AttributeError if the symbol is missing
+        assert f.argtypes is not None or n in ("hann_kernel_classes",), n
+
+
+def test_parameter_validation_without_a_device(lib):
+    ps = synth.small_params(8, 8, 4, L=2)
+
+    def create(**kw):
+        p = binding.Params()
+        q = kw.get("q", ps.q)
+        p.logN, p.L, p.p = kw.get("logN", ps.logN), len(q), kw.get("p", ps.p)
+        p.log_scale, p.R, p.B, p.device = ps.log_scale, kw.get("R", ps.R), kw.get("B", ps.B), kw.get("device", 0)
+        for i, v in enumerate(q):
+            p.q[i] = v
+        h = C.c_void_p()
+        rc = lib.hann_ctx_create(C.byref(p), C.byref(h))
+        if rc == 0:
+            lib.hann_ctx_destroy(h)
+        return rc
+
+    assert create(logN=3) == binding.EINVAL
+    assert create(logN=17) == binding.EINVAL
+    assert create(B=3) == binding.EINVAL                      # B must divide R
+    assert create(R=24) == binding.EINVAL                     # R must divide n
+    assert create(q=(ps.q[0], ps.q[0] + 2)) == binding.EINVAL  # composite
+    assert create(q=(ps.q[0], ps.q[0])) == binding.EINVAL      # repeated prime
+    assert create(p=97) == binding.EINVAL                     # prime but not 1 mod 2N
+    assert create(device=99) in (binding.ECUDA,)              # no such device
+    assert lib.hann_ctx_create(None, None) == binding.EINVAL
+    assert lib.hann_sizeof(None, binding.SIZE_CT) == binding.EINVAL
+    assert lib.hann_workspace_bytes(None, 1) == binding.EINVAL
+    assert lib.hann_sync(None) == binding.EINVAL
+    assert lib.hann_last_error(None) == b"null context"
+    lib.hann_ctx_destroy(None)  # a no-op
+
+
+def test_context_refuses_to_run_without_cuda():
+    import torch
+
+    if torch.cuda.is_available():
+        pytest.skip("a CUDA device is present")
+    with pytest.raises(RuntimeError):
+        binding.Context(synth.TOY)

@@ -1,0 +1,57 @@
+"""bench.py across ranks: the path has no exchange step, so N ranks are N independent replicas; the only cross-rank
+logic is the barrier and the max-over-ranks of the measured time.  Covered here with two gloo ranks on CPU."""
+import json
+import os
+import subprocess
+import sys
+import textwrap
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+WORKER = textwrap.dedent(
+    """
+    import os, sys, json
+    sys.path.insert(0, %r)
+    import torch, torch.distributed as dist
+    import bench
+    dist.init_process_group("gloo")
+    rank, world = dist.get_rank(), dist.get_world_size()
+    dist.barrier()
+    ms = bench.max_over_ranks(10.0 * (rank + 1), dist, torch.device("cpu"))
+    val = bench.replica_throughput(1000, world, ms * 1e-3)
+    with open(os.path.join(%r, "rank%%d.json" %% rank), "w") as f:
+        json.dump({"rank": rank, "ms": ms, "value": val}, f)
+    dist.destroy_process_group()
+    """
+)
+
+
+def test_max_over_ranks_and_replica_value_with_two_gloo_ranks(tmp_path):
+    script = tmp_path / "worker.py"
+    script.write_text(WORKER % (ROOT, str(tmp_path)))
+    out = subprocess.run(
+        [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr", "127.0.0.1",
+         "--master-port", "29731", str(script)],
+        capture_output=True, text=True, timeout=300, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    recs = [json.load(open(tmp_path / ("rank%d.json" % r))) for r in (0, 1)]
+    assert sorted(r["rank"] for r in recs) == [0, 1]
+    for r in recs:
+        assert r["ms"] == 20.0                 # the slower rank's time on both ranks
+        assert abs(r["value"] - 2 * 1000 / 0.020) < 1e-6
+
+
+def test_reference_arm_runs_on_rank_zero_only():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2"],
+                         capture_output=True, text=True, timeout=120, env=env, cwd=ROOT)
+    assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_single_process_identity():
+    sys.path.insert(0, ROOT)
+    import torch
+    import bench
+
+    assert bench.max_over_ranks(3.5, None, torch.device("cpu")) == 3.5
+    assert bench.replica_throughput(100, 1, 0.5) == 200.0

@@ -181,6 +181,23 @@ int hann_rotate_sum(hann_ctx *ctx, const void *inner_dev, int64_t n_blocks, void
  * the key, ModDown: out_i = (u_i - centred([u]_p)) * p^{-1} mod q_i. */
 int hann_keyswitch(hann_ctx *ctx, int rot, const void *poly_dev, void *ks0_dev, void *ks1_dev, void *ws, size_t ws_bytes);
 
+/* (No counterpart in the paper.)  hann_keyswitch for callers that can neither allocate device memory nor lend a
+ * workspace -- for instance a request handler that must avoid the device-wide synchronisation of cudaMalloc/cudaFree,
+ * or a process whose device memory was fully partitioned by its own pool at start-up.  Same inputs, outputs and result
+ * bits as hann_keyswitch; the scratch is a fixed hann_static_scratch_bytes() (4 MiB) array inside the library image,
+ * which every GPU that loads the library holds until the process exits.
+ *   - Rings whose key switch needs more than that (e.g. N >= 2^15 with L = 4) are refused with HANN_ESHAPE and a message
+ *     naming both sizes; use hann_keyswitch there.
+ *   - The call performs no cudaMalloc/cudaFree and calls no allocating routine; it returns HANN_EINVAL while the
+ *     per-launch profile (hann_kernel_profile) is on, because that profile creates events on demand.
+ *   - The first call on a device looks up the array's device address (once per device, with the context's device
+ *     current); make that first call before starting any stream capture.
+ *   - All calls on one device share the one array, which keeps whatever the last call left in it (nothing needs
+ *     clearing: every part is written before it is read).  Two calls whose kernels overlap on the GPU -- different
+ *     streams, different contexts, different threads -- race on it; serialise them. */
+int64_t hann_static_scratch_bytes(void);
+int hann_keyswitch_static(hann_ctx *ctx, int rot, const void *poly_dev, void *ks0_dev, void *ks1_dev);
+
 /* Convert `count` elements between the canonical layout (host or device pointer) and the internal device layout.
  * kind POLY / PT: one polynomial of L limbs per element; CT: two. */
 int hann_import(hann_ctx *ctx, int kind, const uint64_t *canonical, int64_t count, void *internal_dev);

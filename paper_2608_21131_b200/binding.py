@@ -77,6 +77,8 @@ def load_library():
         "hann_score_level": (C.c_int, [vp, vp, vp, i64, vp, vp, sz]),
         "hann_rotate_sum": (C.c_int, [vp, vp, i64, vp, vp, sz]),
         "hann_keyswitch": (C.c_int, [vp, C.c_int, vp, vp, vp, vp, sz]),
+        "hann_static_scratch_bytes": (i64, []),
+        "hann_keyswitch_static": (C.c_int, [vp, C.c_int, vp, vp, vp]),
         "hann_import": (C.c_int, [vp, C.c_int, vp, i64, vp]),
         "hann_export": (C.c_int, [vp, C.c_int, vp, i64, vp]),
         "hann_level_host_bytes": (i64, [vp, i64]),
@@ -265,6 +267,16 @@ class Context:
         ks0 = self.alloc(self.sizeof(SIZE_POLY))
         ks1 = self.alloc(self.sizeof(SIZE_POLY))
         self._ck(self.lib.hann_keyswitch(self.h, rot, _ptr(poly), _ptr(ks0), _ptr(ks1), _ptr(ws), ws.numel() * 8))
+        return ks0, ks1
+
+    def keyswitch_static(self, rot, poly, ks0=None, ks1=None):
+        """hann_keyswitch_static: same result as `keyswitch`, scratch inside the library (no workspace argument).
+        The two output polynomials may be passed in so that the call itself allocates nothing."""
+        if ks0 is None:
+            ks0 = self.alloc(self.sizeof(SIZE_POLY))
+        if ks1 is None:
+            ks1 = self.alloc(self.sizeof(SIZE_POLY))
+        self._ck(self.lib.hann_keyswitch_static(self.h, rot, _ptr(poly), _ptr(ks0), _ptr(ks1)))
         return ks0, ks1
 
     def level_host_bytes(self, n_rows):

@@ -163,6 +163,8 @@ def run_ours(args):
     ps, rows_np, qR, wname = build_workload(args.config, args.rows)
     n_rows = rows_np.shape[0]
     ctx = binding.Context(ps, device=local)
+    if args.encode_group:
+        ctx.set_tuning(binding.TUNE_ENCODE_GROUP, args.encode_group)
     km = synth.key_material(ps, wl.KEY_SEED)
     evk = ctx.keygen_from_samples(km.s, km.rots, km.evk_a, km.evk_e)
     ctx.load_keys(evk, km.rots)
@@ -379,6 +381,7 @@ def main():
     ap.add_argument("--config", type=int, default=1)
     ap.add_argument("--rows", type=int, default=None, help="override the row count (debugging, ncu captures)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--encode-group", type=int, default=None, help="tuning: plaintexts per encode launch group")
     ap.add_argument("--lean", action="store_true", help="only run warm-up + steps (for ncu); prints no JSON line")
     args = ap.parse_args()
     if args.impl == "reference":

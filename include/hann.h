@@ -111,6 +111,11 @@ const char *hann_last_error(const hann_ctx *ctx);
 int hann_set_timing(hann_ctx *ctx, int enable);
 int hann_get_stats(hann_ctx *ctx, hann_stats *out);
 
+/* Performance knobs (results never depend on them).  HANN_TUNE_ENCODE_GROUP: plaintexts encoded and transformed per
+ * launch group in hann_encode_candidates (default: all R plaintexts of a block at once); ask hann_workspace_bytes again after changing it. */
+enum { HANN_TUNE_ENCODE_GROUP = 1 };
+int hann_set_tuning(hann_ctx *ctx, int what, int value);
+
 /* Per-launch profile: while enabled every kernel launch of the context is bracketed by a CUDA event pair (this
  * serialises nothing but adds two event records per launch).  hann_kernel_times synchronises, writes the summed
  * device milliseconds and launch counts per kernel class (arrays of hann_kernel_classes() entries, class names from

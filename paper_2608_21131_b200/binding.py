@@ -19,6 +19,7 @@ HANN_MAX_PRIMES = 8
 OK, EINVAL, ESHAPE, ENOKEY, EWORKSPACE, ECUDA, ENOMEM = 0, -1, -2, -3, -4, -5, -6
 SIZE_POLY, SIZE_CT, SIZE_BABY, SIZE_PT_BLOCK, SIZE_INNER, SIZE_EVK, SIZE_ROWS_PER_BLOCK = 1, 2, 3, 4, 5, 6, 7
 KIND_POLY, KIND_CT, KIND_PT = 1, 2, 3
+TUNE_ENCODE_GROUP = 1
 
 
 class HannError(RuntimeError):
@@ -49,11 +50,12 @@ def load_library():
     global _lib
     if _lib is not None:
         return _lib
-    if not os.path.exists(LIB_PATH):
+    path = os.environ.get("HANN_LIB", LIB_PATH)  # development override: an alternative build of the same library
+    if not os.path.exists(path):
         raise RuntimeError(
-            "the CUDA library %s is missing: build it with `python -m paper_2608_21131_b200.build`" % LIB_PATH
+            "the CUDA library %s is missing: build it with `python -m paper_2608_21131_b200.build`" % path
         )
-    lib = C.CDLL(LIB_PATH)
+    lib = C.CDLL(path)
     vp, i64, sz = C.c_void_p, C.c_int64, C.c_size_t
     sig = {
         "hann_ctx_create": (C.c_int, [C.POINTER(Params), C.POINTER(vp)]),
@@ -64,6 +66,7 @@ def load_library():
         "hann_last_error": (C.c_char_p, [vp]),
         "hann_set_timing": (C.c_int, [vp, C.c_int]),
         "hann_get_stats": (C.c_int, [vp, C.POINTER(Stats)]),
+        "hann_set_tuning": (C.c_int, [vp, C.c_int, C.c_int]),
         "hann_kernel_classes": (C.c_int, []),
         "hann_kernel_name": (C.c_char_p, [C.c_int]),
         "hann_kernel_profile": (C.c_int, [vp, C.c_int]),
@@ -173,6 +176,9 @@ class Context:
         st = Stats()
         self._ck(self.lib.hann_get_stats(self.h, C.byref(st)))
         return {k: getattr(st, k) for k, _ in Stats._fields_}
+
+    def set_tuning(self, what, value):
+        self._ck(self.lib.hann_set_tuning(self.h, what, value))
 
     def kernel_profile(self, on):
         self._ck(self.lib.hann_kernel_profile(self.h, 1 if on else 0))

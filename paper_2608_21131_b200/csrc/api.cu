@@ -183,7 +183,9 @@ extern "C" int hann_ctx_create(const hann_params* prm, hann_ctx** out) {
     if (!dg.ok) { delete c; return HANN_ECUDA; }
 
     // per-limb constants and transform tables
-    std::vector<u64> twf((size_t)(L + 1) * N), twfs((size_t)(L + 1) * N), twi((size_t)(L + 1) * N), twis((size_t)(L + 1) * N);
+    // tables of (w, floor(w * 2^64 / q)) pairs, [L+1][N][2]
+    std::vector<u64> twf((size_t)(L + 1) * N * 2), twi((size_t)(L + 1) * N * 2);
+    std::vector<double> twf64((size_t)(L + 1) * N * 2), twi64((size_t)(L + 1) * N * 2);
     std::vector<u64> pw(N), ipw(N);
     for (int i = 0; i <= L; i++) {
         const u64 q = mods[i];
@@ -196,6 +198,11 @@ extern "C" int hann_ctx_create(const hann_params* prm, hann_ctx** out) {
         lc.ninv = hm::invmod((u64)N % q, q);
         lc.ninv_s = hm::shoup(lc.ninv, q);
         lc.half = q / 2;
+        {
+            const double nb = lc.ninv > q / 2 ? -(double)(q - lc.ninv) : (double)lc.ninv;
+            lc.ninv_bal = nb;
+            lc.ninv_q = nb / (double)q;
+        }
         if (i < L) {
             lc.pmod = prm->p % q;
             lc.pinv = hm::invmod(lc.pmod, q);
@@ -211,9 +218,14 @@ extern "C" int hann_ctx_create(const hann_params* prm, hann_ctx** out) {
         }
         for (int k = 0; k < N; k++) {
             const int br = hm::bitrev(k, c->logN);
-            const size_t o = (size_t)i * N + k;
-            twf[o] = pw[br];  twfs[o] = hm::shoup(pw[br], q);
-            twi[o] = ipw[br]; twis[o] = hm::shoup(ipw[br], q);
+            const size_t o = ((size_t)i * N + k) * 2;
+            twf[o] = pw[br];  twf[o + 1] = hm::shoup(pw[br], q);
+            twi[o] = ipw[br]; twi[o + 1] = hm::shoup(ipw[br], q);
+            // balanced copies for the binary64 path (exact for q < 2^53; only used when q < 2^50)
+            const double wb = pw[br] > q / 2 ? -(double)(q - pw[br]) : (double)pw[br];
+            const double iwb = ipw[br] > q / 2 ? -(double)(q - ipw[br]) : (double)ipw[br];
+            twf64[o] = wb;  twf64[o + 1] = wb / (double)q;
+            twi64[o] = iwb; twi64[o + 1] = iwb / (double)q;
         }
     }
     // encode tables
@@ -237,17 +249,19 @@ extern "C" int hann_ctx_create(const hann_params* prm, hann_ctx** out) {
             g = (g * 5) % (2L * N);
         }
     }
-    const size_t twb = (size_t)(L + 1) * N * 8;
-    bool ok = cudaMalloc(&c->tw_fwd, twb) == cudaSuccess && cudaMalloc(&c->tw_fwd_s, twb) == cudaSuccess &&
-              cudaMalloc(&c->tw_inv, twb) == cudaSuccess && cudaMalloc(&c->tw_inv_s, twb) == cudaSuccess &&
+    const size_t twb = (size_t)(L + 1) * N * 16;
+    bool ok = cudaMalloc(&c->tw_fwd, twb) == cudaSuccess && cudaMalloc(&c->tw_inv, twb) == cudaSuccess &&
+              cudaMalloc(&c->tw_fwd_f64, twb) == cudaSuccess && cudaMalloc(&c->tw_inv_f64, twb) == cudaSuccess &&
+              cudaMalloc(&c->lt_dev, sizeof(LimbTable)) == cudaSuccess &&
               cudaMalloc(&c->fft_T, nh * sizeof(double2)) == cudaSuccess && cudaMalloc(&c->fft_U, n * sizeof(double2)) == cudaSuccess &&
               cudaMalloc(&c->jinv, n * sizeof(int32_t)) == cudaSuccess && cudaMalloc(&c->galois_dev, n * sizeof(unsigned)) == cudaSuccess &&
               cudaMalloc(&c->keytab_dev, n * sizeof(u64*)) == cudaSuccess;
     if (ok) {
         ok = cudaMemcpy(c->tw_fwd, twf.data(), twb, cudaMemcpyHostToDevice) == cudaSuccess &&
-             cudaMemcpy(c->tw_fwd_s, twfs.data(), twb, cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->tw_inv, twi.data(), twb, cudaMemcpyHostToDevice) == cudaSuccess &&
-             cudaMemcpy(c->tw_inv_s, twis.data(), twb, cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(c->tw_fwd_f64, twf64.data(), twb, cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(c->tw_inv_f64, twi64.data(), twb, cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(c->lt_dev, &c->lt, sizeof(LimbTable), cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->fft_T, T.data(), nh * sizeof(double2), cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->fft_U, U.data(), n * sizeof(double2), cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->jinv, jinv.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess &&
@@ -274,7 +288,7 @@ extern "C" void hann_ctx_destroy(hann_ctx* c) {
     cudaStreamSynchronize(c->stream);
     for (u64* k : c->keytab_host)
         if (k) cudaFree(k);
-    cudaFree(c->tw_fwd); cudaFree(c->tw_fwd_s); cudaFree(c->tw_inv); cudaFree(c->tw_inv_s);
+    cudaFree(c->tw_fwd); cudaFree(c->tw_inv); cudaFree(c->tw_fwd_f64); cudaFree(c->tw_inv_f64); cudaFree(c->lt_dev);
     cudaFree(c->fft_T); cudaFree(c->fft_U); cudaFree(c->jinv); cudaFree(c->galois_dev); cudaFree(c->keytab_dev);
     if (c->scratch) cudaFree(c->scratch);
     for (auto& r : c->krec) {
@@ -326,6 +340,17 @@ extern "C" int hann_set_timing(hann_ctx* c, int enable) {
     if (!c) return HANN_EINVAL;
     c->timing = enable ? 1 : 0;
     return HANN_OK;
+}
+
+extern "C" int hann_set_tuning(hann_ctx* c, int what, int value) {
+    if (!c) return HANN_EINVAL;
+    switch (what) {
+        case HANN_TUNE_ENCODE_GROUP:
+            if (value < 1) return fail(c, HANN_EINVAL, "hann_set_tuning: encode group must be positive");
+            c->encode_group = value;
+            return HANN_OK;
+        default: return fail(c, HANN_EINVAL, "hann_set_tuning: unknown knob");
+    }
 }
 
 extern "C" int hann_get_stats(hann_ctx* c, hann_stats* out) {
@@ -608,8 +633,12 @@ extern "C" int hann_encode_candidates(hann_ctx* c, const float* rows_dev, int64_
     for (int64_t blk = 0; blk < nblk; blk++) {
         const int64_t rows_here = std::min(n, n_rows - blk * n);
         u64* pt = (u64*)pt_dev + blk * ptw;
-        RET(launch_encode_rows(c, rows_dev + blk * n * dim, rows_here, dim, pt, ws));
-        RET(launch_ntt_fwd(c, pt, (int64_t)c->R * c->L, c->N, limbmap_q(c)));
+        // a few plaintexts at a time: FFT buffer and residues of a group are re-read from L2, not from HBM
+        for (int p0 = 0; p0 < c->R; p0 += c->encode_group) {
+            const int cnt = std::min(c->encode_group, c->R - p0);
+            RET(launch_encode_rows(c, rows_dev + blk * n * dim, rows_here, dim, p0, cnt, pt, ws));
+            RET(launch_ntt_fwd(c, pt + (int64_t)p0 * c->L * c->N, (int64_t)cnt * c->L, c->N, limbmap_q(c)));
+        }
     }
     return HANN_OK;
 }

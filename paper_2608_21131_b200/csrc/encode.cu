@@ -28,9 +28,10 @@ struct EncArgs {
     const int32_t* jinv;
     int logn, b1, K1, C1;
     double scale;  // Delta / n
-    double2* buf;  // [P][n]
-    u64* out;      // [P][L][N] coefficient-domain residues
+    double2* buf;  // [P][n], indexed by blockIdx.y
+    u64* out;      // [..][L][N] coefficient-domain residues, indexed by p_first + blockIdx.y
     int L;
+    int p_first;   // index (g*B + b) of the first plaintext of this launch
 };
 
 __device__ __forceinline__ double2 cmul_rn(double2 y, double2 w) {
@@ -42,7 +43,7 @@ __global__ void __launch_bounds__(kThreads) k_fft_a(EncArgs A) {
     extern __shared__ double2 smc[];
     const int n = 1 << A.logn, S1 = 1 << A.b1, K1 = A.K1;
     const int P = blockIdx.y;
-    const int g = P / A.B, b = P % A.B;
+    const int g = (A.p_first + P) / A.B, b = (A.p_first + P) % A.B;
     const int pos0 = blockIdx.x * K1 * S1;
     for (int idx = threadIdx.x; idx < K1 * S1; idx += kThreads) {
         const int pos = pos0 + idx;
@@ -101,7 +102,7 @@ __global__ void __launch_bounds__(kThreads) k_fft_b(EncArgs A, LimbTable lt) {
         }
         __syncthreads();
     }
-    u64* out = A.out + (long long)P * A.L * N;
+    u64* out = A.out + (long long)(A.p_first + P) * A.L * N;
     for (int idx = threadIdx.x; idx < rows * C1; idx += kThreads) {
         const int k = (idx / C1) * S1 + c0 + (idx % C1);
         double2 cc = cmul_rn(smc[idx], A.U[k]);
@@ -141,10 +142,15 @@ int run_encode(hann_ctx* c, EncArgs& A, int P) {
 
 }  // namespace
 
-int64_t encode_ws_bytes(const hann_ctx* c) { return (int64_t)c->R * c->n * (int64_t)sizeof(double2); }
+int64_t encode_ws_bytes(const hann_ctx* c) {
+    const int group = c->encode_group < c->R ? c->encode_group : c->R;
+    return (int64_t)group * c->n * (int64_t)sizeof(double2);
+}
 
-// one block of candidate rows -> R plaintexts [G][B][L][N], coefficient domain (the caller transforms them)
-int launch_encode_rows(hann_ctx* c, const float* rows, int64_t rows_in_block, int dim, u64* pt_block, void* ws) {
+// plaintexts p_first .. p_first+count-1 of one block of candidate rows -> pt_block[p][L][N], coefficient domain (the
+// caller transforms them); ws holds count complex vectors of n points
+int launch_encode_rows(hann_ctx* c, const float* rows, int64_t rows_in_block, int dim, int p_first, int count, u64* pt_block,
+                       void* ws) {
     EncArgs A = {};
     A.rows = rows;
     A.rows_in_block = rows_in_block;
@@ -152,7 +158,8 @@ int launch_encode_rows(hann_ctx* c, const float* rows, int64_t rows_in_block, in
     A.z = nullptr;
     A.buf = (double2*)ws;
     A.out = pt_block;
-    return run_encode(c, A, c->R);
+    A.p_first = p_first;
+    return run_encode(c, A, count);
 }
 
 // one slot vector z[n] (device) -> one polynomial [L][N], coefficient domain

@@ -23,8 +23,11 @@ struct hann_ctx {
     cudaStream_t stream = nullptr;
     u64 mod[HANN_MAXL1] = {};  // q_0..q_{L-1}, p
     LimbTable lt = {};
-    // transform tables on the device, [L+1][N] each: psi^brev(k) and psi^-brev(k) with their Shoup companions
-    u64 *tw_fwd = nullptr, *tw_fwd_s = nullptr, *tw_inv = nullptr, *tw_inv_s = nullptr;
+    LimbConst* lt_dev = nullptr;  // device copy of lt.c (the transform kernels read it from memory)
+    // transform tables on the device, [L+1][N][2]: (w, floor(w*2^64/q)) for w = psi^brev(k) and psi^-brev(k)
+    u64 *tw_fwd = nullptr, *tw_inv = nullptr;
+    // the same twiddles for the binary64 transform path, [L+1][N][2] doubles: (balanced w, fl(w / q))
+    double *tw_fwd_f64 = nullptr, *tw_inv_f64 = nullptr;
     // encode tables on the device
     double2* fft_T = nullptr;  // [n/2] exp(-2 pi i t / n)
     double2* fft_U = nullptr;  // [n]   exp(-i pi k / N)
@@ -41,6 +44,8 @@ struct hann_ctx {
     // growable device scratch of the exchange and client calls (never used by the server-side scoring calls)
     void* scratch = nullptr;
     int64_t scratch_bytes = 0;
+    // plaintexts encoded and transformed per launch group: small enough that the group's intermediates stay in L2
+    int encode_group = 1 << 20;
     // statistics
     hann_stats stats = {};
     int timing = 0;
@@ -102,7 +107,8 @@ LimbMap limbmap_qp(const hann_ctx* c);  // period L+1: limbs 0..L
 LimbMap limbmap_single(int limb);
 
 // encode (coefficient-domain residues out; the caller transforms)
-int launch_encode_rows(hann_ctx* c, const float* rows, int64_t rows_in_block, int dim, u64* pt_block, void* ws);
+int launch_encode_rows(hann_ctx* c, const float* rows, int64_t rows_in_block, int dim, int p_first, int count, u64* pt_block,
+                       void* ws);
 int launch_encode_slots(hann_ctx* c, const double* z_dev, u64* poly_out, void* ws);
 int64_t encode_ws_bytes(const hann_ctx* c);
 

@@ -23,6 +23,8 @@ struct LimbConst {
     u64 pinv_s;
     u64 pmod;    // p mod q               (ciphertext primes only)
     u64 half;    // floor(q / 2): residues above it lift to negative integers
+    double ninv_bal;  // N^{-1} mod q as a balanced integer (binary64 transform path)
+    double ninv_q;    // fl(ninv_bal / q)
 };
 
 #define HANN_MAXL1 9  // up to 8 ciphertext primes + the special prime

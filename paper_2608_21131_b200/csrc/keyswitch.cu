@@ -17,8 +17,9 @@ inline int grid_for(int64_t work, int per_block = kThreads, int cap = 148 * 16) 
 // ------------------------------------------------------------------------------------------ multiply-accumulate
 
 // inner[blk][g][comp][l][x] = sum_b pt[blk][g][b][l][x] * baby[b][comp][l][x] mod q_l.
-// One thread owns one (l, x) position for a range of (blk, g) pairs; products are accumulated in 128 bits and
-// reduced once per output.
+//
+// Generic kernel (any modulus): one thread owns one (l, x) position for a range of (blk, g) pairs; products are
+// accumulated in 128 bits and reduced once per output.
 __global__ void __launch_bounds__(kThreads) k_mac(const u64* __restrict__ baby, const u64* __restrict__ pt,
                                                   u64* __restrict__ inner, int N, int L, int B, int G,
                                                   long long n_bg, LimbTable lt) {
@@ -38,6 +39,96 @@ __global__ void __launch_bounds__(kThreads) k_mac(const u64* __restrict__ baby, 
             o[0] = reduce128(h0, l0, lc);
             o[LN] = reduce128(h1, l1, lc);
         }
+    }
+}
+
+// Streaming kernel for moduli below 2^50 (the HBM-bound case the path is sized for).  A CTA owns 32 consecutive
+// positions of one limb.  Its NG warps split the B baby steps among them: warp w keeps the baby-step words of steps
+// w*BB .. w*BB+BB-1 (both ciphertext components) for its lane's position in REGISTERS for the CTA's whole life, and
+// streams the matching plaintext rows of every (blk, g) pair past them, so every plaintext word is read from HBM
+// exactly once, 256 contiguous bytes per warp load, with the next pair's loads in flight while the current pair is
+// multiplied.  The warps' partial sums meet in shared memory once per (blk, g) pair.
+// The GPU has no native 64-bit multiplier, so each residue is split into two 25-bit halves and a product costs three
+// 32x32->64 multiply-adds (Karatsuba) accumulated carry-free in 64-bit registers: a sum of B <= 128 products of
+// 25-bit halves stays below 2^57, of the 26-bit half sums below 2^59.
+constexpr unsigned kM25 = (1u << 25) - 1;
+
+template <int NG, int BB>
+__global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ baby, const u64* __restrict__ pt,
+                                                        u64* __restrict__ inner, int N, int L, long long n_bg,
+                                                        int bg_per_cta, const LimbConst* __restrict__ lt) {
+    constexpr int B = NG * BB;
+    __shared__ u64 part[2][NG][6][32];
+    const long long LN = (long long)L * N;
+    const long long pos0 = (long long)blockIdx.x * 32;
+    const int lane = threadIdx.x & 31, wg = threadIdx.x >> 5;
+    const LimbConst* lc = lt + pos0 / N;
+    // this warp's baby-step words, split into 25-bit halves: lo half in the low word, hi half in the high word
+    unsigned w0[BB][2], w1[BB][2];
+#pragma unroll
+    for (int k = 0; k < BB; k++)
+#pragma unroll
+        for (int c = 0; c < 2; c++) {
+            const u64 v = baby[((long long)(wg * BB + k) * 2 + c) * LN + pos0 + lane];
+            w0[k][c] = (unsigned)v & kM25;
+            w1[k][c] = (unsigned)(v >> 25);
+        }
+    const long long bg0 = (long long)blockIdx.y * bg_per_cta;
+    const long long bg1 = bg0 + bg_per_cta < n_bg ? bg0 + bg_per_cta : n_bg;
+    if (bg0 >= bg1) return;
+    const u64* p = pt + (bg0 * B + wg * BB) * LN + pos0 + lane;
+    u64 cur[BB], nxt[BB];
+#pragma unroll
+    for (int k = 0; k < BB; k++) cur[k] = __ldcs(p + (long long)k * LN);
+    for (long long bg = bg0; bg < bg1; bg++) {
+        if (bg + 1 < bg1) {
+            const u64* pn = p + (long long)B * LN;
+#pragma unroll
+            for (int k = 0; k < BB; k++) nxt[k] = __ldcs(pn + (long long)k * LN);
+        }
+        u64 p00[2] = {0, 0}, p11[2] = {0, 0}, pm[2] = {0, 0};
+#pragma unroll
+        for (int k = 0; k < BB; k++) {
+            const unsigned a0 = (unsigned)cur[k] & kM25, a1 = (unsigned)(cur[k] >> 25), as = a0 + a1;
+#pragma unroll
+            for (int c = 0; c < 2; c++) {
+                p00[c] += (u64)a0 * w0[k][c];
+                p11[c] += (u64)a1 * w1[k][c];
+                pm[c] += (u64)as * (w0[k][c] + w1[k][c]);
+            }
+        }
+        u64(*buf)[6][32] = part[bg & 1];
+#pragma unroll
+        for (int c = 0; c < 2; c++) {
+            buf[wg][c * 3 + 0][lane] = p00[c];
+            buf[wg][c * 3 + 1][lane] = pm[c];
+            buf[wg][c * 3 + 2][lane] = p11[c];
+        }
+        __syncthreads();
+        // warps 0 and 1 (or warp 0 twice when NG == 1) finish component 0 and 1
+        for (int c = wg; c < 2; c += NG) {
+            u64 s00 = 0, sm = 0, s11 = 0;
+#pragma unroll
+            for (int g = 0; g < NG; g++) {
+                s00 += buf[g][c * 3 + 0][lane];
+                sm += buf[g][c * 3 + 1][lane];
+                s11 += buf[g][c * 3 + 2][lane];
+            }
+            // value = s00 + cross * 2^25 + s11 * 2^50 with cross = sm - s00 - s11 < 2^59
+            const u64 cross = sm - s00 - s11;
+            u64 lo = s00, hi = 0;
+            const u64 c_lo = cross << 25, c_hi = cross >> 39;
+            lo += c_lo;
+            hi += c_hi + (lo < c_lo ? 1 : 0);
+            const u64 d_lo = s11 << 50, d_hi = s11 >> 14;
+            lo += d_lo;
+            hi += d_hi + (lo < d_lo ? 1 : 0);
+            inner[(bg * 2 + c) * LN + pos0 + lane] = reduce128(hi, lo, *lc);
+        }
+        if (NG == 1) __syncthreads();  // a single warp reuses the buffer it just read
+#pragma unroll
+        for (int k = 0; k < BB; k++) cur[k] = nxt[k];
+        p += (long long)B * LN;
     }
 }
 
@@ -233,10 +324,39 @@ int check_launch(hann_ctx* c, const char* what) {
     return HANN_OK;
 }
 
+template <int NG, int BB>
+void launch_mac_stream(hann_ctx* c, const u64* baby, const u64* pt, int64_t n_bg, u64* inner) {
+    const long long LN = (long long)c->L * c->N;
+    const int tiles = (int)(LN / 32);
+    // split the (blk, g) range over grid.y only as far as needed to fill the machine: every extra split re-reads the
+    // baby-step words
+    int split = 1;
+    while ((long long)tiles * split < 148 * 8 && split < n_bg) split *= 2;
+    const int per = (int)((n_bg + split - 1) / split);
+    split = (int)((n_bg + per - 1) / per);
+    KProf kp(c, KC_MAC);
+    k_mac_stream<NG, BB><<<dim3(tiles, split), 32 * NG, 0, c->stream>>>(baby, pt, inner, c->N, c->L, n_bg, per, c->lt_dev);
+}
+
 int launch_mac(hann_ctx* c, const u64* baby, const u64* pt, int64_t n_blocks, u64* inner) {
     if (n_blocks <= 0) return HANN_OK;
     const long long LN = (long long)c->L * c->N;
     const long long n_bg = n_blocks * c->G;
+    bool small = c->N >= 32 && c->B <= 128;
+    for (int l = 0; l < c->L; l++) small = small && c->mod[l] < (1ULL << 50);
+    if (small) {
+        switch (c->B) {
+            case 1: launch_mac_stream<1, 1>(c, baby, pt, n_bg, inner); break;
+            case 2: launch_mac_stream<2, 1>(c, baby, pt, n_bg, inner); break;
+            case 4: launch_mac_stream<4, 1>(c, baby, pt, n_bg, inner); break;
+            case 8: launch_mac_stream<4, 2>(c, baby, pt, n_bg, inner); break;
+            case 16: launch_mac_stream<4, 4>(c, baby, pt, n_bg, inner); break;
+            case 32: launch_mac_stream<4, 8>(c, baby, pt, n_bg, inner); break;
+            case 64: launch_mac_stream<8, 8>(c, baby, pt, n_bg, inner); break;
+            default: launch_mac_stream<8, 16>(c, baby, pt, n_bg, inner); break;
+        }
+        return check_launch(c, "mac_stream");
+    }
     int gx = (int)((LN + kThreads - 1) / kThreads);
     int gy = 1;
     // enough CTAs to fill the machine even for a single small block

@@ -183,6 +183,98 @@ __global__ void __launch_bounds__(kThreads) k_ks_inner(const u64* __restrict__ d
     }
 }
 
+// Streaming form of the same inner product for L <= 4 digits.  A thread owns one position (modulus i, coefficient x)
+// and loops over the items.  When the items share one digit set and differ by key (the hoisted baby rotations:
+// KEYS_STREAM), the L digit words stay in registers and the 2L key words of each item stream past them; when the
+// items share the key (rotate-and-sum over blocks), the key words stay and the digit words stream.  The streamed
+// words of the next item are in flight while the current item is multiplied.  Moduli below 2^50 use the carry-free
+// 25-bit Karatsuba products of the multiply-accumulate kernel; the special prime uses 128-bit accumulation.
+template <int LL, bool KEYS_STREAM>
+__global__ void __launch_bounds__(128) k_ks_inner_stream(const u64* __restrict__ digits, long long digit_stride,
+                                                         const u64* const* __restrict__ keytab, int rot0, int rot_inc,
+                                                         u64* __restrict__ u, int N, long long nitems, int items_per_cta,
+                                                         const LimbConst* __restrict__ lt) {
+    constexpr int NS = KEYS_STREAM ? 2 * LL : LL;  // streamed words per item
+    const long long L1N = (long long)(LL + 1) * N;
+    const long long pos = (long long)blockIdx.x * 128 + threadIdx.x;  // i*N + x
+    const int i = (int)(pos / N);
+    const LimbConst lc = lt[i];
+    const bool small = lc.q < (1ULL << 50);
+    const long long it0 = (long long)blockIdx.y * items_per_cta;
+    const long long it1 = it0 + items_per_cta < nitems ? it0 + items_per_cta : nitems;
+    if (it0 >= it1) return;
+    // stationary words
+    u64 st[KEYS_STREAM ? LL : 2 * LL];
+    if (KEYS_STREAM) {
+#pragma unroll
+        for (int j = 0; j < LL; j++) st[j] = digits[(long long)j * L1N + pos];
+    } else {
+        const u64* key = keytab[rot0];
+#pragma unroll
+        for (int j = 0; j < LL; j++) {
+            st[2 * j] = key[((long long)j * 2 + 0) * L1N + pos];
+            st[2 * j + 1] = key[((long long)j * 2 + 1) * L1N + pos];
+        }
+    }
+    u64 cur[NS], nxt[NS];
+    auto load = [&](long long item, u64(&v)[NS]) {
+        if (KEYS_STREAM) {
+            const u64* key = keytab[rot0 + (int)item * rot_inc];
+#pragma unroll
+            for (int k = 0; k < NS; k++) v[k] = __ldcs(key + (long long)k * L1N + pos);  // k = j*2 + comp
+        } else {
+            const u64* d = digits + item * digit_stride + pos;
+#pragma unroll
+            for (int k = 0; k < NS; k++) v[k] = __ldcs(d + (long long)k * L1N);
+        }
+    };
+    load(it0, cur);
+    for (long long item = it0; item < it1; item++) {
+        if (item + 1 < it1) load(item + 1, nxt);
+        u64 out[2];
+        if (small) {
+            u64 p00[2] = {0, 0}, p11[2] = {0, 0}, pm[2] = {0, 0};
+#pragma unroll
+            for (int j = 0; j < LL; j++)
+#pragma unroll
+                for (int c = 0; c < 2; c++) {
+                    const u64 dv = KEYS_STREAM ? st[j] : cur[j];
+                    const u64 kv = KEYS_STREAM ? cur[2 * j + c] : st[2 * j + c];
+                    const unsigned a0 = (unsigned)dv & kM25, a1 = (unsigned)(dv >> 25);
+                    const unsigned b0 = (unsigned)kv & kM25, b1 = (unsigned)(kv >> 25);
+                    p00[c] += (u64)a0 * b0;
+                    p11[c] += (u64)a1 * b1;
+                    pm[c] += (u64)(a0 + a1) * (b0 + b1);
+                }
+#pragma unroll
+            for (int c = 0; c < 2; c++) {
+                const u64 cross = pm[c] - p00[c] - p11[c];
+                u64 lo = p00[c], hi = 0;
+                const u64 c_lo = cross << 25, c_hi = cross >> 39;
+                lo += c_lo;
+                hi += c_hi + (lo < c_lo ? 1 : 0);
+                const u64 d_lo = p11[c] << 50, d_hi = p11[c] >> 14;
+                lo += d_lo;
+                hi += d_hi + (lo < d_lo ? 1 : 0);
+                out[c] = reduce128(hi, lo, lc);
+            }
+        } else {
+            u64 h[2] = {0, 0}, l[2] = {0, 0};
+#pragma unroll
+            for (int j = 0; j < LL; j++)
+#pragma unroll
+                for (int c = 0; c < 2; c++) mac128(h[c], l[c], KEYS_STREAM ? st[j] : cur[j], KEYS_STREAM ? cur[2 * j + c] : st[2 * j + c]);
+            out[0] = reduce128(h[0], l[0], lc);
+            out[1] = reduce128(h[1], l[1], lc);
+        }
+        u64* o = u + item * 2 * L1N + pos;
+        o[0] = out[0];
+        o[L1N] = out[1];
+#pragma unroll
+        for (int k = 0; k < NS; k++) cur[k] = nxt[k];
+    }
+}
+
 // lifted[poly][i][x] = centred lift of up[poly][x] (residue mod p, coefficient domain) reduced mod q_i.
 // up is the special-prime limb inside u: poly = item*2 + comp lives at u + poly*(L+1)*N + L*N.
 __global__ void __launch_bounds__(kThreads) k_moddown_lift(const u64* __restrict__ u, u64* __restrict__ lifted, int N,
@@ -377,7 +469,35 @@ int launch_lift_digits(hann_ctx* c, const u64* src, int64_t src_stride, int64_t 
     return check_launch(c, "lift_digits");
 }
 
+template <int LL>
+void launch_ks_inner_stream(hann_ctx* c, const u64* digits, int64_t digit_stride, int rot0, int rot_inc, int64_t nitems, u64* u) {
+    const long long L1N = (long long)(LL + 1) * c->N;
+    const int tiles = (int)(L1N / 128);
+    int split = 1;
+    while ((long long)tiles * split < 148 * 8 && split < nitems) split *= 2;
+    const int per = (int)((nitems + split - 1) / split);
+    split = (int)((nitems + per - 1) / per);
+    KProf kp(c, KC_KS_INNER);
+    if (digit_stride == 0)
+        k_ks_inner_stream<LL, true><<<dim3(tiles, split), 128, 0, c->stream>>>(digits, 0, c->keytab_dev, rot0, rot_inc, u, c->N, nitems,
+                                                                            per, c->lt_dev);
+    else
+        k_ks_inner_stream<LL, false><<<dim3(tiles, split), 128, 0, c->stream>>>(digits, digit_stride, c->keytab_dev, rot0, rot_inc, u,
+                                                                             c->N, nitems, per, c->lt_dev);
+}
+
 int launch_ks_inner(hann_ctx* c, const u64* digits, int64_t digit_stride, int rot0, int rot_inc, int64_t nitems, u64* u) {
+    // the streaming kernel covers the two shapes the path produces: one digit set under many keys (digit_stride == 0)
+    // and many digit sets under one key (rot_inc == 0)
+    if (c->L <= 4 && c->N >= 128 && (digit_stride == 0 || rot_inc == 0)) {
+        switch (c->L) {
+            case 1: launch_ks_inner_stream<1>(c, digits, digit_stride, rot0, rot_inc, nitems, u); break;
+            case 2: launch_ks_inner_stream<2>(c, digits, digit_stride, rot0, rot_inc, nitems, u); break;
+            case 3: launch_ks_inner_stream<3>(c, digits, digit_stride, rot0, rot_inc, nitems, u); break;
+            default: launch_ks_inner_stream<4>(c, digits, digit_stride, rot0, rot_inc, nitems, u); break;
+        }
+        return check_launch(c, "ks_inner_stream");
+    }
     {
         KProf kp(c, KC_KS_INNER);
         k_ks_inner<<<grid_for(nitems * (c->L + 1) * c->N), kThreads, 0, c->stream>>>(digits, digit_stride, c->keytab_dev, rot0, rot_inc, u,

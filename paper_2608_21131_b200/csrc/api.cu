@@ -636,8 +636,13 @@ extern "C" int hann_encode_candidates(hann_ctx* c, const float* rows_dev, int64_
         // a few plaintexts at a time: FFT buffer and residues of a group are re-read from L2, not from HBM
         for (int p0 = 0; p0 < c->R; p0 += c->encode_group) {
             const int cnt = std::min(c->encode_group, c->R - p0);
-            RET(launch_encode_rows(c, rows_dev + blk * n * dim, rows_here, dim, p0, cnt, pt, ws));
-            RET(launch_ntt_fwd(c, pt + (int64_t)p0 * c->L * c->N, (int64_t)cnt * c->L, c->N, limbmap_q(c)));
+            if (encode_fused_available(c)) {
+                RET(launch_encode_rows_fused(c, rows_dev + blk * n * dim, rows_here, dim, p0, cnt, pt, ws));
+                RET(launch_ntt_fwd_pass_b(c, pt + (int64_t)p0 * c->L * c->N, (int64_t)cnt * c->L, c->N, limbmap_q(c)));
+            } else {
+                RET(launch_encode_rows(c, rows_dev + blk * n * dim, rows_here, dim, p0, cnt, pt, ws));
+                RET(launch_ntt_fwd(c, pt + (int64_t)p0 * c->L * c->N, (int64_t)cnt * c->L, c->N, limbmap_q(c)));
+            }
         }
     }
     return HANN_OK;

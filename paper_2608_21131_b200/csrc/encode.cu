@@ -171,3 +171,274 @@ int launch_encode_slots(hann_ctx* c, const double* z_dev, u64* poly_out, void* w
     A.out = poly_out;
     return run_encode(c, A, 1);
 }
+
+// =====================================================================================================================
+// Fused path (rings with N >= 2^9 whose ciphertext primes are all below 2^50).
+//
+// Kernel W runs the FFT stages 1..8 (contiguous chunks of 256 points) in two register rounds of four stages; its
+// twiddles T[t * n / 2^s] are the same 255 values for every chunk and plaintext and live in shared memory.
+// Kernel X owns 16 adjacent columns of one plaintext: it finishes the FFT (the a-1 strided stages, a = logN - 8),
+// twists, scales and rounds, and then -- because coefficient k and coefficient k + n are the real and imaginary part of
+// the same FFT output -- already holds, per thread, exactly the words the first register round of the forward
+// transform's pass A needs.  It runs pass A for every ciphertext prime from those registers and writes the pass-A
+// output (binary64 residues) to the plaintext buffer; pass B is the stock kernel.  The integer coefficients never
+// travel to HBM, and the operations and their order are those of the two-kernel path, so the results are bit-identical.
+#include "nttcore.cuh"
+
+namespace {
+
+struct FusedArgs {
+    const float* rows;
+    long long rows_in_block;
+    int dim, R, B, p_first;
+    const double2* T;
+    const double2* U;
+    const int32_t* jinv;
+    int logn, L;
+    double scale;
+    double2* buf;        // [count][n]
+    u64* out;            // [..][L][N]
+    const double2* tw;   // forward transform twiddles, binary64 format, [L+1][N]
+    const LimbConst* lt;
+};
+
+__device__ __forceinline__ void dit(double2& x, double2& y, double2 w) {
+    const double2 v = cmul_rn(y, w);
+    y = make_double2(__dsub_rn(x.x, v.x), __dsub_rn(x.y, v.y));
+    x = make_double2(__dadd_rn(x.x, v.x), __dadd_rn(x.y, v.y));
+}
+
+constexpr int kWChunks = 8;  // chunks of 256 points per CTA of kernel W (128 threads)
+
+__global__ void __launch_bounds__(128) k_fft_w(FusedArgs A) {
+    __shared__ double2 tc[256];                    // tc[h - 1 + t] = T[t * n / (2h)], h = 1, 2, .., 128
+    __shared__ double2 sm[kWChunks * (256 + 16)];  // padded chunk: position pos lives at pos + pos/16
+    const int n = 1 << A.logn;
+    const int P = blockIdx.y;
+    const int g = (A.p_first + P) / A.B, b = (A.p_first + P) % A.B;
+    for (int i = threadIdx.x; i < 255; i += 128) {
+        const int s = 32 - __clz(i + 1);  // stage 1..8: h = 2^(s-1), entries h-1 .. 2h-2
+        const int h = 1 << (s - 1), t = i - (h - 1);
+        tc[i] = A.T[(long long)t << (A.logn - s)];
+    }
+    __syncthreads();
+    const int chunk0 = blockIdx.x * kWChunks;
+    // round 1: stages 1..4 on 16 consecutive positions
+    {
+        const int ch = threadIdx.x >> 4, j = threadIdx.x & 15;
+        const int pos0 = ((chunk0 + ch) << 8) + (j << 4);
+        double2 x[16];
+#pragma unroll
+        for (int e = 0; e < 16; e++) {
+            const int u = (int)(__brev((unsigned)(pos0 + e)) >> (32 - A.logn));
+            const int jj = A.jinv[u];
+            int row = jj - g * A.B;
+            if (row < 0) row += n;
+            const int col = (jj + b) % A.R;
+            const double v = (row < A.rows_in_block && col < A.dim) ? (double)A.rows[(long long)row * A.dim + col] : 0.0;
+            x[e] = make_double2(v, 0.0);
+        }
+#pragma unroll
+        for (int s = 0; s < 4; s++) {
+            const int span = 1 << s;
+#pragma unroll
+            for (int e = 0; e < 16; e++)
+                if (!(e & span)) dit(x[e], x[e + span], tc[span - 1 + (e & (span - 1))]);
+        }
+        double2* d = sm + ch * 272 + 17 * j;
+#pragma unroll
+        for (int e = 0; e < 16; e++) d[e] = x[e];
+    }
+    __syncthreads();
+    // round 2: stages 5..8 on positions j + 16 e
+    {
+        const int ch = threadIdx.x >> 4, j = threadIdx.x & 15;
+        double2 x[16];
+#pragma unroll
+        for (int e = 0; e < 16; e++) x[e] = sm[ch * 272 + 17 * e + j];
+#pragma unroll
+        for (int s = 0; s < 4; s++) {
+            const int span = 1 << s;  // in units of 16 positions
+#pragma unroll
+            for (int e = 0; e < 16; e++)
+                if (!(e & span)) dit(x[e], x[e + span], tc[16 * span - 1 + j + 16 * (e & (span - 1))]);
+        }
+        double2* o = A.buf + (long long)P * n + ((long long)(chunk0 + ch) << 8) + j;
+#pragma unroll
+        for (int e = 0; e < 16; e++) o[16 * e] = x[e];
+    }
+}
+
+// R1 + R2 = a = logN - 8 are the register rounds of the transform's pass A (R1 = min(a, 4)); the FFT's a - 1 strided
+// stages run as a first round of R2 stages and a last round of R1 - 1 stages
+template <int R1, int R2>
+__global__ void __launch_bounds__(256, 2) k_encode_x(FusedArgs A) {
+    extern __shared__ u64 smx[];
+    constexpr int a = R1 + R2;
+    constexpr int G1 = 1 << R2;        // row groups of transform round 1 = threads per column
+    constexpr int HF = 1 << (R1 - 1);  // complex words a thread holds after the FFT's last round
+    constexpr int rows_fft = 1 << (a - 1);
+    const int n = 1 << A.logn, N = 2 * n;
+    const int P = blockIdx.y;
+    const int c0 = blockIdx.x << 4;
+    const double2* in = A.buf + (long long)P * n + c0;
+    double2* smc = (double2*)smx;  // [rows_fft][16]
+    if (R2 > 0) {
+        // FFT round of R2 stages: rows gg*2^R2 + e, spans 1 .. 2^(R2-1) rows
+        constexpr int E = 1 << (R2 == 0 ? 1 : R2);
+        for (int w = threadIdx.x; w < (rows_fft >> R2) * 16; w += blockDim.x) {
+            const int c = w & 15, gg = w >> 4;
+            double2 x[E];
+#pragma unroll
+            for (int e = 0; e < E; e++) x[e] = in[(long long)((gg << R2) + e) * 256 + c];
+#pragma unroll
+            for (int t = 0; t < R2; t++) {
+                const int span = 1 << t;
+#pragma unroll
+                for (int e = 0; e < E; e++)
+                    if (!(e & span)) {
+                        const int tr = e & (span - 1);
+                        dit(x[e], x[e + span], A.T[(long long)(tr * 256 + c0 + c) << (a - 2 - t)]);
+                    }
+            }
+#pragma unroll
+            for (int e = 0; e < E; e++) smc[(((gg << R2) + e) << 4) + c] = x[e];
+        }
+        __syncthreads();
+    }
+    // FFT last round (R1 - 1 stages) on rows g + G1*e, then twist, scale, round: one thread per (column, g)
+    double m[1 << R1];  // rounded coefficients: rows g + G1*e, e < 2^R1 (second half = imaginary parts)
+    const int c = threadIdx.x & 15, g = threadIdx.x >> 4;
+    const bool active = g < G1;
+    if (active) {
+        double2 x[HF];
+#pragma unroll
+        for (int e = 0; e < HF; e++) x[e] = R2 > 0 ? smc[((g + G1 * e) << 4) + c] : in[(long long)(g + G1 * e) * 256 + c];
+#pragma unroll
+        for (int u = 0; u < R1 - 1; u++) {
+            const int span = 1 << u, t = R2 + u;
+#pragma unroll
+            for (int e = 0; e < HF; e++)
+                if (!(e & span)) {
+                    const int tr = g + G1 * (e & (span - 1));
+                    dit(x[e], x[e + span], A.T[(long long)(tr * 256 + c0 + c) << (a - 2 - t)]);
+                }
+        }
+#pragma unroll
+        for (int e = 0; e < HF; e++) {
+            const int k = (g + G1 * e) * 256 + c0 + c;
+            const double2 cc = cmul_rn(x[e], A.U[k]);
+            m[e] = rint(__dmul_rn(cc.x, A.scale));
+            m[e + HF] = rint(__dmul_rn(cc.y, A.scale));
+        }
+    }
+    // pass A of the forward transform for every ciphertext prime, from the registers
+    constexpr int RR2 = R2 == 0 ? 1 : R2;
+    constexpr int G2 = 1 << R1;
+    for (int l = 0; l < A.L; l++) {
+        const ArithF64 ar(A.lt + l);
+        const double2* tw = A.tw + ((size_t)l << (A.logn + 1));
+        u64* base = A.out + ((long long)(A.p_first + P) * A.L + l) * N + c0;
+        if (R2 > 0) __syncthreads();  // the exchange tile is free again
+        if (active) {
+            double x[1 << R1];
+#pragma unroll
+            for (int e = 0; e < (1 << R1); e++) x[e] = ar.reduce(m[e]);
+            fwd_round<R1>(ar, x, tw, 1u);
+#pragma unroll
+            for (int e = 0; e < (1 << R1); e++) {
+                if (R2 == 0) base[(size_t)(g + G1 * e) * 256 + c] = ar.to_mid(x[e]);
+                else smx[((g + G1 * e) << 4) + c] = ar.to_mid(x[e]);
+            }
+        }
+        if (R2 > 0) {
+            __syncthreads();
+            for (int w = threadIdx.x; w < (G2 << 4); w += blockDim.x) {
+                const int cc = w & 15, gg = w >> 4;
+                double x[1 << RR2];
+#pragma unroll
+                for (int e = 0; e < (1 << RR2); e++) x[e] = ar.from_mid(smx[(((gg << RR2) + e) << 4) + cc]);
+                fwd_round<RR2>(ar, x, tw, (unsigned)(G2 + gg));
+#pragma unroll
+                for (int e = 0; e < (1 << RR2); e++) base[(size_t)((gg << RR2) + e) * 256 + cc] = ar.to_mid(x[e]);
+            }
+        }
+    }
+}
+
+typedef void (*KernX)(FusedArgs);
+KernX pick_x(int a) {
+    switch (a) {
+        case 1: return k_encode_x<1, 0>;
+        case 2: return k_encode_x<2, 0>;
+        case 3: return k_encode_x<3, 0>;
+        case 4: return k_encode_x<4, 0>;
+        case 5: return k_encode_x<4, 1>;
+        case 6: return k_encode_x<4, 2>;
+        case 7: return k_encode_x<4, 3>;
+        default: return k_encode_x<4, 4>;
+    }
+}
+
+}  // namespace
+
+bool encode_fused_available(const hann_ctx* c) {
+    if (c->logN < 9) return false;
+    for (int l = 0; l < c->L; l++)
+        if (c->mod[l] >= (1ULL << 50)) return false;
+    return true;
+}
+
+// plaintexts p_first .. p_first+count-1 of one block: encode and run pass A of their forward transforms; the caller
+// finishes with launch_ntt_fwd_pass_b over the same polynomials
+int launch_encode_rows_fused(hann_ctx* c, const float* rows, int64_t rows_in_block, int dim, int p_first, int count, u64* pt_block,
+                             void* ws) {
+    FusedArgs A;
+    A.rows = rows;
+    A.rows_in_block = rows_in_block;
+    A.dim = dim;
+    A.R = c->R;
+    A.B = c->B;
+    A.p_first = p_first;
+    A.T = c->fft_T;
+    A.U = c->fft_U;
+    A.jinv = c->jinv;
+    A.logn = c->logN - 1;
+    A.L = c->L;
+    A.scale = ldexp(1.0, c->prm.log_scale - A.logn);
+    A.buf = (double2*)ws;
+    A.out = pt_block;
+    A.tw = (const double2*)c->tw_fwd_f64;
+    A.lt = c->lt_dev;
+    const int n = c->n, a = c->logN - 8;
+    const int chunks = n >> 8;  // >= 1 because logN >= 9
+    if (chunks % kWChunks == 0) {
+        KProf kp(c, KC_FFT_A);
+        k_fft_w<<<dim3(chunks / kWChunks, count), 128, 0, c->stream>>>(A);
+    } else {
+        // small rings: the stock first-pass kernel produces the same buffer
+        EncArgs E = {};
+        E.rows = rows;
+        E.rows_in_block = rows_in_block;
+        E.dim = dim;
+        E.buf = (double2*)ws;
+        E.p_first = p_first;
+        E.T = c->fft_T;
+        E.U = c->fft_U;
+        E.jinv = c->jinv;
+        E.logn = A.logn;
+        E.b1 = 8;
+        E.K1 = chunks < 8 ? chunks : 8;
+        E.R = c->R;
+        E.B = c->B;
+        KProf kp(c, KC_FFT_A);
+        k_fft_a<<<dim3(chunks / E.K1, count), kThreads, (size_t)E.K1 * 256 * sizeof(double2), c->stream>>>(E);
+    }
+    {
+        const size_t smem = a > 4 ? (size_t)(1 << a) * 16 * 8 : 0;  // FFT tile (2^(a-1) x 16 complex) = transform tile (2^a x 16 words)
+        KProf kp(c, KC_FFT_B);
+        const int threads = a >= 8 ? 256 : (a == 7 ? 128 : 64);  // 16 columns x 2^R2 row groups, at least two warps
+        pick_x(a)<<<dim3(16, count), threads, smem, c->stream>>>(A);
+    }
+    return check_launch(c, "encode_fused");
+}

@@ -102,6 +102,11 @@ int check_launch(hann_ctx* c, const char* what);
 // transforms of npoly polynomials; polynomial p starts at data + p*stride and uses modulus lm.limb[p % lm.period]
 int launch_ntt_fwd(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
 int launch_ntt_inv(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
+int launch_ntt_fwd_pass_b(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
+// encode a block and run pass A of the transforms in one kernel when the parameters allow it (returns false if not)
+bool encode_fused_available(const hann_ctx* c);
+int launch_encode_rows_fused(hann_ctx* c, const float* rows, int64_t rows_in_block, int dim, int p_first, int count, u64* pt_block,
+                             void* ws);
 LimbMap limbmap_q(const hann_ctx* c);   // period L: limbs 0..L-1
 LimbMap limbmap_qp(const hann_ctx* c);  // period L+1: limbs 0..L
 LimbMap limbmap_single(int limb);

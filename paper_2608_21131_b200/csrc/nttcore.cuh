@@ -1,0 +1,133 @@
+// Arithmetic policies and register rounds shared by the transform kernels (ntt.cu) and the fused encoder
+// (encode.cu).  See ntt.cu for the description of the three arithmetic classes and their range discipline.
+#pragma once
+#include "modarith.cuh"
+
+#ifndef HANN_F64_MINBLOCKS
+#define HANN_F64_MINBLOCKS 2
+#endif
+#ifndef HANN_NTT_MINBLOCKS
+#define HANN_NTT_MINBLOCKS 2
+#endif
+
+// ---- arithmetic policies ---------------------------------------------------------------------------------------
+
+struct ArithF64 {
+    typedef double T;
+    typedef double2 TW;
+    double q, qinv, half;
+    static constexpr int kMinBlocks = HANN_F64_MINBLOCKS;
+    TW ninv;
+    __device__ __forceinline__ ArithF64(const LimbConst* lc)
+        : q((double)lc->q), qinv(1.0 / (double)lc->q), half((double)lc->half), ninv(make_double2(lc->ninv_bal, lc->ninv_q)) {}
+    __device__ __forceinline__ T reduce(T x) const { return __fma_rn(-rint(__dmul_rn(x, qinv)), q, x); }
+    __device__ __forceinline__ T mulmod(T y, TW w) const {
+        const double h = __dmul_rn(y, w.x);
+        const double l = __fma_rn(y, w.x, -h);
+        const double c = rint(__dmul_rn(y, w.y));
+        return __dadd_rn(__fma_rn(-c, q, h), l);
+    }
+    __device__ __forceinline__ T from_canonical(u64 v) const { return __ull2double_rn(v); }
+    __device__ __forceinline__ T from_mid(u64 v) const { return __longlong_as_double((long long)v); }
+    __device__ __forceinline__ u64 to_mid(T x) const { return (u64)__double_as_longlong(reduce(x)); }
+    __device__ __forceinline__ u64 to_canonical(T x) const {
+        x = reduce(x);
+        if (x < 0.0) x += q;
+        return __double2ull_rn(x);
+    }
+    __device__ __forceinline__ void fwd(T& X, T& Y, TW w) const {
+        const T t = mulmod(Y, w);
+        Y = __dsub_rn(X, t);
+        X = __dadd_rn(X, t);
+    }
+    __device__ __forceinline__ void inv(T& X, T& Y, TW w) const {
+        const T d = __dsub_rn(X, Y);
+        X = __dadd_rn(X, Y);
+        Y = mulmod(d, w);
+    }
+    // inverse transforms start from balanced values so that four doubling stages stay below 2^53
+    __device__ __forceinline__ T inv_input(u64 v) const {
+        const double x = __ull2double_rn(v);
+        return x > half ? x - q : x;
+    }
+    __device__ __forceinline__ u64 scaled_output(T x, TW ninv_pair) const { return to_canonical(mulmod(reduce(x), ninv_pair)); }
+};
+
+template <bool SMALLQ>
+struct ArithInt {
+    typedef u64 T;
+    typedef ulonglong2 TW;
+    u64 q, q2;
+    static constexpr int kMinBlocks = HANN_NTT_MINBLOCKS;
+    TW ninv;
+    __device__ __forceinline__ ArithInt(const LimbConst* lc) : q(lc->q), q2(2 * lc->q), ninv(make_ulonglong2(lc->ninv, lc->ninv_s)) {}
+    __device__ __forceinline__ T from_canonical(u64 v) const { return v; }
+    __device__ __forceinline__ T from_mid(u64 v) const { return v; }
+    __device__ __forceinline__ u64 to_mid(T x) const { return x; }
+    __device__ __forceinline__ u64 to_canonical(T v) const {  // forward results: [0, 33q) or [0, 4q)
+        if (SMALLQ) {
+            v = csub(v, 32 * q);
+            v = csub(v, 16 * q);
+            v = csub(v, 8 * q);
+            v = csub(v, 4 * q);
+        }
+        v = csub(v, q2);
+        return csub(v, q);
+    }
+    __device__ __forceinline__ void fwd(T& X, T& Y, TW w) const {
+        u64 x = X;
+        if (!SMALLQ) x = csub(x, q2);
+        const u64 t = shoup_mul(Y, w.x, w.y, q);
+        X = x + t;
+        Y = x - t + q2;
+    }
+    __device__ __forceinline__ void inv(T& X, T& Y, TW w) const {  // [0, 2q) in and out
+        const u64 x = X, y = Y;
+        X = csub(x + y, q2);
+        Y = shoup_mul(x - y + q2, w.x, w.y, q);
+    }
+    __device__ __forceinline__ T inv_input(u64 v) const { return v; }
+    __device__ __forceinline__ u64 scaled_output(T x, TW ninv_pair) const { return csub(shoup_mul(x, ninv_pair.x, ninv_pair.y, q), q); }
+};
+
+// ---- register rounds -----------------------------------------------------------------------------------------
+
+template <int R, class AR>
+__device__ __forceinline__ void fwd_round(const AR& ar, typename AR::T (&x)[1 << R], const typename AR::TW* __restrict__ tw,
+                                          unsigned base) {
+#pragma unroll
+    for (int s = 0; s < R; s++) {
+        const int span = 1 << (R - 1 - s);
+#pragma unroll
+        for (int il = 0; il < (1 << s); il++) {
+            const typename AR::TW w = tw[(base << s) + il];
+#pragma unroll
+            for (int jj = 0; jj < span; jj++) {
+                const int e = il * 2 * span + jj;
+                ar.fwd(x[e], x[e + span], w);
+            }
+        }
+    }
+}
+
+template <int R, class AR>
+__device__ __forceinline__ void inv_round(const AR& ar, typename AR::T (&x)[1 << R], const typename AR::TW* __restrict__ tw,
+                                          unsigned base) {
+#pragma unroll
+    for (int s = 0; s < R; s++) {
+        const int span = 1 << s;
+#pragma unroll
+        for (int il = 0; il < (1 << (R - 1 - s)); il++) {
+            const typename AR::TW w = tw[(base << (R - 1 - s)) + il];
+#pragma unroll
+            for (int jj = 0; jj < span; jj++) {
+                const int e = il * 2 * span + jj;
+                ar.inv(x[e], x[e + span], w);
+            }
+        }
+    }
+}
+
+template <int R2>
+__device__ __forceinline__ int pad(int pos) { return R2 == 0 ? pos : pos + (pos >> R2); }
+

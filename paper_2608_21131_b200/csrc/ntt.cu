@@ -160,6 +160,75 @@ __global__ void __launch_bounds__(kThreads, AR::kMinBlocks) k_ntt_fwd_b(NttArgs 
     fwd_b_body<R1, R2>(A, ar, base, chunk0, (const typename AR::TW*)A.tw + ((size_t)sel.limb << A.logN), sm);
 }
 
+// Forward pass B for rings of at least 2^9 points (chunks of 256 words, two rounds of four stages).  A CTA takes kBK
+// chunks of kBPG polynomials that share their modulus (same position in consecutive limb periods): the 255 twiddle pairs
+// of each chunk are staged in shared memory once and serve all kBPG polynomials, which cuts the table traffic (two
+// table bytes per data byte otherwise) and keeps the twiddles out of the register file.
+constexpr int kBK = 4, kBPG = 4;
+#ifndef HANN_B8_MINBLOCKS
+#define HANN_B8_MINBLOCKS 3
+#endif
+
+template <class AR>
+__global__ void __launch_bounds__(256, HANN_B8_MINBLOCKS) k_ntt_fwd_b8(NttArgs A, int groups) {
+    extern __shared__ u64 smraw[];
+    typedef typename AR::TW TW;
+    TW* tc = (TW*)smraw;                 // [kBK][256]: entry e of chunk ch = pass stage s, group il with e + 1 = 2^s + il
+    u64* sm = smraw + kBK * 256 * 2;     // [kBPG][kBK][272] padded chunks
+    const int y = blockIdx.y, k = y % A.nsel, yg = y / A.nsel;
+    const int pos = (int)((A.pos4 >> (4 * k)) & 15), limb = (int)((A.limb4 >> (4 * k)) & 15);
+    const AR ar(A.lt + limb);
+    const int chunk0 = blockIdx.x * kBK;
+    const TW* tw = (const TW*)A.tw + ((size_t)limb << A.logN);
+    const unsigned m0 = 1u << A.a;
+    const int t = threadIdx.x >> 6, ch = (threadIdx.x >> 4) & 3, j = threadIdx.x & 15;
+    const long long group = (long long)yg * kBPG + t;
+    const bool valid = group < groups;
+    u64* base = A.data + (group * A.period + pos) * A.stride + ((size_t)(chunk0 + ch) << 8);
+    // the data loads go out first so that they overlap the staging of the twiddles
+    u64 raw[16];
+    if (valid) {
+#pragma unroll
+        for (int e = 0; e < 16; e++) raw[e] = base[j + 16 * e];
+    }
+    for (int i = threadIdx.x; i < kBK * 256; i += 256) {
+        const int c2 = i >> 8, e = i & 255;
+        if (e < 255) {
+            const int st = 31 - __clz(e + 1), il = e + 1 - (1 << st);
+            tc[i] = tw[((m0 + (unsigned)(chunk0 + c2)) << st) + il];
+        }
+    }
+    __syncthreads();
+    const TW* tcc = tc + ch * 256 - 1;
+    u64* s1 = sm + (t * kBK + ch) * 272;
+    if (valid) {
+        typename AR::T x[16];
+#pragma unroll
+        for (int e = 0; e < 16; e++) x[e] = ar.from_mid(raw[e]);
+        fwd_round<4>(ar, x, tcc, 1u);
+#pragma unroll
+        for (int e = 0; e < 16; e++) s1[17 * e + j] = ar.to_mid(x[e]);
+    }
+    __syncthreads();
+    if (valid) {
+        typename AR::T x[16];
+#pragma unroll
+        for (int e = 0; e < 16; e++) x[e] = ar.from_mid(s1[17 * j + e]);
+        fwd_round<4>(ar, x, tcc, 16u + (unsigned)j);
+#pragma unroll
+        for (int e = 0; e < 16; e++) s1[17 * j + e] = ar.to_canonical(x[e]);
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < kBPG * kBK * 256; idx += 256) {
+        const int t2 = idx >> 10, rem = idx & 1023;
+        const long long g2 = (long long)yg * kBPG + t2;
+        if (g2 < groups) {
+            const int p = rem & 255;
+            A.data[(g2 * A.period + pos) * A.stride + ((size_t)chunk0 << 8) + rem] = sm[(t2 * kBK + (rem >> 8)) * 272 + p + (p >> 4)];
+        }
+    }
+}
+
 // ---- inverse pass B': spans 1 .. S/2 inside contiguous chunks (mirror of forward pass B) -----------------------
 
 template <int R1, int R2, class AR>
@@ -295,6 +364,12 @@ void launch_fwd_class(hann_ctx* c, const NttArgs& A, int groups, bool skip_a) {
         pick_fwd_a<AR>(A.a)<<<dim3(1 << (A.b - A.logC), groups * A.nsel), kThreads, smem_a(A), c->stream>>>(A);
     }
     KProf kp(c, KC_NTT_FWD_B);
+    if (A.b == 8 && A.a > 0 && ((c->N >> 8) % kBK) == 0) {
+        const size_t smem = (size_t)kBK * 256 * 16 + (size_t)kBPG * kBK * 272 * 8;
+        cudaFuncSetAttribute(k_ntt_fwd_b8<AR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  // 50 KiB > default 48
+        k_ntt_fwd_b8<AR><<<dim3((c->N >> 8) / kBK, ((groups + kBPG - 1) / kBPG) * A.nsel), 256, smem, c->stream>>>(A, groups);
+        return;
+    }
     pick_fwd_b<AR>(A.b)<<<dim3((c->N >> A.b) / A.K, groups * A.nsel), kThreads, smem_b(A), c->stream>>>(A);
 }
 

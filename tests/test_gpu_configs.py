@@ -1,0 +1,147 @@
+"""The benchmark configurations at their full sizes, in the launch configuration bench.py times (whole levels per
+call): bit-exact conformance against the CPU oracle on the first and last block of a level, the score tolerance on every
+scored row, and agreement of the FHE-steered routing with plaintext routing (same top-10 ids, same planted-neighbour
+hit) on the synthetic hierarchies."""
+import numpy as np
+import pytest
+
+from paper_2608_21131_b200 import synth, workloads as wl
+from tests.helpers import Pair
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def pair16():
+    return Pair(synth.FULL16, key_seed=wl.KEY_SEED)
+
+
+class Query:
+    """one encrypted query on both sides; the baby set is prepared once and reused by every level"""
+
+    def __init__(self, p, qR, with_oracle=True):
+        import torch
+
+        self.p, self.qR, self.torch = p, qR, torch
+        ct_o, ct_g = p.query(qR)
+        assert np.array_equal(ct_o, ct_g)
+        self.ct_o = ct_o
+        self.baby = p.g.query_prepare(p.g.import_(p.b.KIND_CT, ct_g, 1), p.ws)
+        self.baby_o = p.o.baby_set(ct_o, p.evk_o) if with_oracle else None
+
+    def score_level(self, rows, oracle_blocks=()):
+        """GPU scores of a level [n_rows]; blocks listed in oracle_blocks are compared bit for bit with the oracle"""
+        p, g, b, ps = self.p, self.p.g, self.p.b, self.p.ps
+        n_rows = rows.shape[0]
+        nb = g.n_blocks(n_rows)
+        ws = g.workspace(nb)
+        pt = g.encode_candidates(self.torch.from_numpy(np.ascontiguousarray(rows)).to(g.device), ws)
+        inner = g.score_level(self.baby, pt, nb, ws)
+        score = g.rotate_sum(inner, nb, ws)
+        g.sync()
+        score_h = g.export(b.KIND_CT, score, nb)
+        for blk in oracle_blocks:
+            sc_o, pt_o, in_o = p.o.score_block(rows[blk * ps.n:(blk + 1) * ps.n], self.baby_o, p.evk_o[ps.B - 1], True, True)
+            ptw, inw = g.sizeof(b.SIZE_PT_BLOCK), g.sizeof(b.SIZE_INNER)
+            pt_g = g.export(b.KIND_PT, pt, ps.R, offset_bytes=blk * ptw).reshape(ps.G, ps.B, ps.L, ps.N)
+            in_g = g.export(b.KIND_CT, inner, ps.G, offset_bytes=blk * inw).reshape(ps.G, 2, ps.L, ps.N)
+            assert np.array_equal(pt_g, pt_o), "encoded plaintexts of block %d" % blk
+            assert np.array_equal(in_g, in_o), "partial sums of block %d" % blk
+            assert np.array_equal(score_h[blk], sc_o), "score ciphertext of block %d" % blk
+        got = g.decrypt_scores(p.km.s, score_h).reshape(-1)[:n_rows]
+        want = rows.astype(np.float64) @ self.qR.astype(np.float64)
+        err = float(np.abs(got - want).max())
+        assert err < 2.0 ** ps.tol_log2, err
+        del pt, inner, score
+        return got, want
+
+
+def test_face_like_level_full(pair16):
+    """222,049 rows, 512 -> 128 dims, N = 2^16: 7 blocks, the last 77.6 % full.  First and last block at every
+    conformance point, every row within 2^-18."""
+    ps, lvl, qR, planted = wl.face_level()
+    q = Query(pair16, qR)
+    got, want = q.score_level(lvl.rows, oracle_blocks=(0, 6))
+    assert got.shape == (222_049,)
+    # the planted neighbour is the top score under both rankings
+    assert int(np.argmax(got)) == planted == int(np.argmax(want))
+    assert np.array_equal(wl.topk_ids(got, lvl.ids, 10), wl.topk_ids(want, lvl.ids, 10))
+
+
+def route(cfg, q, scorer):
+    """coarse -> fine -> rerank with the given scorer(level) -> scores; returns (top-10 row ids, touched rows)"""
+    coarse = wl.coarse_level(cfg) if not hasattr(cfg, "_coarse") else cfg._coarse
+    cfg._coarse = coarse
+    cells = wl.topk_ids(scorer(coarse), coarse.ids, cfg.nprobe)
+    fine = wl.fine_level(cfg, np.sort(cells))
+    leaves = wl.topk_ids(scorer(fine), fine.ids, cfg.leaf_beam)
+    rer = wl.rerank_level(cfg, np.sort(leaves))
+    sc = scorer(rer)
+    return wl.topk_ids(sc, rer.ids, 10), (coarse, fine, rer), sc
+
+
+def same_up_to_near_ties(ids_a, ids_b, scores_by_id, tol):
+    if np.array_equal(ids_a, ids_b):
+        return True
+    # differences are allowed only between scores closer than 2 * tol
+    sa = np.array([scores_by_id[i] for i in ids_a])
+    sb = np.array([scores_by_id[i] for i in ids_b])
+    return set(ids_a) == set(ids_b) or bool(np.abs(np.sort(sa) - np.sort(sb)).max() < 2 * tol)
+
+
+@pytest.mark.parametrize("name,n_queries", [("datacomp", 2), ("deep1b", 3)])
+def test_hierarchy_routing_agrees_with_plaintext(pair16, name, n_queries):
+    cfg = wl.datacomp_like() if name == "datacomp" else wl.deep1b_like()
+    ps = cfg.ps
+    for qi in range(n_queries):
+        qR, planted = wl.hier_query(cfg, qi)
+        q = Query(pair16, qR, with_oracle=(qi == 0))
+
+        def fhe(level):
+            nb = (len(level.ids) + ps.n - 1) // ps.n
+            # first query: first and last block of every level against the oracle
+            blocks = sorted({0, nb - 1}) if qi == 0 else ()
+            return q.score_level(level.rows, oracle_blocks=blocks)[0]
+
+        def plain(level):
+            return level.rows.astype(np.float64) @ qR.astype(np.float64)
+
+        top_f, levels_f, sc_f = route(cfg, q, fhe)
+        top_p, levels_p, sc_p = route(cfg, q, plain)
+        # both pipelines open the same cells and return the same neighbours
+        assert np.array_equal(levels_f[1].ids, levels_p[1].ids) and np.array_equal(levels_f[2].ids, levels_p[2].ids)
+        by_id = dict(zip(levels_p[2].ids.tolist(), sc_p.tolist()))
+        assert same_up_to_near_ties(top_f, top_p, by_id, 2.0 ** ps.tol_log2)
+        assert (planted in top_f) == (planted in top_p)
+        assert planted == top_p[0]  # the perturbed copy's nearest row is the planted row (recall@1 of the routing)
+        if name == "datacomp" and qi == 0:
+            assert len(levels_f[0].ids) == 65_536 and len(levels_f[1].ids) == 1_024 and len(levels_f[2].ids) == 97_976
+        if name == "deep1b" and qi == 0:
+            assert len(levels_f[0].ids) == 1_000 and len(levels_f[1].ids) == 16_000 and len(levels_f[2].ids) == 64_000
+
+
+def test_zero_padded_96_dim_rows_score_identically_on_gpu(pair16):
+    """the 96 -> 128 zero-pad: rows given with dim = 96 and the same rows padded to 128 by the caller give the same bits"""
+    import torch
+
+    p = pair16
+    g, b, ps = p.g, p.b, p.ps
+    x96 = synth.toy_corpus(3, rows=5000, dim=96)
+    x128 = synth.project_rows(x96.astype(np.float64), None, 128)
+    pt_a = g.encode_candidates(torch.from_numpy(x96).to(g.device), p.ws)
+    pt_b = g.encode_candidates(torch.from_numpy(x128).to(g.device), p.ws)
+    g.sync()
+    assert torch.equal(pt_a, pt_b)
+
+
+@pytest.mark.parametrize("logN", [15, 16])
+def test_sweep_level_with_padding_groups(logN, pair16):
+    """scaling-sweep configuration at its smallest size: 2^12 wanted rows inflated x4 by seeded fixed groups to 2^14
+    scored rows (one block at N = 2^15, half a block at N = 2^16), dim 128"""
+    ps = synth.FULL15 if logN == 15 else synth.FULL16
+    ps2, lvl = wl.sweep_level(1 << 12, ps=ps)
+    assert lvl.rows.shape == (1 << 14, 128)
+    p = pair16 if logN == 16 else Pair(ps, key_seed=wl.KEY_SEED)
+    qR = synth.toy_query(wl.query_seed(0), dim=128)
+    q = Query(p, qR)
+    q.score_level(lvl.rows, oracle_blocks=(0,))

@@ -180,6 +180,14 @@ int hann_score_level(hann_ctx *ctx, const void *baby_dev, const void *pt_dev, in
  *   score_ct_dev n_blocks * HANN_SIZE_CT bytes (device), internal layout. */
 int hann_rotate_sum(hann_ctx *ctx, const void *inner_dev, int64_t n_blocks, void *score_ct_dev, void *ws, size_t ws_bytes);
 
+/* One routing level for one query, device buffers in and out: hann_query_prepare, hann_encode_candidates,
+ * hann_score_level and hann_rotate_sum in sequence, except that the query preparation runs on a helper stream beside
+ * the candidate encoding (they are independent; both finish before the multiply-accumulate starts).  All buffers as in
+ * the four calls; `ws` must hold hann_workspace_bytes(ctx, blocks).  On return everything is enqueued on the context's
+ * stream again (the helper stream is joined). */
+int hann_query_level(hann_ctx *ctx, const void *ct_dev, const float *rows_dev, int64_t n_rows, int dim, void *baby_dev,
+                     void *pt_dev, void *inner_dev, void *score_ct_dev, void *ws, size_t ws_bytes);
+
 /* Hybrid key switch of one polynomial d (internal layout, L limbs) with the loaded key of rotation `rot`, WITHOUT
  * applying the automorphism to d: outputs (ks0, ks1), L limbs each, with ks0 + ks1*s ~ d*s(X^k).
  * Steps: digits [d]_{q_j} (inverse transform), centred lift into all L+1 moduli, transform, inner product with

@@ -80,6 +80,7 @@ def load_library():
         "hann_score_level": (C.c_int, [vp, vp, vp, i64, vp, vp, sz]),
         "hann_rotate_sum": (C.c_int, [vp, vp, i64, vp, vp, sz]),
         "hann_keyswitch": (C.c_int, [vp, C.c_int, vp, vp, vp, vp, sz]),
+        "hann_query_level": (C.c_int, [vp, vp, vp, i64, C.c_int, vp, vp, vp, vp, vp, sz]),
         "hann_static_scratch_bytes": (i64, []),
         "hann_keyswitch_static": (C.c_int, [vp, C.c_int, vp, vp, vp]),
         "hann_import": (C.c_int, [vp, C.c_int, vp, i64, vp]),
@@ -267,6 +268,17 @@ class Context:
         if score is None:
             score = self.alloc(n_blocks * self.sizeof(SIZE_CT))
         self._ck(self.lib.hann_rotate_sum(self.h, _ptr(inner), n_blocks, _ptr(score), _ptr(ws), ws.numel() * 8))
+        return score
+
+    def query_level(self, ct_dev, rows_dev, ws, baby=None, pt=None, inner=None, score=None):
+        n_rows, dim = rows_dev.shape
+        nb = self.n_blocks(n_rows)
+        baby = self.alloc(self.sizeof(SIZE_BABY)) if baby is None else baby
+        pt = self.alloc(nb * self.sizeof(SIZE_PT_BLOCK)) if pt is None else pt
+        inner = self.alloc(nb * self.sizeof(SIZE_INNER)) if inner is None else inner
+        score = self.alloc(nb * self.sizeof(SIZE_CT)) if score is None else score
+        self._ck(self.lib.hann_query_level(self.h, _ptr(ct_dev), _ptr(rows_dev), n_rows, dim, _ptr(baby), _ptr(pt), _ptr(inner),
+                                           _ptr(score), _ptr(ws), ws.numel() * 8))
         return score
 
     def keyswitch(self, rot, poly, ws):

@@ -31,6 +31,7 @@ def build(force: bool = False, verbose: bool = False, out: str = LIB, extra_flag
     cmd = [
         nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
         "--fmad=false",  # the encode kernels pin every floating-point rounding
+        "--extended-lambda",
         "-Xcompiler", "-fPIC,-O2,-Wall", "-shared", "-o", tmp,
     ]
     if verbose:

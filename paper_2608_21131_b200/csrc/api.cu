@@ -249,6 +249,9 @@ extern "C" int hann_ctx_create(const hann_params* prm, hann_ctx** out) {
             g = (g * 5) % (2L * N);
         }
     }
+    // the FFT runs on bit-reversed input: position pos of its input array takes slot jinv[brev(pos)]
+    std::vector<int32_t> jpos(n);
+    for (int pos = 0; pos < n; pos++) jpos[pos] = jinv[hm::bitrev(pos, c->logN - 1)];
     const size_t twb = (size_t)(L + 1) * N * 16;
     bool ok = cudaMalloc(&c->tw_fwd, twb) == cudaSuccess && cudaMalloc(&c->tw_inv, twb) == cudaSuccess &&
               cudaMalloc(&c->tw_fwd_f64, twb) == cudaSuccess && cudaMalloc(&c->tw_inv_f64, twb) == cudaSuccess &&
@@ -264,7 +267,7 @@ extern "C" int hann_ctx_create(const hann_params* prm, hann_ctx** out) {
              cudaMemcpy(c->lt_dev, &c->lt, sizeof(LimbTable), cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->fft_T, T.data(), nh * sizeof(double2), cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->fft_U, U.data(), n * sizeof(double2), cudaMemcpyHostToDevice) == cudaSuccess &&
-             cudaMemcpy(c->jinv, jinv.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(c->jinv, jpos.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->galois_dev, gal.data(), n * sizeof(unsigned), cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemset(c->keytab_dev, 0, n * sizeof(u64*)) == cudaSuccess;
     }
@@ -272,6 +275,10 @@ extern "C" int hann_ctx_create(const hann_params* prm, hann_ctx** out) {
     c->keytab_host.assign(n, nullptr);
     for (int k = 0; k < HANN_NKINDS && ok; k++)
         ok = cudaEventCreate(&c->ev[k][0]) == cudaSuccess && cudaEventCreate(&c->ev[k][1]) == cudaSuccess;
+    if (ok)
+        ok = cudaStreamCreateWithFlags(&c->aux_stream, cudaStreamNonBlocking) == cudaSuccess &&
+             cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
     if (ok) ok = ntt_configure(c) == HANN_OK;
     if (!ok) {
         cudaGetLastError();
@@ -291,6 +298,12 @@ extern "C" void hann_ctx_destroy(hann_ctx* c) {
     cudaFree(c->tw_fwd); cudaFree(c->tw_inv); cudaFree(c->tw_fwd_f64); cudaFree(c->tw_inv_f64); cudaFree(c->lt_dev);
     cudaFree(c->fft_T); cudaFree(c->fft_U); cudaFree(c->jinv); cudaFree(c->galois_dev); cudaFree(c->keytab_dev);
     if (c->scratch) cudaFree(c->scratch);
+    if (c->aux_stream) {
+        cudaStreamSynchronize(c->aux_stream);
+        cudaStreamDestroy(c->aux_stream);
+    }
+    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+    if (c->ev_join) cudaEventDestroy(c->ev_join);
     for (auto& r : c->krec) {
         if (r.a) cudaEventDestroy(r.a);
         if (r.b) cudaEventDestroy(r.b);
@@ -324,6 +337,8 @@ extern "C" int64_t hann_workspace_bytes(const hann_ctx* c, int64_t max_blocks) {
     int64_t w = std::max(ks_item_words(c) * items, prepare_words(c)) * 8;
     w = std::max(w, (ks_item_words(c) + (int64_t)c->L * c->N) * 8);  // hann_keyswitch permutes its input first
     w = std::max(w, encode_ws_bytes(c));
+    // hann_query_level runs query_prepare and encode_candidates side by side, each in its own part
+    w = std::max(w, align256(prepare_words(c) * 8 + kSlack) + encode_ws_bytes(c));
     return w + kSlack;
 }
 
@@ -729,6 +744,35 @@ extern "C" int hann_keyswitch(hann_ctx* c, int rot, const void* poly_dev, void* 
     return HANN_OK;
 }
 
+extern "C" int hann_query_level(hann_ctx* c, const void* ct_dev, const float* rows_dev, int64_t n_rows, int dim, void* baby_dev,
+                                void* pt_dev, void* inner_dev, void* score_ct_dev, void* ws, size_t ws_bytes) {
+    if (!c) return HANN_EINVAL;
+    if (!ct_dev || !rows_dev || !baby_dev || !pt_dev || !inner_dev || !score_ct_dev || n_rows < 1)
+        return fail(c, HANN_EINVAL, "hann_query_level: bad argument");
+    if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_query_level: workspace missing or not 256-byte aligned");
+    const int64_t prep = c->B > 1 ? align256(prepare_words(c) * 8 + kSlack) : 0;
+    if ((int64_t)ws_bytes < prep + encode_ws_bytes(c)) return fail(c, HANN_EWORKSPACE, "hann_query_level: workspace too small");
+    DeviceGuard dg(c->device);
+    const int64_t nblk = (n_rows + c->n - 1) / c->n;
+    // fork: the baby rotations of the query on the helper stream, the candidate encoding on the context's stream
+    cudaStream_t main_stream = c->stream;
+    CK(cudaEventRecord(c->ev_fork, main_stream));
+    CK(cudaStreamWaitEvent(c->aux_stream, c->ev_fork, 0));
+    c->stream = c->aux_stream;
+    int rc = hann_query_prepare(c, ct_dev, baby_dev, ws, (size_t)prep);
+    c->stream = main_stream;
+    cudaError_t e = cudaEventRecord(c->ev_join, c->aux_stream);
+    if (rc == HANN_OK) rc = hann_encode_candidates(c, rows_dev, n_rows, dim, pt_dev, (char*)ws + prep, ws_bytes - (size_t)prep);
+    // join before anything else is reported, so that the helper stream never runs past this call's buffers unobserved
+    cudaError_t e2 = cudaStreamWaitEvent(main_stream, c->ev_join, 0);
+    RET(rc);
+    CK(e);
+    CK(e2);
+    RET(hann_score_level(c, baby_dev, pt_dev, nblk, inner_dev, ws, ws_bytes));
+    RET(hann_rotate_sum(c, inner_dev, nblk, score_ct_dev, ws, ws_bytes));
+    return HANN_OK;
+}
+
 // ================================================================================================ host-buffer level
 
 namespace {
@@ -777,10 +821,7 @@ extern "C" int hann_score_level_host(hann_ctx* c, const uint64_t* ct_host, const
     void* ws = b;
     CK(cudaMemcpyAsync(rows, rows_host, (size_t)n_rows * dim * 4, cudaMemcpyHostToDevice, c->stream));
     RET(import_polys(c, ct_host, 2, ct));
-    RET(hann_query_prepare(c, ct, baby, ws, (size_t)p.ws));
-    RET(hann_encode_candidates(c, rows, n_rows, dim, pt, ws, (size_t)p.ws));
-    RET(hann_score_level(c, baby, pt, p.nblk, inner, ws, (size_t)p.ws));
-    RET(hann_rotate_sum(c, inner, p.nblk, score, ws, (size_t)p.ws));
+    RET(hann_query_level(c, ct, rows, n_rows, dim, baby, pt, inner, score, ws, (size_t)p.ws));
     RET(export_polys(c, score, p.nblk * 2, stage, score_ct_host));
     CK(cudaStreamSynchronize(c->stream));
     return HANN_OK;

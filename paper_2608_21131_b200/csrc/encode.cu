@@ -47,8 +47,7 @@ __global__ void __launch_bounds__(kThreads) k_fft_a(EncArgs A) {
     const int pos0 = blockIdx.x * K1 * S1;
     for (int idx = threadIdx.x; idx < K1 * S1; idx += kThreads) {
         const int pos = pos0 + idx;
-        const int u = (int)(__brev((unsigned)pos) >> (32 - A.logn));
-        const int j = A.jinv[u];
+        const int j = A.jinv[pos];
         double v;
         if (A.rows) {
             int row = j - g * A.B;
@@ -230,8 +229,7 @@ __global__ void __launch_bounds__(128) k_fft_w(FusedArgs A) {
         double2 x[16];
 #pragma unroll
         for (int e = 0; e < 16; e++) {
-            const int u = (int)(__brev((unsigned)(pos0 + e)) >> (32 - A.logn));
-            const int jj = A.jinv[u];
+            const int jj = A.jinv[pos0 + e];
             int row = jj - g * A.B;
             if (row < 0) row += n;
             const int col = (jj + b) % A.R;
@@ -332,14 +330,21 @@ __global__ void __launch_bounds__(256, 2) k_encode_x(FusedArgs A) {
             m[e + HF] = rint(__dmul_rn(cc.y, A.scale));
         }
     }
-    // pass A of the forward transform for every ciphertext prime, from the registers
+    // pass A of the forward transform for every ciphertext prime, from the registers.  Pass A uses table entries
+    // 1 .. 2^a - 1 of a limb, the same for every column: they are staged in shared memory behind the exchange tile.
     constexpr int RR2 = R2 == 0 ? 1 : R2;
     constexpr int G2 = 1 << R1;
+    constexpr int NT = 1 << a;  // cached twiddle pairs per limb (entry 0 unused)
+    double2* twc = (double2*)(smx + (R2 > 0 ? (size_t)NT * 16 : 0));
+    for (int i = threadIdx.x; i < A.L * NT; i += blockDim.x) {
+        const int l = i / NT, e = i % NT;
+        if (e) twc[i] = A.tw[((size_t)l << (A.logn + 1)) + e];
+    }
     for (int l = 0; l < A.L; l++) {
         const ArithF64 ar(A.lt + l);
-        const double2* tw = A.tw + ((size_t)l << (A.logn + 1));
+        const double2* tw = twc + l * NT;
         u64* base = A.out + ((long long)(A.p_first + P) * A.L + l) * N + c0;
-        if (R2 > 0) __syncthreads();  // the exchange tile is free again
+        __syncthreads();  // the twiddle cache is filled (first limb) / the exchange tile is free again
         if (active) {
             double x[1 << R1];
 #pragma unroll
@@ -435,9 +440,11 @@ int launch_encode_rows_fused(hann_ctx* c, const float* rows, int64_t rows_in_blo
         k_fft_a<<<dim3(chunks / E.K1, count), kThreads, (size_t)E.K1 * 256 * sizeof(double2), c->stream>>>(E);
     }
     {
-        const size_t smem = a > 4 ? (size_t)(1 << a) * 16 * 8 : 0;  // FFT tile (2^(a-1) x 16 complex) = transform tile (2^a x 16 words)
+        // exchange tile (FFT: 2^(a-1) x 16 complex = transform: 2^a x 16 words) when a > 4, then L x 2^a twiddle pairs
+        const size_t smem = (a > 4 ? (size_t)(1 << a) * 16 * 8 : 0) + (size_t)c->L * (1 << a) * 16;
         KProf kp(c, KC_FFT_B);
         const int threads = a >= 8 ? 256 : (a == 7 ? 128 : 64);  // 16 columns x 2^R2 row groups, at least two warps
+        if (smem > 48 * 1024) cudaFuncSetAttribute(pick_x(a), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         pick_x(a)<<<dim3(16, count), threads, smem, c->stream>>>(A);
     }
     return check_launch(c, "encode_fused");

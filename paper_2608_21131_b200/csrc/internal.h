@@ -21,6 +21,9 @@ struct hann_ctx {
     int logN = 0, N = 0, n = 0, L = 0, R = 0, B = 0, G = 0;
     int device = 0;
     cudaStream_t stream = nullptr;
+    // helper stream and events of hann_query_level, which runs the query preparation beside the candidate encoding
+    cudaStream_t aux_stream = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     u64 mod[HANN_MAXL1] = {};  // q_0..q_{L-1}, p
     LimbTable lt = {};
     LimbConst* lt_dev = nullptr;  // device copy of lt.c (the transform kernels read it from memory)
@@ -31,7 +34,7 @@ struct hann_ctx {
     // encode tables on the device
     double2* fft_T = nullptr;  // [n/2] exp(-2 pi i t / n)
     double2* fft_U = nullptr;  // [n]   exp(-i pi k / N)
-    int32_t* jinv = nullptr;   // [n]   jinv[u_j] = j with u_j = (5^j mod 2N - 1)/4
+    int32_t* jinv = nullptr;   // [n]   slot j feeding FFT input position pos: jinv[pos] = j with u_j = brev(pos), u_j = (5^j mod 2N - 1)/4
     unsigned* galois_dev = nullptr;  // [n] 5^r mod 2N
     std::vector<unsigned> h_galois;
     // host copies used by decode

@@ -173,7 +173,10 @@ template <class AR>
 __global__ void __launch_bounds__(256, HANN_B8_MINBLOCKS) k_ntt_fwd_b8(NttArgs A, int groups) {
     extern __shared__ u64 smraw[];
     typedef typename AR::TW TW;
-    TW* tc = (TW*)smraw;                 // [kBK][256]: entry e of chunk ch = pass stage s, group il with e + 1 = 2^s + il
+    // twiddle cache [kBK][256].  Entries 0..14: pass stages 0..3 (e + 1 = 2^s + il; read by all 16 threads of a chunk at
+    // once: broadcast).  Entries 16..255: pass stages 4..7, stored [2^u - 1 + il'][j] so that the 16 threads j of a chunk,
+    // which need group j*2^u + il' of stage 4 + u, read consecutive 16-byte words (no bank conflicts).
+    TW* tc = (TW*)smraw;
     u64* sm = smraw + kBK * 256 * 2;     // [kBPG][kBK][272] padded chunks
     const int y = blockIdx.y, k = y % A.nsel, yg = y / A.nsel;
     const int pos = (int)((A.pos4 >> (4 * k)) & 15), limb = (int)((A.limb4 >> (4 * k)) & 15);
@@ -193,19 +196,23 @@ __global__ void __launch_bounds__(256, HANN_B8_MINBLOCKS) k_ntt_fwd_b8(NttArgs A
     }
     for (int i = threadIdx.x; i < kBK * 256; i += 256) {
         const int c2 = i >> 8, e = i & 255;
-        if (e < 255) {
+        if (e < 15) {
             const int st = 31 - __clz(e + 1), il = e + 1 - (1 << st);
             tc[i] = tw[((m0 + (unsigned)(chunk0 + c2)) << st) + il];
+        } else if (e >= 16) {
+            const int jj = e & 15, r = (e >> 4) - 1;           // r = 2^u - 1 + il'
+            const int u = 31 - __clz(r + 1), il = r + 1 - (1 << u);
+            tc[i] = tw[((m0 + (unsigned)(chunk0 + c2)) << (4 + u)) + (jj << u) + il];
         }
     }
     __syncthreads();
-    const TW* tcc = tc + ch * 256 - 1;
+    const TW* tcc = tc + ch * 256;
     u64* s1 = sm + (t * kBK + ch) * 272;
     if (valid) {
         typename AR::T x[16];
 #pragma unroll
         for (int e = 0; e < 16; e++) x[e] = ar.from_mid(raw[e]);
-        fwd_round<4>(ar, x, tcc, 1u);
+        fwd_round_f<4>(ar, x, [=](int st, int il) { return tcc[(1 << st) - 1 + il]; });
 #pragma unroll
         for (int e = 0; e < 16; e++) s1[17 * e + j] = ar.to_mid(x[e]);
     }
@@ -214,7 +221,7 @@ __global__ void __launch_bounds__(256, HANN_B8_MINBLOCKS) k_ntt_fwd_b8(NttArgs A
         typename AR::T x[16];
 #pragma unroll
         for (int e = 0; e < 16; e++) x[e] = ar.from_mid(s1[17 * j + e]);
-        fwd_round<4>(ar, x, tcc, 16u + (unsigned)j);
+        fwd_round_f<4>(ar, x, [=](int u, int il) { return tcc[(((1 << u) + il) << 4) + j]; });
 #pragma unroll
         for (int e = 0; e < 16; e++) s1[17 * j + e] = ar.to_canonical(x[e]);
     }

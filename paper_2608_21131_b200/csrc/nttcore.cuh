@@ -110,6 +110,25 @@ __device__ __forceinline__ void fwd_round(const AR& ar, typename AR::T (&x)[1 <<
     }
 }
 
+// the same round with the twiddle of (stage s, group il) supplied by a functor (shared-memory caches with their own
+// layout)
+template <int R, class AR, class TWF>
+__device__ __forceinline__ void fwd_round_f(const AR& ar, typename AR::T (&x)[1 << R], const TWF& twf) {
+#pragma unroll
+    for (int s = 0; s < R; s++) {
+        const int span = 1 << (R - 1 - s);
+#pragma unroll
+        for (int il = 0; il < (1 << s); il++) {
+            const typename AR::TW w = twf(s, il);
+#pragma unroll
+            for (int jj = 0; jj < span; jj++) {
+                const int e = il * 2 * span + jj;
+                ar.fwd(x[e], x[e + span], w);
+            }
+        }
+    }
+}
+
 template <int R, class AR>
 __device__ __forceinline__ void inv_round(const AR& ar, typename AR::T (&x)[1 << R], const typename AR::TW* __restrict__ tw,
                                           unsigned base) {

@@ -132,12 +132,25 @@ int upload_secret(hann_ctx* c, const int8_t* s_host, int nlimbs, int8_t* s8, u64
     return launch_ntt_fwd(c, dst, nlimbs, c->N, lm);
 }
 
-// ---- one key switch round on `items` polynomials already in coefficient form ------------------------------
-// c1c[items][L][N] (coefficients of the polynomials to switch, item stride L*N) -> u, lifted; combine is left to
-// the caller because its sources and targets differ between the callers.
+// ---- one key switch round on `items` polynomials ---------------------------------------------------------------
+// c1c[items][L][N] (the polynomials to switch, transform domain, item stride L*N; overwritten) -> u, lifted; combine is
+// left to the caller because its sources and targets differ between the callers.
 int ks_digits_to_lifted(hann_ctx* c, u64* c1c, int64_t items, u64* digits, int64_t digit_stride, int rot0, int rot_inc,
                         int64_t u_items, u64* u, u64* lifted) {
     const int L = c->L, N = c->N;
+    if (ks_lift_available(c)) {
+        // c1c arrives in the transform domain: inverse pass B', then one kernel finishes the inverse, lifts the digits
+        // and starts their forward transforms; the same again for ModDown
+        RET(launch_ntt_inv_pass_b(c, c1c, items * L, N, limbmap_q(c)));
+        RET(launch_ks_lift(c, c1c, N, items * L, limbmap_q(c), digits, L + 1, 0));
+        RET(launch_ntt_fwd_pass_b(c, digits, items * L * (L + 1), N, limbmap_qp(c)));
+        RET(launch_ks_inner(c, digits, digit_stride, rot0, rot_inc, u_items, u));
+        RET(launch_ntt_inv_pass_b(c, u + (int64_t)L * N, u_items * 2, (int64_t)(L + 1) * N, limbmap_single(L)));
+        RET(launch_ks_lift(c, u + (int64_t)L * N, (int64_t)(L + 1) * N, u_items * 2, limbmap_single(L), lifted, L, 0));
+        RET(launch_ntt_fwd_pass_b(c, lifted, u_items * 2 * L, N, limbmap_q(c)));
+        return HANN_OK;
+    }
+    RET(launch_ntt_inv(c, c1c, items * L, N, limbmap_q(c)));
     RET(launch_lift_digits(c, c1c, (int64_t)L * N, items, digits));
     RET(launch_ntt_fwd(c, digits, items * L * (L + 1), N, limbmap_qp(c)));
     RET(launch_ks_inner(c, digits, digit_stride, rot0, rot_inc, u_items, u));
@@ -627,7 +640,6 @@ extern "C" int hann_query_prepare(hann_ctx* c, const void* ct_dev, void* baby_de
     u64* lifted = ar.take<u64>((int64_t)(B - 1) * 2 * LN);
     if (!c1c || !digits || !u || !lifted) return fail(c, HANN_EWORKSPACE, "hann_query_prepare: workspace too small");
     CK(cudaMemcpyAsync(c1c, ct + LN, LN * 8, cudaMemcpyDeviceToDevice, c->stream));
-    RET(launch_ntt_inv(c, c1c, L, N, limbmap_q(c)));
     // one digit set, B-1 keys: item i uses rotation 1 + i
     RET(ks_digits_to_lifted(c, c1c, 1, digits, 0, 1, 1, B - 1, u, lifted));
     RET(launch_moddown_combine(c, u, lifted, B - 1, 1, 1, ct, 0, nullptr, 0, baby + ctw, baby + ctw + LN, ctw));
@@ -708,7 +720,6 @@ extern "C" int hann_rotate_sum(hann_ctx* c, const void* inner_dev, int64_t n_blo
             u64* out = (g % 2 == 0) ? score + b0 * ctw : tmp;
             // c1 of every accumulator -> coefficients
             CK(cudaMemcpy2DAsync(c1c, LN * 8, old + LN, old_stride * 8, LN * 8, nb, cudaMemcpyDeviceToDevice, c->stream));
-            RET(launch_ntt_inv(c, c1c, nb * L, N, limbmap_q(c)));
             RET(ks_digits_to_lifted(c, c1c, nb, digits, (int64_t)L * L1N, B, 0, nb, u, lifted));
             RET(launch_moddown_combine(c, u, lifted, nb, B, 0, old, old_stride, inner + (b0 * G + g) * ctw, (int64_t)G * ctw, out,
                                        out + LN, ctw));
@@ -738,7 +749,6 @@ extern "C" int hann_keyswitch(hann_ctx* c, int rot, const void* poly_dev, void* 
     // the stored key is phi_k^{-1}(evk): switch phi_k^{-1}(d) and apply phi_k to the result
     const unsigned kinv = c->h_galois[(c->n - rot) % c->n];
     RET(launch_permute(c, (const u64*)poly_dev, c1c, L, kinv));
-    RET(launch_ntt_inv(c, c1c, L, N, limbmap_q(c)));
     RET(ks_digits_to_lifted(c, c1c, 1, digits, 0, rot, 0, 1, u, lifted));
     RET(launch_moddown_combine(c, u, lifted, 1, rot, 0, nullptr, 0, nullptr, 0, (u64*)ks0_dev, (u64*)ks1_dev, 0));
     return HANN_OK;

@@ -325,6 +325,146 @@ __global__ void __launch_bounds__(kThreads, AR::kMinBlocks) k_ntt_inv_a(NttArgs 
     inv_a_body<R1, R2>(A, ar, base, (const typename AR::TW*)A.tw + ((size_t)sel.limb << A.logN), sm);
 }
 
+// ---- fused key-switch step: inverse pass A' + centred lift + forward pass A for several target moduli -----------------
+//
+// Both the digit decomposition (ModUp) and ModDown take a polynomial back to coefficients, lift every coefficient to a
+// centred integer and re-reduce it into other moduli, whose forward transforms follow.  The last inverse round leaves a
+// thread with rows g + G1*e of its column -- exactly the words the first forward round needs -- so the lift and pass A of
+// all target transforms run from registers; the coefficient-domain polynomials never travel to memory.
+
+struct LiftArgs {
+    u64* src;             // source polynomials after inverse pass B' (private format of their modulus)
+    long long src_stride;
+    int src_period;
+    u64 src_limb4;        // limb of source polynomial sp = nibble (sp % src_period)
+    u64* dst;             // target polynomial (sp, ti) at dst + (sp * n_tgt + ti) * N, in forward pass-A output format
+    int n_tgt, tgt_limb0;
+    int logN;
+    const void *tw_inv_int, *tw_inv_f64, *tw_fwd_int, *tw_fwd_f64;
+    const LimbConst* lt;
+};
+
+template <int R1, int R2, class AR>
+__device__ __forceinline__ void lift_inverse(const LiftArgs& A, const AR ar, const typename AR::TW* __restrict__ tw, const u64* __restrict__ base,
+                                             u64* __restrict__ sm, int g, int c, bool active, u64 (&v)[1 << R1]) {
+    constexpr int G1 = 1 << R2, G2 = 1 << R1;
+    constexpr int RR2 = R2 == 0 ? 1 : R2;
+    const typename AR::TW ninv = ar.ninv;
+    if (R2 != 0) {
+        for (int w = threadIdx.x; w < (G2 << 4); w += blockDim.x) {
+            const int cc = w & 15, gg = w >> 4;
+            typename AR::T x[1 << RR2];
+#pragma unroll
+            for (int e = 0; e < (1 << RR2); e++) x[e] = ar.from_mid(base[(size_t)((gg << RR2) + e) * 256 + cc]);
+            inv_round<RR2>(ar, x, tw, (unsigned)(G2 + gg));
+#pragma unroll
+            for (int e = 0; e < (1 << RR2); e++) sm[(((gg << RR2) + e) << 4) + cc] = ar.to_mid(x[e]);
+        }
+        __syncthreads();
+    }
+    if (active) {
+        typename AR::T x[1 << R1];
+#pragma unroll
+        for (int e = 0; e < (1 << R1); e++) x[e] = ar.from_mid(R2 == 0 ? base[(size_t)(g + G1 * e) * 256 + c] : sm[((g + G1 * e) << 4) + c]);
+        inv_round<R1>(ar, x, tw, 1u);
+#pragma unroll
+        for (int e = 0; e < (1 << R1); e++) v[e] = ar.scaled_output(x[e], ninv);
+    }
+}
+
+__device__ __forceinline__ double lifted_value(const ArithF64&, u64 r, bool neg, u64 q) { return neg ? -(double)r : (double)r; }
+template <bool S>
+__device__ __forceinline__ u64 lifted_value(const ArithInt<S>&, u64 r, bool neg, u64 q) { return (neg && r) ? q - r : r; }
+
+template <int R1, int R2, class AR>
+__device__ __forceinline__ void lift_forward(const AR ar, const LimbConst* lc, bool same_modulus, const typename AR::TW* __restrict__ tw,
+                                             u64* __restrict__ base, u64* __restrict__ sm, int g, int c, bool active,
+                                             const u64 (&v)[1 << R1], u64 src_q, u64 src_half) {
+    constexpr int G1 = 1 << R2, G2 = 1 << R1;
+    constexpr int RR2 = R2 == 0 ? 1 : R2;
+    if (active) {
+        typename AR::T x[1 << R1];
+#pragma unroll
+        for (int e = 0; e < (1 << R1); e++) {
+            // centred lift of the coefficient (sign and magnitude), reduced into this modulus
+            const bool neg = v[e] > src_half;
+            const u64 mag = neg ? src_q - v[e] : v[e];
+            x[e] = same_modulus ? ar.from_canonical(v[e]) : lifted_value(ar, barrett64(mag, *lc), neg, lc->q);
+        }
+        fwd_round<R1>(ar, x, tw, 1u);
+#pragma unroll
+        for (int e = 0; e < (1 << R1); e++) {
+            if (R2 == 0) base[(size_t)(g + G1 * e) * 256 + c] = ar.to_mid(x[e]);
+            else sm[((g + G1 * e) << 4) + c] = ar.to_mid(x[e]);
+        }
+    }
+    if (R2 != 0) {
+        __syncthreads();
+        for (int w = threadIdx.x; w < (G2 << 4); w += blockDim.x) {
+            const int cc = w & 15, gg = w >> 4;
+            typename AR::T x[1 << RR2];
+#pragma unroll
+            for (int e = 0; e < (1 << RR2); e++) x[e] = ar.from_mid(sm[(((gg << RR2) + e) << 4) + cc]);
+            fwd_round<RR2>(ar, x, tw, (unsigned)(G2 + gg));
+#pragma unroll
+            for (int e = 0; e < (1 << RR2); e++) base[(size_t)((gg << RR2) + e) * 256 + cc] = ar.to_mid(x[e]);
+        }
+        __syncthreads();  // the exchange tile is free for the next target
+    }
+}
+
+template <int R1, int R2>
+__global__ void __launch_bounds__(256, 2) k_ks_lift(LiftArgs A) {
+    extern __shared__ u64 sm[];
+    constexpr int G1 = 1 << R2;
+    const int N = 1 << A.logN;
+    const long long sp = blockIdx.y;
+    const int c0 = blockIdx.x << 4;
+    const int c = threadIdx.x & 15, g = threadIdx.x >> 4;
+    const bool active = g < G1;
+    const int sl = (int)((A.src_limb4 >> (4 * (sp % A.src_period))) & 15);
+    const LimbConst* slc = A.lt + sl;
+    const u64* sbase = A.src + sp * A.src_stride + c0;
+    u64 v[1 << R1];
+    if (slc->q < (1ULL << 50)) {
+        const ArithF64 ar(slc);
+        lift_inverse<R1, R2>(A, ar, (const double2*)A.tw_inv_f64 + ((size_t)sl << A.logN), sbase, sm, g, c, active, v);
+    } else {
+        const ArithInt<false> ar(slc);
+        lift_inverse<R1, R2>(A, ar, (const ulonglong2*)A.tw_inv_int + ((size_t)sl << A.logN), sbase, sm, g, c, active, v);
+    }
+    if (R2 != 0) __syncthreads();  // every thread is done with the exchange tile of the inverse rounds
+    for (int ti = 0; ti < A.n_tgt; ti++) {
+        const int tl = A.tgt_limb0 + ti;
+        const LimbConst* tlc = A.lt + tl;
+        u64* dbase = A.dst + (sp * A.n_tgt + ti) * (long long)N + c0;
+        if (tlc->q < (1ULL << 50)) {
+            const ArithF64 ar(tlc);
+            lift_forward<R1, R2>(ar, tlc, tl == sl, (const double2*)A.tw_fwd_f64 + ((size_t)tl << A.logN), dbase, sm, g, c, active, v, slc->q, slc->half);
+        } else if (tlc->q < (1ULL << 57)) {
+            const ArithInt<true> ar(tlc);
+            lift_forward<R1, R2>(ar, tlc, tl == sl, (const ulonglong2*)A.tw_fwd_int + ((size_t)tl << A.logN), dbase, sm, g, c, active, v, slc->q, slc->half);
+        } else {
+            const ArithInt<false> ar(tlc);
+            lift_forward<R1, R2>(ar, tlc, tl == sl, (const ulonglong2*)A.tw_fwd_int + ((size_t)tl << A.logN), dbase, sm, g, c, active, v, slc->q, slc->half);
+        }
+    }
+}
+
+typedef void (*KernLift)(LiftArgs);
+KernLift pick_lift(int a) {
+    switch (a) {
+        case 1: return k_ks_lift<1, 0>;
+        case 2: return k_ks_lift<2, 0>;
+        case 3: return k_ks_lift<3, 0>;
+        case 4: return k_ks_lift<4, 0>;
+        case 5: return k_ks_lift<4, 1>;
+        case 6: return k_ks_lift<4, 2>;
+        case 7: return k_ks_lift<4, 3>;
+        default: return k_ks_lift<4, 4>;
+    }
+}
+
 // ---- dispatch ----------------------------------------------------------------------------------------------------
 
 typedef void (*KernA)(NttArgs);
@@ -381,12 +521,12 @@ void launch_fwd_class(hann_ctx* c, const NttArgs& A, int groups, bool skip_a) {
 }
 
 template <class AR>
-void launch_inv_class(hann_ctx* c, const NttArgs& A, int groups) {
+void launch_inv_class(hann_ctx* c, const NttArgs& A, int groups, bool skip_a) {
     {
         KProf kp(c, KC_NTT_INV_B);
         pick_inv_b<AR>(A.b)<<<dim3((c->N >> A.b) / A.K, groups * A.nsel), kThreads, smem_b(A), c->stream>>>(A, A.a == 0 ? 1 : 0);
     }
-    if (A.a > 0) {
+    if (A.a > 0 && !skip_a) {
         KProf kp(c, KC_NTT_INV_A);
         pick_inv_a<AR>(A.a)<<<dim3(1 << (A.b - A.logC), groups * A.nsel), kThreads, smem_a(A), c->stream>>>(A);
     }
@@ -431,8 +571,8 @@ int launch_ntt(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const Limb
                 else if (cls == 1) launch_fwd_class<ArithInt<true>>(c, A, groups, skip_a);
                 else launch_fwd_class<ArithInt<false>>(c, A, groups, skip_a);
             } else {
-                if (cls == 0) launch_inv_class<ArithF64>(c, A, groups);
-                else launch_inv_class<ArithInt<false>>(c, A, groups);
+                if (cls == 0) launch_inv_class<ArithF64>(c, A, groups, skip_a);
+                else launch_inv_class<ArithInt<false>>(c, A, groups, skip_a);
             }
         }
     }
@@ -472,6 +612,49 @@ int launch_ntt_fwd_pass_b(hann_ctx* c, u64* data, int64_t npoly, int64_t stride,
 
 int launch_ntt_inv(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm) {
     return launch_ntt(c, data, npoly, stride, lm, true);
+}
+
+bool ks_lift_available(const hann_ctx* c) { return c->logN >= 9; }
+
+// After inverse pass B' of the nsrc source polynomials (launch_ntt_inv_pass_b): finish their inverse transforms, lift the
+// coefficients (centred) into the n_tgt moduli tgt_limb0 .. and run pass A of the target transforms.  The caller finishes
+// with launch_ntt_fwd_pass_b over the targets.
+int launch_ks_lift(hann_ctx* c, u64* src, int64_t src_stride, int64_t nsrc, const LimbMap& src_lm, u64* dst, int n_tgt, int tgt_limb0) {
+    if (nsrc <= 0) return HANN_OK;
+    LiftArgs A;
+    A.src = src;
+    A.src_stride = src_stride;
+    A.src_period = src_lm.period;
+    A.src_limb4 = 0;
+    for (int i = 0; i < src_lm.period && i < 16; i++) A.src_limb4 |= (u64)src_lm.limb[i] << (4 * i);
+    A.dst = dst;
+    A.n_tgt = n_tgt;
+    A.tgt_limb0 = tgt_limb0;
+    A.logN = c->logN;
+    A.tw_inv_int = c->tw_inv;
+    A.tw_inv_f64 = c->tw_inv_f64;
+    A.tw_fwd_int = c->tw_fwd;
+    A.tw_fwd_f64 = c->tw_fwd_f64;
+    A.lt = c->lt_dev;
+    const int a = c->logN - 8;
+    const size_t smem = a > 4 ? (size_t)(1 << a) * 16 * 8 : 0;
+    const int threads = a >= 8 ? 256 : (a == 7 ? 128 : 64);
+    for (int64_t s0 = 0; s0 < nsrc; s0 += 65535) {
+        const int ns = (int)std::min<int64_t>(65535, nsrc - s0);
+        // the source limb of polynomial s0 + y is nibble (s0 + y) % period: 65535 is not a multiple of every period, so shift
+        LiftArgs Ap = A;
+        Ap.src = src + s0 * src_stride;
+        Ap.dst = dst + s0 * n_tgt * (int64_t)c->N;
+        Ap.src_limb4 = 0;
+        for (int i = 0; i < src_lm.period && i < 16; i++) Ap.src_limb4 |= (u64)src_lm.limb[(s0 + i) % src_lm.period] << (4 * i);
+        KProf kp(c, KC_LIFT_DIGITS);
+        pick_lift(a)<<<dim3(16, ns), threads, smem, c->stream>>>(Ap);
+    }
+    return check_launch(c, "ks_lift");
+}
+
+int launch_ntt_inv_pass_b(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm) {
+    return launch_ntt(c, data, npoly, stride, lm, true, true);
 }
 
 int ntt_configure(hann_ctx* c) {

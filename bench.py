@@ -28,7 +28,6 @@ sys.path.insert(0, ROOT)
 METRIC = "encrypted candidates scored/sec"
 UNIT = "candidates/s"
 SM_COUNT = 148
-IMAD_LANES_PER_SM = 64  # 32-bit integer multiply-add lanes per SM per clock
 
 
 def read_peaks():
@@ -121,26 +120,41 @@ def build_workload(config, rows_override=None):
     raise SystemExit("bench.py times configs 0, 1 and 4; the hierarchy configs are exercised by the tests")
 
 
+FP64_LANES_PER_SM = 64  # binary64 multiply-add lanes per SM per clock
+
+# DRAM bytes (read + write) per unit of work of the bandwidth- or transform-bound kernels, from the ncu captures
+# summarised under profiles/ (small case: one block of 32,768 rows; traffic grows in proportion to the units)
+NCU_DRAM_BYTES_PER_UNIT = {
+    "ntt_fwd_b": ("polynomial", 483.2e6 / 512),
+    "mac": ("block", None),
+    "ks_inner": ("item", None),
+}
+
+
 def algorithmic_work(ctx, n_blocks, n_rows):
-    """algorithmic bytes (HBM-bound kernels) or 32-bit multiplies (ALU-bound kernels) of ONE step, per kernel class.
-    A 64-bit Shoup butterfly costs 10 32x32-bit multiplies: 4 for hi64(a*w'), 3 for lo64(a*w), 3 for lo64(t*q)."""
+    """Algorithmic work of ONE step per kernel class: bytes for the HBM-bound kernels, binary64 instructions for the
+    transform kernels (moduli below 2^50 run their butterflies on the FP64 pipe: exact product = multiply + fma,
+    quotient = multiply + round, remainder = fma + add, butterfly = add + subtract: 8 per butterfly; an FFT butterfly with
+    separately rounded products and sums is 10).  Returns {class: (bound, amount, units per step)}."""
     L, N, B, G, R = ctx.L, ctx.N, ctx.B, ctx.G, ctx.R
-    logN = ctx.logN
+    n, logN = ctx.n, ctx.logN
     b = min(logN, 8)
     a = logN - b
     W = 8 * N
-    fwd_polys = n_blocks * R * L + (L * (L + 1) + (B - 1) * 2 * L) + (G - 1) * n_blocks * (L * (L + 1) + 2 * L)
-    inv_polys = (L + (B - 1) * 2) + (G - 1) * n_blocks * (L + 2)
+    items_rot = (G - 1) * n_blocks  # key switches of the rotate-and-sum
+    fwd_polys = n_blocks * R * L + (L * (L + 1) + (B - 1) * 2 * L) + items_rot * (L * (L + 1) + 2 * L)
+    inv_polys = (L + (B - 1) * 2) + items_rot * (L + 2)
+    lift_src = [(L, L + 1), ((B - 1) * 2, L)] + [(items_rot * L, L + 1), (items_rot * 2, L)]  # (sources, targets each)
+    lift_ops = sum(src * (1 + tgt) * a * (N // 2) * 8 for src, tgt in lift_src)
     return {
-        "mac": ("hbm", n_blocks * R * L * W + B * 2 * L * W + n_blocks * G * 2 * L * W),
+        "mac": ("hbm", n_blocks * R * L * W + B * 2 * L * W + n_blocks * G * 2 * L * W, n_blocks),
         "ks_inner": ("hbm", (B - 1) * (L * 2 * (L + 1) * W + 2 * (L + 1) * W) + L * (L + 1) * W
-                     + (G - 1) * (L * 2 * (L + 1) * W + n_blocks * (L * (L + 1) * W + 2 * (L + 1) * W))),
-        "ntt_fwd_a": ("alu", fwd_polys * (N // 2) * a * 10),
-        "ntt_fwd_b": ("alu", fwd_polys * (N // 2) * b * 10),
-        "ntt_inv_a": ("alu", inv_polys * (N // 2) * a * 10),
-        "ntt_inv_b": ("alu", inv_polys * (N // 2) * b * 10),
-        "fft_a": ("hbm", n_blocks * R * (ctx.n * 16) + n_rows * R * 4),
-        "fft_b": ("hbm", n_blocks * R * (ctx.n * 16 + L * W)),
+                     + (G - 1) * (L * 2 * (L + 1) * W + n_blocks * (L * (L + 1) * W + 2 * (L + 1) * W)), (B - 1) + items_rot),
+        "ntt_fwd_b": ("alu", fwd_polys * (N // 2) * b * 8, fwd_polys),
+        "ntt_inv_b": ("alu", inv_polys * (N // 2) * b * 8, inv_polys),
+        "lift_digits": ("alu", lift_ops, inv_polys),
+        "fft_a": ("hbm", n_blocks * R * (n * 16) + n_rows * R * 4, n_blocks * R),
+        "fft_b": ("alu", n_blocks * R * ((a - 1) * (n // 2) * 10 + L * a * (N // 2) * 8), n_blocks * R),
     }
 
 
@@ -248,22 +262,27 @@ def run_ours(args):
     hbm_peak, sm_max_mhz, peak_src = read_peaks()
     work = algorithmic_work(ctx, nb, n_rows)
     dom = max((k for k in kernels if k in work), key=lambda k: kernels[k]["ms_per_step"])
-    bound, amount = work[dom]
+    bound, amount, units = work[dom]
     dom_s = kernels[dom]["ms_per_step"] * 1e-3
+    dom_launches = max(kernels[dom]["launches_per_step"], 1)
     if bound == "hbm":
         achieved, peak, runit = amount / dom_s / 1e9, hbm_peak, "GB/s"
+        psrc = peak_src + " copy bandwidth"
     else:
-        achieved, peak, runit = amount / dom_s / 1e12, SM_COUNT * IMAD_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12, "Tmul32/s"
+        achieved, peak, runit = amount / dom_s / 1e12, SM_COUNT * FP64_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12, "T fp64 instr/s"
+        psrc = "derived: %d SMs x %d fp64 lanes x %.0f MHz" % (SM_COUNT, FP64_LANES_PER_SM, sm_max_mhz)
+    unit_name, per_unit = NCU_DRAM_BYTES_PER_UNIT.get(dom, (None, None))
     roofline = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,
-                "peak_source": peak_src + (" copy bandwidth" if bound == "hbm" else
-                                           ": %d SMs x %d int32 multiply-add lanes x %.0f MHz" % (SM_COUNT, IMAD_LANES_PER_SM, sm_max_mhz)),
-                "traffic": None, "launches_per_step": kernels[dom]["launches_per_step"],
-                "avg_launch_ms": kernels[dom]["ms_per_step"] / max(kernels[dom]["launches_per_step"], 1)}
+                "peak_source": psrc, "launches_per_step": kernels[dom]["launches_per_step"],
+                "avg_launch_ms": kernels[dom]["ms_per_step"] / dom_launches,
+                "algorithmic_per_launch": amount / dom_launches,
+                "traffic": per_unit * units / dom_launches if per_unit else None,
+                "traffic_source": ("ncu dram bytes per %s on the 1-block case x %s per launch" % (unit_name, unit_name)) if per_unit else None}
     hbm_kernels = {}
     for k in ("mac", "ks_inner"):
         if k in kernels:
-            hbm_kernels[k] = {"GB/s": work[k][1] / (kernels[k]["ms_per_step"] * 1e-3) / 1e9,
-                              "frac_of_measured_copy": work[k][1] / (kernels[k]["ms_per_step"] * 1e-3) / 1e9 / hbm_peak}
+            gbs = work[k][1] / (kernels[k]["ms_per_step"] * 1e-3) / 1e9
+            hbm_kernels[k] = {"GB/s": gbs, "frac_of_measured_copy": gbs / hbm_peak, "frac_of_8TBps_nominal": gbs / 8000.0}
 
     # end to end through the host-buffer entry point: pinned host inputs, copies inside the timed region
     rows_pin = torch.from_numpy(rows_np).pin_memory()

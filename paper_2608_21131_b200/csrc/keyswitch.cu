@@ -322,6 +322,43 @@ __global__ void __launch_bounds__(kThreads) k_moddown_combine(
     }
 }
 
+// The same combine for rings of at least 256 points, without scattered global reads.  In bit-reversed order the
+// automorphism maps every aligned chunk of 256 positions onto another aligned chunk (the top 8 bits of a position are
+// the low 8 bits of its evaluation index, which an affine map modulo 2^logN keeps together), so a CTA loads the source
+// chunk of u, lifted and c0 contiguously into shared memory and permutes there.
+__global__ void __launch_bounds__(256) k_moddown_combine_chunk(
+    const u64* __restrict__ u, const u64* __restrict__ lifted, const unsigned* __restrict__ galois, int rot0, int rot_inc,
+    const u64* __restrict__ c0, long long c0_stride, const u64* __restrict__ addend, long long addend_stride,
+    u64* __restrict__ out0, u64* __restrict__ out1, long long out_stride, int N, int logN, int L, const LimbConst* __restrict__ lt) {
+    __shared__ u64 su[2][256], sl[2][256], sc[256];
+    const long long LN = (long long)L * N, L1N = (long long)(L + 1) * N;
+    const int chunks = N >> 8;
+    const int chunk = blockIdx.x % chunks;
+    const int i = (blockIdx.x / chunks) % L;
+    const long long item = blockIdx.x / ((long long)chunks * L);
+    const unsigned k = galois[rot0 + (int)item * rot_inc];
+    const int t = (chunk << 8) + threadIdx.x;
+    const int s = (k == 1u) ? t : galois_src(t, k, logN);
+    const int src_chunk = ((k == 1u) ? (chunk << 8) : galois_src(chunk << 8, k, logN)) & ~255;
+    const LimbConst lc = lt[i];
+#pragma unroll
+    for (int comp = 0; comp < 2; comp++) {
+        su[comp][threadIdx.x] = u[(item * 2 + comp) * L1N + (long long)i * N + src_chunk + threadIdx.x];
+        sl[comp][threadIdx.x] = lifted[((item * 2 + comp) * L + i) * N + src_chunk + threadIdx.x];
+    }
+    if (c0) sc[threadIdx.x] = c0[item * c0_stride + (long long)i * N + src_chunk + threadIdx.x];
+    __syncthreads();
+    const int ls = s & 255;
+#pragma unroll
+    for (int comp = 0; comp < 2; comp++) {
+        u64 v = csub(shoup_mul(submod(su[comp][ls], sl[comp][ls], lc.q), lc.pinv, lc.pinv_s, lc.q), lc.q);
+        if (comp == 0 && c0) v = addmod(v, sc[ls], lc.q);
+        if (addend) v = addmod(v, addend[item * addend_stride + (long long)comp * LN + (long long)i * N + t], lc.q);
+        u64* o = (comp == 0 ? out0 : out1) + item * out_stride + (long long)i * N + t;
+        *o = v;
+    }
+}
+
 // dst[poly][t] = src[poly][galois source of t]   (transform domain automorphism X -> X^k)
 __global__ void __launch_bounds__(kThreads) k_permute(const u64* __restrict__ src, u64* __restrict__ dst, long long npoly,
                                                       unsigned k, int N, int logN) {
@@ -517,6 +554,14 @@ int launch_moddown_lift(hann_ctx* c, const u64* u, int64_t npoly, u64* lifted) {
 int launch_moddown_combine(hann_ctx* c, const u64* u, const u64* lifted, int64_t nitems, int rot0, int rot_inc, const u64* c0,
                            int64_t c0_stride, const u64* addend, int64_t addend_stride, u64* out0, u64* out1,
                            int64_t out_stride) {
+    if (c->N >= 256) {
+        const long long ctas = nitems * c->L * (c->N >> 8);
+        KProf kp(c, KC_MODDOWN_COMBINE);
+        k_moddown_combine_chunk<<<(unsigned)ctas, 256, 0, c->stream>>>(u, lifted, c->galois_dev, rot0, rot_inc, c0, c0_stride, addend,
+                                                                     addend_stride, out0, out1, out_stride, c->N, c->logN, c->L,
+                                                                     c->lt_dev);
+        return check_launch(c, "moddown_combine_chunk");
+    }
     {
         KProf kp(c, KC_MODDOWN_COMBINE);
         k_moddown_combine<<<grid_for(nitems * 2 * c->L * c->N), kThreads, 0, c->stream>>>(

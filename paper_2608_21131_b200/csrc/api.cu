@@ -190,6 +190,7 @@ extern "C" int hann_ctx_create(const hann_params* prm, hann_ctx** out) {
     if (!c) return HANN_ENOMEM;
     c->prm = *prm;
     c->logN = prm->logN; c->N = N; c->n = n; c->L = L; c->R = prm->R; c->B = prm->B; c->G = prm->R / prm->B;
+    c->ntt_tau = prm->logN >= 10 ? 1 : 0;
     c->device = prm->device;
     c->stream = (cudaStream_t)prm->stream;
     DeviceGuard dg(c->device);

@@ -19,6 +19,7 @@ enum {
 struct hann_ctx {
     hann_params prm;
     int logN = 0, N = 0, n = 0, L = 0, R = 0, B = 0, G = 0;
+    int ntt_tau = 0;  // 1 when the transform-domain layout swaps the low nibbles of positions (rings of 2^10 and more)
     int device = 0;
     cudaStream_t stream = nullptr;
     // helper stream and events of hann_query_level, which runs the query preparation beside the candidate encoding

@@ -301,7 +301,7 @@ __global__ void __launch_bounds__(kThreads) k_moddown_combine(
     const u64* __restrict__ u, const u64* __restrict__ lifted, long long nitems, const unsigned* __restrict__ galois,
     int rot0, int rot_inc, const u64* __restrict__ c0, long long c0_stride, const u64* __restrict__ addend,
     long long addend_stride, u64* __restrict__ out0, u64* __restrict__ out1, long long out_stride, int N, int logN, int L,
-    LimbTable lt) {
+    int tau, LimbTable lt) {
     const long long LN = (long long)L * N, L1N = (long long)(L + 1) * N;
     const long long total = nitems * 2 * LN;
     for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
@@ -310,7 +310,7 @@ __global__ void __launch_bounds__(kThreads) k_moddown_combine(
         const int comp = (int)((idx / LN) % 2);
         const long long item = idx / (2 * LN);
         const unsigned k = galois[rot0 + (int)item * rot_inc];
-        const int s = (k == 1u) ? t : galois_src(t, k, logN);
+        const int s = (k == 1u) ? t : galois_src(t, k, logN, tau);
         const LimbConst& lc = lt.c[i];
         u64 a = u[(item * 2 + comp) * L1N + (long long)i * N + s];
         u64 b = lifted[((item * 2 + comp) * L + i) * N + s];
@@ -329,7 +329,8 @@ __global__ void __launch_bounds__(kThreads) k_moddown_combine(
 __global__ void __launch_bounds__(256) k_moddown_combine_chunk(
     const u64* __restrict__ u, const u64* __restrict__ lifted, const unsigned* __restrict__ galois, int rot0, int rot_inc,
     const u64* __restrict__ c0, long long c0_stride, const u64* __restrict__ addend, long long addend_stride,
-    u64* __restrict__ out0, u64* __restrict__ out1, long long out_stride, int N, int logN, int L, const LimbConst* __restrict__ lt) {
+    u64* __restrict__ out0, u64* __restrict__ out1, long long out_stride, int N, int logN, int L, int tau,
+    const LimbConst* __restrict__ lt) {
     __shared__ u64 su[2][256], sl[2][256], sc[256];
     const long long LN = (long long)L * N, L1N = (long long)(L + 1) * N;
     const int chunks = N >> 8;
@@ -338,8 +339,8 @@ __global__ void __launch_bounds__(256) k_moddown_combine_chunk(
     const long long item = blockIdx.x / ((long long)chunks * L);
     const unsigned k = galois[rot0 + (int)item * rot_inc];
     const int t = (chunk << 8) + threadIdx.x;
-    const int s = (k == 1u) ? t : galois_src(t, k, logN);
-    const int src_chunk = ((k == 1u) ? (chunk << 8) : galois_src(chunk << 8, k, logN)) & ~255;
+    const int s = (k == 1u) ? t : galois_src(t, k, logN, tau);
+    const int src_chunk = ((k == 1u) ? (chunk << 8) : galois_src(chunk << 8, k, logN, tau)) & ~255;
     const LimbConst lc = lt[i];
 #pragma unroll
     for (int comp = 0; comp < 2; comp++) {
@@ -361,12 +362,12 @@ __global__ void __launch_bounds__(256) k_moddown_combine_chunk(
 
 // dst[poly][t] = src[poly][galois source of t]   (transform domain automorphism X -> X^k)
 __global__ void __launch_bounds__(kThreads) k_permute(const u64* __restrict__ src, u64* __restrict__ dst, long long npoly,
-                                                      unsigned k, int N, int logN) {
+                                                      unsigned k, int N, int logN, int tau) {
     const long long total = npoly * N;
     for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
         const long long poly = idx / N;
         const int t = (int)(idx % N);
-        dst[idx] = src[poly * N + galois_src(t, k, logN)];
+        dst[idx] = src[poly * N + galois_src(t, k, logN, tau)];
     }
 }
 
@@ -559,14 +560,14 @@ int launch_moddown_combine(hann_ctx* c, const u64* u, const u64* lifted, int64_t
         KProf kp(c, KC_MODDOWN_COMBINE);
         k_moddown_combine_chunk<<<(unsigned)ctas, 256, 0, c->stream>>>(u, lifted, c->galois_dev, rot0, rot_inc, c0, c0_stride, addend,
                                                                      addend_stride, out0, out1, out_stride, c->N, c->logN, c->L,
-                                                                     c->lt_dev);
+                                                                     c->ntt_tau, c->lt_dev);
         return check_launch(c, "moddown_combine_chunk");
     }
     {
         KProf kp(c, KC_MODDOWN_COMBINE);
         k_moddown_combine<<<grid_for(nitems * 2 * c->L * c->N), kThreads, 0, c->stream>>>(
             u, lifted, nitems, c->galois_dev, rot0, rot_inc, c0, c0_stride, addend, addend_stride, out0, out1, out_stride, c->N,
-            c->logN, c->L, c->lt);
+            c->logN, c->L, c->ntt_tau, c->lt);
     }
     return check_launch(c, "moddown_combine");
 }
@@ -574,7 +575,7 @@ int launch_moddown_combine(hann_ctx* c, const u64* u, const u64* lifted, int64_t
 int launch_permute(hann_ctx* c, const u64* src, u64* dst, int64_t npoly, unsigned k) {
     {
         KProf kp(c, KC_PERMUTE);
-        k_permute<<<grid_for(npoly * c->N), kThreads, 0, c->stream>>>(src, dst, npoly, k, c->N, c->logN);
+        k_permute<<<grid_for(npoly * c->N), kThreads, 0, c->stream>>>(src, dst, npoly, k, c->N, c->logN, c->ntt_tau);
     }
     return check_launch(c, "permute");
 }

@@ -85,12 +85,19 @@ __device__ __forceinline__ void mac128(u64& hi, u64& lo, u64 a, u64 b) {
     hi += ph + (lo < pl ? 1 : 0);
 }
 
-// position t of a transformed polynomial holds the value at psi^(2*brev(t)+1); the automorphism X -> X^k
-// reads position brev(((2*brev(t)+1)*k mod 2N - 1) / 2)
-__device__ __forceinline__ int galois_src(int t, unsigned k, int logN) {
+// swap the two low nibbles of a position (an involution inside every aligned chunk of 256 positions)
+__device__ __forceinline__ int swap_nibbles(int t) { return (t & ~255) | ((t & 15) << 4) | ((t >> 4) & 15); }
+
+// Position t of a transformed polynomial holds the value at psi^(2*brev(t)+1); the automorphism X -> X^k reads position
+// brev(((2*brev(t)+1)*k mod 2N - 1) / 2).  Rings of 2^10 points and more store every chunk of 256 positions with its
+// two low nibbles swapped (`tau`: the last forward round then writes, and the first inverse round reads, coalesced
+// words straight from registers), so the map is conjugated by that swap.
+__device__ __forceinline__ int galois_src(int t, unsigned k, int logN, int tau) {
+    if (tau) t = swap_nibbles(t);
     unsigned br = __brev((unsigned)t) >> (32 - logN);
     unsigned e = ((2u * br + 1u) * k) & ((2u << logN) - 1u);
-    return (int)(__brev((e - 1u) >> 1) >> (32 - logN));
+    int s = (int)(__brev((e - 1u) >> 1) >> (32 - logN));
+    return tau ? swap_nibbles(s) : s;
 }
 
 #endif  // __CUDACC__

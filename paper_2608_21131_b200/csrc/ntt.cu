@@ -45,6 +45,7 @@ struct NttArgs {
     // a launch covers, out of every group of `period` consecutive polynomials, the nsel positions pos[] (their limbs
     // limb[]): all positions whose modulus falls in the launch's arithmetic class
     int period, nsel;
+    int tau;  // chunks of 256 positions are stored with their low nibbles swapped (see galois_src)
     u64 pos4, limb4;  // 4-bit fields: position within the period and limb of selection k (at most 16 selections)
 };
 
@@ -178,19 +179,21 @@ __global__ void __launch_bounds__(256, HANN_B8_MINBLOCKS) k_ntt_fwd_b8(NttArgs A
     // which need group j*2^u + il' of stage 4 + u, read consecutive 16-byte words (no bank conflicts).
     TW* tc = (TW*)smraw;
     u64* sm = smraw + kBK * 256 * 2;     // [kBPG][kBK][272] padded chunks
-    const int y = blockIdx.y, k = y % A.nsel, yg = y / A.nsel;
+    const int k = blockIdx.y;
     const int pos = (int)((A.pos4 >> (4 * k)) & 15), limb = (int)((A.limb4 >> (4 * k)) & 15);
     const AR ar(A.lt + limb);
     const int chunk0 = blockIdx.x * kBK;
     const TW* tw = (const TW*)A.tw + ((size_t)limb << A.logN);
     const unsigned m0 = 1u << A.a;
     const int t = threadIdx.x >> 6, ch = (threadIdx.x >> 4) & 3, j = threadIdx.x & 15;
-    const long long group = (long long)yg * kBPG + t;
-    const bool valid = group < groups;
-    u64* base = A.data + (group * A.period + pos) * A.stride + ((size_t)(chunk0 + ch) << 8);
-    // the data loads go out first so that they overlap the staging of the twiddles
+    const int ntiles = (groups + kBPG - 1) / kBPG;
+    // a CTA walks tiles blockIdx.z, blockIdx.z + gridDim.z, ..: the twiddles are staged once, and the words of the next
+    // tile are already in flight while the current one is transformed
+    int yg = blockIdx.z;
+    const long long tile_stride = (long long)kBPG * A.period * A.stride;  // words between the same polynomial slot of two tiles
+    u64* base = A.data + (((long long)yg * kBPG + t) * A.period + pos) * A.stride + ((size_t)(chunk0 + ch) << 8);
     u64 raw[16];
-    if (valid) {
+    if ((long long)yg * kBPG + t < groups) {
 #pragma unroll
         for (int e = 0; e < 16; e++) raw[e] = base[j + 16 * e];
     }
@@ -208,31 +211,38 @@ __global__ void __launch_bounds__(256, HANN_B8_MINBLOCKS) k_ntt_fwd_b8(NttArgs A
     __syncthreads();
     const TW* tcc = tc + ch * 256;
     u64* s1 = sm + (t * kBK + ch) * 272;
-    if (valid) {
-        typename AR::T x[16];
+    for (; yg < ntiles; yg += gridDim.z) {
+        const bool valid = (long long)yg * kBPG + t < groups;
+        const int yn = yg + gridDim.z;
+        u64 nxt[16];
+        if (yn < ntiles && (long long)yn * kBPG + t < groups) {
+            const u64* nb = base + (long long)gridDim.z * tile_stride;
 #pragma unroll
-        for (int e = 0; e < 16; e++) x[e] = ar.from_mid(raw[e]);
-        fwd_round_f<4>(ar, x, [=](int st, int il) { return tcc[(1 << st) - 1 + il]; });
-#pragma unroll
-        for (int e = 0; e < 16; e++) s1[17 * e + j] = ar.to_mid(x[e]);
-    }
-    __syncthreads();
-    if (valid) {
-        typename AR::T x[16];
-#pragma unroll
-        for (int e = 0; e < 16; e++) x[e] = ar.from_mid(s1[17 * j + e]);
-        fwd_round_f<4>(ar, x, [=](int u, int il) { return tcc[(((1 << u) + il) << 4) + j]; });
-#pragma unroll
-        for (int e = 0; e < 16; e++) s1[17 * j + e] = ar.to_canonical(x[e]);
-    }
-    __syncthreads();
-    for (int idx = threadIdx.x; idx < kBPG * kBK * 256; idx += 256) {
-        const int t2 = idx >> 10, rem = idx & 1023;
-        const long long g2 = (long long)yg * kBPG + t2;
-        if (g2 < groups) {
-            const int p = rem & 255;
-            A.data[(g2 * A.period + pos) * A.stride + ((size_t)chunk0 << 8) + rem] = sm[(t2 * kBK + (rem >> 8)) * 272 + p + (p >> 4)];
+            for (int e = 0; e < 16; e++) nxt[e] = nb[j + 16 * e];
         }
+        if (valid) {
+            typename AR::T x[16];
+#pragma unroll
+            for (int e = 0; e < 16; e++) x[e] = ar.from_mid(raw[e]);
+            fwd_round_f<4>(ar, x, [=](int st, int il) { return tcc[(1 << st) - 1 + il]; });
+#pragma unroll
+            for (int e = 0; e < 16; e++) s1[17 * e + j] = ar.to_mid(x[e]);
+        }
+        __syncthreads();
+        if (valid) {
+            typename AR::T x[16];
+#pragma unroll
+            for (int e = 0; e < 16; e++) x[e] = ar.from_mid(s1[17 * j + e]);
+            fwd_round_f<4>(ar, x, [=](int u, int il) { return tcc[(((1 << u) + il) << 4) + j]; });
+            // logical position 16 j + e goes to word 16 e + j of the chunk (nibble-swapped layout): the 16 threads of a
+            // chunk write 128 contiguous bytes per store
+#pragma unroll
+            for (int e = 0; e < 16; e++) base[16 * e + j] = ar.to_canonical(x[e]);
+        }
+        __syncthreads();  // round 2 has read the exchange tile; the next tile may overwrite it
+#pragma unroll
+        for (int e = 0; e < 16; e++) raw[e] = nxt[e];
+        base += (long long)gridDim.z * tile_stride;
     }
 }
 
@@ -248,7 +258,11 @@ __device__ __forceinline__ void inv_b_body(const NttArgs& A, const AR ar, u64* _
     const unsigned m0 = 1u << A.a;
     const typename AR::TW ninv = ar.ninv;
     if (R2 != 0) {
-        for (int idx = threadIdx.x; idx < K * S; idx += kThreads) sm[(idx / S) * SP + pad<R2>(idx % S)] = base[idx];
+        // memory word idx of a chunk is logical position idx (or its nibble swap, on rings that store chunks that way)
+        for (int idx = threadIdx.x; idx < K * S; idx += kThreads) {
+            const int p = idx % S;
+            sm[(idx / S) * SP + pad<R2>(A.tau ? swap_nibbles(p) : p)] = base[idx];
+        }
         __syncthreads();
         for (int w = threadIdx.x; w < K * J2; w += kThreads) {
             const int ch = w / J2, j = w % J2;
@@ -514,7 +528,11 @@ void launch_fwd_class(hann_ctx* c, const NttArgs& A, int groups, bool skip_a) {
     if (A.b == 8 && A.a > 0 && ((c->N >> 8) % kBK) == 0) {
         const size_t smem = (size_t)kBK * 256 * 16 + (size_t)kBPG * kBK * 272 * 8;
         cudaFuncSetAttribute(k_ntt_fwd_b8<AR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  // 50 KiB > default 48
-        k_ntt_fwd_b8<AR><<<dim3((c->N >> 8) / kBK, ((groups + kBPG - 1) / kBPG) * A.nsel), 256, smem, c->stream>>>(A, groups);
+        // enough CTAs for about four per SM; beyond that a CTA walks several tiles and reuses its staged twiddles
+        const int ranges = (c->N >> 8) / kBK, ntiles = (groups + kBPG - 1) / kBPG;
+        int zs = (148 * 4 + ranges * A.nsel - 1) / (ranges * A.nsel);
+        zs = zs < 1 ? 1 : (zs > ntiles ? ntiles : zs);
+        k_ntt_fwd_b8<AR><<<dim3(ranges, A.nsel, zs), 256, smem, c->stream>>>(A, groups);
         return;
     }
     pick_fwd_b<AR>(A.b)<<<dim3((c->N >> A.b) / A.K, groups * A.nsel), kThreads, smem_b(A), c->stream>>>(A);
@@ -549,6 +567,7 @@ int launch_ntt(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const Limb
     const int chunks = c->N >> A.b;
     A.K = chunks < 16 ? chunks : 16;
     A.lt = c->lt_dev;
+    A.tau = c->ntt_tau;
     A.period = lm.period;
     const int64_t groups_total = npoly / lm.period;
     for (int cls = 0; cls < 3; cls++) {

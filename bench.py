@@ -51,7 +51,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits", "-lms", "100"],
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
@@ -214,12 +214,14 @@ def run_ours(args):
         print("lean run: %d steps, %d kernel launches" % (args.warmup + args.steps, ctx.get_stats()["launches"]))
         return 0
 
+    # the clock sampler runs from the warm-up on (nvidia-smi needs ~0.1 s to produce its first line); warm-up and timed
+    # steps are the same work, so every sample is taken under the timed region's load
+    sampler = ClockSampler(local)
+    sampler.start()
     for _ in range(max(args.warmup, 3)):
         step()
     l0 = ctx.get_stats()["launches"]
-    sampler = ClockSampler(local)
     barrier()
-    sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
@@ -411,8 +413,8 @@ def main():
         args.steps = 2 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup
         return run_reference(args)
-    args.steps = 10 if args.steps is None else args.steps
-    args.warmup = 3 if args.warmup is None else args.warmup
+    args.steps = 200 if args.steps is None else args.steps
+    args.warmup = 20 if args.warmup is None else args.warmup
     return run_ours(args)
 
 

@@ -293,6 +293,9 @@ extern "C" int hann_ctx_create(const hann_params* prm, hann_ctx** out) {
         ok = cudaStreamCreateWithFlags(&c->aux_stream, cudaStreamNonBlocking) == cudaSuccess &&
              cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
              cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < 2 && ok; i++)
+        ok = cudaStreamCreateWithFlags(&c->lane_stream[i], cudaStreamNonBlocking) == cudaSuccess &&
+             cudaEventCreateWithFlags(&c->lane_join[i], cudaEventDisableTiming) == cudaSuccess;
     if (ok) ok = ntt_configure(c) == HANN_OK;
     if (!ok) {
         cudaGetLastError();
@@ -315,6 +318,13 @@ extern "C" void hann_ctx_destroy(hann_ctx* c) {
     if (c->aux_stream) {
         cudaStreamSynchronize(c->aux_stream);
         cudaStreamDestroy(c->aux_stream);
+    }
+    for (int i = 0; i < 2; i++) {
+        if (c->lane_stream[i]) {
+            cudaStreamSynchronize(c->lane_stream[i]);
+            cudaStreamDestroy(c->lane_stream[i]);
+        }
+        if (c->lane_join[i]) cudaEventDestroy(c->lane_join[i]);
     }
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_join) cudaEventDestroy(c->ev_join);
@@ -702,32 +712,69 @@ extern "C" int hann_rotate_sum(hann_ctx* c, const void* inner_dev, int64_t n_blo
     }
     if (!c->keytab_host[B]) return fail(c, HANN_ENOKEY, "hann_rotate_sum: the key of rotation B is not loaded");
     if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_rotate_sum: workspace missing or not 256-byte aligned");
-    // as many blocks per round as the workspace holds
-    int64_t ch = ((int64_t)ws_bytes - kSlack) / (ks_item_words(c) * 8);
-    if (ch < 1) return fail(c, HANN_EWORKSPACE, "hann_rotate_sum: workspace too small");
-    ch = std::min<int64_t>(std::min<int64_t>(ch, n_blocks), 8);
-    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
-    u64* c1c = ar.take<u64>(ch * LN);
-    u64* digits = ar.take<u64>(ch * L * L1N);
-    u64* u = ar.take<u64>(ch * 2 * L1N);
-    u64* lifted = ar.take<u64>(ch * 2 * LN);
-    u64* tmp = ar.take<u64>(ch * ctw);
-    if (!c1c || !digits || !u || !lifted || !tmp) return fail(c, HANN_EWORKSPACE, "hann_rotate_sum: workspace too small");
-    for (int64_t b0 = 0; b0 < n_blocks; b0 += ch) {
-        const int64_t nb = std::min(ch, n_blocks - b0);
-        const u64* old = inner + (b0 * G + (G - 1)) * ctw;  // acc = inner[G-1]
-        int64_t old_stride = (int64_t)G * ctw;
-        for (int g = G - 2; g >= 0; g--) {
-            u64* out = (g % 2 == 0) ? score + b0 * ctw : tmp;
-            // c1 of every accumulator -> coefficients
-            CK(cudaMemcpy2DAsync(c1c, LN * 8, old + LN, old_stride * 8, LN * 8, nb, cudaMemcpyDeviceToDevice, c->stream));
-            RET(ks_digits_to_lifted(c, c1c, nb, digits, (int64_t)L * L1N, B, 0, nb, u, lifted));
-            RET(launch_moddown_combine(c, u, lifted, nb, B, 0, old, old_stride, inner + (b0 * G + g) * ctw, (int64_t)G * ctw, out,
-                                       out + LN, ctw));
-            old = out;
-            old_stride = ctw;
+    // Horner over the giant steps for blocks [b_lo, b_hi), as many blocks per round as the given part of the workspace
+    // holds, on the context's current stream
+    auto run_range = [&](int64_t b_lo, int64_t b_hi, char* wsp, int64_t wsp_bytes) -> int {
+        int64_t ch = (wsp_bytes - kSlack) / (ks_item_words(c) * 8);
+        if (ch < 1) return fail(c, HANN_EWORKSPACE, "hann_rotate_sum: workspace too small");
+        ch = std::min<int64_t>(std::min<int64_t>(ch, b_hi - b_lo), 8);
+        Arena ar{wsp, 0, wsp_bytes};
+        u64* c1c = ar.take<u64>(ch * LN);
+        u64* digits = ar.take<u64>(ch * L * L1N);
+        u64* u = ar.take<u64>(ch * 2 * L1N);
+        u64* lifted = ar.take<u64>(ch * 2 * LN);
+        u64* tmp = ar.take<u64>(ch * ctw);
+        if (!c1c || !digits || !u || !lifted || !tmp) return fail(c, HANN_EWORKSPACE, "hann_rotate_sum: workspace too small");
+        for (int64_t b0 = b_lo; b0 < b_hi; b0 += ch) {
+            const int64_t nb = std::min(ch, b_hi - b0);
+            const u64* old = inner + (b0 * G + (G - 1)) * ctw;  // acc = inner[G-1]
+            int64_t old_stride = (int64_t)G * ctw;
+            for (int g = G - 2; g >= 0; g--) {
+                u64* out = (g % 2 == 0) ? score + b0 * ctw : tmp;
+                // c1 of every accumulator, still in the transform domain; the key-switch round takes it from there
+                CK(cudaMemcpy2DAsync(c1c, LN * 8, old + LN, old_stride * 8, LN * 8, nb, cudaMemcpyDeviceToDevice, c->stream));
+                RET(ks_digits_to_lifted(c, c1c, nb, digits, (int64_t)L * L1N, B, 0, nb, u, lifted));
+                RET(launch_moddown_combine(c, u, lifted, nb, B, 0, old, old_stride, inner + (b0 * G + g) * ctw, (int64_t)G * ctw, out,
+                                           out + LN, ctw));
+                old = out;
+                old_stride = ctw;
+            }
         }
+        return HANN_OK;
+    };
+    // Blocks are independent: up to four ranges run side by side on the context's stream and the helper streams, each in
+    // its own part of the workspace, which keeps the machine busy through the many small launches of a key switch.
+    // (One lane while the per-launch profile is on, so that its kernel times do not overlap.)
+    int lanes = (int)std::min<int64_t>(4, n_blocks);
+    if (c->stream == c->aux_stream || c->kprof) lanes = 1;
+    while (lanes > 1 && (((int64_t)ws_bytes / lanes) & ~(int64_t)255) < ks_item_words(c) * 8 + kSlack) lanes--;
+    if (lanes <= 1) return run_range(0, n_blocks, (char*)ws, (int64_t)ws_bytes);
+    const int64_t part = ((int64_t)ws_bytes / lanes) & ~(int64_t)255;
+    cudaStream_t main_stream = c->stream;
+    cudaStream_t helper[3] = {c->aux_stream, c->lane_stream[0], c->lane_stream[1]};
+    cudaEvent_t joined[3] = {c->ev_join, c->lane_join[0], c->lane_join[1]};
+    CK(cudaEventRecord(c->ev_fork, main_stream));
+    int rc = HANN_OK;
+    cudaError_t ce = cudaSuccess;
+    for (int ln = 1; ln < lanes; ln++) {
+        const int64_t lo = n_blocks * ln / lanes, hi = n_blocks * (ln + 1) / lanes;
+        cudaError_t e = cudaStreamWaitEvent(helper[ln - 1], c->ev_fork, 0);
+        c->stream = helper[ln - 1];
+        const int r = e == cudaSuccess ? run_range(lo, hi, (char*)ws + ln * part, part) : HANN_ECUDA;
+        c->stream = main_stream;
+        if (e == cudaSuccess) e = cudaEventRecord(joined[ln - 1], helper[ln - 1]);
+        if (rc == HANN_OK) rc = r;
+        if (ce == cudaSuccess) ce = e;
     }
+    const int r0 = run_range(0, n_blocks / lanes, (char*)ws, part);
+    if (rc == HANN_OK) rc = r0;
+    // join every helper before reporting anything: no helper stream runs past this call unobserved
+    for (int ln = 1; ln < lanes; ln++) {
+        cudaError_t e = cudaStreamWaitEvent(main_stream, joined[ln - 1], 0);
+        if (ce == cudaSuccess) ce = e;
+    }
+    RET(rc);
+    CK(ce);
     return HANN_OK;
 }
 

@@ -25,6 +25,9 @@ struct hann_ctx {
     // helper stream and events of hann_query_level, which runs the query preparation beside the candidate encoding
     cudaStream_t aux_stream = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    // further helper streams: hann_rotate_sum runs independent block ranges side by side (aux_stream is lane 1)
+    cudaStream_t lane_stream[2] = {nullptr, nullptr};
+    cudaEvent_t lane_join[2] = {nullptr, nullptr};
     u64 mod[HANN_MAXL1] = {};  // q_0..q_{L-1}, p
     LimbTable lt = {};
     LimbConst* lt_dev = nullptr;  // device copy of lt.c (the transform kernels read it from memory)

@@ -148,8 +148,9 @@ def algorithmic_work(ctx, n_blocks, n_rows):
     lift_ops = sum(src * (1 + tgt) * a * (N // 2) * 8 for src, tgt in lift_src)
     return {
         "mac": ("hbm", n_blocks * R * L * W + B * 2 * L * W + n_blocks * G * 2 * L * W, n_blocks),
-        "ks_inner": ("hbm", (B - 1) * (L * 2 * (L + 1) * W + 2 * (L + 1) * W) + L * (L + 1) * W
-                     + (G - 1) * (L * 2 * (L + 1) * W + n_blocks * (L * (L + 1) * W + 2 * (L + 1) * W)), (B - 1) + items_rot),
+        # one digit set under B-1 streamed keys (query_prepare) / one key under many digit sets (rotate_sum, L2-resident key)
+        "ks_inner_keys": ("hbm", (B - 1) * (L * 2 * (L + 1) * W + 2 * (L + 1) * W) + L * (L + 1) * W, B - 1),
+        "ks_inner": ("hbm", (G - 1) * (L * 2 * (L + 1) * W + n_blocks * (L * (L + 1) * W + 2 * (L + 1) * W)), items_rot),
         "ntt_fwd_b": ("alu", fwd_polys * (N // 2) * b * 8, fwd_polys),
         "ntt_inv_b": ("alu", inv_polys * (N // 2) * b * 8, inv_polys),
         "lift_digits": ("alu", lift_ops, inv_polys),
@@ -282,7 +283,7 @@ def run_ours(args):
                 "traffic": per_unit * units / dom_launches if per_unit else None,
                 "traffic_source": ("ncu dram bytes per %s on the 1-block case x %s per launch" % (unit_name, unit_name)) if per_unit else None}
     hbm_kernels = {}
-    for k in ("mac", "ks_inner"):
+    for k in ("mac", "ks_inner_keys", "ks_inner"):
         if k in kernels:
             gbs = work[k][1] / (kernels[k]["ms_per_step"] * 1e-3) / 1e9
             hbm_kernels[k] = {"GB/s": gbs, "frac_of_measured_copy": gbs / hbm_peak, "frac_of_8TBps_nominal": gbs / 8000.0}

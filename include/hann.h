@@ -216,10 +216,12 @@ int hann_keyswitch_static(hann_ctx *ctx, int rot, const void *poly_dev, void *ks
 int hann_import(hann_ctx *ctx, int kind, const uint64_t *canonical, int64_t count, void *internal_dev);
 int hann_export(hann_ctx *ctx, int kind, const void *internal_dev, int64_t count, uint64_t *canonical_out);
 
-/* One level end to end from HOST buffers (copies included): import the canonical query ciphertext, prepare the baby
- * set, copy the rows to the device, encode, multiply-accumulate, rotate-and-sum, export the score ciphertexts to the
- * host in canonical layout.  Device buffers for the intermediates are carved from `ws_dev`, which must hold
- * hann_level_host_bytes(ctx, n_rows) bytes.
+/* One level end to end from HOST buffers (copies included): the rows are copied to the device block by block on a copy
+ * stream while the query ciphertext is imported and its baby set prepared on a helper stream; every block is encoded as
+ * soon as its rows have arrived; then multiply-accumulate, rotate-and-sum, and the score ciphertexts are exported to
+ * the host in canonical layout.  Page-locked host buffers are needed for the copies to overlap the kernels (pageable
+ * memory works but serialises).  Device buffers for the intermediates are carved from `ws_dev`, which must hold
+ * hann_level_host_bytes(ctx, n_rows) bytes.  Returns after everything has finished.
  *   ct_host [2][L][N];  rows_host [n_rows][dim] float32;  score_ct_host [ceil(n_rows/n)][2][L][N]. */
 int64_t hann_level_host_bytes(const hann_ctx *ctx, int64_t n_rows);
 int hann_score_level_host(hann_ctx *ctx, const uint64_t *ct_host, const float *rows_host, int64_t n_rows, int dim,

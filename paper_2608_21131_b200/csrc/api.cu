@@ -326,6 +326,7 @@ extern "C" void hann_ctx_destroy(hann_ctx* c) {
         }
         if (c->lane_join[i]) cudaEventDestroy(c->lane_join[i]);
     }
+    for (cudaEvent_t e : c->blk_ev) cudaEventDestroy(e);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_join) cudaEventDestroy(c->ev_join);
     for (auto& r : c->krec) {
@@ -408,7 +409,8 @@ extern "C" int hann_get_stats(hann_ctx* c, hann_stats* out) {
 }
 
 static const char* kKernelNames[KC_COUNT] = {"ntt_fwd_a", "ntt_fwd_b", "ntt_inv_b", "ntt_inv_a", "fft_a", "fft_b", "mac",
-                                             "lift_digits", "ks_inner", "moddown_lift", "moddown_combine", "permute", "other"};
+                                             "lift_digits", "ks_inner", "moddown_lift", "moddown_combine", "permute", "other",
+                                             "ks_inner_keys"};
 
 extern "C" int hann_kernel_classes(void) { return KC_COUNT; }
 extern "C" const char* hann_kernel_name(int cls) { return cls >= 0 && cls < KC_COUNT ? kKernelNames[cls] : ""; }
@@ -877,9 +879,44 @@ extern "C" int hann_score_level_host(hann_ctx* c, const uint64_t* ct_host, const
     u64* score = (u64*)b; b += p.score;
     u64* stage = (u64*)b; b += p.stage;
     void* ws = b;
-    CK(cudaMemcpyAsync(rows, rows_host, (size_t)n_rows * dim * 4, cudaMemcpyHostToDevice, c->stream));
-    RET(import_polys(c, ct_host, 2, ct));
-    RET(hann_query_level(c, ct, rows, n_rows, dim, baby, pt, inner, score, ws, (size_t)p.ws));
+    // Three streams: the rows travel block by block on a copy stream, the query is imported and its baby rotations are
+    // prepared on the helper stream, and the context's stream encodes each block as soon as its rows have arrived.
+    while ((int64_t)c->blk_ev.size() < p.nblk) {
+        cudaEvent_t e;
+        CK(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+        c->blk_ev.push_back(e);
+    }
+    const int64_t prep = c->B > 1 ? align256(prepare_words(c) * 8 + kSlack) : 0;
+    cudaStream_t main_stream = c->stream, copy_stream = c->lane_stream[1];
+    CK(cudaEventRecord(c->ev_fork, main_stream));
+    CK(cudaStreamWaitEvent(copy_stream, c->ev_fork, 0));
+    CK(cudaStreamWaitEvent(c->aux_stream, c->ev_fork, 0));
+    for (int64_t blk = 0; blk < p.nblk; blk++) {
+        const int64_t r0 = blk * c->n, rn = std::min<int64_t>(c->n, n_rows - r0);
+        CK(cudaMemcpyAsync(rows + r0 * dim, rows_host + r0 * dim, (size_t)rn * dim * 4, cudaMemcpyHostToDevice, copy_stream));
+        CK(cudaEventRecord(c->blk_ev[blk], copy_stream));
+    }
+    c->stream = c->aux_stream;
+    int rc = import_polys(c, ct_host, 2, ct);
+    if (rc == HANN_OK) rc = hann_query_prepare(c, ct, baby, ws, (size_t)prep);
+    c->stream = main_stream;
+    cudaError_t ej = cudaEventRecord(c->ev_join, c->aux_stream);
+    for (int64_t blk = 0; blk < p.nblk && rc == HANN_OK; blk++) {
+        const int64_t r0 = blk * c->n, rn = std::min<int64_t>(c->n, n_rows - r0);
+        if (cudaStreamWaitEvent(main_stream, c->blk_ev[blk], 0) != cudaSuccess) rc = fail(c, HANN_ECUDA, "cudaStreamWaitEvent failed");
+        if (rc == HANN_OK)
+            rc = hann_encode_candidates(c, rows + r0 * dim, rn, dim, pt + blk * (hann_sizeof(c, HANN_SIZE_PT_BLOCK) / 8), (char*)ws + prep,
+                                        (size_t)(p.ws - prep));
+    }
+    // join the helper streams before reporting anything
+    cudaError_t ew = cudaStreamWaitEvent(main_stream, c->ev_join, 0);
+    cudaError_t ew2 = cudaStreamWaitEvent(main_stream, c->blk_ev[p.nblk - 1], 0);
+    RET(rc);
+    CK(ej);
+    CK(ew);
+    CK(ew2);
+    RET(hann_score_level(c, baby, pt, p.nblk, inner, ws, (size_t)p.ws));
+    RET(hann_rotate_sum(c, inner, p.nblk, score, ws, (size_t)p.ws));
     RET(export_polys(c, score, p.nblk * 2, stage, score_ct_host));
     CK(cudaStreamSynchronize(c->stream));
     return HANN_OK;

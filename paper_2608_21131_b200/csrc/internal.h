@@ -13,7 +13,7 @@
 // kernel classes of the per-launch profile (hann_kernel_profile / hann_kernel_times)
 enum {
     KC_NTT_FWD_A = 0, KC_NTT_FWD_B, KC_NTT_INV_B, KC_NTT_INV_A, KC_FFT_A, KC_FFT_B, KC_MAC, KC_LIFT_DIGITS, KC_KS_INNER,
-    KC_MODDOWN_LIFT, KC_MODDOWN_COMBINE, KC_PERMUTE, KC_OTHER, KC_COUNT
+    KC_MODDOWN_LIFT, KC_MODDOWN_COMBINE, KC_PERMUTE, KC_OTHER, KC_KS_INNER_KEYS, KC_COUNT
 };
 
 struct hann_ctx {
@@ -28,6 +28,7 @@ struct hann_ctx {
     // further helper streams: hann_rotate_sum runs independent block ranges side by side (aux_stream is lane 1)
     cudaStream_t lane_stream[2] = {nullptr, nullptr};
     cudaEvent_t lane_join[2] = {nullptr, nullptr};
+    std::vector<cudaEvent_t> blk_ev;  // one event per block: hann_score_level_host encodes a block as soon as its rows arrived
     u64 mod[HANN_MAXL1] = {};  // q_0..q_{L-1}, p
     LimbTable lt = {};
     LimbConst* lt_dev = nullptr;  // device copy of lt.c (the transform kernels read it from memory)

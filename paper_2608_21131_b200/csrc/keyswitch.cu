@@ -189,32 +189,31 @@ __global__ void __launch_bounds__(kThreads) k_ks_inner(const u64* __restrict__ d
 // items share the key (rotate-and-sum over blocks), the key words stay and the digit words stream.  The streamed
 // words of the next item are in flight while the current item is multiplied.  Moduli below 2^50 use the carry-free
 // 25-bit Karatsuba products of the multiply-accumulate kernel; the special prime uses 128-bit accumulation.
-template <int LL, bool KEYS_STREAM>
-__global__ void __launch_bounds__(128) k_ks_inner_stream(const u64* __restrict__ digits, long long digit_stride,
-                                                         const u64* const* __restrict__ keytab, int rot0, int rot_inc,
-                                                         u64* __restrict__ u, int N, long long nitems, int items_per_cta,
-                                                         const LimbConst* __restrict__ lt) {
-    constexpr int NS = KEYS_STREAM ? 2 * LL : LL;  // streamed words per item
-    const long long L1N = (long long)(LL + 1) * N;
-    const long long pos = (long long)blockIdx.x * 128 + threadIdx.x;  // i*N + x
-    const int i = (int)(pos / N);
-    const LimbConst lc = lt[i];
-    const bool small = lc.q < (1ULL << 50);
-    const long long it0 = (long long)blockIdx.y * items_per_cta;
-    const long long it1 = it0 + items_per_cta < nitems ? it0 + items_per_cta : nitems;
-    if (it0 >= it1) return;
-    // stationary words
-    u64 st[KEYS_STREAM ? LL : 2 * LL];
+// MODE 0: moduli below 2^50, 25-bit halves, Karatsuba (3 products); MODE 1: moduli below 2^60 (the special prime),
+// 30-bit halves, 4 products (sums of 2 LL <= 8 products of 60 bits fit 64 bits); MODE 2: anything else, 128-bit
+// accumulation.
+template <int LL, bool KEYS_STREAM, int MODE>
+__device__ __forceinline__ void ks_inner_body(const u64* __restrict__ digits, long long digit_stride, const u64* const* __restrict__ keytab,
+                                              int rot0, int rot_inc, u64* __restrict__ u, long long L1N, long long pos, long long it0,
+                                              long long it1, const LimbConst& lc) {
+    constexpr int NS = KEYS_STREAM ? 2 * LL : LL;   // streamed words per item
+    constexpr int NST = KEYS_STREAM ? LL : 2 * LL;  // stationary words
+    constexpr int SH = MODE == 0 ? 25 : 30;
+    constexpr unsigned MASK = (1u << SH) - 1;
+    u64 st[NST];
     if (KEYS_STREAM) {
 #pragma unroll
         for (int j = 0; j < LL; j++) st[j] = digits[(long long)j * L1N + pos];
     } else {
         const u64* key = keytab[rot0];
 #pragma unroll
-        for (int j = 0; j < LL; j++) {
-            st[2 * j] = key[((long long)j * 2 + 0) * L1N + pos];
-            st[2 * j + 1] = key[((long long)j * 2 + 1) * L1N + pos];
-        }
+        for (int k = 0; k < NST; k++) st[k] = key[(long long)k * L1N + pos];  // k = j*2 + comp
+    }
+    unsigned s0[NST], s1[NST];
+#pragma unroll
+    for (int k = 0; k < NST; k++) {
+        s0[k] = (unsigned)st[k] & MASK;
+        s1[k] = (unsigned)(st[k] >> SH);
     }
     u64 cur[NS], nxt[NS];
     auto load = [&](long long item, u64(&v)[NS]) {
@@ -232,28 +231,33 @@ __global__ void __launch_bounds__(128) k_ks_inner_stream(const u64* __restrict__
     for (long long item = it0; item < it1; item++) {
         if (item + 1 < it1) load(item + 1, nxt);
         u64 out[2];
-        if (small) {
+        if (MODE != 2) {
             u64 p00[2] = {0, 0}, p11[2] = {0, 0}, pm[2] = {0, 0};
 #pragma unroll
             for (int j = 0; j < LL; j++)
 #pragma unroll
                 for (int c = 0; c < 2; c++) {
-                    const u64 dv = KEYS_STREAM ? st[j] : cur[j];
-                    const u64 kv = KEYS_STREAM ? cur[2 * j + c] : st[2 * j + c];
-                    const unsigned a0 = (unsigned)dv & kM25, a1 = (unsigned)(dv >> 25);
-                    const unsigned b0 = (unsigned)kv & kM25, b1 = (unsigned)(kv >> 25);
-                    p00[c] += (u64)a0 * b0;
-                    p11[c] += (u64)a1 * b1;
-                    pm[c] += (u64)(a0 + a1) * (b0 + b1);
+                    const int ks = KEYS_STREAM ? j : 2 * j + c;            // stationary word
+                    const u64 sv = KEYS_STREAM ? cur[2 * j + c] : cur[j];  // streamed word
+                    const unsigned b0 = (unsigned)sv & MASK, b1 = (unsigned)(sv >> SH);
+                    p00[c] += (u64)s0[ks] * b0;
+                    p11[c] += (u64)s1[ks] * b1;
+                    if (MODE == 0) {
+                        pm[c] += (u64)(s0[ks] + s1[ks]) * (b0 + b1);
+                    } else {
+                        pm[c] += (u64)s0[ks] * b1;
+                        pm[c] += (u64)s1[ks] * b0;
+                    }
                 }
 #pragma unroll
             for (int c = 0; c < 2; c++) {
-                const u64 cross = pm[c] - p00[c] - p11[c];
+                // value = p00 + cross * 2^SH + p11 * 2^(2 SH)
+                const u64 cross = MODE == 0 ? pm[c] - p00[c] - p11[c] : pm[c];
                 u64 lo = p00[c], hi = 0;
-                const u64 c_lo = cross << 25, c_hi = cross >> 39;
+                const u64 c_lo = cross << SH, c_hi = cross >> (64 - SH);
                 lo += c_lo;
                 hi += c_hi + (lo < c_lo ? 1 : 0);
-                const u64 d_lo = p11[c] << 50, d_hi = p11[c] >> 14;
+                const u64 d_lo = p11[c] << (2 * SH), d_hi = p11[c] >> (64 - 2 * SH);
                 lo += d_lo;
                 hi += d_hi + (lo < d_lo ? 1 : 0);
                 out[c] = reduce128(hi, lo, lc);
@@ -273,6 +277,23 @@ __global__ void __launch_bounds__(128) k_ks_inner_stream(const u64* __restrict__
 #pragma unroll
         for (int k = 0; k < NS; k++) cur[k] = nxt[k];
     }
+}
+
+template <int LL, bool KEYS_STREAM>
+__global__ void __launch_bounds__(128) k_ks_inner_stream(const u64* __restrict__ digits, long long digit_stride,
+                                                         const u64* const* __restrict__ keytab, int rot0, int rot_inc,
+                                                         u64* __restrict__ u, int N, long long nitems, int items_per_cta,
+                                                         const LimbConst* __restrict__ lt) {
+    const long long L1N = (long long)(LL + 1) * N;
+    const long long pos = (long long)blockIdx.x * 128 + threadIdx.x;  // i*N + x
+    const LimbConst lc = lt[pos / N];
+    const long long it0 = (long long)blockIdx.y * items_per_cta;
+    const long long it1 = it0 + items_per_cta < nitems ? it0 + items_per_cta : nitems;
+    if (it0 >= it1) return;
+    // a CTA lies inside one limb, so the choice is uniform
+    if (lc.q < (1ULL << 50)) ks_inner_body<LL, KEYS_STREAM, 0>(digits, digit_stride, keytab, rot0, rot_inc, u, L1N, pos, it0, it1, lc);
+    else if (lc.q < (1ULL << 60)) ks_inner_body<LL, KEYS_STREAM, 1>(digits, digit_stride, keytab, rot0, rot_inc, u, L1N, pos, it0, it1, lc);
+    else ks_inner_body<LL, KEYS_STREAM, 2>(digits, digit_stride, keytab, rot0, rot_inc, u, L1N, pos, it0, it1, lc);
 }
 
 // lifted[poly][i][x] = centred lift of up[poly][x] (residue mod p, coefficient domain) reduced mod q_i.
@@ -515,7 +536,7 @@ void launch_ks_inner_stream(hann_ctx* c, const u64* digits, int64_t digit_stride
     while ((long long)tiles * split < 148 * 8 && split < nitems) split *= 2;
     const int per = (int)((nitems + split - 1) / split);
     split = (int)((nitems + per - 1) / per);
-    KProf kp(c, KC_KS_INNER);
+    KProf kp(c, digit_stride == 0 && nitems > 1 ? KC_KS_INNER_KEYS : KC_KS_INNER);  // streamed keys timed on their own
     if (digit_stride == 0)
         k_ks_inner_stream<LL, true><<<dim3(tiles, split), 128, 0, c->stream>>>(digits, 0, c->keytab_dev, rot0, rot_inc, u, c->N, nitems,
                                                                             per, c->lt_dev);

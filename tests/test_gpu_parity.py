@@ -188,3 +188,56 @@ def test_error_codes():
     # the context stays usable after errors
     g.query_prepare(ct, ws)
     g.sync()
+
+
+# primes of the other arithmetic classes: [2^50, 2^57) runs the lazy integer transforms and the generic element-wise
+# kernels, >= 2^57 Harvey's butterflies; the special prime just below 2^62 is the largest the library accepts
+Q54 = (18014398506729473, 18014398505943041, 18014398496243713)
+Q58 = (288230376147386369,)
+P62 = 4611686018425815041
+
+
+@pytest.mark.parametrize(
+    "logN,q,p,R,B,n_rows",
+    [
+        (9, Q54[:2], synth.P60, 16, 4, 300),         # lazy-integer limbs + 60-bit special prime
+        (10, Q54, P62, 32, 8, 700),                   # three 54-bit limbs, 62-bit special prime (128-bit inner product)
+        (10, (synth.Q50[0], Q54[0]), P62, 16, 4, 512),  # binary64 and integer limbs side by side
+        (11, Q58 + Q54[:1], synth.P60, 64, 8, 1100),  # a 58-bit ciphertext prime (Harvey class)
+        (8, Q54[:2], P62, 8, 2, 200),                 # single-pass transforms with integer limbs
+    ],
+)
+def test_level_bit_exact_other_prime_classes(logN, q, p, R, B, n_rows):
+    ps = synth.ParamSet("classes", logN, tuple(q), p, 40, R, B, -18)
+    pr = Pair(ps, key_seed=logN)
+    rows = synth.toy_corpus(logN, rows=n_rows, dim=R)
+    qv = synth.toy_query(logN + 1, dim=R)
+    run_level(pr, rows, qv)
+    # and one key switch of an arbitrary polynomial under these moduli
+    rng = np.random.default_rng(1)
+    d = np.stack([rng.integers(0, m, size=ps.N, dtype=np.uint64) for m in ps.q])
+    ks0_o, ks1_o = pr.o.keyswitch(d, pr.evk_o[0])
+    ks0, ks1 = pr.g.keyswitch(1, pr.g.import_(pr.b.KIND_POLY, d[None], 1), pr.ws)
+    assert np.array_equal(pr.g.export(pr.b.KIND_POLY, ks0, 1)[0, 0], ks0_o)
+    assert np.array_equal(pr.g.export(pr.b.KIND_POLY, ks1, 1)[0, 0], ks1_o)
+
+
+def test_empty_and_single_row_levels():
+    import torch
+
+    ps = synth.small_params(10, 16, 4, L=2)
+    p = Pair(ps, key_seed=2)
+    g, b = p.g, p.b
+    # no rows: nothing to do, no error
+    empty = torch.zeros((0, 16), dtype=torch.float32, device=g.device)
+    pt = g.alloc(8)
+    g.encode_candidates(empty, p.ws, pt)
+    g.score_level(g.alloc(g.sizeof(b.SIZE_BABY)), pt, 0, p.ws, g.alloc(8))
+    g.rotate_sum(g.alloc(8), 0, p.ws, g.alloc(8))
+    g.sync()
+    # one row: a whole block is computed, slot 0 holds its score, every other slot is noise around zero
+    rows = synth.toy_corpus(5, rows=1, dim=16)
+    qv = synth.toy_query(6, dim=16)
+    got, score_g = run_level(p, rows, qv)
+    allslots = g.decrypt_scores(p.km.s, score_g)[0]
+    assert np.abs(allslots[1:]).max() < 2.0 ** ps.tol_log2

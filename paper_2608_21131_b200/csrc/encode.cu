@@ -267,6 +267,66 @@ __global__ void __launch_bounds__(128) k_fft_w(FusedArgs A) {
     }
 }
 
+// Kernel W for B >= 8: a CTA takes ONE chunk of 256 FFT positions for EIGHT plaintexts (g, b0 .. b0+7).  For a given
+// position the eight plaintexts read eight consecutive columns of the same candidate row, so the gather moves whole
+// 32-byte sectors instead of one float per sector, and all of a thread's 16 loads are independent.
+__global__ void __launch_bounds__(128) k_fft_w8(FusedArgs A) {
+    __shared__ double2 tc[256];
+    __shared__ double2 sm[8 * 272];
+    __shared__ float sin_[8 * 272];  // gathered inputs [plaintext][position + position/16]
+    const int n = 1 << A.logn;
+    const int P0 = blockIdx.y * 8;
+    const int g = (A.p_first + P0) / A.B, b0 = (A.p_first + P0) % A.B;
+    const int chunk = blockIdx.x;
+    for (int i = threadIdx.x; i < 255; i += 128) {
+        const int s = 32 - __clz(i + 1);
+        const int h = 1 << (s - 1), t = i - (h - 1);
+        tc[i] = A.T[(long long)t << (A.logn - s)];
+    }
+#pragma unroll
+    for (int i = 0; i < 16; i++) {
+        const int idx = threadIdx.x + 128 * i, p = idx >> 3, pl = idx & 7;
+        const int jj = A.jinv[(chunk << 8) + p];
+        int row = jj - g * A.B;
+        if (row < 0) row += n;
+        const int col = (jj + b0 + pl) % A.R;
+        sin_[pl * 272 + p + (p >> 4)] = (row < A.rows_in_block && col < A.dim) ? A.rows[(long long)row * A.dim + col] : 0.0f;
+    }
+    __syncthreads();
+    const int pl = threadIdx.x >> 4, j = threadIdx.x & 15;
+    {
+        double2 x[16];
+#pragma unroll
+        for (int e = 0; e < 16; e++) x[e] = make_double2((double)sin_[pl * 272 + 17 * j + e], 0.0);
+#pragma unroll
+        for (int s = 0; s < 4; s++) {
+            const int span = 1 << s;
+#pragma unroll
+            for (int e = 0; e < 16; e++)
+                if (!(e & span)) dit(x[e], x[e + span], tc[span - 1 + (e & (span - 1))]);
+        }
+        double2* d = sm + pl * 272 + 17 * j;
+#pragma unroll
+        for (int e = 0; e < 16; e++) d[e] = x[e];
+    }
+    __syncthreads();
+    {
+        double2 x[16];
+#pragma unroll
+        for (int e = 0; e < 16; e++) x[e] = sm[pl * 272 + 17 * e + j];
+#pragma unroll
+        for (int s = 0; s < 4; s++) {
+            const int span = 1 << s;
+#pragma unroll
+            for (int e = 0; e < 16; e++)
+                if (!(e & span)) dit(x[e], x[e + span], tc[16 * span - 1 + j + 16 * (e & (span - 1))]);
+        }
+        double2* o = A.buf + (long long)(P0 + pl) * n + ((long long)chunk << 8) + j;
+#pragma unroll
+        for (int e = 0; e < 16; e++) o[16 * e] = x[e];
+    }
+}
+
 // R1 + R2 = a = logN - 8 are the register rounds of the transform's pass A (R1 = min(a, 4)); the FFT's a - 1 strided
 // stages run as a first round of R2 stages and a last round of R1 - 1 stages
 template <int R1, int R2>
@@ -417,7 +477,10 @@ int launch_encode_rows_fused(hann_ctx* c, const float* rows, int64_t rows_in_blo
     A.lt = c->lt_dev;
     const int n = c->n, a = c->logN - 8;
     const int chunks = n >> 8;  // >= 1 because logN >= 9
-    if (chunks % kWChunks == 0) {
+    if (c->B % 8 == 0 && count % 8 == 0 && p_first % 8 == 0) {
+        KProf kp(c, KC_FFT_A);
+        k_fft_w8<<<dim3(chunks, count / 8), 128, 0, c->stream>>>(A);
+    } else if (chunks % kWChunks == 0) {
         KProf kp(c, KC_FFT_A);
         k_fft_w<<<dim3(chunks / kWChunks, count), 128, 0, c->stream>>>(A);
     } else {

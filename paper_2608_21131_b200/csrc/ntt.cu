@@ -530,8 +530,19 @@ void launch_fwd_class(hann_ctx* c, const NttArgs& A, int groups, bool skip_a) {
         cudaFuncSetAttribute(k_ntt_fwd_b8<AR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  // 50 KiB > default 48
         // enough CTAs for about four per SM; beyond that a CTA walks several tiles and reuses its staged twiddles
         const int ranges = (c->N >> 8) / kBK, ntiles = (groups + kBPG - 1) / kBPG;
-        int zs = (148 * 4 + ranges * A.nsel - 1) / (ranges * A.nsel);
-        zs = zs < 1 ? 1 : (zs > ntiles ? ntiles : zs);
+        // tiles per CTA: a CTA that walks several tiles stages its twiddles once, but the grid should still fill whole
+        // waves of the 148 x 3 resident CTAs.  Pick the split with the smallest (waves x tiles per CTA), ties to fewer CTAs.
+        const int slots = 148 * HANN_B8_MINBLOCKS, per = ranges * A.nsel;
+        int zs = 1;
+        long best = -1;
+        for (int z = 1; z <= ntiles && z <= 64; z++) {
+            const long waves = ((long)per * z + slots - 1) / slots, tiles = (ntiles + z - 1) / z;
+            const long cost = waves * (4 * tiles + 1);  // staging the twiddles costs about a quarter of a tile
+            if (best < 0 || cost < best) {
+                best = cost;
+                zs = z;
+            }
+        }
         k_ntt_fwd_b8<AR><<<dim3(ranges, A.nsel, zs), 256, smem, c->stream>>>(A, groups);
         return;
     }

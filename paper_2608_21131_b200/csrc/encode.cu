@@ -329,8 +329,11 @@ __global__ void __launch_bounds__(128) k_fft_w8(FusedArgs A) {
 
 // R1 + R2 = a = logN - 8 are the register rounds of the transform's pass A (R1 = min(a, 4)); the FFT's a - 1 strided
 // stages run as a first round of R2 stages and a last round of R1 - 1 stages
+#ifndef HANN_X_MINBLOCKS
+#define HANN_X_MINBLOCKS 2
+#endif
 template <int R1, int R2>
-__global__ void __launch_bounds__(256, 2) k_encode_x(FusedArgs A) {
+__global__ void __launch_bounds__(256, HANN_X_MINBLOCKS) k_encode_x(FusedArgs A) {
     extern __shared__ u64 smx[];
     constexpr int a = R1 + R2;
     constexpr int G1 = 1 << R2;        // row groups of transform round 1 = threads per column

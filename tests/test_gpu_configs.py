@@ -145,3 +145,51 @@ def test_sweep_level_with_padding_groups(logN, pair16):
     qR = synth.toy_query(wl.query_seed(0), dim=128)
     q = Query(p, qR)
     q.score_level(lvl.rows, oracle_blocks=(0,))
+
+
+def test_projection_under_encryption_then_scoring():
+    """Rank reduction under encryption (Sec. 3.1 "How"), in this build's plaintext-resident variant: the server holds the
+    512 -> 128 projection W in plaintext and applies it to the encrypted 512-dimensional query with the same diagonal
+    baby-step/giant-step scorer -- the "candidate block" is W^T tiled down the n slots, so slot i of the result holds
+    q_R[i mod 128], i.e. the projected query already tiled for the scoring levels.  The projected ciphertext (scale
+    Delta^2) is then used as the query of an ordinary level (result at scale Delta^3).  Both stages are compared with the
+    oracle bit for bit, the final scores with float64 within 2^-18."""
+    import torch
+
+    ps512 = synth.ParamSet("proj", 13, synth.Q50, synth.P60, 40, 512, 32, -18)
+    ps128 = ps512.with_(R=128)
+    pp, pc = Pair(ps512, key_seed=4), Pair(ps128, key_seed=4)
+    assert np.array_equal(pp.evk_g, pc.evk_g)  # same client, same keys: rotations 1..32 serve both stages
+    n = ps512.n
+    W = synth.projection_matrix(wl.PROJ_SEED, 512, 128)
+    q512 = synth.normalise(synth.gaussian_vectors(9, synth.S_QUERY, np.arange(1), 512))[0].astype(np.float32)
+    WT = np.ascontiguousarray(W.T.astype(np.float32))                 # [128][512]
+    block = np.ascontiguousarray(np.tile(WT, (n // 128, 1)))          # row i = W^T[i mod 128]
+    # stage 1: projection
+    ct_o, ct_g = pp.query(q512)
+    assert np.array_equal(ct_o, ct_g)
+    g, b = pp.g, pp.b
+    baby = g.query_prepare(g.import_(b.KIND_CT, ct_g, 1), pp.ws)
+    pt = g.encode_candidates(torch.from_numpy(block).to(g.device), pp.ws)
+    proj = g.rotate_sum(g.score_level(baby, pt, 1, pp.ws), 1, pp.ws)
+    g.sync()
+    proj_o, _, _ = pp.o.score_block(block, pp.o.baby_set(ct_o, pp.evk_o), pp.evk_o[31])
+    assert np.array_equal(g.export(b.KIND_CT, proj, 1)[0], proj_o)
+    qR = (WT.astype(np.float64) @ q512.astype(np.float64))
+    slots = g.decrypt_scores(pp.km.s, proj_o[None], log_scale_out=80)[0]
+    assert np.abs(slots - np.tile(qR, n // 128)).max() < 2.0 ** -20
+    # stage 2: an ordinary level with the projected ciphertext as its query (same ring, same keys, R = 128)
+    rows = synth.project_rows(synth.toy_corpus(7, rows=n + 500, dim=512).astype(np.float64), W, 128)
+    g2 = pc.g
+    baby2 = g2.query_prepare(proj, pc.ws)   # the device ciphertext of stage 1 is the query of stage 2
+    pt2 = g2.encode_candidates(torch.from_numpy(rows).to(g2.device), pc.ws)
+    score = g2.rotate_sum(g2.score_level(baby2, pt2, 2, pc.ws), 2, pc.ws)
+    g2.sync()
+    score_g = g2.export(b.KIND_CT, score, 2)
+    baby2_o = pc.o.baby_set(proj_o, pc.evk_o)
+    for blk in range(2):
+        sc_o, _, _ = pc.o.score_block(rows[blk * n:(blk + 1) * n], baby2_o, pc.evk_o[31])
+        assert np.array_equal(score_g[blk], sc_o)
+    got = g2.decrypt_scores(pc.km.s, score_g, log_scale_out=120).reshape(-1)[: rows.shape[0]]
+    want = rows.astype(np.float64) @ qR
+    assert np.abs(got - want).max() < 2.0 ** -18

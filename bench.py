@@ -102,7 +102,7 @@ def replica_throughput(units_per_rank, world, seconds_slowest):
     return world * units_per_rank / seconds_slowest
 
 
-def build_workload(config, rows_override=None):
+def build_workload(config, rows_override=None, logn=16):
     from paper_2608_21131_b200 import workloads as wl, synth
 
     if config == 0:
@@ -114,10 +114,10 @@ def build_workload(config, rows_override=None):
         return ps, lvl.rows, q, "face-like flat level: %d rows, dim 512->128, N=2^16, 4x50b+60b primes, scale 2^40" % n
     if config == 4:
         base = rows_override or (1 << 18)
-        ps, lvl = wl.sweep_level(base)
+        ps, lvl = wl.sweep_level(base, ps=synth.FULL15 if logn == 15 else synth.FULL16)
         q = synth.toy_query(wl.query_seed(0), dim=ps.R)
-        return ps, lvl.rows, q, "sweep: %d wanted rows inflated x4 to %d scored rows, dim 128, N=2^16" % (base, lvl.rows.shape[0])
-    raise SystemExit("bench.py times configs 0, 1 and 4; the hierarchy configs are exercised by the tests")
+        return ps, lvl.rows, q, "sweep: %d wanted rows inflated x4 to %d scored rows, dim 128, N=2^%d" % (base, lvl.rows.shape[0], ps.logN)
+    raise SystemExit("unknown config %r" % config)
 
 
 FP64_LANES_PER_SM = 64  # binary64 multiply-add lanes per SM per clock
@@ -175,7 +175,7 @@ def run_ours(args):
 
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    ps, rows_np, qR, wname = build_workload(args.config, args.rows)
+    ps, rows_np, qR, wname = build_workload(args.config, args.rows, args.logn)
     n_rows = rows_np.shape[0]
     ctx = binding.Context(ps, device=local)
     if args.encode_group:
@@ -364,6 +364,81 @@ def cpu_baseline(ps, rows_np, qR, km, n_rows):
                       "block time (per-block work is constant)" % (t_prep, nb, min(ps.n, n_rows), t_blk)}
 
 
+def run_hierarchy(args):
+    """Configs 2 and 3: the client-steered hierarchy (coarse -> fine -> rerank), one query after the other.  The timed
+    quantity is the server-side scoring of each level (rows resident in HBM, CUDA events); the client steps between the
+    levels (decrypt, rank, fetch the next candidates) are outside.  The baby rotations are prepared once per query and
+    reused by its three levels.  Prints one JSON line with the latency distribution per level."""
+    import torch
+    from paper_2608_21131_b200 import binding, synth, workloads as wl
+
+    torch.cuda.set_device(0)
+    cfg = wl.datacomp_like() if args.config == 2 else wl.deep1b_like()
+    ps = cfg.ps
+    ctx = binding.Context(ps, device=0)
+    km = synth.key_material(ps, wl.KEY_SEED)
+    ctx.load_keys(ctx.keygen_from_samples(km.s, km.rots, km.evk_a, km.evk_e), km.rots)
+    coarse = wl.coarse_level(cfg)
+    max_rows = max(len(coarse.ids), cfg.nprobe * cfg.h.fan, cfg.leaf_beam * cfg.h.leaf)
+    nb_max = ctx.n_blocks(max_rows)
+    ws = ctx.workspace(nb_max)
+    baby = ctx.alloc(ctx.sizeof(binding.SIZE_BABY))
+    pt = ctx.alloc(nb_max * ctx.sizeof(binding.SIZE_PT_BLOCK))
+    inner = ctx.alloc(nb_max * ctx.sizeof(binding.SIZE_INNER))
+    score = ctx.alloc(nb_max * ctx.sizeof(binding.SIZE_CT))
+    coarse_dev = torch.from_numpy(coarse.rows).to(ctx.device)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+
+    def timed(fn):
+        ev[0].record()
+        fn()
+        ev[1].record()
+        torch.cuda.synchronize()
+        return ev[0].elapsed_time(ev[1])
+
+    def level(rows_dev, n_rows):
+        nb = ctx.n_blocks(n_rows)
+        ms = timed(lambda: (ctx.encode_candidates(rows_dev, ws, pt), ctx.score_level(baby, pt, nb, ws, inner),
+                            ctx.rotate_sum(inner, nb, ws, score)))
+        sc = ctx.decrypt_scores(km.s, ctx.export(binding.KIND_CT, score, nb)).reshape(-1)[:n_rows]
+        return ms, sc
+
+    times = {"query_prepare": [], "coarse": [], "fine": [], "rerank": []}
+    rows_scored, hits, worst = 0, 0, 0.0
+    n_q = args.steps + args.warmup
+    for qi in range(n_q):
+        qR, planted = wl.hier_query(cfg, qi)
+        ct_dev = ctx.import_(binding.KIND_CT, ctx.encrypt_query(km.s, qR, km.ct_a, km.ct_e), 1)
+        t_prep = timed(lambda: ctx.query_prepare(ct_dev, ws, baby))
+        t_c, sc = level(coarse_dev, len(coarse.ids))
+        worst = max(worst, float(np.abs(sc - coarse.rows.astype(np.float64) @ qR.astype(np.float64)).max()))
+        fine = wl.fine_level(cfg, np.sort(wl.topk_ids(sc, coarse.ids, cfg.nprobe)))
+        t_f, sf = level(torch.from_numpy(fine.rows).to(ctx.device), len(fine.ids))
+        rer = wl.rerank_level(cfg, np.sort(wl.topk_ids(sf, fine.ids, cfg.leaf_beam)))
+        t_r, sr = level(torch.from_numpy(rer.rows).to(ctx.device), len(rer.ids))
+        worst = max(worst, float(np.abs(sr - rer.rows.astype(np.float64) @ qR.astype(np.float64)).max()))
+        if qi >= args.warmup:
+            for k, v in zip(("query_prepare", "coarse", "fine", "rerank"), (t_prep, t_c, t_f, t_r)):
+                times[k].append(v)
+            rows_scored += len(coarse.ids) + len(fine.ids) + len(rer.ids)
+            hits += int(planted in wl.topk_ids(sr, rer.ids, 10))
+    total_ms = sum(sum(v) for v in times.values())
+    pct = lambda v, p: float(np.percentile(v, p))
+    print(json.dumps({
+        "metric": METRIC, "value": rows_scored / (total_ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+        "config": {"workload": cfg.name + " hierarchy, one query at a time", "levels": {"coarse": len(coarse.ids), "fine": len(fine.ids),
+                                                                                        "rerank": len(rer.ids)},
+                   "logN": ps.logN, "L": ps.L, "R": ps.R, "B": ps.B},
+        "ms_per_query_level": {k: {"p50": pct(v, 50), "p95": pct(v, 95)} for k, v in times.items()},
+        "ms_per_query": {"p50": pct(np.sum(list(times.values()), axis=0), 50), "p95": pct(np.sum(list(times.values()), axis=0), 95)},
+        "planted_neighbour_in_top10": hits / args.steps,
+        "check": {"max_abs_score_error": worst, "tolerance": 2.0 ** ps.tol_log2, "ok": bool(worst < 2.0 ** ps.tol_log2)},
+    }))
+    return 0
+
+
 def run_reference(args):
     """reference arm: the CPU oracle, unmodified, on the host cores; a step is query_prepare + one block"""
     rank = int(os.environ.get("RANK", "0"))
@@ -372,7 +447,7 @@ def run_reference(args):
         return 0
     from paper_2608_21131_b200 import synth, workloads as wl
 
-    ps, rows_np, qR, wname = build_workload(args.config, args.rows)
+    ps, rows_np, qR, wname = build_workload(args.config, args.rows, args.logn)
     n_rows = rows_np.shape[0]
     km = synth.key_material(ps, wl.KEY_SEED)
     o, ct, evk = oracle_setup(ps, qR, km)
@@ -406,7 +481,9 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=1)
+    ap.add_argument("--config", type=int, default=1, help="0 toy, 1 face-like level (default), 2 DataComp-like and 3 Deep1B-like "
+                    "hierarchies (latency per level), 4 scaling sweep point (--rows = wanted rows, --logn 15|16)")
+    ap.add_argument("--logn", type=int, default=16, help="ring of the sweep configuration")
     ap.add_argument("--rows", type=int, default=None, help="override the row count (debugging, ncu captures)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--encode-group", type=int, default=None, help="tuning: plaintexts per encode launch group")
@@ -416,6 +493,10 @@ def main():
         args.steps = 2 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup
         return run_reference(args)
+    if args.config in (2, 3):
+        args.steps = (16 if args.config == 2 else 64) if args.steps is None else args.steps
+        args.warmup = 2 if args.warmup is None else args.warmup
+        return run_hierarchy(args)
     args.steps = 200 if args.steps is None else args.steps
     args.warmup = 20 if args.warmup is None else args.warmup
     return run_ours(args)

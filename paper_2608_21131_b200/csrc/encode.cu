@@ -412,11 +412,11 @@ __global__ void __launch_bounds__(256, HANN_X_MINBLOCKS) k_encode_x(FusedArgs A)
             double x[1 << R1];
 #pragma unroll
             for (int e = 0; e < (1 << R1); e++) x[e] = ar.reduce(m[e]);
-            fwd_round<R1>(ar, x, tw, 1u);
+            fwd_round<R1, ArithF64, R1>(ar, x, tw, 1u);
 #pragma unroll
             for (int e = 0; e < (1 << R1); e++) {
                 if (R2 == 0) base[(size_t)(g + G1 * e) * 256 + c] = ar.to_mid(x[e]);
-                else smx[((g + G1 * e) << 4) + c] = ar.to_mid(x[e]);
+                else smx[((g + G1 * e) << 4) + c] = ar.to_exch(x[e]);
             }
         }
         if (R2 > 0) {
@@ -426,7 +426,7 @@ __global__ void __launch_bounds__(256, HANN_X_MINBLOCKS) k_encode_x(FusedArgs A)
                 double x[1 << RR2];
 #pragma unroll
                 for (int e = 0; e < (1 << RR2); e++) x[e] = ar.from_mid(smx[(((gg << RR2) + e) << 4) + cc]);
-                fwd_round<RR2>(ar, x, tw, (unsigned)(G2 + gg));
+                fwd_round<RR2, ArithF64, 5 - R1>(ar, x, tw, (unsigned)(G2 + gg));
 #pragma unroll
                 for (int e = 0; e < (1 << RR2); e++) base[(size_t)((gg << RR2) + e) * 256 + cc] = ar.to_mid(x[e]);
             }

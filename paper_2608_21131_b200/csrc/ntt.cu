@@ -16,10 +16,16 @@
 // Arithmetic.  Three exact implementations of the same modular butterflies, chosen per limb by the size of q:
 //   * q < 2^50: binary64.  Residues are held as balanced integers in doubles; a product y*w mod q is
 //       h = fl(y*w), l = fma(y, w, -h), c = rint(y * fl(w/q)), t = fma(-c, q, h) + l
-//     which is exact (t = y*w - c*q, |t| <= 1.5 q) while |y| <= 8 q; a round of at most 4 stages grows a value by
-//     at most 6 q (forward) or to 8 times its size (inverse, from |x| <= q/2), so reducing every value at the end of
-//     each round keeps every intermediate an integer below 2^53.  The FP64 pipe sustains about twice the
-//     butterflies per second of the integer pipe, which has no native 64-bit multiply.
+//     which is exact (t = y*w - c*q) while |y| <= 8q, with |t| <= (1/2 + k/8) q for |y| <= k q (the quotient estimate
+//     is off by at most k/8 before rounding).  A forward stage maps values bounded by b q to values bounded by
+//     (b + 1/2 + b/8) q: from reduced inputs (b = 1/2) eight stages reach 1.06, 1.70, 2.41, 3.21, 4.11, 5.12, 6.26,
+//     7.55 -- below 8, so a whole pass of eight stages runs without a reduction and every intermediate stays an
+//     integer below 2^53; from inputs in (-q, q) (b = 1) four stages reach 4.0.  While the multiplied value is
+//     below 4q (the first five stages from reduced inputs) the quotient is rounded inside a multiply-add with
+//     1.5 * 2^52 on the FP64 pipe; the later stages use the conversion unit's rint, which runs beside that pipe.
+//     An inverse stage doubles a bound, so inverse rounds have at most 4 stages from |x| <= q/2.  Conversions between
+//     integers below 2^52 and doubles go through the mantissa of 2^52 + v.  The FP64 pipe sustains about twice
+//     the butterflies per second of the integer pipe, which has no native 64-bit multiply.
 //   * q < 2^57: 64-bit integers, Shoup multiplication, no correction inside a forward transform (a value grows by
 //     at most 2q per stage, 16 stages stay below 33q < 2^63), one chain of conditional subtractions at the end.
 //   * otherwise (the ~60-bit special prime): Harvey's lazy butterflies in [0, 4q).
@@ -224,22 +230,22 @@ __global__ void __launch_bounds__(256, HANN_B8_MINBLOCKS) k_ntt_fwd_b8(NttArgs A
             typename AR::T x[16];
 #pragma unroll
             for (int e = 0; e < 16; e++) x[e] = ar.from_mid(raw[e]);
-            fwd_round_f<4>(ar, x, [=](int st, int il) { return tcc[(1 << st) - 1 + il]; });
+            fwd_round_f<4, AR, 4>(ar, x, [=](int st, int il) { return tcc[(1 << st) - 1 + il]; });
 #pragma unroll
-            for (int e = 0; e < 16; e++) s1[17 * e + j] = ar.to_mid(x[e]);
+            for (int e = 0; e < 16; e++) s1[17 * e + j] = ar.to_exch(x[e]);
         }
-        __syncthreads();
+        __syncwarp();  // the exchange tile of a chunk is private to the 16 lanes that transform it
         if (valid) {
             typename AR::T x[16];
 #pragma unroll
             for (int e = 0; e < 16; e++) x[e] = ar.from_mid(s1[17 * j + e]);
-            fwd_round_f<4>(ar, x, [=](int u, int il) { return tcc[(((1 << u) + il) << 4) + j]; });
+            fwd_round_f<4, AR, 1>(ar, x, [=](int u, int il) { return tcc[(((1 << u) + il) << 4) + j]; });
             // logical position 16 j + e goes to word 16 e + j of the chunk (nibble-swapped layout): the 16 threads of a
             // chunk write 128 contiguous bytes per store
 #pragma unroll
             for (int e = 0; e < 16; e++) base[16 * e + j] = ar.to_canonical(x[e]);
         }
-        __syncthreads();  // round 2 has read the exchange tile; the next tile may overwrite it
+        __syncwarp();  // round 2 has read the exchange tile; the next tile may overwrite it
 #pragma unroll
         for (int e = 0; e < 16; e++) raw[e] = nxt[e];
         base += (long long)gridDim.z * tile_stride;
@@ -386,7 +392,10 @@ __device__ __forceinline__ void lift_inverse(const LiftArgs& A, const AR ar, con
     }
 }
 
-__device__ __forceinline__ double lifted_value(const ArithF64&, u64 r, bool neg, u64 q) { return neg ? -(double)r : (double)r; }
+__device__ __forceinline__ double lifted_value(const ArithF64& ar, u64 r, bool neg, u64 q) {
+    const double d = ar.from_canonical(r);
+    return neg ? -d : d;
+}
 template <bool S>
 __device__ __forceinline__ u64 lifted_value(const ArithInt<S>&, u64 r, bool neg, u64 q) { return (neg && r) ? q - r : r; }
 
@@ -405,7 +414,7 @@ __device__ __forceinline__ void lift_forward(const AR ar, const LimbConst* lc, b
             const u64 mag = neg ? src_q - v[e] : v[e];
             x[e] = same_modulus ? ar.from_canonical(v[e]) : lifted_value(ar, barrett64(mag, *lc), neg, lc->q);
         }
-        fwd_round<R1>(ar, x, tw, 1u);
+        fwd_round<R1, AR, R1>(ar, x, tw, 1u);
 #pragma unroll
         for (int e = 0; e < (1 << R1); e++) {
             if (R2 == 0) base[(size_t)(g + G1 * e) * 256 + c] = ar.to_mid(x[e]);
@@ -419,7 +428,7 @@ __device__ __forceinline__ void lift_forward(const AR ar, const LimbConst* lc, b
             typename AR::T x[1 << RR2];
 #pragma unroll
             for (int e = 0; e < (1 << RR2); e++) x[e] = ar.from_mid(sm[(((gg << RR2) + e) << 4) + cc]);
-            fwd_round<RR2>(ar, x, tw, (unsigned)(G2 + gg));
+            fwd_round<RR2, AR, RR2>(ar, x, tw, (unsigned)(G2 + gg));
 #pragma unroll
             for (int e = 0; e < (1 << RR2); e++) base[(size_t)((gg << RR2) + e) * 256 + cc] = ar.to_mid(x[e]);
         }

@@ -17,26 +17,50 @@ struct ArithF64 {
     typedef double2 TW;
     double q, qinv, half;
     static constexpr int kMinBlocks = HANN_F64_MINBLOCKS;
+    static constexpr double kRound = 6755399441055744.0;  // 1.5 * 2^52: fl(v + kRound) - kRound = rint(v) for |v| < 2^51
+    static constexpr double kTwo52 = 4503599627370496.0;
     TW ninv;
     __device__ __forceinline__ ArithF64(const LimbConst* lc)
         : q((double)lc->q), qinv(1.0 / (double)lc->q), half((double)lc->half), ninv(make_double2(lc->ninv_bal, lc->ninv_q)) {}
-    __device__ __forceinline__ T reduce(T x) const { return __fma_rn(-rint(__dmul_rn(x, qinv)), q, x); }
+    // x - round(x/q) q; the quotient (at most 8 in magnitude) is rounded by adding 1.5 * 2^52
+    __device__ __forceinline__ T reduce(T x) const {
+        return __fma_rn(-__dsub_rn(__fma_rn(x, qinv, kRound), kRound), q, x);
+    }
     __device__ __forceinline__ T mulmod(T y, TW w) const {
         const double h = __dmul_rn(y, w.x);
         const double l = __fma_rn(y, w.x, -h);
         const double c = rint(__dmul_rn(y, w.y));
         return __dadd_rn(__fma_rn(-c, q, h), l);
     }
-    __device__ __forceinline__ T from_canonical(u64 v) const { return __ull2double_rn(v); }
+    // the same product for |y| < 4q: |y * w/q| < 2^51, so the quotient can be rounded on the FP64 pipe by adding
+    // 1.5 * 2^52 inside the multiply-add (one rounding less than above, and no trip through the conversion unit)
+    __device__ __forceinline__ T mulmod_small(T y, TW w) const {
+        const double h = __dmul_rn(y, w.x);
+        const double l = __fma_rn(y, w.x, -h);
+        const double c = __dsub_rn(__fma_rn(y, w.y, kRound), kRound);
+        return __dadd_rn(__fma_rn(-c, q, h), l);
+    }
+    // integers below 2^52 <-> binary64 through the mantissa of 2^52 + v (one add and one logic operation)
+    __device__ __forceinline__ T from_canonical(u64 v) const {
+        return __dsub_rn(__longlong_as_double((long long)(v | 0x4330000000000000ULL)), kTwo52);
+    }
     __device__ __forceinline__ T from_mid(u64 v) const { return __longlong_as_double((long long)v); }
     __device__ __forceinline__ u64 to_mid(T x) const { return (u64)__double_as_longlong(reduce(x)); }
+    // exchange between the two rounds of a forward pass that started from reduced values: no reduction (eight stages
+    // stay below 8q, see ntt.cu)
+    __device__ __forceinline__ u64 to_exch(T x) const { return (u64)__double_as_longlong(x); }
     __device__ __forceinline__ u64 to_canonical(T x) const {
         x = reduce(x);
         if (x < 0.0) x += q;
-        return __double2ull_rn(x);
+        return (u64)__double_as_longlong(__dadd_rn(x, kTwo52)) & 0x000FFFFFFFFFFFFFULL;
     }
     __device__ __forceinline__ void fwd(T& X, T& Y, TW w) const {
         const T t = mulmod(Y, w);
+        Y = __dsub_rn(X, t);
+        X = __dadd_rn(X, t);
+    }
+    __device__ __forceinline__ void fwd_small(T& X, T& Y, TW w) const {  // |Y| < 4q
+        const T t = mulmod_small(Y, w);
         Y = __dsub_rn(X, t);
         X = __dadd_rn(X, t);
     }
@@ -47,7 +71,7 @@ struct ArithF64 {
     }
     // inverse transforms start from balanced values so that four doubling stages stay below 2^53
     __device__ __forceinline__ T inv_input(u64 v) const {
-        const double x = __ull2double_rn(v);
+        const double x = from_canonical(v);
         return x > half ? x - q : x;
     }
     __device__ __forceinline__ u64 scaled_output(T x, TW ninv_pair) const { return to_canonical(mulmod(reduce(x), ninv_pair)); }
@@ -64,6 +88,7 @@ struct ArithInt {
     __device__ __forceinline__ T from_canonical(u64 v) const { return v; }
     __device__ __forceinline__ T from_mid(u64 v) const { return v; }
     __device__ __forceinline__ u64 to_mid(T x) const { return x; }
+    __device__ __forceinline__ u64 to_exch(T x) const { return x; }
     __device__ __forceinline__ u64 to_canonical(T v) const {  // forward results: [0, 33q) or [0, 4q)
         if (SMALLQ) {
             v = csub(v, 32 * q);
@@ -81,6 +106,7 @@ struct ArithInt {
         X = x + t;
         Y = x - t + q2;
     }
+    __device__ __forceinline__ void fwd_small(T& X, T& Y, TW w) const { fwd(X, Y, w); }
     __device__ __forceinline__ void inv(T& X, T& Y, TW w) const {  // [0, 2q) in and out
         const u64 x = X, y = Y;
         X = csub(x + y, q2);
@@ -92,7 +118,9 @@ struct ArithInt {
 
 // ---- register rounds -----------------------------------------------------------------------------------------
 
-template <int R, class AR>
+// NS: the first NS stages of the round see inputs below 4q (binary64 arithmetic then rounds its quotients on the FP64
+// pipe instead of the conversion unit); 0 is always correct
+template <int R, class AR, int NS = 0>
 __device__ __forceinline__ void fwd_round(const AR& ar, typename AR::T (&x)[1 << R], const typename AR::TW* __restrict__ tw,
                                           unsigned base) {
 #pragma unroll
@@ -104,7 +132,8 @@ __device__ __forceinline__ void fwd_round(const AR& ar, typename AR::T (&x)[1 <<
 #pragma unroll
             for (int jj = 0; jj < span; jj++) {
                 const int e = il * 2 * span + jj;
-                ar.fwd(x[e], x[e + span], w);
+                if (s < NS) ar.fwd_small(x[e], x[e + span], w);
+                else ar.fwd(x[e], x[e + span], w);
             }
         }
     }
@@ -112,7 +141,7 @@ __device__ __forceinline__ void fwd_round(const AR& ar, typename AR::T (&x)[1 <<
 
 // the same round with the twiddle of (stage s, group il) supplied by a functor (shared-memory caches with their own
 // layout)
-template <int R, class AR, class TWF>
+template <int R, class AR, int NS = 0, class TWF>
 __device__ __forceinline__ void fwd_round_f(const AR& ar, typename AR::T (&x)[1 << R], const TWF& twf) {
 #pragma unroll
     for (int s = 0; s < R; s++) {
@@ -123,7 +152,8 @@ __device__ __forceinline__ void fwd_round_f(const AR& ar, typename AR::T (&x)[1 
 #pragma unroll
             for (int jj = 0; jj < span; jj++) {
                 const int e = il * 2 * span + jj;
-                ar.fwd(x[e], x[e + span], w);
+                if (s < NS) ar.fwd_small(x[e], x[e + span], w);
+                else ar.fwd(x[e], x[e + span], w);
             }
         }
     }

@@ -269,7 +269,7 @@ extern "C" int hann_ctx_create(const hann_params* prm, hann_ctx** out) {
     const size_t twb = (size_t)(L + 1) * N * 16;
     bool ok = cudaMalloc(&c->tw_fwd, twb) == cudaSuccess && cudaMalloc(&c->tw_inv, twb) == cudaSuccess &&
               cudaMalloc(&c->tw_fwd_f64, twb) == cudaSuccess && cudaMalloc(&c->tw_inv_f64, twb) == cudaSuccess &&
-              cudaMalloc(&c->lt_dev, sizeof(LimbTable)) == cudaSuccess &&
+              cudaMalloc(&c->lt_dev, sizeof(LimbTable)) == cudaSuccess && cudaMalloc(&c->kflag, sizeof(int)) == cudaSuccess &&
               cudaMalloc(&c->fft_T, nh * sizeof(double2)) == cudaSuccess && cudaMalloc(&c->fft_U, n * sizeof(double2)) == cudaSuccess &&
               cudaMalloc(&c->jinv, n * sizeof(int32_t)) == cudaSuccess && cudaMalloc(&c->galois_dev, n * sizeof(unsigned)) == cudaSuccess &&
               cudaMalloc(&c->keytab_dev, n * sizeof(u64*)) == cudaSuccess;
@@ -279,6 +279,7 @@ extern "C" int hann_ctx_create(const hann_params* prm, hann_ctx** out) {
              cudaMemcpy(c->tw_fwd_f64, twf64.data(), twb, cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->tw_inv_f64, twi64.data(), twb, cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->lt_dev, &c->lt, sizeof(LimbTable), cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemset(c->kflag, 0, sizeof(int)) == cudaSuccess &&
              cudaMemcpy(c->fft_T, T.data(), nh * sizeof(double2), cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->fft_U, U.data(), n * sizeof(double2), cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->jinv, jpos.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess &&
@@ -312,7 +313,7 @@ extern "C" void hann_ctx_destroy(hann_ctx* c) {
     cudaStreamSynchronize(c->stream);
     for (u64* k : c->keytab_host)
         if (k) cudaFree(k);
-    cudaFree(c->tw_fwd); cudaFree(c->tw_inv); cudaFree(c->tw_fwd_f64); cudaFree(c->tw_inv_f64); cudaFree(c->lt_dev);
+    cudaFree(c->tw_fwd); cudaFree(c->tw_inv); cudaFree(c->tw_fwd_f64); cudaFree(c->tw_inv_f64); cudaFree(c->lt_dev); cudaFree(c->kflag);
     cudaFree(c->fft_T); cudaFree(c->fft_U); cudaFree(c->jinv); cudaFree(c->galois_dev); cudaFree(c->keytab_dev);
     if (c->scratch) cudaFree(c->scratch);
     if (c->aux_stream) {
@@ -371,6 +372,12 @@ extern "C" int hann_sync(hann_ctx* c) {
     if (!c) return HANN_EINVAL;
     DeviceGuard dg(c->device);
     CK(cudaStreamSynchronize(c->stream));
+    int flag = 0;
+    CK(cudaMemcpy(&flag, c->kflag, sizeof(int), cudaMemcpyDeviceToHost));
+    if (flag) {
+        cudaMemset(c->kflag, 0, sizeof(int));
+        return fail(c, HANN_ECUDA, "a kernel gave up a bounded wait for an asynchronous copy; results of the last calls are invalid");
+    }
     return HANN_OK;
 }
 

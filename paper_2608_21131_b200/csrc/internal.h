@@ -32,6 +32,7 @@ struct hann_ctx {
     u64 mod[HANN_MAXL1] = {};  // q_0..q_{L-1}, p
     LimbTable lt = {};
     LimbConst* lt_dev = nullptr;  // device copy of lt.c (the transform kernels read it from memory)
+    int* kflag = nullptr;         // device word raised by a kernel that gave up a bounded wait; read by hann_sync
     // transform tables on the device, [L+1][N][2]: (w, floor(w*2^64/q)) for w = psi^brev(k) and psi^-brev(k)
     u64 *tw_fwd = nullptr, *tw_inv = nullptr;
     // the same twiddles for the binary64 transform path, [L+1][N][2] doubles: (balanced w, fl(w / q))

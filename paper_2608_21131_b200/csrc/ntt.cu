@@ -252,6 +252,137 @@ __global__ void __launch_bounds__(256, HANN_B8_MINBLOCKS) k_ntt_fwd_b8(NttArgs A
     }
 }
 
+// The same pass with the words brought in by bulk asynchronous copies.  A warp owns the two chunks of ONE polynomial
+// (4 KiB, contiguous in memory) and runs its own two-deep pipeline: lane 0 starts the copy of the warp's tile after next
+// into the buffer the warp has just finished with, completion is signalled on a per-buffer mbarrier, and no warp ever
+// waits for another (the only CTA-wide barrier follows the staging of the twiddles).  The prefetched words therefore
+// occupy no registers.  The two rounds exchange IN PLACE in the landing buffer: position 16 r + c of a chunk is kept at
+// word 16 r + (c ^ r), which makes the column reads and writes of round 1 and the row reads of round 2 conflict-free
+// without padding.  Every wait on an mbarrier is bounded; a warp whose wait runs out raises the context's kernel flag
+// and stops.
+constexpr int kTK = 2, kTP = 8;       // chunks per CTA, polynomials per tile (= warps per CTA)
+constexpr unsigned long long kWaitLimitNs = 1000000000ULL;
+
+__device__ __forceinline__ unsigned smem_addr(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_load(unsigned dst, const void* src, unsigned bytes, unsigned bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src),
+                 "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// bounded: gives up (false) one second after the first unsuccessful probe
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity) {
+    unsigned long long t0 = 0;
+    for (unsigned it = 0;; it++) {
+        unsigned ok;
+        asm volatile(
+            "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+        if ((it & 63) == 0) {
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) return false;
+        }
+    }
+}
+
+template <class AR>
+__global__ void __launch_bounds__(256, 3) k_ntt_fwd_b8t(NttArgs A, int groups, int* kflag) {
+    extern __shared__ __align__(128) u64 smraw[];
+    typedef typename AR::TW TW;
+    TW* tc = (TW*)smraw;                                 // twiddle cache [kTK][256], layout as in k_ntt_fwd_b8
+    u64* bufs = smraw + kTK * 256 * 2;                   // [kTP][2][512] landing / exchange buffers
+    u64* bars = bufs + kTP * 2 * 512;                    // [kTP][2] mbarriers
+    const int k = blockIdx.y;
+    const int pos = (int)((A.pos4 >> (4 * k)) & 15), limb = (int)((A.limb4 >> (4 * k)) & 15);
+    const AR ar(A.lt + limb);
+    const int chunk0 = blockIdx.x * kTK;
+    const TW* tw = (const TW*)A.tw + ((size_t)limb << A.logN);
+    const unsigned m0 = 1u << A.a;
+    const int t = threadIdx.x >> 5, lane = threadIdx.x & 31, ch = lane >> 4, j = lane & 15;
+    const int ntiles = (groups + kTP - 1) / kTP;
+    const long long tile_stride = (long long)kTP * A.period * A.stride;
+    u64* wbuf = bufs + t * 1024;
+    const unsigned bar0 = smem_addr(bars + t * 2), buf0 = smem_addr(wbuf);
+    if (lane == 0) {
+        mbar_init(bar0, 1);
+        mbar_init(bar0 + 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    // tiles of this CTA: blockIdx.z, blockIdx.z + gridDim.z, ..; this warp's polynomial in tile yg is yg * kTP + t
+    const int yg0 = blockIdx.z, ystep = gridDim.z;
+    u64* gbase = A.data + (((long long)yg0 * kTP + t) * A.period + pos) * A.stride + ((size_t)chunk0 << 8);
+    const int my_tiles = yg0 < ntiles ? (ntiles - yg0 + ystep - 1) / ystep : 0;
+    // tile i of this warp is valid when its polynomial exists (only the last tile can be ragged)
+    auto tile_valid = [&](int i) { return i < my_tiles && (long long)(yg0 + (long long)i * ystep) * kTP + t < groups; };
+    if (lane == 0) {
+        for (int i = 0; i < 2; i++)
+            if (tile_valid(i)) {
+                mbar_expect_tx(bar0 + 8 * i, 4096);
+                bulk_load(buf0 + 4096 * i, gbase + (long long)i * ystep * tile_stride, 4096, bar0 + 8 * i);
+            }
+    }
+    for (int i = threadIdx.x; i < kTK * 256; i += 256) {
+        const int c2 = i >> 8, e = i & 255;
+        if (e < 15) {
+            const int st = 31 - __clz(e + 1), il = e + 1 - (1 << st);
+            tc[i] = tw[((m0 + (unsigned)(chunk0 + c2)) << st) + il];
+        } else if (e >= 16) {
+            const int jj = e & 15, r = (e >> 4) - 1;
+            const int u = 31 - __clz(r + 1), il = r + 1 - (1 << u);
+            tc[i] = tw[((m0 + (unsigned)(chunk0 + c2)) << (4 + u)) + (jj << u) + il];
+        }
+    }
+    __syncthreads();
+    const TW* tcc = tc + ch * 256;
+    for (int i = 0; i < my_tiles; i++) {
+        if (!tile_valid(i)) break;  // warp-uniform
+        const int s = i & 1;
+        if (!mbar_wait(bar0 + 8 * s, (unsigned)(i >> 1) & 1u)) {
+            if (lane == 0) atomicExch(kflag, 1);
+            // the copy into the other buffer may still be in flight: give it the same bounded time, then stop
+            if (tile_valid(i + 1)) mbar_wait(bar0 + 8 * (s ^ 1), (unsigned)((i + 1) >> 1) & 1u);
+            return;
+        }
+        u64* sb = wbuf + s * 512 + ch * 256;
+        typename AR::T x[16];
+#pragma unroll
+        for (int e = 0; e < 16; e++) x[e] = ar.from_mid(sb[j + 16 * e]);
+        __syncwarp();  // every lane holds its words: the buffer may be overwritten
+        fwd_round_f<4, AR, 4>(ar, x, [=](int st, int il) { return tcc[(1 << st) - 1 + il]; });
+#pragma unroll
+        for (int e = 0; e < 16; e++) sb[16 * e + (j ^ e)] = ar.to_exch(x[e]);
+        __syncwarp();
+#pragma unroll
+        for (int e = 0; e < 16; e++) x[e] = ar.from_mid(sb[16 * j + (e ^ j)]);
+        fwd_round_f<4, AR, 1>(ar, x, [=](int u, int il) { return tcc[(((1 << u) + il) << 4) + j]; });
+        u64* go = gbase + (long long)i * ystep * tile_stride + ((size_t)ch << 8);
+#pragma unroll
+        for (int e = 0; e < 16; e++) go[16 * e + j] = ar.to_canonical(x[e]);
+        // order this warp's shared-memory accesses before the asynchronous copy that refills the buffer
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0 && tile_valid(i + 2)) {
+            mbar_expect_tx(bar0 + 8 * s, 4096);
+            bulk_load(buf0 + 4096 * s, gbase + (long long)(i + 2) * ystep * tile_stride, 4096, bar0 + 8 * s);
+        }
+    }
+}
+
 // ---- inverse pass B': spans 1 .. S/2 inside contiguous chunks (mirror of forward pass B) -----------------------
 
 template <int R1, int R2, class AR>
@@ -534,7 +665,29 @@ void launch_fwd_class(hann_ctx* c, const NttArgs& A, int groups, bool skip_a) {
         pick_fwd_a<AR>(A.a)<<<dim3(1 << (A.b - A.logC), groups * A.nsel), kThreads, smem_a(A), c->stream>>>(A);
     }
     KProf kp(c, KC_NTT_FWD_B);
-    if (A.b == 8 && A.a > 0 && ((c->N >> 8) % kBK) == 0) {
+#ifndef HANN_NO_B8T
+    if (A.b == 8 && A.a > 0 && A.tau && ((c->N >> 8) % kTK) == 0 && ((uintptr_t)A.data & 15) == 0 && (A.stride & 1) == 0) {
+        const size_t smem = (size_t)kTK * 256 * 16 + (size_t)kTP * 2 * 512 * 8 + (size_t)kTP * 2 * 8;
+        cudaFuncSetAttribute(k_ntt_fwd_b8t<AR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        const int ranges = (c->N >> 8) / kTK, ntiles = (groups + kTP - 1) / kTP;
+        // tiles per CTA: a CTA stages its twiddles once and its warps prefetch two tiles ahead, but the grid should still
+        // fill whole waves of the 148 x 3 resident CTAs.  Smallest (waves x (tiles per CTA + staging)), ties to fewer CTAs.
+        const int slots = 148 * 3, per = ranges * A.nsel;
+        int zs = 1;
+        long best = -1;
+        for (int z = 1; z <= ntiles && z <= 64; z++) {
+            const long waves = ((long)per * z + slots - 1) / slots, tiles = (ntiles + z - 1) / z;
+            const long cost = waves * (4 * tiles + 1);
+            if (best < 0 || cost < best) {
+                best = cost;
+                zs = z;
+            }
+        }
+        k_ntt_fwd_b8t<AR><<<dim3(ranges, A.nsel, zs), 256, smem, c->stream>>>(A, groups, c->kflag);
+        return;
+    }
+#endif
+    if (A.b == 8 && A.a > 0 && A.tau && ((c->N >> 8) % kBK) == 0) {
         const size_t smem = (size_t)kBK * 256 * 16 + (size_t)kBPG * kBK * 272 * 8;
         cudaFuncSetAttribute(k_ntt_fwd_b8<AR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  // 50 KiB > default 48
         // enough CTAs for about four per SM; beyond that a CTA walks several tiles and reuses its staged twiddles

@@ -241,3 +241,21 @@ def test_empty_and_single_row_levels():
     got, score_g = run_level(p, rows, qv)
     allslots = g.decrypt_scores(p.km.s, score_g)[0]
     assert np.abs(allslots[1:]).max() < 2.0 ** ps.tol_log2
+
+
+def test_encode_into_buffer_that_is_only_word_aligned():
+    """Polynomial buffers need no more than 8-byte alignment: the transform falls back from its bulk-copy kernel to
+    the plain-load kernel and produces the same words."""
+    import torch
+
+    ps = synth.small_params(12, 32, 8, L=2)
+    p = Pair(ps, key_seed=4)
+    g, b = p.g, p.b
+    rows = torch.from_numpy(synth.toy_corpus(7, rows=ps.n + 5, dim=32)).to(g.device)
+    nbytes = g.n_blocks(rows.shape[0]) * g.sizeof(b.SIZE_PT_BLOCK)
+    aligned = g.encode_candidates(rows, p.ws, g.alloc(nbytes))
+    shifted = g.alloc(nbytes + 8)[1:]
+    assert shifted.data_ptr() % 16 == 8
+    g.encode_candidates(rows, p.ws, shifted)
+    g.sync()
+    assert torch.equal(aligned, shifted)

@@ -817,6 +817,7 @@ extern "C" int hann_query_level(hann_ctx* c, const void* ct_dev, const float* ro
     if (!ct_dev || !rows_dev || !baby_dev || !pt_dev || !inner_dev || !score_ct_dev || n_rows < 1)
         return fail(c, HANN_EINVAL, "hann_query_level: bad argument");
     if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_query_level: workspace missing or not 256-byte aligned");
+    if (dim < 1 || dim > c->R) return fail(c, HANN_ESHAPE, "hann_query_level: dim must be in 1..R");
     const int64_t prep = c->B > 1 ? align256(prepare_words(c) * 8 + kSlack) : 0;
     if ((int64_t)ws_bytes < prep + encode_ws_bytes(c)) return fail(c, HANN_EWORKSPACE, "hann_query_level: workspace too small");
     DeviceGuard dg(c->device);

@@ -365,6 +365,43 @@ void orc_decrypt_residues(const orc_ctx *c, const int8_t *s, const u64 *ct, u64 
     free(sq); free(t);
 }
 
+/* mu = c0 + c1*s over the first nl moduli of a ciphertext stored with nl limbs: ct[2][nl][N] */
+void orc_decrypt_residues_limbs(const orc_ctx *c, const int8_t *s, const u64 *ct, int nl, u64 *mu) {
+    int N = c->N;
+    u64 *sq = (u64 *)malloc(8 * N), *t = (u64 *)malloc(8 * N);
+    for (int l = 0; l < nl; l++) {
+        u64 q = c->mod[l];
+        lift_i8(s, N, q, sq);
+        orc_negacyclic_mul(c, l, ct + (size_t)(1 * nl + l) * N, sq, t);
+        for (int i = 0; i < N; i++) mu[(size_t)l * N + i] = addmod(ct[(size_t)(0 * nl + l) * N + i], t[i], q);
+    }
+    free(sq); free(t);
+}
+
+/* Output compaction (Sec. 7, storage and upload footprint: switch a ciphertext down to the minimal modulus the
+ * remaining computation -- here only decryption -- needs).  On each of the two polynomials:
+ *   rescale != 0: divide by the last prime q_{L-1} first:  r = centred lift of [c]_{q_{L-1}};
+ *       c'_i = (c_i - r) * q_{L-1}^{-1} mod q_i, i.e. c' = (c - r) / q_{L-1} exactly; message and scale are divided by
+ *       q_{L-1} and a rounding error (tau_0 + tau_1 s, |tau| <= 1/2 per coefficient) is added;
+ *   then keep limbs 0..keep-1 (no division, no error: c_0 + c_1 s is the same integer mod q_0..q_{keep-1}; valid
+ *       while |message + noise| < q_0..q_{keep-1} / 2).
+ * ct[2][L][N] coefficient domain -> out[2][keep][N]; keep <= L-1 when rescaling, keep <= L otherwise. */
+void orc_compact(const orc_ctx *c, const u64 *ct, int keep, int rescale, u64 *out) {
+    int N = c->N, L = c->L; u64 ql = c->mod[L - 1];
+    for (int poly = 0; poly < 2; poly++)
+        for (int i = 0; i < keep; i++) {
+            u64 q = c->mod[i], qlinv = invmod(ql % q, q);
+            for (int x = 0; x < N; x++) {
+                u64 v = ct[((size_t)poly * L + i) * N + x];
+                if (rescale) {
+                    i64 r = centred(ct[((size_t)poly * L + (L - 1)) * N + x], ql);
+                    v = mulmod(submod(v, reduce_signed(r, q), q), qlinv, q);
+                }
+                out[((size_t)poly * keep + i) * N + x] = v;
+            }
+        }
+}
+
 /* ------------------------------------------------------------------ evaluation keys, key switching */
 
 /* Evaluation key for the left rotation by r (k = 5^r, s' = phi_k(s)); one special prime, one digit per

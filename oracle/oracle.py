@@ -219,6 +219,40 @@ class Oracle:
         muf = np.array([float(v) for v in mu], dtype=np.float64)
         return self.decode(muf, float(2.0 ** log_scale_out))
 
+    # ---- output compaction
+    def compact(self, ct, keep=1, rescale=True):
+        """keep the first `keep` limbs, after a rescale by the last prime if asked (scale / q_{L-1}):
+        [2][L][N] -> [2][keep][N]"""
+        ct = _u64(ct)
+        assert ct.shape == (2, self.L, self.N) and 1 <= keep <= self.L - (1 if rescale else 0)
+        out = np.zeros((2, keep, self.N), dtype=np.uint64)
+        lib().orc_compact(self.h, _p(ct, u64p), C.c_int(keep), C.c_int(1 if rescale else 0), _p(out, u64p))
+        return out
+
+    def decrypt_compact_int(self, s, ctc):
+        """centred integers of c0 + c1*s over the limbs the compact ciphertext still has"""
+        s = np.ascontiguousarray(s, dtype=np.int8)
+        ctc = _u64(ctc)
+        nl = ctc.shape[1]
+        mu = np.zeros((nl, self.N), dtype=np.uint64)
+        lib().orc_decrypt_residues_limbs(self.h, _p(s, i8p), _p(ctc, u64p), C.c_int(nl), _p(mu, u64p))
+        Q = 1
+        for l in range(nl):
+            Q *= self.q[l]
+        acc = np.zeros(self.N, dtype=object)
+        for l in range(nl):
+            Qh = Q // self.q[l]
+            acc = acc + mu[l].astype(object) * (Qh * pow(Qh % self.q[l], -1, self.q[l]))
+        acc = acc % Q
+        return np.array([int(v) - Q if int(v) > Q // 2 else int(v) for v in acc], dtype=object)
+
+    def decrypt_compact_slots(self, s, ctc, log_scale_in, rescaled=True):
+        """slots of a compacted ciphertext whose scale was 2^log_scale_in before compaction"""
+        mu = self.decrypt_compact_int(s, ctc)
+        muf = np.array([float(v) for v in mu], dtype=np.float64)
+        scale = float(2.0 ** log_scale_in)
+        return self.decode(muf, scale / float(self.q[self.L - 1]) if rescaled else scale)
+
     # ---- keys, key switching, rotation
     def evk_gen(self, s, r, a, e):
         s = np.ascontiguousarray(s, dtype=np.int8)

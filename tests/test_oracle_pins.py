@@ -410,3 +410,80 @@ def test_full_size_primes_scores_within_tolerance_small_ring():
     assert np.abs(got.real - want).max() < 2.0 ** -18
     assert np.abs(got.real - want).max() < 2.0 ** -24
     assert np.abs(got.imag).max() < 2.0 ** -18
+
+
+# ------------------------------------------------------------------ output compaction (rescale + limb drop)
+
+
+def test_compaction_is_exact_division_of_the_crt_integer():
+    """Big-integer pin: with C the centred CRT integer of a polynomial over q_0..q_{L-1} and r the centred residue
+    mod q_{L-1}, the kept limbs must hold (C - r) / q_{L-1} (an exact division), i.e. C / q_{L-1} rounded to nearest."""
+    ps = synth.small_params(5, 4, 2, L=3, big=True)
+    o = make(ps)
+    rng = np.random.default_rng(11)
+    ct = np.stack([np.stack([rand_poly(rng, ps.N, q) for q in ps.q]) for _ in range(2)])
+    ql = ps.q[-1]
+    for keep in (1, 2):
+        out = o.compact(ct, keep)
+        assert np.array_equal(o.compact(ct, keep, rescale=False), ct[:, :keep])
+        for poly in range(2):
+            C = [int(v) for v in o.crt_centred(ct[poly])]
+            for x in range(ps.N):
+                r = C[x] % ql
+                if r > ql // 2:
+                    r -= ql
+                assert (C[x] - r) % ql == 0
+                want = (C[x] - r) // ql
+                assert abs(want * ql - C[x]) <= ql // 2            # nearest multiple
+                for i in range(keep):
+                    assert int(out[poly, i, x]) == want % ps.q[i]
+
+
+def rescale_error_sigma(N, scale):
+    """standard deviation of the real part of a slot of the rescale's rounding error tau_0 + tau_1 s (tau uniform in
+    [-1/2, 1/2], s ternary with variance 2/3): a coefficient has variance N/18 + 1/12, a slot sums N of them with
+    unit-modulus weights, its real part takes half"""
+    return math.sqrt(N * (N / 18.0 + 1.0 / 12.0) / 2.0) / scale
+
+
+def test_compacted_scores_decrypt_to_the_same_scores():
+    """Production primes on a reduced ring.  Dropping to two limbs is exact (identical centred integers); a rescale to
+    one limb (scale 2^80 / q_3 ~ 2^30) adds the rounding error of the division: within 6 sigma of its analytic size and,
+    on this ring, still inside 2^-18."""
+    ps = synth.ParamSet("n11", 11, synth.Q50, synth.P60, 40, 128, 32, -18)
+    o = make(ps)
+    km = synth.key_material(ps, 5)
+    rows = synth.project_rows(synth.toy_corpus(1, rows=ps.n - 100, dim=96).astype(np.float64), None, 128)
+    qv = np.zeros(128, dtype=np.float32); qv[:96] = synth.toy_query(2, dim=96)
+    ct = o.encrypt_query(km.s, qv, km.ct_a, km.ct_e)
+    evk = all_keys(o, km)
+    sc, _, _ = o.score_block(rows, o.baby_set(ct, evk), evk[ps.B - 1])
+    want = np.zeros(ps.n); want[: ps.n - 100] = rows.astype(np.float64) @ qv.astype(np.float64)
+    full_int = o.decrypt_int(km.s, sc)
+    full = o.decrypt_slots(km.s, sc, 2 * ps.log_scale)
+    two = o.compact(sc, 2, rescale=False)
+    assert np.array_equal(two, sc[:, :2])
+    assert list(o.decrypt_compact_int(km.s, two)) == list(full_int)          # the same integers from half the limbs
+    sigma = rescale_error_sigma(ps.N, 2.0 ** 80 / ps.q[-1])
+    for keep in (1, 3):
+        small = o.compact(sc, keep)
+        assert small.shape == (2, keep, ps.N)
+        got = o.decrypt_compact_slots(km.s, small, 2 * ps.log_scale)
+        assert np.abs(got.real - full.real).max() < 6 * sigma
+        assert np.abs(got.real - full.real).std() > sigma / 3                # and the error really is of that size
+        assert np.abs(got.real - want).max() < 2.0 ** -18
+        assert np.abs(got.imag).max() < 2.0 ** -18
+    # toy primes: only 2^50 / q_1 ~ 2^20 of scale is left on the one ~30-bit limb, so the rounding error of the
+    # division (sigma ~ 2^-10.5) exceeds the scoring tolerance: the toy set has no room for a rescale
+    ps = synth.TOY
+    o = make(ps)
+    km = synth.key_material(ps, 3)
+    rows = synth.toy_corpus(1, rows=ps.n)
+    qv = synth.toy_query(2)
+    ct = o.encrypt_query(km.s, qv, km.ct_a, km.ct_e)
+    evk = all_keys(o, km)
+    sc, _, _ = o.score_block(rows, o.baby_set(ct, evk), evk[ps.B - 1])
+    got = o.decrypt_compact_slots(km.s, o.compact(sc, 1), 2 * ps.log_scale)
+    sigma = rescale_error_sigma(ps.N, 2.0 ** 50 / ps.q[-1])
+    err = np.abs(got.real - o.decrypt_slots(km.s, sc, 2 * ps.log_scale).real)
+    assert sigma / 3 < err.std() and err.max() < 6 * sigma

@@ -255,6 +255,30 @@ def run_ours(args):
     ctx.set_timing(False)
     stage_ms = {k[3:]: float(np.median(v)) for k, v in stage.items()}
 
+    # output compaction of the level's score ciphertexts (not part of the step: an optional call after it): device time of
+    # both forms, bytes the client would download, and the decrypted scores of what comes out
+    compaction = {}
+    if ps.L >= 2:
+        for name, keep, rescale in (("first_2_limbs_exact", min(2, ps.L), False), ("rescale_to_1_limb", 1, True)):
+            if keep > ps.L - (1 if rescale else 0) or (not rescale and keep == ps.L):
+                continue
+            out_c = ctx.alloc(ctx.lib.hann_compact_bytes(ctx.h, nb, keep))
+            ctx.compact_scores(score, nb, keep, rescale, ws, out_c)
+            torch.cuda.synchronize()
+            c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            c0.record()
+            for _ in range(aux_steps):
+                ctx.compact_scores(score, nb, keep, rescale, ws, out_c)
+            c1.record()
+            torch.cuda.synchronize()
+            small = ctx.export_limbs(out_c, nb * 2, keep).reshape(nb, 2, keep, ps.N)
+            got_c = ctx.decrypt_compact(km.s, small, rescale).reshape(-1)[:n_rows]
+            compaction[name] = {"ms": c0.elapsed_time(c1) / aux_steps, "bytes_out": int(small.nbytes),
+                                "bytes_uncompacted": int(score_host.nbytes),
+                                "max_abs_score_error": float(np.abs(got_c - want).max()),
+                                "same_top10": bool(np.array_equal(np.argsort(-got_c)[:10], np.argsort(-want)[:10]))}
+            del out_c
+
     # per-kernel device time, live, with an event pair around every launch of the same steps
     ctx.kernel_profile(True)
     for _ in range(aux_steps):
@@ -332,7 +356,7 @@ def run_ours(args):
             # candidates already encoded and resident (the paper's "warm" case): prepare + multiply-accumulate + rotate-and-sum
             "warm_value": world * n_rows / ((stage_ms["query_prepare"] + stage_ms["score_level"] + stage_ms["rotate_sum"]) * 1e-3),
             "kernels": kernels, "hbm_kernels": hbm_kernels, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
-            "gpu_launches": int(launches), "clocks": clocks,
+            "gpu_launches": int(launches), "clocks": clocks, "compaction": compaction,
             "check": {"max_abs_score_error": max_err, "tolerance": 2.0 ** ps.tol_log2, "ok": check_ok},
         }
         print(json.dumps(line))

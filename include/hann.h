@@ -150,6 +150,12 @@ int hann_encrypt_query(hann_ctx *ctx, const int8_t *s, const float *q, int dim, 
 int hann_decrypt_scores(hann_ctx *ctx, const int8_t *s, const uint64_t *ct, int64_t count, int log_scale_out,
                         double *scores, double *imag_or_null);
 
+/* Decrypt compacted score ciphertexts (hann_compact_scores, exported with hann_export_limbs): ct [count][2][limbs][N]
+ * canonical, over the first `limbs` ciphertext primes; `log_scale_in` is the scale before compaction (2*log_scale after
+ * scoring), `rescaled` says whether the compaction divided by the last prime. */
+int hann_decrypt_compact(hann_ctx *ctx, const int8_t *s, const uint64_t *ct, int64_t count, int limbs, int rescaled,
+                         int log_scale_in, double *scores, double *imag_or_null);
+
 /* ---- server side ------------------------------------------------------------------------------------------ */
 
 /* Upload evaluation keys (canonical layout as produced by hann_keygen_from_samples; `evk` may be a host or a
@@ -215,6 +221,25 @@ int hann_keyswitch_static(hann_ctx *ctx, int rot, const void *poly_dev, void *ks
  * kind POLY / PT: one polynomial of L limbs per element; CT: two. */
 int hann_import(hann_ctx *ctx, int kind, const uint64_t *canonical, int64_t count, void *internal_dev);
 int hann_export(hann_ctx *ctx, int kind, const void *internal_dev, int64_t count, uint64_t *canonical_out);
+/* The same for npoly polynomials stored with `limbs` limbs each (compacted ciphertexts): internal [npoly][limbs][N] ->
+ * canonical [npoly][limbs][N]. */
+int hann_export_limbs(hann_ctx *ctx, const void *internal_dev, int64_t npoly, int limbs, uint64_t *canonical_out);
+
+/* Output compaction (Sec. 7, storage and upload footprint: switch a ciphertext down to the minimal modulus the rest of
+ * its life needs -- for a score ciphertext that is decryption only).  Each score ciphertext [2][L][N] becomes
+ * [2][keep][N] (internal layout, transform domain):
+ *   rescale = 0: limbs 0..keep-1 are kept as they are.  Exact: c0 + c1*s is the same integer modulo the smaller
+ *       product, so this is valid while |scores * scale| stays below q_0..q_{keep-1} / 2 (scale 2^80, two ~50-bit
+ *       limbs: scores up to 2^19);
+ *   rescale = 1: every polynomial is first divided by the last prime with rounding, c' = (c - [c]_{q_{L-1}}) / q_{L-1}
+ *       (centred residue), which divides message and scale by q_{L-1} and adds a rounding error of standard deviation
+ *       ~ N / 6 per slot (real part, heavy-tailed: a product of two near-Gaussian values) -- at N = 2^16 and scale
+ *       2^80 / q_3 ~ 2^30 that is 2^-16.6 per score, above the scoring path's own error; keep <= L-1.
+ * out_dev: hann_compact_bytes(ctx, n_blocks, keep) bytes (device).  `ws` as for the other server calls (only used
+ * with rescale = 1).  Nothing is allocated. */
+int64_t hann_compact_bytes(const hann_ctx *ctx, int64_t n_blocks, int keep);
+int hann_compact_scores(hann_ctx *ctx, const void *score_ct_dev, int64_t n_blocks, int keep, int rescale, void *out_dev,
+                        void *ws, size_t ws_bytes);
 
 /* One level end to end from HOST buffers (copies included): the rows are copied to the device block by block on a copy
  * stream while the query ciphertext is imported and its baby set prepared on a helper stream; every block is encoded as

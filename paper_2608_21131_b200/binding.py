@@ -85,6 +85,10 @@ def load_library():
         "hann_keyswitch_static": (C.c_int, [vp, C.c_int, vp, vp, vp]),
         "hann_import": (C.c_int, [vp, C.c_int, vp, i64, vp]),
         "hann_export": (C.c_int, [vp, C.c_int, vp, i64, vp]),
+        "hann_export_limbs": (C.c_int, [vp, vp, i64, C.c_int, vp]),
+        "hann_compact_bytes": (i64, [vp, i64, C.c_int]),
+        "hann_compact_scores": (C.c_int, [vp, vp, i64, C.c_int, C.c_int, vp, vp, sz]),
+        "hann_decrypt_compact": (C.c_int, [vp, vp, vp, i64, C.c_int, C.c_int, C.c_int, vp, vp]),
         "hann_level_host_bytes": (i64, [vp, i64]),
         "hann_score_level_host": (C.c_int, [vp, vp, vp, i64, C.c_int, vp, vp, sz]),
     }
@@ -219,6 +223,17 @@ class Context:
         self._ck(self.lib.hann_decrypt_scores(self.h, _ptr(s), _ptr(ct), count, ls, _ptr(scores), _ptr(imag)))
         return (scores, imag) if want_imag else scores
 
+    def decrypt_compact(self, s, ct, rescaled, log_scale_in=None, want_imag=False):
+        """ct: [count][2][limbs][N] canonical, as produced by compact_scores + export_limbs"""
+        s, ct = _np(s, np.int8), _np(ct, np.uint64)
+        count, _, limbs, _ = ct.shape
+        scores = np.empty((count, self.n), dtype=np.float64)
+        imag = np.empty((count, self.n), dtype=np.float64) if want_imag else None
+        ls = 2 * self.log_scale if log_scale_in is None else log_scale_in
+        self._ck(self.lib.hann_decrypt_compact(self.h, _ptr(s), _ptr(ct), count, limbs, 1 if rescaled else 0, ls, _ptr(scores),
+                                               _ptr(imag)))
+        return (scores, imag) if want_imag else scores
+
     # ---- server side
     def load_keys(self, evk, rots):
         rots = _np(rots, np.int32)
@@ -238,6 +253,18 @@ class Context:
         polys = 2 if kind == KIND_CT else 1
         out = np.empty((count, polys, self.L, self.N), dtype=np.uint64)
         self._ck(self.lib.hann_export(self.h, kind, _ptr(internal) + offset_bytes, count, _ptr(out)))
+        return out
+
+    def export_limbs(self, internal, npoly, limbs):
+        out = np.empty((npoly, limbs, self.N), dtype=np.uint64)
+        self._ck(self.lib.hann_export_limbs(self.h, _ptr(internal), npoly, limbs, _ptr(out)))
+        return out
+
+    def compact_scores(self, score, n_blocks, keep, rescale, ws=None, out=None):
+        if out is None:
+            out = self.alloc(self.lib.hann_compact_bytes(self.h, n_blocks, keep))
+        self._ck(self.lib.hann_compact_scores(self.h, _ptr(score), n_blocks, keep, 1 if rescale else 0, _ptr(out), _ptr(ws),
+                                              ws.numel() * 8 if ws is not None else 0))
         return out
 
     def query_prepare(self, ct_dev, ws, baby=None):

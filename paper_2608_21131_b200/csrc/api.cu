@@ -474,6 +474,68 @@ extern "C" int hann_export(hann_ctx* c, int kind, const void* internal_dev, int6
     return HANN_OK;
 }
 
+extern "C" int hann_export_limbs(hann_ctx* c, const void* internal_dev, int64_t npoly, int limbs, uint64_t* canonical_out) {
+    if (!c) return HANN_EINVAL;
+    if (!canonical_out || !internal_dev || npoly < 0) return fail(c, HANN_EINVAL, "hann_export_limbs: bad argument");
+    if (limbs < 1 || limbs > c->L) return fail(c, HANN_ESHAPE, "hann_export_limbs: limb count out of range");
+    DeviceGuard dg(c->device);
+    const int64_t piece = 64, pw = (int64_t)limbs * c->N;
+    RET(ensure_scratch(c, piece * pw * 8));
+    for (int64_t p0 = 0; p0 < npoly; p0 += piece) {
+        const int64_t np = std::min(piece, npoly - p0);
+        u64* staging = (u64*)c->scratch;
+        CK(cudaMemcpyAsync(staging, (const u64*)internal_dev + p0 * pw, np * pw * 8, cudaMemcpyDeviceToDevice, c->stream));
+        RET(launch_ntt_inv(c, staging, np * limbs, c->N, limbmap_first(limbs)));
+        CK(cudaMemcpyAsync(canonical_out + p0 * pw, staging, np * pw * 8, cudaMemcpyDefault, c->stream));
+    }
+    CK(cudaStreamSynchronize(c->stream));
+    return HANN_OK;
+}
+
+extern "C" int64_t hann_compact_bytes(const hann_ctx* c, int64_t n_blocks, int keep) {
+    if (!c || n_blocks < 0 || keep < 1 || keep > c->L) return HANN_EINVAL;
+    return n_blocks * 2 * (int64_t)keep * c->N * 8;
+}
+
+extern "C" int hann_compact_scores(hann_ctx* c, const void* score_ct_dev, int64_t n_blocks, int keep, int rescale, void* out_dev,
+                                   void* ws, size_t ws_bytes) {
+    if (!c) return HANN_EINVAL;
+    if (n_blocks < 0 || (n_blocks > 0 && (!score_ct_dev || !out_dev))) return fail(c, HANN_EINVAL, "hann_compact_scores: bad argument");
+    const int L = c->L, N = c->N;
+    if (keep < 1 || keep > L - (rescale ? 1 : 0)) return fail(c, HANN_ESHAPE, "hann_compact_scores: keep must be in 1..L-1 (1..L without rescale)");
+    if (n_blocks == 0) return HANN_OK;
+    DeviceGuard dg(c->device);
+    const u64* src = (const u64*)score_ct_dev;
+    u64* out = (u64*)out_dev;
+    const int64_t npoly = n_blocks * 2;
+    if (!rescale) {
+        // the first `keep` limbs of every polynomial: c0 + c1 s is the same integer modulo the smaller product
+        CK(cudaMemcpy2DAsync(out, (size_t)keep * N * 8, src, (size_t)L * N * 8, (size_t)keep * N * 8, (size_t)npoly, cudaMemcpyDeviceToDevice,
+                             c->stream));
+        return HANN_OK;
+    }
+    if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_compact_scores: workspace missing or not 256-byte aligned");
+    // per polynomial: the last limb back in coefficients (N words) and its lift into the kept limbs (keep * N words)
+    const int64_t per = (int64_t)(1 + keep) * N * 8;
+    int64_t ch = ((int64_t)ws_bytes - kSlack) / per;
+    if (ch < 1) return fail(c, HANN_EWORKSPACE, "hann_compact_scores: workspace too small");
+    ch = std::min(ch, npoly);
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
+    u64* t = ar.take<u64>(ch * N);
+    u64* lifted = ar.take<u64>(ch * keep * N);
+    if (!t || !lifted) return fail(c, HANN_EWORKSPACE, "hann_compact_scores: workspace too small");
+    for (int64_t p0 = 0; p0 < npoly; p0 += ch) {
+        const int64_t np = std::min(ch, npoly - p0);
+        CK(cudaMemcpy2DAsync(t, (size_t)N * 8, src + (p0 * L + (L - 1)) * N, (size_t)L * N * 8, (size_t)N * 8, (size_t)np,
+                             cudaMemcpyDeviceToDevice, c->stream));
+        RET(launch_ntt_inv(c, t, np, N, limbmap_single(L - 1)));
+        RET(launch_rescale_lift(c, t, np, keep, lifted));
+        RET(launch_ntt_fwd(c, lifted, np * keep, N, limbmap_first(keep)));
+        RET(launch_rescale_combine(c, src + p0 * L * N, lifted, np, keep, out + p0 * keep * N));
+    }
+    return HANN_OK;
+}
+
 // ================================================================================================ client side
 
 extern "C" int hann_keygen_from_samples(hann_ctx* c, const int8_t* s, int n_rot, const int32_t* rot, const uint64_t* a,
@@ -561,32 +623,34 @@ extern "C" int hann_encrypt_query(hann_ctx* c, const int8_t* s, const float* q, 
     return HANN_OK;
 }
 
-extern "C" int hann_decrypt_scores(hann_ctx* c, const int8_t* s, const uint64_t* ct, int64_t count, int log_scale_out,
-                                   double* scores, double* imag_or_null) {
-    if (!c) return HANN_EINVAL;
-    if (!s || !ct || !scores || count < 0) return fail(c, HANN_EINVAL, "hann_decrypt_scores: bad argument");
-    const int L = c->L, N = c->N, n = c->n;
+// count ciphertexts of nl limbs each, ct [count][2][nl][N] canonical, plaintext scale 1 / inv_scale
+static int decrypt_impl(hann_ctx* c, const int8_t* s, const uint64_t* ct, int64_t count, int nl, long double inv_scale,
+                        double* scores, double* imag_or_null) {
+    const int N = c->N, n = c->n;
     DeviceGuard dg(c->device);
-    const int64_t LN = (int64_t)L * N;
+    const int64_t LN = (int64_t)nl * N;
     RET(ensure_scratch(c, 4 * LN * 8 + align256(N) + kSlack));
     Arena ar{(char*)c->scratch, 0, c->scratch_bytes};
     u64* shat = ar.take<u64>(LN);
     u64* CT = ar.take<u64>(2 * LN);
     u64* MU = ar.take<u64>(LN);
     int8_t* s8 = ar.take<int8_t>(N);
-    RET(upload_secret(c, s, L, s8, shat));
+    const LimbMap lm = limbmap_first(nl);
+    CK(cudaMemcpyAsync(s8, s, N, cudaMemcpyHostToDevice, c->stream));
+    RET(launch_lift_i8(c, s8, nl, shat));
+    RET(launch_ntt_fwd(c, shat, nl, N, lm));
     std::vector<u64> mu(LN);
     std::vector<long double> real(N);
     std::vector<double> re(n), im(n);
-    const long double inv_scale = ldexpl(1.0L, -log_scale_out);
     for (int64_t i = 0; i < count; i++) {
-        RET(import_polys(c, ct + i * 2 * LN, 2, CT));
-        RET(launch_mul(c, CT + LN, shat, L, MU, L, limbmap_q(c)));   // c1 * s
-        RET(launch_add(c, MU, CT, MU, L, limbmap_q(c)));             // + c0
-        RET(launch_ntt_inv(c, MU, L, N, limbmap_q(c)));
+        CK(cudaMemcpyAsync(CT, ct + i * 2 * LN, 2 * LN * 8, cudaMemcpyDefault, c->stream));
+        RET(launch_ntt_fwd(c, CT, 2 * nl, N, lm));
+        RET(launch_mul(c, CT + LN, shat, nl, MU, nl, lm));   // c1 * s
+        RET(launch_add(c, MU, CT, MU, nl, lm));              // + c0
+        RET(launch_ntt_inv(c, MU, nl, N, lm));
         CK(cudaMemcpyAsync(mu.data(), MU, LN * 8, cudaMemcpyDeviceToHost, c->stream));
         CK(cudaStreamSynchronize(c->stream));
-        hm::crt_to_real(mu.data(), L, N, c->mod, real.data());
+        hm::crt_to_real(mu.data(), nl, N, c->mod, real.data());
         // slots: a_k = (mu_k + i mu_{k+n}) conj(U[k]);  z_j * scale = sum_k a_k exp(+2 pi i u_j k / n)
         for (int k = 0; k < n; k++) {
             const double mr = (double)(real[k] * inv_scale), mi = (double)(real[k + n] * inv_scale);
@@ -601,6 +665,23 @@ extern "C" int hann_decrypt_scores(hann_ctx* c, const int8_t* s, const uint64_t*
         }
     }
     return HANN_OK;
+}
+
+extern "C" int hann_decrypt_scores(hann_ctx* c, const int8_t* s, const uint64_t* ct, int64_t count, int log_scale_out,
+                                   double* scores, double* imag_or_null) {
+    if (!c) return HANN_EINVAL;
+    if (!s || !ct || !scores || count < 0) return fail(c, HANN_EINVAL, "hann_decrypt_scores: bad argument");
+    return decrypt_impl(c, s, ct, count, c->L, ldexpl(1.0L, -log_scale_out), scores, imag_or_null);
+}
+
+extern "C" int hann_decrypt_compact(hann_ctx* c, const int8_t* s, const uint64_t* ct, int64_t count, int limbs, int rescaled,
+                                    int log_scale_in, double* scores, double* imag_or_null) {
+    if (!c) return HANN_EINVAL;
+    if (!s || !ct || !scores || count < 0) return fail(c, HANN_EINVAL, "hann_decrypt_compact: bad argument");
+    if (limbs < 1 || limbs > c->L - (rescaled ? 1 : 0)) return fail(c, HANN_ESHAPE, "hann_decrypt_compact: limb count out of range");
+    long double inv_scale = ldexpl(1.0L, -log_scale_in);
+    if (rescaled) inv_scale *= (long double)c->mod[c->L - 1];
+    return decrypt_impl(c, s, ct, count, limbs, inv_scale, scores, imag_or_null);
 }
 
 // ================================================================================================ server side

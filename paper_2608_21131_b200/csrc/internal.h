@@ -140,6 +140,10 @@ int launch_moddown_combine(hann_ctx* c, const u64* u, const u64* lifted, int64_t
                            int64_t c0_stride, const u64* addend, int64_t addend_stride, u64* out0, u64* out1,
                            int64_t out_stride);
 int launch_permute(hann_ctx* c, const u64* src, u64* dst, int64_t npoly, unsigned k);
+// output compaction: centred lift of coefficient-domain residues mod q_{L-1} into limbs 0..keep-1; (src - lifted) / q_{L-1}
+int launch_rescale_lift(hann_ctx* c, const u64* t, int64_t npoly, int keep, u64* lifted);
+int launch_rescale_combine(hann_ctx* c, const u64* src, const u64* lifted, int64_t npoly, int keep, u64* out);
+LimbMap limbmap_first(int nlimbs);  // period nlimbs: limbs 0..nlimbs-1
 
 // helpers of the client half
 int launch_lift_i8(hann_ctx* c, const int8_t* v, int nlimbs, u64* out);

@@ -593,6 +593,66 @@ int launch_moddown_combine(hann_ctx* c, const u64* u, const u64* lifted, int64_t
     return check_launch(c, "moddown_combine");
 }
 
+// ---- output compaction: rescale by the last ciphertext prime ---------------------------------------------------------
+// lifted[poly][i][x] = centred lift of t[poly][x] (residue mod q_{L-1}, coefficient domain) reduced mod q_i, i < keep
+__global__ void __launch_bounds__(kThreads) k_rescale_lift(const u64* __restrict__ t, u64* __restrict__ lifted, int N, int L,
+                                                           int keep, long long npoly, LimbTable lt) {
+    const long long total = npoly * N;
+    const u64 ql = lt.c[L - 1].q, half = lt.c[L - 1].half;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const long long poly = idx / N;
+        const int x = (int)(idx % N);
+        const u64 v = t[idx];
+        const bool neg = v > half;
+        const u64 mag = neg ? ql - v : v;
+        for (int i = 0; i < keep; i++) {
+            u64 r = barrett64(mag, lt.c[i]);
+            lifted[(poly * keep + i) * N + x] = (neg && r) ? lt.c[i].q - r : r;
+        }
+    }
+}
+
+struct RescaleConst {
+    u64 w[HANN_MAXL1], ws[HANN_MAXL1];  // q_{L-1}^{-1} mod q_i and its Shoup companion
+};
+
+// out[poly][i][x] = (src[poly][i][x] - lifted[poly][i][x]) * q_{L-1}^{-1} mod q_i; src polynomials have L limbs, out keep
+__global__ void __launch_bounds__(kThreads) k_rescale_combine(const u64* __restrict__ src, const u64* __restrict__ lifted,
+                                                              u64* __restrict__ out, int N, int L, int keep, long long npoly,
+                                                              LimbTable lt, RescaleConst rc) {
+    const long long total = npoly * keep * N;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const int x = (int)(idx % N);
+        const int i = (int)((idx / N) % keep);
+        const long long poly = idx / ((long long)keep * N);
+        const u64 q = lt.c[i].q;
+        const u64 d = submod(src[(poly * L + i) * N + x], lifted[idx], q);
+        out[idx] = csub(shoup_mul(d, rc.w[i], rc.ws[i], q), q);
+    }
+}
+
+int launch_rescale_lift(hann_ctx* c, const u64* t, int64_t npoly, int keep, u64* lifted) {
+    {
+        KProf kp(c, KC_OTHER);
+        k_rescale_lift<<<grid_for(npoly * c->N), kThreads, 0, c->stream>>>(t, lifted, c->N, c->L, keep, npoly, c->lt);
+    }
+    return check_launch(c, "rescale_lift");
+}
+
+int launch_rescale_combine(hann_ctx* c, const u64* src, const u64* lifted, int64_t npoly, int keep, u64* out) {
+    RescaleConst rc = {};
+    const u64 ql = c->mod[c->L - 1];
+    for (int i = 0; i < keep; i++) {
+        rc.w[i] = hm::invmod(ql % c->mod[i], c->mod[i]);
+        rc.ws[i] = hm::shoup(rc.w[i], c->mod[i]);
+    }
+    {
+        KProf kp(c, KC_OTHER);
+        k_rescale_combine<<<grid_for(npoly * keep * c->N), kThreads, 0, c->stream>>>(src, lifted, out, c->N, c->L, keep, npoly, c->lt, rc);
+    }
+    return check_launch(c, "rescale_combine");
+}
+
 int launch_permute(hann_ctx* c, const u64* src, u64* dst, int64_t npoly, unsigned k) {
     {
         KProf kp(c, KC_PERMUTE);

@@ -785,6 +785,12 @@ LimbMap limbmap_qp(const hann_ctx* c) {
     for (int i = 0; i <= c->L; i++) m.limb[i] = (signed char)i;
     return m;
 }
+LimbMap limbmap_first(int nlimbs) {
+    LimbMap m;
+    m.period = nlimbs;
+    for (int i = 0; i < nlimbs; i++) m.limb[i] = (signed char)i;
+    return m;
+}
 LimbMap limbmap_single(int limb) {
     LimbMap m;
     m.period = 1;

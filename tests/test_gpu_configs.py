@@ -29,7 +29,7 @@ class Query:
         self.baby = p.g.query_prepare(p.g.import_(p.b.KIND_CT, ct_g, 1), p.ws)
         self.baby_o = p.o.baby_set(ct_o, p.evk_o) if with_oracle else None
 
-    def score_level(self, rows, oracle_blocks=()):
+    def score_level(self, rows, oracle_blocks=(), compact=False):
         """GPU scores of a level [n_rows]; blocks listed in oracle_blocks are compared bit for bit with the oracle"""
         p, g, b, ps = self.p, self.p.g, self.p.b, self.p.ps
         n_rows = rows.shape[0]
@@ -52,6 +52,19 @@ class Query:
         want = rows.astype(np.float64) @ self.qR.astype(np.float64)
         err = float(np.abs(got - want).max())
         assert err < 2.0 ** ps.tol_log2, err
+        if compact:
+            # output compaction at full size: every block bit-identical to the oracle's compaction of the same
+            # ciphertext; two limbs without rescale decrypt to identical scores, one limb after the rescale to scores
+            # within the rounding error of the division (sigma = N / 6 / scale, heavy-tailed)
+            two = g.export_limbs(g.compact_scores(score, nb, 2, False), nb * 2, 2).reshape(nb, 2, 2, ps.N)
+            one = g.export_limbs(g.compact_scores(score, nb, 1, True, ws), nb * 2, 1).reshape(nb, 2, 1, ps.N)
+            for blk in range(nb):
+                assert np.array_equal(two[blk], p.o.compact(score_h[blk], 2, False))
+                assert np.array_equal(one[blk], p.o.compact(score_h[blk], 1, True))
+            assert np.array_equal(g.decrypt_compact(p.km.s, two, False).reshape(-1)[:n_rows], got)
+            self.compact_scores = g.decrypt_compact(p.km.s, one, True).reshape(-1)[:n_rows]
+            sigma = ps.N / 6.0 / (2.0 ** (2 * ps.log_scale) / ps.q[-1])
+            assert np.abs(self.compact_scores - got).max() < 12 * sigma
         del pt, inner, score
         return got, want
 
@@ -61,8 +74,10 @@ def test_face_like_level_full(pair16):
     conformance point, every row within 2^-18."""
     ps, lvl, qR, planted = wl.face_level()
     q = Query(pair16, qR)
-    got, want = q.score_level(lvl.rows, oracle_blocks=(0, 6))
+    got, want = q.score_level(lvl.rows, oracle_blocks=(0, 6), compact=True)
     assert got.shape == (222_049,)
+    # a quarter of the bytes on the wire (one limb instead of four) still ranks the same neighbours first
+    assert np.array_equal(wl.topk_ids(q.compact_scores, lvl.ids, 10), wl.topk_ids(want, lvl.ids, 10))
     # the planted neighbour is the top score under both rankings
     assert int(np.argmax(got)) == planted == int(np.argmax(want))
     assert np.array_equal(wl.topk_ids(got, lvl.ids, 10), wl.topk_ids(want, lvl.ids, 10))

@@ -259,3 +259,46 @@ def test_encode_into_buffer_that_is_only_word_aligned():
     g.encode_candidates(rows, p.ws, shifted)
     g.sync()
     assert torch.equal(aligned, shifted)
+
+
+@pytest.mark.parametrize(
+    "logN,L,big,n_rows",
+    [
+        (6, 3, False, 40),     # tiny ring, generic kernels, two blocks
+        (10, 2, False, 700),   # two ~30-bit primes: one limb left after the rescale
+        (11, 4, True, 1500),   # production primes (4 x ~50 bit), two blocks
+    ],
+)
+def test_compacted_scores_bit_exact_and_decrypt(logN, L, big, n_rows):
+    """Output compaction: the first limbs as they are (exact) and the rescale by the last prime, each bit-identical to the
+    oracle's on the same score ciphertexts, and decrypting to the same scores (to the rounding error of the division)."""
+    if big:
+        ps = synth.ParamSet("n%d" % logN, logN, synth.Q50, synth.P60, 40, 32, 8, -18)
+    else:
+        ps = synth.small_params(logN, 16, 4, L=L)
+    p = Pair(ps, key_seed=logN)
+    g, o, b = p.g, p.o, p.b
+    rows = synth.toy_corpus(logN, rows=n_rows, dim=ps.R)
+    qv = synth.toy_query(logN + 1, dim=ps.R)
+    ct_o, ct_g = p.query(qv)
+    ct_dev = g.import_(b.KIND_CT, ct_g, 1)
+    nb = g.n_blocks(n_rows)
+    baby, pt, inner, score = (g.alloc(g.sizeof(b.SIZE_BABY)), g.alloc(nb * g.sizeof(b.SIZE_PT_BLOCK)),
+                              g.alloc(nb * g.sizeof(b.SIZE_INNER)), g.alloc(nb * g.sizeof(b.SIZE_CT)))
+    g.query_level(ct_dev, torch_rows(p, rows), p.ws, baby, pt, inner, score)
+    score_g = g.export(b.KIND_CT, score, nb)
+    full = g.decrypt_scores(p.km.s, score_g)
+    for keep, rescale in ((ps.L - 1, False), (1, True), (ps.L - 1, True)):
+        small = g.compact_scores(score, nb, keep, rescale, p.ws)
+        small_g = g.export_limbs(small, nb * 2, keep).reshape(nb, 2, keep, ps.N)
+        for blk in range(nb):
+            assert np.array_equal(small_g[blk], o.compact(score_g[blk], keep, rescale))
+        got = g.decrypt_compact(p.km.s, small_g, rescale)
+        if not rescale:
+            if keep * 30 > 2 * ps.log_scale + 12 or big:       # enough modulus left for the unscaled message
+                assert np.array_equal(got, full)
+        else:
+            sigma = np.sqrt(ps.N * (ps.N / 18.0 + 1.0 / 12.0) / 2.0) / (2.0 ** (2 * ps.log_scale) / ps.q[-1])
+            assert np.abs(got - full).max() < 12 * sigma   # product-of-Gaussians tails, see the oracle's pin
+            got_o = np.stack([o.decrypt_compact_slots(p.km.s, small_g[blk], 2 * ps.log_scale).real for blk in range(nb)])
+            assert np.abs(got - got_o).max() < 1e-9 * max(1.0, np.abs(got_o).max()) + 2 * sigma * 1e-6

@@ -442,13 +442,14 @@ def test_compaction_is_exact_division_of_the_crt_integer():
 def rescale_error_sigma(N, scale):
     """standard deviation of the real part of a slot of the rescale's rounding error tau_0 + tau_1 s (tau uniform in
     [-1/2, 1/2], s ternary with variance 2/3): a coefficient has variance N/18 + 1/12, a slot sums N of them with
-    unit-modulus weights, its real part takes half"""
+    unit-modulus weights, its real part takes half.  A slot of tau_1 s is the PRODUCT of two near-Gaussian values
+    (tau_1 and s evaluated at the same root), so the tails are heavier than Gaussian: tests allow 12 sigma."""
     return math.sqrt(N * (N / 18.0 + 1.0 / 12.0) / 2.0) / scale
 
 
 def test_compacted_scores_decrypt_to_the_same_scores():
     """Production primes on a reduced ring.  Dropping to two limbs is exact (identical centred integers); a rescale to
-    one limb (scale 2^80 / q_3 ~ 2^30) adds the rounding error of the division: within 6 sigma of its analytic size and,
+    one limb (scale 2^80 / q_3 ~ 2^30) adds the rounding error of the division: within 12 sigma of its analytic size and,
     on this ring, still inside 2^-18."""
     ps = synth.ParamSet("n11", 11, synth.Q50, synth.P60, 40, 128, 32, -18)
     o = make(ps)
@@ -469,7 +470,7 @@ def test_compacted_scores_decrypt_to_the_same_scores():
         small = o.compact(sc, keep)
         assert small.shape == (2, keep, ps.N)
         got = o.decrypt_compact_slots(km.s, small, 2 * ps.log_scale)
-        assert np.abs(got.real - full.real).max() < 6 * sigma
+        assert np.abs(got.real - full.real).max() < 12 * sigma
         assert np.abs(got.real - full.real).std() > sigma / 3                # and the error really is of that size
         assert np.abs(got.real - want).max() < 2.0 ** -18
         assert np.abs(got.imag).max() < 2.0 ** -18
@@ -486,4 +487,4 @@ def test_compacted_scores_decrypt_to_the_same_scores():
     got = o.decrypt_compact_slots(km.s, o.compact(sc, 1), 2 * ps.log_scale)
     sigma = rescale_error_sigma(ps.N, 2.0 ** 50 / ps.q[-1])
     err = np.abs(got.real - o.decrypt_slots(km.s, sc, 2 * ps.log_scale).real)
-    assert sigma / 3 < err.std() and err.max() < 6 * sigma
+    assert sigma / 3 < err.std() and err.max() < 12 * sigma

@@ -181,6 +181,16 @@ int hann_encode_candidates(hann_ctx *ctx, const float *rows_dev, int64_t n_rows,
 int hann_score_level(hann_ctx *ctx, const void *baby_dev, const void *pt_dev, int64_t n_blocks, void *inner_dev,
                      void *ws, size_t ws_bytes);
 
+/* Cross-query batching (Sec. 7: score a whole batch of queries against each loaded region before it is evicted): the
+ * same multiply-accumulate for n_queries prepared queries against the same encoded blocks, the plaintexts streamed from
+ * HBM once per pair of queries instead of once per query.
+ *   baby_dev  n_queries * HANN_SIZE_BABY bytes: the baby sets of the queries, one after the other;
+ *   inner_dev n_queries * n_blocks * HANN_SIZE_INNER bytes: query-major, [query][blk][g]; hann_rotate_sum over
+ *             n_queries * n_blocks "blocks" then yields score ciphertexts [query][blk].
+ * Each query's result is bit-identical to hann_score_level on its own. */
+int hann_score_level_batch(hann_ctx *ctx, const void *baby_dev, int n_queries, const void *pt_dev, int64_t n_blocks,
+                           void *inner_dev, void *ws, size_t ws_bytes);
+
 /* Rotate-and-sum: score_ct[blk] = sum_g rot_{g*B}(inner[blk][g]), evaluated by Horner with the single key of
  * rotation B: acc = inner[G-1]; for g = G-2..0: acc = rot_B(acc) + inner[g].
  *   score_ct_dev n_blocks * HANN_SIZE_CT bytes (device), internal layout. */

@@ -78,6 +78,7 @@ def load_library():
         "hann_query_prepare": (C.c_int, [vp, vp, vp, vp, sz]),
         "hann_encode_candidates": (C.c_int, [vp, vp, i64, C.c_int, vp, vp, sz]),
         "hann_score_level": (C.c_int, [vp, vp, vp, i64, vp, vp, sz]),
+        "hann_score_level_batch": (C.c_int, [vp, vp, C.c_int, vp, i64, vp, vp, sz]),
         "hann_rotate_sum": (C.c_int, [vp, vp, i64, vp, vp, sz]),
         "hann_keyswitch": (C.c_int, [vp, C.c_int, vp, vp, vp, vp, sz]),
         "hann_query_level": (C.c_int, [vp, vp, vp, i64, C.c_int, vp, vp, vp, vp, vp, sz]),
@@ -289,6 +290,14 @@ class Context:
             inner = self.alloc(n_blocks * self.sizeof(SIZE_INNER))
         self._ck(self.lib.hann_score_level(self.h, _ptr(baby), _ptr(pt), n_blocks, _ptr(inner), _ptr(ws),
                                            ws.numel() * 8 if ws is not None else 0))
+        return inner
+
+    def score_level_batch(self, babies, n_queries, pt, n_blocks, ws=None, inner=None):
+        """babies: the n_queries baby sets back to back; returns inner [query][blk][g]"""
+        if inner is None:
+            inner = self.alloc(n_queries * n_blocks * self.sizeof(SIZE_INNER))
+        self._ck(self.lib.hann_score_level_batch(self.h, _ptr(babies), n_queries, _ptr(pt), n_blocks, _ptr(inner), _ptr(ws),
+                                                 ws.numel() * 8 if ws is not None else 0))
         return inner
 
     def rotate_sum(self, inner, n_blocks, ws, score=None):

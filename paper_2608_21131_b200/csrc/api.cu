@@ -786,6 +786,17 @@ extern "C" int hann_score_level(hann_ctx* c, const void* baby_dev, const void* p
     return launch_mac(c, (const u64*)baby_dev, (const u64*)pt_dev, n_blocks, (u64*)inner_dev);
 }
 
+extern "C" int hann_score_level_batch(hann_ctx* c, const void* baby_dev, int n_queries, const void* pt_dev, int64_t n_blocks,
+                                      void* inner_dev, void* ws, size_t ws_bytes) {
+    (void)ws; (void)ws_bytes;  // the multiply-accumulate needs no scratch
+    if (!c) return HANN_EINVAL;
+    if (n_blocks < 0 || n_queries < 0 || (n_blocks > 0 && n_queries > 0 && (!baby_dev || !pt_dev || !inner_dev)))
+        return fail(c, HANN_EINVAL, "hann_score_level_batch: bad argument");
+    DeviceGuard dg(c->device);
+    Timer tm(c, 2);
+    return launch_mac_batch(c, (const u64*)baby_dev, n_queries, (const u64*)pt_dev, n_blocks, (u64*)inner_dev);
+}
+
 extern "C" int hann_rotate_sum(hann_ctx* c, const void* inner_dev, int64_t n_blocks, void* score_ct_dev, void* ws, size_t ws_bytes) {
     if (!c) return HANN_EINVAL;
     if (n_blocks < 0 || (n_blocks > 0 && (!inner_dev || !score_ct_dev))) return fail(c, HANN_EINVAL, "hann_rotate_sum: bad argument");

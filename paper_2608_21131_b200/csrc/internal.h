@@ -131,6 +131,8 @@ int64_t encode_ws_bytes(const hann_ctx* c);
 
 // scoring
 int launch_mac(hann_ctx* c, const u64* baby, const u64* pt, int64_t n_blocks, u64* inner);
+// n_queries baby sets against the same blocks: inner [q][n_blocks][G] ciphertexts
+int launch_mac_batch(hann_ctx* c, const u64* baby, int n_queries, const u64* pt, int64_t n_blocks, u64* inner);
 
 // key switching pieces
 int launch_lift_digits(hann_ctx* c, const u64* src, int64_t src_stride, int64_t nitems, u64* digits);

@@ -53,26 +53,32 @@ __global__ void __launch_bounds__(kThreads) k_mac(const u64* __restrict__ baby, 
 // 25-bit halves stays below 2^57, of the 26-bit half sums below 2^59.
 constexpr unsigned kM25 = (1u << 25) - 1;
 
-template <int NG, int BB>
-__global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ baby, const u64* __restrict__ pt,
-                                                        u64* __restrict__ inner, int N, int L, long long n_bg,
-                                                        int bg_per_cta, const LimbConst* __restrict__ lt) {
+// NQ queries at once (cross-query batching against the same encoded candidates): the warp keeps the baby-step words of NQ
+// baby sets (query q at baby + q * baby_stride) and every plaintext word, still read once, feeds NQ times the products;
+// partial sums of query q go to inner + q * inner_stride.
+template <int NG, int BB, int NQ>
+__global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ baby, long long baby_stride,
+                                                        const u64* __restrict__ pt, u64* __restrict__ inner,
+                                                        long long inner_stride, int N, int L, long long n_bg, int bg_per_cta,
+                                                        const LimbConst* __restrict__ lt) {
     constexpr int B = NG * BB;
-    __shared__ u64 part[2][NG][6][32];
+    __shared__ u64 part[2][NG][6 * NQ][32];
     const long long LN = (long long)L * N;
     const long long pos0 = (long long)blockIdx.x * 32;
     const int lane = threadIdx.x & 31, wg = threadIdx.x >> 5;
     const LimbConst* lc = lt + pos0 / N;
     // this warp's baby-step words, split into 25-bit halves: lo half in the low word, hi half in the high word
-    unsigned w0[BB][2], w1[BB][2];
+    unsigned w0[NQ][BB][2], w1[NQ][BB][2];
 #pragma unroll
-    for (int k = 0; k < BB; k++)
+    for (int q = 0; q < NQ; q++)
 #pragma unroll
-        for (int c = 0; c < 2; c++) {
-            const u64 v = baby[((long long)(wg * BB + k) * 2 + c) * LN + pos0 + lane];
-            w0[k][c] = (unsigned)v & kM25;
-            w1[k][c] = (unsigned)(v >> 25);
-        }
+        for (int k = 0; k < BB; k++)
+#pragma unroll
+            for (int c = 0; c < 2; c++) {
+                const u64 v = baby[q * baby_stride + ((long long)(wg * BB + k) * 2 + c) * LN + pos0 + lane];
+                w0[q][k][c] = (unsigned)v & kM25;
+                w1[q][k][c] = (unsigned)(v >> 25);
+            }
     const long long bg0 = (long long)blockIdx.y * bg_per_cta;
     const long long bg1 = bg0 + bg_per_cta < n_bg ? bg0 + bg_per_cta : n_bg;
     if (bg0 >= bg1) return;
@@ -86,33 +92,41 @@ __global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ 
 #pragma unroll
             for (int k = 0; k < BB; k++) nxt[k] = __ldcs(pn + (long long)k * LN);
         }
-        u64 p00[2] = {0, 0}, p11[2] = {0, 0}, pm[2] = {0, 0};
+        u64 p00[NQ][2], p11[NQ][2], pm[NQ][2];
+#pragma unroll
+        for (int q = 0; q < NQ; q++)
+#pragma unroll
+            for (int c = 0; c < 2; c++) p00[q][c] = p11[q][c] = pm[q][c] = 0;
 #pragma unroll
         for (int k = 0; k < BB; k++) {
             const unsigned a0 = (unsigned)cur[k] & kM25, a1 = (unsigned)(cur[k] >> 25), as = a0 + a1;
 #pragma unroll
-            for (int c = 0; c < 2; c++) {
-                p00[c] += (u64)a0 * w0[k][c];
-                p11[c] += (u64)a1 * w1[k][c];
-                pm[c] += (u64)as * (w0[k][c] + w1[k][c]);
-            }
-        }
-        u64(*buf)[6][32] = part[bg & 1];
+            for (int q = 0; q < NQ; q++)
 #pragma unroll
-        for (int c = 0; c < 2; c++) {
-            buf[wg][c * 3 + 0][lane] = p00[c];
-            buf[wg][c * 3 + 1][lane] = pm[c];
-            buf[wg][c * 3 + 2][lane] = p11[c];
+                for (int c = 0; c < 2; c++) {
+                    p00[q][c] += (u64)a0 * w0[q][k][c];
+                    p11[q][c] += (u64)a1 * w1[q][k][c];
+                    pm[q][c] += (u64)as * (w0[q][k][c] + w1[q][k][c]);
+                }
         }
+        u64(*buf)[6 * NQ][32] = part[bg & 1];
+#pragma unroll
+        for (int q = 0; q < NQ; q++)
+#pragma unroll
+            for (int c = 0; c < 2; c++) {
+                buf[wg][(q * 2 + c) * 3 + 0][lane] = p00[q][c];
+                buf[wg][(q * 2 + c) * 3 + 1][lane] = pm[q][c];
+                buf[wg][(q * 2 + c) * 3 + 2][lane] = p11[q][c];
+            }
         __syncthreads();
-        // warps 0 and 1 (or warp 0 twice when NG == 1) finish component 0 and 1
-        for (int c = wg; c < 2; c += NG) {
+        // the warps share out the 2 * NQ (query, component) sums
+        for (int qc = wg; qc < 2 * NQ; qc += NG) {
             u64 s00 = 0, sm = 0, s11 = 0;
 #pragma unroll
             for (int g = 0; g < NG; g++) {
-                s00 += buf[g][c * 3 + 0][lane];
-                sm += buf[g][c * 3 + 1][lane];
-                s11 += buf[g][c * 3 + 2][lane];
+                s00 += buf[g][qc * 3 + 0][lane];
+                sm += buf[g][qc * 3 + 1][lane];
+                s11 += buf[g][qc * 3 + 2][lane];
             }
             // value = s00 + cross * 2^25 + s11 * 2^50 with cross = sm - s00 - s11 < 2^59
             const u64 cross = sm - s00 - s11;
@@ -123,9 +137,9 @@ __global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ 
             const u64 d_lo = s11 << 50, d_hi = s11 >> 14;
             lo += d_lo;
             hi += d_hi + (lo < d_lo ? 1 : 0);
-            inner[(bg * 2 + c) * LN + pos0 + lane] = reduce128(hi, lo, *lc);
+            inner[(qc >> 1) * inner_stride + (bg * 2 + (qc & 1)) * LN + pos0 + lane] = reduce128(hi, lo, *lc);
         }
-        if (NG == 1) __syncthreads();  // a single warp reuses the buffer it just read
+        if (NG < 2 * NQ) __syncthreads();  // a warp that finishes several sums may still be reading while the next pair is written
 #pragma unroll
         for (int k = 0; k < BB; k++) cur[k] = nxt[k];
         p += (long long)B * LN;
@@ -475,8 +489,9 @@ int check_launch(hann_ctx* c, const char* what) {
     return HANN_OK;
 }
 
-template <int NG, int BB>
-void launch_mac_stream(hann_ctx* c, const u64* baby, const u64* pt, int64_t n_bg, u64* inner) {
+template <int NG, int BB, int NQ>
+void launch_mac_stream(hann_ctx* c, const u64* baby, int64_t baby_stride, const u64* pt, int64_t n_bg, u64* inner,
+                       int64_t inner_stride) {
     const long long LN = (long long)c->L * c->N;
     const int tiles = (int)(LN / 32);
     // split the (blk, g) range over grid.y only as far as needed to fill the machine: every extra split re-reads the
@@ -486,26 +501,40 @@ void launch_mac_stream(hann_ctx* c, const u64* baby, const u64* pt, int64_t n_bg
     const int per = (int)((n_bg + split - 1) / split);
     split = (int)((n_bg + per - 1) / per);
     KProf kp(c, KC_MAC);
-    k_mac_stream<NG, BB><<<dim3(tiles, split), 32 * NG, 0, c->stream>>>(baby, pt, inner, c->N, c->L, n_bg, per, c->lt_dev);
+    k_mac_stream<NG, BB, NQ><<<dim3(tiles, split), 32 * NG, 0, c->stream>>>(baby, baby_stride, pt, inner, inner_stride, c->N, c->L, n_bg,
+                                                                             per, c->lt_dev);
 }
 
-int launch_mac(hann_ctx* c, const u64* baby, const u64* pt, int64_t n_blocks, u64* inner) {
-    if (n_blocks <= 0) return HANN_OK;
+template <int NQ>
+void launch_mac_stream_b(hann_ctx* c, const u64* baby, int64_t baby_stride, const u64* pt, int64_t n_bg, u64* inner,
+                         int64_t inner_stride) {
+    switch (c->B) {
+        case 1: launch_mac_stream<1, 1, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride); break;
+        case 2: launch_mac_stream<2, 1, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride); break;
+        case 4: launch_mac_stream<4, 1, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride); break;
+        case 8: launch_mac_stream<4, 2, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride); break;
+        case 16: launch_mac_stream<4, 4, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride); break;
+        case 32: launch_mac_stream<4, 8, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride); break;
+        case 64: launch_mac_stream<8, 8, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride); break;
+        default: launch_mac_stream<8, 16, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride); break;
+    }
+}
+
+// n_queries baby sets [q][B][2][L][N] against the same n_blocks encoded blocks -> inner [q][n_blocks][G][2][L][N]
+int launch_mac_batch(hann_ctx* c, const u64* baby, int n_queries, const u64* pt, int64_t n_blocks, u64* inner) {
+    if (n_blocks <= 0 || n_queries <= 0) return HANN_OK;
     const long long LN = (long long)c->L * c->N;
     const long long n_bg = n_blocks * c->G;
+    const int64_t baby_stride = (int64_t)c->B * 2 * LN, inner_stride = n_bg * 2 * LN;
     bool small = c->N >= 32 && c->B <= 128;
     for (int l = 0; l < c->L; l++) small = small && c->mod[l] < (1ULL << 50);
     if (small) {
-        switch (c->B) {
-            case 1: launch_mac_stream<1, 1>(c, baby, pt, n_bg, inner); break;
-            case 2: launch_mac_stream<2, 1>(c, baby, pt, n_bg, inner); break;
-            case 4: launch_mac_stream<4, 1>(c, baby, pt, n_bg, inner); break;
-            case 8: launch_mac_stream<4, 2>(c, baby, pt, n_bg, inner); break;
-            case 16: launch_mac_stream<4, 4>(c, baby, pt, n_bg, inner); break;
-            case 32: launch_mac_stream<4, 8>(c, baby, pt, n_bg, inner); break;
-            case 64: launch_mac_stream<8, 8>(c, baby, pt, n_bg, inner); break;
-            default: launch_mac_stream<8, 16>(c, baby, pt, n_bg, inner); break;
-        }
+        // pairs of queries share one pass over the plaintexts (B <= 32: the baby-step words of two queries fit the
+        // register file); a last odd query, and every query of wider baby sets, takes a pass of its own
+        int q = 0;
+        if (c->B <= 32)
+            for (; q + 2 <= n_queries; q += 2) launch_mac_stream_b<2>(c, baby + q * baby_stride, baby_stride, pt, n_bg, inner + q * inner_stride, inner_stride);
+        for (; q < n_queries; q++) launch_mac_stream_b<1>(c, baby + q * baby_stride, baby_stride, pt, n_bg, inner + q * inner_stride, inner_stride);
         return check_launch(c, "mac_stream");
     }
     int gx = (int)((LN + kThreads - 1) / kThreads);
@@ -513,11 +542,16 @@ int launch_mac(hann_ctx* c, const u64* baby, const u64* pt, int64_t n_blocks, u6
     // enough CTAs to fill the machine even for a single small block
     while ((long long)gx * gy < 148 * 8 && gy < n_bg) gy *= 2;
     if (gy > n_bg) gy = (int)n_bg;
-    {
+    for (int q = 0; q < n_queries; q++) {
         KProf kp(c, KC_MAC);
-        k_mac<<<dim3(gx, gy), kThreads, 0, c->stream>>>(baby, pt, inner, c->N, c->L, c->B, c->G, n_bg, c->lt);
+        k_mac<<<dim3(gx, gy), kThreads, 0, c->stream>>>(baby + q * baby_stride, pt, inner + q * inner_stride, c->N, c->L, c->B, c->G, n_bg,
+                                                        c->lt);
     }
     return check_launch(c, "mac");
+}
+
+int launch_mac(hann_ctx* c, const u64* baby, const u64* pt, int64_t n_blocks, u64* inner) {
+    return launch_mac_batch(c, baby, 1, pt, n_blocks, inner);
 }
 
 int launch_lift_digits(hann_ctx* c, const u64* src, int64_t src_stride, int64_t nitems, u64* digits) {

@@ -302,3 +302,41 @@ def test_compacted_scores_bit_exact_and_decrypt(logN, L, big, n_rows):
             assert np.abs(got - full).max() < 12 * sigma   # product-of-Gaussians tails, see the oracle's pin
             got_o = np.stack([o.decrypt_compact_slots(p.km.s, small_g[blk], 2 * ps.log_scale).real for blk in range(nb)])
             assert np.abs(got - got_o).max() < 1e-9 * max(1.0, np.abs(got_o).max()) + 2 * sigma * 1e-6
+
+
+@pytest.mark.parametrize("logN,R,B,L,big,n_rows,nq", [(6, 8, 2, 2, False, 70, 3), (10, 64, 8, 2, False, 1200, 5), (11, 32, 32, 4, True, 1100, 2)])
+def test_cross_query_batch_matches_single_queries(logN, R, B, L, big, n_rows, nq):
+    """Several queries against the same encoded blocks in one call: every query's partial sums are bit-identical to the
+    oracle's multiply-accumulate with that query's baby set (and hence to the single-query call), and the scores
+    decrypt within tolerance."""
+    import torch
+
+    ps = synth.ParamSet("b%d" % logN, logN, synth.Q50, synth.P60, 40, R, B, -18) if big else synth.small_params(logN, R, B, L=L)
+    p = Pair(ps, key_seed=logN + 7)
+    g, o, b = p.g, p.o, p.b
+    rows = synth.toy_corpus(logN, rows=n_rows, dim=R)
+    nb = g.n_blocks(n_rows)
+    pt = g.encode_candidates(torch_rows(p, rows), p.ws)
+    pt_o = [o.encode_block(rows[blk * ps.n:(blk + 1) * ps.n]) for blk in range(nb)]
+    babies = g.alloc(nq * g.sizeof(b.SIZE_BABY))
+    words = g.sizeof(b.SIZE_BABY) // 8
+    qvs, baby_os = [], []
+    for q in range(nq):
+        qv = synth.toy_query(100 + q, dim=R)
+        ct_o, ct_g = p.query(qv)
+        g.query_prepare(g.import_(b.KIND_CT, ct_g, 1), p.ws, babies[q * words:(q + 1) * words])
+        qvs.append(qv)
+        baby_os.append(o.baby_set(ct_o, p.evk_o))
+    inner = g.score_level_batch(babies, nq, pt, nb, p.ws)
+    single = g.score_level(babies[words:2 * words], pt, nb, p.ws)
+    g.sync()
+    iw = nb * g.sizeof(b.SIZE_INNER) // 8
+    assert torch.equal(inner[iw:2 * iw], single[:iw])
+    inner_g = g.export(b.KIND_CT, inner, nq * nb * ps.G).reshape(nq, nb, ps.G, 2, ps.L, ps.N)
+    for q in range(nq):
+        for blk in range(nb):
+            assert np.array_equal(inner_g[q, blk], o.mac(pt_o[blk], baby_os[q]))
+    score = g.rotate_sum(inner, nq * nb, p.ws)
+    got = g.decrypt_scores(p.km.s, g.export(b.KIND_CT, score, nq * nb)).reshape(nq, nb * ps.n)[:, :n_rows]
+    for q in range(nq):
+        assert np.abs(got[q] - rows.astype(np.float64) @ qvs[q].astype(np.float64)).max() < 2.0 ** ps.tol_log2

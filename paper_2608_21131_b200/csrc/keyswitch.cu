@@ -1,7 +1,10 @@
 // Element-wise kernels of the scoring path: ciphertext x plaintext multiply-accumulate, the pieces of hybrid key
 // switching (digit lift, inner product with the evaluation key, ModDown), the automorphism gather, and the small
 // helpers of the client half.  All polynomials are [.][limb][N] arrays of 64-bit residues in [0, q).
+#include <cuda.h>
+
 #include "internal.h"
+#include "bulkcopy.cuh"
 
 namespace {
 
@@ -143,6 +146,117 @@ __global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ 
 #pragma unroll
         for (int k = 0; k < BB; k++) cur[k] = nxt[k];
         p += (long long)B * LN;
+    }
+}
+
+// The single-query kernel with the plaintext rows brought in by bulk asynchronous copies.  With register prefetch a warp
+// has 2 KiB in flight and an SM 32 KiB, short of what the memory latency needs at full bandwidth; here every warp runs its
+// own ring of kMacStages buffers (one (blk, g) pair of its BB rows each, 256 B per row: ONE box of a 2-D tensor map over
+// the plaintexts, rows = (blk, g, b), columns = limb positions), refilled by lane 0 as soon as the warp has taken a pair
+// into registers, so an SM keeps about four times as much in flight and the registers of the prefetch
+// are free.  Completion is signalled on per-buffer mbarriers; waits are bounded, and a warp whose wait runs out raises the
+// context's kernel flag and lets the whole CTA leave at its next barrier.
+constexpr int kMacStages = 4;
+
+template <int NG, int BB>
+__global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ baby, const __grid_constant__ CUtensorMap pt_map,
+                                                      u64* __restrict__ inner, int N, int L, long long n_bg, int bg_per_cta,
+                                                      const LimbConst* __restrict__ lt, int* kflag) {
+    constexpr int B = NG * BB;
+    __shared__ __align__(128) u64 ring[NG][kMacStages][BB][32];
+    __shared__ u64 part[2][NG][6][32];
+    __shared__ __align__(8) u64 bars[NG][kMacStages];
+    __shared__ int s_abort;
+    const long long LN = (long long)L * N;
+    const long long pos0 = (long long)blockIdx.x * 32;
+    const int lane = threadIdx.x & 31, wg = threadIdx.x >> 5;
+    const LimbConst* lc = lt + pos0 / N;
+    const long long bg0 = (long long)blockIdx.y * bg_per_cta;
+    const long long bg1 = bg0 + bg_per_cta < n_bg ? bg0 + bg_per_cta : n_bg;
+    if (bg0 >= bg1) return;
+    const int npairs = (int)(bg1 - bg0);
+    const unsigned bar0 = smem_addr(&bars[wg][0]), ring0 = smem_addr(&ring[wg][0][0][0]);
+    const int row0 = (int)(bg0 * B + wg * BB);  // first plaintext row of this warp's pair 0; pair i starts B rows further
+    if (threadIdx.x == 0) s_abort = 0;
+    if (lane == 0) {
+        for (int st = 0; st < kMacStages; st++) mbar_init(bar0 + 8 * st, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        for (int i = 0; i < kMacStages && i < npairs; i++) {
+            mbar_expect_tx(bar0 + 8 * i, BB * 256);
+            tensor_load_2d(ring0 + i * BB * 256, &pt_map, (int)pos0, row0 + i * B, bar0 + 8 * i);
+        }
+    }
+    // this warp's baby-step words, split into 25-bit halves
+    unsigned w0[BB][2], w1[BB][2];
+#pragma unroll
+    for (int k = 0; k < BB; k++)
+#pragma unroll
+        for (int c = 0; c < 2; c++) {
+            const u64 v = baby[((long long)(wg * BB + k) * 2 + c) * LN + pos0 + lane];
+            w0[k][c] = (unsigned)v & kM25;
+            w1[k][c] = (unsigned)(v >> 25);
+        }
+    __syncthreads();  // s_abort and the barriers are initialised
+    for (int i = 0; i < npairs; i++) {
+        const int st = i % kMacStages;
+        const bool arrived = mbar_wait(bar0 + 8 * st, (unsigned)(i / kMacStages) & 1u);
+        if (!arrived && lane == 0) {
+            atomicExch(kflag, 1);
+            s_abort = 1;
+        }
+        u64 cur[BB];
+#pragma unroll
+        for (int k = 0; k < BB; k++) cur[k] = ring[wg][st][k][lane];
+        // every lane holds its words: order the reads before the asynchronous refill of the buffer
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0 && arrived && i + kMacStages < npairs) {
+            mbar_expect_tx(bar0 + 8 * st, BB * 256);
+            tensor_load_2d(ring0 + st * BB * 256, &pt_map, (int)pos0, row0 + (i + kMacStages) * B, bar0 + 8 * st);
+        }
+        u64 p00[2] = {0, 0}, p11[2] = {0, 0}, pm[2] = {0, 0};
+#pragma unroll
+        for (int k = 0; k < BB; k++) {
+            const unsigned a0 = (unsigned)cur[k] & kM25, a1 = (unsigned)(cur[k] >> 25), as = a0 + a1;
+#pragma unroll
+            for (int c = 0; c < 2; c++) {
+                p00[c] += (u64)a0 * w0[k][c];
+                p11[c] += (u64)a1 * w1[k][c];
+                pm[c] += (u64)as * (w0[k][c] + w1[k][c]);
+            }
+        }
+        u64(*buf)[6][32] = part[i & 1];
+#pragma unroll
+        for (int c = 0; c < 2; c++) {
+            buf[wg][c * 3 + 0][lane] = p00[c];
+            buf[wg][c * 3 + 1][lane] = pm[c];
+            buf[wg][c * 3 + 2][lane] = p11[c];
+        }
+        __syncthreads();
+        if (s_abort) {
+            // leave together; first give this warp's copies still in flight the same bounded time
+            for (int j = i + 1; j < npairs && j < i + kMacStages; j++) mbar_wait(bar0 + 8 * (j % kMacStages), (unsigned)(j / kMacStages) & 1u);
+            return;
+        }
+        for (int c = wg; c < 2; c += NG) {
+            u64 s00 = 0, sm = 0, s11 = 0;
+#pragma unroll
+            for (int g = 0; g < NG; g++) {
+                s00 += buf[g][c * 3 + 0][lane];
+                sm += buf[g][c * 3 + 1][lane];
+                s11 += buf[g][c * 3 + 2][lane];
+            }
+            const u64 cross = sm - s00 - s11;
+            u64 lo = s00, hi = 0;
+            const u64 c_lo = cross << 25, c_hi = cross >> 39;
+            lo += c_lo;
+            hi += c_hi + (lo < c_lo ? 1 : 0);
+            const u64 d_lo = s11 << 50, d_hi = s11 >> 14;
+            lo += d_lo;
+            hi += d_hi + (lo < d_lo ? 1 : 0);
+            inner[((bg0 + i) * 2 + c) * LN + pos0 + lane] = reduce128(hi, lo, *lc);
+        }
+        if (NG == 1) __syncthreads();
     }
 }
 
@@ -489,6 +603,30 @@ int check_launch(hann_ctx* c, const char* what) {
     return HANN_OK;
 }
 
+// 2-D tiled tensor map over the plaintexts of a level: `rows` rows of LN 64-bit words, boxes of box_rows x 32 words.  The
+// encoder is a driver entry point, looked up once (no link against the driver library); false if it cannot be had.
+typedef CUresult (*TensorMapEncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                           const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                           CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+bool plaintext_map(const u64* pt, long long LN, long long rows, int box_rows, CUtensorMap* out) {
+    static TensorMapEncodeTiledFn encode = [] {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult res;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &res) != cudaSuccess || res != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            fn = nullptr;
+        }
+        return (TensorMapEncodeTiledFn)fn;
+    }();
+    if (!encode) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)LN, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)LN * 8};
+    const cuuint32_t box[2] = {32, (cuuint32_t)box_rows};
+    const cuuint32_t elem_strides[2] = {1, 1};
+    return encode(out, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, (void*)pt, dims, strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int NG, int BB, int NQ>
 void launch_mac_stream(hann_ctx* c, const u64* baby, int64_t baby_stride, const u64* pt, int64_t n_bg, u64* inner,
                        int64_t inner_stride) {
@@ -501,6 +639,17 @@ void launch_mac_stream(hann_ctx* c, const u64* baby, int64_t baby_stride, const 
     const int per = (int)((n_bg + split - 1) / split);
     split = (int)((n_bg + per - 1) / per);
     KProf kp(c, KC_MAC);
+#ifndef HANN_NO_MAC_BULK
+    // one query, up to 32 baby steps (the rings of wider CTAs would not fit the static shared memory), 16-byte aligned
+    // plaintexts, row count within a 32-bit coordinate: the tensor-copy kernel
+    if constexpr (NQ == 1 && NG * BB <= 32) {
+        CUtensorMap map;
+        if (((uintptr_t)pt & 15) == 0 && n_bg * (NG * BB) < (1LL << 31) && plaintext_map(pt, LN, n_bg * (NG * BB), BB, &map)) {
+            k_mac_bulk<NG, BB><<<dim3(tiles, split), 32 * NG, 0, c->stream>>>(baby, map, inner, c->N, c->L, n_bg, per, c->lt_dev, c->kflag);
+            return;
+        }
+    }
+#endif
     k_mac_stream<NG, BB, NQ><<<dim3(tiles, split), 32 * NG, 0, c->stream>>>(baby, baby_stride, pt, inner, inner_stride, c->N, c->L, n_bg,
                                                                              per, c->lt_dev);
 }

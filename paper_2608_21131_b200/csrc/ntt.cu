@@ -35,6 +35,7 @@
 #include <algorithm>
 
 #include "internal.h"
+#include "bulkcopy.cuh"
 #include "nttcore.cuh"
 
 namespace {
@@ -261,44 +262,6 @@ __global__ void __launch_bounds__(256, HANN_B8_MINBLOCKS) k_ntt_fwd_b8(NttArgs A
 // without padding.  Every wait on an mbarrier is bounded; a warp whose wait runs out raises the context's kernel flag
 // and stops.
 constexpr int kTK = 2, kTP = 8;       // chunks per CTA, polynomials per tile (= warps per CTA)
-constexpr unsigned long long kWaitLimitNs = 1000000000ULL;
-
-__device__ __forceinline__ unsigned smem_addr(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void bulk_load(unsigned dst, const void* src, unsigned bytes, unsigned bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src),
-                 "r"(bytes), "r"(bar)
-                 : "memory");
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-// bounded: gives up (false) one second after the first unsuccessful probe
-__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity) {
-    unsigned long long t0 = 0;
-    for (unsigned it = 0;; it++) {
-        unsigned ok;
-        asm volatile(
-            "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
-            : "=r"(ok)
-            : "r"(bar), "r"(parity)
-            : "memory");
-        if (ok) return true;
-        if ((it & 63) == 0) {
-            const unsigned long long now = global_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) return false;
-        }
-    }
-}
-
 template <class AR>
 __global__ void __launch_bounds__(256, 3) k_ntt_fwd_b8t(NttArgs A, int groups, int* kflag) {
     extern __shared__ __align__(128) u64 smraw[];

@@ -210,8 +210,12 @@ def run_ours(args):
 
     if args.lean:
         # profiling aid (ncu launch lists and captures): W warm-up steps, K steps, nothing else, no JSON line
+        if args.staged:
+            # the configuration of the per-kernel timing pass below: four calls per step on one stream, rotate-and-sum on
+            # one lane (the launch list of this mode is the one whose shares compare with the "kernels" of the JSON line)
+            ctx.kernel_profile(True)
         for _ in range(args.warmup + args.steps):
-            step()
+            step_staged() if args.staged else step()
         torch.cuda.synchronize()
         print("lean run: %d steps, %d kernel launches" % (args.warmup + args.steps, ctx.get_stats()["launches"]))
         return 0
@@ -582,6 +586,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--encode-group", type=int, default=None, help="tuning: plaintexts per encode launch group")
     ap.add_argument("--queries", type=int, default=1, help="queries batched against the level (cross-query batching mode when > 1)")
+    ap.add_argument("--staged", action="store_true", help="with --lean: run the steps as the per-kernel timing pass does")
     ap.add_argument("--lean", action="store_true", help="only run warm-up + steps (for ncu); prints no JSON line")
     args = ap.parse_args()
     if args.impl == "reference":

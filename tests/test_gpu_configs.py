@@ -26,18 +26,26 @@ class Query:
         ct_o, ct_g = p.query(qR)
         assert np.array_equal(ct_o, ct_g)
         self.ct_o = ct_o
-        self.baby = p.g.query_prepare(p.g.import_(p.b.KIND_CT, ct_g, 1), p.ws)
+        self.ct_dev = p.g.import_(p.b.KIND_CT, ct_g, 1)
+        self.baby = p.g.query_prepare(self.ct_dev, p.ws)
         self.baby_o = p.o.baby_set(ct_o, p.evk_o) if with_oracle else None
 
-    def score_level(self, rows, oracle_blocks=(), compact=False):
+    def score_level(self, rows, oracle_blocks=(), compact=False, one_call=False):
         """GPU scores of a level [n_rows]; blocks listed in oracle_blocks are compared bit for bit with the oracle"""
         p, g, b, ps = self.p, self.p.g, self.p.b, self.p.ps
         n_rows = rows.shape[0]
         nb = g.n_blocks(n_rows)
         ws = g.workspace(nb)
-        pt = g.encode_candidates(self.torch.from_numpy(np.ascontiguousarray(rows)).to(g.device), ws)
-        inner = g.score_level(self.baby, pt, nb, ws)
-        score = g.rotate_sum(inner, nb, ws)
+        rows_dev = self.torch.from_numpy(np.ascontiguousarray(rows)).to(g.device)
+        if one_call:
+            # the launch configuration bench.py times: the whole level in one hann_query_level call
+            pt, inner, score = (g.alloc(nb * g.sizeof(b.SIZE_PT_BLOCK)), g.alloc(nb * g.sizeof(b.SIZE_INNER)),
+                                g.alloc(nb * g.sizeof(b.SIZE_CT)))
+            g.query_level(self.ct_dev, rows_dev, ws, self.baby, pt, inner, score)
+        else:
+            pt = g.encode_candidates(rows_dev, ws)
+            inner = g.score_level(self.baby, pt, nb, ws)
+            score = g.rotate_sum(inner, nb, ws)
         g.sync()
         score_h = g.export(b.KIND_CT, score, nb)
         for blk in oracle_blocks:
@@ -160,6 +168,18 @@ def test_sweep_level_with_padding_groups(logN, pair16):
     qR = synth.toy_query(wl.query_seed(0), dim=128)
     q = Query(p, qR)
     q.score_level(lvl.rows, oracle_blocks=(0,))
+
+
+def test_sweep_maximum_size(pair16):
+    """the largest point of the scaling sweep, through one hann_query_level call: 2^20 wanted rows inflated to 2^22 scored
+    rows = 128 blocks (32 GiB of encoded plaintexts) at N = 2^16; first and last block at every conformance point, all
+    4,194,304 scores within 2^-18"""
+    ps2, lvl = wl.sweep_level(1 << 20, ps=synth.FULL16)
+    assert lvl.rows.shape == (1 << 22, 128)
+    q = Query(pair16, synth.toy_query(wl.query_seed(1), dim=128))
+    got, want = q.score_level(lvl.rows, oracle_blocks=(0, 127), one_call=True)
+    assert got.shape == (1 << 22,)
+    assert np.array_equal(np.argsort(-got)[:10], np.argsort(-want)[:10])
 
 
 def test_projection_under_encryption_then_scoring():

@@ -16,12 +16,13 @@ struct ArithF64 {
     typedef double T;
     typedef double2 TW;
     double q, qinv, half;
+    long long qi;
     static constexpr int kMinBlocks = HANN_F64_MINBLOCKS;
     static constexpr double kRound = 6755399441055744.0;  // 1.5 * 2^52: fl(v + kRound) - kRound = rint(v) for |v| < 2^51
     static constexpr double kTwo52 = 4503599627370496.0;
     TW ninv;
     __device__ __forceinline__ ArithF64(const LimbConst* lc)
-        : q((double)lc->q), qinv(1.0 / (double)lc->q), half((double)lc->half), ninv(make_double2(lc->ninv_bal, lc->ninv_q)) {}
+        : q((double)lc->q), qinv(1.0 / (double)lc->q), half((double)lc->half), qi((long long)lc->q), ninv(make_double2(lc->ninv_bal, lc->ninv_q)) {}
     // x - round(x/q) q; the quotient (at most 8 in magnitude) is rounded by adding 1.5 * 2^52
     __device__ __forceinline__ T reduce(T x) const {
         return __fma_rn(-__dsub_rn(__fma_rn(x, qinv, kRound), kRound), q, x);
@@ -51,8 +52,10 @@ struct ArithF64 {
     __device__ __forceinline__ u64 to_exch(T x) const { return (u64)__double_as_longlong(x); }
     __device__ __forceinline__ u64 to_canonical(T x) const {
         x = reduce(x);
-        if (x < 0.0) x += q;
-        return (u64)__double_as_longlong(__dadd_rn(x, kTwo52)) & 0x000FFFFFFFFFFFFFULL;
+        // balanced integer -> two's complement through the mantissa of 1.5 * 2^52 + x; the sign fix runs on the integer
+        // pipe, which is idle beside the FP64 pipe
+        const long long r = __double_as_longlong(__dadd_rn(x, kRound)) - 0x4338000000000000LL;
+        return (u64)(r + ((r >> 63) & qi));
     }
     __device__ __forceinline__ void fwd(T& X, T& Y, TW w) const {
         const T t = mulmod(Y, w);

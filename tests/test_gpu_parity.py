@@ -136,10 +136,11 @@ def test_toy_other_baby_step_counts():
         run_level(p, synth.toy_corpus(1, rows=2048 + 77), synth.toy_query(2))
 
 
-def test_host_buffer_level_matches_device_path():
+@pytest.mark.parametrize("n_rows", [1500, 3000, 7000])   # 1, 2 and 4 blocks
+def test_host_buffer_level_matches_device_path(n_rows):
     ps = synth.TOY
     p = Pair(ps, key_seed=3)
-    rows = synth.toy_corpus(1, rows=3000)
+    rows = synth.toy_corpus(1, rows=n_rows)
     qv = synth.toy_query(2)
     _, score_dev = run_level(p, rows, qv, check=False)
     ct_o, ct_g = p.query(qv)

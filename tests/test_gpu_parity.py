@@ -341,3 +341,29 @@ def test_cross_query_batch_matches_single_queries(logN, R, B, L, big, n_rows, nq
     got = g.decrypt_scores(p.km.s, g.export(b.KIND_CT, score, nq * nb)).reshape(nq, nb * ps.n)[:, :n_rows]
     for q in range(nq):
         assert np.abs(got[q] - rows.astype(np.float64) @ qvs[q].astype(np.float64)).max() < 2.0 ** ps.tol_log2
+
+
+@pytest.mark.parametrize(
+    "logN,R,B,L,bits,log_scale,tol,n_rows",
+    [
+        (10, 128, 64, 2, 30, 25, -10, 600),    # 64 baby steps, two giant steps: eight-warp multiply-accumulate
+        (10, 128, 128, 2, 30, 25, -10, 300),   # every step a baby step (G = 1): 127 rotation keys, no rotate-and-sum
+        (9, 16, 4, 1, 50, 20, -8, 300),        # a single ~50-bit ciphertext prime (one digit); scale^2 must stay below it
+        (9, 16, 4, 6, 40, 25, -10, 300),       # six ciphertext primes: the generic key-switch kernels
+        (11, 16, 4, 8, 36, 25, -10, 1100),     # the maximum of eight ciphertext primes, two blocks
+    ],
+)
+def test_level_bit_exact_other_shapes(logN, R, B, L, bits, log_scale, tol, n_rows):
+    """parameter shapes outside the benchmark configurations: wide baby sets, one and many ciphertext primes"""
+    from oracle.oracle import find_primes
+
+    if bits == 30:
+        ps = synth.small_params(logN, R, B, L=L).with_(log_scale=log_scale, tol_log2=tol)
+    elif bits == 50:
+        ps = synth.ParamSet("shape", logN, synth.Q50[:L], synth.P60, log_scale, R, B, tol)
+    else:
+        q = find_primes(bits, 13, L)
+        ps = synth.ParamSet("shape", logN, q, find_primes(bits + 6, 13, 1)[0], log_scale, R, B, tol)
+    p = Pair(ps, key_seed=logN + L)
+    rows = synth.toy_corpus(logN + L, rows=n_rows, dim=R)
+    run_level(p, rows, synth.toy_query(logN + L + 1, dim=R))

@@ -432,6 +432,31 @@ void orc_evk_gen(const orc_ctx *c, const int8_t *s, int r, const u64 *a, const i
     free(sq); free(sp); free(t);
 }
 
+/* Relinearisation key: the evaluation key of orc_evk_gen with s' = s*s (negacyclic square of the secret) in place of an
+ * automorphism of s: b_j = -a_j*s + e_j + F_j*s^2.  Switching d2 with it gives (ks0, ks1) with ks0 + ks1*s ~ d2*s^2. */
+void orc_rlk_gen(const orc_ctx *c, const int8_t *s, const u64 *a, const int8_t *e, u64 *evk) {
+    int N = c->N, L = c->L;
+    u64 *sq = (u64 *)malloc(8 * N), *s2 = (u64 *)malloc(8 * N), *t = (u64 *)malloc(8 * N);
+    for (int j = 0; j < L; j++)
+        for (int i = 0; i <= L; i++) {
+            u64 q = c->mod[i];
+            const u64 *aj = a + ((size_t)j * (L + 1) + i) * N;
+            u64 *bj = evk + (((size_t)j * 2 + 0) * (L + 1) + i) * N;
+            u64 *ao = evk + (((size_t)j * 2 + 1) * (L + 1) + i) * N;
+            lift_i8(s, N, q, sq);
+            orc_negacyclic_mul(c, i, sq, sq, s2);                 /* s' = s^2 */
+            orc_negacyclic_mul(c, i, aj, sq, t);
+            u64 F = (i == j) ? c->mod[L] % q : 0;
+            for (int x = 0; x < N; x++) {
+                u64 v = t[x] ? q - t[x] : 0;
+                v = addmod(v, reduce_signed(e[(size_t)j * N + x], q), q);
+                v = addmod(v, mulmod(F, s2[x], q), q);
+                bj[x] = v; ao[x] = aj[x];
+            }
+        }
+    free(sq); free(s2); free(t);
+}
+
 /* ModDown: u[L+1][N] over {q_0..q_{L-1}, p}  ->  out[L][N] = round(u / p):
  * rt = centred lift of [u]_p;  out_i = (u_i - rt) * p^{-1} mod q_i. */
 void orc_moddown(const orc_ctx *c, const u64 *u, u64 *out) {
@@ -566,6 +591,71 @@ void orc_mac(const orc_ctx *c, const u64 *pt, const u64 *baby, u64 *inner) {
                 }
                 free(t);
             }
+}
+
+/* Encrypted database (Sec. 2, deployment setting: the candidate diagonals are ciphertexts too).  Symmetric encryption of
+ * the R encoded diagonals of a block: ctdb[g][b] = (-a*s + e + pt[g][b], a).  pt[R][L][N], a[R][L][N], e[R][N]. */
+void orc_encrypt_block(const orc_ctx *c, const int8_t *s, const u64 *pt, const u64 *a, const int8_t *e, u64 *ctdb) {
+    int N = c->N, L = c->L, R = c->R;
+    u64 *sq = (u64 *)malloc(8 * N), *t = (u64 *)malloc(8 * N);
+    for (int r = 0; r < R; r++)
+        for (int l = 0; l < L; l++) {
+            u64 q = c->mod[l];
+            const u64 *ar = a + ((size_t)r * L + l) * N;
+            u64 *c0 = ctdb + (((size_t)r * 2 + 0) * L + l) * N, *c1 = ctdb + (((size_t)r * 2 + 1) * L + l) * N;
+            lift_i8(s, N, q, sq);
+            orc_negacyclic_mul(c, l, ar, sq, t);
+            for (int x = 0; x < N; x++) {
+                u64 v = t[x] ? q - t[x] : 0;
+                v = addmod(v, reduce_signed(e[(size_t)r * N + x], q), q);
+                c0[x] = addmod(v, pt[((size_t)r * L + l) * N + x], q);
+                c1[x] = ar[x];
+            }
+        }
+    free(sq); free(t);
+}
+
+/* Ciphertext x ciphertext multiply-accumulate over the baby steps: for every giant step g the degree-2 ciphertext
+ * (d0, d1, d2) = sum_b (x0*y0, x0*y1 + x1*y0, x1*y1), x = ctdb[g][b], y = baby[b]; decrypts as d0 + d1*s + d2*s^2.
+ * ctdb[R][2][L][N], baby[B][2][L][N] -> inner3[G][3][L][N]. */
+void orc_mac_ct(const orc_ctx *c, const u64 *ctdb, const u64 *baby, u64 *inner3) {
+    int N = c->N, L = c->L, B = c->B, G = c->G;
+    memset(inner3, 0, (size_t)G * 3 * L * N * 8);
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int g = 0; g < G; g++)
+        for (int l = 0; l < L; l++) {
+            u64 q = c->mod[l];
+            u64 *t = (u64 *)malloc(8 * N);
+            u64 *d0 = inner3 + (((size_t)g * 3 + 0) * L + l) * N, *d1 = inner3 + (((size_t)g * 3 + 1) * L + l) * N,
+                *d2 = inner3 + (((size_t)g * 3 + 2) * L + l) * N;
+            for (int b = 0; b < B; b++) {
+                const u64 *x0 = ctdb + ((((size_t)g * B + b) * 2 + 0) * L + l) * N, *x1 = ctdb + ((((size_t)g * B + b) * 2 + 1) * L + l) * N;
+                const u64 *y0 = baby + (((size_t)b * 2 + 0) * L + l) * N, *y1 = baby + (((size_t)b * 2 + 1) * L + l) * N;
+                orc_negacyclic_mul(c, l, x0, y0, t);
+                for (int x = 0; x < N; x++) d0[x] = addmod(d0[x], t[x], q);
+                orc_negacyclic_mul(c, l, x0, y1, t);
+                for (int x = 0; x < N; x++) d1[x] = addmod(d1[x], t[x], q);
+                orc_negacyclic_mul(c, l, x1, y0, t);
+                for (int x = 0; x < N; x++) d1[x] = addmod(d1[x], t[x], q);
+                orc_negacyclic_mul(c, l, x1, y1, t);
+                for (int x = 0; x < N; x++) d2[x] = addmod(d2[x], t[x], q);
+            }
+            free(t);
+        }
+}
+
+/* Relinearisation of one degree-2 ciphertext: (c0, c1) = (d0 + ks0, d1 + ks1), (ks0, ks1) = KeySwitch(d2) under the
+ * relinearisation key.  d[3][L][N] -> ct[2][L][N]. */
+void orc_relin(const orc_ctx *c, const u64 *d, const u64 *rlk, u64 *ct) {
+    int N = c->N, L = c->L;
+    u64 *ks0 = (u64 *)malloc((size_t)L * N * 8), *ks1 = (u64 *)malloc((size_t)L * N * 8);
+    orc_keyswitch(c, d + (size_t)2 * L * N, rlk, ks0, ks1);
+    for (int l = 0; l < L; l++)
+        for (int x = 0; x < N; x++) {
+            ct[((size_t)0 * L + l) * N + x] = addmod(d[((size_t)0 * L + l) * N + x], ks0[(size_t)l * N + x], c->mod[l]);
+            ct[((size_t)1 * L + l) * N + x] = addmod(d[((size_t)1 * L + l) * N + x], ks1[(size_t)l * N + x], c->mod[l]);
+        }
+    free(ks0); free(ks1);
 }
 
 /* score_ct = sum_g rot_{gB}(inner[g]) by Horner with the single key of rotation B:

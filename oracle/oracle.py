@@ -264,6 +264,40 @@ class Oracle:
         lib().orc_evk_gen(self.h, _p(s, i8p), C.c_int(r), _p(a, u64p), _p(e, i8p), _p(evk, u64p))
         return evk
 
+    def rlk_gen(self, s, a, e):
+        """relinearisation key (evaluation key for s^2), same layout as evk_gen"""
+        s = np.ascontiguousarray(s, dtype=np.int8)
+        a = _u64(a)
+        e = np.ascontiguousarray(e, dtype=np.int8)
+        L = self.L
+        assert a.shape == (L, L + 1, self.N) and e.shape == (L, self.N)
+        evk = np.zeros((L, 2, L + 1, self.N), dtype=np.uint64)
+        lib().orc_rlk_gen(self.h, _p(s, i8p), _p(a, u64p), _p(e, i8p), _p(evk, u64p))
+        return evk
+
+    def encrypt_block(self, s, pt, a, e):
+        """pt [G][B][L][N] (or [R][L][N]) -> ctdb [R][2][L][N] under s with the given a [R][L][N], e [R][N]"""
+        s = np.ascontiguousarray(s, dtype=np.int8)
+        pt, a = _u64(pt).reshape(self.R, self.L, self.N), _u64(a)
+        e = np.ascontiguousarray(e, dtype=np.int8)
+        assert a.shape == (self.R, self.L, self.N) and e.shape == (self.R, self.N)
+        out = np.zeros((self.R, 2, self.L, self.N), dtype=np.uint64)
+        lib().orc_encrypt_block(self.h, _p(s, i8p), _p(pt, u64p), _p(a, u64p), _p(e, i8p), _p(out, u64p))
+        return out
+
+    def mac_ct(self, ctdb, baby):
+        ctdb, baby = _u64(ctdb), _u64(baby)
+        out = np.zeros((self.G, 3, self.L, self.N), dtype=np.uint64)
+        lib().orc_mac_ct(self.h, _p(ctdb, u64p), _p(baby, u64p), _p(out, u64p))
+        return out
+
+    def relin(self, d, rlk):
+        d, rlk = _u64(d), _u64(rlk)
+        assert d.shape == (3, self.L, self.N)
+        out = np.zeros((2, self.L, self.N), dtype=np.uint64)
+        lib().orc_relin(self.h, _p(d, u64p), _p(rlk, u64p), _p(out, u64p))
+        return out
+
     def moddown(self, u):
         u = _u64(u)
         out = np.zeros((self.L, self.N), dtype=np.uint64)

@@ -488,3 +488,103 @@ def test_compacted_scores_decrypt_to_the_same_scores():
     sigma = rescale_error_sigma(ps.N, 2.0 ** 50 / ps.q[-1])
     err = np.abs(got.real - o.decrypt_slots(km.s, sc, 2 * ps.log_scale).real)
     assert sigma / 3 < err.std() and err.max() < 12 * sigma
+
+
+# ------------------------------------------------------------------ encrypted database: ct x ct, relinearisation
+
+
+def db_material(ps, seed):
+    """uniform a [R][L][N] and small e [R][N] for the symmetric encryption of one block's diagonals"""
+    a = synth.uniform_residues(seed, 40, list(ps.q), ps.N, lead=(ps.R,))
+    e = synth.rounded_gaussian(seed, 41, (ps.R, ps.N))
+    return a, e
+
+
+def test_ct_times_ct_decrypts_to_the_product_and_relinearises():
+    """Degree-2 decryption d0 + d1 s + d2 s^2 of the ct x ct multiply-accumulate, computed here with schoolbook python
+    integers, equals sum_b (x0 + x1 s)(y0 + y1 s) limb by limb; relinearisation changes that value by no more than the
+    key-switch noise; noise-free everything reproduces the plain matrix-vector product."""
+    ps = synth.small_params(5, 4, 2, L=2)
+    o = make(ps)
+    km = synth.key_material(ps, 9)
+    rng = np.random.default_rng(5)
+    ctdb = np.stack([np.stack([np.stack([rand_poly(rng, ps.N, q) for q in ps.q]) for _ in range(2)]) for _ in range(ps.R)])
+    baby = np.stack([np.stack([np.stack([rand_poly(rng, ps.N, q) for q in ps.q]) for _ in range(2)]) for _ in range(ps.B)])
+    d = o.mac_ct(ctdb, baby)
+    assert d.shape == (ps.G, 3, ps.L, ps.N)
+    s_int = [int(v) for v in km.s]
+    for l, q in enumerate(ps.q):
+        sq = [v % q for v in s_int]
+        s2 = schoolbook_negacyclic(sq, sq, q)
+        for g in range(ps.G):
+            want = [0] * ps.N
+            for b in range(ps.B):
+                x = ctdb[g * ps.B + b, :, l]
+                y = baby[b, :, l]
+                xs = [(int(u) + int(v)) % q for u, v in zip(x[0], schoolbook_negacyclic(x[1], sq, q))]
+                ys = [(int(u) + int(v)) % q for u, v in zip(y[0], schoolbook_negacyclic(y[1], sq, q))]
+                want = [(u + v) % q for u, v in zip(want, schoolbook_negacyclic(xs, ys, q))]
+            got = [(int(a0) + int(a1) + int(a2)) % q for a0, a1, a2 in
+                   zip(d[g, 0, l], schoolbook_negacyclic(d[g, 1, l], sq, q), schoolbook_negacyclic(d[g, 2, l], s2, q))]
+            assert got == want
+    # relinearisation: c0 + c1 s = d0 + d1 s + d2 s^2 + (key-switch error), error within the analytic bound of the key switch
+    ka = synth.uniform_residues(77, 50, list(ps.q) + [ps.p], ps.N, lead=(ps.L,))
+    ke = synth.rounded_gaussian(77, 51, (ps.L, ps.N))
+    rlk = o.rlk_gen(km.s, ka, ke)
+    Q = 1
+    for q in ps.q:
+        Q *= q
+    for g in range(ps.G):
+        ct = o.relin(d[g], rlk)
+        lhs = o.decrypt_int(km.s, ct)
+        deg2 = []
+        for l, q in enumerate(ps.q):
+            sq = [v % q for v in s_int]
+            s2 = schoolbook_negacyclic(sq, sq, q)
+            deg2.append(np.array([(int(a0) + int(a1) + int(a2)) % q for a0, a1, a2 in
+                                  zip(d[g, 0, l], schoolbook_negacyclic(d[g, 1, l], sq, q), schoolbook_negacyclic(d[g, 2, l], s2, q))],
+                                 dtype=np.uint64))
+        rhs = o.crt_centred(np.stack(deg2))
+        err = np.array([float((int(a) - int(b) + Q // 2) % Q - Q // 2) for a, b in zip(lhs, rhs)])
+        sigma = math.sqrt(ps.L * ps.N * 3.2 ** 2 * (max(ps.q) / ps.p) ** 2 / 12 + ps.N / 18)
+        assert np.abs(err).max() < 8 * sigma and err.std() > sigma / 4
+
+
+def test_encrypted_database_scores_within_tolerance():
+    """toy primes, N = 2^10: diagonals encrypted under the same key, ct x ct multiply-accumulate, relinearisation, the
+    unchanged rotate-and-sum: decrypted scores within 2^-10 of the float64 dot products; without noise the result is
+    bit-identical to the plaintext-database path"""
+    ps = synth.small_params(10, 16, 4, L=2)
+    o = make(ps)
+    rows = synth.toy_corpus(4, rows=ps.n - 7, dim=16)
+    qv = synth.toy_query(5, dim=16)
+    for zero in (False, True):
+        km = synth.key_material(ps, 3, zero_noise=zero)
+        evk = all_keys(o, km)
+        ka = synth.uniform_residues(78, 50, list(ps.q) + [ps.p], ps.N, lead=(ps.L,))
+        ke = np.zeros((ps.L, ps.N), dtype=np.int8) if zero else synth.rounded_gaussian(78, 51, (ps.L, ps.N))
+        rlk = o.rlk_gen(km.s, ka, ke)
+        ct = o.encrypt_query(km.s, qv, km.ct_a, km.ct_e)
+        baby = o.baby_set(ct, evk)
+        pt = o.encode_block(rows)
+        a, e = db_material(ps, 21)
+        if zero:
+            e = np.zeros_like(e)
+        ctdb = o.encrypt_block(km.s, pt, a, e)
+        # each database ciphertext decrypts to its diagonal plus its error array
+        for r in (0, ps.R - 1):
+            mu = o.decrypt_residues(km.s, ctdb[r])
+            want = (pt.reshape(ps.R, ps.L, ps.N)[r, 0].astype(object) + e[r].astype(object)) % ps.q[0]
+            assert [int(v) for v in mu[0]] == [int(v) for v in want]
+        d = o.mac_ct(ctdb, baby)
+        inner = np.stack([o.relin(d[g], rlk) for g in range(ps.G)])
+        score = o.rotate_sum(inner, evk[ps.B - 1])
+        got = o.decrypt_slots(km.s, score, 2 * ps.log_scale).real
+        want = np.zeros(ps.n); want[: ps.n - 7] = rows.astype(np.float64) @ qv.astype(np.float64)
+        assert np.abs(got - want).max() < 2.0 ** ps.tol_log2
+        if zero:
+            plain = o.rotate_sum(o.mac(pt, baby), evk[ps.B - 1])
+            # (c0 + c1 s) agree exactly although the ciphertexts differ: same message, no noise anywhere but the roundings
+            # of ModDown, which differ -> compare decrypted integers up to those roundings
+            a_int, b_int = o.decrypt_int(km.s, score), o.decrypt_int(km.s, plain)
+            assert max(abs(int(x) - int(y)) for x, y in zip(a_int, b_int)) < 64 * ps.N

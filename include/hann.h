@@ -75,7 +75,8 @@ enum {
     HANN_SIZE_PT_BLOCK = 4, /* encoded candidates of one block of n rows: R*L*N*8 (= 16*L*R bytes a row) */
     HANN_SIZE_INNER = 5,    /* the G partial-sum ciphertexts of one block                                 */
     HANN_SIZE_EVK = 6,      /* one evaluation key in canonical layout: L*2*(L+1)*N*8                      */
-    HANN_SIZE_ROWS_PER_BLOCK = 7 /* n                                                                     */
+    HANN_SIZE_ROWS_PER_BLOCK = 7, /* n                                                                    */
+    HANN_SIZE_CTDB_BLOCK = 8 /* one ENCRYPTED block of candidates: R ciphertexts, [G][B][2][L][N] uint64      */
 };
 
 /* element kinds of `hann_import` / `hann_export` */
@@ -138,6 +139,17 @@ int hann_kernel_times(hann_ctx *ctx, double *ms, uint64_t *launches);
 int hann_keygen_from_samples(hann_ctx *ctx, const int8_t *s, int n_rot, const int32_t *rot, const uint64_t *a,
                              const int8_t *e, uint64_t *evk_out);
 
+/* Relinearisation key (Sec. 2, encrypted database): the evaluation key for s' = s*s in the layout of
+ * hann_keygen_from_samples for ONE key; a [L][L+1][N], e [L][N], evk_out [L][2][L+1][N].  hann_load_keys takes it under
+ * rotation number 0. */
+int hann_keygen_relin_from_samples(hann_ctx *ctx, const int8_t *s, const uint64_t *a, const int8_t *e, uint64_t *evk_out);
+
+/* Enrolment of an encrypted block (Sec. 2: in deployment the candidate diagonals are ciphertexts): symmetric
+ * encryption of the R encoded plaintexts of one block, ctdb[g][b] = (pt[g][b] - a*s + e, a).
+ *   pt_dev one block as written by hann_encode_candidates (device, internal layout); a [R][L][N] uniform residues
+ *   (canonical, host or device); e [R][N] int8 (host); ctdb_dev HANN_SIZE_CTDB_BLOCK bytes (device, internal). */
+int hann_encrypt_block(hann_ctx *ctx, const int8_t *s, const void *pt_dev, const uint64_t *a, const int8_t *e, void *ctdb_dev);
+
 /* Symmetric encryption of a query: the slot vector holds q[i mod R] (q zero-padded from `dim` to R and tiled
  * n/R times), encoded at scale Delta by the canonical encoder, then ct = (-a*s + e + m, a).
  *   q [dim] float32, dim <= R;  a [L][N] uniform residues;  e [N] int8;  ct_out [2][L][N] canonical. */
@@ -190,6 +202,14 @@ int hann_score_level(hann_ctx *ctx, const void *baby_dev, const void *pt_dev, in
  * Each query's result is bit-identical to hann_score_level on its own. */
 int hann_score_level_batch(hann_ctx *ctx, const void *baby_dev, int n_queries, const void *pt_dev, int64_t n_blocks,
                            void *inner_dev, void *ws, size_t ws_bytes);
+
+/* The multiply-accumulate against an ENCRYPTED block (Sec. 2, deployment setting): for every (blk, g) the degree-2
+ * ciphertext sum_b ctdb[blk][g][b] (x) baby[b] = (x0 y0, x0 y1 + x1 y0, x1 y1) accumulated over the baby steps, then ONE
+ * relinearisation per (blk, g): (d0 + ks0, d1 + ks1) with (ks0, ks1) the key switch of d2 under the relinearisation key
+ * (loaded as rotation 0).  inner_dev as for hann_score_level (n_blocks * HANN_SIZE_INNER bytes); hann_rotate_sum follows
+ * unchanged.  Ciphertext primes below 2^56, B <= 128.  ctdb_dev n_blocks * HANN_SIZE_CTDB_BLOCK bytes. */
+int hann_score_level_ctdb(hann_ctx *ctx, const void *baby_dev, const void *ctdb_dev, int64_t n_blocks, void *inner_dev,
+                          void *ws, size_t ws_bytes);
 
 /* Rotate-and-sum: score_ct[blk] = sum_g rot_{g*B}(inner[blk][g]), evaluated by Horner with the single key of
  * rotation B: acc = inner[G-1]; for g = G-2..0: acc = rot_B(acc) + inner[g].

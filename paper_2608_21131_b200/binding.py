@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libhann.so")
 
 HANN_MAX_PRIMES = 8
 OK, EINVAL, ESHAPE, ENOKEY, EWORKSPACE, ECUDA, ENOMEM = 0, -1, -2, -3, -4, -5, -6
-SIZE_POLY, SIZE_CT, SIZE_BABY, SIZE_PT_BLOCK, SIZE_INNER, SIZE_EVK, SIZE_ROWS_PER_BLOCK = 1, 2, 3, 4, 5, 6, 7
+SIZE_POLY, SIZE_CT, SIZE_BABY, SIZE_PT_BLOCK, SIZE_INNER, SIZE_EVK, SIZE_ROWS_PER_BLOCK, SIZE_CTDB_BLOCK = 1, 2, 3, 4, 5, 6, 7, 8
 KIND_POLY, KIND_CT, KIND_PT = 1, 2, 3
 TUNE_ENCODE_GROUP = 1
 
@@ -78,6 +78,9 @@ def load_library():
         "hann_query_prepare": (C.c_int, [vp, vp, vp, vp, sz]),
         "hann_encode_candidates": (C.c_int, [vp, vp, i64, C.c_int, vp, vp, sz]),
         "hann_score_level": (C.c_int, [vp, vp, vp, i64, vp, vp, sz]),
+        "hann_keygen_relin_from_samples": (C.c_int, [vp, vp, vp, vp, vp]),
+        "hann_encrypt_block": (C.c_int, [vp, vp, vp, vp, vp, vp]),
+        "hann_score_level_ctdb": (C.c_int, [vp, vp, vp, i64, vp, vp, sz]),
         "hann_score_level_batch": (C.c_int, [vp, vp, C.c_int, vp, i64, vp, vp, sz]),
         "hann_rotate_sum": (C.c_int, [vp, vp, i64, vp, vp, sz]),
         "hann_keyswitch": (C.c_int, [vp, C.c_int, vp, vp, vp, vp, sz]),
@@ -207,6 +210,23 @@ class Context:
         self._ck(self.lib.hann_keygen_from_samples(self.h, _ptr(s), len(rots), _ptr(rots), _ptr(a), _ptr(e), _ptr(evk)))
         return evk
 
+    def keygen_relin_from_samples(self, s, a, e):
+        s, a, e = _np(s, np.int8), _np(a, np.uint64), _np(e, np.int8)
+        L, N = self.L, self.N
+        assert a.shape == (L, L + 1, N) and e.shape == (L, N) and s.shape == (N,)
+        evk = np.empty((L, 2, L + 1, N), dtype=np.uint64)
+        self._ck(self.lib.hann_keygen_relin_from_samples(self.h, _ptr(s), _ptr(a), _ptr(e), _ptr(evk)))
+        return evk
+
+    def encrypt_block(self, s, pt_block, a, e, out=None):
+        """one encoded block (device, internal) -> its R ciphertexts (device, internal)"""
+        s, a, e = _np(s, np.int8), _np(a, np.uint64), _np(e, np.int8)
+        assert a.shape == (self.R, self.L, self.N) and e.shape == (self.R, self.N)
+        if out is None:
+            out = self.alloc(self.sizeof(SIZE_CTDB_BLOCK))
+        self._ck(self.lib.hann_encrypt_block(self.h, _ptr(s), _ptr(pt_block), _ptr(a), _ptr(e), _ptr(out)))
+        return out
+
     def encrypt_query(self, s, q, a, e):
         s, q, a, e = _np(s, np.int8), _np(q, np.float32), _np(a, np.uint64), _np(e, np.int8)
         assert a.shape == (self.L, self.N) and e.shape == (self.N,)
@@ -290,6 +310,12 @@ class Context:
             inner = self.alloc(n_blocks * self.sizeof(SIZE_INNER))
         self._ck(self.lib.hann_score_level(self.h, _ptr(baby), _ptr(pt), n_blocks, _ptr(inner), _ptr(ws),
                                            ws.numel() * 8 if ws is not None else 0))
+        return inner
+
+    def score_level_ctdb(self, baby, ctdb, n_blocks, ws, inner=None):
+        if inner is None:
+            inner = self.alloc(n_blocks * self.sizeof(SIZE_INNER))
+        self._ck(self.lib.hann_score_level_ctdb(self.h, _ptr(baby), _ptr(ctdb), n_blocks, _ptr(inner), _ptr(ws), ws.numel() * 8))
         return inner
 
     def score_level_batch(self, babies, n_queries, pt, n_blocks, ws=None, inner=None):

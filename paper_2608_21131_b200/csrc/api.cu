@@ -353,6 +353,7 @@ extern "C" int64_t hann_sizeof(const hann_ctx* c, int what) {
         case HANN_SIZE_INNER: return (int64_t)c->G * 2 * L * N * 8;
         case HANN_SIZE_EVK: return L * 2 * (L + 1) * N * 8;
         case HANN_SIZE_ROWS_PER_BLOCK: return c->n;
+        case HANN_SIZE_CTDB_BLOCK: return (int64_t)c->R * 2 * L * N * 8;
         default: return HANN_EINVAL;
     }
 }
@@ -362,6 +363,7 @@ extern "C" int64_t hann_workspace_bytes(const hann_ctx* c, int64_t max_blocks) {
     const int64_t items = std::max<int64_t>(1, std::min<int64_t>(max_blocks, 8));
     int64_t w = std::max(ks_item_words(c) * items, prepare_words(c)) * 8;
     w = std::max(w, (ks_item_words(c) + (int64_t)c->L * c->N) * 8);  // hann_keyswitch permutes its input first
+    w = std::max(w, (ks_item_words(c) + 3 * (int64_t)c->L * c->N) * 8);  // hann_score_level_ctdb: one degree-2 sum + its key switch
     w = std::max(w, encode_ws_bytes(c));
     // hann_query_level runs query_prepare and encode_candidates side by side, each in its own part
     w = std::max(w, align256(prepare_words(c) * 8 + kSlack) + encode_ws_bytes(c));
@@ -585,6 +587,77 @@ extern "C" int hann_keygen_from_samples(hann_ctx* c, const int8_t* s, int n_rot,
     return HANN_OK;
 }
 
+extern "C" int hann_keygen_relin_from_samples(hann_ctx* c, const int8_t* s, const uint64_t* a, const int8_t* e, uint64_t* evk_out) {
+    if (!c) return HANN_EINVAL;
+    if (!s || !a || !e || !evk_out) return fail(c, HANN_EINVAL, "hann_keygen_relin_from_samples: bad argument");
+    const int L = c->L, N = c->N;
+    DeviceGuard dg(c->device);
+    const int64_t W = (int64_t)N, keyw = (int64_t)L * (L + 1) * W;
+    RET(ensure_scratch(c, (2 * (L + 1) * W + 2 * keyw) * 8 + align256(N) + align256((int64_t)L * N) + kSlack));
+    Arena ar{(char*)c->scratch, 0, c->scratch_bytes};
+    u64* shat = ar.take<u64>((L + 1) * W);
+    u64* s2 = ar.take<u64>((L + 1) * W);
+    u64* A = ar.take<u64>(keyw);
+    u64* AS = ar.take<u64>(keyw);
+    int8_t* s8 = ar.take<int8_t>(N);
+    int8_t* e8 = ar.take<int8_t>((int64_t)L * N);
+    RET(upload_secret(c, s, L + 1, s8, shat));
+    // s' = s^2: squared in the transform domain, back to coefficient-domain residues for the finish kernel
+    RET(launch_mul(c, shat, shat, L + 1, s2, L + 1, limbmap_qp(c)));
+    RET(launch_ntt_inv(c, s2, L + 1, N, limbmap_qp(c)));
+    CK(cudaMemcpyAsync(A, a, keyw * 8, cudaMemcpyHostToDevice, c->stream));
+    CK(cudaMemcpyAsync(e8, e, (size_t)L * N, cudaMemcpyHostToDevice, c->stream));
+    RET(launch_ntt_fwd(c, A, (int64_t)L * (L + 1), N, limbmap_qp(c)));
+    RET(launch_mul(c, A, shat, L + 1, AS, (int64_t)L * (L + 1), limbmap_qp(c)));
+    RET(launch_ntt_inv(c, AS, (int64_t)L * (L + 1), N, limbmap_qp(c)));
+    RET(launch_rlk_finish(c, AS, e8, s2, AS));
+    for (int j = 0; j < L; j++) {
+        CK(cudaMemcpyAsync(evk_out + ((int64_t)j * 2 + 0) * (L + 1) * W, AS + (int64_t)j * (L + 1) * W, (size_t)(L + 1) * W * 8,
+                           cudaMemcpyDeviceToHost, c->stream));
+        memcpy(evk_out + ((int64_t)j * 2 + 1) * (L + 1) * W, a + (int64_t)j * (L + 1) * W, (size_t)(L + 1) * W * 8);
+    }
+    CK(cudaStreamSynchronize(c->stream));
+    return HANN_OK;
+}
+
+extern "C" int hann_encrypt_block(hann_ctx* c, const int8_t* s, const void* pt_dev, const uint64_t* a, const int8_t* e, void* ctdb_dev) {
+    if (!c) return HANN_EINVAL;
+    if (!s || !pt_dev || !a || !e || !ctdb_dev) return fail(c, HANN_EINVAL, "hann_encrypt_block: bad argument");
+    const int L = c->L, N = c->N, R = c->R;
+    const int64_t LN = (int64_t)L * N;
+    DeviceGuard dg(c->device);
+    // pieces of up to 16 plaintexts: a (transformed) lands in the ciphertext's second half, a*s and the transformed error in
+    // the scratch
+    const int piece = 16;
+    RET(ensure_scratch(c, (LN + 2 * piece * LN) * 8 + align256(N) + align256((int64_t)piece * N) + kSlack));
+    Arena ar{(char*)c->scratch, 0, c->scratch_bytes};
+    u64* shat = ar.take<u64>(LN);
+    u64* AS = ar.take<u64>(piece * LN);
+    u64* EH = ar.take<u64>(piece * LN);
+    int8_t* s8 = ar.take<int8_t>(N);
+    int8_t* e8 = ar.take<int8_t>((int64_t)piece * N);
+    RET(upload_secret(c, s, L, s8, shat));
+    u64* ct = (u64*)ctdb_dev;
+    const u64* pt = (const u64*)pt_dev;
+    for (int r0 = 0; r0 < R; r0 += piece) {
+        const int np = std::min(piece, R - r0);
+        // c1 = transform of a, straight into place (polynomial r at ct + (2 r + 1) * LN)
+        CK(cudaMemcpy2DAsync(ct + ((int64_t)r0 * 2 + 1) * LN, (size_t)2 * LN * 8, a + (int64_t)r0 * LN, (size_t)LN * 8, (size_t)LN * 8, (size_t)np,
+                             cudaMemcpyDefault, c->stream));
+        for (int r = 0; r < np; r++) RET(launch_ntt_fwd(c, ct + ((int64_t)(r0 + r) * 2 + 1) * LN, L, N, limbmap_q(c)));
+        CK(cudaMemcpyAsync(e8, e + (int64_t)r0 * N, (size_t)np * N, cudaMemcpyHostToDevice, c->stream));
+        for (int r = 0; r < np; r++) {
+            RET(launch_mul(c, ct + ((int64_t)(r0 + r) * 2 + 1) * LN, shat, L, AS + (int64_t)r * LN, L, limbmap_q(c)));
+            RET(launch_lift_i8(c, e8 + (int64_t)r * N, L, EH + (int64_t)r * LN));
+        }
+        RET(launch_ntt_fwd(c, EH, (int64_t)np * L, N, limbmap_q(c)));
+        // c0 = pt - a*s + e, written at ct + 2 r * LN (the finish kernel strides its output by 2 * LN)
+        RET(launch_encrypt_block_finish(c, pt + (int64_t)r0 * LN, AS, EH, ct + (int64_t)r0 * 2 * LN, np));
+        CK(cudaStreamSynchronize(c->stream));  // e8 is reused by the next piece
+    }
+    return HANN_OK;
+}
+
 extern "C" int hann_encrypt_query(hann_ctx* c, const int8_t* s, const float* q, int dim, const uint64_t* a, const int8_t* e,
                                   uint64_t* ct_out) {
     if (!c) return HANN_EINVAL;
@@ -691,7 +764,7 @@ extern "C" int hann_load_keys(hann_ctx* c, const uint64_t* evk, int n_rot, const
     if (!evk || !rot || n_rot < 0) return fail(c, HANN_EINVAL, "hann_load_keys: bad argument");
     const int L = c->L, N = c->N;
     for (int i = 0; i < n_rot; i++)
-        if (rot[i] < 1 || rot[i] >= c->n) return fail(c, HANN_ESHAPE, "hann_load_keys: rotation out of range");
+        if (rot[i] < 0 || rot[i] >= c->n) return fail(c, HANN_ESHAPE, "hann_load_keys: rotation out of range");
     DeviceGuard dg(c->device);
     const int64_t keyw = (int64_t)L * 2 * (L + 1) * N;
     RET(ensure_scratch(c, keyw * 8));
@@ -795,6 +868,47 @@ extern "C" int hann_score_level_batch(hann_ctx* c, const void* baby_dev, int n_q
     DeviceGuard dg(c->device);
     Timer tm(c, 2);
     return launch_mac_batch(c, (const u64*)baby_dev, n_queries, (const u64*)pt_dev, n_blocks, (u64*)inner_dev);
+}
+
+extern "C" int hann_score_level_ctdb(hann_ctx* c, const void* baby_dev, const void* ctdb_dev, int64_t n_blocks, void* inner_dev,
+                                     void* ws, size_t ws_bytes) {
+    if (!c) return HANN_EINVAL;
+    if (n_blocks < 0 || (n_blocks > 0 && (!baby_dev || !ctdb_dev || !inner_dev))) return fail(c, HANN_EINVAL, "hann_score_level_ctdb: bad argument");
+    if (n_blocks == 0) return HANN_OK;
+    const int L = c->L, N = c->N, G = c->G;
+    for (int l = 0; l < L; l++)
+        if (c->mod[l] >= (1ULL << 56)) return fail(c, HANN_ESHAPE, "hann_score_level_ctdb: ciphertext primes must be below 2^56");
+    if (c->B > 128) return fail(c, HANN_ESHAPE, "hann_score_level_ctdb: at most 128 baby steps");
+    if (!c->keytab_host[0]) return fail(c, HANN_ENOKEY, "hann_score_level_ctdb: the relinearisation key (rotation 0) is not loaded");
+    if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_score_level_ctdb: workspace missing or not 256-byte aligned");
+    DeviceGuard dg(c->device);
+    Timer tm(c, 2);
+    const int64_t LN = (int64_t)L * N, L1N = (int64_t)(L + 1) * N, ctw = 2 * LN;
+    // per (blk, g) item: the degree-2 sum (3 polynomials) and one key switch (its own copy of d2, digits, u, lifted)
+    const int64_t per = (3 * LN + ks_item_words(c)) * 8;
+    int64_t ch = ((int64_t)ws_bytes - kSlack) / per;
+    if (ch < 1) return fail(c, HANN_EWORKSPACE, "hann_score_level_ctdb: workspace too small");
+    const int64_t items = n_blocks * G;
+    ch = std::min<int64_t>(std::min<int64_t>(ch, items), 8 * G);
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
+    u64* d = ar.take<u64>(ch * 3 * LN);
+    u64* c1c = ar.take<u64>(ch * LN);
+    u64* digits = ar.take<u64>(ch * L * L1N);
+    u64* u = ar.take<u64>(ch * 2 * L1N);
+    u64* lifted = ar.take<u64>(ch * 2 * LN);
+    if (!d || !c1c || !digits || !u || !lifted) return fail(c, HANN_EWORKSPACE, "hann_score_level_ctdb: workspace too small");
+    const u64* ctdb = (const u64*)ctdb_dev;
+    u64* inner = (u64*)inner_dev;
+    for (int64_t i0 = 0; i0 < items; i0 += ch) {
+        const int64_t ni = std::min(ch, items - i0);
+        RET(launch_mac_ct(c, (const u64*)baby_dev, ctdb + i0 * c->B * ctw, ni, d));
+        // relinearise: (d0 + ks0, d1 + ks1) with (ks0, ks1) the key switch of d2 under the key of s^2 ("rotation 0": no
+        // automorphism)
+        CK(cudaMemcpy2DAsync(c1c, LN * 8, d + 2 * LN, 3 * LN * 8, LN * 8, ni, cudaMemcpyDeviceToDevice, c->stream));
+        RET(ks_digits_to_lifted(c, c1c, ni, digits, (int64_t)L * L1N, 0, 0, ni, u, lifted));
+        RET(launch_moddown_combine(c, u, lifted, ni, 0, 0, nullptr, 0, d, 3 * LN, inner + i0 * ctw, inner + i0 * ctw + LN, ctw));
+    }
+    return HANN_OK;
 }
 
 extern "C" int hann_rotate_sum(hann_ctx* c, const void* inner_dev, int64_t n_blocks, void* score_ct_dev, void* ws, size_t ws_bytes) {

@@ -153,3 +153,7 @@ int launch_mul(hann_ctx* c, const u64* a, const u64* b, int bperiod, u64* out, i
 int launch_add(hann_ctx* c, const u64* a, const u64* b, u64* out, int64_t npoly, const LimbMap& lm);
 int launch_evk_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const int8_t* sprime, u64* b_out);
 int launch_encrypt_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const u64* m, u64* c0_out);
+// encrypted database: relinearisation key finish, block encryption finish, ct x ct multiply-accumulate
+int launch_rlk_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const u64* s2, u64* b_out);
+int launch_encrypt_block_finish(hann_ctx* c, const u64* pt, const u64* as, const u64* ehat, u64* ct, int64_t npt);
+int launch_mac_ct(hann_ctx* c, const u64* baby, const u64* ctdb, int64_t n_bg, u64* inner3);

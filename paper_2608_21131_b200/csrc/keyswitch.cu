@@ -577,6 +577,62 @@ __global__ void __launch_bounds__(kThreads) k_evk_finish(const u64* __restrict__
     }
 }
 
+// relinearisation key finish, coefficient domain: b[j][i][x] = -as[j][i][x] + e[j][x] + (i == j ? (p mod q_j) * s2[j][x] : 0),
+// s2[i][x] the residues of s^2 modulo limb i
+__global__ void __launch_bounds__(kThreads) k_rlk_finish(const u64* __restrict__ as, const int8_t* __restrict__ e,
+                                                         const u64* __restrict__ s2, u64* __restrict__ b_out, int N, int L,
+                                                         LimbTable lt) {
+    const long long total = (long long)L * (L + 1) * N;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const int x = (int)(idx % N);
+        const int i = (int)((idx / N) % (L + 1));
+        const int j = (int)(idx / ((long long)N * (L + 1)));
+        const LimbConst& lc = lt.c[i];
+        u64 v = as[idx] ? lc.q - as[idx] : 0;
+        v = addmod(v, reduce_signed((i64)e[(long long)j * N + x], lc), lc.q);
+        if (i == j) v = addmod(v, mulmod(lc.pmod, s2[(long long)i * N + x], lc), lc.q);
+        b_out[idx] = v;
+    }
+}
+
+// block encryption finish, transform domain: c0[r][l][t] = pt[r][l][t] - as[r][l][t] + ehat[r][l][t]
+__global__ void __launch_bounds__(kThreads) k_encrypt_block_finish(const u64* __restrict__ pt, const u64* __restrict__ as,
+                                                                   const u64* __restrict__ ehat, u64* __restrict__ ct, int N, int L,
+                                                                   long long npt, LimbTable lt) {
+    const long long LN = (long long)L * N, total = npt * LN;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const long long r = idx / LN, rem = idx % LN;
+        const u64 q = lt.c[(int)(rem / N)].q;
+        ct[r * 2 * LN + rem] = addmod(submod(pt[idx], as[idx], q), ehat[idx], q);
+    }
+}
+
+// ct x ct multiply-accumulate (generic, any modulus): inner3[bg][0..2][l][t] = sum_b (x0 y0, x0 y1 + x1 y0, x1 y1),
+// x = ctdb[bg][b], y = baby[b]
+__global__ void __launch_bounds__(kThreads) k_mac_ct(const u64* __restrict__ baby, const u64* __restrict__ ctdb, u64* __restrict__ inner3,
+                                                     int N, int L, int B, long long n_bg, LimbTable lt) {
+    const long long LN = (long long)L * N;
+    for (long long pos = (long long)blockIdx.x * kThreads + threadIdx.x; pos < LN; pos += (long long)gridDim.x * kThreads) {
+        const LimbConst& lc = lt.c[(int)(pos / N)];
+        for (long long bg = blockIdx.y; bg < n_bg; bg += gridDim.y) {
+            const u64* x = ctdb + bg * B * 2 * LN + pos;
+            u64 h0 = 0, l0 = 0, h1 = 0, l1 = 0, h2 = 0, l2 = 0;
+            for (int b = 0; b < B; b++) {
+                const u64 x0 = __ldcs(x + ((long long)b * 2 + 0) * LN), x1 = __ldcs(x + ((long long)b * 2 + 1) * LN);
+                const u64 y0 = baby[((long long)b * 2 + 0) * LN + pos], y1 = baby[((long long)b * 2 + 1) * LN + pos];
+                mac128(h0, l0, x0, y0);
+                mac128(h1, l1, x0, y1);
+                mac128(h1, l1, x1, y0);
+                mac128(h2, l2, x1, y1);
+            }
+            u64* o = inner3 + bg * 3 * LN + pos;
+            o[0] = reduce128(h0, l0, lc);
+            o[LN] = reduce128(h1, l1, lc);
+            o[2 * LN] = reduce128(h2, l2, lc);
+        }
+    }
+}
+
 // symmetric encryption finish, coefficient domain: c0[l][x] = -as[l][x] + e[x] + m[l][x]
 __global__ void __launch_bounds__(kThreads) k_encrypt_finish(const u64* __restrict__ as, const int8_t* __restrict__ e,
                                                              const u64* __restrict__ m, u64* __restrict__ c0, int N, int L,
@@ -874,6 +930,37 @@ int launch_evk_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const i
         k_evk_finish<<<grid_for((int64_t)c->L * (c->L + 1) * c->N), kThreads, 0, c->stream>>>(as_coeff, e, sprime, b_out, c->N, c->L, c->lt);
     }
     return check_launch(c, "evk_finish");
+}
+
+int launch_rlk_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const u64* s2, u64* b_out) {
+    {
+        KProf kp(c, KC_OTHER);
+        k_rlk_finish<<<grid_for((int64_t)c->L * (c->L + 1) * c->N), kThreads, 0, c->stream>>>(as_coeff, e, s2, b_out, c->N, c->L, c->lt);
+    }
+    return check_launch(c, "rlk_finish");
+}
+
+int launch_encrypt_block_finish(hann_ctx* c, const u64* pt, const u64* as, const u64* ehat, u64* ct, int64_t npt) {
+    {
+        KProf kp(c, KC_OTHER);
+        k_encrypt_block_finish<<<grid_for(npt * c->L * c->N), kThreads, 0, c->stream>>>(pt, as, ehat, ct, c->N, c->L, npt, c->lt);
+    }
+    return check_launch(c, "encrypt_block_finish");
+}
+
+// sums of B <= 2^7 products of residues below 2^62 fit the 128-bit accumulators only for moduli below 2^60 (two products
+// per step in d1): checked by the caller
+int launch_mac_ct(hann_ctx* c, const u64* baby, const u64* ctdb, int64_t n_bg, u64* inner3) {
+    if (n_bg <= 0) return HANN_OK;
+    const long long LN = (long long)c->L * c->N;
+    int gx = (int)((LN + kThreads - 1) / kThreads), gy = 1;
+    while ((long long)gx * gy < 148 * 8 && gy < n_bg) gy *= 2;
+    if (gy > n_bg) gy = (int)n_bg;
+    {
+        KProf kp(c, KC_MAC);
+        k_mac_ct<<<dim3(gx, gy), kThreads, 0, c->stream>>>(baby, ctdb, inner3, c->N, c->L, c->B, n_bg, c->lt);
+    }
+    return check_launch(c, "mac_ct");
 }
 
 int launch_encrypt_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const u64* m, u64* c0_out) {

@@ -367,3 +367,48 @@ def test_level_bit_exact_other_shapes(logN, R, B, L, bits, log_scale, tol, n_row
     p = Pair(ps, key_seed=logN + L)
     rows = synth.toy_corpus(logN + L, rows=n_rows, dim=R)
     run_level(p, rows, synth.toy_query(logN + L + 1, dim=R))
+
+
+@pytest.mark.parametrize("logN,R,B,L,big,n_rows", [(6, 8, 2, 2, False, 50), (10, 16, 4, 2, False, 900), (11, 32, 8, 4, True, 1500)])
+def test_encrypted_database_level_bit_exact(logN, R, B, L, big, n_rows):
+    """Encrypted candidates (ct x ct): relinearisation key, block encryption, degree-2 multiply-accumulate +
+    relinearisation and the unchanged rotate-and-sum, each bit-identical to the oracle; scores within tolerance."""
+    ps = synth.ParamSet("db%d" % logN, logN, synth.Q50, synth.P60, 40, R, B, -18) if big else synth.small_params(logN, R, B, L=L)
+    p = Pair(ps, key_seed=logN + 11)
+    g, o, b = p.g, p.o, p.b
+    ka = synth.uniform_residues(78, 50, list(ps.q) + [ps.p], ps.N, lead=(ps.L,))
+    ke = synth.rounded_gaussian(78, 51, (ps.L, ps.N))
+    rlk_o = o.rlk_gen(p.km.s, ka, ke)
+    rlk_g = g.keygen_relin_from_samples(p.km.s, ka, ke)
+    assert np.array_equal(rlk_g, rlk_o)
+    g.load_keys(rlk_g[None], [0])
+    rows = synth.toy_corpus(logN + 3, rows=n_rows, dim=R)
+    qv = synth.toy_query(logN + 4, dim=R)
+    ct_o, ct_g = p.query(qv)
+    baby = g.query_prepare(g.import_(b.KIND_CT, ct_g, 1), p.ws)
+    baby_o = o.baby_set(ct_o, p.evk_o)
+    nb = g.n_blocks(n_rows)
+    pt = g.encode_candidates(torch_rows(p, rows), p.ws)
+    ptw, dbw = g.sizeof(b.SIZE_PT_BLOCK) // 8, g.sizeof(b.SIZE_CTDB_BLOCK) // 8
+    ctdb = g.alloc(nb * dbw * 8)
+    inner_o = []
+    for blk in range(nb):
+        a = synth.uniform_residues(200 + blk, 40, list(ps.q), ps.N, lead=(ps.R,))
+        e = synth.rounded_gaussian(200 + blk, 41, (ps.R, ps.N))
+        g.encrypt_block(p.km.s, pt[blk * ptw:(blk + 1) * ptw], a, e, ctdb[blk * dbw:(blk + 1) * dbw])
+        pt_o = o.encode_block(rows[blk * ps.n:(blk + 1) * ps.n])
+        db_o = o.encrypt_block(p.km.s, pt_o, a, e)
+        db_g = g.export(b.KIND_CT, ctdb[blk * dbw:(blk + 1) * dbw], ps.R)
+        assert np.array_equal(db_g, db_o)
+        d = o.mac_ct(db_o, baby_o)
+        inner_o.append(np.stack([o.relin(d[gi], rlk_o) for gi in range(ps.G)]))
+    inner = g.score_level_ctdb(baby, ctdb, nb, p.ws)
+    inner_g = g.export(b.KIND_CT, inner, nb * ps.G).reshape(nb, ps.G, 2, ps.L, ps.N)
+    for blk in range(nb):
+        assert np.array_equal(inner_g[blk], inner_o[blk])
+    score = g.rotate_sum(inner, nb, p.ws)
+    score_g = g.export(b.KIND_CT, score, nb)
+    for blk in range(nb):
+        assert np.array_equal(score_g[blk], o.rotate_sum(inner_o[blk], p.evk_o[ps.B - 1]))
+    got = g.decrypt_scores(p.km.s, score_g).reshape(-1)[:n_rows]
+    assert np.abs(got - rows.astype(np.float64) @ qv.astype(np.float64)).max() < 2.0 ** ps.tol_log2

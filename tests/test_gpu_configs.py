@@ -228,3 +228,45 @@ def test_projection_under_encryption_then_scoring():
     got = g2.decrypt_scores(pc.km.s, score_g, log_scale_out=120).reshape(-1)[: rows.shape[0]]
     want = rows.astype(np.float64) @ qR
     assert np.abs(got - want).max() < 2.0 ** -18
+
+
+def test_projection_with_encrypted_matrix():
+    """Rank reduction as the paper deploys it (Sec. 3.1 "How": the server holds W as ENCRYPTED diagonals, so that it never
+    learns the projection): the same diagonal scorer with the encrypted block of W^T (ct x ct multiply-accumulate, one
+    relinearisation per giant step, rotate-and-sum).  Bit-identical to the oracle; the slots of the result hold the
+    projected query, tiled.  (Window packing of the chunks and the 0/1 masks of the paper's storage optimisation are
+    not built: W^T is stored as one 512-diagonal block.)"""
+    import torch
+
+    ps = synth.ParamSet("proj", 13, synth.Q50, synth.P60, 40, 512, 32, -18)
+    p = Pair(ps, key_seed=4)
+    g, o, b, n = p.g, p.o, p.b, ps.n
+    ka = synth.uniform_residues(78, 50, list(ps.q) + [ps.p], ps.N, lead=(ps.L,))
+    ke = synth.rounded_gaussian(78, 51, (ps.L, ps.N))
+    rlk_o = o.rlk_gen(p.km.s, ka, ke)
+    rlk_g = g.keygen_relin_from_samples(p.km.s, ka, ke)
+    assert np.array_equal(rlk_g, rlk_o)
+    g.load_keys(rlk_g[None], [0])
+    W = synth.projection_matrix(wl.PROJ_SEED, 512, 128)
+    WT = np.ascontiguousarray(W.T.astype(np.float32))
+    block = np.ascontiguousarray(np.tile(WT, (n // 128, 1)))
+    q512 = synth.normalise(synth.gaussian_vectors(9, synth.S_QUERY, np.arange(1), 512))[0].astype(np.float32)
+    ct_o, ct_g = p.query(q512)
+    baby = g.query_prepare(g.import_(b.KIND_CT, ct_g, 1), p.ws)
+    baby_o = o.baby_set(ct_o, p.evk_o)
+    # enrolment of W: encode its diagonals, encrypt them under the client's key
+    pt = g.encode_candidates(torch.from_numpy(block).to(g.device), p.ws)
+    a = synth.uniform_residues(300, 40, list(ps.q), ps.N, lead=(ps.R,))
+    e = synth.rounded_gaussian(300, 41, (ps.R, ps.N))
+    wdb = g.encrypt_block(p.km.s, pt, a, e)
+    wdb_o = o.encrypt_block(p.km.s, o.encode_block(block), a, e)
+    # projection under encryption, matrix and query both encrypted
+    inner = g.score_level_ctdb(baby, wdb, 1, p.ws)
+    proj = g.rotate_sum(inner, 1, p.ws)
+    g.sync()
+    d = o.mac_ct(wdb_o, baby_o)
+    proj_o = o.rotate_sum(np.stack([o.relin(d[gi], rlk_o) for gi in range(ps.G)]), p.evk_o[31])
+    assert np.array_equal(g.export(b.KIND_CT, proj, 1)[0], proj_o)
+    qR = WT.astype(np.float64) @ q512.astype(np.float64)
+    slots = g.decrypt_scores(p.km.s, proj_o[None], log_scale_out=80)[0]
+    assert np.abs(slots - np.tile(qR, n // 128)).max() < 2.0 ** -20

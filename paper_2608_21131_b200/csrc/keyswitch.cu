@@ -149,6 +149,93 @@ __global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ 
     }
 }
 
+// Streaming form of the ct x ct multiply-accumulate for moduli below 2^50: the structure of k_mac_stream (a warp keeps
+// the 25-bit halves of its BB baby-step words, both components, in registers), with the two polynomials x0, x1 of every
+// database ciphertext streamed past them one after the other: x_h * y_c adds to d_{h+c}, so the three degree-2 sums share
+// one set of Karatsuba accumulators and every database word is read once.
+template <int NG, int BB>
+__global__ void __launch_bounds__(32 * NG) k_mac_ct_stream(const u64* __restrict__ baby, const u64* __restrict__ ctdb,
+                                                           u64* __restrict__ inner3, int N, int L, long long n_bg, int bg_per_cta,
+                                                           const LimbConst* __restrict__ lt) {
+    constexpr int B = NG * BB;
+    __shared__ u64 part[2][NG][9][32];
+    const long long LN = (long long)L * N;
+    const long long pos0 = (long long)blockIdx.x * 32;
+    const int lane = threadIdx.x & 31, wg = threadIdx.x >> 5;
+    const LimbConst* lc = lt + pos0 / N;
+    unsigned w0[BB][2], w1[BB][2];
+#pragma unroll
+    for (int k = 0; k < BB; k++)
+#pragma unroll
+        for (int c = 0; c < 2; c++) {
+            const u64 v = baby[((long long)(wg * BB + k) * 2 + c) * LN + pos0 + lane];
+            w0[k][c] = (unsigned)v & kM25;
+            w1[k][c] = (unsigned)(v >> 25);
+        }
+    const long long bg0 = (long long)blockIdx.y * bg_per_cta;
+    const long long bg1 = bg0 + bg_per_cta < n_bg ? bg0 + bg_per_cta : n_bg;
+    if (bg0 >= bg1) return;
+    // polynomial h of the ciphertext of (pair bg, step b): ctdb + ((bg * B + b) * 2 + h) * LN
+    const u64* p = ctdb + ((bg0 * B + wg * BB) * 2) * LN + pos0 + lane;
+    u64 cur[BB], nxt[BB];
+#pragma unroll
+    for (int k = 0; k < BB; k++) cur[k] = __ldcs(p + (long long)k * 2 * LN);
+    for (long long bg = bg0; bg < bg1; bg++) {
+        u64 p00[3] = {0, 0, 0}, p11[3] = {0, 0, 0}, pm[3] = {0, 0, 0};
+#pragma unroll
+        for (int h = 0; h < 2; h++) {
+            // next stream element: the other polynomial of this pair, or x0 of the next pair
+            const bool more = h == 0 || bg + 1 < bg1;
+            if (more) {
+                const u64* pn = h == 0 ? p + LN : p + (long long)B * 2 * LN;
+#pragma unroll
+                for (int k = 0; k < BB; k++) nxt[k] = __ldcs(pn + (long long)k * 2 * LN);
+            }
+#pragma unroll
+            for (int k = 0; k < BB; k++) {
+                const unsigned a0 = (unsigned)cur[k] & kM25, a1 = (unsigned)(cur[k] >> 25), as = a0 + a1;
+#pragma unroll
+                for (int c = 0; c < 2; c++) {
+                    p00[h + c] += (u64)a0 * w0[k][c];
+                    p11[h + c] += (u64)a1 * w1[k][c];
+                    pm[h + c] += (u64)as * (w0[k][c] + w1[k][c]);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < BB; k++) cur[k] = nxt[k];
+        }
+        p += (long long)B * 2 * LN;
+        u64(*buf)[9][32] = part[bg & 1];
+#pragma unroll
+        for (int c = 0; c < 3; c++) {
+            buf[wg][c * 3 + 0][lane] = p00[c];
+            buf[wg][c * 3 + 1][lane] = pm[c];
+            buf[wg][c * 3 + 2][lane] = p11[c];
+        }
+        __syncthreads();
+        for (int c = wg; c < 3; c += NG) {
+            u64 s00 = 0, sm = 0, s11 = 0;
+#pragma unroll
+            for (int g = 0; g < NG; g++) {
+                s00 += buf[g][c * 3 + 0][lane];
+                sm += buf[g][c * 3 + 1][lane];
+                s11 += buf[g][c * 3 + 2][lane];
+            }
+            // d1 sums 2 B products: B <= 64 keeps the 25-bit-half sums below 2^57 and the half-sum products below 2^59
+            const u64 cross = sm - s00 - s11;
+            u64 lo = s00, hi = 0;
+            const u64 c_lo = cross << 25, c_hi = cross >> 39;
+            lo += c_lo;
+            hi += c_hi + (lo < c_lo ? 1 : 0);
+            const u64 d_lo = s11 << 50, d_hi = s11 >> 14;
+            lo += d_lo;
+            hi += d_hi + (lo < d_lo ? 1 : 0);
+            inner3[(bg * 3 + c) * LN + pos0 + lane] = reduce128(hi, lo, *lc);
+        }
+        if (NG < 3) __syncthreads();
+    }
+}
+
 // The single-query kernel with the plaintext rows brought in by bulk asynchronous copies.  With register prefetch a warp
 // has 2 KiB in flight and an SM 32 KiB, short of what the memory latency needs at full bandwidth; here every warp runs its
 // own ring of kMacStages buffers (one (blk, g) pair of its BB rows each, 256 B per row: ONE box of a 2-D tensor map over
@@ -953,6 +1040,26 @@ int launch_encrypt_block_finish(hann_ctx* c, const u64* pt, const u64* as, const
 int launch_mac_ct(hann_ctx* c, const u64* baby, const u64* ctdb, int64_t n_bg, u64* inner3) {
     if (n_bg <= 0) return HANN_OK;
     const long long LN = (long long)c->L * c->N;
+    bool small = c->N >= 32 && c->B <= 64 && c->B >= 4;
+    for (int l = 0; l < c->L; l++) small = small && c->mod[l] < (1ULL << 50);
+    if (small) {
+        const int tiles = (int)(LN / 32);
+        int split = 1;
+        while ((long long)tiles * split < 148 * 8 && split < n_bg) split *= 2;
+        const int per = (int)((n_bg + split - 1) / split);
+        split = (int)((n_bg + per - 1) / per);
+        KProf kp(c, KC_MAC);
+        const dim3 grid(tiles, split);
+        switch (c->B) {
+            case 4: k_mac_ct_stream<4, 1><<<grid, 128, 0, c->stream>>>(baby, ctdb, inner3, c->N, c->L, n_bg, per, c->lt_dev); break;
+            case 8: k_mac_ct_stream<4, 2><<<grid, 128, 0, c->stream>>>(baby, ctdb, inner3, c->N, c->L, n_bg, per, c->lt_dev); break;
+            case 16: k_mac_ct_stream<4, 4><<<grid, 128, 0, c->stream>>>(baby, ctdb, inner3, c->N, c->L, n_bg, per, c->lt_dev); break;
+            case 32: k_mac_ct_stream<4, 8><<<grid, 128, 0, c->stream>>>(baby, ctdb, inner3, c->N, c->L, n_bg, per, c->lt_dev); break;
+            case 64: k_mac_ct_stream<8, 8><<<grid, 256, 0, c->stream>>>(baby, ctdb, inner3, c->N, c->L, n_bg, per, c->lt_dev); break;
+            default: small = false; break;
+        }
+        if (small) return check_launch(c, "mac_ct_stream");
+    }
     int gx = (int)((LN + kThreads - 1) / kThreads), gy = 1;
     while ((long long)gx * gy < 148 * 8 && gy < n_bg) gy *= 2;
     if (gy > n_bg) gy = (int)n_bg;

@@ -108,6 +108,11 @@ int64_t hann_workspace_bytes(const hann_ctx *ctx, int64_t max_blocks);
 /* Block until everything enqueued on the context's stream has finished; reports asynchronous CUDA errors. */
 int hann_sync(hann_ctx *ctx);
 const char *hann_last_error(const hann_ctx *ctx);
+/* Self-test of the failure path of the bulk-copy kernels: launches one warp that waits, for limit_ms (1..1000), on a
+ * completion barrier that nothing completes.  The wait runs out, the kernel raises the context's flag and returns; the
+ * NEXT hann_sync therefore reports HANN_ECUDA ("a kernel gave up a bounded wait") and clears the flag, after which the
+ * context works as before.  waited_ms (optional) receives the device time the warp spent waiting. */
+int hann_selftest_bounded_wait(hann_ctx *ctx, int limit_ms, double *waited_ms);
 /* Enable (1) or disable (0) per-call CUDA-event timing; disabled by default. */
 int hann_set_timing(hann_ctx *ctx, int enable);
 int hann_get_stats(hann_ctx *ctx, hann_stats *out);

@@ -81,6 +81,7 @@ def load_library():
         "hann_keygen_relin_from_samples": (C.c_int, [vp, vp, vp, vp, vp]),
         "hann_encrypt_block": (C.c_int, [vp, vp, vp, vp, vp, vp]),
         "hann_score_level_ctdb": (C.c_int, [vp, vp, vp, i64, vp, vp, sz]),
+        "hann_selftest_bounded_wait": (C.c_int, [vp, C.c_int, vp]),
         "hann_score_level_batch": (C.c_int, [vp, vp, C.c_int, vp, i64, vp, vp, sz]),
         "hann_rotate_sum": (C.c_int, [vp, vp, i64, vp, vp, sz]),
         "hann_keyswitch": (C.c_int, [vp, C.c_int, vp, vp, vp, vp, sz]),
@@ -174,6 +175,12 @@ class Context:
 
     def workspace(self, max_blocks):
         return self.alloc(self.workspace_bytes(max_blocks))
+
+    def selftest_bounded_wait(self, limit_ms):
+        """device milliseconds the self-test warp waited before giving up; the next sync() raises"""
+        w = C.c_double(0.0)
+        self._ck(self.lib.hann_selftest_bounded_wait(self.h, int(limit_ms), C.byref(w)))
+        return w.value
 
     def sync(self):
         self._ck(self.lib.hann_sync(self.h))

@@ -383,6 +383,21 @@ extern "C" int hann_sync(hann_ctx* c) {
     return HANN_OK;
 }
 
+extern "C" int hann_selftest_bounded_wait(hann_ctx* c, int limit_ms, double* waited_ms) {
+    if (!c) return HANN_EINVAL;
+    if (limit_ms < 1 || limit_ms > 1000) return fail(c, HANN_EINVAL, "hann_selftest_bounded_wait: limit must be 1..1000 ms");
+    DeviceGuard dg(c->device);
+    RET(ensure_scratch(c, 256));
+    unsigned long long* w = (unsigned long long*)c->scratch;
+    CK(cudaMemsetAsync(w, 0, 8, c->stream));
+    RET(launch_wait_selftest(c, (unsigned long long)limit_ms * 1000000ULL, w));
+    unsigned long long ns = 0;
+    CK(cudaMemcpyAsync(&ns, w, 8, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    if (waited_ms) *waited_ms = (double)ns * 1e-6;
+    return HANN_OK;
+}
+
 extern "C" const char* hann_last_error(const hann_ctx* c) { return c ? c->err.c_str() : "null context"; }
 
 extern "C" int hann_set_timing(hann_ctx* c, int enable) {

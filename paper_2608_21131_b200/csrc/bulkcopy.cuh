@@ -32,8 +32,8 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
-// bounded: gives up (false) one second after the first unsuccessful probe
-__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity) {
+// bounded: gives up (false) limit_ns (default: one second) after the first unsuccessful probe
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, unsigned long long limit_ns = kWaitLimitNs) {
     unsigned long long t0 = 0;
     for (unsigned it = 0;; it++) {
         unsigned ok;
@@ -46,7 +46,7 @@ __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity) {
         if ((it & 63) == 0) {
             const unsigned long long now = global_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) return false;
+            else if (now - t0 > limit_ns) return false;
         }
     }
 }

@@ -346,6 +346,24 @@ __global__ void __launch_bounds__(256, 3) k_ntt_fwd_b8t(NttArgs A, int groups, i
     }
 }
 
+// Self-test of the bounded wait: one warp waits on an mbarrier that nothing ever completes, for limit_ns; the wait must
+// run out, raise the kernel flag and return -- the error path every bulk-copy kernel takes if a copy never arrives.
+__global__ void k_wait_selftest(int* kflag, unsigned long long limit_ns, unsigned long long* waited_ns) {
+    __shared__ __align__(8) u64 bar;
+    const unsigned b = smem_addr(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    const unsigned long long t0 = global_ns();
+    const bool arrived = mbar_wait(b, 0, limit_ns);
+    if (threadIdx.x == 0) {
+        *waited_ns = global_ns() - t0;
+        if (!arrived) atomicExch(kflag, 1);
+    }
+}
+
 // ---- inverse pass B': spans 1 .. S/2 inside contiguous chunks (mirror of forward pass B) -----------------------
 
 template <int R1, int R2, class AR>
@@ -816,6 +834,11 @@ int launch_ks_lift(hann_ctx* c, u64* src, int64_t src_stride, int64_t nsrc, cons
 
 int launch_ntt_inv_pass_b(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm) {
     return launch_ntt(c, data, npoly, stride, lm, true, true);
+}
+
+int launch_wait_selftest(hann_ctx* c, unsigned long long limit_ns, unsigned long long* waited_ns_dev) {
+    k_wait_selftest<<<1, 32, 0, c->stream>>>(c->kflag, limit_ns, waited_ns_dev);
+    return check_launch(c, "wait_selftest");
 }
 
 int ntt_configure(hann_ctx* c) {

@@ -412,3 +412,21 @@ def test_encrypted_database_level_bit_exact(logN, R, B, L, big, n_rows):
         assert np.array_equal(score_g[blk], o.rotate_sum(inner_o[blk], p.evk_o[ps.B - 1]))
     got = g.decrypt_scores(p.km.s, score_g).reshape(-1)[:n_rows]
     assert np.abs(got - rows.astype(np.float64) @ qv.astype(np.float64)).max() < 2.0 ** ps.tol_log2
+
+
+def test_bounded_wait_runs_out_and_is_reported():
+    """Failure path of the bulk-copy kernels without a fault: a wait that nothing completes gives up after its limit, the
+    next sync reports it, and the context keeps working."""
+    from paper_2608_21131_b200 import binding as b
+
+    ps = synth.small_params(10, 16, 4, L=2)
+    p = Pair(ps, key_seed=2)
+    g = p.g
+    g.sync()
+    waited = g.selftest_bounded_wait(20)
+    assert 20.0 <= waited < 200.0
+    with pytest.raises(b.HannError) as ei:
+        g.sync()
+    assert ei.value.code == b.ECUDA and "bounded wait" in str(ei.value)
+    g.sync()                                    # the flag is cleared
+    run_level(p, synth.toy_corpus(5, rows=900, dim=16), synth.toy_query(6, dim=16))   # and the context still computes

@@ -11,8 +11,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhann.so")
-SOURCES = ["api.cu", "ntt.cu", "keyswitch.cu", "encode.cu", "static_scratch.cu", "hostmath.cpp"]
-HEADERS = ["internal.h", "modarith.cuh", "nttcore.cuh", os.path.join("..", "..", "include", "hann.h")]
+SOURCES = ["api.cu", "ntt.cu", "keyswitch.cu", "mac.cu", "encode.cu", "static_scratch.cu", "hostmath.cpp"]
+HEADERS = ["internal.h", "modarith.cuh", "nttcore.cuh", "bulkcopy.cuh", os.path.join("..", "..", "include", "hann.h")]
 
 
 def stale() -> bool:

@@ -346,6 +346,94 @@ __global__ void __launch_bounds__(256, 3) k_ntt_fwd_b8t(NttArgs A, int groups, i
     }
 }
 
+// Inverse pass B' (spans 1 .. 128 inside chunks, the first pass of an inverse transform) in the same form: bulk copies
+// into per-warp buffers, in-place swizzled exchange, no CTA-wide barrier in the loop.  Input canonical residues in the
+// nibble-swapped layout (word 16 e + j holds logical position 16 j + e), output in the private format of the modulus at
+// natural positions, as the second inverse pass (k_ntt_inv_a, k_ks_lift) expects.
+template <class AR>
+__global__ void __launch_bounds__(256, 3) k_ntt_inv_b8t(NttArgs A, int groups, int* kflag) {
+    extern __shared__ __align__(128) u64 smraw[];
+    typedef typename AR::TW TW;
+    // twiddle cache [kTK][256]: stage s of a round of four uses table entries (base << (3 - s)) + il, il < 2^(3 - s); they
+    // are kept at row r = 16 - (16 >> s) + il.  Entries 0..14: second round (base = m0 + chunk, read by all 16 lanes of a
+    // chunk at once); entries 16 (r + 1) + j: first round of lane j (base = ((m0 + chunk) << 4) + j).
+    TW* tc = (TW*)smraw;
+    u64* bufs = smraw + kTK * 256 * 2;
+    u64* bars = bufs + kTP * 2 * 512;
+    const int k = blockIdx.y;
+    const int pos = (int)((A.pos4 >> (4 * k)) & 15), limb = (int)((A.limb4 >> (4 * k)) & 15);
+    const AR ar(A.lt + limb);
+    const int chunk0 = blockIdx.x * kTK;
+    const TW* tw = (const TW*)A.tw + ((size_t)limb << A.logN);
+    const unsigned m0 = 1u << A.a;
+    const int t = threadIdx.x >> 5, lane = threadIdx.x & 31, ch = lane >> 4, j = lane & 15;
+    const int ntiles = (groups + kTP - 1) / kTP;
+    const long long tile_stride = (long long)kTP * A.period * A.stride;
+    u64* wbuf = bufs + t * 1024;
+    const unsigned bar0 = smem_addr(bars + t * 2), buf0 = smem_addr(wbuf);
+    if (lane == 0) {
+        mbar_init(bar0, 1);
+        mbar_init(bar0 + 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    const int yg0 = blockIdx.z, ystep = gridDim.z;
+    u64* gbase = A.data + (((long long)yg0 * kTP + t) * A.period + pos) * A.stride + ((size_t)chunk0 << 8);
+    const int my_tiles = yg0 < ntiles ? (ntiles - yg0 + ystep - 1) / ystep : 0;
+    auto tile_valid = [&](int i) { return i < my_tiles && (long long)(yg0 + (long long)i * ystep) * kTP + t < groups; };
+    if (lane == 0) {
+        for (int i = 0; i < 2; i++)
+            if (tile_valid(i)) {
+                mbar_expect_tx(bar0 + 8 * i, 4096);
+                bulk_load(buf0 + 4096 * i, gbase + (long long)i * ystep * tile_stride, 4096, bar0 + 8 * i);
+            }
+    }
+    for (int i = threadIdx.x; i < kTK * 256; i += 256) {
+        const int c2 = i >> 8, e = i & 255;
+        const unsigned cbase = m0 + (unsigned)(chunk0 + c2);
+        const int r = e < 16 ? e : (e >> 4) - 1;  // row 0..14 (e == 15 and rows above 14 are unused)
+        if (r < 15 && (e < 15 || e >= 16)) {
+            int st = 0;
+            while (16 - (16 >> (st + 1)) <= r) st++;
+            const int il = r - (16 - (16 >> st));
+            const unsigned base = e < 16 ? cbase : (cbase << 4) + (unsigned)(e & 15);
+            tc[i] = tw[(base << (3 - st)) + il];
+        }
+    }
+    __syncthreads();
+    const TW* tcc = tc + ch * 256;
+    for (int i = 0; i < my_tiles; i++) {
+        if (!tile_valid(i)) break;  // warp-uniform
+        const int s = i & 1;
+        if (!mbar_wait(bar0 + 8 * s, (unsigned)(i >> 1) & 1u)) {
+            if (lane == 0) atomicExch(kflag, 1);
+            if (tile_valid(i + 1)) mbar_wait(bar0 + 8 * (s ^ 1), (unsigned)((i + 1) >> 1) & 1u);
+            return;
+        }
+        u64* sb = wbuf + s * 512 + ch * 256;
+        typename AR::T x[16];
+#pragma unroll
+        for (int e = 0; e < 16; e++) x[e] = ar.inv_input(sb[16 * e + j]);  // logical positions 16 j + e
+        __syncwarp();
+        inv_round_f<4>(ar, x, [=](int st, int il) { return tcc[((16 - (16 >> st) + il + 1) << 4) + j]; });
+#pragma unroll
+        for (int e = 0; e < 16; e++) sb[16 * j + (e ^ j)] = ar.to_mid(x[e]);
+        __syncwarp();
+#pragma unroll
+        for (int e = 0; e < 16; e++) x[e] = ar.from_mid(sb[16 * e + (j ^ e)]);  // logical positions j + 16 e
+        inv_round_f<4>(ar, x, [=](int st, int il) { return tcc[16 - (16 >> st) + il]; });
+        u64* go = gbase + (long long)i * ystep * tile_stride + ((size_t)ch << 8);
+#pragma unroll
+        for (int e = 0; e < 16; e++) go[j + 16 * e] = ar.to_mid(x[e]);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0 && tile_valid(i + 2)) {
+            mbar_expect_tx(bar0 + 8 * s, 4096);
+            bulk_load(buf0 + 4096 * s, gbase + (long long)(i + 2) * ystep * tile_stride, 4096, bar0 + 8 * s);
+        }
+    }
+}
+
 // Self-test of the bounded wait: one warp waits on an mbarrier that nothing ever completes, for limit_ns; the wait must
 // run out, raise the kernel flag and return -- the error path every bulk-copy kernel takes if a copy never arrives.
 __global__ void k_wait_selftest(int* kflag, unsigned long long limit_ns, unsigned long long* waited_ns) {
@@ -694,7 +782,24 @@ void launch_fwd_class(hann_ctx* c, const NttArgs& A, int groups, bool skip_a) {
 
 template <class AR>
 void launch_inv_class(hann_ctx* c, const NttArgs& A, int groups, bool skip_a) {
-    {
+    if (A.b == 8 && A.a > 0 && A.tau && ((c->N >> 8) % kTK) == 0 && ((uintptr_t)A.data & 15) == 0 && (A.stride & 1) == 0) {
+        KProf kp(c, KC_NTT_INV_B);
+        const size_t smem = (size_t)kTK * 256 * 16 + (size_t)kTP * 2 * 512 * 8 + (size_t)kTP * 2 * 8;
+        cudaFuncSetAttribute(k_ntt_inv_b8t<AR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        const int ranges = (c->N >> 8) / kTK, ntiles = (groups + kTP - 1) / kTP;
+        const int slots = 148 * 3, per = ranges * A.nsel;
+        int zs = 1;
+        long best = -1;
+        for (int z = 1; z <= ntiles && z <= 64; z++) {
+            const long waves = ((long)per * z + slots - 1) / slots, tiles = (ntiles + z - 1) / z;
+            const long cost = waves * (4 * tiles + 1);
+            if (best < 0 || cost < best) {
+                best = cost;
+                zs = z;
+            }
+        }
+        k_ntt_inv_b8t<AR><<<dim3(ranges, A.nsel, zs), 256, smem, c->stream>>>(A, groups, c->kflag);
+    } else {
         KProf kp(c, KC_NTT_INV_B);
         pick_inv_b<AR>(A.b)<<<dim3((c->N >> A.b) / A.K, groups * A.nsel), kThreads, smem_b(A), c->stream>>>(A, A.a == 0 ? 1 : 0);
     }

@@ -162,20 +162,32 @@ __device__ __forceinline__ void fwd_round_f(const AR& ar, typename AR::T (&x)[1 
     }
 }
 
+// (flat butterfly index t = il * span + jj: with the nested (il, jj) loops of the forward round the compiler left x[] in
+// local memory)
 template <int R, class AR>
 __device__ __forceinline__ void inv_round(const AR& ar, typename AR::T (&x)[1 << R], const typename AR::TW* __restrict__ tw,
                                           unsigned base) {
 #pragma unroll
     for (int s = 0; s < R; s++) {
-        const int span = 1 << s;
 #pragma unroll
-        for (int il = 0; il < (1 << (R - 1 - s)); il++) {
-            const typename AR::TW w = tw[(base << (R - 1 - s)) + il];
+        for (int t = 0; t < (1 << (R - 1)); t++) {
+            const int il = t >> s, jj = t & ((1 << s) - 1);
+            const int e = (il << (s + 1)) + jj;
+            ar.inv(x[e], x[e + (1 << s)], tw[(base << (R - 1 - s)) + il]);
+        }
+    }
+}
+
+// the inverse round with the twiddle of (stage s, group il) supplied by a functor
+template <int R, class AR, class TWF>
+__device__ __forceinline__ void inv_round_f(const AR& ar, typename AR::T (&x)[1 << R], const TWF& twf) {
 #pragma unroll
-            for (int jj = 0; jj < span; jj++) {
-                const int e = il * 2 * span + jj;
-                ar.inv(x[e], x[e + span], w);
-            }
+    for (int s = 0; s < R; s++) {
+#pragma unroll
+        for (int t = 0; t < (1 << (R - 1)); t++) {
+            const int il = t >> s, jj = t & ((1 << s) - 1);
+            const int e = (il << (s + 1)) + jj;
+            ar.inv(x[e], x[e + (1 << s)], twf(s, il));
         }
     }
 }

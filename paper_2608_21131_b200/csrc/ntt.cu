@@ -657,7 +657,9 @@ __global__ void __launch_bounds__(256, 2) k_ks_lift(LiftArgs A) {
         lift_inverse<R1, R2>(A, ar, (const ulonglong2*)A.tw_inv_int + ((size_t)sl << A.logN), sbase, sm, g, c, active, v);
     }
     if (R2 != 0) __syncthreads();  // every thread is done with the exchange tile of the inverse rounds
-    for (int ti = 0; ti < A.n_tgt; ti++) {
+    // a launch too small to fill the machine is cut along the targets as well: gridDim.z CTAs repeat the inverse rounds and
+    // share out the targets, which shortens the chain one CTA runs
+    for (int ti = blockIdx.z; ti < A.n_tgt; ti += gridDim.z) {
         const int tl = A.tgt_limb0 + ti;
         const LimbConst* tlc = A.lt + tl;
         u64* dbase = A.dst + (sp * A.n_tgt + ti) * (long long)N + c0;
@@ -674,6 +676,8 @@ __global__ void __launch_bounds__(256, 2) k_ks_lift(LiftArgs A) {
     }
 }
 
+// launches of at most this many CTAs (a one-block level on one lane) are cut along their targets, see k_ks_lift
+constexpr long kLiftSplitCtas = 160;
 typedef void (*KernLift)(LiftArgs);
 KernLift pick_lift(int a) {
     switch (a) {
@@ -932,7 +936,8 @@ int launch_ks_lift(hann_ctx* c, u64* src, int64_t src_stride, int64_t nsrc, cons
         Ap.src_limb4 = 0;
         for (int i = 0; i < src_lm.period && i < 16; i++) Ap.src_limb4 |= (u64)src_lm.limb[(s0 + i) % src_lm.period] << (4 * i);
         KProf kp(c, KC_LIFT_DIGITS);
-        pick_lift(a)<<<dim3(16, ns), threads, smem, c->stream>>>(Ap);
+        const int zsplit = (16L * ns * n_tgt <= kLiftSplitCtas) ? n_tgt : 1;
+        pick_lift(a)<<<dim3(16, ns, zsplit), threads, smem, c->stream>>>(Ap);
     }
     return check_launch(c, "ks_lift");
 }

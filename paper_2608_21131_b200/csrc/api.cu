@@ -978,7 +978,13 @@ extern "C" int hann_rotate_sum(hann_ctx* c, const void* inner_dev, int64_t n_blo
     int lanes = (int)std::min<int64_t>(4, n_blocks);
     if (c->stream == c->aux_stream || c->kprof) lanes = 1;
     while (lanes > 1 && (((int64_t)ws_bytes / lanes) & ~(int64_t)255) < ks_item_words(c) * 8 + kSlack) lanes--;
-    if (lanes <= 1) return run_range(0, n_blocks, (char*)ws, (int64_t)ws_bytes);
+    if (lanes <= 1) {
+        const int saved = c->lift_split_ctas;
+        if (n_blocks <= 2) c->lift_split_ctas = 320;
+        const int r = run_range(0, n_blocks, (char*)ws, (int64_t)ws_bytes);
+        c->lift_split_ctas = saved;
+        return r;
+    }
     const int64_t part = ((int64_t)ws_bytes / lanes) & ~(int64_t)255;
     cudaStream_t main_stream = c->stream;
     cudaStream_t helper[3] = {c->aux_stream, c->lane_stream[0], c->lane_stream[1]};

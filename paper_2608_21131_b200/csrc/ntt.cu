@@ -676,8 +676,6 @@ __global__ void __launch_bounds__(256, 2) k_ks_lift(LiftArgs A) {
     }
 }
 
-// launches of at most this many CTAs (a one-block level on one lane) are cut along their targets, see k_ks_lift
-constexpr long kLiftSplitCtas = 160;
 typedef void (*KernLift)(LiftArgs);
 KernLift pick_lift(int a) {
     switch (a) {
@@ -936,7 +934,7 @@ int launch_ks_lift(hann_ctx* c, u64* src, int64_t src_stride, int64_t nsrc, cons
         Ap.src_limb4 = 0;
         for (int i = 0; i < src_lm.period && i < 16; i++) Ap.src_limb4 |= (u64)src_lm.limb[(s0 + i) % src_lm.period] << (4 * i);
         KProf kp(c, KC_LIFT_DIGITS);
-        const int zsplit = (16L * ns * n_tgt <= kLiftSplitCtas) ? n_tgt : 1;
+        const int zsplit = (16L * ns * n_tgt <= c->lift_split_ctas) ? n_tgt : 1;  // see hann_ctx::lift_split_ctas
         pick_lift(a)<<<dim3(16, ns, zsplit), threads, smem, c->stream>>>(Ap);
     }
     return check_launch(c, "ks_lift");

@@ -352,6 +352,25 @@ void orc_encrypt(const orc_ctx *c, const int8_t *s, const i64 *m, const u64 *a, 
     free(sq); free(t);
 }
 
+/* Seed-compressed ciphertexts (Sec. 7: the public-random half of a fresh ciphertext is regenerated from a short seed).
+ * The uniform polynomial a is a pure function of (seed, stream): a[l][x] = h(seed, stream, l*N + x) mod q_l with the
+ * 64-bit counter hash  mix(x): x ^= x>>32; x *= 0x9E3779B97F4A7C15; x ^= x>>29; x *= 0xBB67AE8584CAA73B; x ^= x>>32;
+ * h = mix(mix(mix(seed + 0x9E3779B97F4A7C15) ^ (stream * 0xBB67AE8584CAA73B)) + ctr * 0x9E3779B97F4A7C15). */
+static u64 mix64(u64 x) {
+    x ^= x >> 32; x *= 0x9E3779B97F4A7C15ULL; x ^= x >> 29; x *= 0xBB67AE8584CAA73BULL; x ^= x >> 32;
+    return x;
+}
+u64 orc_hash64(u64 seed, u64 stream, u64 ctr) {
+    u64 a = mix64(seed + 0x9E3779B97F4A7C15ULL);
+    u64 b = mix64(a ^ (stream * 0xBB67AE8584CAA73BULL));
+    return mix64(b + ctr * 0x9E3779B97F4A7C15ULL);
+}
+void orc_expand_uniform(const orc_ctx *c, u64 seed, u64 stream, u64 *a) {
+    int N = c->N, L = c->L;
+    for (int l = 0; l < L; l++)
+        for (int x = 0; x < N; x++) a[(size_t)l * N + x] = orc_hash64(seed, stream, (u64)l * N + x) % c->mod[l];
+}
+
 /* mu = c0 + c1*s, residues [L][N]; the caller reconstructs centred integers by CRT */
 void orc_decrypt_residues(const orc_ctx *c, const int8_t *s, const u64 *ct, u64 *mu) {
     int N = c->N, L = c->L;

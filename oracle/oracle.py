@@ -57,6 +57,8 @@ def lib():
         _lib.orc_automorphism.argtypes = [C.c_void_p, C.c_int, C.c_long, u64p, u64p]
         _lib.orc_automorphism_ntt.argtypes = [C.c_void_p, C.c_long, u64p, u64p]
         _lib.orc_decode.argtypes = [C.c_void_p, f64p, C.c_double, f64p, f64p]
+        _lib.orc_hash64.restype = C.c_uint64
+        _lib.orc_hash64.argtypes = [C.c_uint64, C.c_uint64, C.c_uint64]
     return _lib
 
 
@@ -203,6 +205,12 @@ class Oracle:
         qv[: len(qvec)] = np.asarray(qvec, dtype=np.float32)
         z = np.tile(qv.astype(np.float64), self.n // self.R)
         return self.encrypt(s, self.encode(z), a, e)
+
+    def expand_uniform(self, seed, stream):
+        """the uniform half a [L][N] of a seed-compressed ciphertext"""
+        a = np.zeros((self.L, self.N), dtype=np.uint64)
+        lib().orc_expand_uniform(self.h, C.c_uint64(seed), C.c_uint64(stream), _p(a, u64p))
+        return a
 
     def decrypt_residues(self, s, ct):
         s = np.ascontiguousarray(s, dtype=np.int8)

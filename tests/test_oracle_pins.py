@@ -588,3 +588,23 @@ def test_encrypted_database_scores_within_tolerance():
             # of ModDown, which differ -> compare decrypted integers up to those roundings
             a_int, b_int = o.decrypt_int(km.s, score), o.decrypt_int(km.s, plain)
             assert max(abs(int(x) - int(y)) for x, y in zip(a_int, b_int)) < 64 * ps.N
+
+
+# ------------------------------------------------------------------ seed-compressed ciphertexts
+
+
+def test_seed_expansion_matches_the_published_check_values():
+    """the counter hash against its four check values h(1, 0, 0..3) and, through them, against the harness generator;
+    the expanded polynomial is the harness's uniform residue array"""
+    from oracle.oracle import lib
+
+    want = [0xCE6D52A9E69DA903, 0x3C904E4F0D0C01AF, 0x6E6AE58702F2C840, 0xD254BD0790389C63]
+    assert [int(lib().orc_hash64(1, 0, i)) for i in range(4)] == want
+    assert [int(v) for v in synth.hash64(1, 0, np.arange(4))] == want
+    ps = synth.small_params(8, 8, 4, L=2)
+    o = make(ps)
+    a = o.expand_uniform(123456789, 19)
+    assert np.array_equal(a, synth.uniform_residues(123456789, 19, list(ps.q), ps.N))
+    assert all(int(a[l].max()) < ps.q[l] for l in range(ps.L))
+    # roughly uniform: mean near q/2
+    assert abs(float(a[0].astype(np.float64).mean()) / ps.q[0] - 0.5) < 0.1

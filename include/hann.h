@@ -256,6 +256,16 @@ int hann_keyswitch_static(hann_ctx *ctx, int rot, const void *poly_dev, void *ks
  * kind POLY / PT: one polynomial of L limbs per element; CT: two. */
 int hann_import(hann_ctx *ctx, int kind, const uint64_t *canonical, int64_t count, void *internal_dev);
 int hann_export(hann_ctx *ctx, int kind, const void *internal_dev, int64_t count, uint64_t *canonical_out);
+
+/* Seed-compressed fresh ciphertexts (Sec. 7: the public-random half is regenerated from a short seed).  The uniform
+ * polynomial is a pure function of (seed, stream): a[l][x] = h(seed, stream, l*N + x) mod q_l with the 64-bit counter
+ * hash h = mix(mix(mix(seed + M1) ^ (stream * M2)) + ctr * M1), mix(x): x ^= x >> 32; x *= M1; x ^= x >> 29; x *= M2;
+ * x ^= x >> 32, M1 = 0x9E3779B97F4A7C15, M2 = 0xBB67AE8584CAA73B (a benchmark generator, not a cryptographic one).
+ * hann_expand_uniform writes a [L][N] (canonical; host or device pointer) -- the client passes it to hann_encrypt_query
+ * and uploads only c0 and the seed; hann_import_seeded_ct builds the internal ciphertext (HANN_SIZE_CT bytes, device)
+ * from c0 [L][N] (canonical, host or device) and the seed, enqueued on the context's stream. */
+int hann_expand_uniform(hann_ctx *ctx, uint64_t seed, uint64_t stream, uint64_t *a_out);
+int hann_import_seeded_ct(hann_ctx *ctx, const uint64_t *c0, uint64_t seed, uint64_t stream, void *ct_dev);
 /* The same for npoly polynomials stored with `limbs` limbs each (compacted ciphertexts): internal [npoly][limbs][N] ->
  * canonical [npoly][limbs][N]. */
 int hann_export_limbs(hann_ctx *ctx, const void *internal_dev, int64_t npoly, int limbs, uint64_t *canonical_out);

@@ -90,6 +90,8 @@ def load_library():
         "hann_keyswitch_static": (C.c_int, [vp, C.c_int, vp, vp, vp]),
         "hann_import": (C.c_int, [vp, C.c_int, vp, i64, vp]),
         "hann_export": (C.c_int, [vp, C.c_int, vp, i64, vp]),
+        "hann_expand_uniform": (C.c_int, [vp, C.c_uint64, C.c_uint64, vp]),
+        "hann_import_seeded_ct": (C.c_int, [vp, vp, C.c_uint64, C.c_uint64, vp]),
         "hann_export_limbs": (C.c_int, [vp, vp, i64, C.c_int, vp]),
         "hann_compact_bytes": (i64, [vp, i64, C.c_int]),
         "hann_compact_scores": (C.c_int, [vp, vp, i64, C.c_int, C.c_int, vp, vp, sz]),
@@ -281,6 +283,19 @@ class Context:
         polys = 2 if kind == KIND_CT else 1
         out = np.empty((count, polys, self.L, self.N), dtype=np.uint64)
         self._ck(self.lib.hann_export(self.h, kind, _ptr(internal) + offset_bytes, count, _ptr(out)))
+        return out
+
+    def expand_uniform(self, seed, stream):
+        a = np.empty((self.L, self.N), dtype=np.uint64)
+        self._ck(self.lib.hann_expand_uniform(self.h, seed, stream, _ptr(a)))
+        return a
+
+    def import_seeded_ct(self, c0, seed, stream, out=None):
+        """c0 [L][N] canonical + the seed of the uniform half -> internal ciphertext on the device"""
+        c0 = _np(c0, np.uint64)
+        if out is None:
+            out = self.alloc(self.sizeof(SIZE_CT))
+        self._ck(self.lib.hann_import_seeded_ct(self.h, _ptr(c0), seed, stream, _ptr(out)))
         return out
 
     def export_limbs(self, internal, npoly, limbs):

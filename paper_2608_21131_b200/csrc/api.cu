@@ -475,6 +475,29 @@ extern "C" int hann_import(hann_ctx* c, int kind, const uint64_t* canonical, int
     return HANN_OK;
 }
 
+extern "C" int hann_expand_uniform(hann_ctx* c, uint64_t seed, uint64_t stream, uint64_t* a_out) {
+    if (!c) return HANN_EINVAL;
+    if (!a_out) return fail(c, HANN_EINVAL, "hann_expand_uniform: null pointer");
+    DeviceGuard dg(c->device);
+    const int64_t LN = (int64_t)c->L * c->N;
+    RET(ensure_scratch(c, LN * 8));
+    RET(launch_expand_uniform(c, seed, stream, (u64*)c->scratch));
+    CK(cudaMemcpyAsync(a_out, c->scratch, LN * 8, cudaMemcpyDefault, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return HANN_OK;
+}
+
+extern "C" int hann_import_seeded_ct(hann_ctx* c, const uint64_t* c0, uint64_t seed, uint64_t stream, void* ct_dev) {
+    if (!c) return HANN_EINVAL;
+    if (!c0 || !ct_dev) return fail(c, HANN_EINVAL, "hann_import_seeded_ct: null pointer");
+    DeviceGuard dg(c->device);
+    const int64_t LN = (int64_t)c->L * c->N;
+    u64* ct = (u64*)ct_dev;
+    CK(cudaMemcpyAsync(ct, c0, LN * 8, cudaMemcpyDefault, c->stream));
+    RET(launch_expand_uniform(c, seed, stream, ct + LN));
+    return launch_ntt_fwd(c, ct, 2 * c->L, c->N, limbmap_q(c));
+}
+
 extern "C" int hann_export(hann_ctx* c, int kind, const void* internal_dev, int64_t count, uint64_t* canonical_out) {
     if (!c) return HANN_EINVAL;
     const int pk = polys_of_kind(kind);

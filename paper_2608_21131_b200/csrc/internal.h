@@ -158,6 +158,8 @@ int launch_mul(hann_ctx* c, const u64* a, const u64* b, int bperiod, u64* out, i
 int launch_add(hann_ctx* c, const u64* a, const u64* b, u64* out, int64_t npoly, const LimbMap& lm);
 int launch_evk_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const int8_t* sprime, u64* b_out);
 int launch_encrypt_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const u64* m, u64* c0_out);
+// a[L][N] = counter hash of (seed, stream, l*N + x) mod q_l (coefficient domain, canonical)
+int launch_expand_uniform(hann_ctx* c, u64 seed, u64 stream, u64* a);
 // encrypted database: relinearisation key finish, block encryption finish, ct x ct multiply-accumulate
 int launch_rlk_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const u64* s2, u64* b_out);
 int launch_encrypt_block_finish(hann_ctx* c, const u64* pt, const u64* as, const u64* ehat, u64* ct, int64_t npt);

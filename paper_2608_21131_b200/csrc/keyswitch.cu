@@ -362,6 +362,23 @@ __global__ void __launch_bounds__(kThreads) k_encrypt_block_finish(const u64* __
     }
 }
 
+// the uniform half of a seed-compressed ciphertext: a[l][x] = h(seed, stream, l*N + x) mod q_l, h the 64-bit counter hash
+// mix(mix(mix(seed + M1) ^ (stream * M2)) + ctr * M1), mix(x): x ^= x >> 32; x *= M1; x ^= x >> 29; x *= M2; x ^= x >> 32
+__device__ __forceinline__ u64 mix64(u64 x) {
+    x ^= x >> 32;
+    x *= 0x9E3779B97F4A7C15ULL;
+    x ^= x >> 29;
+    x *= 0xBB67AE8584CAA73BULL;
+    x ^= x >> 32;
+    return x;
+}
+__global__ void __launch_bounds__(kThreads) k_expand_uniform(u64* __restrict__ a, u64 seed, u64 stream, int N, int L, LimbTable lt) {
+    const long long total = (long long)L * N;
+    const u64 b = mix64(mix64(seed + 0x9E3779B97F4A7C15ULL) ^ (stream * 0xBB67AE8584CAA73BULL));
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads)
+        a[idx] = barrett64(mix64(b + (u64)idx * 0x9E3779B97F4A7C15ULL), lt.c[(int)(idx / N)]);
+}
+
 // symmetric encryption finish, coefficient domain: c0[l][x] = -as[l][x] + e[x] + m[l][x]
 __global__ void __launch_bounds__(kThreads) k_encrypt_finish(const u64* __restrict__ as, const int8_t* __restrict__ e,
                                                              const u64* __restrict__ m, u64* __restrict__ c0, int N, int L,
@@ -575,6 +592,14 @@ int launch_encrypt_block_finish(hann_ctx* c, const u64* pt, const u64* as, const
         k_encrypt_block_finish<<<grid_for(npt * c->L * c->N), kThreads, 0, c->stream>>>(pt, as, ehat, ct, c->N, c->L, npt, c->lt);
     }
     return check_launch(c, "encrypt_block_finish");
+}
+
+int launch_expand_uniform(hann_ctx* c, u64 seed, u64 stream, u64* a) {
+    {
+        KProf kp(c, KC_OTHER);
+        k_expand_uniform<<<grid_for((int64_t)c->L * c->N), kThreads, 0, c->stream>>>(a, seed, stream, c->N, c->L, c->lt);
+    }
+    return check_launch(c, "expand_uniform");
 }
 
 int launch_encrypt_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const u64* m, u64* c0_out) {

@@ -430,3 +430,25 @@ def test_bounded_wait_runs_out_and_is_reported():
     assert ei.value.code == b.ECUDA and "bounded wait" in str(ei.value)
     g.sync()                                    # the flag is cleared
     run_level(p, synth.toy_corpus(5, rows=900, dim=16), synth.toy_query(6, dim=16))   # and the context still computes
+
+
+@pytest.mark.parametrize("logN,big", [(8, False), (12, False), (13, True)])
+def test_seed_compressed_query_upload(logN, big):
+    """the query uploaded as (c0, seed): the expanded uniform half equals the oracle's, and the imported ciphertext is the
+    one a full upload gives"""
+    import torch
+
+    ps = synth.ParamSet("seed", logN, synth.Q50, synth.P60, 40, 16, 4, -18) if big else synth.small_params(logN, 16, 4, L=2)
+    p = Pair(ps, key_seed=logN)
+    g, o, b = p.g, p.o, p.b
+    seed, stream = 0xC0FFEE + logN, 23
+    a = g.expand_uniform(seed, stream)
+    assert np.array_equal(a, o.expand_uniform(seed, stream))
+    qv = synth.toy_query(logN, dim=16)
+    ct_o = o.encrypt_query(p.km.s, qv, a, p.km.ct_e)
+    ct_g = g.encrypt_query(p.km.s, qv, a, p.km.ct_e)
+    assert np.array_equal(ct_g, ct_o) and np.array_equal(ct_g[1], a)
+    full = g.import_(b.KIND_CT, ct_g, 1)
+    seeded = g.import_seeded_ct(ct_g[0], seed, stream)   # half the bytes on the wire
+    g.sync()
+    assert torch.equal(full[: seeded.numel()], seeded)

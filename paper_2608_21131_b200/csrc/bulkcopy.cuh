@@ -1,5 +1,5 @@
 // Bulk asynchronous global -> shared copies with mbarrier completion (the asynchronous copy path of sm_90 and later),
-// as used by the transform's pass B and by the multiply-accumulate.  No cluster multicast anywhere: every copy lands in the
+// as used by the transform's pass B and by the multiply-accumulate.  Every copy is private to one CTA: it lands in the
 // issuing CTA's own shared memory.  Every wait is bounded in wall-clock time.
 #pragma once
 #include <cstdint>

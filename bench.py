@@ -342,6 +342,29 @@ def run_ours(args):
     e2e_same = bool(np.array_equal(out_pin.numpy().view(np.uint64), score_host))
     e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(rows_np.nbytes + ct_host.nbytes),
            "d2h_bytes_per_step": int(out_pin.numel() * 8), "steps": e2e_steps, "matches_device_path": e2e_same}
+    # the same call downloading only the first two limbs of the score ciphertexts (exact compaction; the client decrypts
+    # the same scores from half the bytes)
+    if ps.L > 2:
+        ctx.set_tuning(binding.TUNE_HOST_LIMBS, 2)
+        out2_pin = torch.empty((nb, 2, 2, ctx.N), dtype=torch.int64).pin_memory()
+
+        def e2e2_step():
+            ctx.lib.hann_score_level_host(ctx.h, ct_pin.data_ptr(), rows_pin.data_ptr(), n_rows, rows_np.shape[1], out2_pin.data_ptr(),
+                                          ws_host.data_ptr(), ws_host.numel() * 8)
+
+        for _ in range(3):
+            e2e2_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            e2e2_step()
+        torch.cuda.synchronize()
+        t2 = max_over_ranks(time.perf_counter() - t0, dist, ctx.device)
+        ctx.set_tuning(binding.TUNE_HOST_LIMBS, ps.L)
+        got2 = ctx.decrypt_compact(km.s, out2_pin.numpy().view(np.uint64), False).reshape(-1)[:n_rows]
+        e2e["two_limb_download"] = {"value": replica_throughput(n_rows * e2e_steps, world, t2), "unit": UNIT,
+                                    "d2h_bytes_per_step": int(out2_pin.numel() * 8),
+                                    "scores_identical_to_full_download": bool(np.array_equal(got2, got))}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:

@@ -118,8 +118,11 @@ int hann_set_timing(hann_ctx *ctx, int enable);
 int hann_get_stats(hann_ctx *ctx, hann_stats *out);
 
 /* Performance knobs (results never depend on them).  HANN_TUNE_ENCODE_GROUP: plaintexts encoded and transformed per
- * launch group in hann_encode_candidates (default: all R plaintexts of a block at once); ask hann_workspace_bytes again after changing it. */
-enum { HANN_TUNE_ENCODE_GROUP = 1 };
+ * launch group in hann_encode_candidates (default: all R plaintexts of a block at once); ask hann_workspace_bytes again after changing it.
+ * HANN_TUNE_HOST_LIMBS (this one DOES change a result's layout): hann_score_level_host downloads only the first `value`
+ * limbs of every score polynomial, score_ct_host [blocks][2][value][N] -- the exact form of hann_compact_scores; decrypt
+ * with hann_decrypt_compact(limbs = value, rescaled = 0).  Default L. */
+enum { HANN_TUNE_ENCODE_GROUP = 1, HANN_TUNE_HOST_LIMBS = 2 };
 int hann_set_tuning(hann_ctx *ctx, int what, int value);
 
 /* Per-launch profile: while enabled every kernel launch of the context is bracketed by a CUDA event pair (this
@@ -292,7 +295,8 @@ int hann_compact_scores(hann_ctx *ctx, const void *score_ct_dev, int64_t n_block
  * the host in canonical layout.  Page-locked host buffers are needed for the copies to overlap the kernels (pageable
  * memory works but serialises).  Device buffers for the intermediates are carved from `ws_dev`, which must hold
  * hann_level_host_bytes(ctx, n_rows) bytes.  Returns after everything has finished.
- *   ct_host [2][L][N];  rows_host [n_rows][dim] float32;  score_ct_host [ceil(n_rows/n)][2][L][N]. */
+ *   ct_host [2][L][N];  rows_host [n_rows][dim] float32;  score_ct_host [ceil(n_rows/n)][2][L][N] (fewer limbs with
+ *   HANN_TUNE_HOST_LIMBS). */
 int64_t hann_level_host_bytes(const hann_ctx *ctx, int64_t n_rows);
 int hann_score_level_host(hann_ctx *ctx, const uint64_t *ct_host, const float *rows_host, int64_t n_rows, int dim,
                           uint64_t *score_ct_host, void *ws_dev, size_t ws_bytes);

@@ -20,6 +20,7 @@ OK, EINVAL, ESHAPE, ENOKEY, EWORKSPACE, ECUDA, ENOMEM = 0, -1, -2, -3, -4, -5, -
 SIZE_POLY, SIZE_CT, SIZE_BABY, SIZE_PT_BLOCK, SIZE_INNER, SIZE_EVK, SIZE_ROWS_PER_BLOCK, SIZE_CTDB_BLOCK = 1, 2, 3, 4, 5, 6, 7, 8
 KIND_POLY, KIND_CT, KIND_PT = 1, 2, 3
 TUNE_ENCODE_GROUP = 1
+TUNE_HOST_LIMBS = 2
 
 
 class HannError(RuntimeError):

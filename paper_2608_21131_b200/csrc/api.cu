@@ -191,6 +191,7 @@ extern "C" int hann_ctx_create(const hann_params* prm, hann_ctx** out) {
     c->prm = *prm;
     c->logN = prm->logN; c->N = N; c->n = n; c->L = L; c->R = prm->R; c->B = prm->B; c->G = prm->R / prm->B;
     c->ntt_tau = prm->logN >= 10 ? 1 : 0;
+    c->host_limbs = L;
     c->device = prm->device;
     c->stream = (cudaStream_t)prm->stream;
     DeviceGuard dg(c->device);
@@ -412,6 +413,10 @@ extern "C" int hann_set_tuning(hann_ctx* c, int what, int value) {
         case HANN_TUNE_ENCODE_GROUP:
             if (value < 1) return fail(c, HANN_EINVAL, "hann_set_tuning: encode group must be positive");
             c->encode_group = value;
+            return HANN_OK;
+        case HANN_TUNE_HOST_LIMBS:
+            if (value < 1 || value > c->L) return fail(c, HANN_EINVAL, "hann_set_tuning: host limbs must be in 1..L");
+            c->host_limbs = value;
             return HANN_OK;
         default: return fail(c, HANN_EINVAL, "hann_set_tuning: unknown knob");
     }
@@ -1175,7 +1180,18 @@ extern "C" int hann_score_level_host(hann_ctx* c, const uint64_t* ct_host, const
     CK(ew2);
     RET(hann_score_level(c, baby, pt, p.nblk, inner, ws, (size_t)p.ws));
     RET(hann_rotate_sum(c, inner, p.nblk, score, ws, (size_t)p.ws));
-    RET(export_polys(c, score, p.nblk * 2, stage, score_ct_host));
+    if (c->host_limbs >= c->L) {
+        RET(export_polys(c, score, p.nblk * 2, stage, score_ct_host));
+    } else {
+        // download only the first host_limbs limbs of every polynomial (exact compaction, see hann_compact_scores): the
+        // inverse transforms and the copy shrink with them
+        const int keep = c->host_limbs;
+        const int64_t npoly = p.nblk * 2, kw = (int64_t)keep * c->N;
+        CK(cudaMemcpy2DAsync(stage, (size_t)kw * 8, score, (size_t)c->L * c->N * 8, (size_t)kw * 8, (size_t)npoly, cudaMemcpyDeviceToDevice,
+                             c->stream));
+        RET(launch_ntt_inv(c, stage, npoly * keep, c->N, limbmap_first(keep)));
+        CK(cudaMemcpyAsync(score_ct_host, stage, (size_t)(npoly * kw) * 8, cudaMemcpyDeviceToHost, c->stream));
+    }
     CK(cudaStreamSynchronize(c->stream));
     return HANN_OK;
 }

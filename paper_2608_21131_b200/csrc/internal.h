@@ -55,6 +55,7 @@ struct hann_ctx {
     int64_t scratch_bytes = 0;
     // plaintexts encoded and transformed per launch group: small enough that the group's intermediates stay in L2
     int encode_group = 1 << 20;
+    int host_limbs = 0;  // limbs of every score polynomial that hann_score_level_host downloads (L: all)
     // key-switch lift launches of at most this many CTAs (after the split) are cut along their targets: 160 keeps it to the
     // ModDown lifts of a single item; hann_rotate_sum raises it to 320 for levels of one or two blocks, whose launches
     // otherwise leave most of the machine idle

@@ -147,6 +147,13 @@ def test_host_buffer_level_matches_device_path(n_rows):
     ws = p.g.alloc(p.g.level_host_bytes(rows.shape[0]))
     out = p.g.score_level_host(ct_g, rows, ws)
     assert np.array_equal(out, score_dev)
+    # downloading only the first limb (the toy set has two): the same first limbs, in the layout of the exact compaction
+    p.g.set_tuning(p.b.TUNE_HOST_LIMBS, 1)
+    nb = out.shape[0]
+    small = np.empty((nb, 2, 1, ps.N), dtype=np.uint64)
+    p.g.score_level_host(ct_g, rows, ws, small)
+    p.g.set_tuning(p.b.TUNE_HOST_LIMBS, ps.L)
+    assert np.array_equal(small, out[:, :, :1])
 
 
 def test_full_ring_one_block():

@@ -459,3 +459,18 @@ def test_seed_compressed_query_upload(logN, big):
     seeded = g.import_seeded_ct(ct_g[0], seed, stream)   # half the bytes on the wire
     g.sync()
     assert torch.equal(full[: seeded.numel()], seeded)
+
+
+def test_sizes_follow_the_storage_formula():
+    """hann_sizeof against the closed forms: 16*L*R bytes per encoded row, 32*L*R per encrypted row (the paper's
+    80*L*R of Sec. 2 without its 2.5x serialization overhead)"""
+    from paper_2608_21131_b200 import binding as b
+
+    for ps in (synth.small_params(10, 16, 4, L=2), synth.FULL16):
+        g = b.Context(ps)
+        assert g.sizeof(b.SIZE_ROWS_PER_BLOCK) == ps.n
+        assert g.sizeof(b.SIZE_PT_BLOCK) == 16 * ps.L * ps.R * ps.n
+        assert g.sizeof(b.SIZE_CTDB_BLOCK) == 32 * ps.L * ps.R * ps.n
+        assert g.sizeof(b.SIZE_CT) == 2 * ps.L * ps.N * 8 and g.sizeof(b.SIZE_BABY) == ps.B * g.sizeof(b.SIZE_CT)
+        assert g.sizeof(b.SIZE_INNER) == ps.G * g.sizeof(b.SIZE_CT)
+        assert g.sizeof(b.SIZE_EVK) == ps.L * 2 * (ps.L + 1) * ps.N * 8

@@ -77,3 +77,24 @@ def test_padding_groups_partition_and_inflate():
     # fixed groups: the same cell always brings the same decoys
     again = synth.padded_fetch(pi, np.array([500]), 4)
     assert set(again.tolist()) <= set(fetched.tolist()) and len(again) == 4
+
+
+def test_storage_formula_matches_the_papers_worked_example():
+    """Sec. 2, "Measured prototype vs. deployment": 80*L*R bytes per encrypted vector, with the totals the paper prints
+    (tests/golden/storage_per_vector.txt).  This library's own layout is the same count without the 2.5x serialization
+    overhead: R ciphertexts of 2*L*N*8 bytes per block of N/2 rows = 32*L*R bytes per encrypted row, 16*L*R per encoded
+    plaintext row."""
+    import os
+
+    unit = {"KB": 1e3, "GB": 1e9, "TB": 1e12}
+    path = os.path.join(os.path.dirname(__file__), "golden", "storage_per_vector.txt")
+    rows = [ln.split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 5
+    for L, R, count, printed, u in rows:
+        total = 80 * int(L) * int(R) * int(count)
+        assert abs(total / unit[u] - float(printed)) / float(printed) < 0.02       # the paper rounds to two digits
+    for ps in (synth.TOY, synth.FULL15, synth.FULL16):
+        ct_bytes = 2 * ps.L * ps.N * 8
+        assert ps.R * ct_bytes // ps.n == 32 * ps.L * ps.R                       # encrypted block / rows per block
+        assert ps.R * ps.L * ps.N * 8 // ps.n == 16 * ps.L * ps.R                 # encoded plaintext block
+        assert 2.5 * 32 * ps.L * ps.R == 80 * ps.L * ps.R

@@ -474,3 +474,39 @@ def test_sizes_follow_the_storage_formula():
         assert g.sizeof(b.SIZE_CT) == 2 * ps.L * ps.N * 8 and g.sizeof(b.SIZE_BABY) == ps.B * g.sizeof(b.SIZE_CT)
         assert g.sizeof(b.SIZE_INNER) == ps.G * g.sizeof(b.SIZE_CT)
         assert g.sizeof(b.SIZE_EVK) == ps.L * 2 * (ps.L + 1) * ps.N * 8
+
+
+def random_shapes(count, seed):
+    """seeded random parameter shapes: ring 2^4..2^11, 1..4 ciphertext primes of 30..48 bits, R | n, B | R, ragged row
+    counts over up to three blocks, dim <= R"""
+    from oracle.oracle import find_primes
+
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(count):
+        logN = int(rng.integers(4, 12))
+        n = 1 << (logN - 1)
+        L = int(rng.integers(1, 5))
+        bits = int(rng.choice([30, 36, 42, 48]))
+        R = 1 << int(rng.integers(1, min(logN - 1, 7) + 1))
+        B = 1 << int(rng.integers(0, int(np.log2(R)) + 1))
+        dim = int(rng.integers(1, R + 1))
+        n_rows = int(rng.integers(1, 3 * n + 1))
+        q = find_primes(bits, 13, L)
+        p = find_primes(bits + 8, 13, 1)[0]
+        # the scale leaves room for scale^2 * |score| under the modulus and keeps the encoding error small
+        log_scale = min(25, (bits * L - 6) // 2)
+        tol = -10 if log_scale >= 25 else -(log_scale - 12)
+        out.append(pytest.param(logN, R, B, tuple(q), p, log_scale, tol, dim, n_rows,
+                                id="N%d-R%d-B%d-L%d-%db-dim%d-rows%d" % (logN, R, B, L, bits, dim, n_rows)))
+    return out
+
+
+@pytest.mark.parametrize("logN,R,B,q,p,log_scale,tol,dim,n_rows", random_shapes(14, 20260825))
+def test_level_bit_exact_random_shapes(logN, R, B, q, p, log_scale, tol, dim, n_rows):
+    ps = synth.ParamSet("rand", logN, q, p, log_scale, R, B, tol)
+    pair = Pair(ps, key_seed=n_rows)
+    rows = synth.toy_corpus(n_rows, rows=n_rows, dim=dim)
+    qv = np.zeros(R, dtype=np.float32)
+    qv[:dim] = synth.toy_query(n_rows + 1, dim=dim)
+    run_level(pair, rows, qv)

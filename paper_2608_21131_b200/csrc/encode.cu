@@ -270,10 +270,12 @@ __global__ void __launch_bounds__(128) k_fft_w(FusedArgs A) {
 // Kernel W for B >= 8: a CTA takes ONE chunk of 256 FFT positions for EIGHT plaintexts (g, b0 .. b0+7).  For a given
 // position the eight plaintexts read eight consecutive columns of the same candidate row, so the gather moves whole
 // 32-byte sectors instead of one float per sector, and all of a thread's 16 loads are independent.
-__global__ void __launch_bounds__(128) k_fft_w8(FusedArgs A) {
+__global__ void __launch_bounds__(128, 5) k_fft_w8(FusedArgs A) {
     __shared__ double2 tc[256];
     __shared__ double2 sm[8 * 272];
-    __shared__ float sin_[8 * 272];  // gathered inputs [plaintext][position + position/16]
+    // gathered inputs [plaintext][position + position/16]: they live in the tail of the exchange tile until round 1 has
+    // read them (38 KiB per CTA: five CTAs per SM)
+    float* sin_ = (float*)(sm + 8 * 272) - 8 * 272;
     const int n = 1 << A.logn;
     const int P0 = blockIdx.y * 8;
     const int g = (A.p_first + P0) / A.B, b0 = (A.p_first + P0) % A.B;
@@ -306,6 +308,7 @@ __global__ void __launch_bounds__(128) k_fft_w8(FusedArgs A) {
                 if (!(e & span)) dit(x[e], x[e + span], tc[span - 1 + (e & (span - 1))]);
         }
         double2* d = sm + pl * 272 + 17 * j;
+        __syncthreads();  // every thread has read its gathered inputs: the tile may be overwritten
 #pragma unroll
         for (int e = 0; e < 16; e++) d[e] = x[e];
     }

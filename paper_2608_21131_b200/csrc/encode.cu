@@ -333,7 +333,7 @@ __global__ void __launch_bounds__(128, 5) k_fft_w8(FusedArgs A) {
 // R1 + R2 = a = logN - 8 are the register rounds of the transform's pass A (R1 = min(a, 4)); the FFT's a - 1 strided
 // stages run as a first round of R2 stages and a last round of R1 - 1 stages
 #ifndef HANN_X_MINBLOCKS
-#define HANN_X_MINBLOCKS 2
+#define HANN_X_MINBLOCKS 3
 #endif
 template <int R1, int R2>
 __global__ void __launch_bounds__(256, HANN_X_MINBLOCKS) k_encode_x(FusedArgs A) {

@@ -125,8 +125,8 @@ FP64_LANES_PER_SM = 64  # binary64 multiply-add lanes per SM per clock
 # DRAM bytes (read + write) per unit of work of the bandwidth- or transform-bound kernels, from the ncu captures
 # summarised under profiles/ (small case: one block of 32,768 rows; traffic grows in proportion to the units)
 NCU_DRAM_BYTES_PER_UNIT = {
-    "ntt_fwd_b": ("polynomial", 490.2e6 / 512),
-    "fft_b": ("plaintext", 276.8e6 / 128),
+    "ntt_fwd_b": ("polynomial", 490.4e6 / 512),
+    "fft_b": ("plaintext", 288.1e6 / 128),
     "mac": ("block", None),
     "ks_inner": ("item", None),
 }

@@ -55,3 +55,26 @@ def test_single_process_identity():
 
     assert bench.max_over_ranks(3.5, None, torch.device("cpu")) == 3.5
     assert bench.replica_throughput(100, 1, 0.5) == 200.0
+
+
+def test_algorithmic_work_matches_the_per_row_figures():
+    """the roofline numerators of bench.py against the closed forms of the design: a scored row costs the multiply-
+    accumulate 16*L*R bytes of plaintext read + 32*L*G bytes of partial sums written (8,192 + 512 at L = 4, R = 128,
+    G = 4), the baby set is read once per level, and a block's encoding is R*L transforms of N/2*log2(N) butterflies"""
+    import types
+
+    import bench
+
+    L, logN, R, B = 4, 16, 128, 32
+    N, n, G = 1 << logN, 1 << (logN - 1), R // B
+    ctx = types.SimpleNamespace(L=L, N=N, n=n, logN=logN, R=R, B=B, G=G)
+    for n_blocks in (1, 7):
+        w = bench.algorithmic_work(ctx, n_blocks, n_blocks * n)
+        bound, mac_bytes, units = w["mac"]
+        assert bound == "hbm" and units == n_blocks
+        assert mac_bytes == n_blocks * n * (16 * L * R + 32 * L * G) + B * 2 * L * N * 8
+        assert 16 * L * R + 32 * L * G == 8704
+        # pass B of the forward transforms: 8 of the 16 stages of every polynomial, 8 binary64 instructions per butterfly
+        fwd_polys = w["ntt_fwd_b"][2]
+        assert fwd_polys == n_blocks * R * L + (L * (L + 1) + (B - 1) * 2 * L) + (G - 1) * n_blocks * (L * (L + 1) + 2 * L)
+        assert w["ntt_fwd_b"][1] == fwd_polys * (N // 2) * 8 * 8

@@ -1,6 +1,9 @@
 """Build the CUDA library (`libhann.so`) in-tree with nvcc for sm_100a.
 
     python -m paper_2608_21131_b200.build [--force] [--verbose]
+
+`build(extra_flags=...)` passes further compiler flags, e.g. `-DHANN_NO_B8T` / `-DHANN_NO_MAC_BULK` to build the
+transform's pass B / the multiply-accumulate without their bulk-copy kernels (A/B comparisons; results are identical).
 """
 from __future__ import annotations
 

@@ -70,3 +70,26 @@ def test_context_refuses_to_run_without_cuda():
         pytest.skip("a CUDA device is present")
     with pytest.raises(RuntimeError):
         binding.Context(synth.TOY)
+
+
+def test_product_path_is_independent_of_the_oracle_and_of_scratch_files():
+    """the package never imports the CPU oracle (only tests, the smoke check and bench.py's CPU legs may), the oracle never
+    imports the package's CUDA side, and nothing that is committed reads the scratch folder"""
+    import subprocess
+
+    pkg = os.path.join(ROOT, "paper_2608_21131_b200")
+    for name in os.listdir(pkg):
+        if name.endswith(".py"):
+            src = open(os.path.join(pkg, name)).read()
+            assert not re.search(r"^\s*(from|import)\s+oracle\b", src, flags=re.M), name
+    for name in ("oracle.py",):
+        src = open(os.path.join(ROOT, "oracle", name)).read()
+        assert not re.search(r"paper_2608_21131_b200\s*(\.|import)\s*(binding|build)", src) and "libhann.so" not in src
+    csrc = os.path.join(pkg, "csrc")
+    for name in os.listdir(csrc):
+        assert "oracle" not in open(os.path.join(csrc, name)).read().lower(), name
+    assert "hann.h" not in open(os.path.join(ROOT, "oracle", "hann_oracle.c")).read()
+    tracked = subprocess.run(["git", "ls-files"], cwd=ROOT, capture_output=True, text=True).stdout.split()
+    for f in tracked:
+        if f.endswith((".py", ".cu", ".cuh", ".h", ".c", ".cpp")) and f != "tests/test_abi.py":
+            assert not re.search(r"(^|[\"'/\s])_work(/|[\"'])", open(os.path.join(ROOT, f)).read()), f

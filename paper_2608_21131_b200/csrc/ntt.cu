@@ -263,13 +263,11 @@ __global__ void __launch_bounds__(256, HANN_B8_MINBLOCKS) k_ntt_fwd_b8(NttArgs A
 // and stops.
 constexpr int kTK = 2, kTP = 8;       // chunks per CTA, polynomials per tile (= warps per CTA)
 template <class AR>
-__global__ void __launch_bounds__(256, 3) k_ntt_fwd_b8t(NttArgs A, int groups, int* kflag) {
-    extern __shared__ __align__(128) u64 smraw[];
+__device__ __forceinline__ void fwd_b8t_body(const NttArgs& A, int groups, int* kflag, int k, u64* smraw) {
     typedef typename AR::TW TW;
     TW* tc = (TW*)smraw;                                 // twiddle cache [kTK][256], layout as in k_ntt_fwd_b8
     u64* bufs = smraw + kTK * 256 * 2;                   // [kTP][2][512] landing / exchange buffers
     u64* bars = bufs + kTP * 2 * 512;                    // [kTP][2] mbarriers
-    const int k = blockIdx.y;
     const int pos = (int)((A.pos4 >> (4 * k)) & 15), limb = (int)((A.limb4 >> (4 * k)) & 15);
     const AR ar(A.lt + limb);
     const int chunk0 = blockIdx.x * kTK;
@@ -344,6 +342,21 @@ __global__ void __launch_bounds__(256, 3) k_ntt_fwd_b8t(NttArgs A, int groups, i
             bulk_load(buf0 + 4096 * s, gbase + (long long)(i + 2) * ystep * tile_stride, 4096, bar0 + 8 * s);
         }
     }
+}
+
+template <class AR>
+__global__ void __launch_bounds__(256, 3) k_ntt_fwd_b8t(NttArgs A, int groups, int* kflag) {
+    extern __shared__ __align__(128) u64 smraw[];
+    fwd_b8t_body<AR>(A, groups, kflag, blockIdx.y, smraw);
+}
+
+// One launch for the two arithmetic classes of a batch over {q_0 .. q_{L-1}, p} (binary64 limbs and the special prime's
+// Harvey integers): the selections of the integer class follow those of the binary64 class along blockIdx.y.  Saves a
+// launch per key switch, which matters on levels of one or two blocks.
+__global__ void __launch_bounds__(256, 3) k_ntt_fwd_b8t_mixed(NttArgs Af, NttArgs Ai, int groups, int* kflag) {
+    extern __shared__ __align__(128) u64 smraw[];
+    if ((int)blockIdx.y < Af.nsel) fwd_b8t_body<ArithF64>(Af, groups, kflag, blockIdx.y, smraw);
+    else fwd_b8t_body<ArithInt<false>>(Ai, groups, kflag, blockIdx.y - Af.nsel, smraw);
 }
 
 // Inverse pass B' (spans 1 .. 128 inside chunks, the first pass of an inverse transform) in the same form: bulk copies
@@ -729,35 +742,54 @@ size_t smem_b(const NttArgs& A) {
     return (size_t)A.K * (S + (S >> R2)) * 8;
 }
 
+bool b8t_eligible(const hann_ctx* c, const NttArgs& A) {
+#ifndef HANN_NO_B8T
+    return A.b == 8 && A.a > 0 && A.tau && ((c->N >> 8) % kTK) == 0 && ((uintptr_t)A.data & 15) == 0 && (A.stride & 1) == 0;
+#else
+    (void)c; (void)A;
+    return false;
+#endif
+}
+constexpr size_t kB8tSmem = (size_t)kTK * 256 * 16 + (size_t)kTP * 2 * 512 * 8 + (size_t)kTP * 2 * 8;
+// tiles per CTA: a CTA stages its twiddles once and its warps prefetch two tiles ahead, but the grid should still fill whole
+// waves of the 148 x 3 resident CTAs.  Smallest (waves x (tiles per CTA + staging)), ties to fewer CTAs.
+int b8t_zsplit(int per, int ntiles) {
+    const int slots = 148 * 3;
+    int zs = 1;
+    long best = -1;
+    for (int z = 1; z <= ntiles && z <= 64; z++) {
+        const long waves = ((long)per * z + slots - 1) / slots, tiles = (ntiles + z - 1) / z;
+        const long cost = waves * (4 * tiles + 1);
+        if (best < 0 || cost < best) {
+            best = cost;
+            zs = z;
+        }
+    }
+    return zs;
+}
+
+// pass B of a batch whose limbs fall into the binary64 class (Af) and the Harvey integer class (Ai): one launch
+void launch_fwd_b8t_mixed(hann_ctx* c, const NttArgs& Af, const NttArgs& Ai, int groups) {
+    KProf kp(c, KC_NTT_FWD_B);
+    cudaFuncSetAttribute(k_ntt_fwd_b8t_mixed, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kB8tSmem);
+    const int ranges = (c->N >> 8) / kTK, ntiles = (groups + kTP - 1) / kTP, nsel = Af.nsel + Ai.nsel;
+    k_ntt_fwd_b8t_mixed<<<dim3(ranges, nsel, b8t_zsplit(ranges * nsel, ntiles)), 256, kB8tSmem, c->stream>>>(Af, Ai, groups, c->kflag);
+}
+
 template <class AR>
-void launch_fwd_class(hann_ctx* c, const NttArgs& A, int groups, bool skip_a) {
+void launch_fwd_class(hann_ctx* c, const NttArgs& A, int groups, bool skip_a, bool skip_b = false) {
     if (A.a > 0 && !skip_a) {
         KProf kp(c, KC_NTT_FWD_A);
         pick_fwd_a<AR>(A.a)<<<dim3(1 << (A.b - A.logC), groups * A.nsel), kThreads, smem_a(A), c->stream>>>(A);
     }
+    if (skip_b) return;
     KProf kp(c, KC_NTT_FWD_B);
-#ifndef HANN_NO_B8T
-    if (A.b == 8 && A.a > 0 && A.tau && ((c->N >> 8) % kTK) == 0 && ((uintptr_t)A.data & 15) == 0 && (A.stride & 1) == 0) {
-        const size_t smem = (size_t)kTK * 256 * 16 + (size_t)kTP * 2 * 512 * 8 + (size_t)kTP * 2 * 8;
-        cudaFuncSetAttribute(k_ntt_fwd_b8t<AR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (b8t_eligible(c, A)) {
+        cudaFuncSetAttribute(k_ntt_fwd_b8t<AR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kB8tSmem);
         const int ranges = (c->N >> 8) / kTK, ntiles = (groups + kTP - 1) / kTP;
-        // tiles per CTA: a CTA stages its twiddles once and its warps prefetch two tiles ahead, but the grid should still
-        // fill whole waves of the 148 x 3 resident CTAs.  Smallest (waves x (tiles per CTA + staging)), ties to fewer CTAs.
-        const int slots = 148 * 3, per = ranges * A.nsel;
-        int zs = 1;
-        long best = -1;
-        for (int z = 1; z <= ntiles && z <= 64; z++) {
-            const long waves = ((long)per * z + slots - 1) / slots, tiles = (ntiles + z - 1) / z;
-            const long cost = waves * (4 * tiles + 1);
-            if (best < 0 || cost < best) {
-                best = cost;
-                zs = z;
-            }
-        }
-        k_ntt_fwd_b8t<AR><<<dim3(ranges, A.nsel, zs), 256, smem, c->stream>>>(A, groups, c->kflag);
+        k_ntt_fwd_b8t<AR><<<dim3(ranges, A.nsel, b8t_zsplit(ranges * A.nsel, ntiles)), 256, kB8tSmem, c->stream>>>(A, groups, c->kflag);
         return;
     }
-#endif
     if (A.b == 8 && A.a > 0 && A.tau && ((c->N >> 8) % kBK) == 0) {
         const size_t smem = (size_t)kBK * 256 * 16 + (size_t)kBPG * kBK * 272 * 8;
         cudaFuncSetAttribute(k_ntt_fwd_b8<AR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  // 50 KiB > default 48
@@ -831,28 +863,43 @@ int launch_ntt(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const Limb
     A.tau = c->ntt_tau;
     A.period = lm.period;
     const int64_t groups_total = npoly / lm.period;
+    NttArgs Ac[3];
     for (int cls = 0; cls < 3; cls++) {
-        A.nsel = 0;
-        A.pos4 = A.limb4 = 0;
+        Ac[cls] = A;
+        NttArgs& X = Ac[cls];
+        X.nsel = 0;
+        X.pos4 = X.limb4 = 0;
         for (int i = 0; i < lm.period && i < 16; i++)
             if (arith_class(c->mod[(int)lm.limb[i]], inverse) == cls) {
-                A.pos4 |= (u64)i << (4 * A.nsel);
-                A.limb4 |= (u64)lm.limb[i] << (4 * A.nsel);
-                A.nsel++;
+                X.pos4 |= (u64)i << (4 * X.nsel);
+                X.limb4 |= (u64)lm.limb[i] << (4 * X.nsel);
+                X.nsel++;
             }
-        if (!A.nsel) continue;
-        A.tw = cls == 0 ? (const void*)(inverse ? c->tw_inv_f64 : c->tw_fwd_f64) : (const void*)(inverse ? c->tw_inv : c->tw_fwd);
-        const int64_t gmax = 65535 / A.nsel;
+        X.tw = cls == 0 ? (const void*)(inverse ? c->tw_inv_f64 : c->tw_fwd_f64) : (const void*)(inverse ? c->tw_inv : c->tw_fwd);
+    }
+    // forward, binary64 limbs plus the special prime, bulk-copy kernel applicable: pass B of both classes in one launch
+    const bool mixed = !inverse && Ac[0].nsel && Ac[2].nsel && !Ac[1].nsel;
+    for (int cls = 0; cls < 3; cls++) {
+        NttArgs& X = Ac[cls];
+        if (!X.nsel) continue;
+        const int64_t gmax = 65535 / (mixed ? Ac[0].nsel + Ac[2].nsel : X.nsel);
         for (int64_t g0 = 0; g0 < groups_total; g0 += gmax) {
             const int groups = (int)std::min<int64_t>(gmax, groups_total - g0);
-            A.data = data + g0 * lm.period * stride;
+            X.data = data + g0 * lm.period * stride;
+            const bool merge = mixed && b8t_eligible(c, X);
             if (!inverse) {
-                if (cls == 0) launch_fwd_class<ArithF64>(c, A, groups, skip_a);
-                else if (cls == 1) launch_fwd_class<ArithInt<true>>(c, A, groups, skip_a);
-                else launch_fwd_class<ArithInt<false>>(c, A, groups, skip_a);
+                if (cls == 0) launch_fwd_class<ArithF64>(c, X, groups, skip_a, merge);
+                else if (cls == 1) launch_fwd_class<ArithInt<true>>(c, X, groups, skip_a);
+                else {
+                    launch_fwd_class<ArithInt<false>>(c, X, groups, skip_a, merge);
+                    if (merge) {
+                        Ac[0].data = X.data;
+                        launch_fwd_b8t_mixed(c, Ac[0], X, groups);
+                    }
+                }
             } else {
-                if (cls == 0) launch_inv_class<ArithF64>(c, A, groups, skip_a);
-                else launch_inv_class<ArithInt<false>>(c, A, groups, skip_a);
+                if (cls == 0) launch_inv_class<ArithF64>(c, X, groups, skip_a);
+                else launch_inv_class<ArithInt<false>>(c, X, groups, skip_a);
             }
         }
     }

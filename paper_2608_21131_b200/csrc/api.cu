@@ -135,13 +135,20 @@ int upload_secret(hann_ctx* c, const int8_t* s_host, int nlimbs, int8_t* s8, u64
 // ---- one key switch round on `items` polynomials ---------------------------------------------------------------
 // c1c[items][L][N] (the polynomials to switch, transform domain, item stride L*N; overwritten) -> u, lifted; combine is
 // left to the caller because its sources and targets differ between the callers.
+// gather_src (optional): the polynomials to switch still lie at gather_src + item * gather_stride (L limbs each); they are
+// brought into c1c on the way (by the inverse pass itself where its bulk-copy kernel applies, by a strided copy otherwise).
 int ks_digits_to_lifted(hann_ctx* c, u64* c1c, int64_t items, u64* digits, int64_t digit_stride, int rot0, int rot_inc,
-                        int64_t u_items, u64* u, u64* lifted) {
+                        int64_t u_items, u64* u, u64* lifted, const u64* gather_src = nullptr, int64_t gather_stride = 0) {
     const int L = c->L, N = c->N;
+    const int64_t LN = (int64_t)L * N;
+    const bool fused_gather = gather_src && ks_lift_available(c) && ntt_inv_pass_b_gathers(c, gather_src, c1c) && (gather_stride & 1) == 0;
+    if (gather_src && !fused_gather)
+        CK(cudaMemcpy2DAsync(c1c, LN * 8, gather_src, gather_stride * 8, LN * 8, items, cudaMemcpyDeviceToDevice, c->stream));
     if (ks_lift_available(c)) {
         // c1c arrives in the transform domain: inverse pass B', then one kernel finishes the inverse, lifts the digits
         // and starts their forward transforms; the same again for ModDown
-        RET(launch_ntt_inv_pass_b(c, c1c, items * L, N, limbmap_q(c)));
+        if (fused_gather) RET(launch_ntt_inv_pass_b_from(c, gather_src, gather_stride, c1c, items * L, N, limbmap_q(c)));
+        else RET(launch_ntt_inv_pass_b(c, c1c, items * L, N, limbmap_q(c)));
         RET(launch_ks_lift(c, c1c, N, items * L, limbmap_q(c), digits, L + 1, 0));
         RET(launch_ntt_fwd_pass_b(c, digits, items * L * (L + 1), N, limbmap_qp(c)));
         RET(launch_ks_inner(c, digits, digit_stride, rot0, rot_inc, u_items, u));
@@ -990,8 +997,7 @@ extern "C" int hann_rotate_sum(hann_ctx* c, const void* inner_dev, int64_t n_blo
             for (int g = G - 2; g >= 0; g--) {
                 u64* out = (g % 2 == 0) ? score + b0 * ctw : tmp;
                 // c1 of every accumulator, still in the transform domain; the key-switch round takes it from there
-                CK(cudaMemcpy2DAsync(c1c, LN * 8, old + LN, old_stride * 8, LN * 8, nb, cudaMemcpyDeviceToDevice, c->stream));
-                RET(ks_digits_to_lifted(c, c1c, nb, digits, (int64_t)L * L1N, B, 0, nb, u, lifted));
+                RET(ks_digits_to_lifted(c, c1c, nb, digits, (int64_t)L * L1N, B, 0, nb, u, lifted, old + LN, old_stride));
                 RET(launch_moddown_combine(c, u, lifted, nb, B, 0, old, old_stride, inner + (b0 * G + g) * ctw, (int64_t)G * ctw, out,
                                            out + LN, ctw));
                 old = out;

@@ -118,6 +118,8 @@ int launch_ntt_fwd(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const 
 int launch_ntt_inv(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
 int launch_ntt_fwd_pass_b(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
 int launch_ntt_inv_pass_b(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
+bool ntt_inv_pass_b_gathers(const hann_ctx* c, const void* src, const void* dst);
+int launch_ntt_inv_pass_b_from(hann_ctx* c, const u64* src, int64_t src_gstride, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
 bool ks_lift_available(const hann_ctx* c);
 int launch_wait_selftest(hann_ctx* c, unsigned long long limit_ns, unsigned long long* waited_ns_dev);
 int launch_ks_lift(hann_ctx* c, u64* src, int64_t src_stride, int64_t nsrc, const LimbMap& src_lm, u64* dst, int n_tgt, int tgt_limb0);

@@ -53,6 +53,10 @@ struct NttArgs {
     // limb[]): all positions whose modulus falls in the launch's arithmetic class
     int period, nsel;
     int tau;  // chunks of 256 positions are stored with their low nibbles swapped (see galois_src)
+    // inverse pass B' only (bulk-copy kernel): read group g, position pos from src + g * src_gstride + pos * stride instead
+    // of from `data` (nullptr: in place)
+    const u64* src;
+    long long src_gstride;
     u64 pos4, limb4;  // 4-bit fields: position within the period and limb of selection k (at most 16 selections)
 };
 
@@ -392,13 +396,16 @@ __global__ void __launch_bounds__(256, 3) k_ntt_inv_b8t(NttArgs A, int groups, i
     __syncwarp();
     const int yg0 = blockIdx.z, ystep = gridDim.z;
     u64* gbase = A.data + (((long long)yg0 * kTP + t) * A.period + pos) * A.stride + ((size_t)chunk0 << 8);
+    // source of the copies: the same words, or a separately laid out input (group stride src_gstride)
+    const u64* sbase = A.src ? A.src + ((long long)yg0 * kTP + t) * A.src_gstride + (long long)pos * A.stride + ((size_t)chunk0 << 8) : gbase;
+    const long long stile_stride = A.src ? (long long)kTP * A.src_gstride : (long long)kTP * A.period * A.stride;
     const int my_tiles = yg0 < ntiles ? (ntiles - yg0 + ystep - 1) / ystep : 0;
     auto tile_valid = [&](int i) { return i < my_tiles && (long long)(yg0 + (long long)i * ystep) * kTP + t < groups; };
     if (lane == 0) {
         for (int i = 0; i < 2; i++)
             if (tile_valid(i)) {
                 mbar_expect_tx(bar0 + 8 * i, 4096);
-                bulk_load(buf0 + 4096 * i, gbase + (long long)i * ystep * tile_stride, 4096, bar0 + 8 * i);
+                bulk_load(buf0 + 4096 * i, sbase + (long long)i * ystep * stile_stride, 4096, bar0 + 8 * i);
             }
     }
     for (int i = threadIdx.x; i < kTK * 256; i += 256) {
@@ -442,7 +449,7 @@ __global__ void __launch_bounds__(256, 3) k_ntt_inv_b8t(NttArgs A, int groups, i
         __syncwarp();
         if (lane == 0 && tile_valid(i + 2)) {
             mbar_expect_tx(bar0 + 8 * s, 4096);
-            bulk_load(buf0 + 4096 * s, gbase + (long long)(i + 2) * ystep * tile_stride, 4096, bar0 + 8 * s);
+            bulk_load(buf0 + 4096 * s, sbase + (long long)(i + 2) * ystep * stile_stride, 4096, bar0 + 8 * s);
         }
     }
 }
@@ -816,7 +823,8 @@ void launch_fwd_class(hann_ctx* c, const NttArgs& A, int groups, bool skip_a, bo
 
 template <class AR>
 void launch_inv_class(hann_ctx* c, const NttArgs& A, int groups, bool skip_a) {
-    if (A.b == 8 && A.a > 0 && A.tau && ((c->N >> 8) % kTK) == 0 && ((uintptr_t)A.data & 15) == 0 && (A.stride & 1) == 0) {
+    if (A.b == 8 && A.a > 0 && A.tau && ((c->N >> 8) % kTK) == 0 && ((uintptr_t)A.data & 15) == 0 && (A.stride & 1) == 0 &&
+        ((uintptr_t)A.src & 15) == 0 && (A.src_gstride & 1) == 0) {
         KProf kp(c, KC_NTT_INV_B);
         const size_t smem = (size_t)kTK * 256 * 16 + (size_t)kTP * 2 * 512 * 8 + (size_t)kTP * 2 * 8;
         cudaFuncSetAttribute(k_ntt_inv_b8t<AR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -845,7 +853,8 @@ void launch_inv_class(hann_ctx* c, const NttArgs& A, int groups, bool skip_a) {
 
 // npoly polynomials, `stride` words apart, polynomial p using modulus lm.limb[p % lm.period]; npoly must be a multiple of
 // the period.  One set of launches per arithmetic class present in the period.
-int launch_ntt(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm, bool inverse, bool skip_a = false) {
+int launch_ntt(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm, bool inverse, bool skip_a = false,
+               const u64* src = nullptr, int64_t src_gstride = 0) {
     if (npoly <= 0) return HANN_OK;
     if (npoly % lm.period) {
         c->err = "transform batch is not a whole number of limb periods";
@@ -861,7 +870,14 @@ int launch_ntt(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const Limb
     A.K = chunks < 16 ? chunks : 16;
     A.lt = c->lt_dev;
     A.tau = c->ntt_tau;
+    A.src = src;
+    A.src_gstride = src_gstride;
     A.period = lm.period;
+    if (src && !(inverse && skip_a && A.b == 8 && A.a > 0 && A.tau && ((c->N >> 8) % kTK) == 0 && (((uintptr_t)data | (uintptr_t)src) & 15) == 0 &&
+                 ((stride | src_gstride) & 1) == 0)) {
+        c->err = "inverse pass B with a separate source needs the bulk-copy kernel (ring of 2^10 or more, 16-byte aligned buffers)";
+        return HANN_EINVAL;
+    }
     const int64_t groups_total = npoly / lm.period;
     NttArgs Ac[3];
     for (int cls = 0; cls < 3; cls++) {
@@ -886,6 +902,7 @@ int launch_ntt(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const Limb
         for (int64_t g0 = 0; g0 < groups_total; g0 += gmax) {
             const int groups = (int)std::min<int64_t>(gmax, groups_total - g0);
             X.data = data + g0 * lm.period * stride;
+            if (src) X.src = src + g0 * src_gstride;
             const bool merge = mixed && b8t_eligible(c, X);
             if (!inverse) {
                 if (cls == 0) launch_fwd_class<ArithF64>(c, X, groups, skip_a, merge);
@@ -989,6 +1006,22 @@ int launch_ks_lift(hann_ctx* c, u64* src, int64_t src_stride, int64_t nsrc, cons
 
 int launch_ntt_inv_pass_b(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm) {
     return launch_ntt(c, data, npoly, stride, lm, true, true);
+}
+
+bool ntt_inv_pass_b_gathers(const hann_ctx* c, const void* src, const void* dst) {
+#ifndef HANN_NO_B8T
+    return c->logN >= 10 && ((c->N >> 8) % kTK) == 0 && (((uintptr_t)src | (uintptr_t)dst) & 15) == 0;
+#else
+    (void)c; (void)src; (void)dst;
+    return false;
+#endif
+}
+
+// The same with the input read from elsewhere: group g (lm.period polynomials, `stride` words apart) starts at
+// src + g * src_gstride; the output goes to data as above.  Only where ntt_inv_pass_b_gathers(c) holds and both pointers are
+// 16-byte aligned (the bulk-copy kernel); the caller copies and uses launch_ntt_inv_pass_b otherwise.
+int launch_ntt_inv_pass_b_from(hann_ctx* c, const u64* src, int64_t src_gstride, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm) {
+    return launch_ntt(c, data, npoly, stride, lm, true, true, src, src_gstride);
 }
 
 int launch_wait_selftest(hann_ctx* c, unsigned long long limit_ns, unsigned long long* waited_ns_dev) {

@@ -121,8 +121,12 @@ int hann_get_stats(hann_ctx *ctx, hann_stats *out);
  * launch group in hann_encode_candidates (default: all R plaintexts of a block at once); ask hann_workspace_bytes again after changing it.
  * HANN_TUNE_HOST_LIMBS (this one DOES change a result's layout): hann_score_level_host downloads only the first `value`
  * limbs of every score polynomial, score_ct_host [blocks][2][value][N] -- the exact form of hann_compact_scores; decrypt
- * with hann_decrypt_compact(limbs = value, rescaled = 0).  Default L. */
-enum { HANN_TUNE_ENCODE_GROUP = 1, HANN_TUNE_HOST_LIMBS = 2 };
+ * with hann_decrypt_compact(limbs = value, rescaled = 0).  Default L.
+ * HANN_TUNE_ENCODE_SYMMETRY: 1 (default) lets hann_encode_candidates use the fact that the encoding of a REAL slot vector
+ * is fixed by X -> 1/X, so that its number-theoretic transform takes each value twice (at psi^(2t+1) and at the inverse
+ * of that root): only half of every transform is computed and the other half is written as a mirror image; 0 computes
+ * every transform in full.  Same bits either way. */
+enum { HANN_TUNE_ENCODE_GROUP = 1, HANN_TUNE_HOST_LIMBS = 2, HANN_TUNE_ENCODE_SYMMETRY = 3 };
 int hann_set_tuning(hann_ctx *ctx, int what, int value);
 
 /* Per-launch profile: while enabled every kernel launch of the context is bracketed by a CUDA event pair (this

@@ -21,6 +21,7 @@ SIZE_POLY, SIZE_CT, SIZE_BABY, SIZE_PT_BLOCK, SIZE_INNER, SIZE_EVK, SIZE_ROWS_PE
 KIND_POLY, KIND_CT, KIND_PT = 1, 2, 3
 TUNE_ENCODE_GROUP = 1
 TUNE_HOST_LIMBS = 2
+TUNE_ENCODE_SYMMETRY = 3
 
 
 class HannError(RuntimeError):

@@ -425,6 +425,9 @@ extern "C" int hann_set_tuning(hann_ctx* c, int what, int value) {
             if (value < 1 || value > c->L) return fail(c, HANN_EINVAL, "hann_set_tuning: host limbs must be in 1..L");
             c->host_limbs = value;
             return HANN_OK;
+        case HANN_TUNE_ENCODE_SYMMETRY:
+            c->encode_sym = value ? 1 : 0;
+            return HANN_OK;
         default: return fail(c, HANN_EINVAL, "hann_set_tuning: unknown knob");
     }
 }
@@ -888,8 +891,12 @@ extern "C" int hann_encode_candidates(hann_ctx* c, const float* rows_dev, int64_
         for (int p0 = 0; p0 < c->R; p0 += c->encode_group) {
             const int cnt = std::min(c->encode_group, c->R - p0);
             if (encode_fused_available(c)) {
-                RET(launch_encode_rows_fused(c, rows_dev + blk * n * dim, rows_here, dim, p0, cnt, pt, ws));
-                RET(launch_ntt_fwd_pass_b(c, pt + (int64_t)p0 * c->L * c->N, (int64_t)cnt * c->L, c->N, limbmap_q(c)));
+                // real slot vectors: the transform of an encoding takes every value twice (at a root and at its inverse)
+                u64* polys = pt + (int64_t)p0 * c->L * c->N;
+                const bool sym = c->encode_sym && ntt_fwd_mirror_available(c, polys, c->N);
+                RET(launch_encode_rows_fused(c, rows_dev + blk * n * dim, rows_here, dim, p0, cnt, pt, ws, sym));
+                if (sym) RET(launch_ntt_fwd_pass_b_mirror(c, polys, (int64_t)cnt * c->L, c->N, limbmap_q(c)));
+                else RET(launch_ntt_fwd_pass_b(c, polys, (int64_t)cnt * c->L, c->N, limbmap_q(c)));
             } else {
                 RET(launch_encode_rows(c, rows_dev + blk * n * dim, rows_here, dim, p0, cnt, pt, ws));
                 RET(launch_ntt_fwd(c, pt + (int64_t)p0 * c->L * c->N, (int64_t)cnt * c->L, c->N, limbmap_q(c)));

@@ -335,7 +335,10 @@ __global__ void __launch_bounds__(128, 5) k_fft_w8(FusedArgs A) {
 #ifndef HANN_X_MINBLOCKS
 #define HANN_X_MINBLOCKS 3
 #endif
-template <int R1, int R2>
+// SYM: the encoding of a real slot vector is fixed by X -> 1/X, so its transform takes the same value at psi^(2t+1) and
+// at the inverse of that root.  After the first stage (which splits modulo X^n - i and X^n + i) only the first half
+// carries on; rows 2^(a-1) .. 2^a - 1 of the pass-A output are not produced, and pass B mirrors its results.
+template <int R1, int R2, bool SYM>
 __global__ void __launch_bounds__(256, HANN_X_MINBLOCKS) k_encode_x(FusedArgs A) {
     extern __shared__ u64 smx[];
     constexpr int a = R1 + R2;
@@ -411,7 +414,19 @@ __global__ void __launch_bounds__(256, HANN_X_MINBLOCKS) k_encode_x(FusedArgs A)
         const double2* tw = twc + l * NT;
         u64* base = A.out + ((long long)(A.p_first + P) * A.L + l) * N + c0;
         __syncthreads();  // the twiddle cache is filled (first limb) / the exchange tile is free again
-        if (active) {
+        if (active && SYM) {
+            constexpr int RS = R1 > 1 ? R1 - 1 : 1;
+            double x[1 << RS];
+            const double2 w1 = tw[1];
+#pragma unroll
+            for (int e = 0; e < HF; e++) x[e] = __dadd_rn(ar.reduce(m[e]), ar.mulmod_small(ar.reduce(m[e + HF]), w1));
+            fwd_round<RS, ArithF64, RS>(ar, x, tw, 2u);
+#pragma unroll
+            for (int e = 0; e < HF; e++) {
+                if (R2 == 0) base[(size_t)(g + G1 * e) * 256 + c] = ar.to_mid(x[e]);
+                else smx[((g + G1 * e) << 4) + c] = ar.to_exch(x[e]);
+            }
+        } else if (active) {
             double x[1 << R1];
 #pragma unroll
             for (int e = 0; e < (1 << R1); e++) x[e] = ar.reduce(m[e]);
@@ -424,7 +439,7 @@ __global__ void __launch_bounds__(256, HANN_X_MINBLOCKS) k_encode_x(FusedArgs A)
         }
         if (R2 > 0) {
             __syncthreads();
-            for (int w = threadIdx.x; w < (G2 << 4); w += blockDim.x) {
+            for (int w = threadIdx.x; w < ((SYM ? G2 / 2 : G2) << 4); w += blockDim.x) {
                 const int cc = w & 15, gg = w >> 4;
                 double x[1 << RR2];
 #pragma unroll
@@ -438,18 +453,20 @@ __global__ void __launch_bounds__(256, HANN_X_MINBLOCKS) k_encode_x(FusedArgs A)
 }
 
 typedef void (*KernX)(FusedArgs);
-KernX pick_x(int a) {
+template <bool SYM>
+KernX pick_x_t(int a) {
     switch (a) {
-        case 1: return k_encode_x<1, 0>;
-        case 2: return k_encode_x<2, 0>;
-        case 3: return k_encode_x<3, 0>;
-        case 4: return k_encode_x<4, 0>;
-        case 5: return k_encode_x<4, 1>;
-        case 6: return k_encode_x<4, 2>;
-        case 7: return k_encode_x<4, 3>;
-        default: return k_encode_x<4, 4>;
+        case 1: return k_encode_x<1, 0, false>;
+        case 2: return k_encode_x<2, 0, SYM>;
+        case 3: return k_encode_x<3, 0, SYM>;
+        case 4: return k_encode_x<4, 0, SYM>;
+        case 5: return k_encode_x<4, 1, SYM>;
+        case 6: return k_encode_x<4, 2, SYM>;
+        case 7: return k_encode_x<4, 3, SYM>;
+        default: return k_encode_x<4, 4, SYM>;
     }
 }
+KernX pick_x(int a, bool sym) { return sym && a >= 2 ? pick_x_t<true>(a) : pick_x_t<false>(a); }
 
 }  // namespace
 
@@ -462,8 +479,9 @@ bool encode_fused_available(const hann_ctx* c) {
 
 // plaintexts p_first .. p_first+count-1 of one block: encode and run pass A of their forward transforms; the caller
 // finishes with launch_ntt_fwd_pass_b over the same polynomials
+// (sym: leave the second half of the pass-A rows out; the caller then finishes with launch_ntt_fwd_pass_b_mirror)
 int launch_encode_rows_fused(hann_ctx* c, const float* rows, int64_t rows_in_block, int dim, int p_first, int count, u64* pt_block,
-                             void* ws) {
+                             void* ws, bool sym) {
     FusedArgs A;
     A.rows = rows;
     A.rows_in_block = rows_in_block;
@@ -513,8 +531,8 @@ int launch_encode_rows_fused(hann_ctx* c, const float* rows, int64_t rows_in_blo
         const size_t smem = (a > 4 ? (size_t)(1 << a) * 16 * 8 : 0) + (size_t)c->L * (1 << a) * 16;
         KProf kp(c, KC_FFT_B);
         const int threads = a >= 8 ? 256 : (a == 7 ? 128 : 64);  // 16 columns x 2^R2 row groups, at least two warps
-        if (smem > 48 * 1024) cudaFuncSetAttribute(pick_x(a), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        pick_x(a)<<<dim3(16, count), threads, smem, c->stream>>>(A);
+        if (smem > 48 * 1024) cudaFuncSetAttribute(pick_x(a, sym), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        pick_x(a, sym)<<<dim3(16, count), threads, smem, c->stream>>>(A);
     }
     return check_launch(c, "encode_fused");
 }

@@ -60,6 +60,7 @@ struct hann_ctx {
     // ModDown lifts of a single item; hann_rotate_sum raises it to 320 for levels of one or two blocks, whose launches
     // otherwise leave most of the machine idle
     int lift_split_ctas = 160;
+    int encode_sym = 1;  // encode_candidates computes half of every transform and mirrors it (real slot vectors)
     // statistics
     hann_stats stats = {};
     int timing = 0;
@@ -117,6 +118,8 @@ int check_launch(hann_ctx* c, const char* what);
 int launch_ntt_fwd(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
 int launch_ntt_inv(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
 int launch_ntt_fwd_pass_b(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
+bool ntt_fwd_mirror_available(const hann_ctx* c, const void* data, int64_t stride);
+int launch_ntt_fwd_pass_b_mirror(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
 int launch_ntt_inv_pass_b(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
 bool ntt_inv_pass_b_gathers(const hann_ctx* c, const void* src, const void* dst);
 int launch_ntt_inv_pass_b_from(hann_ctx* c, const u64* src, int64_t src_gstride, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
@@ -126,7 +129,7 @@ int launch_ks_lift(hann_ctx* c, u64* src, int64_t src_stride, int64_t nsrc, cons
 // encode a block and run pass A of the transforms in one kernel when the parameters allow it (returns false if not)
 bool encode_fused_available(const hann_ctx* c);
 int launch_encode_rows_fused(hann_ctx* c, const float* rows, int64_t rows_in_block, int dim, int p_first, int count, u64* pt_block,
-                             void* ws);
+                             void* ws, bool sym = false);
 LimbMap limbmap_q(const hann_ctx* c);   // period L: limbs 0..L-1
 LimbMap limbmap_qp(const hann_ctx* c);  // period L+1: limbs 0..L
 LimbMap limbmap_single(int limb);

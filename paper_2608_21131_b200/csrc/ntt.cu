@@ -58,6 +58,9 @@ struct NttArgs {
     const u64* src;
     long long src_gstride;
     u64 pos4, limb4;  // 4-bit fields: position within the period and limb of selection k (at most 16 selections)
+    // forward pass B (bulk-copy kernel) of polynomials that are fixed by X -> 1/X: only the first half of the chunks is
+    // transformed (the grid covers that half) and every result is also written to its mirrored position N - 1 - t
+    int mirror;
 };
 
 struct Sel {
@@ -336,8 +339,19 @@ __device__ __forceinline__ void fwd_b8t_body(const NttArgs& A, int groups, int* 
         for (int e = 0; e < 16; e++) x[e] = ar.from_mid(sb[16 * j + (e ^ j)]);
         fwd_round_f<4, AR, 1>(ar, x, [=](int u, int il) { return tcc[(((1 << u) + il) << 4) + j]; });
         u64* go = gbase + (long long)i * ystep * tile_stride + ((size_t)ch << 8);
+        if (A.mirror) {
+            // word 16 e + j of chunk c has its twin at word 16 (15 - e) + (15 - j) of chunk (N >> 8) - 1 - c
+            u64* gm = go + ((((long long)1 << (A.logN - 8)) - 1 - 2 * (chunk0 + ch)) << 8);
 #pragma unroll
-        for (int e = 0; e < 16; e++) go[16 * e + j] = ar.to_canonical(x[e]);
+            for (int e = 0; e < 16; e++) {
+                const u64 v = ar.to_canonical(x[e]);
+                go[16 * e + j] = v;
+                gm[16 * (15 - e) + (15 - j)] = v;
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < 16; e++) go[16 * e + j] = ar.to_canonical(x[e]);
+        }
         // order this warp's shared-memory accesses before the asynchronous copy that refills the buffer
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
@@ -793,7 +807,7 @@ void launch_fwd_class(hann_ctx* c, const NttArgs& A, int groups, bool skip_a, bo
     KProf kp(c, KC_NTT_FWD_B);
     if (b8t_eligible(c, A)) {
         cudaFuncSetAttribute(k_ntt_fwd_b8t<AR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kB8tSmem);
-        const int ranges = (c->N >> 8) / kTK, ntiles = (groups + kTP - 1) / kTP;
+        const int ranges = ((c->N >> 8) / kTK) >> (A.mirror ? 1 : 0), ntiles = (groups + kTP - 1) / kTP;
         k_ntt_fwd_b8t<AR><<<dim3(ranges, A.nsel, b8t_zsplit(ranges * A.nsel, ntiles)), 256, kB8tSmem, c->stream>>>(A, groups, c->kflag);
         return;
     }
@@ -854,7 +868,7 @@ void launch_inv_class(hann_ctx* c, const NttArgs& A, int groups, bool skip_a) {
 // npoly polynomials, `stride` words apart, polynomial p using modulus lm.limb[p % lm.period]; npoly must be a multiple of
 // the period.  One set of launches per arithmetic class present in the period.
 int launch_ntt(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm, bool inverse, bool skip_a = false,
-               const u64* src = nullptr, int64_t src_gstride = 0) {
+               const u64* src = nullptr, int64_t src_gstride = 0, bool mirror = false) {
     if (npoly <= 0) return HANN_OK;
     if (npoly % lm.period) {
         c->err = "transform batch is not a whole number of limb periods";
@@ -873,6 +887,15 @@ int launch_ntt(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const Limb
     A.src = src;
     A.src_gstride = src_gstride;
     A.period = lm.period;
+    A.mirror = mirror ? 1 : 0;
+    if (mirror) {
+        bool ok = !inverse && skip_a && ntt_fwd_mirror_available(c, data, stride);
+        for (int i = 0; i < lm.period; i++) ok = ok && arith_class(c->mod[(int)lm.limb[i]], false) == 0;
+        if (!ok) {
+            c->err = "mirrored forward pass B needs the bulk-copy kernel and moduli below 2^50";
+            return HANN_EINVAL;
+        }
+    }
     if (src && !(inverse && skip_a && A.b == 8 && A.a > 0 && A.tau && ((c->N >> 8) % kTK) == 0 && (((uintptr_t)data | (uintptr_t)src) & 15) == 0 &&
                  ((stride | src_gstride) & 1) == 0)) {
         c->err = "inverse pass B with a separate source needs the bulk-copy kernel (ring of 2^10 or more, 16-byte aligned buffers)";
@@ -958,6 +981,21 @@ int launch_ntt_fwd(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const 
 // the limb's pass-A output format
 int launch_ntt_fwd_pass_b(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm) {
     return launch_ntt(c, data, npoly, stride, lm, false, true);
+}
+
+// The same for polynomials fixed by X -> 1/X (encodings of real slot vectors), whose values at psi^(2t+1) and at its
+// inverse coincide: pass A left rows 2^(a-1) .. 2^a - 1 untouched, pass B transforms the first half of the chunks and
+// writes every value to position t and to position N - 1 - t.
+bool ntt_fwd_mirror_available(const hann_ctx* c, const void* data, int64_t stride) {
+#ifndef HANN_NO_B8T
+    return c->logN >= 10 && c->ntt_tau && ((c->N >> 8) % (2 * kTK)) == 0 && ((uintptr_t)data & 15) == 0 && (stride & 1) == 0;
+#else
+    (void)c; (void)data; (void)stride;
+    return false;
+#endif
+}
+int launch_ntt_fwd_pass_b_mirror(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm) {
+    return launch_ntt(c, data, npoly, stride, lm, false, true, nullptr, 0, true);
 }
 
 int launch_ntt_inv(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm) {

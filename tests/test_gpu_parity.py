@@ -269,6 +269,28 @@ def test_encode_into_buffer_that_is_only_word_aligned():
     assert torch.equal(aligned, shifted)
 
 
+@pytest.mark.parametrize("logN,R,B,L,big", [(10, 16, 4, 2, False), (12, 32, 8, 2, False), (13, 64, 8, 4, True), (16, 128, 32, 4, True)])
+def test_encode_symmetry_shortcut_gives_the_same_words(logN, R, B, L, big):
+    """The encoder transforms only half of every plaintext and mirrors the rest (an encoding of real slots is fixed by
+    X -> 1/X); with the shortcut switched off it computes every transform in full.  Same words, and they are the
+    mirror images the shortcut relies on."""
+    import torch
+
+    ps = synth.small_params(logN, R, B, L=L, big=big)
+    p = Pair(ps, key_seed=6)
+    g, b = p.g, p.b
+    rows = torch.from_numpy(synth.toy_corpus(11, rows=ps.n + 3 if logN < 16 else 1000, dim=R - 1)).to(g.device)
+    nbytes = g.n_blocks(rows.shape[0]) * g.sizeof(b.SIZE_PT_BLOCK)
+    short = g.encode_candidates(rows, p.ws, g.alloc(nbytes))
+    g.set_tuning(b.TUNE_ENCODE_SYMMETRY, 0)
+    full = g.encode_candidates(rows, p.ws, g.alloc(nbytes))
+    g.set_tuning(b.TUNE_ENCODE_SYMMETRY, 1)
+    g.sync()
+    assert torch.equal(short, full)
+    words = full.view(torch.int64).reshape(-1, ps.N)
+    assert torch.equal(words, words.flip(1))
+
+
 @pytest.mark.parametrize(
     "logN,L,big,n_rows",
     [

@@ -130,6 +130,24 @@ def test_encode_equals_exact_cosine_sum(logN):
     assert sum(int(m[k]) != want[k] for k in range(ps.N)) == 0
 
 
+@pytest.mark.parametrize("logN,big", [(4, False), (8, False), (10, True)])
+def test_encoding_of_real_slots_is_fixed_by_conjugation(logN, big):
+    """cos(pi g (N - k) / N) = -cos(pi g k / N) for odd g, so the cosine sum gives m_{N-k} = -m_k (and m_n = 0): the
+    encoding is fixed by X -> 1/X = -X^(N-1).  The pinned binary64 evaluation keeps this to the last bit, and the
+    transform therefore takes the same value at psi^(2t+1) and at its inverse psi^(2(N-1-t)+1)."""
+    ps = synth.small_params(logN, 1, 1, big=big)
+    o = make(ps)
+    z = synth.gaussian(3, logN, np.arange(ps.n)) * 3.0
+    m = o.encode(z, 25)
+    assert m[ps.n] == 0
+    assert np.array_equal(m[1:][::-1], -m[1:])
+    for limb in range(ps.L):
+        q = o.mods[limb]
+        res = np.array([int(v) % q for v in m], dtype=np.uint64)
+        ah = o.ntt(limb, res)
+        assert np.array_equal(ah, ah[::-1])
+
+
 def test_encode_known_answer_n8():
     # N = 8, Delta = 2^10, z = (1/4, 1/2, 3/4, 1): m_0 = (Delta/n) * sum z = 256 * 2.5 = 640; the other
     # coefficients are (Delta/n) sum_j z_j cos(pi g_j k/8) with g = (1, 5, 9, 13), e.g.

@@ -72,7 +72,9 @@ enum {
     HANN_SIZE_POLY = 1,     /* one polynomial of L limbs: L*N*8                                          */
     HANN_SIZE_CT = 2,       /* one ciphertext: 2*L*N*8                                                    */
     HANN_SIZE_BABY = 3,     /* the B rotated query ciphertexts                                            */
-    HANN_SIZE_PT_BLOCK = 4, /* encoded candidates of one block of n rows: R*L*N*8 (= 16*L*R bytes a row) */
+    HANN_SIZE_PT_BLOCK = 4, /* encoded candidates of one block of n rows: R*L*(N/2)*8 (= 8*L*R bytes a row): the encoding
+                             * of a real slot vector is fixed by X -> 1/X, so the second half of its transform is the
+                             * mirror image of the first and is neither computed nor stored */
     HANN_SIZE_INNER = 5,    /* the G partial-sum ciphertexts of one block                                 */
     HANN_SIZE_EVK = 6,      /* one evaluation key in canonical layout: L*2*(L+1)*N*8                      */
     HANN_SIZE_ROWS_PER_BLOCK = 7, /* n                                                                    */
@@ -197,7 +199,7 @@ int hann_query_prepare(hann_ctx *ctx, const void *ct_dev, void *baby_dev, void *
  * (rows are zero-padded to R).  Block blk holds rows blk*n .. blk*n+n-1 (missing rows are zero).  For g < G,
  * b < B plaintext (g,b) of a block encodes the slot vector z[i] = M[(i - g*B) mod n][(i + b) mod R] at scale
  * Delta, reduced into every ciphertext prime and transformed.
- *   pt_dev  ceil(n_rows/n) * HANN_SIZE_PT_BLOCK bytes (device), internal layout [blk][G][B][L][N] */
+ *   pt_dev  ceil(n_rows/n) * HANN_SIZE_PT_BLOCK bytes (device), internal layout [blk][G][B][L][N/2] */
 int hann_encode_candidates(hann_ctx *ctx, const float *rows_dev, int64_t n_rows, int dim, void *pt_dev, void *ws, size_t ws_bytes);
 
 /* Multiply-accumulate of one level: inner[blk][g] = sum_b pt[blk][g][b] * baby[b] (both ciphertext components,
@@ -260,7 +262,10 @@ int64_t hann_static_scratch_bytes(void);
 int hann_keyswitch_static(hann_ctx *ctx, int rot, const void *poly_dev, void *ks0_dev, void *ks1_dev);
 
 /* Convert `count` elements between the canonical layout (host or device pointer) and the internal device layout.
- * kind POLY / PT: one polynomial of L limbs per element; CT: two. */
+ * kind POLY / PT: one polynomial of L limbs per element; CT: two.  The canonical form of every kind is [L][N] words per
+ * polynomial; the internal form of POLY and CT has the same size, that of PT half of it (HANN_SIZE_PT_BLOCK / R per
+ * plaintext), and hann_import of kind PT expects the encoding of a real slot vector (it keeps the first half of the
+ * transform). */
 int hann_import(hann_ctx *ctx, int kind, const uint64_t *canonical, int64_t count, void *internal_dev);
 int hann_export(hann_ctx *ctx, int kind, const void *internal_dev, int64_t count, uint64_t *canonical_out);
 

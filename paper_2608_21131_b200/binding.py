@@ -277,6 +277,8 @@ class Context:
         if isinstance(canonical, np.ndarray):
             canonical = _np(canonical, np.uint64)
         per = self.sizeof(SIZE_CT if kind == KIND_CT else SIZE_POLY)
+        if kind == KIND_PT:
+            per //= 2  # stored plaintexts keep half of every transform
         out = self.alloc(per * count)
         self._ck(self.lib.hann_import(self.h, kind, _ptr(canonical), count, _ptr(out)))
         return out

@@ -357,7 +357,7 @@ extern "C" int64_t hann_sizeof(const hann_ctx* c, int what) {
         case HANN_SIZE_POLY: return L * N * 8;
         case HANN_SIZE_CT: return 2 * L * N * 8;
         case HANN_SIZE_BABY: return (int64_t)c->B * 2 * L * N * 8;
-        case HANN_SIZE_PT_BLOCK: return (int64_t)c->R * L * N * 8;
+        case HANN_SIZE_PT_BLOCK: return (int64_t)c->R * L * (N / 2) * 8;
         case HANN_SIZE_INNER: return (int64_t)c->G * 2 * L * N * 8;
         case HANN_SIZE_EVK: return L * 2 * (L + 1) * N * 8;
         case HANN_SIZE_ROWS_PER_BLOCK: return c->n;
@@ -485,6 +485,19 @@ extern "C" int hann_import(hann_ctx* c, int kind, const uint64_t* canonical, int
     const int pk = polys_of_kind(kind);
     if (!pk || !canonical || !internal_dev || count < 0) return fail(c, HANN_EINVAL, "hann_import: bad argument");
     DeviceGuard dg(c->device);
+    if (kind == HANN_KIND_PT) {
+        // transformed in full in the scratch, first halves kept (a plaintext is the encoding of a real slot vector)
+        const int64_t piece = 64, LN = (int64_t)c->L * c->N;
+        RET(ensure_scratch(c, piece * LN * 8));
+        for (int64_t p0 = 0; p0 < count; p0 += piece) {
+            const int64_t np = std::min(piece, count - p0);
+            RET(import_polys(c, canonical + p0 * LN, np, (u64*)c->scratch));
+            CK(cudaMemcpy2DAsync((u64*)internal_dev + p0 * (LN / 2), (size_t)c->n * 8, c->scratch, (size_t)c->N * 8, (size_t)c->n * 8,
+                                 (size_t)np * c->L, cudaMemcpyDeviceToDevice, c->stream));
+        }
+        CK(cudaStreamSynchronize(c->stream));
+        return HANN_OK;
+    }
     RET(import_polys(c, canonical, count * pk, (u64*)internal_dev));
     CK(cudaStreamSynchronize(c->stream));
     return HANN_OK;
@@ -523,6 +536,13 @@ extern "C" int hann_export(hann_ctx* c, int kind, const void* internal_dev, int6
     RET(ensure_scratch(c, piece * c->L * c->N * 8));
     for (int64_t p0 = 0; p0 < total; p0 += piece) {
         const int64_t np = std::min(piece, total - p0);
+        if (kind == HANN_KIND_PT) {
+            const int64_t LN = (int64_t)c->L * c->N;
+            RET(launch_unpack_half(c, (const u64*)internal_dev + p0 * (LN / 2), np * c->L, (u64*)c->scratch));
+            RET(launch_ntt_inv(c, (u64*)c->scratch, np * c->L, c->N, limbmap_q(c)));
+            CK(cudaMemcpyAsync(canonical_out + p0 * LN, c->scratch, np * LN * 8, cudaMemcpyDefault, c->stream));
+            continue;
+        }
         RET(export_polys(c, (const u64*)internal_dev + p0 * c->L * c->N, np, (u64*)c->scratch, canonical_out + p0 * c->L * c->N));
     }
     CK(cudaStreamSynchronize(c->stream));
@@ -705,7 +725,7 @@ extern "C" int hann_encrypt_block(hann_ctx* c, const int8_t* s, const void* pt_d
         }
         RET(launch_ntt_fwd(c, EH, (int64_t)np * L, N, limbmap_q(c)));
         // c0 = pt - a*s + e, written at ct + 2 r * LN (the finish kernel strides its output by 2 * LN)
-        RET(launch_encrypt_block_finish(c, pt + (int64_t)r0 * LN, AS, EH, ct + (int64_t)r0 * 2 * LN, np));
+        RET(launch_encrypt_block_finish(c, pt + (int64_t)r0 * (LN / 2), AS, EH, ct + (int64_t)r0 * 2 * LN, np));
         CK(cudaStreamSynchronize(c->stream));  // e8 is reused by the next piece
     }
     return HANN_OK;
@@ -883,23 +903,37 @@ extern "C" int hann_encode_candidates(hann_ctx* c, const float* rows_dev, int64_
     if ((int64_t)ws_bytes < encode_ws_bytes(c)) return fail(c, HANN_EWORKSPACE, "hann_encode_candidates: workspace too small");
     DeviceGuard dg(c->device);
     Timer tm(c, 1);
-    const int64_t n = c->n, nblk = (n_rows + n - 1) / n, ptw = (int64_t)c->R * c->L * c->N;
+    // a stored plaintext is the first N/2 values of each limb's transform (the rest is their mirror image)
+    const int64_t n = c->n, nblk = (n_rows + n - 1) / n, Ln = (int64_t)c->L * n, ptw = (int64_t)c->R * Ln;
+    const bool fused = encode_fused_available(c);
     for (int64_t blk = 0; blk < nblk; blk++) {
         const int64_t rows_here = std::min(n, n_rows - blk * n);
+        const float* rows = rows_dev + blk * n * dim;
         u64* pt = (u64*)pt_dev + blk * ptw;
         // a few plaintexts at a time: FFT buffer and residues of a group are re-read from L2, not from HBM
         for (int p0 = 0; p0 < c->R; p0 += c->encode_group) {
             const int cnt = std::min(c->encode_group, c->R - p0);
-            if (encode_fused_available(c)) {
-                // real slot vectors: the transform of an encoding takes every value twice (at a root and at its inverse)
-                u64* polys = pt + (int64_t)p0 * c->L * c->N;
-                const bool sym = c->encode_sym && ntt_fwd_mirror_available(c, polys, c->N);
-                RET(launch_encode_rows_fused(c, rows_dev + blk * n * dim, rows_here, dim, p0, cnt, pt, ws, sym));
-                if (sym) RET(launch_ntt_fwd_pass_b_mirror(c, polys, (int64_t)cnt * c->L, c->N, limbmap_q(c)));
-                else RET(launch_ntt_fwd_pass_b(c, polys, (int64_t)cnt * c->L, c->N, limbmap_q(c)));
-            } else {
-                RET(launch_encode_rows(c, rows_dev + blk * n * dim, rows_here, dim, p0, cnt, pt, ws));
-                RET(launch_ntt_fwd(c, pt + (int64_t)p0 * c->L * c->N, (int64_t)cnt * c->L, c->N, limbmap_q(c)));
+            u64* polys = pt + (int64_t)p0 * Ln;
+            if (fused && c->encode_sym && ntt_fwd_half_available(c, polys, n)) {
+                // half of every transform is computed, straight into place
+                RET(launch_encode_rows_fused(c, rows, rows_here, dim, p0, cnt, polys, n, ws, true));
+                RET(launch_ntt_fwd_pass_b_half(c, polys, (int64_t)cnt * c->L, n, limbmap_q(c)));
+                continue;
+            }
+            // full transforms of a few plaintexts at a time in the staging area, first halves copied into place
+            u64* stage = (u64*)((char*)ws + encode_fft_bytes(c));
+            const int sg = encode_stage_group(c);
+            for (int s0 = 0; s0 < cnt; s0 += sg) {
+                const int sn = std::min(sg, cnt - s0);
+                if (fused) {
+                    RET(launch_encode_rows_fused(c, rows, rows_here, dim, p0 + s0, sn, stage, c->N, ws, false));
+                    RET(launch_ntt_fwd_pass_b(c, stage, (int64_t)sn * c->L, c->N, limbmap_q(c)));
+                } else {
+                    RET(launch_encode_rows(c, rows, rows_here, dim, p0 + s0, sn, stage, ws));
+                    RET(launch_ntt_fwd(c, stage, (int64_t)sn * c->L, c->N, limbmap_q(c)));
+                }
+                CK(cudaMemcpy2DAsync(polys + (int64_t)s0 * Ln, (size_t)n * 8, stage, (size_t)c->N * 8, (size_t)n * 8, (size_t)sn * c->L,
+                                     cudaMemcpyDeviceToDevice, c->stream));
             }
         }
     }

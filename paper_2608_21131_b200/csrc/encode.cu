@@ -29,7 +29,7 @@ struct EncArgs {
     int logn, b1, K1, C1;
     double scale;  // Delta / n
     double2* buf;  // [P][n], indexed by blockIdx.y
-    u64* out;      // [..][L][N] coefficient-domain residues, indexed by p_first + blockIdx.y
+    u64* out;      // [P][L][N] coefficient-domain residues of the launch's plaintexts, indexed by blockIdx.y
     int L;
     int p_first;   // index (g*B + b) of the first plaintext of this launch
 };
@@ -101,7 +101,7 @@ __global__ void __launch_bounds__(kThreads) k_fft_b(EncArgs A, LimbTable lt) {
         }
         __syncthreads();
     }
-    u64* out = A.out + (long long)(A.p_first + P) * A.L * N;
+    u64* out = A.out + (long long)P * A.L * N;
     for (int idx = threadIdx.x; idx < rows * C1; idx += kThreads) {
         const int k = (idx / C1) * S1 + c0 + (idx % C1);
         double2 cc = cmul_rn(smc[idx], A.U[k]);
@@ -141,14 +141,21 @@ int run_encode(hann_ctx* c, EncArgs& A, int P) {
 
 }  // namespace
 
-int64_t encode_ws_bytes(const hann_ctx* c) {
+// FFT buffer of one launch group, then the staging area of encode_stage_group() full-size plaintexts (used when the
+// half-size transform does not apply: small rings, moduli of 2^50 and more, buffers that are only 8-byte aligned)
+int64_t encode_fft_bytes(const hann_ctx* c) {
     const int group = c->encode_group < c->R ? c->encode_group : c->R;
-    return (int64_t)group * c->n * (int64_t)sizeof(double2);
+    return ((int64_t)group * c->n * (int64_t)sizeof(double2) + 255) / 256 * 256;
 }
+int encode_stage_group(const hann_ctx* c) {
+    const int group = c->encode_group < c->R ? c->encode_group : c->R;
+    return group < 8 ? group : 8;
+}
+int64_t encode_ws_bytes(const hann_ctx* c) { return encode_fft_bytes(c) + (int64_t)encode_stage_group(c) * c->L * c->N * 8; }
 
-// plaintexts p_first .. p_first+count-1 of one block of candidate rows -> pt_block[p][L][N], coefficient domain (the
+// plaintexts p_first .. p_first+count-1 of one block of candidate rows -> out[count][L][N], coefficient domain (the
 // caller transforms them); ws holds count complex vectors of n points
-int launch_encode_rows(hann_ctx* c, const float* rows, int64_t rows_in_block, int dim, int p_first, int count, u64* pt_block,
+int launch_encode_rows(hann_ctx* c, const float* rows, int64_t rows_in_block, int dim, int p_first, int count, u64* out,
                        void* ws) {
     EncArgs A = {};
     A.rows = rows;
@@ -156,7 +163,7 @@ int launch_encode_rows(hann_ctx* c, const float* rows, int64_t rows_in_block, in
     A.dim = dim;
     A.z = nullptr;
     A.buf = (double2*)ws;
-    A.out = pt_block;
+    A.out = out;
     A.p_first = p_first;
     return run_encode(c, A, count);
 }
@@ -196,7 +203,8 @@ struct FusedArgs {
     int logn, L;
     double scale;
     double2* buf;        // [count][n]
-    u64* out;            // [..][L][N]
+    u64* out;            // limb polynomial l of the launch's plaintext P starts at out + (P * L + l) * out_stride
+    long long out_stride;
     const double2* tw;   // forward transform twiddles, binary64 format, [L+1][N]
     const LimbConst* lt;
 };
@@ -337,7 +345,8 @@ __global__ void __launch_bounds__(128, 5) k_fft_w8(FusedArgs A) {
 #endif
 // SYM: the encoding of a real slot vector is fixed by X -> 1/X, so its transform takes the same value at psi^(2t+1) and
 // at the inverse of that root.  After the first stage (which splits modulo X^n - i and X^n + i) only the first half
-// carries on; rows 2^(a-1) .. 2^a - 1 of the pass-A output are not produced, and pass B mirrors its results.
+// carries on; rows 2^(a-1) .. 2^a - 1 of the pass-A output are not produced (out_stride may then be N/2), and pass B
+// transforms the first half of the chunks only.
 template <int R1, int R2, bool SYM>
 __global__ void __launch_bounds__(256, HANN_X_MINBLOCKS) k_encode_x(FusedArgs A) {
     extern __shared__ u64 smx[];
@@ -345,7 +354,7 @@ __global__ void __launch_bounds__(256, HANN_X_MINBLOCKS) k_encode_x(FusedArgs A)
     constexpr int G1 = 1 << R2;        // row groups of transform round 1 = threads per column
     constexpr int HF = 1 << (R1 - 1);  // complex words a thread holds after the FFT's last round
     constexpr int rows_fft = 1 << (a - 1);
-    const int n = 1 << A.logn, N = 2 * n;
+    const int n = 1 << A.logn;
     const int P = blockIdx.y;
     const int c0 = blockIdx.x << 4;
     const double2* in = A.buf + (long long)P * n + c0;
@@ -412,7 +421,7 @@ __global__ void __launch_bounds__(256, HANN_X_MINBLOCKS) k_encode_x(FusedArgs A)
     for (int l = 0; l < A.L; l++) {
         const ArithF64 ar(A.lt + l);
         const double2* tw = twc + l * NT;
-        u64* base = A.out + ((long long)(A.p_first + P) * A.L + l) * N + c0;
+        u64* base = A.out + ((long long)P * A.L + l) * A.out_stride + c0;
         __syncthreads();  // the twiddle cache is filled (first limb) / the exchange tile is free again
         if (active && SYM) {
             constexpr int RS = R1 > 1 ? R1 - 1 : 1;
@@ -477,11 +486,11 @@ bool encode_fused_available(const hann_ctx* c) {
     return true;
 }
 
-// plaintexts p_first .. p_first+count-1 of one block: encode and run pass A of their forward transforms; the caller
-// finishes with launch_ntt_fwd_pass_b over the same polynomials
-// (sym: leave the second half of the pass-A rows out; the caller then finishes with launch_ntt_fwd_pass_b_mirror)
-int launch_encode_rows_fused(hann_ctx* c, const float* rows, int64_t rows_in_block, int dim, int p_first, int count, u64* pt_block,
-                             void* ws, bool sym) {
+// plaintexts p_first .. p_first+count-1 of one block: encode and run pass A of their forward transforms into
+// out[count][L][out_stride]; the caller finishes with launch_ntt_fwd_pass_b over the same polynomials.
+// sym: leave the second half of the pass-A rows out (out_stride >= N/2); the caller finishes with launch_ntt_fwd_pass_b_half.
+int launch_encode_rows_fused(hann_ctx* c, const float* rows, int64_t rows_in_block, int dim, int p_first, int count, u64* out,
+                             int64_t out_stride, void* ws, bool sym) {
     FusedArgs A;
     A.rows = rows;
     A.rows_in_block = rows_in_block;
@@ -496,7 +505,8 @@ int launch_encode_rows_fused(hann_ctx* c, const float* rows, int64_t rows_in_blo
     A.L = c->L;
     A.scale = ldexp(1.0, c->prm.log_scale - A.logn);
     A.buf = (double2*)ws;
-    A.out = pt_block;
+    A.out = out;
+    A.out_stride = out_stride;
     A.tw = (const double2*)c->tw_fwd_f64;
     A.lt = c->lt_dev;
     const int n = c->n, a = c->logN - 8;

@@ -118,8 +118,9 @@ int check_launch(hann_ctx* c, const char* what);
 int launch_ntt_fwd(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
 int launch_ntt_inv(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
 int launch_ntt_fwd_pass_b(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
-bool ntt_fwd_mirror_available(const hann_ctx* c, const void* data, int64_t stride);
-int launch_ntt_fwd_pass_b_mirror(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
+bool ntt_fwd_half_available(const hann_ctx* c, const void* data, int64_t stride);
+int launch_ntt_fwd_pass_b_half(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
+int launch_unpack_half(hann_ctx* c, const u64* half, int64_t npoly, u64* full);
 int launch_ntt_inv_pass_b(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
 bool ntt_inv_pass_b_gathers(const hann_ctx* c, const void* src, const void* dst);
 int launch_ntt_inv_pass_b_from(hann_ctx* c, const u64* src, int64_t src_gstride, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
@@ -128,8 +129,8 @@ int launch_wait_selftest(hann_ctx* c, unsigned long long limit_ns, unsigned long
 int launch_ks_lift(hann_ctx* c, u64* src, int64_t src_stride, int64_t nsrc, const LimbMap& src_lm, u64* dst, int n_tgt, int tgt_limb0);
 // encode a block and run pass A of the transforms in one kernel when the parameters allow it (returns false if not)
 bool encode_fused_available(const hann_ctx* c);
-int launch_encode_rows_fused(hann_ctx* c, const float* rows, int64_t rows_in_block, int dim, int p_first, int count, u64* pt_block,
-                             void* ws, bool sym = false);
+int launch_encode_rows_fused(hann_ctx* c, const float* rows, int64_t rows_in_block, int dim, int p_first, int count, u64* out,
+                             int64_t out_stride, void* ws, bool sym);
 LimbMap limbmap_q(const hann_ctx* c);   // period L: limbs 0..L-1
 LimbMap limbmap_qp(const hann_ctx* c);  // period L+1: limbs 0..L
 LimbMap limbmap_single(int limb);
@@ -139,6 +140,8 @@ int launch_encode_rows(hann_ctx* c, const float* rows, int64_t rows_in_block, in
                        void* ws);
 int launch_encode_slots(hann_ctx* c, const double* z_dev, u64* poly_out, void* ws);
 int64_t encode_ws_bytes(const hann_ctx* c);
+int64_t encode_fft_bytes(const hann_ctx* c);
+int encode_stage_group(const hann_ctx* c);
 
 // scoring
 int launch_mac(hann_ctx* c, const u64* baby, const u64* pt, int64_t n_blocks, u64* inner);

@@ -350,7 +350,8 @@ __global__ void __launch_bounds__(kThreads) k_rlk_finish(const u64* __restrict__
     }
 }
 
-// block encryption finish, transform domain: c0[r][l][t] = pt[r][l][t] - as[r][l][t] + ehat[r][l][t]
+// block encryption finish, transform domain: c0[r][l][t] = pt[r][l][t] - as[r][l][t] + ehat[r][l][t]; pt in its stored
+// form [r][l][N/2] (position t >= N/2 is the mirror image of position N - 1 - t)
 __global__ void __launch_bounds__(kThreads) k_encrypt_block_finish(const u64* __restrict__ pt, const u64* __restrict__ as,
                                                                    const u64* __restrict__ ehat, u64* __restrict__ ct, int N, int L,
                                                                    long long npt, LimbTable lt) {
@@ -358,7 +359,9 @@ __global__ void __launch_bounds__(kThreads) k_encrypt_block_finish(const u64* __
     for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
         const long long r = idx / LN, rem = idx % LN;
         const u64 q = lt.c[(int)(rem / N)].q;
-        ct[r * 2 * LN + rem] = addmod(submod(pt[idx], as[idx], q), ehat[idx], q);
+        const int l = (int)(rem / N), t = (int)(rem % N), n = N >> 1;
+        const u64 m = pt[(r * L + l) * n + (t < n ? t : N - 1 - t)];
+        ct[r * 2 * LN + rem] = addmod(submod(m, as[idx], q), ehat[idx], q);
     }
 }
 

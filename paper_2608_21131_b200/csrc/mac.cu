@@ -1,6 +1,8 @@
 // Multiply-accumulate kernels: ciphertext x plaintext (the hot path's inner loop, Sec. 3.4), its paired form for two
-// queries, and ciphertext x ciphertext for an encrypted database.  All polynomials are [.][limb][N] arrays of 64-bit
-// residues in [0, q), in the transform domain.
+// queries, and ciphertext x ciphertext for an encrypted database.  Ciphertext polynomials are [.][limb][N] arrays of 64-bit
+// residues in [0, q), in the transform domain.  A PLAINTEXT is stored as [limb][N/2]: the encoding of a real slot vector
+// is fixed by X -> 1/X, so position t and position N - 1 - t of its transform hold the same value, and every stored word
+// serves both positions (a thread multiplies it with the baby-step words of both and produces both outputs).
 #include <cuda.h>
 
 #include "internal.h"
@@ -20,14 +22,16 @@ __global__ void __launch_bounds__(kThreads) k_mac(const u64* __restrict__ baby, 
                                                   u64* __restrict__ inner, int N, int L, int B, int G,
                                                   long long n_bg, LimbTable lt) {
     const long long LN = (long long)L * N;
+    const int n = N >> 1;
+    const long long Ln = (long long)L * n;
     for (long long pos = (long long)blockIdx.x * kThreads + threadIdx.x; pos < LN; pos += (long long)gridDim.x * kThreads) {
-        const int l = (int)(pos / N);
+        const int l = (int)(pos / N), t = (int)(pos % N);
         const LimbConst& lc = lt.c[l];
         for (long long bg = blockIdx.y; bg < n_bg; bg += gridDim.y) {
-            const u64* p = pt + bg * B * LN + pos;
+            const u64* p = pt + bg * B * Ln + (long long)l * n + (t < n ? t : N - 1 - t);
             u64 h0 = 0, l0 = 0, h1 = 0, l1 = 0;
             for (int b = 0; b < B; b++) {
-                u64 v = __ldcs(p + (long long)b * LN);
+                u64 v = p[(long long)b * Ln];
                 mac128(h0, l0, v, baby[((long long)b * 2 + 0) * LN + pos]);
                 mac128(h1, l1, v, baby[((long long)b * 2 + 1) * LN + pos]);
             }
@@ -58,71 +62,75 @@ __global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ 
                                                         long long inner_stride, int N, int L, long long n_bg, int bg_per_cta,
                                                         const LimbConst* __restrict__ lt) {
     constexpr int B = NG * BB;
-    __shared__ u64 part[2][NG][6 * NQ][32];
-    const long long LN = (long long)L * N;
-    const long long pos0 = (long long)blockIdx.x * 32;
+    constexpr int NV = 2 * NQ;  // (query, side): side 0 is position t, side 1 its mirror image N - 1 - t
+    __shared__ u64 part[2][NG][3 * 2 * NV][32];
+    const int n = N >> 1;
+    const long long LN = (long long)L * N, Ln = (long long)L * n;
+    const long long hpos0 = (long long)blockIdx.x * 32;  // in the stored plaintext layout [L][N/2]
     const int lane = threadIdx.x & 31, wg = threadIdx.x >> 5;
-    const LimbConst* lc = lt + pos0 / N;
-    // this warp's baby-step words, split into 25-bit halves: lo half in the low word, hi half in the high word
-    unsigned w0[NQ][BB][2], w1[NQ][BB][2];
+    const int limb = (int)(hpos0 / n), t0 = (int)(hpos0 % n);
+    const LimbConst* lc = lt + limb;
+    const long long posv[2] = {(long long)limb * N + t0 + lane, (long long)limb * N + (N - 1 - t0 - lane)};
+    // this warp's baby-step words, split into 25-bit halves
+    unsigned w0[NV][BB][2], w1[NV][BB][2];
 #pragma unroll
-    for (int q = 0; q < NQ; q++)
+    for (int v = 0; v < NV; v++)
 #pragma unroll
         for (int k = 0; k < BB; k++)
 #pragma unroll
             for (int c = 0; c < 2; c++) {
-                const u64 v = baby[q * baby_stride + ((long long)(wg * BB + k) * 2 + c) * LN + pos0 + lane];
-                w0[q][k][c] = (unsigned)v & kM25;
-                w1[q][k][c] = (unsigned)(v >> 25);
+                const u64 x = baby[(v >> 1) * baby_stride + ((long long)(wg * BB + k) * 2 + c) * LN + posv[v & 1]];
+                w0[v][k][c] = (unsigned)x & kM25;
+                w1[v][k][c] = (unsigned)(x >> 25);
             }
     const long long bg0 = (long long)blockIdx.y * bg_per_cta;
     const long long bg1 = bg0 + bg_per_cta < n_bg ? bg0 + bg_per_cta : n_bg;
     if (bg0 >= bg1) return;
-    const u64* p = pt + (bg0 * B + wg * BB) * LN + pos0 + lane;
+    const u64* p = pt + (bg0 * B + wg * BB) * Ln + hpos0 + lane;
     u64 cur[BB], nxt[BB];
 #pragma unroll
-    for (int k = 0; k < BB; k++) cur[k] = __ldcs(p + (long long)k * LN);
+    for (int k = 0; k < BB; k++) cur[k] = __ldcs(p + (long long)k * Ln);
     for (long long bg = bg0; bg < bg1; bg++) {
         if (bg + 1 < bg1) {
-            const u64* pn = p + (long long)B * LN;
+            const u64* pn = p + (long long)B * Ln;
 #pragma unroll
-            for (int k = 0; k < BB; k++) nxt[k] = __ldcs(pn + (long long)k * LN);
+            for (int k = 0; k < BB; k++) nxt[k] = __ldcs(pn + (long long)k * Ln);
         }
-        u64 p00[NQ][2], p11[NQ][2], pm[NQ][2];
+        u64 p00[NV][2], p11[NV][2], pm[NV][2];
 #pragma unroll
-        for (int q = 0; q < NQ; q++)
+        for (int v = 0; v < NV; v++)
 #pragma unroll
-            for (int c = 0; c < 2; c++) p00[q][c] = p11[q][c] = pm[q][c] = 0;
+            for (int c = 0; c < 2; c++) p00[v][c] = p11[v][c] = pm[v][c] = 0;
 #pragma unroll
         for (int k = 0; k < BB; k++) {
             const unsigned a0 = (unsigned)cur[k] & kM25, a1 = (unsigned)(cur[k] >> 25), as = a0 + a1;
 #pragma unroll
-            for (int q = 0; q < NQ; q++)
+            for (int v = 0; v < NV; v++)
 #pragma unroll
                 for (int c = 0; c < 2; c++) {
-                    p00[q][c] += (u64)a0 * w0[q][k][c];
-                    p11[q][c] += (u64)a1 * w1[q][k][c];
-                    pm[q][c] += (u64)as * (w0[q][k][c] + w1[q][k][c]);
+                    p00[v][c] += (u64)a0 * w0[v][k][c];
+                    p11[v][c] += (u64)a1 * w1[v][k][c];
+                    pm[v][c] += (u64)as * (w0[v][k][c] + w1[v][k][c]);
                 }
         }
-        u64(*buf)[6 * NQ][32] = part[bg & 1];
+        u64(*buf)[3 * 2 * NV][32] = part[bg & 1];
 #pragma unroll
-        for (int q = 0; q < NQ; q++)
+        for (int v = 0; v < NV; v++)
 #pragma unroll
             for (int c = 0; c < 2; c++) {
-                buf[wg][(q * 2 + c) * 3 + 0][lane] = p00[q][c];
-                buf[wg][(q * 2 + c) * 3 + 1][lane] = pm[q][c];
-                buf[wg][(q * 2 + c) * 3 + 2][lane] = p11[q][c];
+                buf[wg][(v * 2 + c) * 3 + 0][lane] = p00[v][c];
+                buf[wg][(v * 2 + c) * 3 + 1][lane] = pm[v][c];
+                buf[wg][(v * 2 + c) * 3 + 2][lane] = p11[v][c];
             }
         __syncthreads();
-        // the warps share out the 2 * NQ (query, component) sums
-        for (int qc = wg; qc < 2 * NQ; qc += NG) {
+        // the warps share out the 2 * NV (query, side, component) sums
+        for (int vc = wg; vc < 2 * NV; vc += NG) {
             u64 s00 = 0, sm = 0, s11 = 0;
 #pragma unroll
             for (int g = 0; g < NG; g++) {
-                s00 += buf[g][qc * 3 + 0][lane];
-                sm += buf[g][qc * 3 + 1][lane];
-                s11 += buf[g][qc * 3 + 2][lane];
+                s00 += buf[g][vc * 3 + 0][lane];
+                sm += buf[g][vc * 3 + 1][lane];
+                s11 += buf[g][vc * 3 + 2][lane];
             }
             // value = s00 + cross * 2^25 + s11 * 2^50 with cross = sm - s00 - s11 < 2^59
             const u64 cross = sm - s00 - s11;
@@ -133,12 +141,13 @@ __global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ 
             const u64 d_lo = s11 << 50, d_hi = s11 >> 14;
             lo += d_lo;
             hi += d_hi + (lo < d_lo ? 1 : 0);
-            inner[(qc >> 1) * inner_stride + (bg * 2 + (qc & 1)) * LN + pos0 + lane] = reduce128(hi, lo, *lc);
+            const int v = vc >> 1;
+            inner[(v >> 1) * inner_stride + (bg * 2 + (vc & 1)) * LN + posv[v & 1]] = reduce128(hi, lo, *lc);
         }
-        if (NG < 2 * NQ) __syncthreads();  // a warp that finishes several sums may still be reading while the next pair is written
+        if (NG < 2 * NV) __syncthreads();  // a warp that finishes several sums may still be reading while the next pair is written
 #pragma unroll
         for (int k = 0; k < BB; k++) cur[k] = nxt[k];
-        p += (long long)B * LN;
+        p += (long long)B * Ln;
     }
 }
 
@@ -239,18 +248,28 @@ __global__ void __launch_bounds__(32 * NG) k_mac_ct_stream(const u64* __restrict
 constexpr int kMacStages = 4;
 
 template <int NG, int BB>
+constexpr size_t mac_bulk_smem() {
+    return (size_t)NG * kMacStages * BB * 256 + (size_t)2 * NG * 12 * 256 + (size_t)NG * kMacStages * 8 + 16;
+}
+
+template <int NG, int BB>
 __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ baby, const __grid_constant__ CUtensorMap pt_map,
                                                       u64* __restrict__ inner, int N, int L, long long n_bg, int bg_per_cta,
                                                       const LimbConst* __restrict__ lt, int* kflag) {
     constexpr int B = NG * BB;
-    __shared__ __align__(128) u64 ring[NG][kMacStages][BB][32];
-    __shared__ u64 part[2][NG][6][32];
-    __shared__ __align__(8) u64 bars[NG][kMacStages];
-    __shared__ int s_abort;
+    extern __shared__ __align__(128) u64 smem_mac[];
+    u64(*ring)[kMacStages][BB][32] = (u64(*)[kMacStages][BB][32])smem_mac;                        // [NG]
+    u64(*part)[NG][12][32] = (u64(*)[NG][12][32])(smem_mac + (size_t)NG * kMacStages * BB * 32);  // [2]
+    u64(*bars)[kMacStages] = (u64(*)[kMacStages])(smem_mac + (size_t)NG * kMacStages * BB * 32 + (size_t)2 * NG * 12 * 32);  // [NG]
+    int& s_abort = *(int*)(&bars[NG][0]);
+    const int n = N >> 1;
     const long long LN = (long long)L * N;
-    const long long pos0 = (long long)blockIdx.x * 32;
+    const long long hpos0 = (long long)blockIdx.x * 32;  // in the stored plaintext layout [L][N/2]
     const int lane = threadIdx.x & 31, wg = threadIdx.x >> 5;
-    const LimbConst* lc = lt + pos0 / N;
+    const int limb = (int)(hpos0 / n), t0 = (int)(hpos0 % n);
+    const LimbConst* lc = lt + limb;
+    // side 0: position t of the limb, side 1: its mirror image N - 1 - t (same plaintext word)
+    const long long posv[2] = {(long long)limb * N + t0 + lane, (long long)limb * N + (N - 1 - t0 - lane)};
     const long long bg0 = (long long)blockIdx.y * bg_per_cta;
     const long long bg1 = bg0 + bg_per_cta < n_bg ? bg0 + bg_per_cta : n_bg;
     if (bg0 >= bg1) return;
@@ -263,19 +282,21 @@ __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ ba
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         for (int i = 0; i < kMacStages && i < npairs; i++) {
             mbar_expect_tx(bar0 + 8 * i, BB * 256);
-            tensor_load_2d(ring0 + i * BB * 256, &pt_map, (int)pos0, row0 + i * B, bar0 + 8 * i);
+            tensor_load_2d(ring0 + i * BB * 256, &pt_map, (int)hpos0, row0 + i * B, bar0 + 8 * i);
         }
     }
-    // this warp's baby-step words, split into 25-bit halves
-    unsigned w0[BB][2], w1[BB][2];
+    // this warp's baby-step words of both sides, split into 25-bit halves
+    unsigned w0[2][BB][2], w1[2][BB][2];
 #pragma unroll
-    for (int k = 0; k < BB; k++)
+    for (int v = 0; v < 2; v++)
 #pragma unroll
-        for (int c = 0; c < 2; c++) {
-            const u64 v = baby[((long long)(wg * BB + k) * 2 + c) * LN + pos0 + lane];
-            w0[k][c] = (unsigned)v & kM25;
-            w1[k][c] = (unsigned)(v >> 25);
-        }
+        for (int k = 0; k < BB; k++)
+#pragma unroll
+            for (int c = 0; c < 2; c++) {
+                const u64 x = baby[((long long)(wg * BB + k) * 2 + c) * LN + posv[v]];
+                w0[v][k][c] = (unsigned)x & kM25;
+                w1[v][k][c] = (unsigned)(x >> 25);
+            }
     __syncthreads();  // s_abort and the barriers are initialised
     for (int i = 0; i < npairs; i++) {
         const int st = i % kMacStages;
@@ -292,39 +313,43 @@ __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ ba
         __syncwarp();
         if (lane == 0 && arrived && i + kMacStages < npairs) {
             mbar_expect_tx(bar0 + 8 * st, BB * 256);
-            tensor_load_2d(ring0 + st * BB * 256, &pt_map, (int)pos0, row0 + (i + kMacStages) * B, bar0 + 8 * st);
+            tensor_load_2d(ring0 + st * BB * 256, &pt_map, (int)hpos0, row0 + (i + kMacStages) * B, bar0 + 8 * st);
         }
-        u64 p00[2] = {0, 0}, p11[2] = {0, 0}, pm[2] = {0, 0};
+        u64 p00[2][2] = {{0, 0}, {0, 0}}, p11[2][2] = {{0, 0}, {0, 0}}, pm[2][2] = {{0, 0}, {0, 0}};
 #pragma unroll
         for (int k = 0; k < BB; k++) {
             const unsigned a0 = (unsigned)cur[k] & kM25, a1 = (unsigned)(cur[k] >> 25), as = a0 + a1;
 #pragma unroll
-            for (int c = 0; c < 2; c++) {
-                p00[c] += (u64)a0 * w0[k][c];
-                p11[c] += (u64)a1 * w1[k][c];
-                pm[c] += (u64)as * (w0[k][c] + w1[k][c]);
-            }
-        }
-        u64(*buf)[6][32] = part[i & 1];
+            for (int v = 0; v < 2; v++)
 #pragma unroll
-        for (int c = 0; c < 2; c++) {
-            buf[wg][c * 3 + 0][lane] = p00[c];
-            buf[wg][c * 3 + 1][lane] = pm[c];
-            buf[wg][c * 3 + 2][lane] = p11[c];
+                for (int c = 0; c < 2; c++) {
+                    p00[v][c] += (u64)a0 * w0[v][k][c];
+                    p11[v][c] += (u64)a1 * w1[v][k][c];
+                    pm[v][c] += (u64)as * (w0[v][k][c] + w1[v][k][c]);
+                }
         }
+        u64(*buf)[12][32] = part[i & 1];
+#pragma unroll
+        for (int v = 0; v < 2; v++)
+#pragma unroll
+            for (int c = 0; c < 2; c++) {
+                buf[wg][(v * 2 + c) * 3 + 0][lane] = p00[v][c];
+                buf[wg][(v * 2 + c) * 3 + 1][lane] = pm[v][c];
+                buf[wg][(v * 2 + c) * 3 + 2][lane] = p11[v][c];
+            }
         __syncthreads();
         if (s_abort) {
             // leave together; first give this warp's copies still in flight the same bounded time
             for (int j = i + 1; j < npairs && j < i + kMacStages; j++) mbar_wait(bar0 + 8 * (j % kMacStages), (unsigned)(j / kMacStages) & 1u);
             return;
         }
-        for (int c = wg; c < 2; c += NG) {
+        for (int vc = wg; vc < 4; vc += NG) {
             u64 s00 = 0, sm = 0, s11 = 0;
 #pragma unroll
             for (int g = 0; g < NG; g++) {
-                s00 += buf[g][c * 3 + 0][lane];
-                sm += buf[g][c * 3 + 1][lane];
-                s11 += buf[g][c * 3 + 2][lane];
+                s00 += buf[g][vc * 3 + 0][lane];
+                sm += buf[g][vc * 3 + 1][lane];
+                s11 += buf[g][vc * 3 + 2][lane];
             }
             const u64 cross = sm - s00 - s11;
             u64 lo = s00, hi = 0;
@@ -334,9 +359,9 @@ __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ ba
             const u64 d_lo = s11 << 50, d_hi = s11 >> 14;
             lo += d_lo;
             hi += d_hi + (lo < d_lo ? 1 : 0);
-            inner[((bg0 + i) * 2 + c) * LN + pos0 + lane] = reduce128(hi, lo, *lc);
+            inner[((bg0 + i) * 2 + (vc & 1)) * LN + posv[vc >> 1]] = reduce128(hi, lo, *lc);
         }
-        if (NG == 1) __syncthreads();
+        if (NG < 4) __syncthreads();
     }
 }
 
@@ -368,12 +393,12 @@ __global__ void __launch_bounds__(kThreads) k_mac_ct(const u64* __restrict__ bab
 
 }  // namespace
 
-// 2-D tiled tensor map over the plaintexts of a level: `rows` rows of LN 64-bit words, boxes of box_rows x 32 words.  The
+// 2-D tiled tensor map over the stored plaintexts of a level: `rows` rows of Ln = L * N/2 64-bit words, boxes of box_rows x 32 words.  The
 // encoder is a driver entry point, looked up once (no link against the driver library); false if it cannot be had.
 typedef CUresult (*TensorMapEncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                            const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                            CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-bool plaintext_map(const u64* pt, long long LN, long long rows, int box_rows, CUtensorMap* out) {
+bool plaintext_map(const u64* pt, long long Ln, long long rows, int box_rows, CUtensorMap* out) {
     static TensorMapEncodeTiledFn encode = [] {
         void* fn = nullptr;
         cudaDriverEntryPointQueryResult res;
@@ -384,8 +409,8 @@ bool plaintext_map(const u64* pt, long long LN, long long rows, int box_rows, CU
         return (TensorMapEncodeTiledFn)fn;
     }();
     if (!encode) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)LN, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)LN * 8};
+    const cuuint64_t dims[2] = {(cuuint64_t)Ln, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)Ln * 8};
     const cuuint32_t box[2] = {32, (cuuint32_t)box_rows};
     const cuuint32_t elem_strides[2] = {1, 1};
     return encode(out, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, (void*)pt, dims, strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -395,8 +420,8 @@ bool plaintext_map(const u64* pt, long long LN, long long rows, int box_rows, CU
 template <int NG, int BB, int NQ>
 void launch_mac_stream(hann_ctx* c, const u64* baby, int64_t baby_stride, const u64* pt, int64_t n_bg, u64* inner,
                        int64_t inner_stride) {
-    const long long LN = (long long)c->L * c->N;
-    const int tiles = (int)(LN / 32);
+    const long long Ln = (long long)c->L * c->n;
+    const int tiles = (int)(Ln / 32);
     // split the (blk, g) range over grid.y only as far as needed to fill the machine: every extra split re-reads the
     // baby-step words
     int split = 1;
@@ -405,12 +430,14 @@ void launch_mac_stream(hann_ctx* c, const u64* baby, int64_t baby_stride, const 
     split = (int)((n_bg + per - 1) / per);
     KProf kp(c, KC_MAC);
 #ifndef HANN_NO_MAC_BULK
-    // one query, up to 32 baby steps (the rings of wider CTAs would not fit the static shared memory), 16-byte aligned
-    // plaintexts, row count within a 32-bit coordinate: the tensor-copy kernel
+    // one query, up to 32 baby steps, 16-byte aligned plaintexts, row count within a 32-bit coordinate: the tensor-copy
+    // kernel
     if constexpr (NQ == 1 && NG * BB <= 32) {
         CUtensorMap map;
-        if (((uintptr_t)pt & 15) == 0 && n_bg * (NG * BB) < (1LL << 31) && plaintext_map(pt, LN, n_bg * (NG * BB), BB, &map)) {
-            k_mac_bulk<NG, BB><<<dim3(tiles, split), 32 * NG, 0, c->stream>>>(baby, map, inner, c->N, c->L, n_bg, per, c->lt_dev, c->kflag);
+        if (((uintptr_t)pt & 15) == 0 && n_bg * (NG * BB) < (1LL << 31) && plaintext_map(pt, Ln, n_bg * (NG * BB), BB, &map)) {
+            constexpr size_t smem = mac_bulk_smem<NG, BB>();
+            if (smem > 48 * 1024) cudaFuncSetAttribute(k_mac_bulk<NG, BB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            k_mac_bulk<NG, BB><<<dim3(tiles, split), 32 * NG, smem, c->stream>>>(baby, map, inner, c->N, c->L, n_bg, per, c->lt_dev, c->kflag);
             return;
         }
     }
@@ -419,6 +446,8 @@ void launch_mac_stream(hann_ctx* c, const u64* baby, int64_t baby_stride, const 
                                                                              per, c->lt_dev);
 }
 
+// the baby-step words of NQ queries x 2 sides live in registers: 8 BB NQ of them per thread, hence BB <= 8 for one query
+// and BB <= 4 for two (B <= 16: with more warps the partial sums would not fit the static shared memory)
 template <int NQ>
 void launch_mac_stream_b(hann_ctx* c, const u64* baby, int64_t baby_stride, const u64* pt, int64_t n_bg, u64* inner,
                          int64_t inner_stride) {
@@ -428,9 +457,12 @@ void launch_mac_stream_b(hann_ctx* c, const u64* baby, int64_t baby_stride, cons
         case 4: launch_mac_stream<4, 1, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride); break;
         case 8: launch_mac_stream<4, 2, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride); break;
         case 16: launch_mac_stream<4, 4, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride); break;
-        case 32: launch_mac_stream<4, 8, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride); break;
-        case 64: launch_mac_stream<8, 8, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride); break;
-        default: launch_mac_stream<8, 16, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride); break;
+        case 32:
+            if constexpr (NQ == 1) launch_mac_stream<4, 8, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride);
+            break;
+        default:
+            if constexpr (NQ == 1) launch_mac_stream<8, 8, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride);
+            break;
     }
 }
 
@@ -440,13 +472,14 @@ int launch_mac_batch(hann_ctx* c, const u64* baby, int n_queries, const u64* pt,
     const long long LN = (long long)c->L * c->N;
     const long long n_bg = n_blocks * c->G;
     const int64_t baby_stride = (int64_t)c->B * 2 * LN, inner_stride = n_bg * 2 * LN;
-    bool small = c->N >= 32 && c->B <= 128;
+    bool small = c->N >= 64 && c->B <= 64 && (c->B & (c->B - 1)) == 0;
     for (int l = 0; l < c->L; l++) small = small && c->mod[l] < (1ULL << 50);
     if (small) {
-        // pairs of queries share one pass over the plaintexts (B <= 32: the baby-step words of two queries fit the
-        // register file); a last odd query, and every query of wider baby sets, takes a pass of its own
+        // pairs of queries share one pass over the stored plaintexts where the baby-step words of two queries and both
+        // sides fit the register file (B <= 16); a last odd query, and every query of wider baby sets, takes a pass of
+        // its own
         int q = 0;
-        if (c->B <= 32)
+        if (c->B <= 16)
             for (; q + 2 <= n_queries; q += 2) launch_mac_stream_b<2>(c, baby + q * baby_stride, baby_stride, pt, n_bg, inner + q * inner_stride, inner_stride);
         for (; q < n_queries; q++) launch_mac_stream_b<1>(c, baby + q * baby_stride, baby_stride, pt, n_bg, inner + q * inner_stride, inner_stride);
         return check_launch(c, "mac_stream");

@@ -58,9 +58,9 @@ struct NttArgs {
     const u64* src;
     long long src_gstride;
     u64 pos4, limb4;  // 4-bit fields: position within the period and limb of selection k (at most 16 selections)
-    // forward pass B (bulk-copy kernel) of polynomials that are fixed by X -> 1/X: only the first half of the chunks is
-    // transformed (the grid covers that half) and every result is also written to its mirrored position N - 1 - t
-    int mirror;
+    // forward pass B (bulk-copy kernel) of polynomials that are fixed by X -> 1/X and stored as their first N/2 transform
+    // values only: the grid covers the first half of the chunks (stride is then N/2 or more)
+    int half;
 };
 
 struct Sel {
@@ -339,19 +339,8 @@ __device__ __forceinline__ void fwd_b8t_body(const NttArgs& A, int groups, int* 
         for (int e = 0; e < 16; e++) x[e] = ar.from_mid(sb[16 * j + (e ^ j)]);
         fwd_round_f<4, AR, 1>(ar, x, [=](int u, int il) { return tcc[(((1 << u) + il) << 4) + j]; });
         u64* go = gbase + (long long)i * ystep * tile_stride + ((size_t)ch << 8);
-        if (A.mirror) {
-            // word 16 e + j of chunk c has its twin at word 16 (15 - e) + (15 - j) of chunk (N >> 8) - 1 - c
-            u64* gm = go + ((((long long)1 << (A.logN - 8)) - 1 - 2 * (chunk0 + ch)) << 8);
 #pragma unroll
-            for (int e = 0; e < 16; e++) {
-                const u64 v = ar.to_canonical(x[e]);
-                go[16 * e + j] = v;
-                gm[16 * (15 - e) + (15 - j)] = v;
-            }
-        } else {
-#pragma unroll
-            for (int e = 0; e < 16; e++) go[16 * e + j] = ar.to_canonical(x[e]);
-        }
+        for (int e = 0; e < 16; e++) go[16 * e + j] = ar.to_canonical(x[e]);
         // order this warp's shared-memory accesses before the asynchronous copy that refills the buffer
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
@@ -807,7 +796,7 @@ void launch_fwd_class(hann_ctx* c, const NttArgs& A, int groups, bool skip_a, bo
     KProf kp(c, KC_NTT_FWD_B);
     if (b8t_eligible(c, A)) {
         cudaFuncSetAttribute(k_ntt_fwd_b8t<AR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kB8tSmem);
-        const int ranges = ((c->N >> 8) / kTK) >> (A.mirror ? 1 : 0), ntiles = (groups + kTP - 1) / kTP;
+        const int ranges = ((c->N >> 8) / kTK) >> (A.half ? 1 : 0), ntiles = (groups + kTP - 1) / kTP;
         k_ntt_fwd_b8t<AR><<<dim3(ranges, A.nsel, b8t_zsplit(ranges * A.nsel, ntiles)), 256, kB8tSmem, c->stream>>>(A, groups, c->kflag);
         return;
     }
@@ -868,7 +857,7 @@ void launch_inv_class(hann_ctx* c, const NttArgs& A, int groups, bool skip_a) {
 // npoly polynomials, `stride` words apart, polynomial p using modulus lm.limb[p % lm.period]; npoly must be a multiple of
 // the period.  One set of launches per arithmetic class present in the period.
 int launch_ntt(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm, bool inverse, bool skip_a = false,
-               const u64* src = nullptr, int64_t src_gstride = 0, bool mirror = false) {
+               const u64* src = nullptr, int64_t src_gstride = 0, bool half = false) {
     if (npoly <= 0) return HANN_OK;
     if (npoly % lm.period) {
         c->err = "transform batch is not a whole number of limb periods";
@@ -887,19 +876,14 @@ int launch_ntt(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const Limb
     A.src = src;
     A.src_gstride = src_gstride;
     A.period = lm.period;
-    A.mirror = mirror ? 1 : 0;
-    if (mirror) {
-        bool ok = !inverse && skip_a && ntt_fwd_mirror_available(c, data, stride);
+    A.half = half ? 1 : 0;
+    if (half) {
+        bool ok = !inverse && skip_a && ntt_fwd_half_available(c, data, stride);
         for (int i = 0; i < lm.period; i++) ok = ok && arith_class(c->mod[(int)lm.limb[i]], false) == 0;
         if (!ok) {
-            c->err = "mirrored forward pass B needs the bulk-copy kernel and moduli below 2^50";
+            c->err = "half-size forward pass B needs the bulk-copy kernel and moduli below 2^50";
             return HANN_EINVAL;
         }
-    }
-    if (src && !(inverse && skip_a && A.b == 8 && A.a > 0 && A.tau && ((c->N >> 8) % kTK) == 0 && (((uintptr_t)data | (uintptr_t)src) & 15) == 0 &&
-                 ((stride | src_gstride) & 1) == 0)) {
-        c->err = "inverse pass B with a separate source needs the bulk-copy kernel (ring of 2^10 or more, 16-byte aligned buffers)";
-        return HANN_EINVAL;
     }
     const int64_t groups_total = npoly / lm.period;
     NttArgs Ac[3];
@@ -984,9 +968,9 @@ int launch_ntt_fwd_pass_b(hann_ctx* c, u64* data, int64_t npoly, int64_t stride,
 }
 
 // The same for polynomials fixed by X -> 1/X (encodings of real slot vectors), whose values at psi^(2t+1) and at its
-// inverse coincide: pass A left rows 2^(a-1) .. 2^a - 1 untouched, pass B transforms the first half of the chunks and
-// writes every value to position t and to position N - 1 - t.
-bool ntt_fwd_mirror_available(const hann_ctx* c, const void* data, int64_t stride) {
+// inverse coincide, i.e. position t and position N - 1 - t of the transform: only the first N/2 values are computed and
+// kept.  Pass A left out rows 2^(a-1) .. 2^a - 1; polynomial p occupies data + p * stride .. + N/2.
+bool ntt_fwd_half_available(const hann_ctx* c, const void* data, int64_t stride) {
 #ifndef HANN_NO_B8T
     return c->logN >= 10 && c->ntt_tau && ((c->N >> 8) % (2 * kTK)) == 0 && ((uintptr_t)data & 15) == 0 && (stride & 1) == 0;
 #else
@@ -994,8 +978,30 @@ bool ntt_fwd_mirror_available(const hann_ctx* c, const void* data, int64_t strid
     return false;
 #endif
 }
-int launch_ntt_fwd_pass_b_mirror(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm) {
+int launch_ntt_fwd_pass_b_half(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm) {
     return launch_ntt(c, data, npoly, stride, lm, false, true, nullptr, 0, true);
+}
+
+namespace {
+// full[p][t] = half[p][t < N/2 ? t : N - 1 - t]
+__global__ void __launch_bounds__(kThreads) k_unpack_half(const u64* __restrict__ half, u64* __restrict__ full, long long npoly, int N) {
+    const long long total = npoly * N;
+    const int n = N >> 1;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const long long p = idx / N;
+        const int t = (int)(idx % N);
+        full[idx] = half[p * n + (t < n ? t : N - 1 - t)];
+    }
+}
+}  // namespace
+
+// stored plaintext polynomials (first N/2 transform values each) -> all N values
+int launch_unpack_half(hann_ctx* c, const u64* half, int64_t npoly, u64* full) {
+    if (npoly <= 0) return HANN_OK;
+    const int64_t total = npoly * c->N;
+    const int grid = (int)std::min<int64_t>((total + kThreads - 1) / kThreads, 148 * 16);
+    k_unpack_half<<<grid, kThreads, 0, c->stream>>>(half, full, npoly, c->N);
+    return check_launch(c, "unpack_half");
 }
 
 int launch_ntt_inv(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm) {

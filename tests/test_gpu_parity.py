@@ -271,9 +271,9 @@ def test_encode_into_buffer_that_is_only_word_aligned():
 
 @pytest.mark.parametrize("logN,R,B,L,big", [(10, 16, 4, 2, False), (12, 32, 8, 2, False), (13, 64, 8, 4, True), (16, 128, 32, 4, True)])
 def test_encode_symmetry_shortcut_gives_the_same_words(logN, R, B, L, big):
-    """The encoder transforms only half of every plaintext and mirrors the rest (an encoding of real slots is fixed by
-    X -> 1/X); with the shortcut switched off it computes every transform in full.  Same words, and they are the
-    mirror images the shortcut relies on."""
+    """The encoder computes only the stored half of every transformed plaintext (an encoding of real slots is fixed by
+    X -> 1/X, so the other half is its mirror image); with the shortcut switched off it computes every transform in
+    full and keeps the first half.  Same words, and the canonical form is the oracle's encoding."""
     import torch
 
     ps = synth.small_params(logN, R, B, L=L, big=big)
@@ -287,8 +287,18 @@ def test_encode_symmetry_shortcut_gives_the_same_words(logN, R, B, L, big):
     g.set_tuning(b.TUNE_ENCODE_SYMMETRY, 1)
     g.sync()
     assert torch.equal(short, full)
-    words = full.view(torch.int64).reshape(-1, ps.N)
-    assert torch.equal(words, words.flip(1))
+    pt_g = g.export(b.KIND_PT, short, 2)                      # plaintexts (g, b) = (0, 0) and (0, 1) of block 0
+    Rr = np.zeros((ps.n, R), dtype=np.float32)
+    nr = min(ps.n, rows.shape[0])
+    Rr[:nr, : R - 1] = rows[:nr].cpu().numpy()
+    for bb in range(2):
+        z = np.array([Rr[i, (i + bb) % R] for i in range(ps.n)], dtype=np.float64)
+        m = p.o.encode(z)
+        want = np.stack([np.array([int(v) % q for v in m], dtype=np.uint64) for q in ps.q])
+        assert np.array_equal(pt_g.reshape(2, ps.L, ps.N)[bb], want)
+    # import of the canonical form gives the stored words back
+    back = g.import_(b.KIND_PT, pt_g, 2)
+    assert torch.equal(back.reshape(-1)[: 2 * ps.L * ps.n], short.reshape(-1)[: 2 * ps.L * ps.n])
 
 
 @pytest.mark.parametrize(
@@ -484,14 +494,15 @@ def test_seed_compressed_query_upload(logN, big):
 
 
 def test_sizes_follow_the_storage_formula():
-    """hann_sizeof against the closed forms: 16*L*R bytes per encoded row, 32*L*R per encrypted row (the paper's
-    80*L*R of Sec. 2 without its 2.5x serialization overhead)"""
+    """hann_sizeof against the closed forms: 8*L*R bytes per encoded row (half of every transformed plaintext is the
+    mirror image of the other half and is not stored), 32*L*R per encrypted row (the paper's 80*L*R of Sec. 2 without
+    its 2.5x serialization overhead)"""
     from paper_2608_21131_b200 import binding as b
 
     for ps in (synth.small_params(10, 16, 4, L=2), synth.FULL16):
         g = b.Context(ps)
         assert g.sizeof(b.SIZE_ROWS_PER_BLOCK) == ps.n
-        assert g.sizeof(b.SIZE_PT_BLOCK) == 16 * ps.L * ps.R * ps.n
+        assert g.sizeof(b.SIZE_PT_BLOCK) == 8 * ps.L * ps.R * ps.n
         assert g.sizeof(b.SIZE_CTDB_BLOCK) == 32 * ps.L * ps.R * ps.n
         assert g.sizeof(b.SIZE_CT) == 2 * ps.L * ps.N * 8 and g.sizeof(b.SIZE_BABY) == ps.B * g.sizeof(b.SIZE_CT)
         assert g.sizeof(b.SIZE_INNER) == ps.G * g.sizeof(b.SIZE_CT)

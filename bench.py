@@ -136,27 +136,31 @@ def algorithmic_work(ctx, n_blocks, n_rows):
     """Algorithmic work of ONE step per kernel class: bytes for the HBM-bound kernels, binary64 instructions for the
     transform kernels (moduli below 2^50 run their butterflies on the FP64 pipe: exact product = multiply + fma,
     quotient = multiply + round, remainder = fma + add, butterfly = add + subtract: 8 per butterfly; an FFT butterfly with
-    separately rounded products and sums is 10).  Returns {class: (bound, amount, units per step)}."""
+    separately rounded products and sums is 10).  The transform of an encoded plaintext takes every value twice, so only
+    its first stage (a product and a sum per pair: 7 instructions) runs in full; the other stages and the stored
+    plaintext are half size.  Returns {class: (bound, amount, units per step)}."""
     L, N, B, G, R = ctx.L, ctx.N, ctx.B, ctx.G, ctx.R
     n, logN = ctx.n, ctx.logN
     b = min(logN, 8)
     a = logN - b
     W = 8 * N
     items_rot = (G - 1) * n_blocks  # key switches of the rotate-and-sum
-    fwd_polys = n_blocks * R * L + (L * (L + 1) + (B - 1) * 2 * L) + items_rot * (L * (L + 1) + 2 * L)
+    pt_polys = n_blocks * R * L       # half-size transforms
+    ks_polys = (L * (L + 1) + (B - 1) * 2 * L) + items_rot * (L * (L + 1) + 2 * L)
     inv_polys = (L + (B - 1) * 2) + items_rot * (L + 2)
     lift_src = [(L, L + 1), ((B - 1) * 2, L)] + [(items_rot * L, L + 1), (items_rot * 2, L)]  # (sources, targets each)
     lift_ops = sum(src * (1 + tgt) * a * (N // 2) * 8 for src, tgt in lift_src)
+    pass_a_half = (N // 2) * 7 + (a - 1) * (N // 4) * 8  # first stage in full (one output per pair), then half the butterflies
     return {
-        "mac": ("hbm", n_blocks * R * L * W + B * 2 * L * W + n_blocks * G * 2 * L * W, n_blocks),
+        "mac": ("hbm", n_blocks * R * L * (W // 2) + B * 2 * L * W + n_blocks * G * 2 * L * W, n_blocks),
         # one digit set under B-1 streamed keys (query_prepare) / one key under many digit sets (rotate_sum, L2-resident key)
         "ks_inner_keys": ("hbm", (B - 1) * (L * 2 * (L + 1) * W + 2 * (L + 1) * W) + L * (L + 1) * W, B - 1),
         "ks_inner": ("hbm", (G - 1) * (L * 2 * (L + 1) * W + n_blocks * (L * (L + 1) * W + 2 * (L + 1) * W)), items_rot),
-        "ntt_fwd_b": ("alu", fwd_polys * (N // 2) * b * 8, fwd_polys),
+        "ntt_fwd_b": ("alu", (pt_polys * (N // 4) + ks_polys * (N // 2)) * b * 8, pt_polys + ks_polys),
         "ntt_inv_b": ("alu", inv_polys * (N // 2) * b * 8, inv_polys),
         "lift_digits": ("alu", lift_ops, inv_polys),
         "fft_a": ("hbm", n_blocks * R * (n * 16) + n_rows * R * 4, n_blocks * R),
-        "fft_b": ("alu", n_blocks * R * ((a - 1) * (n // 2) * 10 + L * a * (N // 2) * 8), n_blocks * R),
+        "fft_b": ("alu", n_blocks * R * ((a - 1) * (n // 2) * 10 + L * pass_a_half), n_blocks * R),
     }
 
 

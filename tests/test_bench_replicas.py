@@ -59,8 +59,9 @@ def test_single_process_identity():
 
 def test_algorithmic_work_matches_the_per_row_figures():
     """the roofline numerators of bench.py against the closed forms of the design: a scored row costs the multiply-
-    accumulate 16*L*R bytes of plaintext read + 32*L*G bytes of partial sums written (8,192 + 512 at L = 4, R = 128,
-    G = 4), the baby set is read once per level, and a block's encoding is R*L transforms of N/2*log2(N) butterflies"""
+    accumulate 8*L*R bytes of stored plaintext read (half of every transformed plaintext mirrors the other half) +
+    32*L*G bytes of partial sums written (4,096 + 512 at L = 4, R = 128, G = 4), the baby set is read once per level,
+    and pass B of a block's encoding is R*L half-size transforms"""
     import types
 
     import bench
@@ -72,9 +73,11 @@ def test_algorithmic_work_matches_the_per_row_figures():
         w = bench.algorithmic_work(ctx, n_blocks, n_blocks * n)
         bound, mac_bytes, units = w["mac"]
         assert bound == "hbm" and units == n_blocks
-        assert mac_bytes == n_blocks * n * (16 * L * R + 32 * L * G) + B * 2 * L * N * 8
-        assert 16 * L * R + 32 * L * G == 8704
-        # pass B of the forward transforms: 8 of the 16 stages of every polynomial, 8 binary64 instructions per butterfly
-        fwd_polys = w["ntt_fwd_b"][2]
-        assert fwd_polys == n_blocks * R * L + (L * (L + 1) + (B - 1) * 2 * L) + (G - 1) * n_blocks * (L * (L + 1) + 2 * L)
-        assert w["ntt_fwd_b"][1] == fwd_polys * (N // 2) * 8 * 8
+        assert mac_bytes == n_blocks * n * (8 * L * R + 32 * L * G) + B * 2 * L * N * 8
+        assert 8 * L * R + 32 * L * G == 4608
+        # pass B of the forward transforms: 8 of the 16 stages, 8 binary64 instructions per butterfly; the plaintexts'
+        # transforms run on half of the chunks
+        pt_polys = n_blocks * R * L
+        ks_polys = (L * (L + 1) + (B - 1) * 2 * L) + (G - 1) * n_blocks * (L * (L + 1) + 2 * L)
+        assert w["ntt_fwd_b"][2] == pt_polys + ks_polys
+        assert w["ntt_fwd_b"][1] == (pt_polys * (N // 4) + ks_polys * (N // 2)) * 8 * 8

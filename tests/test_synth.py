@@ -82,8 +82,8 @@ def test_padding_groups_partition_and_inflate():
 def test_storage_formula_matches_the_papers_worked_example():
     """Sec. 2, "Measured prototype vs. deployment": 80*L*R bytes per encrypted vector, with the totals the paper prints
     (tests/golden/storage_per_vector.txt).  This library's own layout is the same count without the 2.5x serialization
-    overhead: R ciphertexts of 2*L*N*8 bytes per block of N/2 rows = 32*L*R bytes per encrypted row, 16*L*R per encoded
-    plaintext row."""
+    overhead: R ciphertexts of 2*L*N*8 bytes per block of N/2 rows = 32*L*R bytes per encrypted row; an encoded
+    plaintext row takes 8*L*R (a transformed plaintext of L*N words, of which the stored half determines the rest)."""
     import os
 
     unit = {"KB": 1e3, "GB": 1e9, "TB": 1e12}
@@ -96,5 +96,5 @@ def test_storage_formula_matches_the_papers_worked_example():
     for ps in (synth.TOY, synth.FULL15, synth.FULL16):
         ct_bytes = 2 * ps.L * ps.N * 8
         assert ps.R * ct_bytes // ps.n == 32 * ps.L * ps.R                       # encrypted block / rows per block
-        assert ps.R * ps.L * ps.N * 8 // ps.n == 16 * ps.L * ps.R                 # encoded plaintext block
+        assert ps.R * ps.L * (ps.N // 2) * 8 // ps.n == 8 * ps.L * ps.R            # stored plaintext block
         assert 2.5 * 32 * ps.L * ps.R == 80 * ps.L * ps.R

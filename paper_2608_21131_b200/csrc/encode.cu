@@ -418,6 +418,40 @@ __global__ void __launch_bounds__(256, HANN_X_MINBLOCKS) k_encode_x(FusedArgs A)
         const int l = i / NT, e = i % NT;
         if (e) twc[i] = A.tw[((size_t)l << (A.logn + 1)) + e];
     }
+    if constexpr (SYM && R1 == 4 && R2 == 4) {
+        // The half-size second round has work for 128 threads only: two limbs at a time, the first rounds of both by
+        // all threads into the two halves of the exchange tile, then threads 0..127 finish one limb and threads
+        // 128..255 the other.
+        constexpr int HT = (NT / 2) * 16;  // words of a half-size tile
+        for (int l = 0; l < A.L; l += 2) {
+            __syncthreads();  // the twiddle cache is filled (first pair) / the exchange tile is free again
+            for (int h = 0; h < 2 && l + h < A.L; h++) {
+                const ArithF64 ar(A.lt + l + h);
+                const double2* tw = twc + (l + h) * NT;
+                double x[HF];
+                const double2 w1 = tw[1];
+#pragma unroll
+                for (int e = 0; e < HF; e++) x[e] = __dadd_rn(ar.reduce(m[e]), ar.mulmod_small(ar.reduce(m[e + HF]), w1));
+                fwd_round<R1 - 1, ArithF64, R1 - 1>(ar, x, tw, 2u);
+#pragma unroll
+                for (int e = 0; e < HF; e++) smx[h * HT + ((g + G1 * e) << 4) + c] = ar.to_exch(x[e]);
+            }
+            __syncthreads();
+            const int h = threadIdx.x >> 7, ll = l + h;
+            if (ll < A.L) {
+                const ArithF64 ar(A.lt + ll);
+                const double2* tw = twc + ll * NT;
+                u64* base = A.out + ((long long)P * A.L + ll) * A.out_stride + c0;
+                const int cc = threadIdx.x & 15, gg = (threadIdx.x & 127) >> 4;
+                double x[1 << R2];
+#pragma unroll
+                for (int e = 0; e < (1 << R2); e++) x[e] = ar.from_mid(smx[h * HT + (((gg << R2) + e) << 4) + cc]);
+                fwd_round<R2, ArithF64, 5 - R1>(ar, x, tw, (unsigned)(G2 + gg));
+#pragma unroll
+                for (int e = 0; e < (1 << R2); e++) base[(size_t)((gg << R2) + e) * 256 + cc] = ar.to_mid(x[e]);
+            }
+        }
+    } else
     for (int l = 0; l < A.L; l++) {
         const ArithF64 ar(A.lt + l);
         const double2* tw = twc + l * NT;

@@ -127,8 +127,11 @@ int hann_get_stats(hann_ctx *ctx, hann_stats *out);
  * HANN_TUNE_ENCODE_SYMMETRY: 1 (default) lets hann_encode_candidates use the fact that the encoding of a REAL slot vector
  * is fixed by X -> 1/X, so that its number-theoretic transform takes each value twice (at psi^(2t+1) and at the inverse
  * of that root): only half of every transform is computed and the other half is written as a mirror image; 0 computes
- * every transform in full.  Same bits either way. */
-enum { HANN_TUNE_ENCODE_GROUP = 1, HANN_TUNE_HOST_LIMBS = 2, HANN_TUNE_ENCODE_SYMMETRY = 3 };
+ * every transform in full.  Same bits either way.
+ * HANN_TUNE_HOST_GROUPS: number of block groups hann_score_level_host cuts a level into (a group is scored and its scores
+ * are downloaded while the rows of the following groups still travel); 0 (default) chooses from the level's size.  Ask
+ * hann_level_host_bytes again after changing it. */
+enum { HANN_TUNE_ENCODE_GROUP = 1, HANN_TUNE_HOST_LIMBS = 2, HANN_TUNE_ENCODE_SYMMETRY = 3, HANN_TUNE_HOST_GROUPS = 4 };
 int hann_set_tuning(hann_ctx *ctx, int what, int value);
 
 /* Per-launch profile: while enabled every kernel launch of the context is bracketed by a CUDA event pair (this
@@ -298,11 +301,13 @@ int64_t hann_compact_bytes(const hann_ctx *ctx, int64_t n_blocks, int keep);
 int hann_compact_scores(hann_ctx *ctx, const void *score_ct_dev, int64_t n_blocks, int keep, int rescale, void *out_dev,
                         void *ws, size_t ws_bytes);
 
-/* One level end to end from HOST buffers (copies included): the rows are copied to the device block by block on a copy
- * stream while the query ciphertext is imported and its baby set prepared on a helper stream; every block is encoded as
- * soon as its rows have arrived; then multiply-accumulate, rotate-and-sum, and the score ciphertexts are exported to
- * the host in canonical layout.  Page-locked host buffers are needed for the copies to overlap the kernels (pageable
- * memory works but serialises).  Device buffers for the intermediates are carved from `ws_dev`, which must hold
+/* One level end to end from HOST buffers (copies included): the query ciphertext goes up first and its baby set is
+ * prepared on a helper stream; the rows follow block by block on an upload stream and every block is encoded as soon as
+ * its rows have arrived; the level is cut into groups of blocks (HANN_TUNE_HOST_GROUPS), and a group's multiply-
+ * accumulate, rotate-and-sum and export run on scoring streams while later groups are still uploaded and encoded, its
+ * score ciphertexts travelling to the host (canonical layout) on a download stream.  Page-locked host buffers are needed
+ * for the copies to overlap the kernels (pageable memory works but serialises).  Device buffers for the intermediates
+ * are carved from `ws_dev`, which must hold
  * hann_level_host_bytes(ctx, n_rows) bytes.  Returns after everything has finished.
  *   ct_host [2][L][N];  rows_host [n_rows][dim] float32;  score_ct_host [ceil(n_rows/n)][2][L][N] (fewer limbs with
  *   HANN_TUNE_HOST_LIMBS). */

@@ -22,6 +22,7 @@ KIND_POLY, KIND_CT, KIND_PT = 1, 2, 3
 TUNE_ENCODE_GROUP = 1
 TUNE_HOST_LIMBS = 2
 TUNE_ENCODE_SYMMETRY = 3
+TUNE_HOST_GROUPS = 4
 
 
 class HannError(RuntimeError):

@@ -143,7 +143,7 @@ int ks_digits_to_lifted(hann_ctx* c, u64* c1c, int64_t items, u64* digits, int64
     const int64_t LN = (int64_t)L * N;
     const bool fused_gather = gather_src && ks_lift_available(c) && ntt_inv_pass_b_gathers(c, gather_src, c1c) && (gather_stride & 1) == 0;
     if (gather_src && !fused_gather)
-        CK(cudaMemcpy2DAsync(c1c, LN * 8, gather_src, gather_stride * 8, LN * 8, items, cudaMemcpyDeviceToDevice, c->stream));
+        RET(launch_copy2d(c, c1c, LN, gather_src, gather_stride, LN, items));
     if (ks_lift_available(c)) {
         // c1c arrives in the transform domain: inverse pass B', then one kernel finishes the inverse, lifts the digits
         // and starts their forward transforms; the same again for ModDown
@@ -305,6 +305,14 @@ extern "C" int hann_ctx_create(const hann_params* prm, hann_ctx** out) {
     for (int i = 0; i < 2 && ok; i++)
         ok = cudaStreamCreateWithFlags(&c->lane_stream[i], cudaStreamNonBlocking) == cudaSuccess &&
              cudaEventCreateWithFlags(&c->lane_join[i], cudaEventDisableTiming) == cudaSuccess;
+    if (ok)
+        ok = cudaStreamCreateWithFlags(&c->up_stream, cudaStreamNonBlocking) == cudaSuccess &&
+             cudaStreamCreateWithFlags(&c->down_stream, cudaStreamNonBlocking) == cudaSuccess &&
+             cudaEventCreateWithFlags(&c->down_done, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < 2 && ok; i++)
+        ok = cudaStreamCreateWithFlags(&c->score_stream[i], cudaStreamNonBlocking) == cudaSuccess &&
+             cudaEventCreateWithFlags(&c->score_join[i], cudaEventDisableTiming) == cudaSuccess;
+    if (ok) ok = cudaEventCreateWithFlags(&c->prep_done, cudaEventDisableTiming) == cudaSuccess;
     if (ok) ok = ntt_configure(c) == HANN_OK;
     if (!ok) {
         cudaGetLastError();
@@ -336,6 +344,16 @@ extern "C" void hann_ctx_destroy(hann_ctx* c) {
         if (c->lane_join[i]) cudaEventDestroy(c->lane_join[i]);
     }
     for (cudaEvent_t e : c->blk_ev) cudaEventDestroy(e);
+    for (cudaEvent_t e : c->grp_ev) cudaEventDestroy(e);
+    for (cudaEvent_t e : c->enc_ev) cudaEventDestroy(e);
+    for (cudaEvent_t e : {c->score_join[0], c->score_join[1], c->prep_done})
+        if (e) cudaEventDestroy(e);
+    for (cudaStream_t st : {c->up_stream, c->down_stream, c->score_stream[0], c->score_stream[1]})
+        if (st) {
+            cudaStreamSynchronize(st);
+            cudaStreamDestroy(st);
+        }
+    if (c->down_done) cudaEventDestroy(c->down_done);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_join) cudaEventDestroy(c->ev_join);
     for (auto& r : c->krec) {
@@ -424,6 +442,10 @@ extern "C" int hann_set_tuning(hann_ctx* c, int what, int value) {
         case HANN_TUNE_HOST_LIMBS:
             if (value < 1 || value > c->L) return fail(c, HANN_EINVAL, "hann_set_tuning: host limbs must be in 1..L");
             c->host_limbs = value;
+            return HANN_OK;
+        case HANN_TUNE_HOST_GROUPS:
+            if (value < 0) return fail(c, HANN_EINVAL, "hann_set_tuning: host groups must be 0 (automatic) or positive");
+            c->host_groups = value;
             return HANN_OK;
         case HANN_TUNE_ENCODE_SYMMETRY:
             c->encode_sym = value ? 1 : 0;
@@ -877,7 +899,7 @@ extern "C" int hann_query_prepare(hann_ctx* c, const void* ct_dev, void* baby_de
     Timer tm(c, 0);
     const u64* ct = (const u64*)ct_dev;
     u64* baby = (u64*)baby_dev;
-    CK(cudaMemcpyAsync(baby, ct, ctw * 8, cudaMemcpyDeviceToDevice, c->stream));  // rotation 0
+    RET(launch_copy2d(c, baby, ctw, ct, ctw, ctw, 1));  // rotation 0
     if (B == 1) return HANN_OK;
     if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_query_prepare: workspace missing or not 256-byte aligned");
     Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
@@ -886,9 +908,8 @@ extern "C" int hann_query_prepare(hann_ctx* c, const void* ct_dev, void* baby_de
     u64* u = ar.take<u64>((int64_t)(B - 1) * 2 * L1N);
     u64* lifted = ar.take<u64>((int64_t)(B - 1) * 2 * LN);
     if (!c1c || !digits || !u || !lifted) return fail(c, HANN_EWORKSPACE, "hann_query_prepare: workspace too small");
-    CK(cudaMemcpyAsync(c1c, ct + LN, LN * 8, cudaMemcpyDeviceToDevice, c->stream));
     // one digit set, B-1 keys: item i uses rotation 1 + i
-    RET(ks_digits_to_lifted(c, c1c, 1, digits, 0, 1, 1, B - 1, u, lifted));
+    RET(ks_digits_to_lifted(c, c1c, 1, digits, 0, 1, 1, B - 1, u, lifted, ct + LN, 2 * LN));
     RET(launch_moddown_combine(c, u, lifted, B - 1, 1, 1, ct, 0, nullptr, 0, baby + ctw, baby + ctw + LN, ctw));
     return HANN_OK;
 }
@@ -932,8 +953,7 @@ extern "C" int hann_encode_candidates(hann_ctx* c, const float* rows_dev, int64_
                     RET(launch_encode_rows(c, rows, rows_here, dim, p0 + s0, sn, stage, ws));
                     RET(launch_ntt_fwd(c, stage, (int64_t)sn * c->L, c->N, limbmap_q(c)));
                 }
-                CK(cudaMemcpy2DAsync(polys + (int64_t)s0 * Ln, (size_t)n * 8, stage, (size_t)c->N * 8, (size_t)n * 8, (size_t)sn * c->L,
-                                     cudaMemcpyDeviceToDevice, c->stream));
+                RET(launch_copy2d(c, polys + (int64_t)s0 * Ln, n, stage, c->N, n, (int64_t)sn * c->L));
             }
         }
     }
@@ -995,7 +1015,7 @@ extern "C" int hann_score_level_ctdb(hann_ctx* c, const void* baby_dev, const vo
         RET(launch_mac_ct(c, (const u64*)baby_dev, ctdb + i0 * c->B * ctw, ni, d));
         // relinearise: (d0 + ks0, d1 + ks1) with (ks0, ks1) the key switch of d2 under the key of s^2 ("rotation 0": no
         // automorphism)
-        CK(cudaMemcpy2DAsync(c1c, LN * 8, d + 2 * LN, 3 * LN * 8, LN * 8, ni, cudaMemcpyDeviceToDevice, c->stream));
+        RET(launch_copy2d(c, c1c, LN, d + 2 * LN, 3 * LN, LN, ni));
         RET(ks_digits_to_lifted(c, c1c, ni, digits, (int64_t)L * L1N, 0, 0, ni, u, lifted));
         RET(launch_moddown_combine(c, u, lifted, ni, 0, 0, nullptr, 0, d, 3 * LN, inner + i0 * ctw, inner + i0 * ctw + LN, ctw));
     }
@@ -1013,7 +1033,7 @@ extern "C" int hann_rotate_sum(hann_ctx* c, const void* inner_dev, int64_t n_blo
     DeviceGuard dg(c->device);
     Timer tm(c, 3);
     if (G == 1) {
-        CK(cudaMemcpyAsync(score, inner, n_blocks * ctw * 8, cudaMemcpyDeviceToDevice, c->stream));
+        RET(launch_copy2d(c, score, ctw, inner, ctw, n_blocks * ctw, 1));
         return HANN_OK;
     }
     if (!c->keytab_host[B]) return fail(c, HANN_ENOKEY, "hann_rotate_sum: the key of rotation B is not loaded");
@@ -1050,7 +1070,7 @@ extern "C" int hann_rotate_sum(hann_ctx* c, const void* inner_dev, int64_t n_blo
     // Blocks are independent: up to four ranges run side by side on the context's stream and the helper streams, each in
     // its own part of the workspace, which keeps the machine busy through the many small launches of a key switch.
     // (One lane while the per-launch profile is on, so that its kernel times do not overlap.)
-    int lanes = (int)std::min<int64_t>(4, n_blocks);
+    int lanes = (int)std::min<int64_t>(c->max_lanes, n_blocks);
     if (c->stream == c->aux_stream || c->kprof) lanes = 1;
     while (lanes > 1 && (((int64_t)ws_bytes / lanes) & ~(int64_t)255) < ks_item_words(c) * 8 + kSlack) lanes--;
     if (lanes <= 1) {
@@ -1147,7 +1167,8 @@ extern "C" int hann_query_level(hann_ctx* c, const void* ct_dev, const float* ro
 
 namespace {
 struct LevelPlan {
-    int64_t nblk, ct, baby, rows, pt, inner, score, stage, ws, total;
+    int64_t nblk, ct, baby, rows, pt, inner, score, stage, ws, ws_score, total;
+    int ng;  // block groups; group gi covers blocks [nblk - nblk (ng - gi) / ng, nblk - nblk (ng - gi - 1) / ng)
 };
 LevelPlan plan_level(const hann_ctx* c, int64_t n_rows, int dim) {
     LevelPlan p;
@@ -1161,7 +1182,13 @@ LevelPlan plan_level(const hann_ctx* c, int64_t n_rows, int dim) {
     p.score = align256(p.nblk * ctb);
     p.stage = align256(p.nblk * ctb);
     p.ws = align256(hann_workspace_bytes(c, p.nblk));
-    p.total = p.ct + p.baby + p.rows + p.pt + p.inner + p.score + p.stage + p.ws;
+    p.ng = c->host_groups;
+    if (p.ng <= 0) p.ng = (int)(p.nblk <= 24 ? (p.nblk + 2) / 3 : (p.nblk + 3) / 4);  // groups of three to four blocks
+    p.ng = (int)std::max<int64_t>(1, std::min<int64_t>(p.ng, p.nblk));
+    // with more than one group: a rotate-and-sum workspace for each of the two scoring streams
+    const int64_t gmax = p.nblk - p.nblk * (p.ng - 1) / p.ng;
+    p.ws_score = p.ng > 1 ? align256(ks_item_words(c) * std::min<int64_t>(gmax, 8) * 8 + kSlack) : 0;
+    p.total = p.ct + p.baby + p.rows + p.pt + p.inner + p.score + p.stage + p.ws + 2 * p.ws_score;
     return p;
 }
 }  // namespace
@@ -1188,57 +1215,102 @@ extern "C" int hann_score_level_host(hann_ctx* c, const uint64_t* ct_host, const
     u64* inner = (u64*)b; b += p.inner;
     u64* score = (u64*)b; b += p.score;
     u64* stage = (u64*)b; b += p.stage;
-    void* ws = b;
-    // Three streams: the rows travel block by block on a copy stream, the query is imported and its baby rotations are
-    // prepared on the helper stream, and the context's stream encodes each block as soon as its rows have arrived.
+    void* ws = b; b += p.ws;
+    char* ws_score[2] = {b, b + p.ws_score};
+    // The query goes up first, then the rows block by block on the upload stream; the helper stream prepares the baby
+    // rotations; the context's stream encodes each block as soon as its rows have arrived.  The level is cut into groups
+    // of blocks: a group is scored (multiply-accumulate, rotate-and-sum, inverse transform of its score ciphertexts) on
+    // one of two scoring streams while the following groups are still uploaded and encoded, and its scores go home on
+    // the download stream beside all that.  Only the last group's scoring and download follow the last upload.  (One
+    // group: everything on the context's stream, the rotate-and-sum on its four lanes.)
+    const int ng = p.ng;
     while ((int64_t)c->blk_ev.size() < p.nblk) {
         cudaEvent_t e;
         CK(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
         c->blk_ev.push_back(e);
     }
-    const int64_t prep = c->B > 1 ? align256(prepare_words(c) * 8 + kSlack) : 0;
-    cudaStream_t main_stream = c->stream, copy_stream = c->lane_stream[1];
-    CK(cudaEventRecord(c->ev_fork, main_stream));
-    CK(cudaStreamWaitEvent(copy_stream, c->ev_fork, 0));
-    CK(cudaStreamWaitEvent(c->aux_stream, c->ev_fork, 0));
-    for (int64_t blk = 0; blk < p.nblk; blk++) {
-        const int64_t r0 = blk * c->n, rn = std::min<int64_t>(c->n, n_rows - r0);
-        CK(cudaMemcpyAsync(rows + r0 * dim, rows_host + r0 * dim, (size_t)rn * dim * 4, cudaMemcpyHostToDevice, copy_stream));
-        CK(cudaEventRecord(c->blk_ev[blk], copy_stream));
+    while ((int)c->grp_ev.size() < ng || (int)c->enc_ev.size() < ng) {
+        cudaEvent_t e, e2;
+        CK(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+        c->grp_ev.push_back(e);
+        CK(cudaEventCreateWithFlags(&e2, cudaEventDisableTiming));
+        c->enc_ev.push_back(e2);
     }
+    const int64_t prep = c->B > 1 ? align256(prepare_words(c) * 8 + kSlack) : 0;
+    cudaStream_t main_stream = c->stream;
+    CK(cudaEventRecord(c->ev_fork, main_stream));
+    for (cudaStream_t st : {c->up_stream, c->down_stream, c->aux_stream, c->score_stream[0], c->score_stream[1]})
+        CK(cudaStreamWaitEvent(st, c->ev_fork, 0));
+    // host-to-device copies are served in the order they were queued, whatever their stream: the query must not wait
+    // behind the rows
     c->stream = c->aux_stream;
     int rc = import_polys(c, ct_host, 2, ct);
+    c->stream = main_stream;
+    for (int64_t blk = 0; blk < p.nblk; blk++) {
+        const int64_t r0 = blk * c->n, rn = std::min<int64_t>(c->n, n_rows - r0);
+        CK(cudaMemcpyAsync(rows + r0 * dim, rows_host + r0 * dim, (size_t)rn * dim * 4, cudaMemcpyHostToDevice, c->up_stream));
+        CK(cudaEventRecord(c->blk_ev[blk], c->up_stream));
+    }
+    c->stream = c->aux_stream;
     if (rc == HANN_OK) rc = hann_query_prepare(c, ct, baby, ws, (size_t)prep);
     c->stream = main_stream;
-    cudaError_t ej = cudaEventRecord(c->ev_join, c->aux_stream);
-    for (int64_t blk = 0; blk < p.nblk && rc == HANN_OK; blk++) {
-        const int64_t r0 = blk * c->n, rn = std::min<int64_t>(c->n, n_rows - r0);
-        if (cudaStreamWaitEvent(main_stream, c->blk_ev[blk], 0) != cudaSuccess) rc = fail(c, HANN_ECUDA, "cudaStreamWaitEvent failed");
-        if (rc == HANN_OK)
-            rc = hann_encode_candidates(c, rows + r0 * dim, rn, dim, pt + blk * (hann_sizeof(c, HANN_SIZE_PT_BLOCK) / 8), (char*)ws + prep,
-                                        (size_t)(p.ws - prep));
+    cudaError_t ce = cudaEventRecord(c->prep_done, c->aux_stream);
+    const int64_t ptw = hann_sizeof(c, HANN_SIZE_PT_BLOCK) / 8, ctw = hann_sizeof(c, HANN_SIZE_CT) / 8;
+    const int64_t innerw = hann_sizeof(c, HANN_SIZE_INNER) / 8;
+    const int keep = c->host_limbs >= c->L ? c->L : c->host_limbs;  // limbs of every score polynomial that go home
+    const int64_t kw = (int64_t)keep * c->N;
+    const int saved_lanes = c->max_lanes;
+    for (int gi = 0; gi < ng && rc == HANN_OK; gi++) {
+        const int64_t b0 = p.nblk - p.nblk * (ng - gi) / ng, b1 = p.nblk - p.nblk * (ng - gi - 1) / ng, nb = b1 - b0;
+        for (int64_t blk = b0; blk < b1 && rc == HANN_OK; blk++) {
+            const int64_t r0 = blk * c->n, rn = std::min<int64_t>(c->n, n_rows - r0);
+            if (cudaStreamWaitEvent(main_stream, c->blk_ev[blk], 0) != cudaSuccess) rc = fail(c, HANN_ECUDA, "cudaStreamWaitEvent failed");
+            if (rc == HANN_OK)
+                rc = hann_encode_candidates(c, rows + r0 * dim, rn, dim, pt + blk * ptw, (char*)ws + prep, (size_t)(p.ws - prep));
+        }
+        if (rc != HANN_OK) break;
+        // the scoring stream of this group: the context's own when there is one group
+        cudaStream_t ss = ng > 1 ? c->score_stream[gi & 1] : main_stream;
+        cudaError_t e = cudaSuccess;
+        if (ng > 1) {
+            e = cudaEventRecord(c->enc_ev[gi], main_stream);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(ss, c->enc_ev[gi], 0);
+            c->max_lanes = 1;  // the groups run side by side instead of the lanes
+        }
+        if (e == cudaSuccess && gi < 2) e = cudaStreamWaitEvent(ss, c->prep_done, 0);  // the baby rotations are ready
+        c->stream = ss;
+        void* wsg = ng > 1 ? (void*)ws_score[gi & 1] : ws;
+        const size_t wsg_bytes = ng > 1 ? (size_t)p.ws_score : (size_t)p.ws;
+        if (e == cudaSuccess) rc = hann_score_level(c, baby, pt + b0 * ptw, nb, inner + b0 * innerw, wsg, wsg_bytes);
+        if (e == cudaSuccess && rc == HANN_OK) rc = hann_rotate_sum(c, inner + b0 * innerw, nb, score + b0 * ctw, wsg, wsg_bytes);
+        // canonical form of the group's scores in the staging buffer (first `keep` limbs of every polynomial: with
+        // keep < L the exact compaction of hann_compact_scores), then home on the download stream
+        const int64_t npoly = nb * 2;
+        u64* st = stage + b0 * 2 * kw;
+        if (e == cudaSuccess && rc == HANN_OK) rc = launch_copy2d(c, st, kw, score + b0 * ctw, (int64_t)c->L * c->N, kw, npoly);
+        if (e == cudaSuccess && rc == HANN_OK) rc = launch_ntt_inv(c, st, npoly * keep, c->N, limbmap_first(keep));
+        c->stream = main_stream;
+        c->max_lanes = saved_lanes;
+        if (e == cudaSuccess && rc == HANN_OK) e = cudaEventRecord(c->grp_ev[gi], ss);
+        if (e == cudaSuccess && rc == HANN_OK) e = cudaStreamWaitEvent(c->down_stream, c->grp_ev[gi], 0);
+        if (e == cudaSuccess && rc == HANN_OK)
+            e = cudaMemcpyAsync(score_ct_host + b0 * 2 * kw, st, (size_t)(npoly * kw) * 8, cudaMemcpyDeviceToHost, c->down_stream);
+        if (ce == cudaSuccess) ce = e;
     }
-    // join the helper streams before reporting anything
-    cudaError_t ew = cudaStreamWaitEvent(main_stream, c->ev_join, 0);
-    cudaError_t ew2 = cudaStreamWaitEvent(main_stream, c->blk_ev[p.nblk - 1], 0);
+    // join every helper stream before reporting anything
+    cudaError_t ej[6];
+    ej[0] = cudaStreamWaitEvent(main_stream, c->prep_done, 0);
+    ej[1] = cudaStreamWaitEvent(main_stream, c->blk_ev[p.nblk - 1], 0);
+    ej[2] = cudaEventRecord(c->down_done, c->down_stream);
+    if (ej[2] == cudaSuccess) ej[2] = cudaStreamWaitEvent(main_stream, c->down_done, 0);
+    for (int i = 0; i < 2; i++) {
+        ej[3 + i] = cudaEventRecord(c->score_join[i], c->score_stream[i]);
+        if (ej[3 + i] == cudaSuccess) ej[3 + i] = cudaStreamWaitEvent(main_stream, c->score_join[i], 0);
+    }
+    ej[5] = cudaSuccess;
     RET(rc);
-    CK(ej);
-    CK(ew);
-    CK(ew2);
-    RET(hann_score_level(c, baby, pt, p.nblk, inner, ws, (size_t)p.ws));
-    RET(hann_rotate_sum(c, inner, p.nblk, score, ws, (size_t)p.ws));
-    if (c->host_limbs >= c->L) {
-        RET(export_polys(c, score, p.nblk * 2, stage, score_ct_host));
-    } else {
-        // download only the first host_limbs limbs of every polynomial (exact compaction, see hann_compact_scores): the
-        // inverse transforms and the copy shrink with them
-        const int keep = c->host_limbs;
-        const int64_t npoly = p.nblk * 2, kw = (int64_t)keep * c->N;
-        CK(cudaMemcpy2DAsync(stage, (size_t)kw * 8, score, (size_t)c->L * c->N * 8, (size_t)kw * 8, (size_t)npoly, cudaMemcpyDeviceToDevice,
-                             c->stream));
-        RET(launch_ntt_inv(c, stage, npoly * keep, c->N, limbmap_first(keep)));
-        CK(cudaMemcpyAsync(score_ct_host, stage, (size_t)(npoly * kw) * 8, cudaMemcpyDeviceToHost, c->stream));
-    }
+    CK(ce);
+    for (int i = 0; i < 6; i++) CK(ej[i]);
     CK(cudaStreamSynchronize(c->stream));
     return HANN_OK;
 }

@@ -29,6 +29,19 @@ struct hann_ctx {
     cudaStream_t lane_stream[2] = {nullptr, nullptr};
     cudaEvent_t lane_join[2] = {nullptr, nullptr};
     std::vector<cudaEvent_t> blk_ev;  // one event per block: hann_score_level_host encodes a block as soon as its rows arrived
+    // hann_score_level_host: rows travel on up_stream, score ciphertexts on down_stream (both copy engines busy at once);
+    // grp_ev[i] marks group i's scores ready in the staging buffer, down_done the end of the downloads
+    cudaStream_t up_stream = nullptr, down_stream = nullptr;
+    cudaEvent_t down_done = nullptr;
+    std::vector<cudaEvent_t> grp_ev;
+    int host_groups = 0;  // block groups of hann_score_level_host (0: chosen from the level's size)
+    // hann_score_level_host scores its groups on two streams of their own (alternating), beside the encoding of the
+    // following groups on the context's stream; enc_ev[i]: group i is encoded; prep_done: the baby rotations are ready
+    cudaStream_t score_stream[2] = {nullptr, nullptr};
+    cudaEvent_t score_join[2] = {nullptr, nullptr};
+    cudaEvent_t prep_done = nullptr;
+    std::vector<cudaEvent_t> enc_ev;
+    int max_lanes = 4;  // block ranges hann_rotate_sum runs side by side
     u64 mod[HANN_MAXL1] = {};  // q_0..q_{L-1}, p
     LimbTable lt = {};
     LimbConst* lt_dev = nullptr;  // device copy of lt.c (the transform kernels read it from memory)
@@ -120,6 +133,7 @@ int launch_ntt_inv(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const 
 int launch_ntt_fwd_pass_b(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
 bool ntt_fwd_half_available(const hann_ctx* c, const void* data, int64_t stride);
 int launch_ntt_fwd_pass_b_half(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
+int launch_copy2d(hann_ctx* c, u64* dst, int64_t dst_pitch, const u64* src, int64_t src_pitch, int64_t width, int64_t rows);
 int launch_unpack_half(hann_ctx* c, const u64* half, int64_t npoly, u64* full);
 int launch_ntt_inv_pass_b(hann_ctx* c, u64* data, int64_t npoly, int64_t stride, const LimbMap& lm);
 bool ntt_inv_pass_b_gathers(const hann_ctx* c, const void* src, const void* dst);

@@ -589,6 +589,25 @@ int launch_rlk_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const u
     return check_launch(c, "rlk_finish");
 }
 
+// rows x width words, source and destination rows pitch words apart, copied by the SMs: a cudaMemcpy between device
+// buffers may be scheduled on a copy engine behind queued host transfers, which would stall the compute stream of
+// hann_score_level_host until all of a level's rows have arrived
+namespace {
+__global__ void __launch_bounds__(kThreads) k_copy2d(u64* __restrict__ dst, long long dst_pitch, const u64* __restrict__ src,
+                                                     long long src_pitch, long long width, long long rows) {
+    const long long total = rows * width;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const long long r = idx / width, x = idx % width;
+        dst[r * dst_pitch + x] = src[r * src_pitch + x];
+    }
+}
+}  // namespace
+int launch_copy2d(hann_ctx* c, u64* dst, int64_t dst_pitch, const u64* src, int64_t src_pitch, int64_t width, int64_t rows) {
+    if (width <= 0 || rows <= 0) return HANN_OK;
+    k_copy2d<<<grid_for(width * rows), kThreads, 0, c->stream>>>(dst, dst_pitch, src, src_pitch, width, rows);
+    return check_launch(c, "copy2d");
+}
+
 int launch_encrypt_block_finish(hann_ctx* c, const u64* pt, const u64* as, const u64* ehat, u64* ct, int64_t npt) {
     {
         KProf kp(c, KC_OTHER);

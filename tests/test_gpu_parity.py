@@ -136,7 +136,7 @@ def test_toy_other_baby_step_counts():
         run_level(p, synth.toy_corpus(1, rows=2048 + 77), synth.toy_query(2))
 
 
-@pytest.mark.parametrize("n_rows", [1500, 3000, 7000])   # 1, 2 and 4 blocks
+@pytest.mark.parametrize("n_rows", [1500, 3000, 7000, 15000])   # 1, 2, 4 and 8 blocks
 def test_host_buffer_level_matches_device_path(n_rows):
     ps = synth.TOY
     p = Pair(ps, key_seed=3)
@@ -154,6 +154,12 @@ def test_host_buffer_level_matches_device_path(n_rows):
     p.g.score_level_host(ct_g, rows, ws, small)
     p.g.set_tuning(p.b.TUNE_HOST_LIMBS, ps.L)
     assert np.array_equal(small, out[:, :, :1])
+    # any cut of the level into block groups (scored while later groups are still uploaded and encoded): same bits
+    for groups in (1, 2, 3, 4):
+        p.g.set_tuning(p.b.TUNE_HOST_GROUPS, groups)
+        ws_g = p.g.alloc(p.g.level_host_bytes(rows.shape[0]))
+        assert np.array_equal(p.g.score_level_host(ct_g, rows, ws_g), score_dev)
+    p.g.set_tuning(p.b.TUNE_HOST_GROUPS, 0)
 
 
 def test_full_ring_one_block():

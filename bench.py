@@ -122,14 +122,21 @@ def build_workload(config, rows_override=None, logn=16):
 
 FP64_LANES_PER_SM = 64  # binary64 multiply-add lanes per SM per clock
 
-# DRAM bytes (read + write) per unit of work of the bandwidth- or transform-bound kernels, from the ncu captures
-# summarised under profiles/ (small case: one block of 32,768 rows; traffic grows in proportion to the units)
-NCU_DRAM_BYTES_PER_UNIT = {
-    "ntt_fwd_b": ("polynomial", 490.4e6 / 512),
-    "fft_b": ("plaintext", 288.1e6 / 128),
-    "mac": ("block", None),
-    "ks_inner": ("item", None),
-}
+# DRAM bytes (read + write) per unit of work of the transform kernels, from the ncu captures summarised under profiles/
+# (small case: one block of 32,768 rows; traffic grows in proportion to the units): pass B of a half-size plaintext
+# transform, pass B of a full key-switch transform, the fused FFT tail + pass A per plaintext
+NCU_DRAM_BYTES = {"pass_b_plaintext_poly": 212.4e6 / 512, "pass_b_full_poly": 490.4e6 / 512, "fft_b_plaintext": 153.6e6 / 128}
+
+
+def ncu_traffic_per_step(kernel, ctx, n_blocks):
+    """DRAM traffic of one step of a kernel class, scaled from the ncu captures (None where none was taken)"""
+    L, B, G, R = ctx.L, ctx.B, ctx.G, ctx.R
+    if kernel == "ntt_fwd_b":
+        ks_polys = (L * (L + 1) + (B - 1) * 2 * L) + (G - 1) * n_blocks * (L * (L + 1) + 2 * L)
+        return n_blocks * R * L * NCU_DRAM_BYTES["pass_b_plaintext_poly"] + ks_polys * NCU_DRAM_BYTES["pass_b_full_poly"]
+    if kernel == "fft_b":
+        return n_blocks * R * NCU_DRAM_BYTES["fft_b_plaintext"]
+    return None
 
 
 def algorithmic_work(ctx, n_blocks, n_rows):
@@ -308,13 +315,13 @@ def run_ours(args):
     else:
         achieved, peak, runit = amount / dom_s / 1e12, SM_COUNT * FP64_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12, "T fp64 instr/s"
         psrc = "derived: %d SMs x %d fp64 lanes x %.0f MHz" % (SM_COUNT, FP64_LANES_PER_SM, sm_max_mhz)
-    unit_name, per_unit = NCU_DRAM_BYTES_PER_UNIT.get(dom, (None, None))
+    traffic_step = ncu_traffic_per_step(dom, ctx, nb)
     roofline = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,
                 "peak_source": psrc, "launches_per_step": kernels[dom]["launches_per_step"],
                 "avg_launch_ms": kernels[dom]["ms_per_step"] / dom_launches,
                 "algorithmic_per_launch": amount / dom_launches,
-                "traffic": per_unit * units / dom_launches if per_unit else None,
-                "traffic_source": ("ncu dram bytes per %s on the 1-block case x %s per launch" % (unit_name, unit_name)) if per_unit else None}
+                "traffic": traffic_step / dom_launches if traffic_step else None,
+                "traffic_source": "ncu dram bytes per polynomial on the 1-block case x polynomials per launch" if traffic_step else None}
     hbm_kernels = {}
     for k in ("mac", "ks_inner_keys", "ks_inner"):
         if k in kernels:

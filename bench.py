@@ -158,6 +158,14 @@ def algorithmic_work(ctx, n_blocks, n_rows):
     lift_src = [(L, L + 1), ((B - 1) * 2, L)] + [(items_rot * L, L + 1), (items_rot * 2, L)]  # (sources, targets each)
     lift_ops = sum(src * (1 + tgt) * a * (N // 2) * 8 for src, tgt in lift_src)
     pass_a_half = (N // 2) * 7 + (a - 1) * (N // 4) * 8  # first stage in full (one output per pair), then half the butterflies
+    # the transform kernels also move their polynomials through HBM once in and once out (half-size plaintexts: W/2 each
+    # way); whichever ceiling gives the longer ideal time is the bound the roofline reports
+    transform_bytes = {
+        "ntt_fwd_b": pt_polys * W + ks_polys * 2 * W,
+        "ntt_inv_b": inv_polys * 2 * W,
+        "fft_b": n_blocks * R * (n * 16 + L * (W // 2)),
+    }
+    algorithmic_work.transform_bytes = transform_bytes
     return {
         "mac": ("hbm", n_blocks * R * L * (W // 2) + B * 2 * L * W + n_blocks * G * 2 * L * W, n_blocks),
         # one digit set under B-1 streamed keys (query_prepare) / one key under many digit sets (rotate_sum, L2-resident key)
@@ -309,17 +317,31 @@ def run_ours(args):
     bound, amount, units = work[dom]
     dom_s = kernels[dom]["ms_per_step"] * 1e-3
     dom_launches = max(kernels[dom]["launches_per_step"], 1)
+    alu_peak = SM_COUNT * FP64_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12
+    other = None
+    if bound == "alu":
+        # a transform kernel has two ceilings: its binary64 instructions and its polynomial bytes; report the tighter
+        tbytes = algorithmic_work.transform_bytes.get(dom)
+        alu_frac = amount / dom_s / 1e12 / alu_peak
+        if tbytes:
+            hbm_frac = tbytes / dom_s / 1e9 / hbm_peak
+            if hbm_frac > alu_frac:
+                other = {"bound": "alu", "achieved": amount / dom_s / 1e12, "peak": alu_peak, "unit": "T fp64 instr/s", "frac": alu_frac}
+                bound, amount = "hbm", tbytes
+            else:
+                other = {"bound": "hbm", "achieved": tbytes / dom_s / 1e9, "peak": hbm_peak, "unit": "GB/s", "frac": hbm_frac}
     if bound == "hbm":
         achieved, peak, runit = amount / dom_s / 1e9, hbm_peak, "GB/s"
         psrc = peak_src + " copy bandwidth"
     else:
-        achieved, peak, runit = amount / dom_s / 1e12, SM_COUNT * FP64_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12, "T fp64 instr/s"
+        achieved, peak, runit = amount / dom_s / 1e12, alu_peak, "T fp64 instr/s"
         psrc = "derived: %d SMs x %d fp64 lanes x %.0f MHz" % (SM_COUNT, FP64_LANES_PER_SM, sm_max_mhz)
     traffic_step = ncu_traffic_per_step(dom, ctx, nb)
     roofline = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,
                 "peak_source": psrc, "launches_per_step": kernels[dom]["launches_per_step"],
                 "avg_launch_ms": kernels[dom]["ms_per_step"] / dom_launches,
                 "algorithmic_per_launch": amount / dom_launches,
+                "other_ceiling": other,
                 "traffic": traffic_step / dom_launches if traffic_step else None,
                 "traffic_source": "ncu dram bytes per polynomial on the 1-block case x polynomials per launch" if traffic_step else None}
     hbm_kernels = {}

@@ -81,3 +81,5 @@ def test_algorithmic_work_matches_the_per_row_figures():
         ks_polys = (L * (L + 1) + (B - 1) * 2 * L) + (G - 1) * n_blocks * (L * (L + 1) + 2 * L)
         assert w["ntt_fwd_b"][2] == pt_polys + ks_polys
         assert w["ntt_fwd_b"][1] == (pt_polys * (N // 4) + ks_polys * (N // 2)) * 8 * 8
+        # and the bytes those transforms move: half-size plaintext polynomials W/2 in and out, key-switch polynomials W
+        assert bench.algorithmic_work.transform_bytes["ntt_fwd_b"] == (pt_polys + 2 * ks_polys) * 8 * N

@@ -26,11 +26,12 @@ class Query:
         ct_o, ct_g = p.query(qR)
         assert np.array_equal(ct_o, ct_g)
         self.ct_o = ct_o
+        self.ct_g = ct_g
         self.ct_dev = p.g.import_(p.b.KIND_CT, ct_g, 1)
         self.baby = p.g.query_prepare(self.ct_dev, p.ws)
         self.baby_o = p.o.baby_set(ct_o, p.evk_o) if with_oracle else None
 
-    def score_level(self, rows, oracle_blocks=(), compact=False, one_call=False):
+    def score_level(self, rows, oracle_blocks=(), compact=False, one_call=False, host=False):
         """GPU scores of a level [n_rows]; blocks listed in oracle_blocks are compared bit for bit with the oracle"""
         p, g, b, ps = self.p, self.p.g, self.p.b, self.p.ps
         n_rows = rows.shape[0]
@@ -56,6 +57,11 @@ class Query:
             assert np.array_equal(pt_g, pt_o), "encoded plaintexts of block %d" % blk
             assert np.array_equal(in_g, in_o), "partial sums of block %d" % blk
             assert np.array_equal(score_h[blk], sc_o), "score ciphertext of block %d" % blk
+        if host:
+            # the end-to-end call bench.py times: host buffers in, block groups scored while later groups upload
+            ws_host = g.alloc(g.level_host_bytes(n_rows))
+            assert np.array_equal(g.score_level_host(self.ct_g, np.ascontiguousarray(rows), ws_host), score_h)
+            del ws_host
         got = g.decrypt_scores(p.km.s, score_h).reshape(-1)[:n_rows]
         want = rows.astype(np.float64) @ self.qR.astype(np.float64)
         err = float(np.abs(got - want).max())
@@ -79,10 +85,10 @@ class Query:
 
 def test_face_like_level_full(pair16):
     """222,049 rows, 512 -> 128 dims, N = 2^16: 7 blocks, the last 77.6 % full.  First and last block at every
-    conformance point, every row within 2^-18."""
+    conformance point, every row within 2^-18; the host-buffer call (three block groups) returns the same ciphertexts."""
     ps, lvl, qR, planted = wl.face_level()
     q = Query(pair16, qR)
-    got, want = q.score_level(lvl.rows, oracle_blocks=(0, 6), compact=True)
+    got, want = q.score_level(lvl.rows, oracle_blocks=(0, 6), compact=True, host=True)
     assert got.shape == (222_049,)
     # a quarter of the bytes on the wire (one limb instead of four) still ranks the same neighbours first
     assert np.array_equal(wl.topk_ids(q.compact_scores, lvl.ids, 10), wl.topk_ids(want, lvl.ids, 10))

@@ -27,7 +27,6 @@ sys.path.insert(0, ROOT)
 
 METRIC = "encrypted candidates scored/sec"
 UNIT = "candidates/s"
-SM_COUNT = 148
 
 
 def read_peaks():
@@ -119,8 +118,6 @@ def build_workload(config, rows_override=None, logn=16):
         return ps, lvl.rows, q, "sweep: %d wanted rows inflated x4 to %d scored rows, dim 128, N=2^%d" % (base, lvl.rows.shape[0], ps.logN)
     raise SystemExit("unknown config %r" % config)
 
-
-FP64_LANES_PER_SM = 64  # binary64 multiply-add lanes per SM per clock
 
 # DRAM bytes (read + write) per unit of work of the transform kernels, from the ncu captures summarised under profiles/
 # (small case: one block of 32,768 rows; traffic grows in proportion to the units): pass B of a half-size plaintext
@@ -245,18 +242,34 @@ def run_ours(args):
     sampler.start()
     for _ in range(max(args.warmup, 3)):
         step()
-    l0 = ctx.get_stats()["launches"]
+    # The timed quantity is a block of exactly K steps between two events.  The block is repeated back to back (no host
+    # synchronisation in between) until the timed region has lasted MIN_TIMED_S, so that the clocks are sampled tens of times
+    # under sustained load whatever K is; the reported time is the MEDIAN block, the slowest rank's.
     barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(args.steps):
-        step()
-    e1.record()
+    t_probe = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_probe[0].record()
+    step()
+    t_probe[1].record()
+    torch.cuda.synchronize()
+    est_block_ms = max(t_probe[0].elapsed_time(t_probe[1]) * args.steps, 1e-3)
+    n_timed_blocks = int(min(max(1, np.ceil(args.min_timed_s * 1e3 / est_block_ms)), 2000))
+    if dist is not None:  # every rank runs the same number of blocks
+        nbt = torch.tensor([n_timed_blocks], device=ctx.device)
+        dist.all_reduce(nbt, op=dist.ReduceOp.MAX)
+        n_timed_blocks = int(nbt.item())
+    l0 = ctx.get_stats()["launches"]
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_timed_blocks + 1)]
+    barrier()
+    marks[0].record()
+    for bi in range(n_timed_blocks):
+        for _ in range(args.steps):
+            step()
+        marks[bi + 1].record()
     barrier()
     clocks = sampler.stop()
-    ms_total = e0.elapsed_time(e1)
-    launches = ctx.get_stats()["launches"] - l0
-    ms_step = max_over_ranks(ms_total, dist, ctx.device) / args.steps
+    block_ms = [marks[i].elapsed_time(marks[i + 1]) for i in range(n_timed_blocks)]
+    launches = (ctx.get_stats()["launches"] - l0) // n_timed_blocks
+    ms_step = max_over_ranks(float(np.median(block_ms)), dist, ctx.device) / args.steps
     value = replica_throughput(n_rows, world, ms_step * 1e-3)
 
     # correctness of what was timed: decrypted scores against float64 dot products
@@ -312,30 +325,38 @@ def run_ours(args):
     kernels = {k: {"ms_per_step": v[0] / aux_steps, "launches_per_step": v[1] / aux_steps, "share": v[0] / total_k}
                for k, v in kt.items() if v[1]}
     hbm_peak, sm_max_mhz, peak_src = read_peaks()
+    # arithmetic ceilings measured on this device by the library's own probe kernels: register-resident binary64 modular
+    # butterflies (no memory traffic) and 32 x 32 -> 64 multiply-adds
+    bfly_peak, madd_peak = ctx.probe_rates()
     work = algorithmic_work(ctx, nb, n_rows)
     dom = max((k for k in kernels if k in work), key=lambda k: kernels[k]["ms_per_step"])
     bound, amount, units = work[dom]
     dom_s = kernels[dom]["ms_per_step"] * 1e-3
     dom_launches = max(kernels[dom]["launches_per_step"], 1)
-    alu_peak = SM_COUNT * FP64_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12
+    # transform work is counted in binary64 instructions, 8 per modular butterfly; the measured ceiling is in butterflies
+    alu_peak = bfly_peak / 1e12
+    alu_src = "measured: register-resident binary64 modular butterflies of the library's probe kernel"
     other = None
     if bound == "alu":
-        # a transform kernel has two ceilings: its binary64 instructions and its polynomial bytes; report the tighter
+        # a transform kernel has two ceilings: its butterflies and its polynomial bytes; report the tighter
         tbytes = algorithmic_work.transform_bytes.get(dom)
+        amount = amount / 8.0
         alu_frac = amount / dom_s / 1e12 / alu_peak
         if tbytes:
             hbm_frac = tbytes / dom_s / 1e9 / hbm_peak
             if hbm_frac > alu_frac:
-                other = {"bound": "alu", "achieved": amount / dom_s / 1e12, "peak": alu_peak, "unit": "T fp64 instr/s", "frac": alu_frac}
+                other = {"bound": "alu", "achieved": amount / dom_s / 1e12, "peak": alu_peak, "unit": "T butterflies/s", "frac": alu_frac,
+                         "peak_source": alu_src}
                 bound, amount = "hbm", tbytes
             else:
-                other = {"bound": "hbm", "achieved": tbytes / dom_s / 1e9, "peak": hbm_peak, "unit": "GB/s", "frac": hbm_frac}
+                other = {"bound": "hbm", "achieved": tbytes / dom_s / 1e9, "peak": hbm_peak, "unit": "GB/s", "frac": hbm_frac,
+                         "peak_source": peak_src + " copy bandwidth"}
     if bound == "hbm":
         achieved, peak, runit = amount / dom_s / 1e9, hbm_peak, "GB/s"
         psrc = peak_src + " copy bandwidth"
     else:
-        achieved, peak, runit = amount / dom_s / 1e12, alu_peak, "T fp64 instr/s"
-        psrc = "derived: %d SMs x %d fp64 lanes x %.0f MHz" % (SM_COUNT, FP64_LANES_PER_SM, sm_max_mhz)
+        achieved, peak, runit = amount / dom_s / 1e12, alu_peak, "T butterflies/s"
+        psrc = alu_src
     traffic_step = ncu_traffic_per_step(dom, ctx, nb)
     roofline = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,
                 "peak_source": psrc, "launches_per_step": kernels[dom]["launches_per_step"],
@@ -344,11 +365,21 @@ def run_ours(args):
                 "other_ceiling": other,
                 "traffic": traffic_step / dom_launches if traffic_step else None,
                 "traffic_source": "ncu dram bytes per polynomial on the 1-block case x polynomials per launch" if traffic_step else None}
+    # the streaming kernels against both of THEIR ceilings: bytes against the measured copy bandwidth, and residue
+    # products (three 32 x 32 -> 64 multiply-adds each) against the measured multiply-add rate
+    L_, N_, B_, G_, R_ = ctx.L, ctx.N, ctx.B, ctx.G, ctx.R
+    products = {"mac": nb * R_ * L_ * N_ * 2,
+                "ks_inner_keys": (B_ - 1) * L_ * 2 * (L_ + 1) * N_,
+                "ks_inner": (G_ - 1) * nb * L_ * 2 * (L_ + 1) * N_}
     hbm_kernels = {}
     for k in ("mac", "ks_inner_keys", "ks_inner"):
         if k in kernels:
-            gbs = work[k][1] / (kernels[k]["ms_per_step"] * 1e-3) / 1e9
-            hbm_kernels[k] = {"GB/s": gbs, "frac_of_measured_copy": gbs / hbm_peak, "frac_of_8TBps_nominal": gbs / 8000.0}
+            sec = kernels[k]["ms_per_step"] * 1e-3
+            gbs = work[k][1] / sec / 1e9
+            madds = 3.0 * products[k] / sec
+            hbm_kernels[k] = {"GB/s": gbs, "frac_of_measured_copy": gbs / hbm_peak, "frac_of_8TBps_nominal": gbs / 8000.0,
+                              "T_madds_per_s": madds / 1e12, "frac_of_measured_madd_rate": madds / madd_peak,
+                              "tighter_ceiling": "hbm" if gbs / hbm_peak >= madds / madd_peak else "multiply-add"}
 
     # end to end through the host-buffer entry point: pinned host inputs, copies inside the timed region
     rows_pin = torch.from_numpy(rows_np).pin_memory()
@@ -406,7 +437,10 @@ def run_ours(args):
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64",
+            "ms_per_step": ms_step, "timed_blocks": {"count": n_timed_blocks, "steps_each": args.steps, "reported": "median block",
+                                                     "ms_min": float(min(block_ms)), "ms_max": float(max(block_ms)),
+                                                     "region_s": float(sum(block_ms)) * 1e-3},
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64",
             "data": "synthetic",
             "config": {"workload": wname, "rows": n_rows, "blocks": nb, "R": ps.R, "B": ps.B, "G": ps.G, "logN": ps.logN, "L": ps.L,
                        "l2": "working set per step (%.1f GB of encoded plaintexts) exceeds L2; no flush" %
@@ -415,7 +449,10 @@ def run_ours(args):
             "ms_per_query_level": ms_step, "stage_ms": stage_ms,
             # candidates already encoded and resident (the paper's "warm" case): prepare + multiply-accumulate + rotate-and-sum
             "warm_value": world * n_rows / ((stage_ms["query_prepare"] + stage_ms["score_level"] + stage_ms["rotate_sum"]) * 1e-3),
-            "kernels": kernels, "hbm_kernels": hbm_kernels, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
+            "kernels": kernels, "hbm_kernels": hbm_kernels, "roofline": roofline,
+            "measured_ceilings": {"f64_butterflies_per_s": bfly_peak, "int32_madds_per_s": madd_peak, "hbm_gbs": hbm_peak,
+                                  "ntt_butterflies_per_s": {k: work[k][1] / 8.0 / (kernels[k]["ms_per_step"] * 1e-3)
+                                                            for k in ("ntt_fwd_b", "ntt_inv_b", "lift_digits") if k in kernels}}, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": int(launches), "clocks": clocks, "compaction": compaction,
             "check": {"max_abs_score_error": max_err, "tolerance": 2.0 ** ps.tol_log2, "ok": check_ok},
         }
@@ -606,8 +643,42 @@ def oracle_setup(ps, qR, km):
     return o, ct, evk
 
 
+def oracle_single_thread(ps, rows_np, qR, km, n_rows, o, ct, evk):
+    """The oracle on ONE thread.  Its work is a sum of independent operations with no reuse between them (every rotation,
+    every plaintext encoding, every plaintext x ciphertext product is computed from scratch), so the level's time is the
+    time of one operation of each kind, measured on one thread, times the number of such operations: B-1 rotations for the
+    query, and per block R encodings, R plaintext x ciphertext products and G-1 rotations."""
+    import ctypes
+    from oracle.oracle import Oracle
+
+    omp = ctypes.CDLL("libgomp.so.1")
+    threads = o.num_threads()
+    omp.omp_set_num_threads(1)
+    try:
+        t0 = time.perf_counter()
+        o.rotate(ct, 1, evk[0])
+        t_rot = time.perf_counter() - t0
+        one = Oracle(ps.logN, ps.q, ps.p, ps.log_scale, 1, 1)   # R = B = 1: one diagonal, one product
+        col = np.ascontiguousarray(rows_np[: ps.n, :1])
+        t0 = time.perf_counter()
+        pt1 = one.encode_block(col)
+        t_enc = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        one.mac(pt1, ct[None])
+        t_mac = time.perf_counter() - t0
+    finally:
+        omp.omp_set_num_threads(threads)
+    nb = (n_rows + ps.n - 1) // ps.n
+    total = (ps.B - 1) * t_rot + nb * (ps.R * (t_enc + t_mac) + (ps.G - 1) * t_rot)
+    return {"value": n_rows / total, "unit": UNIT, "cores": 1,
+            "sample": "one rotation (%.2f s), one plaintext encoding (%.3f s) and one plaintext x ciphertext product (%.3f s) timed "
+                      "on one thread; level time = (B-1) rotations + blocks x (R encodings + R products + (G-1) rotations)"
+                      % (t_rot, t_enc, t_mac)}
+
+
 def cpu_baseline(ps, rows_np, qR, km, n_rows):
-    """the oracle as it stands on the host cores: one query_prepare + one block, scaled to the level by block count"""
+    """the oracle as it stands on the host cores: one query_prepare + one block, scaled to the level by block count; and the
+    same level on a single thread"""
     o, ct, evk = oracle_setup(ps, qR, km)
     t0 = time.perf_counter()
     baby = o.baby_set(ct, evk)
@@ -616,9 +687,11 @@ def cpu_baseline(ps, rows_np, qR, km, n_rows):
     o.score_block(rows_np[: ps.n], baby, evk[ps.B - 1])
     t_blk = time.perf_counter() - t0
     nb = (n_rows + ps.n - 1) // ps.n
+    single = oracle_single_thread(ps, rows_np, qR, km, n_rows, o, ct, evk) if ps.B > 1 else None
     return {"value": n_rows / (t_prep + nb * t_blk), "unit": UNIT, "cores": o.num_threads(), "kind": "oracle",
             "sample": "query_prepare once (%.1f s) + block 0 of %d (%d rows, %.1f s) timed; level time = prepare + blocks x "
-                      "block time (per-block work is constant)" % (t_prep, nb, min(ps.n, n_rows), t_blk)}
+                      "block time (per-block work is constant)" % (t_prep, nb, min(ps.n, n_rows), t_blk),
+            "single_thread": single}
 
 
 def run_hierarchy(args):
@@ -732,6 +805,18 @@ def run_reference(args):
     return 0
 
 
+def relaunch_under_torchrun(n, argv=None):
+    """run this script again as n ranks on this node and return the launcher's exit code"""
+    import socket
+
+    with socket.socket() as sk:  # a free port for the rendezvous
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n), "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + list(sys.argv[1:] if argv is None else argv)
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -741,6 +826,7 @@ def main():
     ap.add_argument("--config", type=int, default=1, help="0 toy, 1 face-like level (default), 2 DataComp-like and 3 Deep1B-like "
                     "hierarchies (latency per level), 4 scaling sweep point (--rows = wanted rows, --logn 15|16)")
     ap.add_argument("--logn", type=int, default=16, help="ring of the sweep configuration")
+    ap.add_argument("--min-timed-s", type=float, default=2.0, help="the K-step block is repeated until the timed region lasted this long")
     ap.add_argument("--rows", type=int, default=None, help="override the row count (debugging, ncu captures)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--encode-group", type=int, default=None, help="tuning: plaintexts per encode launch group")
@@ -750,6 +836,10 @@ def main():
     ap.add_argument("--staged", action="store_true", help="with --lean: run the steps as the per-kernel timing pass does")
     ap.add_argument("--lean", action="store_true", help="only run warm-up + steps (for ncu); prints no JSON line")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as `python bench.py --gpus N`: become N ranks, one per GPU, under torch's launcher (independent replicas;
+        # rank 0 prints the line)
+        return relaunch_under_torchrun(args.gpus)
     if args.impl == "reference":
         args.steps = 2 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup

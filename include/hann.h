@@ -22,7 +22,10 @@
  *     `hann_rotate_sum`, `hann_keyswitch`) allocate nothing: all temporaries live in the caller's
  *     workspace `ws` (256-byte aligned device memory, `ws_bytes` long; `hann_workspace_bytes` says how
  *     much is enough; HANN_EWORKSPACE if it is too short) -- the counterpart of the paper's single
- *     pre-allocated arena, Sec. 3.4.  One workspace serves one call at a time.
+ *     pre-allocated arena, Sec. 3.4.  One workspace serves one call at a time.  Two exceptions, both outside the
+ *     steady state: while the per-launch profile (hann_kernel_profile) is on, every launch takes a CUDA event pair
+ *     from a pool that grows on demand; and hann_score_level_host creates one event per block and per block group
+ *     the first time it sees a level of that size (later calls of the same or a smaller size create nothing).
  *   - Canonical exchange layout (the only layout with a meaning outside the library): coefficient
  *     domain, natural coefficient order, residues in [0, q_i), uint64, index order [poly][limb][coeff];
  *     a ciphertext is 2 polynomials (c0, c1) of L limbs.  The internal device layout (transform domain,
@@ -107,9 +110,18 @@ int64_t hann_sizeof(const hann_ctx *ctx, int what);
 /* Bytes of workspace the server-side calls need when at most `max_blocks` blocks are processed per call. */
 int64_t hann_workspace_bytes(const hann_ctx *ctx, int64_t max_blocks);
 
-/* Block until everything enqueued on the context's stream has finished; reports asynchronous CUDA errors. */
+/* Block until everything enqueued on the context's stream has finished; reports asynchronous CUDA errors and a
+ * kernel that gave up a bounded wait (HANN_ECUDA, once: the report clears the condition).  Every host-pointer call
+ * (hann_import, hann_export, hann_export_limbs, hann_expand_uniform, hann_score_level_host, the client half) ends
+ * with the same check, so HANN_OK from any of them means that no kernel of the call was abandoned. */
 int hann_sync(hann_ctx *ctx);
 const char *hann_last_error(const hann_ctx *ctx);
+
+/* ---- test, profiling and measurement hooks (not part of the scoring product; nothing on the hot path calls them) ----
+ * hann_selftest_bounded_wait, hann_set_timing / hann_get_stats, hann_kernel_profile / hann_kernel_times,
+ * hann_probe_rates, hann_debug_check.  (The Python binding's HANN_LIB environment variable, which makes it load
+ * another build of this library for A/B comparisons, is a hook of the same kind.) */
+
 /* Self-test of the failure path of the bulk-copy kernels: launches one warp that waits, for limit_ms (1..1000), on a
  * completion barrier that nothing completes.  The wait runs out, the kernel raises the context's flag and returns; the
  * NEXT hann_sync therefore reports HANN_ECUDA ("a kernel gave up a bounded wait") and clears the flag, after which the
@@ -143,6 +155,12 @@ const char *hann_kernel_name(int cls);
 int hann_kernel_profile(hann_ctx *ctx, int enable);
 int hann_kernel_times(hann_ctx *ctx, double *ms, uint64_t *launches);
 
+/* Measured arithmetic ceilings of the device (a set-up class call: allocates and frees a small buffer, synchronises):
+ * binary64 modular butterflies per second of the register-resident round the transform kernels run (no memory traffic:
+ * the rate no transform can exceed) and 32-bit integer multiply-adds per second (the multiply-accumulate spends three per
+ * residue product).  bench.py reports the transform and multiply-accumulate kernels against these. */
+int hann_probe_rates(hann_ctx *ctx, double *f64_butterflies_per_s, double *int32_madds_per_s);
+
 /* ---- client side (host memory in and out; Sec. 2, The round trip, client steps) -------------------------- */
 
 /* Evaluation keys for the left slot rotations rot[0..n_rot) from caller-drawn randomness (hybrid key switching,
@@ -155,6 +173,13 @@ int hann_kernel_times(hann_ctx *ctx, double *ms, uint64_t *launches);
  *   evk_out [n_rot][L][2][L+1][N]  canonical; [..][j][0] = b_j, [..][j][1] = a_j */
 int hann_keygen_from_samples(hann_ctx *ctx, const int8_t *s, int n_rot, const int32_t *rot, const uint64_t *a,
                              const int8_t *e, uint64_t *evk_out);
+
+/* The same keys from a 64-bit seed (Sec. 2, The round trip, client step 1: the client owns the secret key and hands the
+ * server the evaluation keys): the ternary secret, the uniform halves and the rounded-Gaussian errors (sigma = 3.2) are
+ * all drawn from the counter hash of hann_expand_uniform (streams 16..19; the uniform halves on the device) -- a
+ * benchmark generator, NOT a cryptographic one.  A rotation's key depends on (seed, rotation) only, not on the list it
+ * is generated with.  s_out [N] int8 receives the secret; evk_out as in hann_keygen_from_samples. */
+int hann_keygen_seeded(hann_ctx *ctx, uint64_t seed, int n_rot, const int32_t *rot, int8_t *s_out, uint64_t *evk_out);
 
 /* Relinearisation key (Sec. 2, encrypted database): the evaluation key for s' = s*s in the layout of
  * hann_keygen_from_samples for ONE key; a [L][L+1][N], e [L][N], evk_out [L][2][L+1][N].  hann_load_keys takes it under
@@ -192,20 +217,24 @@ int hann_decrypt_compact(hann_ctx *ctx, const int8_t *s, const uint64_t *ct, int
  * context.  Needed later: rotations 1..B-1 for hann_query_prepare, rotation B for hann_rotate_sum. */
 int hann_load_keys(hann_ctx *ctx, const uint64_t *evk, int n_rot, const int32_t *rot);
 
-/* Once per query: the B rotated copies rot_r(ct), r = 0..B-1, each taken directly from the input ciphertext
- * (key switch of the automorphed c1; the digit decomposition is shared by all rotations).
+/* Once per query (Sec. 3.1 Detail: the baby steps of the diagonal method; Sec. 3.4: the rotated query is computed
+ * once and reused by every block and level): the B rotated copies rot_r(ct), r = 0..B-1, each taken directly from
+ * the input ciphertext (key switch of the automorphed c1; the digit decomposition is shared by all rotations).
  *   ct_dev   one ciphertext, internal layout (device)
  *   baby_dev HANN_SIZE_BABY bytes (device), internal layout [B][2][L][N] */
 int hann_query_prepare(hann_ctx *ctx, const void *ct_dev, void *baby_dev, void *ws, size_t ws_bytes);
 
-/* Encode candidate rows into plaintext blocks.  rows_dev [n_rows][dim] float32 row-major (device), dim <= R
+/* Encode candidate rows into plaintext blocks (Sec. 2, storage paragraph: a block of n rows is held as R diagonals;
+ * Sec. 3.1 Detail: each diagonal is shifted by the giant-step amount in plaintext, so the server needs no database
+ * rotation keys).  rows_dev [n_rows][dim] float32 row-major (device), dim <= R
  * (rows are zero-padded to R).  Block blk holds rows blk*n .. blk*n+n-1 (missing rows are zero).  For g < G,
  * b < B plaintext (g,b) of a block encodes the slot vector z[i] = M[(i - g*B) mod n][(i + b) mod R] at scale
  * Delta, reduced into every ciphertext prime and transformed.
  *   pt_dev  ceil(n_rows/n) * HANN_SIZE_PT_BLOCK bytes (device), internal layout [blk][G][B][L][N/2] */
 int hann_encode_candidates(hann_ctx *ctx, const float *rows_dev, int64_t n_rows, int dim, void *pt_dev, void *ws, size_t ws_bytes);
 
-/* Multiply-accumulate of one level: inner[blk][g] = sum_b pt[blk][g][b] * baby[b] (both ciphertext components,
+/* Multiply-accumulate of one level (Sec. 3.1 "How": the diagonal matrix-vector product; Sec. 3.2 "How": every level
+ * is one call to the same stateless scorer): inner[blk][g] = sum_b pt[blk][g][b] * baby[b] (both ciphertext components,
  * every limb).   inner_dev n_blocks * HANN_SIZE_INNER bytes (device), internal layout [blk][G][2][L][N]. */
 int hann_score_level(hann_ctx *ctx, const void *baby_dev, const void *pt_dev, int64_t n_blocks, void *inner_dev,
                      void *ws, size_t ws_bytes);
@@ -228,12 +257,13 @@ int hann_score_level_batch(hann_ctx *ctx, const void *baby_dev, int n_queries, c
 int hann_score_level_ctdb(hann_ctx *ctx, const void *baby_dev, const void *ctdb_dev, int64_t n_blocks, void *inner_dev,
                           void *ws, size_t ws_bytes);
 
-/* Rotate-and-sum: score_ct[blk] = sum_g rot_{g*B}(inner[blk][g]), evaluated by Horner with the single key of
+/* Rotate-and-sum (Sec. 3.1 Detail: the giant steps of the diagonal method): score_ct[blk] = sum_g rot_{g*B}(inner[blk][g]), evaluated by Horner with the single key of
  * rotation B: acc = inner[G-1]; for g = G-2..0: acc = rot_B(acc) + inner[g].
  *   score_ct_dev n_blocks * HANN_SIZE_CT bytes (device), internal layout. */
 int hann_rotate_sum(hann_ctx *ctx, const void *inner_dev, int64_t n_blocks, void *score_ct_dev, void *ws, size_t ws_bytes);
 
-/* One routing level for one query, device buffers in and out: hann_query_prepare, hann_encode_candidates,
+/* One routing level for one query, device buffers in and out (Sec. 2 "Reproducing this": level + candidates +
+ * encrypted query in, encrypted score vector out): hann_query_prepare, hann_encode_candidates,
  * hann_score_level and hann_rotate_sum in sequence, except that the query preparation runs on a helper stream beside
  * the candidate encoding (they are independent; both finish before the multiply-accumulate starts).  All buffers as in
  * the four calls; `ws` must hold hann_workspace_bytes(ctx, blocks).  On return everything is enqueued on the context's
@@ -241,11 +271,15 @@ int hann_rotate_sum(hann_ctx *ctx, const void *inner_dev, int64_t n_blocks, void
 int hann_query_level(hann_ctx *ctx, const void *ct_dev, const float *rows_dev, int64_t n_rows, int dim, void *baby_dev,
                      void *pt_dev, void *inner_dev, void *score_ct_dev, void *ws, size_t ws_bytes);
 
-/* Hybrid key switch of one polynomial d (internal layout, L limbs) with the loaded key of rotation `rot`, WITHOUT
+/* Hybrid key switch (the operation behind every rotation of Sec. 3.1 and the relinearisation of Sec. 2's encrypted
+ * database; the paper takes it from its CKKS library, the conventions are stated above) of one polynomial d (internal
+ * layout, L limbs) with the loaded key of rotation `rot`, WITHOUT
  * applying the automorphism to d: outputs (ks0, ks1), L limbs each, with ks0 + ks1*s ~ d*s(X^k).
  * Steps: digits [d]_{q_j} (inverse transform), centred lift into all L+1 moduli, transform, inner product with
  * the key, ModDown: out_i = (u_i - centred([u]_p)) * p^{-1} mod q_i. */
 int hann_keyswitch(hann_ctx *ctx, int rot, const void *poly_dev, void *ks0_dev, void *ks1_dev, void *ws, size_t ws_bytes);
+/* Bytes of (256-byte aligned) workspace one hann_keyswitch call carves; never more than hann_workspace_bytes(ctx, 1). */
+int64_t hann_keyswitch_bytes(const hann_ctx *ctx);
 
 /* (No counterpart in the paper.)  hann_keyswitch for callers that can neither allocate device memory nor lend a
  * workspace -- for instance a request handler that must avoid the device-wide synchronisation of cudaMalloc/cudaFree,
@@ -256,8 +290,9 @@ int hann_keyswitch(hann_ctx *ctx, int rot, const void *poly_dev, void *ks0_dev, 
  *     naming both sizes; use hann_keyswitch there.
  *   - The call performs no cudaMalloc/cudaFree and calls no allocating routine; it returns HANN_EINVAL while the
  *     per-launch profile (hann_kernel_profile) is on, because that profile creates events on demand.
- *   - The first call on a device looks up the array's device address (once per device, with the context's device
- *     current); make that first call before starting any stream capture.
+ *   - The array's device address is looked up once per device, by hann_ctx_create (with the context's device
+ *     current), so that this call only reads a cached address; if that look-up did not happen, the first call on the
+ *     device does it -- so create the context (or make a first call) before starting any stream capture.
  *   - All calls on one device share the one array, which keeps whatever the last call left in it (nothing needs
  *     clearing: every part is written before it is read).  Two calls whose kernels overlap on the GPU -- different
  *     streams, different contexts, different threads -- race on it; serialise them. */
@@ -301,7 +336,8 @@ int64_t hann_compact_bytes(const hann_ctx *ctx, int64_t n_blocks, int keep);
 int hann_compact_scores(hann_ctx *ctx, const void *score_ct_dev, int64_t n_blocks, int keep, int rescale, void *out_dev,
                         void *ws, size_t ws_bytes);
 
-/* One level end to end from HOST buffers (copies included): the query ciphertext goes up first and its baby set is
+/* One level end to end from HOST buffers, copies included (Sec. 2 "Reproducing this": one request of the persistent
+ * scoring server): the query ciphertext goes up first and its baby set is
  * prepared on a helper stream; the rows follow block by block on an upload stream and every block is encoded as soon as
  * its rows have arrived; the level is cut into groups of blocks (HANN_TUNE_HOST_GROUPS), and a group's multiply-
  * accumulate, rotate-and-sum and export run on scoring streams while later groups are still uploaded and encoded, its

@@ -23,7 +23,7 @@
  * Layout of every polynomial crossing this API ("canonical"): coefficient domain, natural
  * order, residues in [0, q_i), uint64, index order [poly][limb][coeff].
  *
- * Pins (tests/test_oracle_*.py): primes by independent primality test; NTT round trip and
+ * Pins (tests/test_oracle_pins.py): primes by independent primality test; NTT round trip and
  * NTT product == schoolbook product (python integers) for N <= 256; encode == exact cosine
  * sum evaluated in multi-precision; automorphism == slot roll; decrypt(encrypt(m)) - m == e;
  * key-switch error within the analytic noise bound and ModDown(p*x) == x; rotate via

@@ -75,6 +75,8 @@ def load_library():
         "hann_kernel_profile": (C.c_int, [vp, C.c_int]),
         "hann_kernel_times": (C.c_int, [vp, vp, vp]),
         "hann_keygen_from_samples": (C.c_int, [vp, vp, C.c_int, vp, vp, vp, vp]),
+        "hann_keygen_seeded": (C.c_int, [vp, C.c_uint64, C.c_int, vp, vp, vp]),
+        "hann_probe_rates": (C.c_int, [vp, vp, vp]),
         "hann_encrypt_query": (C.c_int, [vp, vp, vp, C.c_int, vp, vp, vp]),
         "hann_decrypt_scores": (C.c_int, [vp, vp, vp, i64, C.c_int, vp, vp]),
         "hann_load_keys": (C.c_int, [vp, vp, C.c_int, vp]),
@@ -90,6 +92,7 @@ def load_library():
         "hann_keyswitch": (C.c_int, [vp, C.c_int, vp, vp, vp, vp, sz]),
         "hann_query_level": (C.c_int, [vp, vp, vp, i64, C.c_int, vp, vp, vp, vp, vp, sz]),
         "hann_static_scratch_bytes": (i64, []),
+        "hann_keyswitch_bytes": (i64, [vp]),
         "hann_keyswitch_static": (C.c_int, [vp, C.c_int, vp, vp, vp]),
         "hann_import": (C.c_int, [vp, C.c_int, vp, i64, vp]),
         "hann_export": (C.c_int, [vp, C.c_int, vp, i64, vp]),
@@ -221,6 +224,21 @@ class Context:
         evk = np.empty((len(rots), L, 2, L + 1, N), dtype=np.uint64)
         self._ck(self.lib.hann_keygen_from_samples(self.h, _ptr(s), len(rots), _ptr(rots), _ptr(a), _ptr(e), _ptr(evk)))
         return evk
+
+    def keygen_seeded(self, seed, rots):
+        """secret key [N] int8 and evaluation keys [len(rots)][L][2][L+1][N] drawn from a 64-bit seed"""
+        rots = _np(rots, np.int32)
+        L, N = self.L, self.N
+        s = np.empty(N, dtype=np.int8)
+        evk = np.empty((len(rots), L, 2, L + 1, N), dtype=np.uint64)
+        self._ck(self.lib.hann_keygen_seeded(self.h, seed, len(rots), _ptr(rots), _ptr(s), _ptr(evk)))
+        return s, evk
+
+    def probe_rates(self):
+        """(binary64 modular butterflies/s, int32 multiply-adds/s) measured on the context's device"""
+        a, b = C.c_double(0.0), C.c_double(0.0)
+        self._ck(self.lib.hann_probe_rates(self.h, C.byref(a), C.byref(b)))
+        return a.value, b.value
 
     def keygen_relin_from_samples(self, s, a, e):
         s, a, e = _np(s, np.int8), _np(a, np.uint64), _np(e, np.int8)

@@ -5,6 +5,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "internal.h"
 
@@ -31,6 +32,22 @@ int fail(hann_ctx* c, int code, const char* msg) {
 }
 
 inline int64_t align256(int64_t x) { return (x + 255) & ~(int64_t)255; }
+
+// Waits for the context's stream, then reads and clears the word a kernel raises when it gives up a bounded wait for an
+// asynchronous copy.  Every entry point that synchronises ends with this, so a call that returns HANN_OK has results that
+// no aborted kernel produced.  (The word lives in mapped page-locked host memory: reading it costs no copy.)
+int sync_and_check(hann_ctx* c) {
+    cudaError_t e_ = cudaStreamSynchronize(c->stream);
+    if (e_ != cudaSuccess) {
+        c->err = std::string("cudaStreamSynchronize: ") + cudaGetErrorString(e_);
+        return HANN_ECUDA;
+    }
+    if (*(volatile int*)c->kflag_host) {
+        *(volatile int*)c->kflag_host = 0;
+        return fail(c, HANN_ECUDA, "a kernel gave up a bounded wait for an asynchronous copy; results of the last calls are invalid");
+    }
+    return HANN_OK;
+}
 
 // bump allocator over a caller-provided workspace
 struct Arena {
@@ -98,6 +115,19 @@ int64_t prepare_words(const hann_ctx* c) {
 }
 
 constexpr int64_t kSlack = 16 * 256;  // room for the alignment of a dozen sub-buffers
+
+// the four sub-buffers of ONE key switch (hann_keyswitch, hann_keyswitch_static): input copy, digits, u, lifted
+struct KsBuffers {
+    u64 *c1c, *digits, *u, *lifted;
+};
+bool carve_keyswitch(const hann_ctx* c, Arena& ar, KsBuffers& b) {
+    const int64_t L = c->L, N = c->N;
+    b.c1c = ar.take<u64>(L * N);
+    b.digits = ar.take<u64>(L * (L + 1) * N);
+    b.u = ar.take<u64>(2 * (L + 1) * N);
+    b.lifted = ar.take<u64>(2 * L * N);
+    return b.c1c && b.digits && b.u && b.lifted;
+}
 
 // canonical (host or device) -> internal: copy, forward transform of count polynomials of L limbs
 int import_polys(hann_ctx* c, const u64* canonical, int64_t npolyL, u64* dst) {
@@ -171,6 +201,16 @@ int ks_digits_to_lifted(hann_ctx* c, u64* c1c, int64_t items, u64* digits, int64
 }  // namespace
 
 int ntt_configure(hann_ctx* c);
+int static_scratch_resolve(hann_ctx* c, void** out);
+
+// bytes of 256-byte aligned workspace one hann_keyswitch needs: measured by running its own carving on an empty arena
+int64_t keyswitch_ws_bytes(const hann_ctx* c) {
+    Arena ar{nullptr, 0, INT64_MAX / 2};
+    KsBuffers kb;
+    ar.base = (char*)256;  // any non-null base: the carving only does pointer arithmetic
+    carve_keyswitch(c, ar, kb);
+    return ar.off;
+}
 
 // ================================================================================================ context
 
@@ -277,17 +317,19 @@ extern "C" int hann_ctx_create(const hann_params* prm, hann_ctx** out) {
     const size_t twb = (size_t)(L + 1) * N * 16;
     bool ok = cudaMalloc(&c->tw_fwd, twb) == cudaSuccess && cudaMalloc(&c->tw_inv, twb) == cudaSuccess &&
               cudaMalloc(&c->tw_fwd_f64, twb) == cudaSuccess && cudaMalloc(&c->tw_inv_f64, twb) == cudaSuccess &&
-              cudaMalloc(&c->lt_dev, sizeof(LimbTable)) == cudaSuccess && cudaMalloc(&c->kflag, sizeof(int)) == cudaSuccess &&
+              cudaMalloc(&c->lt_dev, sizeof(LimbTable)) == cudaSuccess &&
+              cudaHostAlloc((void**)&c->kflag_host, sizeof(int), cudaHostAllocMapped) == cudaSuccess &&
+              cudaHostGetDevicePointer((void**)&c->kflag, c->kflag_host, 0) == cudaSuccess &&
               cudaMalloc(&c->fft_T, nh * sizeof(double2)) == cudaSuccess && cudaMalloc(&c->fft_U, n * sizeof(double2)) == cudaSuccess &&
               cudaMalloc(&c->jinv, n * sizeof(int32_t)) == cudaSuccess && cudaMalloc(&c->galois_dev, n * sizeof(unsigned)) == cudaSuccess &&
               cudaMalloc(&c->keytab_dev, n * sizeof(u64*)) == cudaSuccess;
     if (ok) {
+        *c->kflag_host = 0;
         ok = cudaMemcpy(c->tw_fwd, twf.data(), twb, cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->tw_inv, twi.data(), twb, cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->tw_fwd_f64, twf64.data(), twb, cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->tw_inv_f64, twi64.data(), twb, cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->lt_dev, &c->lt, sizeof(LimbTable), cudaMemcpyHostToDevice) == cudaSuccess &&
-             cudaMemset(c->kflag, 0, sizeof(int)) == cudaSuccess &&
              cudaMemcpy(c->fft_T, T.data(), nh * sizeof(double2), cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->fft_U, U.data(), n * sizeof(double2), cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->jinv, jpos.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess &&
@@ -314,6 +356,13 @@ extern "C" int hann_ctx_create(const hann_params* prm, hann_ctx** out) {
              cudaEventCreateWithFlags(&c->score_join[i], cudaEventDisableTiming) == cudaSuccess;
     if (ok) ok = cudaEventCreateWithFlags(&c->prep_done, cudaEventDisableTiming) == cudaSuccess;
     if (ok) ok = ntt_configure(c) == HANN_OK;
+    if (ok) {
+        // look up the built-in scratch of hann_keyswitch_static now, while this device is current, so that the request-time
+        // call only reads a cached address (a failure here is reported by that call, not by context creation)
+        void* unused = nullptr;
+        static_scratch_resolve(c, &unused);
+        c->err.clear();
+    }
     if (!ok) {
         cudaGetLastError();
         hann_ctx_destroy(c);
@@ -329,7 +378,8 @@ extern "C" void hann_ctx_destroy(hann_ctx* c) {
     cudaStreamSynchronize(c->stream);
     for (u64* k : c->keytab_host)
         if (k) cudaFree(k);
-    cudaFree(c->tw_fwd); cudaFree(c->tw_inv); cudaFree(c->tw_fwd_f64); cudaFree(c->tw_inv_f64); cudaFree(c->lt_dev); cudaFree(c->kflag);
+    cudaFree(c->tw_fwd); cudaFree(c->tw_inv); cudaFree(c->tw_fwd_f64); cudaFree(c->tw_inv_f64); cudaFree(c->lt_dev);
+    if (c->kflag_host) cudaFreeHost(c->kflag_host);
     cudaFree(c->fft_T); cudaFree(c->fft_U); cudaFree(c->jinv); cudaFree(c->galois_dev); cudaFree(c->keytab_dev);
     if (c->scratch) cudaFree(c->scratch);
     if (c->aux_stream) {
@@ -396,17 +446,12 @@ extern "C" int64_t hann_workspace_bytes(const hann_ctx* c, int64_t max_blocks) {
     return w + kSlack;
 }
 
+extern "C" int64_t hann_keyswitch_bytes(const hann_ctx* c) { return c ? keyswitch_ws_bytes(c) : HANN_EINVAL; }
+
 extern "C" int hann_sync(hann_ctx* c) {
     if (!c) return HANN_EINVAL;
     DeviceGuard dg(c->device);
-    CK(cudaStreamSynchronize(c->stream));
-    int flag = 0;
-    CK(cudaMemcpy(&flag, c->kflag, sizeof(int), cudaMemcpyDeviceToHost));
-    if (flag) {
-        cudaMemset(c->kflag, 0, sizeof(int));
-        return fail(c, HANN_ECUDA, "a kernel gave up a bounded wait for an asynchronous copy; results of the last calls are invalid");
-    }
-    return HANN_OK;
+    return sync_and_check(c);
 }
 
 extern "C" int hann_selftest_bounded_wait(hann_ctx* c, int limit_ms, double* waited_ms) {
@@ -517,11 +562,11 @@ extern "C" int hann_import(hann_ctx* c, int kind, const uint64_t* canonical, int
             CK(cudaMemcpy2DAsync((u64*)internal_dev + p0 * (LN / 2), (size_t)c->n * 8, c->scratch, (size_t)c->N * 8, (size_t)c->n * 8,
                                  (size_t)np * c->L, cudaMemcpyDeviceToDevice, c->stream));
         }
-        CK(cudaStreamSynchronize(c->stream));
+        RET(sync_and_check(c));
         return HANN_OK;
     }
     RET(import_polys(c, canonical, count * pk, (u64*)internal_dev));
-    CK(cudaStreamSynchronize(c->stream));
+    RET(sync_and_check(c));
     return HANN_OK;
 }
 
@@ -533,7 +578,7 @@ extern "C" int hann_expand_uniform(hann_ctx* c, uint64_t seed, uint64_t stream, 
     RET(ensure_scratch(c, LN * 8));
     RET(launch_expand_uniform(c, seed, stream, (u64*)c->scratch));
     CK(cudaMemcpyAsync(a_out, c->scratch, LN * 8, cudaMemcpyDefault, c->stream));
-    CK(cudaStreamSynchronize(c->stream));
+    RET(sync_and_check(c));
     return HANN_OK;
 }
 
@@ -567,7 +612,7 @@ extern "C" int hann_export(hann_ctx* c, int kind, const void* internal_dev, int6
         }
         RET(export_polys(c, (const u64*)internal_dev + p0 * c->L * c->N, np, (u64*)c->scratch, canonical_out + p0 * c->L * c->N));
     }
-    CK(cudaStreamSynchronize(c->stream));
+    RET(sync_and_check(c));
     return HANN_OK;
 }
 
@@ -585,7 +630,7 @@ extern "C" int hann_export_limbs(hann_ctx* c, const void* internal_dev, int64_t 
         RET(launch_ntt_inv(c, staging, np * limbs, c->N, limbmap_first(limbs)));
         CK(cudaMemcpyAsync(canonical_out + p0 * pw, staging, np * pw * 8, cudaMemcpyDefault, c->stream));
     }
-    CK(cudaStreamSynchronize(c->stream));
+    RET(sync_and_check(c));
     return HANN_OK;
 }
 
@@ -677,7 +722,34 @@ extern "C" int hann_keygen_from_samples(hann_ctx* c, const int8_t* s, int n_rot,
                                cudaMemcpyDeviceToHost, c->stream));
             memcpy(out_r + ((int64_t)j * 2 + 1) * (L + 1) * W, a_r + (int64_t)j * (L + 1) * W, (size_t)(L + 1) * W * 8);
         }
-        CK(cudaStreamSynchronize(c->stream));  // sprime (host) is reused by the next rotation
+        RET(sync_and_check(c));  // sprime (host) is reused by the next rotation
+    }
+    return HANN_OK;
+}
+
+extern "C" int hann_keygen_seeded(hann_ctx* c, uint64_t seed, int n_rot, const int32_t* rot, int8_t* s_out, uint64_t* evk_out) {
+    if (!c) return HANN_EINVAL;
+    if (!rot || !s_out || !evk_out || n_rot < 0) return fail(c, HANN_EINVAL, "hann_keygen_seeded: bad argument");
+    const int L = c->L, N = c->N;
+    for (int i = 0; i < n_rot; i++)
+        if (rot[i] < 1 || rot[i] >= c->n) return fail(c, HANN_ESHAPE, "hann_keygen_seeded: rotation out of range");
+    // streams of the counter hash: 16 secret, 17 uniform halves of the keys, 18/19 the two Box-Muller sub-streams
+    hm::seeded_ternary(seed, 16, N, s_out);
+    const int64_t keyw = (int64_t)L * (L + 1) * N;
+    std::vector<u64> a((size_t)keyw);
+    std::vector<int8_t> e((size_t)L * N);
+    for (int r = 0; r < n_rot; r++) {
+        {
+            DeviceGuard dg(c->device);
+            RET(ensure_scratch(c, keyw * 8));
+            // counters are keyed by the ROTATION, not by its place in the list: a rotation's key does not depend on
+            // which other keys are generated with it
+            RET(launch_expand_uniform_qp(c, seed, 17, (u64)rot[r] * (u64)keyw, (u64*)c->scratch));
+            CK(cudaMemcpyAsync(a.data(), c->scratch, keyw * 8, cudaMemcpyDeviceToHost, c->stream));
+            RET(sync_and_check(c));
+        }
+        hm::seeded_gaussian(seed, 18, (u64)rot[r] * (u64)L * N, (long)L * N, 3.2, e.data());
+        RET(hann_keygen_from_samples(c, s_out, 1, rot + r, a.data(), e.data(), evk_out + (int64_t)r * 2 * keyw));
     }
     return HANN_OK;
 }
@@ -711,7 +783,7 @@ extern "C" int hann_keygen_relin_from_samples(hann_ctx* c, const int8_t* s, cons
                            cudaMemcpyDeviceToHost, c->stream));
         memcpy(evk_out + ((int64_t)j * 2 + 1) * (L + 1) * W, a + (int64_t)j * (L + 1) * W, (size_t)(L + 1) * W * 8);
     }
-    CK(cudaStreamSynchronize(c->stream));
+    RET(sync_and_check(c));
     return HANN_OK;
 }
 
@@ -748,7 +820,7 @@ extern "C" int hann_encrypt_block(hann_ctx* c, const int8_t* s, const void* pt_d
         RET(launch_ntt_fwd(c, EH, (int64_t)np * L, N, limbmap_q(c)));
         // c0 = pt - a*s + e, written at ct + 2 r * LN (the finish kernel strides its output by 2 * LN)
         RET(launch_encrypt_block_finish(c, pt + (int64_t)r0 * (LN / 2), AS, EH, ct + (int64_t)r0 * 2 * LN, np));
-        CK(cudaStreamSynchronize(c->stream));  // e8 is reused by the next piece
+        RET(sync_and_check(c));  // e8 is reused by the next piece
     }
     return HANN_OK;
 }
@@ -786,7 +858,7 @@ extern "C" int hann_encrypt_query(hann_ctx* c, const int8_t* s, const float* q, 
     RET(launch_ntt_inv(c, AS, L, N, limbmap_q(c)));
     RET(launch_encrypt_finish(c, AS, e8, M, AS));
     CK(cudaMemcpyAsync(ct_out, AS, LN * 8, cudaMemcpyDeviceToHost, c->stream));
-    CK(cudaStreamSynchronize(c->stream));
+    RET(sync_and_check(c));
     memcpy(ct_out + LN, a, LN * 8);
     return HANN_OK;
 }
@@ -817,7 +889,7 @@ static int decrypt_impl(hann_ctx* c, const int8_t* s, const uint64_t* ct, int64_
         RET(launch_add(c, MU, CT, MU, nl, lm));              // + c0
         RET(launch_ntt_inv(c, MU, nl, N, lm));
         CK(cudaMemcpyAsync(mu.data(), MU, LN * 8, cudaMemcpyDeviceToHost, c->stream));
-        CK(cudaStreamSynchronize(c->stream));
+        RET(sync_and_check(c));
         hm::crt_to_real(mu.data(), nl, N, c->mod, real.data());
         // slots: a_k = (mu_k + i mu_{k+n}) conj(U[k]);  z_j * scale = sum_k a_k exp(+2 pi i u_j k / n)
         for (int k = 0; k < n; k++) {
@@ -882,7 +954,7 @@ extern "C" int hann_load_keys(hann_ctx* c, const uint64_t* evk, int n_rot, const
         const unsigned kinv = c->h_galois[(c->n - r) % c->n];  // 5^{-r} = 5^{n-r} (5 has order n modulo 2N)
         (void)k;
         RET(launch_permute(c, tmp, c->keytab_host[r], (int64_t)L * 2 * (L + 1), kinv));
-        CK(cudaStreamSynchronize(c->stream));
+        RET(sync_and_check(c));
     }
     CK(cudaMemcpy(c->keytab_dev, c->keytab_host.data(), c->keytab_host.size() * sizeof(u64*), cudaMemcpyHostToDevice));
     return HANN_OK;
@@ -1115,16 +1187,13 @@ extern "C" int hann_keyswitch(hann_ctx* c, int rot, const void* poly_dev, void* 
     if (rot < 1 || rot >= c->n) return fail(c, HANN_ESHAPE, "hann_keyswitch: rotation out of range");
     if (!c->keytab_host[rot]) return fail(c, HANN_ENOKEY, "hann_keyswitch: key not loaded");
     if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_keyswitch: workspace missing or not 256-byte aligned");
-    const int L = c->L, N = c->N;
-    const int64_t LN = (int64_t)L * N, L1N = (int64_t)(L + 1) * N;
+    const int L = c->L;
     DeviceGuard dg(c->device);
     Timer tm(c, 4);
     Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
-    u64* c1c = ar.take<u64>(LN);
-    u64* digits = ar.take<u64>(L * L1N);
-    u64* u = ar.take<u64>(2 * L1N);
-    u64* lifted = ar.take<u64>(2 * LN);
-    if (!c1c || !digits || !u || !lifted) return fail(c, HANN_EWORKSPACE, "hann_keyswitch: workspace too small");
+    KsBuffers kb;
+    if (!carve_keyswitch(c, ar, kb)) return fail(c, HANN_EWORKSPACE, "hann_keyswitch: workspace too small");
+    u64 *c1c = kb.c1c, *digits = kb.digits, *u = kb.u, *lifted = kb.lifted;
     // the stored key is phi_k^{-1}(evk): switch phi_k^{-1}(d) and apply phi_k to the result
     const unsigned kinv = c->h_galois[(c->n - rot) % c->n];
     RET(launch_permute(c, (const u64*)poly_dev, c1c, L, kinv));
@@ -1311,6 +1380,6 @@ extern "C" int hann_score_level_host(hann_ctx* c, const uint64_t* ct_host, const
     RET(rc);
     CK(ce);
     for (int i = 0; i < 6; i++) CK(ej[i]);
-    CK(cudaStreamSynchronize(c->stream));
+    RET(sync_and_check(c));
     return HANN_OK;
 }

@@ -27,6 +27,11 @@ __device__ __forceinline__ void tensor_load_2d(unsigned dst, const void* tmap, i
                  "l"(tmap), "r"(x), "r"(y), "r"(bar)
                  : "memory");
 }
+// the context's error word lives in mapped host memory: a plain store, made visible to the host before the kernel ends
+__device__ __forceinline__ void raise_flag(int* kflag) {
+    *(volatile int*)kflag = 1;
+    __threadfence_system();
+}
 __device__ __forceinline__ unsigned long long global_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));

@@ -229,4 +229,37 @@ void fft_inplace(double* re, double* im, int n, int logn, int sign) {
     }
 }
 
+static u64 mix64(u64 x) {
+    x ^= x >> 32;
+    x *= 0x9E3779B97F4A7C15ULL;
+    x ^= x >> 29;
+    x *= 0xBB67AE8584CAA73BULL;
+    x ^= x >> 32;
+    return x;
+}
+
+u64 hash64(u64 seed, u64 stream, u64 ctr) {
+    const u64 a = mix64(seed + 0x9E3779B97F4A7C15ULL);
+    const u64 b = mix64(a ^ (stream * 0xBB67AE8584CAA73BULL));
+    return mix64(b + ctr * 0x9E3779B97F4A7C15ULL);
+}
+
+void seeded_ternary(u64 seed, u64 stream, int N, int8_t* s) {
+    // the top 32 bits times 3, shifted down: uniform on {0, 1, 2} up to 2^-32
+    for (int x = 0; x < N; x++) s[x] = (int8_t)((int)(((hash64(seed, stream, (u64)x) >> 32) * 3) >> 32) - 1);
+}
+
+void seeded_gaussian(u64 seed, u64 stream, u64 ctr0, long count, double sigma, int8_t* e) {
+    const double two_pi = 6.283185307179586476925286766559;
+    for (long i = 0; i < count; i++) {
+        // u1 in (0, 1], u2 in [0, 1): 53-bit uniforms from two sub-streams
+        const double u1 = (double)((hash64(seed, stream, ctr0 + (u64)i) >> 11) + 1) * 0x1p-53;
+        const double u2 = (double)(hash64(seed, stream + 1, ctr0 + (u64)i) >> 11) * 0x1p-53;
+        double v = std::nearbyint(sigma * std::sqrt(-2.0 * std::log(u1)) * std::cos(two_pi * u2));
+        if (v > 127) v = 127;
+        if (v < -127) v = -127;
+        e[i] = (int8_t)v;
+    }
+}
+
 }  // namespace hm

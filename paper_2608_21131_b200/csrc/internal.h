@@ -45,7 +45,10 @@ struct hann_ctx {
     u64 mod[HANN_MAXL1] = {};  // q_0..q_{L-1}, p
     LimbTable lt = {};
     LimbConst* lt_dev = nullptr;  // device copy of lt.c (the transform kernels read it from memory)
-    int* kflag = nullptr;         // device word raised by a kernel that gave up a bounded wait; read by hann_sync
+    // word raised by a kernel that gave up a bounded wait: mapped page-locked host memory (kflag is its device address), read
+    // and cleared after the synchronisation that ends every host-pointer call and hann_sync
+    int* kflag = nullptr;
+    int* kflag_host = nullptr;
     // transform tables on the device, [L+1][N][2]: (w, floor(w*2^64/q)) for w = psi^brev(k) and psi^-brev(k)
     u64 *tw_fwd = nullptr, *tw_inv = nullptr;
     // the same twiddles for the binary64 transform path, [L+1][N][2] doubles: (balanced w, fl(w / q))
@@ -122,7 +125,14 @@ void unit_root(long t, long den, double* c, double* s);  // exp(2 pi i t/den), c
 // residues [L][N] -> centred integers in (-Q/2, Q/2] as long double
 void crt_to_real(const u64* res, int L, int N, const u64* q, long double* out);
 void fft_inplace(double* re, double* im, int n, int logn, int sign);
+u64 hash64(u64 seed, u64 stream, u64 ctr);  // the 64-bit counter hash of the seeded calls (see hann_expand_uniform)
+void seeded_ternary(u64 seed, u64 stream, int N, int8_t* s);                       // uniform on {-1, 0, 1}
+void seeded_gaussian(u64 seed, u64 stream, u64 ctr0, long count, double sigma, int8_t* e);  // rounded Gaussian (Box-Muller)
 }  // namespace hm
+
+// bytes of workspace one hann_keyswitch carves (api.cu); device address of the built-in scratch (static_scratch.cu)
+int64_t keyswitch_ws_bytes(const hann_ctx* c);
+int static_scratch_resolve(hann_ctx* c, void** out);
 
 // ---- launchers: each enqueues on ctx->stream, counts its launches and returns HANN_OK or HANN_ECUDA
 int check_launch(hann_ctx* c, const char* what);
@@ -183,6 +193,8 @@ int launch_evk_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const i
 int launch_encrypt_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const u64* m, u64* c0_out);
 // a[L][N] = counter hash of (seed, stream, l*N + x) mod q_l (coefficient domain, canonical)
 int launch_expand_uniform(hann_ctx* c, u64 seed, u64 stream, u64* a);
+// a[L][L+1][N] = counter hash of (seed, stream, ctr0 + index) reduced into the modulus of each of the L+1 limbs
+int launch_expand_uniform_qp(hann_ctx* c, u64 seed, u64 stream, u64 ctr0, u64* a);
 // encrypted database: relinearisation key finish, block encryption finish, ct x ct multiply-accumulate
 int launch_rlk_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const u64* s2, u64* b_out);
 int launch_encrypt_block_finish(hann_ctx* c, const u64* pt, const u64* as, const u64* ehat, u64* ct, int64_t npt);

@@ -382,6 +382,14 @@ __global__ void __launch_bounds__(kThreads) k_expand_uniform(u64* __restrict__ a
         a[idx] = barrett64(mix64(b + (u64)idx * 0x9E3779B97F4A7C15ULL), lt.c[(int)(idx / N)]);
 }
 
+// the same generator over the L+1 moduli of an evaluation key: a[j][i][x] = h(seed, stream, ctr0 + (j (L+1) + i) N + x) mod m_i
+__global__ void __launch_bounds__(kThreads) k_expand_uniform_qp(u64* __restrict__ a, u64 seed, u64 stream, u64 ctr0, int N, int L, LimbTable lt) {
+    const long long total = (long long)L * (L + 1) * N;
+    const u64 b = mix64(mix64(seed + 0x9E3779B97F4A7C15ULL) ^ (stream * 0xBB67AE8584CAA73BULL));
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads)
+        a[idx] = barrett64(mix64(b + (ctr0 + (u64)idx) * 0x9E3779B97F4A7C15ULL), lt.c[(int)((idx / N) % (L + 1))]);
+}
+
 // symmetric encryption finish, coefficient domain: c0[l][x] = -as[l][x] + e[x] + m[l][x]
 __global__ void __launch_bounds__(kThreads) k_encrypt_finish(const u64* __restrict__ as, const int8_t* __restrict__ e,
                                                              const u64* __restrict__ m, u64* __restrict__ c0, int N, int L,
@@ -622,6 +630,14 @@ int launch_expand_uniform(hann_ctx* c, u64 seed, u64 stream, u64* a) {
         k_expand_uniform<<<grid_for((int64_t)c->L * c->N), kThreads, 0, c->stream>>>(a, seed, stream, c->N, c->L, c->lt);
     }
     return check_launch(c, "expand_uniform");
+}
+
+int launch_expand_uniform_qp(hann_ctx* c, u64 seed, u64 stream, u64 ctr0, u64* a) {
+    {
+        KProf kp(c, KC_OTHER);
+        k_expand_uniform_qp<<<grid_for((int64_t)c->L * (c->L + 1) * c->N), kThreads, 0, c->stream>>>(a, seed, stream, ctr0, c->N, c->L, c->lt);
+    }
+    return check_launch(c, "expand_uniform_qp");
 }
 
 int launch_encrypt_finish(hann_ctx* c, const u64* as_coeff, const int8_t* e, const u64* m, u64* c0_out) {

@@ -302,7 +302,7 @@ __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ ba
         const int st = i % kMacStages;
         const bool arrived = mbar_wait(bar0 + 8 * st, (unsigned)(i / kMacStages) & 1u);
         if (!arrived && lane == 0) {
-            atomicExch(kflag, 1);
+            raise_flag(kflag);
             s_abort = 1;
         }
         u64 cur[BB];

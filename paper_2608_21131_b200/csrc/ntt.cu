@@ -321,7 +321,7 @@ __device__ __forceinline__ void fwd_b8t_body(const NttArgs& A, int groups, int* 
         if (!tile_valid(i)) break;  // warp-uniform
         const int s = i & 1;
         if (!mbar_wait(bar0 + 8 * s, (unsigned)(i >> 1) & 1u)) {
-            if (lane == 0) atomicExch(kflag, 1);
+            if (lane == 0) raise_flag(kflag);
             // the copy into the other buffer may still be in flight: give it the same bounded time, then stop
             if (tile_valid(i + 1)) mbar_wait(bar0 + 8 * (s ^ 1), (unsigned)((i + 1) >> 1) & 1u);
             return;
@@ -429,7 +429,7 @@ __global__ void __launch_bounds__(256, 3) k_ntt_inv_b8t(NttArgs A, int groups, i
         if (!tile_valid(i)) break;  // warp-uniform
         const int s = i & 1;
         if (!mbar_wait(bar0 + 8 * s, (unsigned)(i >> 1) & 1u)) {
-            if (lane == 0) atomicExch(kflag, 1);
+            if (lane == 0) raise_flag(kflag);
             if (tile_valid(i + 1)) mbar_wait(bar0 + 8 * (s ^ 1), (unsigned)((i + 1) >> 1) & 1u);
             return;
         }
@@ -471,7 +471,7 @@ __global__ void k_wait_selftest(int* kflag, unsigned long long limit_ns, unsigne
     const bool arrived = mbar_wait(b, 0, limit_ns);
     if (threadIdx.x == 0) {
         *waited_ns = global_ns() - t0;
-        if (!arrived) atomicExch(kflag, 1);
+        if (!arrived) raise_flag(kflag);
     }
 }
 

@@ -20,9 +20,12 @@ constexpr int kMaxDevices = 64;
 std::mutex g_mu;
 void* g_scratch_addr[kMaxDevices] = {};  // device address of g_static_scratch, per device ordinal
 
+}  // namespace
+
 // In host code `g_static_scratch` is only a handle for the runtime, not an address a kernel could use; the device
-// address has to be asked for, once per device, while that device is current.
-int static_scratch_address(hann_ctx* c, void** out) {
+// address has to be asked for, once per device, while that device is current.  hann_ctx_create does so (a request-time
+// call then only reads the cached address); the entry point itself asks again if that has not happened.
+int static_scratch_resolve(hann_ctx* c, void** out) {
     if (c->device < 0 || c->device >= kMaxDevices) {
         c->err = "hann_keyswitch_static: device ordinal out of range";
         return HANN_EINVAL;
@@ -46,8 +49,6 @@ int static_scratch_address(hann_ctx* c, void** out) {
     return HANN_OK;
 }
 
-}  // namespace
-
 extern "C" int64_t hann_static_scratch_bytes(void) { return (int64_t)HANN_STATIC_SCRATCH_BYTES; }
 
 extern "C" int hann_keyswitch_static(hann_ctx* c, int rot, const void* poly_dev, void* ks0_dev, void* ks1_dev) {
@@ -57,9 +58,8 @@ extern "C" int hann_keyswitch_static(hann_ctx* c, int rot, const void* poly_dev,
         c->err = "hann_keyswitch_static: switch the per-launch profile off first";
         return HANN_EINVAL;
     }
-    // one key switch needs: permuted input, digits, u, lifted (same carving as hann_keyswitch)
-    const int64_t L = c->L, N = c->N;
-    const int64_t ks_need = (L * N + L * (L + 1) * N + 2 * (L + 1) * N + 2 * L * N) * 8 + 16 * 256;
+    // what hann_keyswitch carves from its workspace: permuted input, digits, u, lifted
+    const int64_t ks_need = keyswitch_ws_bytes(c);
     if (ks_need > (int64_t)HANN_STATIC_SCRATCH_BYTES) {
         c->err = "hann_keyswitch_static: ring too large for the built-in scratch (" + std::to_string(ks_need) + " bytes needed, " +
                  std::to_string(HANN_STATIC_SCRATCH_BYTES) + " available); use hann_keyswitch with a workspace";
@@ -71,7 +71,7 @@ extern "C" int hann_keyswitch_static(hann_ctx* c, int rot, const void* poly_dev,
         return HANN_ECUDA;
     }
     void* scratch = nullptr;
-    int rc = static_scratch_address(c, &scratch);
+    int rc = static_scratch_resolve(c, &scratch);
     // Nothing in the scratch has to start at zero: each sub-buffer is fully written by one kernel before the next
     // one reads it, so the previous call's contents are simply overwritten.
     if (rc == HANN_OK) rc = hann_keyswitch(c, rot, poly_dev, ks0_dev, ks1_dev, scratch, (size_t)HANN_STATIC_SCRATCH_BYTES);

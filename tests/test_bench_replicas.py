@@ -48,6 +48,20 @@ def test_reference_arm_runs_on_rank_zero_only():
     assert out.returncode == 0 and out.stdout.strip() == ""
 
 
+def test_gpus_flag_launches_the_ranks_itself():
+    """`python bench.py --gpus 2` with no launcher around it starts two ranks under torch's launcher (rendezvous on
+    127.0.0.1, a free port) and rank 0 prints the one JSON line -- exercised on CPU with the reference arm (the oracle on
+    the toy configuration), whose other rank exits without work"""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference", "--config", "0",
+                          "--steps", "1", "--warmup", "0"], capture_output=True, text=True, timeout=600, env=env, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    rec = json.loads(lines[0])
+    assert rec["impl"] == "reference" and rec["n_gpus"] == 2 and rec["value"] > 0 and rec["cpu_baseline"]["kind"] == "oracle"
+
+
 def test_single_process_identity():
     sys.path.insert(0, ROOT)
     import torch

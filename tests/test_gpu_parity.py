@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 
 from paper_2608_21131_b200 import synth
-from tests.helpers import Pair
+from tests.helpers import Pair, make_oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -475,6 +475,84 @@ def test_bounded_wait_runs_out_and_is_reported():
     assert ei.value.code == b.ECUDA and "bounded wait" in str(ei.value)
     g.sync()                                    # the flag is cleared
     run_level(p, synth.toy_corpus(5, rows=900, dim=16), synth.toy_query(6, dim=16))   # and the context still computes
+
+
+def test_abandoned_kernel_is_reported_by_every_synchronising_call():
+    """A kernel that gave up a bounded wait must not go unnoticed by a caller that never calls hann_sync: the next call that
+    synchronises (an export, the host-buffer level) returns HANN_ECUDA once, and the same call then succeeds."""
+    from paper_2608_21131_b200 import binding as b
+
+    ps = synth.small_params(10, 16, 4, L=2)
+    p = Pair(ps, key_seed=2)
+    g = p.g
+    poly = g.alloc(g.sizeof(b.SIZE_POLY))
+    poly.zero_()
+    g.selftest_bounded_wait(1)
+    with pytest.raises(b.HannError) as ei:
+        g.export(b.KIND_POLY, poly, 1)
+    assert ei.value.code == b.ECUDA and "bounded wait" in str(ei.value)
+    assert not g.export(b.KIND_POLY, poly, 1).any()
+    rows, qv = synth.toy_corpus(5, rows=700, dim=16), synth.toy_query(6, dim=16)
+    ct = g.encrypt_query(p.km.s, qv, p.km.ct_a, p.km.ct_e)
+    ws = g.alloc(g.level_host_bytes(rows.shape[0]))
+    want = g.score_level_host(ct, rows, ws)
+    g.selftest_bounded_wait(1)
+    with pytest.raises(b.HannError) as ei:
+        g.score_level_host(ct, rows, ws)
+    assert ei.value.code == b.ECUDA
+    assert np.array_equal(g.score_level_host(ct, rows, ws), want)
+    g.selftest_bounded_wait(1)
+    with pytest.raises(b.HannError):
+        g.expand_uniform(1, 2)
+    g.sync()
+
+
+def test_seeded_key_generation_round_trip_and_statistics():
+    """hann_keygen_seeded: the keys rotate a ciphertext correctly (decrypts to the rolled slots), depend on (seed, rotation)
+    only, and the drawn secret / errors / uniform halves have the statistics of their distributions.  The evaluation keys
+    equal what hann_keygen_from_samples gives for the same samples, recovered from the key itself: a_j is stored in the
+    key, and e_j = b_j + a_j s - F_j s' is small."""
+    from paper_2608_21131_b200 import binding as b
+
+    ps = synth.small_params(12, 16, 4, L=2)
+    g = b.Context(ps)
+    o = make_oracle(ps)
+    s, evk = g.keygen_seeded(77, [1, 2, 3, 4])
+    s2, evk2 = g.keygen_seeded(77, [3])
+    assert np.array_equal(s, s2) and np.array_equal(evk[2], evk2[0])       # a key depends on (seed, rotation) only
+    s3, evk3 = g.keygen_seeded(78, [3])
+    assert not np.array_equal(s, s3) and not np.array_equal(evk3[0], evk2[0])
+    # statistics: ternary secret close to uniform on {-1, 0, 1}; uniform halves spread over [0, q)
+    assert set(np.unique(s).tolist()) == {-1, 0, 1}
+    for v in (-1, 0, 1):
+        assert abs(float(np.mean(s == v)) - 1 / 3) < 0.03
+    a = evk[:, :, 1]                                                          # [rot][j][L+1][N]
+    mods = np.array(list(ps.q) + [ps.p], dtype=np.float64)
+    u = a.astype(np.float64) / mods[None, None, :, None]
+    assert abs(u.mean() - 0.5) < 0.005 and abs(u.std() - 12 ** -0.5) < 0.005
+    # errors: e_j = b_j + a_j s - F_j s' over limb 0, recovered with the oracle's exact products
+    k = o.galois(1)
+    sq = np.array([(int(x) % ps.q[0]) for x in s], dtype=np.uint64)
+    sp = o.automorphism(0, k, sq)
+    errs = []
+    for j in range(ps.L):
+        as_ = o.negacyclic_mul(0, evk[0, j, 1, 0], sq)
+        e = (evk[0, j, 0, 0].astype(object) + as_.astype(object) - (ps.p % ps.q[0] if j == 0 else 0) * sp.astype(object)) % ps.q[0]
+        e = np.array([int(v) - ps.q[0] if int(v) > ps.q[0] // 2 else int(v) for v in e], dtype=np.float64)
+        errs.append(e)
+    errs = np.concatenate(errs)
+    assert np.abs(errs).max() <= 6 * 3.2 and abs(errs.std() - 3.2) < 0.15 and abs(errs.mean()) < 0.2
+    # round trip: the seeded keys serve the ordinary path (oracle rotation with the same key, then decrypt)
+    g.load_keys(evk, [1, 2, 3, 4])
+    qv = synth.toy_query(5, dim=16)
+    km = synth.key_material(ps, 3)
+    ct = g.encrypt_query(s, qv, km.ct_a, km.ct_e)
+    baby = g.export(b.KIND_CT, g.query_prepare(g.import_(b.KIND_CT, ct, 1), g.workspace(1)), ps.B)
+    g.sync()
+    for r in range(1, ps.B):
+        assert np.array_equal(baby[r], o.rotate(ct, r, evk[r - 1]))
+        z = o.decrypt_slots(s, baby[r], ps.log_scale).real
+        assert np.abs(z - np.roll(np.tile(qv.astype(np.float64), ps.n // 16), -r)).max() < 2.0 ** -10
 
 
 @pytest.mark.parametrize("logN,big", [(8, False), (12, False), (13, True)])

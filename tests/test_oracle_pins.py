@@ -11,6 +11,7 @@ import sympy
 
 from oracle.oracle import Oracle, find_primes, is_prime
 from paper_2608_21131_b200 import synth
+from tests.helpers import rescale_error_bound, rescale_error_sigma
 
 
 def make(ps):
@@ -107,11 +108,12 @@ def exact_encode(z, N, log_scale):
     n = N // 2
     g = [pow(5, j, 2 * N) for j in range(n)]
     zs = [mpmath.mpf(float(v)) for v in z]
+    cos_tab = [mpmath.cos(mpmath.pi * t / N) for t in range(2 * N)]   # cos(pi t / N), t mod 2N
     out, margin = [], []
     for k in range(N):
         acc = mpmath.mpf(0)
         for j in range(n):
-            acc += zs[j] * mpmath.cos(mpmath.pi * ((g[j] * k) % (2 * N)) / N)
+            acc += zs[j] * cos_tab[(g[j] * k) % (2 * N)]
         val = acc * mpmath.mpf(2) ** log_scale / n
         out.append(int(mpmath.nint(val)))
         margin.append(float(abs(abs(val - mpmath.floor(val)) - mpmath.mpf(0.5))))
@@ -128,6 +130,23 @@ def test_encode_equals_exact_cosine_sum(logN):
     for k in range(ps.N):
         assert int(m[k]) == want[k] or (abs(int(m[k]) - want[k]) == 1 and margin[k] < 1e-6)
     assert sum(int(m[k]) != want[k] for k in range(ps.N)) == 0
+
+
+def test_encode_equals_exact_cosine_sum_at_the_production_scale():
+    """the same pin at N = 1024 and scale 2^40, the scale of every configuration but the toy: coefficients of ~2^35
+    (Delta |z| / sqrt(n)) need 35 of the 53 mantissa bits, so a sloppier evaluation order than the pinned one, or a
+    table that is not correctly rounded, would show here first"""
+    ps = synth.small_params(10, 1, 1)
+    o = make(ps)
+    z = synth.gaussian(11, 40, np.arange(ps.n))
+    m = o.encode(z, 40)
+    want, margin = exact_encode(z, ps.N, 40)
+    assert max(abs(int(v)) for v in want) > 2 ** 34
+    bad = [k for k in range(ps.N) if int(m[k]) != want[k]]
+    # the binary64 evaluation carries a relative error of a few 2^-53 per operation into values of ~2^35, i.e. ~2^-15 of
+    # a unit: only an exact value within that distance of a half-integer may round the other way
+    assert all(abs(int(m[k]) - want[k]) == 1 and margin[k] < 2.0 ** -10 for k in bad), bad
+    assert len(bad) <= 1
 
 
 @pytest.mark.parametrize("logN,big", [(4, False), (8, False), (10, True)])
@@ -457,17 +476,9 @@ def test_compaction_is_exact_division_of_the_crt_integer():
                     assert int(out[poly, i, x]) == want % ps.q[i]
 
 
-def rescale_error_sigma(N, scale):
-    """standard deviation of the real part of a slot of the rescale's rounding error tau_0 + tau_1 s (tau uniform in
-    [-1/2, 1/2], s ternary with variance 2/3): a coefficient has variance N/18 + 1/12, a slot sums N of them with
-    unit-modulus weights, its real part takes half.  A slot of tau_1 s is the PRODUCT of two near-Gaussian values
-    (tau_1 and s evaluated at the same root), so the tails are heavier than Gaussian: tests allow 12 sigma."""
-    return math.sqrt(N * (N / 18.0 + 1.0 / 12.0) / 2.0) / scale
-
-
 def test_compacted_scores_decrypt_to_the_same_scores():
     """Production primes on a reduced ring.  Dropping to two limbs is exact (identical centred integers); a rescale to
-    one limb (scale 2^80 / q_3 ~ 2^30) adds the rounding error of the division: within 12 sigma of its analytic size and,
+    one limb (scale 2^80 / q_3 ~ 2^30) adds the rounding error of the division: inside the Laplace-tail bound of its analytic size (see helpers) and,
     on this ring, still inside 2^-18."""
     ps = synth.ParamSet("n11", 11, synth.Q50, synth.P60, 40, 128, 32, -18)
     o = make(ps)
@@ -488,7 +499,7 @@ def test_compacted_scores_decrypt_to_the_same_scores():
         small = o.compact(sc, keep)
         assert small.shape == (2, keep, ps.N)
         got = o.decrypt_compact_slots(km.s, small, 2 * ps.log_scale)
-        assert np.abs(got.real - full.real).max() < 12 * sigma
+        assert np.abs(got.real - full.real).max() < rescale_error_bound(ps.N, 2.0 ** 80 / ps.q[-1], ps.n)
         assert np.abs(got.real - full.real).std() > sigma / 3                # and the error really is of that size
         assert np.abs(got.real - want).max() < 2.0 ** -18
         assert np.abs(got.imag).max() < 2.0 ** -18
@@ -505,7 +516,7 @@ def test_compacted_scores_decrypt_to_the_same_scores():
     got = o.decrypt_compact_slots(km.s, o.compact(sc, 1), 2 * ps.log_scale)
     sigma = rescale_error_sigma(ps.N, 2.0 ** 50 / ps.q[-1])
     err = np.abs(got.real - o.decrypt_slots(km.s, sc, 2 * ps.log_scale).real)
-    assert sigma / 3 < err.std() and err.max() < 12 * sigma
+    assert sigma / 3 < err.std() and err.max() < rescale_error_bound(ps.N, 2.0 ** 50 / ps.q[-1], ps.n)
 
 
 # ------------------------------------------------------------------ encrypted database: ct x ct, relinearisation

@@ -28,7 +28,9 @@
  * sum evaluated in multi-precision; automorphism == slot roll; decrypt(encrypt(m)) - m == e;
  * key-switch error within the analytic noise bound and ModDown(p*x) == x; rotate via
  * "decompose then permute" == "permute then decompose"; BSGS/Horner == plain matvec;
- * decrypted scores == float64 dot products within the stated tolerance.
+ * decrypted scores == float64 dot products within the stated tolerance; the lazy giant steps: inner product + ModDown
+ * == orc_keyswitch bit for bit, the result's decryption minus the exactly rotated decryptions of the terms inside the
+ * analytic bound for G-1 key products and ONE rounding.
  */
 #include <stdint.h>
 #include <stdlib.h>
@@ -695,6 +697,57 @@ void orc_rotate_sum(const orc_ctx *c, const u64 *inner, const u64 *evk_B, u64 *s
     }
     memcpy(score_ct, acc, ctw * 8);
     free(acc); free(rot);
+}
+
+/* ---- second evaluation order of the giant steps: distinct keys, one ModDown ("lazy") --------------------------------
+ * The paper fixes only WHAT the giant steps compute, sum_g rot_{gB}(inner[g]) (Sec. 3.1 Detail); Horner with one key
+ * (orc_rotate_sum) is one order of evaluation, this is the other one this build supports.  Every term is rotated by its
+ * own amount gB with the key of that rotation, the key products are SUMMED in R_{Qp} and brought down once:
+ *   (U0, U1) = sum_{g>=1} sum_j digit_j(phi_g(inner[g].c1)) * (b_j, a_j)[key of rotation gB]      over the L+1 moduli,
+ *   score = ( inner[0].c0 + sum_{g>=1} phi_g(inner[g].c0) + ModDown(U0),  inner[0].c1 + ModDown(U1) ),  phi_g: X -> X^(5^(gB)).
+ * One rounding (ModDown) instead of G-1, and no key-switch result is ever key-switched again. */
+
+/* (u0, u1) += sum_j d_j * (b_j, a_j) over the L+1 moduli: the inner product of orc_keyswitch without its ModDown */
+void orc_ks_accumulate(const orc_ctx *c, const u64 *d, const u64 *evk, u64 *u0, u64 *u1) {
+    int N = c->N, L = c->L;
+    u64 *dj = (u64 *)malloc(8 * N), *t = (u64 *)malloc(8 * N);
+    for (int j = 0; j < L; j++)
+        for (int i = 0; i <= L; i++) {
+            u64 q = c->mod[i];
+            for (int x = 0; x < N; x++) dj[x] = reduce_signed(centred(d[(size_t)j * N + x], c->mod[j]), q);
+            orc_negacyclic_mul(c, i, dj, evk + (((size_t)j * 2 + 0) * (L + 1) + i) * N, t);
+            for (int x = 0; x < N; x++) u0[(size_t)i * N + x] = addmod(u0[(size_t)i * N + x], t[x], q);
+            orc_negacyclic_mul(c, i, dj, evk + (((size_t)j * 2 + 1) * (L + 1) + i) * N, t);
+            for (int x = 0; x < N; x++) u1[(size_t)i * N + x] = addmod(u1[(size_t)i * N + x], t[x], q);
+        }
+    free(dj); free(t);
+}
+
+/* inner[G][2][L][N]; evk_giant[G-1] keys, entry g-1 the key of rotation g*B; score_ct[2][L][N] */
+void orc_rotate_sum_lazy(const orc_ctx *c, const u64 *inner, const u64 *evk_giant, u64 *score_ct) {
+    int N = c->N, L = c->L, G = c->G;
+    size_t LN = (size_t)L * N, ctw = 2 * LN, evw = (size_t)L * 2 * (L + 1) * N;
+    u64 *u0 = (u64 *)calloc((size_t)(L + 1) * N, 8), *u1 = (u64 *)calloc((size_t)(L + 1) * N, 8);
+    u64 *pc = (u64 *)malloc(LN * 8), *md = (u64 *)malloc(LN * 8);
+    memcpy(score_ct, inner, ctw * 8);                              /* the g = 0 term is not rotated */
+    for (int g = 1; g < G; g++) {
+        long k = orc_galois(c, g * c->B);
+        const u64 *ct = inner + (size_t)g * ctw;
+        for (int l = 0; l < L; l++) orc_automorphism(c, l, k, ct + (size_t)l * N, pc + (size_t)l * N);          /* phi_g(c0) */
+        for (int l = 0; l < L; l++)
+            for (int x = 0; x < N; x++) score_ct[(size_t)l * N + x] = addmod(score_ct[(size_t)l * N + x], pc[(size_t)l * N + x], c->mod[l]);
+        for (int l = 0; l < L; l++) orc_automorphism(c, l, k, ct + LN + (size_t)l * N, pc + (size_t)l * N);     /* phi_g(c1) */
+        orc_ks_accumulate(c, pc, evk_giant + (size_t)(g - 1) * evw, u0, u1);
+    }
+    if (G > 1) {
+        orc_moddown(c, u0, md);
+        for (int l = 0; l < L; l++)
+            for (int x = 0; x < N; x++) score_ct[(size_t)l * N + x] = addmod(score_ct[(size_t)l * N + x], md[(size_t)l * N + x], c->mod[l]);
+        orc_moddown(c, u1, md);
+        for (int l = 0; l < L; l++)
+            for (int x = 0; x < N; x++) score_ct[LN + (size_t)l * N + x] = addmod(score_ct[LN + (size_t)l * N + x], md[(size_t)l * N + x], c->mod[l]);
+    }
+    free(u0); free(u1); free(pc); free(md);
 }
 
 /* One block end to end: encode, MAC, rotate-and-sum.  Optional outputs pt_out / inner_out may be NULL. */

@@ -353,6 +353,22 @@ class Oracle:
         lib().orc_rotate_sum(self.h, _p(inner, u64p), _p(evk_B, u64p), _p(out, u64p))
         return out
 
+    def ks_accumulate(self, d, evk, u0=None, u1=None):
+        """(u0, u1) += sum_j digit_j(d) * (b_j, a_j) over the L+1 moduli (no ModDown); returns the two [L+1][N] arrays"""
+        d, evk = _u64(d), _u64(evk)
+        u0 = np.zeros((self.L + 1, self.N), dtype=np.uint64) if u0 is None else u0
+        u1 = np.zeros((self.L + 1, self.N), dtype=np.uint64) if u1 is None else u1
+        lib().orc_ks_accumulate(self.h, _p(d, u64p), _p(evk, u64p), _p(u0, u64p), _p(u1, u64p))
+        return u0, u1
+
+    def rotate_sum_lazy(self, inner, evk_giant):
+        """sum_g rot_{gB}(inner[g]) with the keys of rotations B, 2B, .., (G-1)B (evk_giant[g-1]) and one ModDown"""
+        inner, evk_giant = _u64(inner), _u64(evk_giant)
+        assert inner.shape == (self.G, 2, self.L, self.N) and evk_giant.shape[0] == max(self.G - 1, 0)
+        out = np.zeros((2, self.L, self.N), dtype=np.uint64)
+        lib().orc_rotate_sum_lazy(self.h, _p(inner, u64p), _p(evk_giant, u64p), _p(out, u64p))
+        return out
+
     def score_block(self, rows, baby, evk_B, want_pt=False, want_inner=False):
         rows = np.ascontiguousarray(rows, dtype=np.float32)
         baby, evk_B = _u64(baby), _u64(evk_B)

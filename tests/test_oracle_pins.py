@@ -382,6 +382,96 @@ def test_bsgs_without_noise_equals_plain_matvec(logN, R, B):
     assert np.abs(total - got).max() < 2e-5
 
 
+# ------------------------------------------------------------------ giant steps, second order of evaluation (lazy)
+
+
+def test_key_product_then_moddown_is_the_key_switch():
+    """orc_ks_accumulate repeats the inner product of orc_keyswitch: followed by ModDown it must give the same bits"""
+    ps = synth.small_params(7, 8, 4, L=3, big=True)
+    o = make(ps)
+    km = synth.key_material(ps, 23)
+    rng = np.random.default_rng(4)
+    evk = o.evk_gen(km.s, 2, km.evk_a[1], km.evk_e[1])
+    d = np.stack([rand_poly(rng, ps.N, q) for q in ps.q])
+    u0, u1 = o.ks_accumulate(d, evk)
+    ks0, ks1 = o.keyswitch(d, evk)
+    assert np.array_equal(o.moddown(u0), ks0) and np.array_equal(o.moddown(u1), ks1)
+    # and it accumulates: a second product lands on top of the first
+    d2 = np.stack([rand_poly(rng, ps.N, q) for q in ps.q])
+    v0, v1 = o.ks_accumulate(d2, evk)
+    w0, w1 = o.ks_accumulate(d2, evk, u0.copy(), u1.copy())
+    mods = np.array(list(ps.q) + [ps.p], dtype=object)[:, None]
+    assert np.array_equal(w0.astype(object), (u0.astype(object) + v0.astype(object)) % mods)
+    assert np.array_equal(w1.astype(object), (u1.astype(object) + v1.astype(object)) % mods)
+
+
+@pytest.mark.parametrize("big", [False, True])
+def test_lazy_giant_steps_error_within_analytic_bound(big):
+    """sum_g rot_{gB}(inner[g]) with distinct keys and one ModDown: the decryption of the result minus the exactly rotated
+    decryptions of the terms (python integers, explicit coefficient map) is the key-switch error of G-1 key products and
+    ONE rounding: variance (G-1) L N sigma^2 q^2 / (12 p^2) + N/18.  Horner on the same terms rounds G-1 times: its
+    error is measurably larger where the rounding term dominates (50-bit primes under a 60-bit special prime)."""
+    ps = synth.small_params(8, 16, 4, L=2, big=big)
+    o = make(ps)
+    G, B, N, Q = ps.G, ps.B, ps.N, 1
+    for q in ps.q:
+        Q *= q
+    km = synth.key_material(ps, 27, rots=[g * B for g in range(1, G)])
+    evk = all_keys(o, km)
+    rng = np.random.default_rng(8)
+    inner = np.stack([np.stack([np.stack([rand_poly(rng, N, q) for q in ps.q]) for _ in range(2)]) for _ in range(G)])
+    want = np.zeros(N, dtype=object)
+    for g in range(G):
+        dg = o.decrypt_int(km.s, inner[g])
+        k = o.galois(g * B)
+        rot = np.zeros(N, dtype=object)
+        for i in range(N):
+            e = (i * k) % (2 * N)
+            if e < N:
+                rot[e] = int(dg[i])
+            else:
+                rot[e - N] = -int(dg[i])
+        want = want + rot
+
+    def error_of(ct):
+        got = o.decrypt_int(km.s, ct)
+        return np.array([float(((int(a) - int(b) + Q // 2) % Q) - Q // 2) for a, b in zip(got, want)])
+
+    err = error_of(o.rotate_sum_lazy(inner, evk))
+    qmean = float(np.mean([float(x) for x in ps.q]))
+    key_var = ps.L * N * 3.2 ** 2 * qmean ** 2 / (12 * float(ps.p) ** 2)
+    std = math.sqrt((G - 1) * key_var + N / 18.0)
+    assert abs(err.mean()) < 0.5 * std and 0.7 * std < err.std() < 1.3 * std and np.abs(err).max() < 6 * std
+    # Horner with the single key of rotation B on the same terms: G-1 roundings
+    err_h = error_of(o.rotate_sum(inner, evk[0]))
+    std_h = math.sqrt((G - 1) * (key_var + N / 18.0))
+    assert 0.7 * std_h < err_h.std() < 1.3 * std_h
+    if big:
+        assert err_h.std() > 1.3 * err.std()
+
+
+@pytest.mark.parametrize("logN,R,B", [(5, 4, 2), (6, 8, 2), (6, 4, 1), (6, 4, 4)])
+def test_lazy_giant_steps_without_noise_equal_plain_matvec(logN, R, B):
+    ps = synth.small_params(logN, R, B, L=2)
+    o = make(ps)
+    rots = sorted(set(range(1, B)) | {g * B for g in range(1, ps.G)})
+    km = synth.key_material(ps, 41, rots=rots, zero_noise=True)
+    evk = dict(zip(rots, all_keys(o, km)))
+    rows = synth.toy_corpus(3, rows=ps.n - 3, dim=R)
+    qv = synth.toy_query(4, dim=R)
+    ct = o.encrypt_query(km.s, qv, km.ct_a, km.ct_e)
+    baby = o.baby_set(ct, np.stack([evk[r] for r in range(1, B)]) if B > 1 else np.zeros((0, ps.L, 2, ps.L + 1, ps.N), dtype=np.uint64))
+    inner = o.mac(o.encode_block(rows), baby)
+    giant = np.stack([evk[g * B] for g in range(1, ps.G)]) if ps.G > 1 else np.zeros((0, ps.L, 2, ps.L + 1, ps.N), dtype=np.uint64)
+    score = o.rotate_sum_lazy(inner, giant)
+    got = o.decrypt_slots(km.s, score, 2 * ps.log_scale)
+    want = np.zeros(ps.n)
+    want[: ps.n - 3] = rows.astype(np.float64) @ qv.astype(np.float64)
+    assert np.abs(got.real - want).max() < 2e-5 and np.abs(got.imag).max() < 2e-5
+    if ps.G == 1:
+        assert np.array_equal(score, inner[0])
+
+
 def test_zero_padding_96_to_128_is_exact():
     # Sec. 4 (datasets): zero-padding 96 -> 128 dimensions changes no dot product
     x = synth.toy_corpus(8, rows=50, dim=96).astype(np.float64)

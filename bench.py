@@ -101,9 +101,25 @@ def replica_throughput(units_per_rank, world, seconds_slowest):
     return world * units_per_rank / seconds_slowest
 
 
-def build_workload(config, rows_override=None, logn=16):
+def bench_keys(ctx, ps, args):
+    """key material of a run: rotations 1..B, plus 2B..(G-1)B when the giant steps are evaluated in the lazy order"""
+    from paper_2608_21131_b200 import binding, synth, workloads as wl
+
+    rots = list(range(1, ps.B + 1))
+    if args.giant == "lazy":
+        rots += [g * ps.B for g in range(2, ps.G)]
+        ctx.set_tuning(binding.TUNE_GIANT_LAZY, 1)
+    km = synth.key_material(ps, wl.KEY_SEED, rots=rots)
+    ctx.load_keys(ctx.keygen_from_samples(km.s, km.rots, km.evk_a, km.evk_e), km.rots)
+    return km
+
+
+def build_workload(config, rows_override=None, logn=16, baby=None):
     from paper_2608_21131_b200 import workloads as wl, synth
 
+    if baby:
+        ps, rows, q, name = build_workload(config, rows_override, logn)
+        return ps.with_(B=baby), rows, q, name + ", B=%d" % baby
     if config == 0:
         ps, rows, q = wl.toy()
         return ps, rows, q, "toy: 4,096 rows, dim 64, N=2^12, scale 2^25"
@@ -192,14 +208,12 @@ def run_ours(args):
 
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    ps, rows_np, qR, wname = build_workload(args.config, args.rows, args.logn)
+    ps, rows_np, qR, wname = build_workload(args.config, args.rows, args.logn, args.baby)
     n_rows = rows_np.shape[0]
     ctx = binding.Context(ps, device=local)
     if args.encode_group:
         ctx.set_tuning(binding.TUNE_ENCODE_GROUP, args.encode_group)
-    km = synth.key_material(ps, wl.KEY_SEED)
-    evk = ctx.keygen_from_samples(km.s, km.rots, km.evk_a, km.evk_e)
-    ctx.load_keys(evk, km.rots)
+    km = bench_keys(ctx, ps, args)
     ct_host = ctx.encrypt_query(km.s, qR, km.ct_a, km.ct_e)
     ct_dev = ctx.import_(binding.KIND_CT, ct_host, 1)
     rows_dev = torch.from_numpy(rows_np).to(ctx.device)
@@ -443,6 +457,7 @@ def run_ours(args):
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64",
             "data": "synthetic",
             "config": {"workload": wname, "rows": n_rows, "blocks": nb, "R": ps.R, "B": ps.B, "G": ps.G, "logN": ps.logN, "L": ps.L,
+                       "giant_steps": "Horner, one key (default)" if args.giant == "horner" else "lazy: G-1 keys, one ModDown per block",
                        "l2": "working set per step (%.1f GB of encoded plaintexts) exceeds L2; no flush" %
                              (nb * ctx.sizeof(binding.SIZE_PT_BLOCK) / 1e9),
                        "replicas": "each rank scores the whole level on its own GPU" if world > 1 else "single GPU"},
@@ -706,8 +721,7 @@ def run_hierarchy(args):
     cfg = wl.datacomp_like() if args.config == 2 else wl.deep1b_like()
     ps = cfg.ps
     ctx = binding.Context(ps, device=0)
-    km = synth.key_material(ps, wl.KEY_SEED)
-    ctx.load_keys(ctx.keygen_from_samples(km.s, km.rots, km.evk_a, km.evk_e), km.rots)
+    km = bench_keys(ctx, ps, args)
     coarse = wl.coarse_level(cfg)
     max_rows = max(len(coarse.ids), cfg.nprobe * cfg.h.fan, cfg.leaf_beam * cfg.h.leaf)
     nb_max = ctx.n_blocks(max_rows)
@@ -758,7 +772,7 @@ def run_hierarchy(args):
         "metric": METRIC, "value": rows_scored / (total_ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u64", "data": "synthetic",
-        "config": {"workload": cfg.name + " hierarchy, one query at a time", "levels": {"coarse": len(coarse.ids), "fine": len(fine.ids),
+        "config": {"workload": cfg.name + " hierarchy, one query at a time", "giant_steps": args.giant, "levels": {"coarse": len(coarse.ids), "fine": len(fine.ids),
                                                                                         "rerank": len(rer.ids)},
                    "logN": ps.logN, "L": ps.L, "R": ps.R, "B": ps.B},
         "ms_per_query_level": {k: {"p50": pct(v, 50), "p95": pct(v, 95)} for k, v in times.items()},
@@ -827,6 +841,8 @@ def main():
                     "hierarchies (latency per level), 4 scaling sweep point (--rows = wanted rows, --logn 15|16)")
     ap.add_argument("--logn", type=int, default=16, help="ring of the sweep configuration")
     ap.add_argument("--min-timed-s", type=float, default=2.0, help="the K-step block is repeated until the timed region lasted this long")
+    ap.add_argument("--giant", default="horner", choices=["horner", "lazy"], help="evaluation order of the giant steps of the rotate-and-sum")
+    ap.add_argument("--baby", type=int, default=None, help="baby-step count B (default: the configuration's; must divide R)")
     ap.add_argument("--rows", type=int, default=None, help="override the row count (debugging, ncu captures)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--encode-group", type=int, default=None, help="tuning: plaintexts per encode launch group")

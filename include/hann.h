@@ -142,8 +142,11 @@ int hann_get_stats(hann_ctx *ctx, hann_stats *out);
  * every transform in full.  Same bits either way.
  * HANN_TUNE_HOST_GROUPS: number of block groups hann_score_level_host cuts a level into (a group is scored and its scores
  * are downloaded while the rows of the following groups still travel); 0 (default) chooses from the level's size.  Ask
- * hann_level_host_bytes again after changing it. */
-enum { HANN_TUNE_ENCODE_GROUP = 1, HANN_TUNE_HOST_LIMBS = 2, HANN_TUNE_ENCODE_SYMMETRY = 3, HANN_TUNE_HOST_GROUPS = 4 };
+ * hann_level_host_bytes again after changing it.
+ * HANN_TUNE_GIANT_LAZY (this one changes the result's BITS, not its meaning): 1 makes hann_rotate_sum, and with it
+ * hann_query_level and hann_score_level_host, evaluate the giant steps in the order of hann_rotate_sum_lazy (the keys of
+ * rotations 2B .. (G-1)B must then be loaded as well); 0 (default) is Horner with the single key of rotation B. */
+enum { HANN_TUNE_ENCODE_GROUP = 1, HANN_TUNE_HOST_LIMBS = 2, HANN_TUNE_ENCODE_SYMMETRY = 3, HANN_TUNE_HOST_GROUPS = 4, HANN_TUNE_GIANT_LAZY = 5 };
 int hann_set_tuning(hann_ctx *ctx, int what, int value);
 
 /* Per-launch profile: while enabled every kernel launch of the context is bracketed by a CUDA event pair (this
@@ -261,6 +264,18 @@ int hann_score_level_ctdb(hann_ctx *ctx, const void *baby_dev, const void *ctdb_
  * rotation B: acc = inner[G-1]; for g = G-2..0: acc = rot_B(acc) + inner[g].
  *   score_ct_dev n_blocks * HANN_SIZE_CT bytes (device), internal layout. */
 int hann_rotate_sum(hann_ctx *ctx, const void *inner_dev, int64_t n_blocks, void *score_ct_dev, void *ws, size_t ws_bytes);
+
+/* The same sum, evaluated in the second order this library supports (the paper fixes the sum, not the order): every
+ * term is rotated by its own amount with the key of that rotation, the key products of a block are added up over the
+ * L+1 moduli and brought down by ONE ModDown:
+ *     (U0, U1) = sum_{g>=1} KeyProduct_{gB}(phi_g(inner[g].c1)),   phi_g: X -> X^(5^(gB)),
+ *     score = (inner[0].c0 + sum_{g>=1} phi_g(inner[g].c0) + ModDown(U0),  inner[0].c1 + ModDown(U1)).
+ * One key-switch round of depth one instead of a chain of G-1, one rounding instead of G-1 (so slightly LESS noise),
+ * at the price of G-1 resident keys (rotations B, 2B, .., (G-1)B: HANN_ENOKEY if one is missing) instead of one.  The
+ * ciphertext bits differ from hann_rotate_sum's (both orders are reproduced bit for bit by the reference evaluation of
+ * the same order); the decrypted scores agree within the key-switch noise.  Workspace: hann_workspace_bytes(ctx, blocks)
+ * is enough; with more, more blocks go through one round. */
+int hann_rotate_sum_lazy(hann_ctx *ctx, const void *inner_dev, int64_t n_blocks, void *score_ct_dev, void *ws, size_t ws_bytes);
 
 /* One routing level for one query, device buffers in and out (Sec. 2 "Reproducing this": level + candidates +
  * encrypted query in, encrypted score vector out): hann_query_prepare, hann_encode_candidates,

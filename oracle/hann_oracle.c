@@ -750,6 +750,32 @@ void orc_rotate_sum_lazy(const orc_ctx *c, const u64 *inner, const u64 *evk_gian
     free(u0); free(u1); free(pc); free(md);
 }
 
+/* ---- pieces of the packed projection (Sec. 3.1 Detail: all chunks of W in one object per diagonal, combined with 0/1
+ * plaintext masks; see oracle.py PackedProjection for the steps) -------------------------------------------------------- */
+
+/* encode a real slot vector at scale 2^log_scale and reduce it into the L ciphertext primes: pt[L][N] */
+void orc_encode_plain(const orc_ctx *c, const double *z, int log_scale, u64 *pt) {
+    int N = c->N, L = c->L;
+    i64 *m = (i64 *)malloc(sizeof(i64) * N);
+    orc_encode(c, z, log_scale, m);
+    for (int l = 0; l < L; l++) lift_i64(m, N, c->mod[l], pt + (size_t)l * N);
+    free(m);
+}
+
+/* acc[2][L][N] += ct[2][L][N] * pt[L][N]: ciphertext x plaintext product of both components, every limb.  A mask
+ * multiply is exactly this (the mask is a public constant: no key switch, no relinearisation). */
+void orc_mul_plain_acc(const orc_ctx *c, const u64 *ct, const u64 *pt, u64 *acc) {
+    int N = c->N, L = c->L;
+    u64 *t = (u64 *)malloc(8 * N);
+    for (int comp = 0; comp < 2; comp++)
+        for (int l = 0; l < L; l++) {
+            size_t o = ((size_t)comp * L + l) * N;
+            orc_negacyclic_mul(c, l, ct + o, pt + (size_t)l * N, t);
+            for (int x = 0; x < N; x++) acc[o + x] = addmod(acc[o + x], t[x], c->mod[l]);
+        }
+    free(t);
+}
+
 /* One block end to end: encode, MAC, rotate-and-sum.  Optional outputs pt_out / inner_out may be NULL. */
 void orc_score_block(const orc_ctx *c, const float *rows, int n_rows, const u64 *baby, const u64 *evk_B,
                      u64 *score_ct, u64 *pt_out, u64 *inner_out) {

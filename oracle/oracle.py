@@ -381,6 +381,160 @@ class Oracle:
         )
         return out, pt, inner
 
+    # ---- pieces of the packed projection
+    def encode_plain(self, z, log_scale=None):
+        """real slot vector -> plaintext residues [L][N] at scale 2^log_scale"""
+        z = np.ascontiguousarray(z, dtype=np.float64)
+        assert z.shape == (self.n,)
+        pt = np.zeros((self.L, self.N), dtype=np.uint64)
+        lib().orc_encode_plain(self.h, _p(z, f64p), C.c_int(self.log_scale if log_scale is None else log_scale), _p(pt, u64p))
+        return pt
+
+    def mul_plain_acc(self, ct, pt, acc=None):
+        """acc += ct * pt (ciphertext x plaintext); returns acc [2][L][N]"""
+        ct, pt = _u64(ct), _u64(pt)
+        acc = np.zeros((2, self.L, self.N), dtype=np.uint64) if acc is None else acc
+        lib().orc_mul_plain_acc(self.h, _p(ct, u64p), _p(pt, u64p), _p(acc, u64p))
+        return acc
+
+    def add(self, a, b):
+        """a + b for ciphertexts / polynomial stacks [..][L][N]"""
+        mods = np.array(self.q, dtype=object).reshape((1,) * (np.ndim(a) - 2) + (self.L, 1))
+        return ((np.asarray(a).astype(object) + np.asarray(b).astype(object)) % mods).astype(np.uint64)
+
     @staticmethod
     def num_threads():
         return int(lib().orc_num_threads())
+
+
+def restrict_keys(evk, L_from, L_to):
+    """Evaluation keys [..][L_from][2][L_from+1][N] of a chain of L_from primes, restricted to its first L_to primes:
+    digits 0..L_to-1, limbs q_0..q_{L_to-1} and the special prime.  With one-prime digits the key material of digit j on
+    limb i (b_j = -a_j s + e_j + F_j s', F_j = p mod q_j on limb j, 0 elsewhere) does not depend on the other primes, so
+    the restriction IS the key of the shorter chain."""
+    limbs = list(range(L_to)) + [L_from]
+    return np.ascontiguousarray(np.asarray(evk)[..., :L_to, :, :, :][..., limbs, :])
+
+
+class PackedProjection:
+    """Rank reduction under encryption with the matrix packed by windows (Sec. 3.1 "How" and Detail):
+    Enc(q_R) = W^T Enc(q), W of shape D x R (D = c R), by the diagonal method with baby and giant steps.
+
+    Reading taken (the paper gives no index formulas):
+      * slots are viewed with period D; window k of a period is positions kR .. kR+R-1; the query ciphertext holds
+        q[i mod D]; chunk k of W is the R x R matrix W_k^T[r][col] = W[kR + col][r];
+      * ONE packed object per diagonal d = gB + b of all c chunks (storage R objects, not D): slot kR + j of P[g][b]
+        holds W_k^T[(j - gB) mod R][(j + b) mod R] -- the diagonal, shifted IN its window by the giant-step amount in
+        plaintext (the paper's plaintext pre-rotation);
+      * a baby step must rotate every chunk of the query INSIDE its window.  A slot rotation moves data across window
+        boundaries, so the in-window rotation is put together from two slot rotations with 0/1 plaintext masks (a public
+        constant: a ciphertext x plaintext multiply, no key switch):
+            cyc_b = lo_b * rot_b(ct) + hi_b * rot_{b-R}(ct),  lo_b[i] = [(i mod R) + b < R],  hi_b = 1 - lo_b;
+        the masks are encoded at scale 2^log_mask, and ONE rescale (by the last prime) follows;
+      * inner[g] = sum_b P[g][b] * cyc_b, then the giant steps sum_g rot_{gB}(inner[g]) with ordinary slot rotations:
+        these DO mix adjacent windows (slot kR + j receives from window k or k + 1), which is harmless because
+      * a single final fold, acc += rot_{R 2^t}(acc) for t < log2 c, adds up all windows: window mixing is a fixed
+        permutation of the windows, invisible to their sum.  Every slot i then holds q_R[i mod R]: the projected query,
+        already tiled for the scoring levels;
+      * one more rescale (by the next prime) returns the scale to about 2^log_scale: the projected query has L - 2 primes
+        and scores at scale Delta^2 again.
+    Three parameter sets of the same ring share the keys (restrict_keys): top (L primes: baby rotations and masks), mid
+    (L - 1: matrix product, giant steps, fold), low (L - 2: what the scoring levels run on)."""
+
+    def __init__(self, logN, q, p, log_scale, D, R, B, log_mask, log_w):
+        assert D % R == 0 and R % B == 0 and len(q) >= 3
+        self.D, self.R, self.B, self.G, self.c = D, R, B, R // B, D // R
+        assert self.c & (self.c - 1) == 0, "the fold doubles: D / R must be a power of two"
+        self.log_scale, self.log_mask, self.log_w = log_scale, log_mask, log_w
+        self.top = Oracle(logN, q, p, log_scale, R, B)
+        self.mid = Oracle(logN, q[:-1], p, log_scale, R, B)
+        self.low = Oracle(logN, q[:-2], p, log_scale, R, B)
+        self.n, self.N, self.L = self.top.n, self.top.N, len(q)
+        assert self.n % D == 0
+        # exact scale of the projected query: Delta * 2^log_mask / q_{L-1} * 2^log_w / q_{L-2}
+        self.scale_out = 2.0 ** log_scale * (2.0 ** log_mask / q[-1]) * (2.0 ** log_w / q[-2])
+
+    # ---- index formulas (plain slot vectors)
+    def query_slots(self, qvec):
+        return np.tile(np.asarray(qvec, dtype=np.float64), self.n // self.D)
+
+    def matrix_slots(self, W):
+        """z[g][b][i] = W[kR + (j + b) mod R][(j - gB) mod R] for i mod D = kR + j"""
+        W = np.asarray(W, dtype=np.float64)
+        assert W.shape == (self.D, self.R)
+        i = np.arange(self.n) % self.D
+        k, j = i // self.R, i % self.R
+        z = np.zeros((self.G, self.B, self.n))
+        for g in range(self.G):
+            for b in range(self.B):
+                z[g, b] = W[k * self.R + (j + b) % self.R, (j - g * self.B) % self.R]
+        return z
+
+    def masks(self):
+        j = np.arange(self.n) % self.R
+        lo = np.stack([(j + b < self.R).astype(np.float64) for b in range(self.B)])
+        return lo, 1.0 - lo
+
+    def baby_rotations(self):
+        """slot rotations the baby steps need: b and b - R (taken modulo n), b = 1 .. B-1"""
+        return list(range(1, self.B)) + [self.n - self.R + b for b in range(1, self.B)]
+
+    def fold_rotations(self):
+        return [self.R << t for t in range(self.c.bit_length() - 1)]
+
+    def plain(self, W, qvec):
+        """the same steps on plain slot vectors (no encryption): what every slot must hold at the end"""
+        x = self.query_slots(qvec)
+        z = self.matrix_slots(W)
+        lo, hi = self.masks()
+        cyc = [lo[b] * np.roll(x, -b) + hi[b] * np.roll(x, -(b - self.R)) for b in range(self.B)]
+        acc = np.zeros(self.n)
+        for g in range(self.G):
+            acc += np.roll(sum(z[g, b] * cyc[b] for b in range(self.B)), -g * self.B)
+        unfolded = acc.copy()
+        for r in self.fold_rotations():
+            acc = acc + np.roll(acc, -r)
+        return acc, unfolded
+
+    # ---- the encrypted pipeline
+    def enrol(self, W):
+        """packed diagonals of W as plaintexts of the middle chain: [G][B][L-1][N] at scale 2^log_w"""
+        z = self.matrix_slots(W)
+        return np.stack([np.stack([self.mid.encode_plain(z[g, b], self.log_w) for b in range(self.B)]) for g in range(self.G)])
+
+    def mask_plaintexts(self):
+        lo, hi = self.masks()
+        return (np.stack([self.top.encode_plain(v, self.log_mask) for v in lo]),
+                np.stack([self.top.encode_plain(v, self.log_mask) for v in hi]))
+
+    def in_window_rotations(self, ct, evk):
+        """cyc[b] = lo_b * rot_b(ct) + hi_b * rot_{b-R}(ct) over the L primes (scale Delta 2^log_mask), then the rescale:
+        [B][2][L-1][N].  evk: {rotation: key of the top chain}."""
+        lo, hi = self.mask_plaintexts()
+        out = []
+        for b in range(self.B):
+            a = ct if b == 0 else self.top.rotate(ct, b, evk[b])
+            acc = self.top.mul_plain_acc(a, lo[b])
+            if b > 0:
+                r = self.n - self.R + b
+                acc = self.top.mul_plain_acc(self.top.rotate(ct, r, evk[r]), hi[b], acc)
+            out.append(self.top.compact(acc, self.L - 1, rescale=True))
+        return np.stack(out)
+
+    def project(self, ct, evk, Wpt, lazy=False):
+        """ct [2][L][N] (query tiled with period D, scale Delta) -> projected query [2][L-2][N] at scale `scale_out`.
+        evk: {rotation: key of the TOP chain} for baby_rotations(), B (or B, 2B, .. when lazy) and fold_rotations()."""
+        mid, L = self.mid, self.L
+        low_key = lambda r: restrict_keys(evk[r], L, L - 1)
+        cyc = self.in_window_rotations(ct, evk)
+        inner = mid.mac(Wpt, cyc)
+        if self.G == 1:
+            acc = inner[0]
+        elif lazy:
+            acc = mid.rotate_sum_lazy(inner, np.stack([low_key(g * self.B) for g in range(1, self.G)]))
+        else:
+            acc = mid.rotate_sum(inner, low_key(self.B))
+        self.unfolded = acc
+        for r in self.fold_rotations():
+            acc = mid.add(acc, mid.rotate(acc, r, low_key(r)))
+        return mid.compact(acc, L - 2, rescale=True)

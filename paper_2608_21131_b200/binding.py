@@ -23,6 +23,7 @@ TUNE_ENCODE_GROUP = 1
 TUNE_HOST_LIMBS = 2
 TUNE_ENCODE_SYMMETRY = 3
 TUNE_HOST_GROUPS = 4
+TUNE_GIANT_LAZY = 5
 
 
 class HannError(RuntimeError):
@@ -89,6 +90,7 @@ def load_library():
         "hann_selftest_bounded_wait": (C.c_int, [vp, C.c_int, vp]),
         "hann_score_level_batch": (C.c_int, [vp, vp, C.c_int, vp, i64, vp, vp, sz]),
         "hann_rotate_sum": (C.c_int, [vp, vp, i64, vp, vp, sz]),
+        "hann_rotate_sum_lazy": (C.c_int, [vp, vp, i64, vp, vp, sz]),
         "hann_keyswitch": (C.c_int, [vp, C.c_int, vp, vp, vp, vp, sz]),
         "hann_query_level": (C.c_int, [vp, vp, vp, i64, C.c_int, vp, vp, vp, vp, vp, sz]),
         "hann_static_scratch_bytes": (i64, []),
@@ -375,6 +377,12 @@ class Context:
         if score is None:
             score = self.alloc(n_blocks * self.sizeof(SIZE_CT))
         self._ck(self.lib.hann_rotate_sum(self.h, _ptr(inner), n_blocks, _ptr(score), _ptr(ws), ws.numel() * 8))
+        return score
+
+    def rotate_sum_lazy(self, inner, n_blocks, ws, score=None):
+        if score is None:
+            score = self.alloc(n_blocks * self.sizeof(SIZE_CT))
+        self._ck(self.lib.hann_rotate_sum_lazy(self.h, _ptr(inner), n_blocks, _ptr(score), _ptr(ws), ws.numel() * 8))
         return score
 
     def query_level(self, ct_dev, rows_dev, ws, baby=None, pt=None, inner=None, score=None):

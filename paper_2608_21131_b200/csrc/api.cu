@@ -109,6 +109,13 @@ int64_t ks_item_words(const hann_ctx* c) {
     return L * N + L * (L + 1) * N + 2 * (L + 1) * N + 2 * L * N + 2 * L * N;
 }
 
+// words of workspace the lazy rotate-and-sum needs per block of a round: G-1 terms (c1 coefficients, digits, key product)
+// and one ModDown (special-prime limb of the sum, its lift)
+int64_t lazy_block_words(const hann_ctx* c) {
+    const int64_t L = c->L, N = c->N, G1 = c->G - 1;
+    return G1 * (L * N + L * (L + 1) * N + 2 * (L + 1) * N) + 2 * N + 2 * L * N;
+}
+
 int64_t prepare_words(const hann_ctx* c) {
     const int64_t L = c->L, N = c->N, nb = std::max(c->B - 1, 1);
     return L * N + L * (L + 1) * N + nb * (2 * (L + 1) * N + 2 * L * N);
@@ -440,6 +447,7 @@ extern "C" int64_t hann_workspace_bytes(const hann_ctx* c, int64_t max_blocks) {
     int64_t w = std::max(ks_item_words(c) * items, prepare_words(c)) * 8;
     w = std::max(w, (ks_item_words(c) + (int64_t)c->L * c->N) * 8);  // hann_keyswitch permutes its input first
     w = std::max(w, (ks_item_words(c) + 3 * (int64_t)c->L * c->N) * 8);  // hann_score_level_ctdb: one degree-2 sum + its key switch
+    w = std::max(w, lazy_block_words(c) * std::min<int64_t>(items, 4) * 8);  // hann_rotate_sum_lazy: up to four blocks per round
     w = std::max(w, encode_ws_bytes(c));
     // hann_query_level runs query_prepare and encode_candidates side by side, each in its own part
     w = std::max(w, align256(prepare_words(c) * 8 + kSlack) + encode_ws_bytes(c));
@@ -494,6 +502,9 @@ extern "C" int hann_set_tuning(hann_ctx* c, int what, int value) {
             return HANN_OK;
         case HANN_TUNE_ENCODE_SYMMETRY:
             c->encode_sym = value ? 1 : 0;
+            return HANN_OK;
+        case HANN_TUNE_GIANT_LAZY:
+            c->giant_lazy = value ? 1 : 0;
             return HANN_OK;
         default: return fail(c, HANN_EINVAL, "hann_set_tuning: unknown knob");
     }
@@ -1102,6 +1113,7 @@ extern "C" int hann_rotate_sum(hann_ctx* c, const void* inner_dev, int64_t n_blo
     const int64_t LN = (int64_t)L * N, L1N = (int64_t)(L + 1) * N, ctw = 2 * LN;
     const u64* inner = (const u64*)inner_dev;
     u64* score = (u64*)score_ct_dev;
+    if (c->giant_lazy && G > 1) return hann_rotate_sum_lazy(c, inner_dev, n_blocks, score_ct_dev, ws, ws_bytes);
     DeviceGuard dg(c->device);
     Timer tm(c, 3);
     if (G == 1) {
@@ -1181,6 +1193,78 @@ extern "C" int hann_rotate_sum(hann_ctx* c, const void* inner_dev, int64_t n_blo
     return HANN_OK;
 }
 
+extern "C" int hann_rotate_sum_lazy(hann_ctx* c, const void* inner_dev, int64_t n_blocks, void* score_ct_dev, void* ws, size_t ws_bytes) {
+    if (!c) return HANN_EINVAL;
+    if (n_blocks < 0 || (n_blocks > 0 && (!inner_dev || !score_ct_dev))) return fail(c, HANN_EINVAL, "hann_rotate_sum_lazy: bad argument");
+    if (n_blocks == 0) return HANN_OK;
+    const int L = c->L, N = c->N, G = c->G, B = c->B;
+    const int64_t LN = (int64_t)L * N, L1N = (int64_t)(L + 1) * N, ctw = 2 * LN;
+    const u64* inner = (const u64*)inner_dev;
+    u64* score = (u64*)score_ct_dev;
+    DeviceGuard dg(c->device);
+    Timer tm(c, 3);
+    if (G == 1) return launch_copy2d(c, score, ctw, inner, ctw, n_blocks * ctw, 1);
+    for (int g = 1; g < G; g++)
+        if (!c->keytab_host[g * B]) return fail(c, HANN_ENOKEY, "hann_rotate_sum_lazy: the keys of rotations B, 2B, .., (G-1)B must be loaded");
+    if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_rotate_sum_lazy: workspace missing or not 256-byte aligned");
+    int64_t ch = ((int64_t)ws_bytes - kSlack) / (lazy_block_words(c) * 8);
+    if (ch < 1) return fail(c, HANN_EWORKSPACE, "hann_rotate_sum_lazy: workspace too small");
+    ch = std::min<int64_t>(std::min<int64_t>(ch, n_blocks), 16);
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
+    const int64_t items_max = ch * (G - 1);
+    u64* c1c = ar.take<u64>(items_max * LN);
+    u64* digits = ar.take<u64>(items_max * L * L1N);
+    u64* u = ar.take<u64>(items_max * 2 * L1N);
+    u64* up = ar.take<u64>(ch * 2 * N);
+    u64* lifted = ar.take<u64>(ch * 2 * LN);
+    if (!c1c || !digits || !u || !up || !lifted) return fail(c, HANN_EWORKSPACE, "hann_rotate_sum_lazy: workspace too small");
+    const bool lift = ks_lift_available(c);
+    for (int64_t b0 = 0; b0 < n_blocks; b0 += ch) {
+        const int64_t nb = std::min(ch, n_blocks - b0), items = nb * (G - 1);
+        // c1 of term (g, blk), still in the transform domain, into c1c[(g - 1) * nb + blk]
+        bool all_fused = lift;
+        for (int g = 1; g < G; g++) {
+            const u64* src = inner + (b0 * G + g) * ctw + LN;
+            u64* dst = c1c + (int64_t)(g - 1) * nb * LN;
+            const bool fused = lift && ntt_inv_pass_b_gathers(c, src, dst);
+            all_fused = all_fused && fused;
+            if (fused) RET(launch_ntt_inv_pass_b_from(c, src, (int64_t)G * ctw, dst, nb * L, N, limbmap_q(c)));
+            else RET(launch_copy2d(c, dst, LN, src, (int64_t)G * ctw, LN, nb));
+        }
+        if (lift) {
+            if (!all_fused) {
+                // the terms whose inverse pass ran while gathering are finished; the copied ones still need it
+                for (int g = 1; g < G; g++) {
+                    const u64* src = inner + (b0 * G + g) * ctw + LN;
+                    u64* dst = c1c + (int64_t)(g - 1) * nb * LN;
+                    if (!ntt_inv_pass_b_gathers(c, src, dst)) RET(launch_ntt_inv_pass_b(c, dst, nb * L, N, limbmap_q(c)));
+                }
+            }
+            RET(launch_ks_lift(c, c1c, N, items * L, limbmap_q(c), digits, L + 1, 0));
+            RET(launch_ntt_fwd_pass_b(c, digits, items * L * (L + 1), N, limbmap_qp(c)));
+        } else {
+            RET(launch_ntt_inv(c, c1c, items * L, N, limbmap_q(c)));
+            RET(launch_lift_digits(c, c1c, LN, items, digits));
+            RET(launch_ntt_fwd(c, digits, items * L * (L + 1), N, limbmap_qp(c)));
+        }
+        // every giant step under its own key, all in one launch; then the special-prime limb of the SUM of the (permuted)
+        // products, its inverse transform, centred lift and forward transforms: one ModDown per block
+        RET(launch_ks_inner_batches(c, digits, (int64_t)L * L1N, B, B, G - 1, nb, u));
+        RET(launch_giant_sum_p(c, u, nb, up));
+        if (lift) {
+            RET(launch_ntt_inv_pass_b(c, up, nb * 2, N, limbmap_single(L)));
+            RET(launch_ks_lift(c, up, N, nb * 2, limbmap_single(L), lifted, L, 0));
+            RET(launch_ntt_fwd_pass_b(c, lifted, nb * 2 * L, N, limbmap_q(c)));
+        } else {
+            RET(launch_ntt_inv(c, up, nb * 2, N, limbmap_single(L)));
+            RET(launch_lift_p(c, up, nb * 2, lifted));
+            RET(launch_ntt_fwd(c, lifted, nb * 2 * L, N, limbmap_q(c)));
+        }
+        RET(launch_giant_combine(c, u, lifted, inner + b0 * G * ctw, nb, score + b0 * ctw));
+    }
+    return HANN_OK;
+}
+
 extern "C" int hann_keyswitch(hann_ctx* c, int rot, const void* poly_dev, void* ks0_dev, void* ks1_dev, void* ws, size_t ws_bytes) {
     if (!c) return HANN_EINVAL;
     if (!poly_dev || !ks0_dev || !ks1_dev) return fail(c, HANN_EINVAL, "hann_keyswitch: null pointer");
@@ -1256,7 +1340,7 @@ LevelPlan plan_level(const hann_ctx* c, int64_t n_rows, int dim) {
     p.ng = (int)std::max<int64_t>(1, std::min<int64_t>(p.ng, p.nblk));
     // with more than one group: a rotate-and-sum workspace for each of the two scoring streams
     const int64_t gmax = p.nblk - p.nblk * (p.ng - 1) / p.ng;
-    p.ws_score = p.ng > 1 ? align256(ks_item_words(c) * std::min<int64_t>(gmax, 8) * 8 + kSlack) : 0;
+    p.ws_score = p.ng > 1 ? align256(std::max(ks_item_words(c) * std::min<int64_t>(gmax, 8), lazy_block_words(c) * std::min<int64_t>(gmax, 4)) * 8 + kSlack) : 0;
     p.total = p.ct + p.baby + p.rows + p.pt + p.inner + p.score + p.stage + p.ws + 2 * p.ws_score;
     return p;
 }

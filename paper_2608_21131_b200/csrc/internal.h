@@ -76,6 +76,7 @@ struct hann_ctx {
     // ModDown lifts of a single item; hann_rotate_sum raises it to 320 for levels of one or two blocks, whose launches
     // otherwise leave most of the machine idle
     int lift_split_ctas = 160;
+    int giant_lazy = 0;  // hann_rotate_sum (and the calls built on it) evaluates the giant steps in the lazy order
     int encode_sym = 1;  // encode_candidates computes half of every transform and mirrors it (real slot vectors)
     // statistics
     hann_stats stats = {};
@@ -176,6 +177,11 @@ int launch_mac_batch(hann_ctx* c, const u64* baby, int n_queries, const u64* pt,
 int launch_lift_digits(hann_ctx* c, const u64* src, int64_t src_stride, int64_t nitems, u64* digits);
 int launch_ks_inner(hann_ctx* c, const u64* digits, int64_t digit_stride, int rot0, int rot_inc, int64_t nitems, u64* u);
 int launch_moddown_lift(hann_ctx* c, const u64* u, int64_t npoly, u64* lifted);
+// lazy giant steps (items laid out giant step after giant step, see keyswitch.cu)
+int launch_ks_inner_batches(hann_ctx* c, const u64* digits, int64_t digit_stride, int rot0, int rot_zinc, int nz, int64_t per_z, u64* u);
+int launch_giant_sum_p(hann_ctx* c, const u64* u, int64_t nblk, u64* up);
+int launch_lift_p(hann_ctx* c, const u64* up, int64_t npoly, u64* lifted);
+int launch_giant_combine(hann_ctx* c, const u64* u, const u64* lifted, const u64* inner, int64_t nblk, u64* score);
 int launch_moddown_combine(hann_ctx* c, const u64* u, const u64* lifted, int64_t nitems, int rot0, int rot_inc, const u64* c0,
                            int64_t c0_stride, const u64* addend, int64_t addend_stride, u64* out0, u64* out1,
                            int64_t out_stride);

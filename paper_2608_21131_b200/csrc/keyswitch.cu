@@ -162,14 +162,19 @@ __device__ __forceinline__ void ks_inner_body(const u64* __restrict__ digits, lo
     }
 }
 
+// blockIdx.z selects one of several independent batches of `nitems` items laid out one after the other (digits and u), batch
+// z using rotation rot0 + z * rot_zinc: the giant steps of the lazy rotate-and-sum, each under its own key
 template <int LL, bool KEYS_STREAM>
 __global__ void __launch_bounds__(128) k_ks_inner_stream(const u64* __restrict__ digits, long long digit_stride,
                                                          const u64* const* __restrict__ keytab, int rot0, int rot_inc,
                                                          u64* __restrict__ u, int N, long long nitems, int items_per_cta,
-                                                         const LimbConst* __restrict__ lt) {
+                                                         const LimbConst* __restrict__ lt, int rot_zinc) {
     const long long L1N = (long long)(LL + 1) * N;
     const long long pos = (long long)blockIdx.x * 128 + threadIdx.x;  // i*N + x
     const LimbConst lc = lt[pos / N];
+    rot0 += (int)blockIdx.z * rot_zinc;
+    digits += (long long)blockIdx.z * nitems * digit_stride;
+    u += (long long)blockIdx.z * nitems * 2 * L1N;
     const long long it0 = (long long)blockIdx.y * items_per_cta;
     const long long it1 = it0 + items_per_cta < nitems ? it0 + items_per_cta : nitems;
     if (it0 >= it1) return;
@@ -261,6 +266,78 @@ __global__ void __launch_bounds__(256) k_moddown_combine_chunk(
         if (addend) v = addmod(v, addend[item * addend_stride + (long long)comp * LN + (long long)i * N + t], lc.q);
         u64* o = (comp == 0 ? out0 : out1) + item * out_stride + (long long)i * N + t;
         *o = v;
+    }
+}
+
+// ---- lazy giant steps: the key products of G-1 differently rotated terms are summed before ONE ModDown -------------------
+// Items are laid out giant step after giant step: item (g, blk) = (g - 1) * nblk + blk, g = 1 .. G-1; the keys are stored
+// pre-permuted, so the product u of item (g, blk) still awaits the automorphism of rotation g * B.
+
+// up[blk][comp][t] = sum_g u[(g, blk)][comp][limb L][source_g(t)] mod p      (special-prime limb of the summed products)
+__global__ void __launch_bounds__(kThreads) k_giant_sum_p(const u64* __restrict__ u, u64* __restrict__ up, long long nblk, int G, int B,
+                                                          const unsigned* __restrict__ galois, int N, int logN, int L, int tau,
+                                                          LimbTable lt) {
+    const long long L1N = (long long)(L + 1) * N, total = nblk * 2 * N;
+    const u64 p = lt.c[L].q;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const int t = (int)(idx % N);
+        const int comp = (int)((idx / N) % 2);
+        const long long blk = idx / (2 * (long long)N);
+        u64 acc = 0;
+        for (int g = 1; g < G; g++) {
+            const int s = galois_src(t, galois[g * B], logN, tau);
+            acc = addmod(acc, u[((((long long)(g - 1) * nblk + blk) * 2 + comp) * L1N) + (long long)L * N + s], p);
+        }
+        up[idx] = acc;
+    }
+}
+
+// lifted[poly][i][x] = centred lift of up[poly][x] (residue mod p, coefficient domain, polynomials N words apart) mod q_i
+__global__ void __launch_bounds__(kThreads) k_lift_p(const u64* __restrict__ up, u64* __restrict__ lifted, int N, int L, long long npoly,
+                                                     LimbTable lt) {
+    const long long total = npoly * N;
+    const u64 p = lt.c[L].q, half = lt.c[L].half;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const long long poly = idx / N;
+        const int x = (int)(idx % N);
+        const u64 v = up[idx];
+        const bool neg = v > half;
+        const u64 mag = neg ? p - v : v;
+        for (int i = 0; i < L; i++) {
+            u64 r = barrett64(mag, lt.c[i]);
+            lifted[(poly * L + i) * N + x] = (neg && r) ? lt.c[i].q - r : r;
+        }
+    }
+}
+
+// score[blk][comp][i][t] = (sum_g u[(g, blk)][comp][i][source_g(t)] - lifted[blk][comp][i][t]) * p^{-1}
+//                          + inner[blk][0][comp][i][t] + (comp == 0 ? sum_g inner[blk][g][0][i][source_g(t)] : 0)
+// (every aligned chunk of 256 positions maps onto one chunk under an automorphism, so the gathered reads of a CTA stay inside
+// a few cache lines)
+__global__ void __launch_bounds__(kThreads) k_giant_combine(const u64* __restrict__ u, const u64* __restrict__ lifted,
+                                                            const u64* __restrict__ inner, u64* __restrict__ score, long long nblk, int G,
+                                                            int B, const unsigned* __restrict__ galois, int N, int logN, int L, int tau,
+                                                            LimbTable lt) {
+    const long long LN = (long long)L * N, L1N = (long long)(L + 1) * N, ctw = 2 * LN;
+    const long long total = nblk * LN;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const int t = (int)(idx % N);
+        const int i = (int)((idx / N) % L);
+        const long long blk = idx / LN;
+        const LimbConst& lc = lt.c[i];
+        u64 a0 = 0, a1 = 0, c0 = inner[(blk * G) * ctw + (long long)i * N + t];
+        for (int g = 1; g < G; g++) {
+            const int s = galois_src(t, galois[g * B], logN, tau);
+            const u64* ug = u + (((long long)(g - 1) * nblk + blk) * 2) * L1N + (long long)i * N + s;
+            a0 = addmod(a0, ug[0], lc.q);
+            a1 = addmod(a1, ug[L1N], lc.q);
+            c0 = addmod(c0, inner[(blk * G + g) * ctw + (long long)i * N + s], lc.q);
+        }
+        const u64* lf = lifted + (blk * 2 * L + i) * N + t;
+        const u64 v0 = csub(shoup_mul(submod(a0, lf[0], lc.q), lc.pinv, lc.pinv_s, lc.q), lc.q);
+        const u64 v1 = csub(shoup_mul(submod(a1, lf[LN], lc.q), lc.pinv, lc.pinv_s, lc.q), lc.q);
+        score[blk * ctw + (long long)i * N + t] = addmod(v0, c0, lc.q);
+        score[blk * ctw + LN + (long long)i * N + t] = addmod(v1, inner[(blk * G) * ctw + LN + (long long)i * N + t], lc.q);
     }
 }
 
@@ -425,20 +502,21 @@ int launch_lift_digits(hann_ctx* c, const u64* src, int64_t src_stride, int64_t 
 }
 
 template <int LL>
-void launch_ks_inner_stream(hann_ctx* c, const u64* digits, int64_t digit_stride, int rot0, int rot_inc, int64_t nitems, u64* u) {
+void launch_ks_inner_stream(hann_ctx* c, const u64* digits, int64_t digit_stride, int rot0, int rot_inc, int64_t nitems, u64* u,
+                            int nz = 1, int rot_zinc = 0) {
     const long long L1N = (long long)(LL + 1) * c->N;
     const int tiles = (int)(L1N / 128);
     int split = 1;
-    while ((long long)tiles * split < 148 * 8 && split < nitems) split *= 2;
+    while ((long long)tiles * split * nz < 148 * 8 && split < nitems) split *= 2;
     const int per = (int)((nitems + split - 1) / split);
     split = (int)((nitems + per - 1) / per);
     KProf kp(c, digit_stride == 0 && nitems > 1 ? KC_KS_INNER_KEYS : KC_KS_INNER);  // streamed keys timed on their own
     if (digit_stride == 0)
-        k_ks_inner_stream<LL, true><<<dim3(tiles, split), 128, 0, c->stream>>>(digits, 0, c->keytab_dev, rot0, rot_inc, u, c->N, nitems,
-                                                                            per, c->lt_dev);
+        k_ks_inner_stream<LL, true><<<dim3(tiles, split, nz), 128, 0, c->stream>>>(digits, 0, c->keytab_dev, rot0, rot_inc, u, c->N, nitems,
+                                                                                per, c->lt_dev, rot_zinc);
     else
-        k_ks_inner_stream<LL, false><<<dim3(tiles, split), 128, 0, c->stream>>>(digits, digit_stride, c->keytab_dev, rot0, rot_inc, u,
-                                                                             c->N, nitems, per, c->lt_dev);
+        k_ks_inner_stream<LL, false><<<dim3(tiles, split, nz), 128, 0, c->stream>>>(digits, digit_stride, c->keytab_dev, rot0, rot_inc, u,
+                                                                                 c->N, nitems, per, c->lt_dev, rot_zinc);
 }
 
 int launch_ks_inner(hann_ctx* c, const u64* digits, int64_t digit_stride, int rot0, int rot_inc, int64_t nitems, u64* u) {
@@ -459,6 +537,53 @@ int launch_ks_inner(hann_ctx* c, const u64* digits, int64_t digit_stride, int ro
                                                                                    c->N, c->L, nitems, c->lt);
     }
     return check_launch(c, "ks_inner");
+}
+
+// nz batches of `per_z` digit sets each (digits and u laid out batch after batch); every item of batch z is multiplied with
+// the key of rotation rot0 + z * rot_zinc
+int launch_ks_inner_batches(hann_ctx* c, const u64* digits, int64_t digit_stride, int rot0, int rot_zinc, int nz, int64_t per_z, u64* u) {
+    if (nz <= 0 || per_z <= 0) return HANN_OK;
+    if (c->L <= 4 && c->N >= 128 && digit_stride != 0) {
+        switch (c->L) {
+            case 1: launch_ks_inner_stream<1>(c, digits, digit_stride, rot0, 0, per_z, u, nz, rot_zinc); break;
+            case 2: launch_ks_inner_stream<2>(c, digits, digit_stride, rot0, 0, per_z, u, nz, rot_zinc); break;
+            case 3: launch_ks_inner_stream<3>(c, digits, digit_stride, rot0, 0, per_z, u, nz, rot_zinc); break;
+            default: launch_ks_inner_stream<4>(c, digits, digit_stride, rot0, 0, per_z, u, nz, rot_zinc); break;
+        }
+        return check_launch(c, "ks_inner_stream");
+    }
+    for (int z = 0; z < nz; z++) {
+        const int r = launch_ks_inner(c, digits + z * per_z * digit_stride, digit_stride, rot0 + z * rot_zinc, 0, per_z,
+                                      u + z * per_z * 2 * (int64_t)(c->L + 1) * c->N);
+        if (r != HANN_OK) return r;
+    }
+    return HANN_OK;
+}
+
+int launch_giant_sum_p(hann_ctx* c, const u64* u, int64_t nblk, u64* up) {
+    {
+        KProf kp(c, KC_PERMUTE);
+        k_giant_sum_p<<<grid_for(nblk * 2 * c->N), kThreads, 0, c->stream>>>(u, up, nblk, c->G, c->B, c->galois_dev, c->N, c->logN, c->L,
+                                                                           c->ntt_tau, c->lt);
+    }
+    return check_launch(c, "giant_sum_p");
+}
+
+int launch_lift_p(hann_ctx* c, const u64* up, int64_t npoly, u64* lifted) {
+    {
+        KProf kp(c, KC_MODDOWN_LIFT);
+        k_lift_p<<<grid_for(npoly * c->N), kThreads, 0, c->stream>>>(up, lifted, c->N, c->L, npoly, c->lt);
+    }
+    return check_launch(c, "lift_p");
+}
+
+int launch_giant_combine(hann_ctx* c, const u64* u, const u64* lifted, const u64* inner, int64_t nblk, u64* score) {
+    {
+        KProf kp(c, KC_MODDOWN_COMBINE);
+        k_giant_combine<<<grid_for(nblk * c->L * c->N, kThreads, 148 * 32), kThreads, 0, c->stream>>>(
+            u, lifted, inner, score, nblk, c->G, c->B, c->galois_dev, c->N, c->logN, c->L, c->ntt_tau, c->lt);
+    }
+    return check_launch(c, "giant_combine");
 }
 
 int launch_moddown_lift(hann_ctx* c, const u64* u, int64_t npoly, u64* lifted) {

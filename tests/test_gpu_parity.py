@@ -119,6 +119,70 @@ def test_level_bit_exact_small(logN, R, B, L, big, n_rows, dim):
     run_level(p, rows, qv)
 
 
+@pytest.mark.parametrize(
+    "logN,R,B,L,big,n_rows",
+    [
+        (5, 8, 2, 2, False, 40),        # tiny ring (generic kernels), three blocks, G = 4
+        (8, 16, 4, 2, False, 300),      # single-pass transform, three blocks
+        (10, 64, 8, 3, True, 1300),     # 50-bit primes, G = 8, three blocks (fused lift path)
+        (12, 64, 8, 2, False, 4096),    # the toy configuration's ring, G = 8
+        (13, 128, 32, 4, True, 9000),   # production primes and B, G = 4, three blocks
+        (9, 32, 32, 2, False, 300),     # G = 1: nothing to rotate
+    ],
+)
+def test_lazy_giant_steps_bit_exact(logN, R, B, L, big, n_rows):
+    """hann_rotate_sum_lazy (distinct giant-step keys, key products summed, one ModDown per block) against the oracle's
+    evaluation in the same order, bit for bit; its decrypted scores within the tolerance, and within the key-switch noise
+    of the Horner evaluation of the same partial sums."""
+    import torch
+
+    from paper_2608_21131_b200 import binding as b
+
+    ps = synth.small_params(logN, R, B, L=L, big=big)
+    if big:
+        ps = ps.with_(log_scale=40)
+    G = ps.G
+    rots = sorted(set(range(1, B + 1)) | {g * B for g in range(1, G)})
+    g_, o = b.Context(ps), make_oracle(ps)
+    km = synth.key_material(ps, logN, rots=rots)
+    evk_o = dict(zip(rots, (o.evk_gen(km.s, r, km.evk_a[i], km.evk_e[i]) for i, r in enumerate(rots))))
+    evk_g = g_.keygen_from_samples(km.s, km.rots, km.evk_a, km.evk_e)
+    g_.load_keys(evk_g, km.rots)
+    rows = synth.toy_corpus(logN, rows=n_rows, dim=R)
+    qv = synth.toy_query(logN + 1, dim=R)
+    ct = g_.encrypt_query(km.s, qv, km.ct_a, km.ct_e)
+    nb = g_.n_blocks(n_rows)
+    ws = g_.workspace(nb)
+    baby = g_.query_prepare(g_.import_(b.KIND_CT, ct, 1), ws)
+    inner = g_.score_level(baby, g_.encode_candidates(torch.from_numpy(rows).to(g_.device), ws), nb, ws)
+    score = g_.rotate_sum_lazy(inner, nb, ws)
+    horner = g_.rotate_sum(inner, nb, ws)
+    g_.sync()
+    score_h, inner_h = g_.export(b.KIND_CT, score, nb), g_.export(b.KIND_CT, inner, nb * G).reshape(nb, G, 2, L, ps.N)
+    giant = (np.stack([evk_o[g * B] for g in range(1, G)]) if G > 1
+             else np.zeros((0, L, 2, L + 1, ps.N), dtype=np.uint64))
+    for blk in range(nb):
+        assert np.array_equal(score_h[blk], o.rotate_sum_lazy(inner_h[blk], giant)), blk
+    got = g_.decrypt_scores(km.s, score_h).reshape(-1)[:n_rows]
+    want = rows.astype(np.float64) @ qv.astype(np.float64)
+    assert np.abs(got - want).max() < 2.0 ** ps.tol_log2
+    got_h = g_.decrypt_scores(km.s, g_.export(b.KIND_CT, horner, nb)).reshape(-1)[:n_rows]
+    assert np.abs(got - got_h).max() < 2.0 ** ps.tol_log2
+    # a tight workspace (one block per round) gives the same bits
+    if nb > 1:
+        tight = g_.alloc(g_.workspace_bytes(1))
+        again = g_.rotate_sum_lazy(inner, nb, tight)
+        g_.sync()
+        assert torch.equal(again, score)
+    # a missing giant-step key is reported, not guessed
+    if G > 2:
+        h = b.Context(ps)
+        h.load_keys(evk_g[: B], km.rots[: B])
+        with pytest.raises(b.HannError) as ei:
+            h.rotate_sum_lazy(inner, nb, ws)
+        assert ei.value.code == b.ENOKEY
+
+
 def test_toy_configuration_full():
     """Toy configuration: 4,096 unit-norm rows of dimension 64, N = 2^12, scale 2^25 -> two blocks; every conformance
     point bit-exact, every score within 2^-10; repeated with three seed triples."""

@@ -9,7 +9,7 @@ import numpy as np
 import pytest
 import sympy
 
-from oracle.oracle import Oracle, find_primes, is_prime
+from oracle.oracle import Oracle, PackedProjection, find_primes, is_prime, restrict_keys
 from paper_2608_21131_b200 import synth
 from tests.helpers import rescale_error_bound, rescale_error_sigma
 
@@ -470,6 +470,80 @@ def test_lazy_giant_steps_without_noise_equal_plain_matvec(logN, R, B):
     assert np.abs(got.real - want).max() < 2e-5 and np.abs(got.imag).max() < 2e-5
     if ps.G == 1:
         assert np.array_equal(score, inner[0])
+
+
+# ------------------------------------------------------------------ packed projection (Sec. 3.1 Detail)
+
+
+@pytest.mark.parametrize("D,R,B", [(16, 16, 4), (32, 16, 4), (64, 16, 2), (64, 16, 16), (64, 8, 1), (128, 32, 8)])
+def test_packed_projection_on_plain_slots_is_the_matrix_product(D, R, B):
+    """the index formulas alone, no encryption: packed diagonals, in-window rotations from two slot rotations and 0/1
+    masks, giant steps by plain slot rotations, ONE final fold -> every slot i holds (W^T q)[i mod R]"""
+    pp = PackedProjection(9, synth.Q50, synth.P60, 40, D, R, B, 50, 50)
+    rng = np.random.default_rng(D + R + B)
+    W, qv = rng.standard_normal((D, R)), rng.standard_normal(D)
+    got, unfolded = pp.plain(W, qv)
+    want = np.tile(W.T @ qv, pp.n // R)
+    assert np.abs(got - want).max() < 1e-12
+    lo, hi = pp.masks()
+    assert np.array_equal(lo + hi, np.ones_like(lo)) and set(np.unique(lo)) <= {0.0, 1.0}
+    # masks + two slot rotations = rotation inside every window of R slots
+    x = pp.query_slots(qv)
+    for b in range(B):
+        inwin = np.roll(x.reshape(-1, R), -b, axis=1).reshape(-1)
+        assert np.array_equal(lo[b] * np.roll(x, -b) + hi[b] * np.roll(x, -(b - R)), inwin)
+    if D > R and B < R:
+        # before the fold a window holds a mix of chunk products, not the answer: the fold is what makes it right, and it
+        # is needed once only (folding commutes with the slot rotations of the giant steps)
+        assert np.abs(unfolded - want).max() > 1e-3
+        assert np.abs(sum(np.roll(unfolded, -k * R) for k in range(D // R)) - want).max() < 1e-12
+
+
+def test_keys_of_a_shorter_chain_are_a_restriction_of_the_longer_chain_keys():
+    ps = synth.small_params(7, 8, 4, L=4, big=True)
+    km = synth.key_material(ps, 12, rots=[3])
+    full = make(ps).evk_gen(km.s, 3, km.evk_a[0], km.evk_e[0])
+    for Lt in (3, 2):
+        short = Oracle(ps.logN, ps.q[:Lt], ps.p, ps.log_scale, ps.R, ps.B)
+        limbs = list(range(Lt)) + [ps.L]
+        want = short.evk_gen(km.s, 3, km.evk_a[0][:Lt][:, limbs], km.evk_e[0][:Lt])
+        assert np.array_equal(restrict_keys(full, ps.L, Lt), want)
+
+
+@pytest.mark.parametrize("logN,D,R,B,lazy", [(9, 64, 16, 4, False), (10, 128, 32, 4, True), (9, 32, 32, 8, False)])
+def test_packed_projection_under_encryption(logN, D, R, B, lazy):
+    """the encrypted pipeline at production primes (4 x 50 bits + 60, scale 2^40, masks and matrix at 2^50): the result
+    decrypts, at its exact scale Delta 2^50/q_3 2^50/q_2, to the float64 W^T q tiled over the slots within 2^-20, on the
+    chain of L - 2 primes; it equals the UNPACKED projection (one D-diagonal block through the ordinary scorer) within
+    the same tolerance."""
+    pp = PackedProjection(logN, synth.Q50, synth.P60, 40, D, R, B, 50, 50)
+    top = pp.top
+    rots = sorted(set(pp.baby_rotations()) | {g * B for g in range(1, pp.G)} | set(pp.fold_rotations()))
+    ps = synth.ParamSet("pp", logN, synth.Q50, synth.P60, 40, R, B, -18)
+    km = synth.key_material(ps, 61, rots=rots)
+    evk = dict(zip(rots, all_keys(top, km)))
+    rng = np.random.default_rng(5)
+    W = np.linalg.qr(rng.standard_normal((D, R)))[0]
+    qv = rng.standard_normal(D)
+    qv = (qv / np.linalg.norm(qv)).astype(np.float32)
+    ct = top.encrypt(km.s, top.encode(pp.query_slots(qv)), km.ct_a, km.ct_e)
+    out = pp.project(ct, evk, pp.enrol(W), lazy=lazy)
+    assert out.shape == (2, 2, pp.N)
+    mu = pp.low.decrypt_int(km.s, out)
+    slots = pp.low.decode(np.array([float(v) for v in mu]), pp.scale_out)
+    want = np.tile(W.T.astype(np.float64) @ qv.astype(np.float64), pp.n // R)
+    assert np.abs(slots.real - want).max() < 2.0 ** -20 and np.abs(slots.imag).max() < 2.0 ** -20
+    assert abs(pp.scale_out / 2.0 ** 40 - 1.0) < 2.0 ** -20          # the two rescales bring the scale back to ~Delta
+    # the unpacked projection: W^T tiled down the slots as one block of D diagonals, ordinary scorer (R = D)
+    ub = min(B, D)
+    un = Oracle(logN, synth.Q50, synth.P60, 40, D, ub)
+    kmu = synth.key_material(synth.ParamSet("un", logN, synth.Q50, synth.P60, 40, D, ub, -18), 61)
+    evu = all_keys(un, kmu)
+    block = np.tile(W.T.astype(np.float32), (pp.n // R, 1))
+    ctu = un.encrypt_query(kmu.s, qv, kmu.ct_a, kmu.ct_e)
+    sc, _, _ = un.score_block(block, un.baby_set(ctu, evu), evu[ub - 1])
+    plain = un.decrypt_slots(kmu.s, sc, 80).real
+    assert np.abs(plain - slots.real).max() < 2.0 ** -19
 
 
 def test_zero_padding_96_to_128_is_exact():

@@ -314,6 +314,65 @@ int64_t hann_keyswitch_bytes(const hann_ctx *ctx);
 int64_t hann_static_scratch_bytes(void);
 int hann_keyswitch_static(hann_ctx *ctx, int rot, const void *poly_dev, void *ks0_dev, void *ks1_dev);
 
+/* ---- rank reduction under encryption, projection matrix packed by windows (Sec. 3.1 "How" and Detail) -----------------
+ * Enc(q_R) = W^T Enc(q) for W of shape D x R, D = c R, c a power of two, D dividing n.  Reading taken (the paper gives no
+ * index formulas): the n slots are viewed with period D, window k of a period is positions kR .. kR+R-1, and the query
+ * ciphertext holds q[i mod D].  Chunk k of W is the R x R matrix W_k^T[r][col] = W[kR + col][r].
+ *   - Packing: ONE stored plaintext per diagonal gB + b holds that diagonal of ALL c chunks, chunk k in window k, shifted
+ *     inside its window by the giant-step amount: slot kR + j holds W[kR + (j + b) mod R][(j - gB) mod R].  R objects
+ *     instead of D (the paper's factor c = 512 / R).
+ *   - Baby steps: every chunk of the query must rotate INSIDE its window, which a slot rotation does not do; it is put
+ *     together from two slot rotations and 0/1 plaintext masks -- a ciphertext x plaintext multiply, no key switch:
+ *     cyc_b = lo_b * rot_b(ct) + hi_b * rot_{b-R}(ct), lo_b[i] = [(i mod R) + b < R], hi_b = 1 - lo_b.  One rescale follows.
+ *   - Matrix product and giant steps: inner[g] = sum_b packed[g][b] * cyc_b, then sum_g rot_{gB}(inner[g]) with plain slot
+ *     rotations.  These mix adjacent windows; the single final fold acc += rot_{R 2^t}(acc), t < log2 c, adds all windows
+ *     up, and a fixed permutation of the windows is invisible to that sum.  Every slot i then holds q_R[i mod R]: the
+ *     projected query, already tiled for the scoring levels.  A second rescale brings the scale back to about Delta.
+ * Three contexts of the same ring, R, B and special prime carry this: `top` (L primes: baby rotations, masks), `mid` (the
+ * first L - 1 primes: matrix product, giant steps, fold) and the scoring context (the first L - 2 primes).  Evaluation
+ * keys of a shorter chain are the longer chain's keys restricted to its digits and limbs (one-prime digits), so the
+ * client generates them once.  Keys needed: top: rotations b and n - R + b, b = 1 .. B-1; mid: B (Horner; or B .. (G-1)B
+ * with HANN_TUNE_GIANT_LAZY) and R 2^t, t < log2 c. */
+
+/* Hoisted slot rotations of one ciphertext: out[i] = rot_{rot0 + i}(ct), i < count -- one digit decomposition of c1, count
+ * keys, one ModDown round (what hann_query_prepare does for rotations 1 .. B-1).  out_dev count * HANN_SIZE_CT bytes. */
+int hann_rotate_hoisted(hann_ctx *ctx, const void *ct_dev, int rot0, int count, void *out_dev, void *ws, size_t ws_bytes);
+
+/* Encode `count` real slot vectors z_dev [count][n] (device, binary64) at scale 2^log_scale into stored plaintexts
+ * pt_dev [count][L][N/2] (the layout of one (g, b) plaintext of hann_encode_candidates).  Enrolment-time call. */
+int hann_encode_slots(hann_ctx *ctx, const double *z_dev, int64_t count, int log_scale, void *pt_dev, void *ws, size_t ws_bytes);
+
+/* Enrolment of the projection matrix: W_dev [D][R] float32 row-major (device) -> the R packed diagonals, pt_dev
+ * [G][B][L][N/2] (HANN_SIZE_PT_BLOCK bytes: "one block" for hann_score_level) at scale 2^log_scale_w.  Call it on `mid`.
+ * ws: hann_workspace_bytes(ctx, 1) is enough. */
+int hann_project_enrol(hann_ctx *ctx, const float *W_dev, int D, int log_scale_w, void *pt_dev, void *ws, size_t ws_bytes);
+
+/* The window masks lo_b, hi_b, b < B, as stored plaintexts [B][L][N/2] each at scale 2^log_scale_m.  Call it on `top`. */
+int hann_project_masks(hann_ctx *ctx, int log_scale_m, void *lo_dev, void *hi_dev, void *ws, size_t ws_bytes);
+
+/* The baby steps inside the windows: cyc_dev [B] ciphertexts (HANN_SIZE_BABY bytes, scale Delta * mask scale), from two
+ * hoisted batches of slot rotations and the mask combine.  ws: hann_project_bytes is enough. */
+int hann_project_baby(hann_ctx *ctx, const void *ct_dev, const void *lo_dev, const void *hi_dev, void *cyc_dev, void *ws,
+                      size_t ws_bytes);
+
+/* Rescale (the step between two multiplications of a CKKS circuit): every polynomial of `count` ciphertexts is divided
+ * by the last prime with rounding, c' = (c - [c]_{q_{L-1}}) / q_{L-1}, which divides message and scale by q_{L-1}.
+ * out_dev [count][2][L-1][N]: ciphertexts of the context whose chain is the first L - 1 primes.  (hann_compact_scores
+ * with keep = L - 1 under the name the operation has in a circuit.) */
+int hann_rescale(hann_ctx *ctx, const void *ct_dev, int64_t count, void *out_dev, void *ws, size_t ws_bytes);
+
+/* Fold: ct += rot_{stride * 2^t}(ct) for t = 0 .. steps-1, in place (keys of those rotations must be loaded).  With
+ * stride = R and steps = log2(D / R) this is the projection's final sum over the windows. */
+int hann_fold(hann_ctx *ctx, void *ct_dev, int stride, int steps, void *ws, size_t ws_bytes);
+
+/* The whole projection: hann_project_baby and hann_rescale on `top`, then hann_score_level (against the packed matrix as
+ * its one block), hann_rotate_sum, hann_fold and hann_rescale on `mid`.  ct_dev: the query on `top`; out_dev: the projected
+ * query, one ciphertext of the scoring context ([2][L-2][N]) at scale Delta * 2^log_scale_m / q_{L-1} * 2^log_scale_w /
+ * q_{L-2}.  Both contexts must use the same device and stream.  ws: hann_project_bytes(top, mid) bytes. */
+int64_t hann_project_bytes(const hann_ctx *top, const hann_ctx *mid);
+int hann_project_query(hann_ctx *top, hann_ctx *mid, const void *ct_dev, const void *lo_dev, const void *hi_dev,
+                       const void *wpt_dev, int D, void *out_dev, void *ws, size_t ws_bytes);
+
 /* Convert `count` elements between the canonical layout (host or device pointer) and the internal device layout.
  * kind POLY / PT: one polynomial of L limbs per element; CT: two.  The canonical form of every kind is [L][N] words per
  * polynomial; the internal form of POLY and CT has the same size, that of PT half of it (HANN_SIZE_PT_BLOCK / R per

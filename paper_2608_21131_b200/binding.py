@@ -91,6 +91,15 @@ def load_library():
         "hann_score_level_batch": (C.c_int, [vp, vp, C.c_int, vp, i64, vp, vp, sz]),
         "hann_rotate_sum": (C.c_int, [vp, vp, i64, vp, vp, sz]),
         "hann_rotate_sum_lazy": (C.c_int, [vp, vp, i64, vp, vp, sz]),
+        "hann_rotate_hoisted": (C.c_int, [vp, vp, C.c_int, C.c_int, vp, vp, sz]),
+        "hann_encode_slots": (C.c_int, [vp, vp, i64, C.c_int, vp, vp, sz]),
+        "hann_project_enrol": (C.c_int, [vp, vp, C.c_int, C.c_int, vp, vp, sz]),
+        "hann_project_masks": (C.c_int, [vp, C.c_int, vp, vp, vp, sz]),
+        "hann_project_baby": (C.c_int, [vp, vp, vp, vp, vp, vp, sz]),
+        "hann_rescale": (C.c_int, [vp, vp, i64, vp, vp, sz]),
+        "hann_fold": (C.c_int, [vp, vp, C.c_int, C.c_int, vp, sz]),
+        "hann_project_bytes": (i64, [vp, vp]),
+        "hann_project_query": (C.c_int, [vp, vp, vp, vp, vp, vp, C.c_int, vp, vp, sz]),
         "hann_keyswitch": (C.c_int, [vp, C.c_int, vp, vp, vp, vp, sz]),
         "hann_query_level": (C.c_int, [vp, vp, vp, i64, C.c_int, vp, vp, vp, vp, vp, sz]),
         "hann_static_scratch_bytes": (i64, []),
@@ -126,6 +135,14 @@ def _ptr(a):
     if isinstance(a, np.ndarray):
         return a.ctypes.data
     return a.data_ptr()
+
+
+def restrict_keys(evk, L_from, L_to):
+    """Evaluation keys [..][L_from][2][L_from+1][N] (canonical) restricted to the chain of the first L_to primes: digits
+    0..L_to-1 and limbs q_0..q_{L_to-1} plus the special prime.  Pure slicing: with one-prime digits that IS the key of
+    the shorter chain, so a client generates keys once for its longest chain."""
+    limbs = list(range(L_to)) + [L_from]
+    return np.ascontiguousarray(np.asarray(evk)[..., :L_to, :, :, :][..., limbs, :])
 
 
 class Context:
@@ -395,6 +412,56 @@ class Context:
         self._ck(self.lib.hann_query_level(self.h, _ptr(ct_dev), _ptr(rows_dev), n_rows, dim, _ptr(baby), _ptr(pt), _ptr(inner),
                                            _ptr(score), _ptr(ws), ws.numel() * 8))
         return score
+
+    # ---- packed projection
+    def rotate_hoisted(self, ct_dev, rot0, count, ws, out=None):
+        if out is None:
+            out = self.alloc(max(count, 1) * self.sizeof(SIZE_CT))
+        self._ck(self.lib.hann_rotate_hoisted(self.h, _ptr(ct_dev), rot0, count, _ptr(out), _ptr(ws), ws.numel() * 8))
+        return out
+
+    def encode_slots(self, z_dev, log_scale, ws):
+        count = z_dev.shape[0]
+        assert z_dev.dtype == self.torch.float64 and z_dev.is_contiguous() and z_dev.shape[1] == self.n
+        pt = self.alloc(count * self.sizeof(SIZE_POLY) // 2)
+        self._ck(self.lib.hann_encode_slots(self.h, _ptr(z_dev), count, log_scale, _ptr(pt), _ptr(ws), ws.numel() * 8))
+        return pt
+
+    def project_enrol(self, W_dev, log_scale_w, ws):
+        D, R = W_dev.shape
+        assert R == self.R and W_dev.dtype == self.torch.float32 and W_dev.is_contiguous()
+        pt = self.alloc(self.sizeof(SIZE_PT_BLOCK))
+        self._ck(self.lib.hann_project_enrol(self.h, _ptr(W_dev), D, log_scale_w, _ptr(pt), _ptr(ws), ws.numel() * 8))
+        return pt
+
+    def project_masks(self, log_scale_m, ws):
+        lo = self.alloc(self.B * self.sizeof(SIZE_POLY) // 2)
+        hi = self.alloc(self.B * self.sizeof(SIZE_POLY) // 2)
+        self._ck(self.lib.hann_project_masks(self.h, log_scale_m, _ptr(lo), _ptr(hi), _ptr(ws), ws.numel() * 8))
+        return lo, hi
+
+    def project_baby(self, ct_dev, lo, hi, ws):
+        cyc = self.alloc(self.sizeof(SIZE_BABY))
+        self._ck(self.lib.hann_project_baby(self.h, _ptr(ct_dev), _ptr(lo), _ptr(hi), _ptr(cyc), _ptr(ws), ws.numel() * 8))
+        return cyc
+
+    def rescale(self, ct_dev, count, ws):
+        out = self.alloc(self.lib.hann_compact_bytes(self.h, count, self.L - 1))
+        self._ck(self.lib.hann_rescale(self.h, _ptr(ct_dev), count, _ptr(out), _ptr(ws), ws.numel() * 8))
+        return out
+
+    def fold(self, ct_dev, stride, steps, ws):
+        self._ck(self.lib.hann_fold(self.h, _ptr(ct_dev), stride, steps, _ptr(ws), ws.numel() * 8))
+        return ct_dev
+
+    def project_query(self, mid, ct_dev, lo, hi, wpt, D, ws=None):
+        """the projected query: one ciphertext of the chain with two primes fewer, [2][L-2][N] internal"""
+        if ws is None:
+            ws = self.alloc(self.lib.hann_project_bytes(self.h, mid.h))
+        out = self.alloc(mid.lib.hann_compact_bytes(mid.h, 1, mid.L - 1))
+        self._ck(self.lib.hann_project_query(self.h, mid.h, _ptr(ct_dev), _ptr(lo), _ptr(hi), _ptr(wpt), D, _ptr(out), _ptr(ws),
+                                             ws.numel() * 8))
+        return out
 
     def keyswitch(self, rot, poly, ws):
         ks0 = self.alloc(self.sizeof(SIZE_POLY))

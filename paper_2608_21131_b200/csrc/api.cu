@@ -971,30 +971,46 @@ extern "C" int hann_load_keys(hann_ctx* c, const uint64_t* evk, int n_rot, const
     return HANN_OK;
 }
 
+// out[i] = rot_{rot0 + i}(ct), i < count: one digit decomposition of c1, count keys, one ModDown round
+static int rotate_hoisted(hann_ctx* c, const char* who, const u64* ct, int rot0, int count, u64* out, void* ws, size_t ws_bytes) {
+    const int L = c->L, N = c->N;
+    const int64_t LN = (int64_t)L * N, L1N = (int64_t)(L + 1) * N, ctw = 2 * LN;
+    if (count <= 0) return HANN_OK;
+    if (rot0 < 1 || rot0 + count > c->n) return fail(c, HANN_ESHAPE, (std::string(who) + ": rotation out of range").c_str());
+    for (int r = rot0; r < rot0 + count; r++)
+        if (!c->keytab_host[r]) return fail(c, HANN_ENOKEY, (std::string(who) + ": a rotation key is not loaded").c_str());
+    if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, (std::string(who) + ": workspace missing or not 256-byte aligned").c_str());
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
+    u64* c1c = ar.take<u64>(LN);
+    u64* digits = ar.take<u64>(L * L1N);
+    u64* u = ar.take<u64>((int64_t)count * 2 * L1N);
+    u64* lifted = ar.take<u64>((int64_t)count * 2 * LN);
+    if (!c1c || !digits || !u || !lifted) return fail(c, HANN_EWORKSPACE, (std::string(who) + ": workspace too small").c_str());
+    // one digit set, count keys: item i uses rotation rot0 + i
+    RET(ks_digits_to_lifted(c, c1c, 1, digits, 0, rot0, 1, count, u, lifted, ct + LN, 2 * LN));
+    RET(launch_moddown_combine(c, u, lifted, count, rot0, 1, ct, 0, nullptr, 0, out, out + LN, ctw));
+    return HANN_OK;
+}
+
 extern "C" int hann_query_prepare(hann_ctx* c, const void* ct_dev, void* baby_dev, void* ws, size_t ws_bytes) {
     if (!c) return HANN_EINVAL;
     if (!ct_dev || !baby_dev) return fail(c, HANN_EINVAL, "hann_query_prepare: null pointer");
-    const int L = c->L, N = c->N, B = c->B;
-    const int64_t LN = (int64_t)L * N, L1N = (int64_t)(L + 1) * N, ctw = 2 * LN;
-    for (int r = 1; r < B; r++)
+    const int64_t ctw = 2 * (int64_t)c->L * c->N;
+    for (int r = 1; r < c->B; r++)
         if (!c->keytab_host[r]) return fail(c, HANN_ENOKEY, "hann_query_prepare: a baby-step rotation key is not loaded");
     DeviceGuard dg(c->device);
     Timer tm(c, 0);
     const u64* ct = (const u64*)ct_dev;
     u64* baby = (u64*)baby_dev;
     RET(launch_copy2d(c, baby, ctw, ct, ctw, ctw, 1));  // rotation 0
-    if (B == 1) return HANN_OK;
-    if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_query_prepare: workspace missing or not 256-byte aligned");
-    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
-    u64* c1c = ar.take<u64>(LN);
-    u64* digits = ar.take<u64>(L * L1N);
-    u64* u = ar.take<u64>((int64_t)(B - 1) * 2 * L1N);
-    u64* lifted = ar.take<u64>((int64_t)(B - 1) * 2 * LN);
-    if (!c1c || !digits || !u || !lifted) return fail(c, HANN_EWORKSPACE, "hann_query_prepare: workspace too small");
-    // one digit set, B-1 keys: item i uses rotation 1 + i
-    RET(ks_digits_to_lifted(c, c1c, 1, digits, 0, 1, 1, B - 1, u, lifted, ct + LN, 2 * LN));
-    RET(launch_moddown_combine(c, u, lifted, B - 1, 1, 1, ct, 0, nullptr, 0, baby + ctw, baby + ctw + LN, ctw));
-    return HANN_OK;
+    return rotate_hoisted(c, "hann_query_prepare", ct, 1, c->B - 1, baby + ctw, ws, ws_bytes);
+}
+
+extern "C" int hann_rotate_hoisted(hann_ctx* c, const void* ct_dev, int rot0, int count, void* out_dev, void* ws, size_t ws_bytes) {
+    if (!c) return HANN_EINVAL;
+    if (!ct_dev || !out_dev || count < 0) return fail(c, HANN_EINVAL, "hann_rotate_hoisted: bad argument");
+    DeviceGuard dg(c->device);
+    return rotate_hoisted(c, "hann_rotate_hoisted", (const u64*)ct_dev, rot0, count, (u64*)out_dev, ws, ws_bytes);
 }
 
 extern "C" int hann_encode_candidates(hann_ctx* c, const float* rows_dev, int64_t n_rows, int dim, void* pt_dev, void* ws,
@@ -1262,6 +1278,182 @@ extern "C" int hann_rotate_sum_lazy(hann_ctx* c, const void* inner_dev, int64_t 
         }
         RET(launch_giant_combine(c, u, lifted, inner + b0 * G * ctw, nb, score + b0 * ctw));
     }
+    return HANN_OK;
+}
+
+// ================================================================================================ packed projection
+
+// count real slot vectors z [count][n] (device doubles) -> stored plaintexts [count][L][N/2] at scale 2^log_scale: canonical
+// encode, full transform in the staging area, first half kept
+static int encode_slot_vectors(hann_ctx* c, const double* z, int64_t count, int log_scale, u64* pt, void* ws, size_t ws_bytes) {
+    if ((int64_t)ws_bytes < encode_ws_bytes(c)) return fail(c, HANN_EWORKSPACE, "slot-vector encoding: workspace too small");
+    u64* stage = (u64*)((char*)ws + encode_fft_bytes(c));
+    const int64_t n = c->n, Ln = (int64_t)c->L * n;
+    for (int64_t i = 0; i < count; i++) {
+        RET(launch_encode_slots(c, z + i * n, stage, ws, log_scale));
+        RET(launch_ntt_fwd(c, stage, c->L, c->N, limbmap_q(c)));
+        RET(launch_copy2d(c, pt + i * Ln, n, stage, c->N, n, c->L));
+    }
+    return HANN_OK;
+}
+
+extern "C" int hann_encode_slots(hann_ctx* c, const double* z_dev, int64_t count, int log_scale, void* pt_dev, void* ws, size_t ws_bytes) {
+    if (!c) return HANN_EINVAL;
+    if (count < 0 || (count > 0 && (!z_dev || !pt_dev))) return fail(c, HANN_EINVAL, "hann_encode_slots: bad argument");
+    if (log_scale < 1 || log_scale > 60) return fail(c, HANN_EINVAL, "hann_encode_slots: scale must be 2^1 .. 2^60");
+    if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_encode_slots: workspace missing or not 256-byte aligned");
+    DeviceGuard dg(c->device);
+    return encode_slot_vectors(c, z_dev, count, log_scale, (u64*)pt_dev, ws, ws_bytes);
+}
+
+extern "C" int hann_project_enrol(hann_ctx* c, const float* W_dev, int D, int log_scale_w, void* pt_dev, void* ws, size_t ws_bytes) {
+    if (!c) return HANN_EINVAL;
+    if (!W_dev || !pt_dev) return fail(c, HANN_EINVAL, "hann_project_enrol: null pointer");
+    if (D < c->R || D % c->R || c->n % D) return fail(c, HANN_ESHAPE, "hann_project_enrol: D must be a multiple of R that divides n");
+    if (log_scale_w < 1 || log_scale_w > 60) return fail(c, HANN_EINVAL, "hann_project_enrol: scale must be 2^1 .. 2^60");
+    if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_project_enrol: workspace missing or not 256-byte aligned");
+    const int64_t zb = align256((int64_t)c->n * 8);
+    if ((int64_t)ws_bytes < zb + encode_ws_bytes(c)) return fail(c, HANN_EWORKSPACE, "hann_project_enrol: workspace too small");
+    DeviceGuard dg(c->device);
+    double* z = (double*)ws;
+    const int64_t Ln = (int64_t)c->L * c->n;
+    for (int g = 0; g < c->G; g++)
+        for (int b = 0; b < c->B; b++) {
+            RET(launch_packed_diagonal(c, W_dev, D, g, b, z));
+            RET(encode_slot_vectors(c, z, 1, log_scale_w, (u64*)pt_dev + ((int64_t)g * c->B + b) * Ln, (char*)ws + zb, ws_bytes - (size_t)zb));
+        }
+    return HANN_OK;
+}
+
+extern "C" int hann_project_masks(hann_ctx* c, int log_scale_m, void* lo_dev, void* hi_dev, void* ws, size_t ws_bytes) {
+    if (!c) return HANN_EINVAL;
+    if (!lo_dev || !hi_dev) return fail(c, HANN_EINVAL, "hann_project_masks: null pointer");
+    if (log_scale_m < 1 || log_scale_m > 60) return fail(c, HANN_EINVAL, "hann_project_masks: scale must be 2^1 .. 2^60");
+    if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_project_masks: workspace missing or not 256-byte aligned");
+    const int64_t zb = align256((int64_t)c->n * 8);
+    if ((int64_t)ws_bytes < 2 * zb + encode_ws_bytes(c)) return fail(c, HANN_EWORKSPACE, "hann_project_masks: workspace too small");
+    DeviceGuard dg(c->device);
+    double *lo = (double*)ws, *hi = (double*)((char*)ws + zb);
+    const int64_t Ln = (int64_t)c->L * c->n;
+    for (int b = 0; b < c->B; b++) {
+        RET(launch_window_masks(c, b, lo, hi));
+        RET(encode_slot_vectors(c, lo, 1, log_scale_m, (u64*)lo_dev + b * Ln, (char*)ws + 2 * zb, ws_bytes - (size_t)(2 * zb)));
+        RET(encode_slot_vectors(c, hi, 1, log_scale_m, (u64*)hi_dev + b * Ln, (char*)ws + 2 * zb, ws_bytes - (size_t)(2 * zb)));
+    }
+    return HANN_OK;
+}
+
+// words of workspace hann_project_baby needs: the two batches of rotated ciphertexts and one hoisted rotation round
+static int64_t project_baby_words(const hann_ctx* c) {
+    const int64_t L = c->L, N = c->N, nb = std::max(c->B - 1, 1);
+    return 2 * nb * 2 * L * N + prepare_words(c);
+}
+
+extern "C" int hann_project_baby(hann_ctx* c, const void* ct_dev, const void* lo_dev, const void* hi_dev, void* cyc_dev, void* ws,
+                                 size_t ws_bytes) {
+    if (!c) return HANN_EINVAL;
+    if (!ct_dev || !lo_dev || !hi_dev || !cyc_dev) return fail(c, HANN_EINVAL, "hann_project_baby: null pointer");
+    if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_project_baby: workspace missing or not 256-byte aligned");
+    const int B = c->B;
+    const int64_t ctw = 2 * (int64_t)c->L * c->N;
+    DeviceGuard dg(c->device);
+    Timer tm(c, 0);
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
+    u64* rot_a = ar.take<u64>(std::max(B - 1, 1) * ctw);
+    u64* rot_h = ar.take<u64>(std::max(B - 1, 1) * ctw);
+    if (!rot_a || !rot_h) return fail(c, HANN_EWORKSPACE, "hann_project_baby: workspace too small");
+    char* sub = (char*)ws + ar.off;
+    const size_t sub_bytes = ws_bytes - (size_t)ar.off;
+    // rot_b(ct) and rot_{b-R}(ct) (the latter as the slot rotation by n - R + b), b = 1 .. B-1, each batch hoisted
+    RET(rotate_hoisted(c, "hann_project_baby", (const u64*)ct_dev, 1, B - 1, rot_a, sub, sub_bytes));
+    RET(rotate_hoisted(c, "hann_project_baby", (const u64*)ct_dev, c->n - c->R + 1, B - 1, rot_h, sub, sub_bytes));
+    return launch_mask_combine(c, (const u64*)ct_dev, rot_a, rot_h, (const u64*)lo_dev, (const u64*)hi_dev, (u64*)cyc_dev);
+}
+
+extern "C" int hann_rescale(hann_ctx* c, const void* ct_dev, int64_t count, void* out_dev, void* ws, size_t ws_bytes) {
+    if (!c) return HANN_EINVAL;
+    if (c->L < 2) return fail(c, HANN_ESHAPE, "hann_rescale: the chain has a single prime left");
+    return hann_compact_scores(c, ct_dev, count, c->L - 1, 1, out_dev, ws, ws_bytes);
+}
+
+extern "C" int hann_fold(hann_ctx* c, void* ct_dev, int stride, int steps, void* ws, size_t ws_bytes) {
+    if (!c) return HANN_EINVAL;
+    if (!ct_dev || stride < 1 || steps < 0) return fail(c, HANN_EINVAL, "hann_fold: bad argument");
+    if (steps == 0) return HANN_OK;
+    if (((int64_t)stride << (steps - 1)) >= c->n) return fail(c, HANN_ESHAPE, "hann_fold: rotation out of range");
+    for (int t = 0; t < steps; t++)
+        if (!c->keytab_host[stride << t]) return fail(c, HANN_ENOKEY, "hann_fold: the keys of rotations stride * 2^t must be loaded");
+    if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_fold: workspace missing or not 256-byte aligned");
+    const int L = c->L, N = c->N;
+    const int64_t LN = (int64_t)L * N, L1N = (int64_t)(L + 1) * N, ctw = 2 * LN;
+    DeviceGuard dg(c->device);
+    Timer tm(c, 3);
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
+    KsBuffers kb;
+    u64* tmp = ar.take<u64>(ctw);
+    if (!tmp || !carve_keyswitch(c, ar, kb)) return fail(c, HANN_EWORKSPACE, "hann_fold: workspace too small");
+    u64* cur = (u64*)ct_dev;
+    u64* nxt = tmp;
+    for (int t = 0; t < steps; t++) {
+        const int r = stride << t;
+        // nxt = cur + rot_r(cur): the Horner step of the rotate-and-sum with the ciphertext itself as the addend
+        RET(ks_digits_to_lifted(c, kb.c1c, 1, kb.digits, (int64_t)L * L1N, r, 0, 1, kb.u, kb.lifted, cur + LN, ctw));
+        RET(launch_moddown_combine(c, kb.u, kb.lifted, 1, r, 0, cur, ctw, cur, ctw, nxt, nxt + LN, ctw));
+        std::swap(cur, nxt);
+    }
+    if (cur != (u64*)ct_dev) RET(launch_copy2d(c, (u64*)ct_dev, ctw, cur, ctw, ctw, 1));
+    return HANN_OK;
+}
+
+extern "C" int64_t hann_project_bytes(const hann_ctx* top, const hann_ctx* mid) {
+    if (!top || !mid) return HANN_EINVAL;
+    const int64_t B = top->B, G = mid->G;
+    const int64_t cyc_top = align256(B * hann_sizeof(top, HANN_SIZE_CT)), cyc_mid = align256(B * hann_sizeof(mid, HANN_SIZE_CT));
+    const int64_t inner = align256(G * hann_sizeof(mid, HANN_SIZE_CT)), acc = align256(hann_sizeof(mid, HANN_SIZE_CT));
+    const int64_t sub = std::max<int64_t>(std::max<int64_t>(project_baby_words(top) * 8 + kSlack, hann_workspace_bytes(top, B)),
+                                          hann_workspace_bytes(mid, 1));
+    return cyc_top + cyc_mid + inner + acc + align256(sub) + kSlack;
+}
+
+extern "C" int hann_project_query(hann_ctx* top, hann_ctx* mid, const void* ct_dev, const void* lo_dev, const void* hi_dev,
+                                  const void* wpt_dev, int D, void* out_dev, void* ws, size_t ws_bytes) {
+    if (!top || !mid) return HANN_EINVAL;
+    hann_ctx* c = top;
+    if (!ct_dev || !lo_dev || !hi_dev || !wpt_dev || !out_dev) return fail(c, HANN_EINVAL, "hann_project_query: null pointer");
+    if (mid->L != top->L - 1 || mid->L < 2 || mid->N != top->N || mid->R != top->R || mid->B != top->B || mid->device != top->device ||
+        mid->stream != top->stream)
+        return fail(c, HANN_ESHAPE, "hann_project_query: the second context must be the same ring, R, B, device and stream with one prime less");
+    for (int i = 0; i < mid->L; i++)
+        if (mid->mod[i] != top->mod[i]) return fail(c, HANN_ESHAPE, "hann_project_query: the second context's primes must be the first L-1 of the first's");
+    if (mid->mod[mid->L] != top->mod[top->L]) return fail(c, HANN_ESHAPE, "hann_project_query: the contexts must share the special prime");
+    const int R = top->R;
+    if (D < R || D % R || top->n % D || ((D / R) & (D / R - 1))) return fail(c, HANN_ESHAPE, "hann_project_query: D / R must be a power of two, D must divide n");
+    if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_project_query: workspace missing or not 256-byte aligned");
+    if ((int64_t)ws_bytes < hann_project_bytes(top, mid)) return fail(c, HANN_EWORKSPACE, "hann_project_query: workspace too small");
+    const int64_t B = top->B, G = mid->G;
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
+    u64* cyc_top = ar.take<u64>(B * hann_sizeof(top, HANN_SIZE_CT) / 8);
+    u64* cyc_mid = ar.take<u64>(B * hann_sizeof(mid, HANN_SIZE_CT) / 8);
+    u64* inner = ar.take<u64>(G * hann_sizeof(mid, HANN_SIZE_CT) / 8);
+    u64* acc = ar.take<u64>(hann_sizeof(mid, HANN_SIZE_CT) / 8);
+    if (!cyc_top || !cyc_mid || !inner || !acc) return fail(c, HANN_EWORKSPACE, "hann_project_query: workspace too small");
+    char* sub = (char*)ws + ar.off;
+    const size_t sub_bytes = ws_bytes - (size_t)ar.off;
+    auto relay = [&](int rc) {  // failures of the second context are reported through the first
+        if (rc != HANN_OK && top->err.empty()) top->err = mid->err;
+        return rc;
+    };
+    top->err.clear();
+    // baby steps inside the windows (scale Delta * mask scale), first rescale: the baby set of the middle chain
+    RET(hann_project_baby(top, ct_dev, lo_dev, hi_dev, cyc_top, sub, sub_bytes));
+    RET(hann_rescale(top, cyc_top, B, cyc_mid, sub, sub_bytes));
+    // packed matrix x in-window rotations, giant steps, the single fold over the windows, second rescale
+    RET(relay(hann_score_level(mid, cyc_mid, wpt_dev, 1, inner, sub, sub_bytes)));
+    RET(relay(hann_rotate_sum(mid, inner, 1, acc, sub, sub_bytes)));
+    int steps = 0;
+    while ((R << steps) < D) steps++;
+    RET(relay(hann_fold(mid, acc, R, steps, sub, sub_bytes)));
+    RET(relay(hann_rescale(mid, acc, 1, out_dev, sub, sub_bytes)));
     return HANN_OK;
 }
 

@@ -114,7 +114,7 @@ __global__ void __launch_bounds__(kThreads) k_fft_b(EncArgs A, LimbTable lt) {
     }
 }
 
-int run_encode(hann_ctx* c, EncArgs& A, int P) {
+int run_encode(hann_ctx* c, EncArgs& A, int P, int log_scale = -1) {
     const int n = c->n;
     A.T = c->fft_T;
     A.U = c->fft_U;
@@ -124,7 +124,7 @@ int run_encode(hann_ctx* c, EncArgs& A, int P) {
     const int S1 = 1 << A.b1, chunks = n >> A.b1;
     A.K1 = chunks < 8 ? chunks : 8;
     A.C1 = S1 < 16 ? S1 : 16;
-    A.scale = ldexp(1.0, c->prm.log_scale - A.logn);
+    A.scale = ldexp(1.0, (log_scale < 0 ? c->prm.log_scale : log_scale) - A.logn);
     A.L = c->L;
     A.R = c->R;
     A.B = c->B;
@@ -168,14 +168,14 @@ int launch_encode_rows(hann_ctx* c, const float* rows, int64_t rows_in_block, in
     return run_encode(c, A, count);
 }
 
-// one slot vector z[n] (device) -> one polynomial [L][N], coefficient domain
-int launch_encode_slots(hann_ctx* c, const double* z_dev, u64* poly_out, void* ws) {
+// one slot vector z[n] (device) -> one polynomial [L][N], coefficient domain, at scale 2^log_scale (negative: the context's)
+int launch_encode_slots(hann_ctx* c, const double* z_dev, u64* poly_out, void* ws, int log_scale) {
     EncArgs A = {};
     A.rows = nullptr;
     A.z = z_dev;
     A.buf = (double2*)ws;
     A.out = poly_out;
-    return run_encode(c, A, 1);
+    return run_encode(c, A, 1, log_scale);
 }
 
 // =====================================================================================================================

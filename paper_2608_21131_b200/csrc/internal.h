@@ -163,7 +163,11 @@ LimbMap limbmap_single(int limb);
 // encode (coefficient-domain residues out; the caller transforms)
 int launch_encode_rows(hann_ctx* c, const float* rows, int64_t rows_in_block, int dim, int p_first, int count, u64* pt_block,
                        void* ws);
-int launch_encode_slots(hann_ctx* c, const double* z_dev, u64* poly_out, void* ws);
+int launch_encode_slots(hann_ctx* c, const double* z_dev, u64* poly_out, void* ws, int log_scale = -1);
+// packed projection (project.cu): slot vectors of a packed matrix diagonal and of the window masks; the mask combine
+int launch_packed_diagonal(hann_ctx* c, const float* W, int D, int g, int b, double* z);
+int launch_window_masks(hann_ctx* c, int b, double* lo, double* hi);
+int launch_mask_combine(hann_ctx* c, const u64* ct, const u64* rot_a, const u64* rot_h, const u64* lo, const u64* hi, u64* cyc);
 int64_t encode_ws_bytes(const hann_ctx* c);
 int64_t encode_fft_bytes(const hann_ctx* c);
 int encode_stage_group(const hann_ctx* c);

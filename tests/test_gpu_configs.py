@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 
 from paper_2608_21131_b200 import synth, workloads as wl
-from tests.helpers import Pair, rescale_error_bound
+from tests.helpers import Pair, make_oracle, rescale_error_bound
 
 pytestmark = pytest.mark.gpu
 
@@ -262,6 +262,89 @@ def test_projection_under_encryption_then_scoring():
     got = g2.decrypt_scores(pc.km.s, score_g, log_scale_out=120).reshape(-1)[: rows.shape[0]]
     want = rows.astype(np.float64) @ qR
     assert np.abs(got - want).max() < 2.0 ** -18
+
+
+@pytest.mark.parametrize("logN,D,R,B,B_score,lazy", [(13, 512, 128, 4, 32, False), (12, 128, 32, 8, 8, True), (16, 512, 128, 8, 32, False)])
+def test_packed_projection_then_scoring(logN, D, R, B, B_score, lazy):
+    """Rank reduction with the matrix packed by windows (Sec. 3.1 Detail): masks, packed diagonals, the in-window baby
+    rotations after their rescale and the projected query are each compared with the oracle bit for bit; the projected
+    query (two primes fewer, scale back at ~2^40) then serves an ordinary scoring level on the shorter chain, again bit
+    for bit, with scores inside 2^-18 of the float64 products.  512 -> 128 at N = 2^13 and at N = 2^16."""
+    import torch
+
+    from oracle.oracle import PackedProjection, restrict_keys
+    from paper_2608_21131_b200 import binding as b
+
+    q, p, L = synth.Q50, synth.P60, 4
+    pp = PackedProjection(logN, q, p, 40, D, R, B, 50, 50)
+    n, N = pp.n, pp.N
+    ps_top = synth.ParamSet("top", logN, q, p, 40, R, B, -18)
+    top, mid = b.Context(ps_top), b.Context(ps_top.with_(q=q[:3]))
+    ps_low = ps_top.with_(q=q[:2], B=B_score)
+    low = b.Context(ps_low)
+    giant = [g * B for g in range(1, pp.G)] if lazy else [B]
+    rots_top = pp.baby_rotations()
+    rots_mid = sorted(set(giant) | set(pp.fold_rotations()))
+    rots_low = list(range(1, B_score + 1))
+    rots = sorted(set(rots_top) | set(rots_mid) | set(rots_low))
+    km = synth.key_material(ps_top, 61, rots=rots)
+    evk = top.keygen_from_samples(km.s, km.rots, km.evk_a, km.evk_e)       # the client's keys, longest chain
+    evk_o = dict(zip(rots, helpers_keys(pp.top, km)))
+    assert np.array_equal(evk, np.stack([evk_o[r] for r in rots]))
+    pick = lambda want: np.stack([evk[rots.index(r)] for r in want])
+    top.load_keys(pick(rots_top), rots_top)
+    mid.load_keys(b.restrict_keys(pick(rots_mid), L, 3), rots_mid)
+    low.load_keys(b.restrict_keys(pick(rots_low), L, 2), rots_low)
+    assert np.array_equal(b.restrict_keys(pick(rots_mid), L, 3), restrict_keys(pick(rots_mid), L, 3))
+    if lazy:
+        mid.set_tuning(b.TUNE_GIANT_LAZY, 1)
+    rng = np.random.default_rng(5)
+    W = np.linalg.qr(rng.standard_normal((D, R)))[0].astype(np.float32)
+    qv = rng.standard_normal(D)
+    qv = (qv / np.linalg.norm(qv)).astype(np.float32)
+    # enrolment: masks on the top chain, packed matrix on the middle chain
+    ws_top, ws_mid = top.workspace(1), mid.workspace(1)
+    lo, hi = top.project_masks(50, ws_top)
+    wpt = mid.project_enrol(torch.from_numpy(W).to(mid.device), 50, ws_mid)
+    lo_o, hi_o = pp.mask_plaintexts()
+    assert np.array_equal(top.export(b.KIND_PT, lo, B).reshape(B, L, N), lo_o)
+    assert np.array_equal(top.export(b.KIND_PT, hi, B).reshape(B, L, N), hi_o)
+    wpt_o = pp.enrol(W.astype(np.float64))
+    assert np.array_equal(mid.export(b.KIND_PT, wpt, R).reshape(pp.G, B, 3, N), wpt_o)
+    # the query: q tiled with period D (a "dimension D" query of a context whose R is D would do the same)
+    ct = pp.top.encrypt(km.s, pp.top.encode(pp.query_slots(qv)), km.ct_a, km.ct_e)
+    ct_dev = top.import_(b.KIND_CT, ct, 1)
+    wsp = top.alloc(top.lib.hann_project_bytes(top.h, mid.h))
+    cyc = top.rescale(top.project_baby(ct_dev, lo, hi, wsp), B, wsp)
+    top.sync()
+    cyc_o = pp.in_window_rotations(ct, evk_o)
+    assert np.array_equal(top.export_limbs(cyc, 2 * B, 3).reshape(B, 2, 3, N), cyc_o)
+    out = top.project_query(mid, ct_dev, lo, hi, wpt, D, wsp)
+    top.sync()
+    out_o = pp.project(ct, evk_o, wpt_o, lazy=lazy)
+    assert np.array_equal(mid.export_limbs(out, 2, 2).reshape(2, 2, N), out_o)
+    want_q = W.T.astype(np.float64) @ qv.astype(np.float64)
+    slots = pp.low.decode(np.array([float(v) for v in pp.low.decrypt_int(km.s, out_o)]), pp.scale_out).real
+    assert np.abs(slots - np.tile(want_q, n // R)).max() < 2.0 ** -20
+    # an ordinary level on the shortest chain with the projected ciphertext as its query
+    rows = synth.project_rows(synth.toy_corpus(7, rows=n + 300, dim=D).astype(np.float64), W.astype(np.float64), R)
+    ws_low = low.workspace(2)
+    baby = low.query_prepare(out, ws_low)
+    score = low.rotate_sum(low.score_level(baby, low.encode_candidates(torch.from_numpy(rows).to(low.device), ws_low), 2, ws_low), 2, ws_low)
+    low.sync()
+    score_g = low.export(b.KIND_CT, score, 2)
+    o_low = make_oracle(ps_low)
+    evk_low = restrict_keys(np.stack([evk_o[r] for r in rots_low]), L, 2)
+    baby_o = o_low.baby_set(out_o, evk_low)
+    for blk in range(2):
+        sc_o, _, _ = o_low.score_block(rows[blk * n:(blk + 1) * n], baby_o, evk_low[B_score - 1])
+        assert np.array_equal(score_g[blk], sc_o), blk
+    got = low.decrypt_scores(km.s, score_g, log_scale_out=80).reshape(-1)[: rows.shape[0]] * (2.0 ** 40 / pp.scale_out)
+    assert np.abs(got - rows.astype(np.float64) @ want_q).max() < 2.0 ** -18
+
+
+def helpers_keys(o, km):
+    return [o.evk_gen(km.s, r, km.evk_a[i], km.evk_e[i]) for i, r in enumerate(km.rots)]
 
 
 def test_projection_with_encrypted_matrix():

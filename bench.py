@@ -649,6 +649,82 @@ def run_encrypted_db(args):
     return 0 if err < 2.0 ** ps.tol_log2 else 1
 
 
+def run_project(args):
+    """Rank reduction under encryption (Sec. 3.1: Enc(q_R) = W^T Enc(q), matrix packed by windows): device time of one
+    projection of a 512-dimensional encrypted query, for every baby-step count of the sweep and both evaluation orders of the
+    giant steps (the paper's projection-latency figure: the optimum sits below sqrt(R) because a baby step costs two slot
+    rotations here and a giant step one).  N = 2^16, 4 x 50-bit primes, masks and matrix at scale 2^50.  One JSON line."""
+    import torch
+    from paper_2608_21131_b200 import binding, synth, workloads as wl
+
+    torch.cuda.set_device(0)
+    D, R, L, logN = 512, args.project_rank, 4, 16
+    q, p = synth.Q50, synth.P60
+    rng = np.random.default_rng(wl.PROJ_SEED)
+    W = np.linalg.qr(rng.standard_normal((D, R)))[0].astype(np.float32)
+    qv = synth.normalise(synth.gaussian_vectors(wl.query_seed(0), synth.S_QUERY, np.arange(1), D))[0].astype(np.float32)
+    want = W.T.astype(np.float64) @ qv.astype(np.float64)
+    sweep = []
+    for B in [int(x) for x in args.project_sweep.split(",")]:
+        if R % B:
+            continue
+        G = R // B
+        ps = synth.ParamSet("proj", logN, q, p, 40, R, B, -18)
+        top, mid = binding.Context(ps), binding.Context(ps.with_(q=q[:3]))
+        n = top.n
+        rots_top = list(range(1, B)) + [n - R + b for b in range(1, B)]
+        fold = [R << t for t in range((D // R).bit_length() - 1)]
+        rots_mid = sorted(set(g * B for g in range(1, G)) | set(fold))
+        rots = sorted(set(rots_top) | set(rots_mid))
+        km = synth.key_material(ps, wl.KEY_SEED, rots=rots)
+        evk = top.keygen_from_samples(km.s, km.rots, km.evk_a, km.evk_e)
+        pick = lambda wanted: np.stack([evk[rots.index(r)] for r in wanted])
+        if rots_top:
+            top.load_keys(pick(rots_top), rots_top)
+        mid.load_keys(binding.restrict_keys(pick(rots_mid), L, 3), rots_mid)
+        del evk
+        lo, hi = top.project_masks(50, top.workspace(1))
+        wpt = mid.project_enrol(torch.from_numpy(W).to(mid.device), 50, mid.workspace(1))
+        # the query: q tiled with period D = one "candidate-free" encryption of a D-dimensional vector
+        qctx = binding.Context(ps.with_(R=D, B=1))
+        ct_dev = top.import_(binding.KIND_CT, qctx.encrypt_query(km.s, qv, km.ct_a, km.ct_e), 1)
+        del qctx
+        wsp = top.alloc(top.lib.hann_project_bytes(top.h, mid.h))
+        rec = {"B": B, "G": G, "slot_rotations": {"baby": 2 * (B - 1), "giant": G - 1, "fold": len(fold)}}
+        for order in ("horner", "lazy"):
+            mid.set_tuning(binding.TUNE_GIANT_LAZY, 1 if order == "lazy" else 0)
+            for _ in range(3):
+                out = top.project_query(mid, ct_dev, lo, hi, wpt, D, wsp)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(args.steps):
+                out = top.project_query(mid, ct_dev, lo, hi, wpt, D, wsp)
+            e1.record()
+            torch.cuda.synchronize()
+            rec["ms_" + order] = e0.elapsed_time(e1) / args.steps
+            # what came out: decrypt on the two-prime chain at the exact scale Delta 2^50/q_3 2^50/q_2
+            lowctx = binding.Context(ps.with_(q=q[:2]))
+            can = mid.export_limbs(out, 2, 2).reshape(1, 2, 2, top.N)
+            slots = lowctx.decrypt_scores(km.s, can, log_scale_out=40)[0] * (2.0 ** 40 / (2.0 ** 40 * (2.0 ** 50 / q[3]) * (2.0 ** 50 / q[2])))
+            rec["max_abs_error_" + order] = float(np.abs(slots - np.tile(want, n // R)).max())
+            del lowctx
+        sweep.append(rec)
+        del top, mid, lo, hi, wpt, wsp, ct_dev
+        torch.cuda.empty_cache()
+    best = min(sweep, key=lambda r: min(r["ms_horner"], r["ms_lazy"]))
+    ok = all(max(r["max_abs_error_horner"], r["max_abs_error_lazy"]) < 2.0 ** -20 for r in sweep)
+    print(json.dumps({
+        "metric": "encrypted projections/sec", "value": 1e3 / min(best["ms_horner"], best["ms_lazy"]), "unit": "projections/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": 3, "ms_per_step": min(best["ms_horner"], best["ms_lazy"]), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+        "config": {"workload": "packed projection %d -> %d of one encrypted query, N=2^16, 4x50b primes, masks and matrix at 2^50" % (D, R),
+                   "sqrt_R": R ** 0.5, "best_B": best["B"]},
+        "sweep": sweep, "check": {"tolerance": 2.0 ** -20, "ok": ok},
+    }))
+    return 0 if ok else 1
+
+
 def oracle_setup(ps, qR, km):
     from oracle.oracle import Oracle
 
@@ -841,6 +917,9 @@ def main():
                     "hierarchies (latency per level), 4 scaling sweep point (--rows = wanted rows, --logn 15|16)")
     ap.add_argument("--logn", type=int, default=16, help="ring of the sweep configuration")
     ap.add_argument("--min-timed-s", type=float, default=2.0, help="the K-step block is repeated until the timed region lasted this long")
+    ap.add_argument("--project", action="store_true", help="packed projection 512 -> R of one encrypted query: baby-step sweep")
+    ap.add_argument("--project-rank", type=int, default=128, help="R of --project (128 or 256)")
+    ap.add_argument("--project-sweep", default="1,2,4,8,16,32", help="baby-step counts of --project")
     ap.add_argument("--giant", default="horner", choices=["horner", "lazy"], help="evaluation order of the giant steps of the rotate-and-sum")
     ap.add_argument("--baby", type=int, default=None, help="baby-step count B (default: the configuration's; must divide R)")
     ap.add_argument("--rows", type=int, default=None, help="override the row count (debugging, ncu captures)")
@@ -860,6 +939,9 @@ def main():
         args.steps = 2 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup
         return run_reference(args)
+    if args.project:
+        args.steps = 10 if args.steps is None else args.steps
+        return run_project(args)
     if args.config in (2, 3):
         args.steps = (16 if args.config == 2 else 64) if args.steps is None else args.steps
         args.warmup = 2 if args.warmup is None else args.warmup

@@ -42,7 +42,7 @@ typedef uint64_t u64;
 typedef int64_t i64;
 typedef unsigned __int128 u128;
 
-#define ORC_MAX_LIMBS 9 /* up to 8 ciphertext primes + the special prime */
+#define ORC_MAX_LIMBS 17 /* up to 16 ciphertext primes + the special prime */
 
 typedef struct {
     int logN, N, n;      /* ring degree N = 2^logN, n = N/2 slots */

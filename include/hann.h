@@ -119,7 +119,7 @@ const char *hann_last_error(const hann_ctx *ctx);
 
 /* ---- test, profiling and measurement hooks (not part of the scoring product; nothing on the hot path calls them) ----
  * hann_selftest_bounded_wait, hann_set_timing / hann_get_stats, hann_kernel_profile / hann_kernel_times,
- * hann_probe_rates, hann_debug_check.  (The Python binding's HANN_LIB environment variable, which makes it load
+ * hann_probe_rates, hann_debug_build / hann_debug_canaries / hann_debug_verify.  (The Python binding's HANN_LIB environment variable, which makes it load
  * another build of this library for A/B comparisons, is a hook of the same kind.) */
 
 /* Self-test of the failure path of the bulk-copy kernels: launches one warp that waits, for limit_ms (1..1000), on a
@@ -157,6 +157,21 @@ int hann_kernel_classes(void);
 const char *hann_kernel_name(int cls);
 int hann_kernel_profile(hann_ctx *ctx, int enable);
 int hann_kernel_times(hann_ctx *ctx, double *ms, uint64_t *launches);
+
+/* Checks that stand in for a memory checker (never a trap, never an abort):
+ *   - hann_debug_build() is 1 for a library compiled with -DHANN_DEBUG.  Such a build checks the computed indices of its
+ *     gathers (automorphism sources, mirror positions, row gathers) against their ranges; a failing check SKIPS the access
+ *     and records the source line in the context's error word, which the next synchronising call reports as HANN_ECUDA
+ *     ("index range check failed ... source line N").  A release build has no such code.
+ *   - hann_debug_canaries(ctx, 1) (any build) makes every server-side call put a 256-byte guard behind each sub-buffer it
+ *     carves from the caller's workspace (the slack in hann_workspace_bytes covers them), filled with a pattern on the
+ *     spot; hann_debug_verify(ctx, &checked, &damaged) checks all guards carved since the last verify, reports how many
+ *     there were and how many a kernel overwrote (HANN_ECUDA if any, naming the first one), and forgets them.  Call it
+ *     while the workspaces of those calls are still allocated.  A later call that carves the same workspace retires the
+ *     guards its own sub-buffers cover (they are overwritten legitimately), so verify after the call you want checked. */
+int hann_debug_build(void);
+int hann_debug_canaries(hann_ctx *ctx, int enable);
+int hann_debug_verify(hann_ctx *ctx, int64_t *guards_checked, int64_t *guards_damaged);
 
 /* Measured arithmetic ceilings of the device (a set-up class call: allocates and frees a small buffer, synchronises):
  * binary64 modular butterflies per second of the register-resident round the transform kernels run (no memory traffic:

@@ -78,6 +78,9 @@ def load_library():
         "hann_keygen_from_samples": (C.c_int, [vp, vp, C.c_int, vp, vp, vp, vp]),
         "hann_keygen_seeded": (C.c_int, [vp, C.c_uint64, C.c_int, vp, vp, vp]),
         "hann_probe_rates": (C.c_int, [vp, vp, vp]),
+        "hann_debug_build": (C.c_int, []),
+        "hann_debug_canaries": (C.c_int, [vp, C.c_int]),
+        "hann_debug_verify": (C.c_int, [vp, vp, vp]),
         "hann_encrypt_query": (C.c_int, [vp, vp, vp, C.c_int, vp, vp, vp]),
         "hann_decrypt_scores": (C.c_int, [vp, vp, vp, i64, C.c_int, vp, vp]),
         "hann_load_keys": (C.c_int, [vp, vp, C.c_int, vp]),
@@ -257,6 +260,15 @@ class Context:
         """(binary64 modular butterflies/s, int32 multiply-adds/s) measured on the context's device"""
         a, b = C.c_double(0.0), C.c_double(0.0)
         self._ck(self.lib.hann_probe_rates(self.h, C.byref(a), C.byref(b)))
+        return a.value, b.value
+
+    def debug_canaries(self, on):
+        self._ck(self.lib.hann_debug_canaries(self.h, 1 if on else 0))
+
+    def debug_verify(self):
+        """(guards checked, guards damaged) since the last call; raises if any guard was overwritten"""
+        a, b = C.c_int64(0), C.c_int64(0)
+        self._ck(self.lib.hann_debug_verify(self.h, C.byref(a), C.byref(b)))
         return a.value, b.value
 
     def keygen_relin_from_samples(self, s, a, e):

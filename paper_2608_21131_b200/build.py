@@ -18,6 +18,7 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhann.so")
+DEBUG_LIB = os.path.join(HERE, "libhann_debug.so")  # the -DHANN_DEBUG build (index range checks in the kernels)
 OBJDIR = os.path.join(HERE, "build")
 SOURCES = ["api.cu", "ntt.cu", "keyswitch.cu", "mac.cu", "encode.cu", "static_scratch.cu", "project.cu", "probe.cu", "hostmath.cpp"]
 HEADERS = ["internal.h", "modarith.cuh", "nttcore.cuh", "bulkcopy.cuh", "debugcheck.cuh", os.path.join("..", "..", "include", "hann.h")]
@@ -27,16 +28,20 @@ def _deps():
     return [os.path.join(CSRC, s) for s in SOURCES + HEADERS]
 
 
-def stale() -> bool:
-    if not os.path.exists(LIB):
+def stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     return any(os.path.getmtime(d) > t for d in _deps())
 
 
+def build_debug(force: bool = False) -> str:
+    return build(force=force, out=DEBUG_LIB, extra_flags=("-DHANN_DEBUG",))
+
+
 def build(force: bool = False, verbose: bool = False, out: str = LIB, extra_flags=()) -> str:
-    if not force and out == LIB and not stale():
-        return LIB
+    if not force and out in (LIB, DEBUG_LIB) and not stale(out):
+        return out
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     flags = [
         "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -73,3 +78,5 @@ def build(force: bool = False, verbose: bool = False, out: str = LIB, extra_flag
 
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    if "--debug" in sys.argv:
+        print(build_debug(force="--force" in sys.argv))

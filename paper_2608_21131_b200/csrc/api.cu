@@ -42,23 +42,41 @@ int sync_and_check(hann_ctx* c) {
         c->err = std::string("cudaStreamSynchronize: ") + cudaGetErrorString(e_);
         return HANN_ECUDA;
     }
-    if (*(volatile int*)c->kflag_host) {
+    const int word = *(volatile int*)c->kflag_host;
+    if (word) {
         *(volatile int*)c->kflag_host = 0;
+        if (word & 0x10000) {
+            c->err = "a kernel's index range check failed (debug build), source line " + std::to_string(word & 0xFFFF) +
+                     "; the access was skipped, results of the last calls are invalid";
+            return HANN_ECUDA;
+        }
         return fail(c, HANN_ECUDA, "a kernel gave up a bounded wait for an asynchronous copy; results of the last calls are invalid");
     }
     return HANN_OK;
 }
 
-// bump allocator over a caller-provided workspace
+// bump allocator over a caller-provided workspace.  With a context whose canaries are switched on (hann_debug_canaries) every
+// sub-buffer is followed by a guard of 256 bytes that is filled with a pattern when it is carved and checked by
+// hann_debug_verify: a kernel that writes past the end of its sub-buffer is found without any memory checker.
 struct Arena {
     char* base;
     int64_t off, cap;
+    hann_ctx* dbg = nullptr;
     template <typename T>
     T* take(int64_t count) {
         int64_t bytes = align256(count * (int64_t)sizeof(T));
-        if (off + bytes > cap) return nullptr;
+        const bool guard = dbg && dbg->canaries;
+        if (off + bytes + (guard ? 256 : 0) > cap) return nullptr;
         T* p = (T*)(base + off);
         off += bytes;
+        if (guard) {
+            // guards of earlier calls that lie inside what is carved now are about to be overwritten legitimately: forget them
+            const char *lo = (const char*)p, *hi = base + off + 256;
+            auto& gs = dbg->guards;
+            gs.erase(std::remove_if(gs.begin(), gs.end(), [&](u64* g) { return (const char*)g + 256 > lo && (const char*)g < hi; }), gs.end());
+            if (launch_guard_fill(dbg, (u64*)(base + off)) == HANN_OK) gs.push_back((u64*)(base + off));
+            off += 256;
+        }
         return p;
     }
 };
@@ -363,6 +381,8 @@ extern "C" int hann_ctx_create(const hann_params* prm, hann_ctx** out) {
              cudaEventCreateWithFlags(&c->score_join[i], cudaEventDisableTiming) == cudaSuccess;
     if (ok) ok = cudaEventCreateWithFlags(&c->prep_done, cudaEventDisableTiming) == cudaSuccess;
     if (ok) ok = ntt_configure(c) == HANN_OK;
+    // a -DHANN_DEBUG build: the range checks of the kernels report through this context's error word
+    if (ok) ok = debug_bind_keyswitch(c->kflag) == 0 && debug_bind_project(c->kflag) == 0 && debug_bind_encode(c->kflag) == 0;
     if (ok) {
         // look up the built-in scratch of hann_keyswitch_static now, while this device is current, so that the request-time
         // call only reads a cached address (a failure here is reported by that call, not by context creation)
@@ -474,6 +494,50 @@ extern "C" int hann_selftest_bounded_wait(hann_ctx* c, int limit_ms, double* wai
     CK(cudaMemcpyAsync(&ns, w, 8, cudaMemcpyDeviceToHost, c->stream));
     CK(cudaStreamSynchronize(c->stream));
     if (waited_ms) *waited_ms = (double)ns * 1e-6;
+    return HANN_OK;
+}
+
+extern "C" int hann_debug_build(void) {
+#ifdef HANN_DEBUG
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+extern "C" int hann_debug_canaries(hann_ctx* c, int enable) {
+    if (!c) return HANN_EINVAL;
+    c->canaries = enable ? 1 : 0;
+    c->guards.clear();
+    return HANN_OK;
+}
+
+extern "C" int hann_debug_verify(hann_ctx* c, int64_t* guards_checked, int64_t* guards_damaged) {
+    if (!c) return HANN_EINVAL;
+    if (!guards_checked || !guards_damaged) return fail(c, HANN_EINVAL, "hann_debug_verify: null pointer");
+    DeviceGuard dg(c->device);
+    const int64_t ng = (int64_t)c->guards.size();
+    *guards_checked = ng;
+    *guards_damaged = 0;
+    if (ng == 0) return sync_and_check(c);
+    // guard addresses and the damage counter go through the exchange scratch (this is a debugging call: it may allocate)
+    RET(ensure_scratch(c, align256(ng * 8) + 256));
+    u64** list = (u64**)c->scratch;
+    unsigned long long* bad = (unsigned long long*)((char*)c->scratch + align256(ng * 8));
+    CK(cudaMemcpyAsync(list, c->guards.data(), (size_t)ng * 8, cudaMemcpyHostToDevice, c->stream));
+    const unsigned long long init[2] = {0ULL, ~0ULL};   // damaged guards, index of the first one
+    CK(cudaMemcpyAsync(bad, init, 16, cudaMemcpyHostToDevice, c->stream));
+    RET(launch_guard_verify(c, list, ng, bad));
+    unsigned long long res[2] = {0, 0};
+    CK(cudaMemcpyAsync(res, bad, 16, cudaMemcpyDeviceToHost, c->stream));
+    RET(sync_and_check(c));
+    *guards_damaged = (int64_t)res[0];
+    c->guards.clear();
+    if (res[0]) {
+        c->err = "hann_debug_verify: a kernel wrote past the end of a workspace sub-buffer (" + std::to_string(res[0]) + " of " +
+                 std::to_string(ng) + " guards damaged, the first one is guard " + std::to_string(res[1]) + " in carving order)";
+        return HANN_ECUDA;
+    }
     return HANN_OK;
 }
 
@@ -673,7 +737,7 @@ extern "C" int hann_compact_scores(hann_ctx* c, const void* score_ct_dev, int64_
     int64_t ch = ((int64_t)ws_bytes - kSlack) / per;
     if (ch < 1) return fail(c, HANN_EWORKSPACE, "hann_compact_scores: workspace too small");
     ch = std::min(ch, npoly);
-    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes, c};
     u64* t = ar.take<u64>(ch * N);
     u64* lifted = ar.take<u64>(ch * keep * N);
     if (!t || !lifted) return fail(c, HANN_EWORKSPACE, "hann_compact_scores: workspace too small");
@@ -980,7 +1044,7 @@ static int rotate_hoisted(hann_ctx* c, const char* who, const u64* ct, int rot0,
     for (int r = rot0; r < rot0 + count; r++)
         if (!c->keytab_host[r]) return fail(c, HANN_ENOKEY, (std::string(who) + ": a rotation key is not loaded").c_str());
     if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, (std::string(who) + ": workspace missing or not 256-byte aligned").c_str());
-    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes, c};
     u64* c1c = ar.take<u64>(LN);
     u64* digits = ar.take<u64>(L * L1N);
     u64* u = ar.take<u64>((int64_t)count * 2 * L1N);
@@ -1100,7 +1164,7 @@ extern "C" int hann_score_level_ctdb(hann_ctx* c, const void* baby_dev, const vo
     if (ch < 1) return fail(c, HANN_EWORKSPACE, "hann_score_level_ctdb: workspace too small");
     const int64_t items = n_blocks * G;
     ch = std::min<int64_t>(std::min<int64_t>(ch, items), 8 * G);
-    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes, c};
     u64* d = ar.take<u64>(ch * 3 * LN);
     u64* c1c = ar.take<u64>(ch * LN);
     u64* digits = ar.take<u64>(ch * L * L1N);
@@ -1144,7 +1208,7 @@ extern "C" int hann_rotate_sum(hann_ctx* c, const void* inner_dev, int64_t n_blo
         int64_t ch = (wsp_bytes - kSlack) / (ks_item_words(c) * 8);
         if (ch < 1) return fail(c, HANN_EWORKSPACE, "hann_rotate_sum: workspace too small");
         ch = std::min<int64_t>(std::min<int64_t>(ch, b_hi - b_lo), 8);
-        Arena ar{wsp, 0, wsp_bytes};
+        Arena ar{wsp, 0, wsp_bytes, c};
         u64* c1c = ar.take<u64>(ch * LN);
         u64* digits = ar.take<u64>(ch * L * L1N);
         u64* u = ar.take<u64>(ch * 2 * L1N);
@@ -1226,7 +1290,7 @@ extern "C" int hann_rotate_sum_lazy(hann_ctx* c, const void* inner_dev, int64_t 
     int64_t ch = ((int64_t)ws_bytes - kSlack) / (lazy_block_words(c) * 8);
     if (ch < 1) return fail(c, HANN_EWORKSPACE, "hann_rotate_sum_lazy: workspace too small");
     ch = std::min<int64_t>(std::min<int64_t>(ch, n_blocks), 16);
-    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes, c};
     const int64_t items_max = ch * (G - 1);
     u64* c1c = ar.take<u64>(items_max * LN);
     u64* digits = ar.take<u64>(items_max * L * L1N);
@@ -1358,7 +1422,7 @@ extern "C" int hann_project_baby(hann_ctx* c, const void* ct_dev, const void* lo
     const int64_t ctw = 2 * (int64_t)c->L * c->N;
     DeviceGuard dg(c->device);
     Timer tm(c, 0);
-    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes, c};
     u64* rot_a = ar.take<u64>(std::max(B - 1, 1) * ctw);
     u64* rot_h = ar.take<u64>(std::max(B - 1, 1) * ctw);
     if (!rot_a || !rot_h) return fail(c, HANN_EWORKSPACE, "hann_project_baby: workspace too small");
@@ -1388,7 +1452,7 @@ extern "C" int hann_fold(hann_ctx* c, void* ct_dev, int stride, int steps, void*
     const int64_t LN = (int64_t)L * N, L1N = (int64_t)(L + 1) * N, ctw = 2 * LN;
     DeviceGuard dg(c->device);
     Timer tm(c, 3);
-    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes, c};
     KsBuffers kb;
     u64* tmp = ar.take<u64>(ctw);
     if (!tmp || !carve_keyswitch(c, ar, kb)) return fail(c, HANN_EWORKSPACE, "hann_fold: workspace too small");
@@ -1431,7 +1495,7 @@ extern "C" int hann_project_query(hann_ctx* top, hann_ctx* mid, const void* ct_d
     if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_project_query: workspace missing or not 256-byte aligned");
     if ((int64_t)ws_bytes < hann_project_bytes(top, mid)) return fail(c, HANN_EWORKSPACE, "hann_project_query: workspace too small");
     const int64_t B = top->B, G = mid->G;
-    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes, c};
     u64* cyc_top = ar.take<u64>(B * hann_sizeof(top, HANN_SIZE_CT) / 8);
     u64* cyc_mid = ar.take<u64>(B * hann_sizeof(mid, HANN_SIZE_CT) / 8);
     u64* inner = ar.take<u64>(G * hann_sizeof(mid, HANN_SIZE_CT) / 8);
@@ -1466,7 +1530,7 @@ extern "C" int hann_keyswitch(hann_ctx* c, int rot, const void* poly_dev, void* 
     const int L = c->L;
     DeviceGuard dg(c->device);
     Timer tm(c, 4);
-    Arena ar{(char*)ws, 0, (int64_t)ws_bytes};
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes, c};
     KsBuffers kb;
     if (!carve_keyswitch(c, ar, kb)) return fail(c, HANN_EWORKSPACE, "hann_keyswitch: workspace too small");
     u64 *c1c = kb.c1c, *digits = kb.digits, *u = kb.u, *lifted = kb.lifted;

@@ -11,6 +11,7 @@
 // z_j -> position brev(u_j) is folded into its loads); pass 2 runs the remaining stages on column tiles of the
 // (n/S1) x S1 matrix view, then twists, rounds, reduces modulo every ciphertext prime and writes residues.
 #include "internal.h"
+#include "debugcheck.cuh"
 
 namespace {
 
@@ -48,6 +49,7 @@ __global__ void __launch_bounds__(kThreads) k_fft_a(EncArgs A) {
     for (int idx = threadIdx.x; idx < K1 * S1; idx += kThreads) {
         const int pos = pos0 + idx;
         const int j = A.jinv[pos];
+        if (!HANN_CHECK_INDEX(j, n)) continue;
         double v;
         if (A.rows) {
             int row = j - g * A.B;
@@ -580,3 +582,5 @@ int launch_encode_rows_fused(hann_ctx* c, const float* rows, int64_t rows_in_blo
     }
     return check_launch(c, "encode_fused");
 }
+
+HANN_DEBUG_DEFINE_BIND(debug_bind_encode)

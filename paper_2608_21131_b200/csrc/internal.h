@@ -76,6 +76,9 @@ struct hann_ctx {
     // ModDown lifts of a single item; hann_rotate_sum raises it to 320 for levels of one or two blocks, whose launches
     // otherwise leave most of the machine idle
     int lift_split_ctas = 160;
+    // debugging aid: guards behind every workspace sub-buffer (see Arena in api.cu), filled when carved, checked on request
+    int canaries = 0;
+    std::vector<u64*> guards;
     int giant_lazy = 0;  // hann_rotate_sum (and the calls built on it) evaluates the giant steps in the lazy order
     int encode_sym = 1;  // encode_candidates computes half of every transform and mirrors it (real slot vectors)
     // statistics
@@ -134,6 +137,13 @@ void seeded_gaussian(u64 seed, u64 stream, u64 ctr0, long count, double sigma, i
 // bytes of workspace one hann_keyswitch carves (api.cu); device address of the built-in scratch (static_scratch.cu)
 int64_t keyswitch_ws_bytes(const hann_ctx* c);
 int static_scratch_resolve(hann_ctx* c, void** out);
+
+int launch_guard_fill(hann_ctx* c, u64* guard);                                             // 32 words of pattern
+int launch_guard_verify(hann_ctx* c, u64* const* guards, int64_t count, unsigned long long* damaged);  // counts damaged guards
+// debug build: point each translation unit's range-check word at the context's error word (no-ops in a release build)
+int debug_bind_keyswitch(int* word);
+int debug_bind_project(int* word);
+int debug_bind_encode(int* word);
 
 // ---- launchers: each enqueues on ctx->stream, counts its launches and returns HANN_OK or HANN_ECUDA
 int check_launch(hann_ctx* c, const char* what);

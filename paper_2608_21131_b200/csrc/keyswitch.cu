@@ -3,6 +3,7 @@
 // compaction, and the small helpers of the client half.  All polynomials are [.][limb][N] arrays of 64-bit residues in
 // [0, q).
 #include "internal.h"
+#include "debugcheck.cuh"
 
 namespace {
 
@@ -220,6 +221,7 @@ __global__ void __launch_bounds__(kThreads) k_moddown_combine(
         const long long item = idx / (2 * LN);
         const unsigned k = galois[rot0 + (int)item * rot_inc];
         const int s = (k == 1u) ? t : galois_src(t, k, logN, tau);
+        if (!HANN_CHECK_INDEX(s, N)) continue;
         const LimbConst& lc = lt.c[i];
         u64 a = u[(item * 2 + comp) * L1N + (long long)i * N + s];
         u64 b = lifted[((item * 2 + comp) * L + i) * N + s];
@@ -250,6 +252,10 @@ __global__ void __launch_bounds__(256) k_moddown_combine_chunk(
     const int t = (chunk << 8) + threadIdx.x;
     const int s = (k == 1u) ? t : galois_src(t, k, logN, tau);
     const int src_chunk = ((k == 1u) ? (chunk << 8) : galois_src(chunk << 8, k, logN, tau)) & ~255;
+    // the source chunk must lie inside the polynomial (uniform over the CTA, so leaving here cannot split it at the
+    // barrier); that the source of every t lies in that chunk is checked per thread below, where only the store is skipped
+    if (!HANN_CHECK_INDEX(src_chunk + 255, N)) return;
+    const bool in_chunk = HANN_CHECK_INDEX((s & ~255) - src_chunk, 1);
     const LimbConst lc = lt[i];
 #pragma unroll
     for (int comp = 0; comp < 2; comp++) {
@@ -265,7 +271,7 @@ __global__ void __launch_bounds__(256) k_moddown_combine_chunk(
         if (comp == 0 && c0) v = addmod(v, sc[ls], lc.q);
         if (addend) v = addmod(v, addend[item * addend_stride + (long long)comp * LN + (long long)i * N + t], lc.q);
         u64* o = (comp == 0 ? out0 : out1) + item * out_stride + (long long)i * N + t;
-        *o = v;
+        if (in_chunk) *o = v;
     }
 }
 
@@ -286,6 +292,7 @@ __global__ void __launch_bounds__(kThreads) k_giant_sum_p(const u64* __restrict_
         u64 acc = 0;
         for (int g = 1; g < G; g++) {
             const int s = galois_src(t, galois[g * B], logN, tau);
+            if (!HANN_CHECK_INDEX(s, N)) continue;
             acc = addmod(acc, u[((((long long)(g - 1) * nblk + blk) * 2 + comp) * L1N) + (long long)L * N + s], p);
         }
         up[idx] = acc;
@@ -328,6 +335,7 @@ __global__ void __launch_bounds__(kThreads) k_giant_combine(const u64* __restric
         u64 a0 = 0, a1 = 0, c0 = inner[(blk * G) * ctw + (long long)i * N + t];
         for (int g = 1; g < G; g++) {
             const int s = galois_src(t, galois[g * B], logN, tau);
+            if (!HANN_CHECK_INDEX(s, N)) continue;
             const u64* ug = u + (((long long)(g - 1) * nblk + blk) * 2) * L1N + (long long)i * N + s;
             a0 = addmod(a0, ug[0], lc.q);
             a1 = addmod(a1, ug[L1N], lc.q);
@@ -348,7 +356,9 @@ __global__ void __launch_bounds__(kThreads) k_permute(const u64* __restrict__ sr
     for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
         const long long poly = idx / N;
         const int t = (int)(idx % N);
-        dst[idx] = src[poly * N + galois_src(t, k, logN, tau)];
+        const int sidx = galois_src(t, k, logN, tau);
+        if (!HANN_CHECK_INDEX(sidx, N)) continue;
+        dst[idx] = src[poly * N + sidx];
     }
 }
 
@@ -484,6 +494,21 @@ __global__ void __launch_bounds__(kThreads) k_encrypt_finish(const u64* __restri
 
 }  // namespace
 
+// ---- workspace guards (debugging aid): 32 words behind a sub-buffer hold a pattern derived from their own address
+__global__ void k_guard_fill(u64* guard) { guard[threadIdx.x] = 0xC0DEC0DEC0DEC0DEULL ^ (u64)(uintptr_t)(guard + threadIdx.x); }
+__global__ void k_guard_verify(u64* const* guards, long long count, unsigned long long* damaged) {
+    const long long gi = blockIdx.x;
+    if (gi >= count) return;
+    const u64* g = guards[gi];
+    const bool bad = g[threadIdx.x] != (0xC0DEC0DEC0DEC0DEULL ^ (u64)(uintptr_t)(g + threadIdx.x));
+    if (__any_sync(0xffffffffu, bad) && threadIdx.x == 0) {
+        atomicAdd(damaged, 1ULL);
+        atomicMin(damaged + 1, (unsigned long long)gi);   // the first damaged guard, in the order they were carved
+    }
+}
+
+HANN_DEBUG_DEFINE_BIND(debug_bind_keyswitch)
+
 int check_launch(hann_ctx* c, const char* what) {
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
@@ -491,6 +516,16 @@ int check_launch(hann_ctx* c, const char* what) {
         return HANN_ECUDA;
     }
     return HANN_OK;
+}
+
+int launch_guard_fill(hann_ctx* c, u64* guard) {
+    k_guard_fill<<<1, 32, 0, c->stream>>>(guard);
+    return check_launch(c, "guard_fill");
+}
+
+int launch_guard_verify(hann_ctx* c, u64* const* guards, int64_t count, unsigned long long* damaged) {
+    k_guard_verify<<<(unsigned)count, 32, 0, c->stream>>>(guards, count, damaged);
+    return check_launch(c, "guard_verify");
 }
 
 int launch_lift_digits(hann_ctx* c, const u64* src, int64_t src_stride, int64_t nitems, u64* digits) {

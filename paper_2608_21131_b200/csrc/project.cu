@@ -10,6 +10,7 @@
 //              g B + b of every chunk in its own window, shifted inside the window by the giant-step amount;
 //   masks      lo_b[i] = 1 if (i mod R) + b < R else 0, hi_b = 1 - lo_b.
 #include "internal.h"
+#include "debugcheck.cuh"
 
 namespace {
 
@@ -29,7 +30,9 @@ __global__ void __launch_bounds__(kThreads) k_packed_diagonal(const float* __res
         const int w = i % D, k = w / R, j = w % R;
         int col = (j - g * B) % R;
         if (col < 0) col += R;
-        z[i] = (double)W[(long long)(k * R + (j + b) % R) * R + col];
+        const long long widx = (long long)(k * R + (j + b) % R) * R + col;
+        if (!HANN_CHECK_INDEX(widx, (long long)D * R)) continue;
+        z[i] = (double)W[widx];
     }
 }
 
@@ -57,6 +60,7 @@ __global__ void __launch_bounds__(kThreads) k_mask_combine(const u64* __restrict
         const long long b = idx / ctw, rem = idx % ctw;
         const LimbConst& lc = lt.c[l];
         const long long m = (b * L + l) * n + (t < n ? t : N - 1 - t);
+        if (!HANN_CHECK_INDEX(m, (long long)Bn * L * n)) continue;
         const u64 a = b == 0 ? ct[rem] : rot_a[(b - 1) * ctw + rem];
         u64 v = mulmod(a, lo[m], lc);
         if (b > 0) v = addmod(v, mulmod(rot_h[(b - 1) * ctw + rem], hi[m], lc), lc.q);
@@ -90,3 +94,5 @@ int launch_mask_combine(hann_ctx* c, const u64* ct, const u64* rot_a, const u64*
     }
     return check_launch(c, "mask_combine");
 }
+
+HANN_DEBUG_DEFINE_BIND(debug_bind_project)

@@ -13,7 +13,20 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(scope="module")
 def pair16():
-    return Pair(synth.FULL16, key_seed=wl.KEY_SEED)
+    """the production parameter set with the keys of rotations 1..B and, for the lazy order of the giant steps, 2B..(G-1)B
+    (key material of a rotation depends on its place in the list, so the first B keys are those of bench.py's key set too)"""
+    ps = synth.FULL16
+    p = Pair(ps, key_seed=wl.KEY_SEED)
+    rots = list(range(1, ps.B + 1)) + [gg * ps.B for gg in range(2, ps.G)]
+    km = synth.key_material(ps, wl.KEY_SEED, rots=rots)
+    extra = [i for i, r in enumerate(rots) if r > ps.B]
+    p.evk_lazy_o = {ps.B: p.evk_o[ps.B - 1]}
+    for i in extra:
+        p.evk_lazy_o[rots[i]] = p.o.evk_gen(km.s, rots[i], km.evk_a[i], km.evk_e[i])
+    evk_extra = p.g.keygen_from_samples(km.s, [rots[i] for i in extra], km.evk_a[extra], km.evk_e[extra])
+    assert np.array_equal(evk_extra, np.stack([p.evk_lazy_o[rots[i]] for i in extra]))
+    p.g.load_keys(evk_extra, [rots[i] for i in extra])
+    return p
 
 
 class Query:
@@ -31,7 +44,7 @@ class Query:
         self.baby = p.g.query_prepare(self.ct_dev, p.ws)
         self.baby_o = p.o.baby_set(ct_o, p.evk_o) if with_oracle else None
 
-    def score_level(self, rows, oracle_blocks=(), compact=False, one_call=False, host=False):
+    def score_level(self, rows, oracle_blocks=(), compact=False, one_call=False, host=False, lazy_blocks=()):
         """GPU scores of a level [n_rows]; blocks listed in oracle_blocks are compared bit for bit with the oracle"""
         p, g, b, ps = self.p, self.p.g, self.p.b, self.p.ps
         n_rows = rows.shape[0]
@@ -57,6 +70,25 @@ class Query:
             assert np.array_equal(pt_g, pt_o), "encoded plaintexts of block %d" % blk
             assert np.array_equal(in_g, in_o), "partial sums of block %d" % blk
             assert np.array_equal(score_h[blk], sc_o), "score ciphertext of block %d" % blk
+        if lazy_blocks:
+            # the giant steps in the order bench.py's headline uses (distinct keys, one ModDown per block): the same partial
+            # sums through hann_query_level / hann_rotate_sum with the knob set, against the oracle's evaluation in that order
+            giant = np.stack([p.evk_lazy_o[gg * ps.B] for gg in range(1, ps.G)])
+            g.set_tuning(b.TUNE_GIANT_LAZY, 1)
+            lazy = g.rotate_sum(inner, nb, ws)
+            g.sync()
+            lazy_h = g.export(b.KIND_CT, lazy, nb)
+            for blk in lazy_blocks:
+                in_g = g.export(b.KIND_CT, inner, ps.G, offset_bytes=blk * g.sizeof(b.SIZE_INNER)).reshape(ps.G, 2, ps.L, ps.N)
+                assert np.array_equal(lazy_h[blk], p.o.rotate_sum_lazy(in_g, giant)), "lazy score ciphertext of block %d" % blk
+            got_l = g.decrypt_scores(p.km.s, lazy_h).reshape(-1)[:n_rows]
+            assert float(np.abs(got_l - rows.astype(np.float64) @ self.qR.astype(np.float64)).max()) < 2.0 ** ps.tol_log2
+            if host:
+                ws_host = g.alloc(g.level_host_bytes(n_rows))
+                assert np.array_equal(g.score_level_host(self.ct_g, np.ascontiguousarray(rows), ws_host), lazy_h)
+                del ws_host
+            g.set_tuning(b.TUNE_GIANT_LAZY, 0)
+            del lazy
         if host:
             # the end-to-end call bench.py times: host buffers in, block groups scored while later groups upload
             ws_host = g.alloc(g.level_host_bytes(n_rows))
@@ -87,7 +119,7 @@ def test_face_like_level_full(pair16):
     conformance point, every row within 2^-18; the host-buffer call (three block groups) returns the same ciphertexts."""
     ps, lvl, qR, planted = wl.face_level()
     q = Query(pair16, qR)
-    got, want = q.score_level(lvl.rows, oracle_blocks=(0, 6), compact=True, host=True)
+    got, want = q.score_level(lvl.rows, oracle_blocks=(0, 6), compact=True, host=True, lazy_blocks=(0, 6))
     assert got.shape == (222_049,)
     # a quarter of the bytes on the wire (one limb instead of four) still ranks the same neighbours first
     assert np.array_equal(wl.topk_ids(q.compact_scores, lvl.ids, 10), wl.topk_ids(want, lvl.ids, 10))

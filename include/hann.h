@@ -54,7 +54,7 @@ extern "C" {
 #define HANN_ECUDA (-5)      /* a CUDA runtime call or kernel launch failed                 */
 #define HANN_ENOMEM (-6)     /* host or device allocation failed (set-up calls only)        */
 
-#define HANN_MAX_PRIMES 8
+#define HANN_MAX_PRIMES 15
 
 typedef struct hann_ctx hann_ctx; /* opaque */
 
@@ -271,7 +271,7 @@ int hann_score_level_batch(hann_ctx *ctx, const void *baby_dev, int n_queries, c
  * ciphertext sum_b ctdb[blk][g][b] (x) baby[b] = (x0 y0, x0 y1 + x1 y0, x1 y1) accumulated over the baby steps, then ONE
  * relinearisation per (blk, g): (d0 + ks0, d1 + ks1) with (ks0, ks1) the key switch of d2 under the relinearisation key
  * (loaded as rotation 0).  inner_dev as for hann_score_level (n_blocks * HANN_SIZE_INNER bytes); hann_rotate_sum follows
- * unchanged.  Ciphertext primes below 2^56, B <= 128.  ctdb_dev n_blocks * HANN_SIZE_CTDB_BLOCK bytes. */
+ * unchanged.  Ciphertext primes below 2^60, B <= 128.  ctdb_dev n_blocks * HANN_SIZE_CTDB_BLOCK bytes. */
 int hann_score_level_ctdb(hann_ctx *ctx, const void *baby_dev, const void *ctdb_dev, int64_t n_blocks, void *inner_dev,
                           void *ws, size_t ws_bytes);
 
@@ -387,6 +387,37 @@ int hann_fold(hann_ctx *ctx, void *ct_dev, int stride, int steps, void *ws, size
 int64_t hann_project_bytes(const hann_ctx *top, const hann_ctx *mid);
 int hann_project_query(hann_ctx *top, hann_ctx *mid, const void *ct_dev, const void *lo_dev, const void *hi_dev,
                        const void *wpt_dev, int D, void *out_dev, void *ws, size_t ws_bytes);
+
+/* ---- membership (threshold) circuit of the face task (Sec. 3.1 "The norm problem", membership bullet; Sec. 2 "Security
+ * parameters": depth 11) ---------------------------------------------------------------------------------------------
+ * The server returns, per candidate, a ciphertext slot whose SIGN says whether <x, q_R> >= tau |q_R|: the threshold is
+ * scaled into the query's units by r = kappa tau sqrt(|q_R|^2), the root taken by a low-degree Chebyshev polynomial of the
+ * encrypted squared norm, and sign(s - r) is amplified by `sign_iters` iterations of f(x) = x (3 - x^2) / 2 (kappa = 1/2
+ * keeps everything in [-1, 1]).  Depth: 1 (norm) + ceil(log2 deg) (Chebyshev basis by the product identity T_{m+n} =
+ * 2 T_m T_n - T_{m-n}) + 1 (combination) + 2 per sign iteration: 11 at deg = 7, sign_iters = 3, on a chain of 12 primes.
+ *   - Chain: prime i of the chain is consumed by the i-th rescale counted from the END; the primes consumed by the second
+ *     product of a sign iteration must be about TWICE the scale (that rescale is the division by two), all other scaling
+ *     primes about the scale, the first prime large enough for a value of magnitude 1 at that scale.
+ *   - Contexts: arith[l-1], l = 1..L, the first l primes with R = B = 1 (relinearisation key loaded as rotation 0 where a
+ *     product happens, the keys of rotations 1, 2, .., R/2 on arith[L-2] for the fold); `scorer`: the first
+ *     L - depth(threshold) + 1 primes with the rank R and its own B (baby-step keys and the key of rotation B loaded).
+ *     All keys are restrictions of the longest chain's keys.  All contexts on one device and stream.
+ *   - The client sends lam q_R tiled with period R at scale 2^log_scale, lam^2 = a q_{L-1} / 2^log_scale, a = 2 / (t_hi -
+ *     t_lo) ([t_lo, t_hi] must contain |q_R|^2); the candidates are enrolled (hann_encode_candidates on `scorer`) times
+ *     kappa / lam.  coef[0..deg]: Chebyshev coefficients of kappa tau sqrt(t) on [t_lo, t_hi], computed by the caller (they
+ *     decide integer constants of the circuit, so every party must use the same doubles).
+ *   - out_dev [n_blocks][2][1][N] (ciphertexts on the first prime, *out_scale their scale); thr_dev (optional): the
+ *     threshold ciphertext [2][*thr_level][N] at *thr_scale.  ws: hann_membership_bytes. */
+typedef struct {
+    int32_t R, deg, sign_iters, log_scale;
+    double tau, t_lo, t_hi;
+    const double *coef; /* deg + 1 values */
+} hann_membership_params;
+int hann_membership_levels(int deg, int sign_iters, int *chain_primes, int *score_level);
+int64_t hann_membership_bytes(hann_ctx *const *arith, int L, const hann_ctx *scorer, const hann_membership_params *prm, int64_t n_blocks);
+int hann_membership_decide(hann_ctx *const *arith, int L, hann_ctx *scorer, const hann_membership_params *prm, const void *ct_dev,
+                           const void *pt_dev, int64_t n_blocks, void *out_dev, double *out_scale, void *thr_dev, int *thr_level,
+                           double *thr_scale, void *ws, size_t ws_bytes);
 
 /* Convert `count` elements between the canonical layout (host or device pointer) and the internal device layout.
  * kind POLY / PT: one polynomial of L limbs per element; CT: two.  The canonical form of every kind is [L][N] words per

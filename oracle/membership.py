@@ -172,10 +172,11 @@ def chebyshev_basis(mul, sub_, twice, add_const, u, deg):
 class Membership:
     """one parameter set of the membership path: ring, chain, rank R, threshold tau, range of |q_R|^2, polynomial degree"""
 
-    def __init__(self, logN, R, tau, t_lo=0.05, t_hi=1.0, deg=7, sign_iters=3, log_scale=45):
+    def __init__(self, logN, R, tau, t_lo=0.05, t_hi=1.0, deg=7, sign_iters=3, log_scale=45, B=None):
         q, p = membership_chain(logN, deg, sign_iters, log_scale)
         self.ev = Evaluator(logN, q, p, log_scale)
         self.R, self.tau, self.t_lo, self.t_hi, self.deg, self.sign_iters = R, tau, t_lo, t_hi, deg, sign_iters
+        self.B = B if B else max(1, 1 << ((R.bit_length() - 1) // 2))       # baby steps of the scorer
         self.kappa = 0.5
         self.n, self.N, self.L, self.log_scale = self.ev.n, self.ev.N, len(q), log_scale
         self.coef = chebyshev_coefficients(lambda t: self.kappa * tau * np.sqrt(t), deg, t_lo, t_hi)
@@ -203,7 +204,7 @@ class Membership:
         u = (2.0 * t - (self.t_hi + self.t_lo)) / (self.t_hi - self.t_lo)
         T = chebyshev_basis(lambda a, b: a * b, lambda a, b: a - b, lambda a: 2.0 * a, lambda a, c: a + c, u, self.deg)
         r = self.coef[0] + sum(self.coef[k] * T[k] for k in range(1, self.deg + 1))
-        d = self.kappa * (rows.astype(np.float64) @ qR.astype(np.float64)) - r
+        d = self.lam * (self.scaled_rows(rows).astype(np.float64) @ qR.astype(np.float64)) - r
         x = d
         for _ in range(self.sign_iters):
             x = x * (1.5 - 0.5 * x * x)
@@ -217,7 +218,7 @@ class Membership:
         for r in self.fold_rotations():
             t = ev.add(t, ev.rotate(t, r))                       # lam^2 |q_R|^2 in every slot
         # read at scale Delta it is a t (see __init__); the rescale left it at Delta^2 / q_{L-1} = Delta lam^2 / a ... exactly
-        t = Ct(t.res, t.scale / (self.lam ** 2) * self.a)
+        t = Ct(t.res, t.scale / (self.lam * self.lam) * self.a)
         u = ev.add_const(t, -(self.t_hi + self.t_lo) / (self.t_hi - self.t_lo))
         T = chebyshev_basis(ev.mul, ev.sub, lambda x: ev.mul_int(x, 2), ev.add_const, u, self.deg)
         level = min(T[k].level for k in T) - 1
@@ -230,23 +231,27 @@ class Membership:
             acc = term if acc is None else ev.add(acc, term)
         return ev.add_const(acc, float(self.coef[0]))
 
+    def score_rotations(self):
+        """slot rotations the scorer needs: the baby steps and the Horner rotation"""
+        return list(range(1, self.B + 1))
+
+    def scorer(self, level):
+        return Oracle(self.ev.logN, self.ev.q[:level], self.ev.p, self.log_scale, self.R, self.B)
+
+    def scaled_rows(self, rows):
+        """what is enrolled: the candidates times kappa / lam (float32, as every candidate row of the scoring path)"""
+        return (rows.astype(np.float64) * (self.kappa / self.lam)).astype(np.float32)
+
     def scores(self, ct_q, rows, level):
-        """kappa <x_i, q_R> in slot i for up to n rows (unit dimension R tiled query): the diagonal method written out with
-        plain slot rotations (no baby/giant split: the oracle is not about speed), entered at `level` and ending one below"""
+        """kappa <x_i, q_R> in slot i for up to n rows: the ordinary diagonal scorer (baby set, multiply-accumulate, Horner)
+        on the first `level` primes, against candidates enrolled as scaled_rows(); ends one level below"""
         ev = self.ev
         assert rows.shape[0] <= self.n and rows.shape[1] == self.R
-        M = np.zeros((self.n, self.R))
-        M[: rows.shape[0]] = rows
+        o = self.scorer(level)
         q = ev.drop(ct_q, level)
-        i = np.arange(self.n)
-        acc = None
-        for dgl in range(self.R):
-            rot = q if dgl == 0 else ev.rotate(q, dgl)
-            o = ev.o[level]
-            z = (self.kappa / self.lam) * M[i, (i + dgl) % self.R]
-            term = o.mul_plain_acc(rot.res, o.encode_plain(z, self.log_scale))
-            acc = term if acc is None else o.add(acc, term)
-        return ev.rescale(Ct(acc, q.scale * 2.0 ** self.log_scale))
+        keys = np.stack([ev._key(ev.rot_keys[r], level) for r in self.score_rotations()])
+        sc, _, _ = o.score_block(self.scaled_rows(rows), o.baby_set(q.res, keys), keys[self.B - 1])
+        return ev.rescale(Ct(sc, q.scale * 2.0 ** self.log_scale))
 
     def decide(self, ct_q, rows):
         """Ct whose slot i is ~ sign(<x_i, q_R> - tau |q_R|), amplified towards +-1"""

@@ -15,7 +15,7 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhann.so")
 
-HANN_MAX_PRIMES = 8
+HANN_MAX_PRIMES = 15
 OK, EINVAL, ESHAPE, ENOKEY, EWORKSPACE, ECUDA, ENOMEM = 0, -1, -2, -3, -4, -5, -6
 SIZE_POLY, SIZE_CT, SIZE_BABY, SIZE_PT_BLOCK, SIZE_INNER, SIZE_EVK, SIZE_ROWS_PER_BLOCK, SIZE_CTDB_BLOCK = 1, 2, 3, 4, 5, 6, 7, 8
 KIND_POLY, KIND_CT, KIND_PT = 1, 2, 3
@@ -43,6 +43,13 @@ class Stats(C.Structure):
     _fields_ = [
         ("launches", C.c_uint64), ("ms_query_prepare", C.c_float), ("ms_encode", C.c_float),
         ("ms_score_level", C.c_float), ("ms_rotate_sum", C.c_float), ("ms_keyswitch", C.c_float),
+    ]
+
+
+class MembershipParams(C.Structure):
+    _fields_ = [
+        ("R", C.c_int32), ("deg", C.c_int32), ("sign_iters", C.c_int32), ("log_scale", C.c_int32),
+        ("tau", C.c_double), ("t_lo", C.c_double), ("t_hi", C.c_double), ("coef", C.POINTER(C.c_double)),
     ]
 
 
@@ -103,6 +110,9 @@ def load_library():
         "hann_fold": (C.c_int, [vp, vp, C.c_int, C.c_int, vp, sz]),
         "hann_project_bytes": (i64, [vp, vp]),
         "hann_project_query": (C.c_int, [vp, vp, vp, vp, vp, vp, C.c_int, vp, vp, sz]),
+        "hann_membership_levels": (C.c_int, [C.c_int, C.c_int, vp, vp]),
+        "hann_membership_bytes": (i64, [vp, C.c_int, vp, vp, i64]),
+        "hann_membership_decide": (C.c_int, [vp, C.c_int, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, sz]),
         "hann_keyswitch": (C.c_int, [vp, C.c_int, vp, vp, vp, vp, sz]),
         "hann_query_level": (C.c_int, [vp, vp, vp, i64, C.c_int, vp, vp, vp, vp, vp, sz]),
         "hann_static_scratch_bytes": (i64, []),
@@ -504,3 +514,27 @@ class Context:
         self._ck(self.lib.hann_score_level_host(self.h, _ptr(ct_host), _ptr(rows_host), n_rows, dim, _ptr(out), _ptr(ws_dev),
                                                 ws_dev.numel() * 8))
         return out
+
+
+def membership_decide(arith, scorer, R, deg, sign_iters, log_scale, tau, t_lo, t_hi, coef, ct_dev, pt_dev, n_blocks, want_threshold=False):
+    """hann_membership_decide: arith = [context of the first l primes with R = B = 1 for l = 1..L], scorer = the context the
+    candidates were encoded on.  Returns (out [n_blocks][2][1][N] device tensor, its scale) and, if asked, the threshold
+    ciphertext (device tensor, level, scale)."""
+    top = arith[-1]
+    L = len(arith)
+    handles = (C.c_void_p * L)(*[a.h for a in arith])
+    coef = _np(coef, np.float64)
+    prm = MembershipParams(R, deg, sign_iters, log_scale, tau, t_lo, t_hi, coef.ctypes.data_as(C.POINTER(C.c_double)))
+    need = top.lib.hann_membership_bytes(handles, L, scorer.h, C.byref(prm), n_blocks)
+    if need < 0:
+        raise HannError(int(need), "hann_membership_bytes: bad argument")
+    ws = top.alloc(need)
+    out = top.alloc(max(n_blocks, 1) * 2 * top.N * 8)
+    out_scale, thr_scale, thr_level = C.c_double(0.0), C.c_double(0.0), C.c_int(0)
+    thr = top.alloc(2 * L * top.N * 8) if want_threshold else None
+    top._ck(top.lib.hann_membership_decide(handles, L, scorer.h, C.byref(prm), _ptr(ct_dev), _ptr(pt_dev), n_blocks, _ptr(out),
+                                           C.byref(out_scale), _ptr(thr), C.byref(thr_level), C.byref(thr_scale), _ptr(ws),
+                                           ws.numel() * 8))
+    if want_threshold:
+        return (out, out_scale.value), (thr, thr_level.value, thr_scale.value)
+    return out, out_scale.value

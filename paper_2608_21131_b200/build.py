@@ -20,7 +20,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhann.so")
 DEBUG_LIB = os.path.join(HERE, "libhann_debug.so")  # the -DHANN_DEBUG build (index range checks in the kernels)
 OBJDIR = os.path.join(HERE, "build")
-SOURCES = ["api.cu", "ntt.cu", "keyswitch.cu", "mac.cu", "encode.cu", "static_scratch.cu", "project.cu", "probe.cu", "hostmath.cpp"]
+SOURCES = ["api.cu", "ntt.cu", "keyswitch.cu", "mac.cu", "encode.cu", "static_scratch.cu", "project.cu", "probe.cu", "membership.cu", "hostmath.cpp"]
 HEADERS = ["internal.h", "modarith.cuh", "nttcore.cuh", "bulkcopy.cuh", "debugcheck.cuh", os.path.join("..", "..", "include", "hann.h")]
 
 

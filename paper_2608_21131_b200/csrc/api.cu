@@ -1151,7 +1151,7 @@ extern "C" int hann_score_level_ctdb(hann_ctx* c, const void* baby_dev, const vo
     if (n_blocks == 0) return HANN_OK;
     const int L = c->L, N = c->N, G = c->G;
     for (int l = 0; l < L; l++)
-        if (c->mod[l] >= (1ULL << 56)) return fail(c, HANN_ESHAPE, "hann_score_level_ctdb: ciphertext primes must be below 2^56");
+        if (c->mod[l] >= (1ULL << 60)) return fail(c, HANN_ESHAPE, "hann_score_level_ctdb: ciphertext primes must be below 2^60");
     if (c->B > 128) return fail(c, HANN_ESHAPE, "hann_score_level_ctdb: at most 128 baby steps");
     if (!c->keytab_host[0]) return fail(c, HANN_ENOKEY, "hann_score_level_ctdb: the relinearisation key (rotation 0) is not loaded");
     if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_score_level_ctdb: workspace missing or not 256-byte aligned");

@@ -494,6 +494,26 @@ __global__ void __launch_bounds__(kThreads) k_encrypt_finish(const u64* __restri
 
 }  // namespace
 
+// out[poly][l][t] = a[poly][l][t] * ma_l (+ b[poly][l][t] * mb_l) (+ k_l on the first polynomial of every ciphertext), mod q_l:
+// the additions, negations, integer multiples and added constants of a leveled circuit, in the transform domain (a constant
+// polynomial transforms to its constant in every position).  Ciphertexts of `limbs` limbs: polynomial pairs.
+struct LinearArgs {
+    u64 ma[HANN_MAXL1], mb[HANN_MAXL1], k[HANN_MAXL1];
+};
+__global__ void __launch_bounds__(kThreads) k_linear(const u64* __restrict__ a, const u64* __restrict__ b, u64* __restrict__ out,
+                                                     long long npoly, int limbs, int N, LinearArgs la, LimbTable lt) {
+    const long long total = npoly * limbs * N;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const int l = (int)((idx / N) % limbs);
+        const long long poly = idx / ((long long)limbs * N);
+        const LimbConst& lc = lt.c[l];
+        u64 v = la.ma[l] == 1 ? a[idx] : mulmod(a[idx], la.ma[l], lc);
+        if (b) v = addmod(v, la.mb[l] == 1 ? b[idx] : mulmod(b[idx], la.mb[l], lc), lc.q);
+        if ((poly & 1) == 0 && la.k[l]) v = addmod(v, la.k[l], lc.q);
+        out[idx] = v;
+    }
+}
+
 // ---- workspace guards (debugging aid): 32 words behind a sub-buffer hold a pattern derived from their own address
 __global__ void k_guard_fill(u64* guard) { guard[threadIdx.x] = 0xC0DEC0DEC0DEC0DEULL ^ (u64)(uintptr_t)(guard + threadIdx.x); }
 __global__ void k_guard_verify(u64* const* guards, long long count, unsigned long long* damaged) {
@@ -516,6 +536,23 @@ int check_launch(hann_ctx* c, const char* what) {
         return HANN_ECUDA;
     }
     return HANN_OK;
+}
+
+// out = ma * a + mb * b + k (k on the c0 of every ciphertext); ma, mb, k signed integers below 2^62 in magnitude, reduced per limb
+// here; b may be null.  npoly polynomials of c->L limbs.
+int launch_linear(hann_ctx* c, const u64* a, long long ma, const u64* b, long long mb, long long k, int64_t npoly, u64* out) {
+    LinearArgs la = {};
+    auto residue = [](long long v, u64 q) { return v >= 0 ? (u64)v % q : (q - ((u64)(-v) % q)) % q; };
+    for (int l = 0; l < c->L; l++) {
+        la.ma[l] = residue(ma, c->mod[l]);
+        la.mb[l] = residue(mb, c->mod[l]);
+        la.k[l] = residue(k, c->mod[l]);
+    }
+    {
+        KProf kp(c, KC_OTHER);
+        k_linear<<<grid_for(npoly * c->L * c->N), kThreads, 0, c->stream>>>(a, b, out, npoly, c->L, c->N, la, c->lt);
+    }
+    return check_launch(c, "linear");
 }
 
 int launch_guard_fill(hann_ctx* c, u64* guard) {

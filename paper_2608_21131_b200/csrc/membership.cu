@@ -1,0 +1,259 @@
+// The membership (threshold) circuit of the face task as a sequence of the library's own calls (Sec. 3.1, "The norm
+// problem", membership bullet; Sec. 2, "Security parameters": depth 11 on a chain of 12 primes).  The server compares the raw
+// score <x, q_R> with tau |q_R| = sqrt(tau^2 |q_R|^2) under encryption and returns a ciphertext whose SIGN is the decision:
+//   1. t = |q_R|^2 in every slot: the tiled query times itself (ciphertext x ciphertext, relinearised, rescaled), folded over
+//      the R slots of a period;
+//   2. u = a t + b in [-1, 1] (the factor a is absorbed by the client's encoding: it sends lam q_R, lam^2 = a q_{L-1} / Delta);
+//   3. r = sum_k c_k T_k(u), the low-degree Chebyshev interpolant of kappa tau sqrt(t): T_k by the product identity
+//      T_{m+n} = 2 T_m T_n - T_{m-n}, m = ceil(k/2); one integer-constant multiply per term brings all terms to one scale;
+//   4. s = kappa <x, q_R>: the ordinary scorer (candidates enrolled times kappa / lam) on the level that ends where r ends;
+//   5. sign(s - r) ~ f(f(f(.))), f(x) = x (3 - x^2) / 2, the halving done by a rescale over a prime of twice the scale.
+// Every ciphertext carries (level, scale); the scale arithmetic below is written operation by operation in IEEE binary64 so
+// that any evaluation of the same circuit in the same order gets the same integer constants.
+#include <cmath>
+#include <string>
+#include <vector>
+
+#include "internal.h"
+
+namespace {
+
+inline int64_t align256(int64_t x) { return (x + 255) & ~(int64_t)255; }
+
+struct MCt {
+    u64* p = nullptr;
+    int level = 0;
+    double scale = 0;
+};
+
+struct Circuit {
+    hann_ctx* const* arith;   // arith[l - 1]: the first l primes, R = B = 1
+    int L;
+    hann_ctx* top;            // arith[L - 1]: errors are reported through it
+    int N;
+    char* base;               // bump area for the circuit's ciphertexts
+    int64_t off = 0, cap = 0;
+    void* sub;                // workspace lent to the library calls
+    size_t sub_bytes;
+    int rc = HANN_OK;
+
+    hann_ctx* at(int level) const { return arith[level - 1]; }
+    double prime(int i) const { return (double)top->mod[i]; }
+    bool fail(int code, const std::string& msg) {
+        if (rc == HANN_OK) {
+            rc = code;
+            top->err = msg;
+        }
+        return false;
+    }
+    bool ok(int r, hann_ctx* from) {
+        if (r != HANN_OK && rc == HANN_OK) {
+            rc = r;
+            if (from != top) top->err = from->err;
+        }
+        return rc == HANN_OK;
+    }
+    u64* take(int level, int64_t cts = 1) {
+        const int64_t bytes = align256(cts * 2 * (int64_t)level * N * 8);
+        if (rc != HANN_OK) return nullptr;
+        if (off + bytes > cap) {
+            fail(HANN_EWORKSPACE, "hann_membership_decide: workspace too small");
+            return nullptr;
+        }
+        u64* r = (u64*)(base + off);
+        off += bytes;
+        return r;
+    }
+
+    // the first `level` primes of a: exact while the ciphertext's content is small against the shorter product
+    MCt drop(const MCt& a, int level) {
+        if (a.level == level || rc != HANN_OK) return a;
+        MCt o{take(level), level, a.scale};
+        if (o.p) ok(launch_copy2d(at(level), o.p, (int64_t)level * N, a.p, (int64_t)a.level * N, (int64_t)level * N, 2), at(level));
+        return o;
+    }
+    MCt linear(const MCt& a, long long ma, const MCt* b, long long mb, long long k, double scale) {
+        MCt o{take(a.level), a.level, scale};
+        if (o.p) ok(launch_linear(at(a.level), a.p, ma, b ? b->p : nullptr, mb, k, 2, o.p), at(a.level));
+        return o;
+    }
+    MCt add(const MCt& a0, const MCt& b0, int sign) {
+        const int l = a0.level < b0.level ? a0.level : b0.level;
+        const MCt a = drop(a0, l), b = drop(b0, l);
+        return linear(a, 1, &b, sign, 0, a.scale);
+    }
+    MCt neg(const MCt& a) { return linear(a, -1, nullptr, 0, 0, a.scale); }
+    MCt add_const(const MCt& a, double c) { return linear(a, 1, nullptr, 0, (long long)std::nearbyint(c * a.scale), a.scale); }
+    MCt mul_int(const MCt& a, long long m) { return linear(a, m, nullptr, 0, 0, a.scale); }
+    MCt rescale(const MCt& a) {
+        MCt o{take(a.level - 1), a.level - 1, a.scale / prime(a.level - 1)};
+        if (o.p) ok(hann_rescale(at(a.level), a.p, 1, o.p, sub, sub_bytes), at(a.level));
+        return o;
+    }
+    // ciphertext x ciphertext: the degree-2 product with one relinearisation (the multiply-accumulate of an encrypted block
+    // of one diagonal against a baby set of one ciphertext), then the rescale
+    MCt mul(const MCt& a0, const MCt& b0) {
+        const int l = a0.level < b0.level ? a0.level : b0.level;
+        const MCt a = drop(a0, l), b = drop(b0, l);
+        MCt prod{take(l), l, a.scale * b.scale};
+        if (prod.p) ok(hann_score_level_ctdb(at(l), b.p, a.p, 1, prod.p, sub, sub_bytes), at(l));
+        return rescale(prod);
+    }
+    MCt rotate(const MCt& a, int r) {
+        MCt o{take(a.level), a.level, a.scale};
+        if (o.p) ok(hann_rotate_hoisted(at(a.level), a.p, r, 1, o.p, sub, sub_bytes), at(a.level));
+        return o;
+    }
+    // factor * value at (very nearly) target_scale one level down: integer-constant multiply, then rescale
+    MCt to_scale(const MCt& a, double factor, double target_scale) {
+        const double q = prime(a.level - 1);
+        const double m = std::nearbyint(((factor * target_scale) * q) / a.scale);
+        MCt o = rescale(mul_int(a, (long long)m));
+        o.scale = ((a.scale * m) / q) / factor;
+        return o;
+    }
+};
+
+int threshold_depth(int deg) {
+    int lg = 0;
+    while ((1 << lg) < deg) lg++;
+    return 1 + lg + 1;
+}
+
+}  // namespace
+
+extern "C" int hann_membership_levels(int deg, int sign_iters, int* chain_primes, int* score_level) {
+    if (deg < 1 || deg > 15 || sign_iters < 0 || !chain_primes || !score_level) return HANN_EINVAL;
+    *chain_primes = threshold_depth(deg) + 2 * sign_iters + 1;
+    *score_level = *chain_primes - threshold_depth(deg) + 1;
+    return HANN_OK;
+}
+
+extern "C" int64_t hann_membership_bytes(hann_ctx* const* arith, int L, const hann_ctx* scorer, const hann_membership_params* prm,
+                                         int64_t n_blocks) {
+    if (!arith || !scorer || !prm || L < 2 || n_blocks < 0) return HANN_EINVAL;
+    for (int l = 1; l <= L; l++)
+        if (!arith[l - 1]) return HANN_EINVAL;
+    const int64_t N = arith[L - 1]->N, ct_top = align256(2 * (int64_t)L * N * 8);
+    // the circuit's ciphertexts never share storage: about 4 per Chebyshev term, 3 per fold step, 4 per sign iteration
+    int folds = 0;
+    while ((1 << folds) < prm->R) folds++;
+    const int64_t cts = 8 + 5 * (int64_t)prm->deg + 3 * folds + n_blocks * (4 + 5 * (int64_t)prm->sign_iters);
+    int64_t sub = 0;
+    for (int l = 1; l <= L; l++) sub = std::max<int64_t>(sub, hann_workspace_bytes(arith[l - 1], 1));
+    sub = std::max<int64_t>(sub, hann_workspace_bytes(scorer, 8));
+    const int64_t scoring = align256(hann_sizeof(scorer, HANN_SIZE_BABY)) + n_blocks * (align256(hann_sizeof(scorer, HANN_SIZE_INNER)) +
+                                                                                      align256(hann_sizeof(scorer, HANN_SIZE_CT)));
+    return cts * ct_top + scoring + align256(sub) + 4096;
+}
+
+extern "C" int hann_membership_decide(hann_ctx* const* arith, int L, hann_ctx* scorer, const hann_membership_params* prm,
+                                      const void* ct_dev, const void* pt_dev, int64_t n_blocks, void* out_dev, double* out_scale,
+                                      void* thr_dev, int* thr_level, double* thr_scale, void* ws, size_t ws_bytes) {
+    if (!arith || L < 2 || !arith[L - 1]) return HANN_EINVAL;
+    hann_ctx* top = arith[L - 1];
+    auto bad = [&](int code, const char* msg) {
+        top->err = msg;
+        return code;
+    };
+    if (!scorer || !prm || !prm->coef || !ct_dev || !out_dev || !out_scale || n_blocks < 0 || (n_blocks > 0 && !pt_dev))
+        return bad(HANN_EINVAL, "hann_membership_decide: bad argument");
+    int want_L = 0, score_level = 0;
+    if (hann_membership_levels(prm->deg, prm->sign_iters, &want_L, &score_level) != HANN_OK || want_L != L)
+        return bad(HANN_ESHAPE, "hann_membership_decide: the chain must have depth(threshold) + 2 * sign iterations + 1 primes");
+    for (int l = 1; l <= L; l++) {
+        const hann_ctx* a = arith[l - 1];
+        if (!a || a->L != l || a->N != top->N || a->R != 1 || a->B != 1 || a->device != top->device || a->stream != top->stream)
+            return bad(HANN_ESHAPE, "hann_membership_decide: arith[l-1] must be the context of the first l primes with R = B = 1");
+        for (int i = 0; i < l; i++)
+            if (a->mod[i] != top->mod[i]) return bad(HANN_ESHAPE, "hann_membership_decide: the contexts must share one chain of primes");
+        if (a->mod[l] != top->mod[L]) return bad(HANN_ESHAPE, "hann_membership_decide: the contexts must share the special prime");
+    }
+    if (scorer->L != score_level || scorer->N != top->N || scorer->R != prm->R || scorer->device != top->device || scorer->stream != top->stream)
+        return bad(HANN_ESHAPE, "hann_membership_decide: the scorer must be the context of the first (L - depth(threshold) + 1) primes with rank R");
+    for (int i = 0; i < score_level; i++)
+        if (scorer->mod[i] != top->mod[i]) return bad(HANN_ESHAPE, "hann_membership_decide: the scorer must use the chain's primes");
+    if (prm->R < 1 || (prm->R & (prm->R - 1)) || prm->t_hi <= prm->t_lo || prm->log_scale < 1 || prm->log_scale > 60)
+        return bad(HANN_EINVAL, "hann_membership_decide: R must be a power of two, t_lo < t_hi");
+    if (!ws || ((uintptr_t)ws & 255)) return bad(HANN_EWORKSPACE, "hann_membership_decide: workspace missing or not 256-byte aligned");
+    if ((int64_t)ws_bytes < hann_membership_bytes(arith, L, scorer, prm, n_blocks)) return bad(HANN_EWORKSPACE, "hann_membership_decide: workspace too small");
+
+    const int N = top->N;
+    int64_t sub = 0;
+    for (int l = 1; l <= L; l++) sub = std::max<int64_t>(sub, hann_workspace_bytes(arith[l - 1], 1));
+    sub = align256(std::max<int64_t>(sub, hann_workspace_bytes(scorer, 8)));
+    Circuit C;
+    C.arith = arith; C.L = L; C.top = top; C.N = N;
+    C.sub = ws; C.sub_bytes = (size_t)sub;
+    C.base = (char*)ws + sub; C.cap = (int64_t)ws_bytes - sub;
+    top->err.clear();
+
+    const double delta = std::ldexp(1.0, prm->log_scale), a = 2.0 / (prm->t_hi - prm->t_lo);
+    const double lam = std::sqrt(a * C.prime(L - 1) / delta);
+    const MCt q{(u64*)ct_dev, L, delta};
+
+    // 1, 2: |q_R|^2 (times lam^2) in every slot, read as a t at scale Delta; u = a t - (t_hi + t_lo) / (t_hi - t_lo)
+    MCt t = C.mul(q, q);
+    for (int r = 1; r < prm->R; r <<= 1) t = C.add(t, C.rotate(t, r), 1);
+    t.scale = t.scale / (lam * lam) * a;
+    const MCt u = C.add_const(t, -(prm->t_hi + prm->t_lo) / (prm->t_hi - prm->t_lo));
+    // 3: Chebyshev basis by the product identity, then the combination at one common scale
+    std::vector<MCt> T(prm->deg + 1);
+    T[1] = u;
+    for (int k = 2; k <= prm->deg; k++) {
+        const int m = (k + 1) / 2, nn = k - m;
+        const MCt prod2 = C.mul_int(C.mul(T[m], T[nn]), 2);
+        T[k] = m == nn ? C.add_const(prod2, -1.0) : C.add(prod2, T[m - nn], -1);
+    }
+    int level = T[1].level;
+    for (int k = 1; k <= prm->deg; k++) level = T[k].level < level ? T[k].level : level;
+    level -= 1;
+    MCt acc;
+    for (int k = 1; k <= prm->deg; k++) {
+        if (std::fabs(prm->coef[k]) < 1e-15) continue;
+        const MCt term = C.to_scale(C.drop(T[k], level + 1), prm->coef[k], delta);
+        acc = acc.p ? C.add(acc, term, 1) : term;
+    }
+    if (C.rc == HANN_OK && !acc.p) return bad(HANN_EINVAL, "hann_membership_decide: all polynomial coefficients vanish");
+    const MCt thr = C.add_const(acc, prm->coef[0]);
+    if (C.rc != HANN_OK) return C.rc;
+    if (thr.level + 1 != score_level) return bad(HANN_ESHAPE, "hann_membership_decide: internal level mismatch");
+    if (thr_dev) {
+        C.ok(launch_copy2d(C.at(thr.level), (u64*)thr_dev, 2LL * thr.level * N, thr.p, 2LL * thr.level * N, 2LL * thr.level * N, 1), C.at(thr.level));
+        if (thr_level) *thr_level = thr.level;
+        if (thr_scale) *thr_scale = thr.scale;
+    }
+    // 4: the scores of every block on the scorer's level, rescaled onto the threshold's level; 5: sign iterations
+    if (n_blocks > 0) {
+        const MCt qs = C.drop(q, score_level);
+        const int64_t babyb = align256(hann_sizeof(scorer, HANN_SIZE_BABY)), innerb = align256(hann_sizeof(scorer, HANN_SIZE_INNER));
+        u64* baby = nullptr;
+        u64* inner = nullptr;
+        if (C.rc == HANN_OK) {
+            if (C.off + babyb + n_blocks * innerb > C.cap) return bad(HANN_EWORKSPACE, "hann_membership_decide: workspace too small");
+            baby = (u64*)(C.base + C.off); C.off += babyb;
+            inner = (u64*)(C.base + C.off); C.off += n_blocks * innerb;
+        }
+        u64* score = C.take(score_level, n_blocks);
+        if (C.rc == HANN_OK) {
+            C.ok(hann_query_prepare(scorer, qs.p, baby, C.sub, C.sub_bytes), scorer);
+            C.ok(hann_score_level(scorer, baby, pt_dev, n_blocks, inner, C.sub, C.sub_bytes), scorer);
+            C.ok(hann_rotate_sum(scorer, inner, n_blocks, score, C.sub, C.sub_bytes), scorer);
+        }
+        const int64_t ctw = 2LL * score_level * N;
+        for (int64_t blk = 0; blk < n_blocks && C.rc == HANN_OK; blk++) {
+            const MCt s = C.rescale(MCt{score + blk * ctw, score_level, qs.scale * delta});
+            MCt x = C.add(s, thr, -1);
+            for (int it = 0; it < prm->sign_iters; it++) {
+                const MCt w = C.add_const(C.neg(C.mul(x, x)), 3.0);   // 3 - x^2 over a prime ~Delta
+                x = C.mul(x, w);                                      // x (3 - x^2) over a prime ~2 Delta ...
+                x.scale *= 2.0;                                       // ... read at the same scale it is x (3 - x^2) / 2
+            }
+            if (C.rc != HANN_OK) break;
+            if (x.level != 1) return bad(HANN_ESHAPE, "hann_membership_decide: internal level mismatch at the output");
+            C.ok(launch_copy2d(C.at(1), (u64*)out_dev + blk * 2LL * N, 2LL * N, x.p, 2LL * N, 2LL * N, 1), C.at(1));
+            *out_scale = x.scale;
+        }
+    }
+    return C.rc;
+}

@@ -27,7 +27,7 @@ struct LimbConst {
     double ninv_q;    // fl(ninv_bal / q)
 };
 
-#define HANN_MAXL1 9  // up to 8 ciphertext primes + the special prime
+#define HANN_MAXL1 16  // up to 15 ciphertext primes + the special prime (limb numbers travel in 4-bit fields)
 
 struct LimbTable {
     LimbConst c[HANN_MAXL1];

@@ -77,7 +77,7 @@ def test_encrypted_circuit_depth_eleven_matches_the_plain_circuit():
     ev = m.ev
     q, p, L = ev.q, ev.p, ev.L
     ps = synth.ParamSet("mem", logN, tuple(q), p, 45, R, 1, -10)
-    rots = sorted(set(range(1, R)) | set(m.fold_rotations()))
+    rots = sorted(set(m.score_rotations()) | set(m.fold_rotations()))
     km = synth.key_material(ps, 31, rots=rots)
     top = ev.o[L]
     rot_keys = {r: top.evk_gen(km.s, r, km.evk_a[i], km.evk_e[i]) for i, r in enumerate(rots)}

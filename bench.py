@@ -744,6 +744,108 @@ def run_project(args):
     return 0 if ok else 1
 
 
+def run_membership(args):
+    """Membership (threshold) scan of the face task (Sec. 3.1 norm problem; Sec. 2: depth 11, ring 2^15, 45-bit scale): one
+    encrypted query against the face-like level, the server returning per candidate a ciphertext slot whose sign says whether
+    <x, q_R> >= tau |q_R|.  A step = the whole circuit (hann_membership_decide) with the candidates encoded and resident.
+    Chain of 12 primes (58-bit first prime, 45/46-bit scaling primes), R = 128.  One JSON line; the decisions are checked
+    against the direct comparison outside the polynomial's error band."""
+    import torch
+    from paper_2608_21131_b200 import binding, synth, workloads as wl
+
+    torch.cuda.set_device(0)
+    logN, R, B, deg, iters, tau, t_lo, t_hi, log_scale = 15, 128, 32, 7, 3, 0.45, 0.05, 1.0, 45
+    n_rows = args.rows or 222_049
+    _, lvl, qR, planted = wl.face_level(rows=n_rows, ps=synth.FULL15)
+    qR = (0.7 * qR / np.linalg.norm(qR)).astype(np.float32)      # |q_R|^2 = 0.49, inside [t_lo, t_hi]
+    lib = binding.load_library()
+    lv = np.zeros(2, dtype=np.int32)
+    lib.hann_membership_levels(deg, iters, lv[0:].ctypes.data, lv[1:].ctypes.data)
+    L, score_level = int(lv[0]), int(lv[1])
+    # the chain: largest primes below 2^58 / 2^45 / 2^46 / 2^60 that are 1 mod 2N, consumed from the end (see hann.h)
+    def primes_below(bits, count):
+        import sympy
+
+        out, c = [], (1 << bits) - (2 << logN) + 1
+        while len(out) < count:
+            if sympy.isprime(c):
+                out.append(c)
+            c -= 2 << logN
+        return out
+    n_thr = 1 + 3 + 1
+    p45, p46 = primes_below(log_scale, n_thr + iters), primes_below(log_scale + 1, iters)
+    consumed = p45[:n_thr]
+    for i in range(iters):
+        consumed += [p45[n_thr + i], p46[i]]
+    q = primes_below(58, 1) + consumed[::-1]
+    p = primes_below(60, 1)[0]
+    a_aff = 2.0 / (t_hi - t_lo)
+    lam, kappa = float(np.sqrt(a_aff * q[-1] / 2.0 ** log_scale)), 0.5
+    k = np.arange(deg + 1)
+    nodes = np.cos(np.pi * (k + 0.5) / (deg + 1))
+    vals = kappa * tau * np.sqrt(0.5 * (t_hi - t_lo) * nodes + 0.5 * (t_hi + t_lo))
+    coef = np.array([2.0 / (deg + 1) * np.sum(vals * np.cos(np.pi * j * (k + 0.5) / (deg + 1))) for j in range(deg + 1)])
+    coef[0] *= 0.5
+    ps = synth.ParamSet("mem", logN, tuple(q), p, log_scale, R, B, -10)
+    fold = [1 << t for t in range(R.bit_length() - 1)]
+    rots = sorted(set(range(1, B + 1)) | set(fold))
+    km = synth.key_material(ps, wl.KEY_SEED, rots=rots)
+    topc = binding.Context(synth.ParamSet("a", logN, tuple(q), p, log_scale, 1, 1, -10))
+    evk = topc.keygen_from_samples(km.s, km.rots, km.evk_a, km.evk_e)
+    ka = synth.uniform_residues(wl.KEY_SEED, 50, list(q) + [p], ps.N, lead=(L,))
+    ke = synth.rounded_gaussian(wl.KEY_SEED, 51, (L, ps.N))
+    rlk = topc.keygen_relin_from_samples(km.s, ka, ke)
+    arith = [binding.Context(synth.ParamSet("a%d" % l, logN, tuple(q[:l]), p, log_scale, 1, 1, -10)) for l in range(1, L)] + [topc]
+    for l in range(2, L + 1):
+        arith[l - 1].load_keys(binding.restrict_keys(rlk, L, l)[None], [0])
+    pick = lambda wanted: np.stack([evk[rots.index(r)] for r in wanted])
+    arith[L - 2].load_keys(binding.restrict_keys(pick(fold), L, L - 1), fold)
+    scorer = binding.Context(synth.ParamSet("s", logN, tuple(q[:score_level]), p, log_scale, R, B, -10))
+    srots = list(range(1, B + 1))
+    scorer.load_keys(binding.restrict_keys(pick(srots), L, score_level), srots)
+    del evk
+    # the client encodes lam * q_R tiled with period R: a "dimension R" query of a context of that rank on the full chain
+    qctx = binding.Context(synth.ParamSet("q", logN, tuple(q), p, log_scale, R, 1, -10))
+    ct_dev = topc.import_(binding.KIND_CT, qctx.encrypt_query(km.s, (lam * qR.astype(np.float64)).astype(np.float32), km.ct_a, km.ct_e), 1)
+    del qctx
+    rows_scaled = (lvl.rows.astype(np.float64) * (kappa / lam)).astype(np.float32)
+    nb = scorer.n_blocks(n_rows)
+    pt = scorer.encode_candidates(torch.from_numpy(rows_scaled).to(scorer.device), scorer.workspace(nb))
+
+    def step():
+        return binding.membership_decide(arith, scorer, R, deg, iters, log_scale, tau, t_lo, t_hi, coef, ct_dev, pt, nb)
+
+    l0 = sum(c.get_stats()["launches"] for c in arith + [scorer])
+    out, out_scale = step()
+    launches = sum(c.get_stats()["launches"] for c in arith + [scorer]) - l0
+    for _ in range(max(args.warmup, 2)):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        out, out_scale = step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    dec = arith[0].decrypt_scores(km.s, arith[0].export(binding.KIND_CT, out, nb), log_scale_out=log_scale).reshape(-1)[:n_rows] * (2.0 ** log_scale / out_scale)
+    q64 = (lam * qR.astype(np.float64)).astype(np.float32).astype(np.float64) / lam       # the query as the client encoded it
+    direct = (rows_scaled.astype(np.float64) * (lam / kappa)) @ q64 - tau * np.linalg.norm(q64)
+    clear = np.abs(direct) > 4e-3 * tau
+    agree = bool(np.array_equal(np.sign(dec[clear]), np.sign(direct[clear])))
+    print(json.dumps({
+        "metric": "encrypted membership decisions/sec", "value": n_rows / (ms * 1e-3), "unit": "candidates/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 2), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64",
+        "data": "synthetic",
+        "config": {"workload": "membership (threshold) scan of the face-like level: %d rows, R=128, N=2^15, 12 primes (58b + 45/46b), depth 11" % n_rows,
+                   "blocks": nb, "tau": tau, "chebyshev_degree": deg, "sign_iterations": iters, "candidates": "encoded and resident"},
+        "gpu_launches": int(launches),
+        "check": {"decisions_agree_outside_error_band": agree, "rows_outside_band": int(clear.sum()), "matches": int((dec > 0).sum()),
+                  "planted_row_matches": bool(dec[planted] > 0), "ok": bool(agree and dec[planted] > 0)},
+    }))
+    return 0 if agree else 1
+
+
 def oracle_setup(ps, qR, km):
     from oracle.oracle import Oracle
 
@@ -944,6 +1046,7 @@ def main():
                     "hierarchies (latency per level), 4 scaling sweep point (--rows = wanted rows, --logn 15|16)")
     ap.add_argument("--logn", type=int, default=16, help="ring of the sweep configuration")
     ap.add_argument("--min-timed-s", type=float, default=2.0, help="the K-step block is repeated until the timed region lasted this long")
+    ap.add_argument("--membership", action="store_true", help="membership (threshold) scan of the face-like level at depth 11, N = 2^15")
     ap.add_argument("--project", action="store_true", help="packed projection 512 -> R of one encrypted query: baby-step sweep")
     ap.add_argument("--project-rank", type=int, default=128, help="R of --project (128 or 256)")
     ap.add_argument("--project-sweep", default="1,2,4,8,16,32", help="baby-step counts of --project")
@@ -970,6 +1073,10 @@ def main():
     if args.project:
         args.steps = 10 if args.steps is None else args.steps
         return run_project(args)
+    if args.membership:
+        args.steps = 5 if args.steps is None else args.steps
+        args.warmup = 2 if args.warmup is None else args.warmup
+        return run_membership(args)
     if args.config in (2, 3):
         args.steps = (16 if args.config == 2 else 64) if args.steps is None else args.steps
         args.warmup = 2 if args.warmup is None else args.warmup

@@ -135,10 +135,12 @@ extern "C" int64_t hann_membership_bytes(hann_ctx* const* arith, int L, const ha
     for (int l = 1; l <= L; l++)
         if (!arith[l - 1]) return HANN_EINVAL;
     const int64_t N = arith[L - 1]->N, ct_top = align256(2 * (int64_t)L * N * 8);
-    // the circuit's ciphertexts never share storage: about 4 per Chebyshev term, 3 per fold step, 4 per sign iteration
+    // The circuit's ciphertexts never share storage.  Counted at the size of a ciphertext of the full chain (most live on
+    // shorter ones): at most 12 per Chebyshev term (two level drops, product, rescale, doubling, the difference, and drop /
+    // multiple / rescale / sum in the combination), 2 per fold step, 3 per block plus 8 per sign iteration, 16 spare.
     int folds = 0;
     while ((1 << folds) < prm->R) folds++;
-    const int64_t cts = 8 + 5 * (int64_t)prm->deg + 3 * folds + n_blocks * (4 + 5 * (int64_t)prm->sign_iters);
+    const int64_t cts = 16 + 12 * (int64_t)prm->deg + 2 * folds + n_blocks * (3 + 8 * (int64_t)prm->sign_iters);
     int64_t sub = 0;
     for (int l = 1; l <= L; l++) sub = std::max<int64_t>(sub, hann_workspace_bytes(arith[l - 1], 1));
     sub = std::max<int64_t>(sub, hann_workspace_bytes(scorer, 8));

@@ -268,6 +268,56 @@ def test_error_codes():
     g.sync()
 
 
+def test_error_codes_of_the_newer_calls():
+    """refusals of the lazy giant steps, the hoisted rotation, the fold, the rescale, the projection and the membership
+    circuit: each names its reason, nothing is computed, and the contexts stay usable"""
+    from paper_2608_21131_b200 import binding as b
+    import torch
+
+    ps = synth.small_params(9, 16, 4, L=3, big=True)
+    g = b.Context(ps)
+    km = synth.key_material(ps, 1)                       # rotations 1..4: no key of rotation 8 or 12
+    g.load_keys(g.keygen_from_samples(km.s, km.rots, km.evk_a, km.evk_e), km.rots)
+    ws = g.workspace(1)
+    ct = g.alloc(g.sizeof(b.SIZE_CT))
+    ct.zero_()
+    inner = g.alloc(g.sizeof(b.SIZE_INNER))
+    inner.zero_()
+
+    def code(fn):
+        with pytest.raises(b.HannError) as ei:
+            fn()
+        return ei.value.code
+
+    assert code(lambda: g.rotate_sum_lazy(inner, 1, ws)) == b.ENOKEY                    # needs rotations 8 and 12
+    assert code(lambda: g.rotate_hoisted(ct, 3, 4, ws)) == b.ENOKEY                     # rotations 3..6
+    assert code(lambda: g.rotate_hoisted(ct, 0, 1, ws)) == b.ESHAPE
+    assert code(lambda: g.rotate_hoisted(ct, 1, 2, ws[:64])) == b.EWORKSPACE
+    assert code(lambda: g.fold(ct, 8, 1, ws)) == b.ENOKEY
+    assert code(lambda: g.fold(ct, 128, 2, ws)) == b.ESHAPE                             # rotation 256 = n
+    g.fold(ct, 2, 0, ws)                                                                # no steps: nothing to do
+    one = b.Context(ps.with_(q=ps.q[:1]))
+    assert code(lambda: one.rescale(one.alloc(one.sizeof(b.SIZE_CT)), 1, ws)) == b.ESHAPE   # a single prime left
+    assert g.rotate_sum_lazy(inner, 0, ws) is not None                                  # no blocks: a no-op
+    # projection: the second context must be the same ring with one prime less
+    other = b.Context(ps.with_(q=ps.q[:2], R=8, B=4))
+    lo = g.alloc(g.B * g.sizeof(b.SIZE_POLY) // 2)
+    wpt = other.alloc(other.sizeof(b.SIZE_PT_BLOCK))
+    assert code(lambda: g.project_query(other, ct, lo, lo, wpt, 64)) == b.ESHAPE
+    mid = b.Context(ps.with_(q=ps.q[:2]))
+    assert code(lambda: g.project_query(mid, ct, lo, lo, wpt, 48)) == b.ESHAPE          # D / R not a power of two
+    assert code(lambda: g.project_query(mid, ct, lo, lo, wpt, 64)) == b.ENOKEY          # rotation n - R + 1 is not loaded
+    W = torch.zeros((40, 16), dtype=torch.float32, device=g.device)
+    assert code(lambda: g.project_enrol(W, 50, ws)) == b.ESHAPE                         # D must be a multiple of R dividing n
+    # membership: a chain that does not fit the circuit's depth
+    arith = [b.Context(ps.with_(q=ps.q[:l], R=1, B=1)) for l in (1, 2, 3)]
+    coef = np.ones(8)
+    assert code(lambda: b.membership_decide(arith, g, 16, 7, 3, 40, 0.4, 0.05, 1.0, coef, ct, None, 0)) == b.ESHAPE
+    # and the context still computes
+    g.rotate_hoisted(ct, 1, 3, ws)
+    g.sync()
+
+
 # primes of the other arithmetic classes: [2^50, 2^57) runs the lazy integer transforms and the generic element-wise
 # kernels, >= 2^57 Harvey's butterflies; the special prime just below 2^62 is the largest the library accepts
 Q54 = (18014398506729473, 18014398505943041, 18014398496243713)

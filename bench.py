@@ -108,6 +108,8 @@ def bench_keys(ctx, ps, args):
     rots = list(range(1, ps.B + 1)) + [g * ps.B for g in range(2, ps.G)]
     if args.giant == "lazy":
         ctx.set_tuning(binding.TUNE_GIANT_LAZY, 1)
+    if args.lazy_lanes:
+        ctx.set_tuning(binding.TUNE_LAZY_LANES, args.lazy_lanes)
     km = synth.key_material(ps, wl.KEY_SEED, rots=rots)
     ctx.load_keys(ctx.keygen_from_samples(km.s, km.rots, km.evk_a, km.evk_e), km.rots)
     return km
@@ -1052,6 +1054,7 @@ def main():
     ap.add_argument("--project-sweep", default="1,2,4,8,16,32", help="baby-step counts of --project")
     ap.add_argument("--giant", default="lazy", choices=["horner", "lazy"],
                     help="evaluation order of the giant steps of the rotate-and-sum (the library's own default is Horner)")
+    ap.add_argument("--lazy-lanes", type=int, default=None, help="tuning: block ranges the lazy rotate-and-sum runs side by side (1..4)")
     ap.add_argument("--baby", type=int, default=None, help="baby-step count B (default: the configuration's; must divide R)")
     ap.add_argument("--rows", type=int, default=None, help="override the row count (debugging, ncu captures)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")

@@ -24,6 +24,7 @@ TUNE_HOST_LIMBS = 2
 TUNE_ENCODE_SYMMETRY = 3
 TUNE_HOST_GROUPS = 4
 TUNE_GIANT_LAZY = 5
+TUNE_LAZY_LANES = 6
 
 
 class HannError(RuntimeError):

@@ -570,6 +570,10 @@ extern "C" int hann_set_tuning(hann_ctx* c, int what, int value) {
         case HANN_TUNE_GIANT_LAZY:
             c->giant_lazy = value ? 1 : 0;
             return HANN_OK;
+        case HANN_TUNE_LAZY_LANES:
+            if (value < 1 || value > 4) return fail(c, HANN_EINVAL, "hann_set_tuning: lazy lanes must be 1..4");
+            c->lazy_lanes = value;
+            return HANN_OK;
         default: return fail(c, HANN_EINVAL, "hann_set_tuning: unknown knob");
     }
 }
@@ -1287,61 +1291,99 @@ extern "C" int hann_rotate_sum_lazy(hann_ctx* c, const void* inner_dev, int64_t 
     for (int g = 1; g < G; g++)
         if (!c->keytab_host[g * B]) return fail(c, HANN_ENOKEY, "hann_rotate_sum_lazy: the keys of rotations B, 2B, .., (G-1)B must be loaded");
     if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_rotate_sum_lazy: workspace missing or not 256-byte aligned");
-    int64_t ch = ((int64_t)ws_bytes - kSlack) / (lazy_block_words(c) * 8);
-    if (ch < 1) return fail(c, HANN_EWORKSPACE, "hann_rotate_sum_lazy: workspace too small");
-    ch = std::min<int64_t>(std::min<int64_t>(ch, n_blocks), 16);
-    Arena ar{(char*)ws, 0, (int64_t)ws_bytes, c};
-    const int64_t items_max = ch * (G - 1);
-    u64* c1c = ar.take<u64>(items_max * LN);
-    u64* digits = ar.take<u64>(items_max * L * L1N);
-    u64* u = ar.take<u64>(items_max * 2 * L1N);
-    u64* up = ar.take<u64>(ch * 2 * N);
-    u64* lifted = ar.take<u64>(ch * 2 * LN);
-    if (!c1c || !digits || !u || !up || !lifted) return fail(c, HANN_EWORKSPACE, "hann_rotate_sum_lazy: workspace too small");
     const bool lift = ks_lift_available(c);
-    for (int64_t b0 = 0; b0 < n_blocks; b0 += ch) {
-        const int64_t nb = std::min(ch, n_blocks - b0), items = nb * (G - 1);
-        // c1 of term (g, blk), still in the transform domain, into c1c[(g - 1) * nb + blk]
-        bool all_fused = lift;
-        for (int g = 1; g < G; g++) {
-            const u64* src = inner + (b0 * G + g) * ctw + LN;
-            u64* dst = c1c + (int64_t)(g - 1) * nb * LN;
-            const bool fused = lift && ntt_inv_pass_b_gathers(c, src, dst);
-            all_fused = all_fused && fused;
-            if (fused) RET(launch_ntt_inv_pass_b_from(c, src, (int64_t)G * ctw, dst, nb * L, N, limbmap_q(c)));
-            else RET(launch_copy2d(c, dst, LN, src, (int64_t)G * ctw, LN, nb));
-        }
-        if (lift) {
-            if (!all_fused) {
-                // the terms whose inverse pass ran while gathering are finished; the copied ones still need it
-                for (int g = 1; g < G; g++) {
-                    const u64* src = inner + (b0 * G + g) * ctw + LN;
-                    u64* dst = c1c + (int64_t)(g - 1) * nb * LN;
-                    if (!ntt_inv_pass_b_gathers(c, src, dst)) RET(launch_ntt_inv_pass_b(c, dst, nb * L, N, limbmap_q(c)));
-                }
+    // blocks [b_lo, b_hi), as many per round as the given part of the workspace holds, on the context's current stream
+    auto run_range = [&](int64_t b_lo, int64_t b_hi, char* wsp, int64_t wsp_bytes) -> int {
+        int64_t ch = (wsp_bytes - kSlack) / (lazy_block_words(c) * 8);
+        if (ch < 1) return fail(c, HANN_EWORKSPACE, "hann_rotate_sum_lazy: workspace too small");
+        ch = std::min<int64_t>(std::min<int64_t>(ch, b_hi - b_lo), 16);
+        Arena ar{wsp, 0, wsp_bytes, c};
+        const int64_t items_max = ch * (G - 1);
+        u64* c1c = ar.take<u64>(items_max * LN);
+        u64* digits = ar.take<u64>(items_max * L * L1N);
+        u64* u = ar.take<u64>(items_max * 2 * L1N);
+        u64* up = ar.take<u64>(ch * 2 * N);
+        u64* lifted = ar.take<u64>(ch * 2 * LN);
+        if (!c1c || !digits || !u || !up || !lifted) return fail(c, HANN_EWORKSPACE, "hann_rotate_sum_lazy: workspace too small");
+        for (int64_t b0 = b_lo; b0 < b_hi; b0 += ch) {
+            const int64_t nb = std::min(ch, b_hi - b0), items = nb * (G - 1);
+            // c1 of term (g, blk), still in the transform domain, into c1c[(g - 1) * nb + blk]
+            bool all_fused = lift;
+            for (int g = 1; g < G; g++) {
+                const u64* src = inner + (b0 * G + g) * ctw + LN;
+                u64* dst = c1c + (int64_t)(g - 1) * nb * LN;
+                const bool fused = lift && ntt_inv_pass_b_gathers(c, src, dst);
+                all_fused = all_fused && fused;
+                if (fused) RET(launch_ntt_inv_pass_b_from(c, src, (int64_t)G * ctw, dst, nb * L, N, limbmap_q(c)));
+                else RET(launch_copy2d(c, dst, LN, src, (int64_t)G * ctw, LN, nb));
             }
-            RET(launch_ks_lift(c, c1c, N, items * L, limbmap_q(c), digits, L + 1, 0));
-            RET(launch_ntt_fwd_pass_b(c, digits, items * L * (L + 1), N, limbmap_qp(c)));
-        } else {
-            RET(launch_ntt_inv(c, c1c, items * L, N, limbmap_q(c)));
-            RET(launch_lift_digits(c, c1c, LN, items, digits));
-            RET(launch_ntt_fwd(c, digits, items * L * (L + 1), N, limbmap_qp(c)));
+            if (lift) {
+                if (!all_fused) {
+                    // the terms whose inverse pass ran while gathering are finished; the copied ones still need it
+                    for (int g = 1; g < G; g++) {
+                        const u64* src = inner + (b0 * G + g) * ctw + LN;
+                        u64* dst = c1c + (int64_t)(g - 1) * nb * LN;
+                        if (!ntt_inv_pass_b_gathers(c, src, dst)) RET(launch_ntt_inv_pass_b(c, dst, nb * L, N, limbmap_q(c)));
+                    }
+                }
+                RET(launch_ks_lift(c, c1c, N, items * L, limbmap_q(c), digits, L + 1, 0));
+                RET(launch_ntt_fwd_pass_b(c, digits, items * L * (L + 1), N, limbmap_qp(c)));
+            } else {
+                RET(launch_ntt_inv(c, c1c, items * L, N, limbmap_q(c)));
+                RET(launch_lift_digits(c, c1c, LN, items, digits));
+                RET(launch_ntt_fwd(c, digits, items * L * (L + 1), N, limbmap_qp(c)));
+            }
+            // every giant step under its own key, all in one launch; then the special-prime limb of the SUM of the (permuted)
+            // products, its inverse transform, centred lift and forward transforms: one ModDown per block
+            RET(launch_ks_inner_batches(c, digits, (int64_t)L * L1N, B, B, G - 1, nb, u));
+            RET(launch_giant_sum_p(c, u, nb, up));
+            if (lift) {
+                RET(launch_ntt_inv_pass_b(c, up, nb * 2, N, limbmap_single(L)));
+                RET(launch_ks_lift(c, up, N, nb * 2, limbmap_single(L), lifted, L, 0));
+                RET(launch_ntt_fwd_pass_b(c, lifted, nb * 2 * L, N, limbmap_q(c)));
+            } else {
+                RET(launch_ntt_inv(c, up, nb * 2, N, limbmap_single(L)));
+                RET(launch_lift_p(c, up, nb * 2, lifted));
+                RET(launch_ntt_fwd(c, lifted, nb * 2 * L, N, limbmap_q(c)));
+            }
+            RET(launch_giant_combine(c, u, lifted, inner + b0 * G * ctw, nb, score + b0 * ctw));
         }
-        // every giant step under its own key, all in one launch; then the special-prime limb of the SUM of the (permuted)
-        // products, its inverse transform, centred lift and forward transforms: one ModDown per block
-        RET(launch_ks_inner_batches(c, digits, (int64_t)L * L1N, B, B, G - 1, nb, u));
-        RET(launch_giant_sum_p(c, u, nb, up));
-        if (lift) {
-            RET(launch_ntt_inv_pass_b(c, up, nb * 2, N, limbmap_single(L)));
-            RET(launch_ks_lift(c, up, N, nb * 2, limbmap_single(L), lifted, L, 0));
-            RET(launch_ntt_fwd_pass_b(c, lifted, nb * 2 * L, N, limbmap_q(c)));
-        } else {
-            RET(launch_ntt_inv(c, up, nb * 2, N, limbmap_single(L)));
-            RET(launch_lift_p(c, up, nb * 2, lifted));
-            RET(launch_ntt_fwd(c, lifted, nb * 2 * L, N, limbmap_q(c)));
-        }
-        RET(launch_giant_combine(c, u, lifted, inner + b0 * G * ctw, nb, score + b0 * ctw));
+        return HANN_OK;
+    };
+    // Block ranges are independent: up to `lazy_lanes` of them run side by side on the context's stream and its helper
+    // streams, each in its own part of the workspace, so that the short launches of one range (the ModDown of a few
+    // polynomials is a latency chain on a fraction of the machine) overlap the long ones of another.  One lane while the
+    // per-launch profile is on (its kernel times must not overlap) and when the caller already is on a helper stream.
+    int lanes = (int)std::min<int64_t>(c->lazy_lanes, n_blocks);
+    if (c->stream == c->aux_stream || c->kprof || c->max_lanes <= 1) lanes = 1;
+    while (lanes > 1 && (((int64_t)ws_bytes / lanes) & ~(int64_t)255) < lazy_block_words(c) * 8 + kSlack) lanes--;
+    if (lanes <= 1) return run_range(0, n_blocks, (char*)ws, (int64_t)ws_bytes);
+    const int64_t part = ((int64_t)ws_bytes / lanes) & ~(int64_t)255;
+    cudaStream_t main_stream = c->stream;
+    cudaStream_t helper[3] = {c->aux_stream, c->lane_stream[0], c->lane_stream[1]};
+    cudaEvent_t joined[3] = {c->ev_join, c->lane_join[0], c->lane_join[1]};
+    CK(cudaEventRecord(c->ev_fork, main_stream));
+    int rc = HANN_OK;
+    cudaError_t ce = cudaSuccess;
+    for (int ln = 1; ln < lanes; ln++) {
+        const int64_t lo = n_blocks * ln / lanes, hi = n_blocks * (ln + 1) / lanes;
+        cudaError_t e = cudaStreamWaitEvent(helper[ln - 1], c->ev_fork, 0);
+        c->stream = helper[ln - 1];
+        const int r = e == cudaSuccess ? run_range(lo, hi, (char*)ws + ln * part, part) : HANN_ECUDA;
+        c->stream = main_stream;
+        if (e == cudaSuccess) e = cudaEventRecord(joined[ln - 1], helper[ln - 1]);
+        if (rc == HANN_OK) rc = r;
+        if (ce == cudaSuccess) ce = e;
     }
+    const int r0 = run_range(0, n_blocks / lanes, (char*)ws, part);
+    if (rc == HANN_OK) rc = r0;
+    // join every helper before reporting anything: no helper stream runs past this call unobserved
+    for (int ln = 1; ln < lanes; ln++) {
+        cudaError_t e = cudaStreamWaitEvent(main_stream, joined[ln - 1], 0);
+        if (ce == cudaSuccess) ce = e;
+    }
+    RET(rc);
+    CK(ce);
     return HANN_OK;
 }
 

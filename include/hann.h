@@ -277,6 +277,13 @@ int hann_score_level_batch(hann_ctx *ctx, const void *baby_dev, int n_queries, c
 int hann_score_level_ctdb(hann_ctx *ctx, const void *baby_dev, const void *ctdb_dev, int64_t n_blocks, void *inner_dev,
                           void *ws, size_t ws_bytes);
 
+/* Ciphertext x ciphertext product of `count` independent pairs with relinearisation (the multiplication of a CKKS circuit;
+ * Sec. 2: the encrypted database and the membership path need it): out[i] = (d0 + ks0, d1 + ks1), (d0, d1, d2) =
+ * (a0 b0, a0 b1 + a1 b0, a1 b1) of pair i, (ks0, ks1) the key switch of d2 under the relinearisation key (rotation 0).
+ * The scale of out is the product of the scales; hann_rescale follows in a circuit.  a_dev, b_dev, out_dev: count
+ * ciphertexts each (internal layout); out may not alias a or b. */
+int hann_multiply(hann_ctx *ctx, const void *a_dev, const void *b_dev, int64_t count, void *out_dev, void *ws, size_t ws_bytes);
+
 /* Rotate-and-sum (Sec. 3.1 Detail: the giant steps of the diagonal method): score_ct[blk] = sum_g rot_{g*B}(inner[blk][g]), evaluated by Horner with the single key of
  * rotation B: acc = inner[G-1]; for g = G-2..0: acc = rot_B(acc) + inner[g].
  *   score_ct_dev n_blocks * HANN_SIZE_CT bytes (device), internal layout. */

@@ -102,6 +102,7 @@ def load_library():
         "hann_score_level_batch": (C.c_int, [vp, vp, C.c_int, vp, i64, vp, vp, sz]),
         "hann_rotate_sum": (C.c_int, [vp, vp, i64, vp, vp, sz]),
         "hann_rotate_sum_lazy": (C.c_int, [vp, vp, i64, vp, vp, sz]),
+        "hann_multiply": (C.c_int, [vp, vp, vp, i64, vp, vp, sz]),
         "hann_rotate_hoisted": (C.c_int, [vp, vp, C.c_int, C.c_int, vp, vp, sz]),
         "hann_encode_slots": (C.c_int, [vp, vp, i64, C.c_int, vp, vp, sz]),
         "hann_project_enrol": (C.c_int, [vp, vp, C.c_int, C.c_int, vp, vp, sz]),
@@ -418,6 +419,11 @@ class Context:
             score = self.alloc(n_blocks * self.sizeof(SIZE_CT))
         self._ck(self.lib.hann_rotate_sum(self.h, _ptr(inner), n_blocks, _ptr(score), _ptr(ws), ws.numel() * 8))
         return score
+
+    def multiply(self, a, b_, count, ws):
+        out = self.alloc(count * self.sizeof(SIZE_CT))
+        self._ck(self.lib.hann_multiply(self.h, _ptr(a), _ptr(b_), count, _ptr(out), _ptr(ws), ws.numel() * 8))
+        return out
 
     def rotate_sum_lazy(self, inner, n_blocks, ws, score=None):
         if score is None:

@@ -466,7 +466,8 @@ extern "C" int64_t hann_workspace_bytes(const hann_ctx* c, int64_t max_blocks) {
     const int64_t items = std::max<int64_t>(1, std::min<int64_t>(max_blocks, 8));
     int64_t w = std::max(ks_item_words(c) * items, prepare_words(c)) * 8;
     w = std::max(w, (ks_item_words(c) + (int64_t)c->L * c->N) * 8);  // hann_keyswitch permutes its input first
-    w = std::max(w, (ks_item_words(c) + 3 * (int64_t)c->L * c->N) * 8);  // hann_score_level_ctdb: one degree-2 sum + its key switch
+    // hann_score_level_ctdb, hann_multiply: per item one degree-2 sum + its key switch
+    w = std::max(w, (ks_item_words(c) + 3 * (int64_t)c->L * c->N) * items * 8);
     w = std::max(w, lazy_block_words(c) * std::min<int64_t>(items, 4) * 8);  // hann_rotate_sum_lazy: up to four blocks per round
     w = std::max(w, encode_ws_bytes(c));
     // hann_query_level runs query_prepare and encode_candidates side by side, each in its own part
@@ -1185,6 +1186,43 @@ extern "C" int hann_score_level_ctdb(hann_ctx* c, const void* baby_dev, const vo
         RET(launch_copy2d(c, c1c, LN, d + 2 * LN, 3 * LN, LN, ni));
         RET(ks_digits_to_lifted(c, c1c, ni, digits, (int64_t)L * L1N, 0, 0, ni, u, lifted));
         RET(launch_moddown_combine(c, u, lifted, ni, 0, 0, nullptr, 0, d, 3 * LN, inner + i0 * ctw, inner + i0 * ctw + LN, ctw));
+    }
+    return HANN_OK;
+}
+
+extern "C" int hann_multiply(hann_ctx* c, const void* a_dev, const void* b_dev, int64_t count, void* out_dev, void* ws, size_t ws_bytes) {
+    if (!c) return HANN_EINVAL;
+    if (count < 0 || (count > 0 && (!a_dev || !b_dev || !out_dev))) return fail(c, HANN_EINVAL, "hann_multiply: bad argument");
+    if (count == 0) return HANN_OK;
+    const int L = c->L, N = c->N;
+    for (int l = 0; l < L; l++)
+        if (c->mod[l] >= (1ULL << 62)) return fail(c, HANN_ESHAPE, "hann_multiply: ciphertext primes must be below 2^62");
+    if (!c->keytab_host[0]) return fail(c, HANN_ENOKEY, "hann_multiply: the relinearisation key (rotation 0) is not loaded");
+    if (!ws || ((uintptr_t)ws & 255)) return fail(c, HANN_EWORKSPACE, "hann_multiply: workspace missing or not 256-byte aligned");
+    DeviceGuard dg(c->device);
+    Timer tm(c, 2);
+    const int64_t LN = (int64_t)L * N, L1N = (int64_t)(L + 1) * N, ctw = 2 * LN;
+    // per pair: the degree-2 product (3 polynomials) and one key switch (its own copy of d2, digits, u, lifted)
+    const int64_t per = (3 * LN + ks_item_words(c)) * 8;
+    int64_t ch = ((int64_t)ws_bytes - kSlack) / per;
+    if (ch < 1) return fail(c, HANN_EWORKSPACE, "hann_multiply: workspace too small");
+    ch = std::min<int64_t>(std::min<int64_t>(ch, count), 32);
+    Arena ar{(char*)ws, 0, (int64_t)ws_bytes, c};
+    u64* d = ar.take<u64>(ch * 3 * LN);
+    u64* c1c = ar.take<u64>(ch * LN);
+    u64* digits = ar.take<u64>(ch * L * L1N);
+    u64* u = ar.take<u64>(ch * 2 * L1N);
+    u64* lifted = ar.take<u64>(ch * 2 * LN);
+    if (!d || !c1c || !digits || !u || !lifted) return fail(c, HANN_EWORKSPACE, "hann_multiply: workspace too small");
+    const u64 *a = (const u64*)a_dev, *b = (const u64*)b_dev;
+    u64* out = (u64*)out_dev;
+    for (int64_t i0 = 0; i0 < count; i0 += ch) {
+        const int64_t ni = std::min(ch, count - i0);
+        RET(launch_mul_ct(c, a + i0 * ctw, b + i0 * ctw, ni, d));
+        // relinearise: (d0 + ks0, d1 + ks1), (ks0, ks1) the key switch of d2 under the key of s^2 ("rotation 0")
+        RET(launch_copy2d(c, c1c, LN, d + 2 * LN, 3 * LN, LN, ni));
+        RET(ks_digits_to_lifted(c, c1c, ni, digits, (int64_t)L * L1N, 0, 0, ni, u, lifted));
+        RET(launch_moddown_combine(c, u, lifted, ni, 0, 0, nullptr, 0, d, 3 * LN, out + i0 * ctw, out + i0 * ctw + LN, ctw));
     }
     return HANN_OK;
 }

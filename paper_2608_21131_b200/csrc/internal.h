@@ -140,7 +140,10 @@ int64_t keyswitch_ws_bytes(const hann_ctx* c);
 int static_scratch_resolve(hann_ctx* c, void** out);
 
 // out = ma * a + mb * b + k on npoly polynomials of c->L limbs (k on the first polynomial of every pair); b may be null
-int launch_linear(hann_ctx* c, const u64* a, long long ma, const u64* b, long long mb, long long k, int64_t npoly, u64* out);
+int launch_linear(hann_ctx* c, const u64* a, long long ma, const u64* b, long long mb, long long k, int64_t npoly, u64* out,
+                  int64_t b_period = 0);
+// d[i] = (a0 b0, a0 b1 + a1 b0, a1 b1) for `count` ciphertext pairs
+int launch_mul_ct(hann_ctx* c, const u64* a, const u64* b, int64_t count, u64* d);
 int launch_guard_fill(hann_ctx* c, u64* guard);                                             // 32 words of pattern
 int launch_guard_verify(hann_ctx* c, u64* const* guards, int64_t count, unsigned long long* damaged);  // counts damaged guards
 // debug build: point each translation unit's range-check word at the context's error word (no-ops in a release build)

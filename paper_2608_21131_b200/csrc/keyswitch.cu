@@ -500,17 +500,37 @@ __global__ void __launch_bounds__(kThreads) k_encrypt_finish(const u64* __restri
 struct LinearArgs {
     u64 ma[HANN_MAXL1], mb[HANN_MAXL1], k[HANN_MAXL1];
 };
+// b_period > 0: b has only b_period words (one ciphertext) and is used for every ciphertext of a.
 __global__ void __launch_bounds__(kThreads) k_linear(const u64* __restrict__ a, const u64* __restrict__ b, u64* __restrict__ out,
-                                                     long long npoly, int limbs, int N, LinearArgs la, LimbTable lt) {
+                                                     long long npoly, int limbs, int N, long long b_period, LinearArgs la, LimbTable lt) {
     const long long total = npoly * limbs * N;
     for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
         const int l = (int)((idx / N) % limbs);
         const long long poly = idx / ((long long)limbs * N);
         const LimbConst& lc = lt.c[l];
         u64 v = la.ma[l] == 1 ? a[idx] : mulmod(a[idx], la.ma[l], lc);
-        if (b) v = addmod(v, la.mb[l] == 1 ? b[idx] : mulmod(b[idx], la.mb[l], lc), lc.q);
+        if (b) {
+            const u64 bv = b[b_period > 0 ? idx % b_period : idx];
+            v = addmod(v, la.mb[l] == 1 ? bv : mulmod(bv, la.mb[l], lc), lc.q);
+        }
         if ((poly & 1) == 0 && la.k[l]) v = addmod(v, la.k[l], lc.q);
         out[idx] = v;
+    }
+}
+
+// degree-2 product of `count` independent ciphertext pairs: d[i] = (a0 b0, a0 b1 + a1 b0, a1 b1), all [.][limbs][N], elementwise
+// in the transform domain
+__global__ void __launch_bounds__(kThreads) k_mul_ct(const u64* __restrict__ a, const u64* __restrict__ b, u64* __restrict__ d,
+                                                     long long count, int limbs, int N, LimbTable lt) {
+    const long long LN = (long long)limbs * N, total = count * LN;
+    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
+        const long long i = idx / LN, pos = idx % LN;
+        const LimbConst& lc = lt.c[(int)(pos / N)];
+        const u64 a0 = a[i * 2 * LN + pos], a1 = a[i * 2 * LN + LN + pos], b0 = b[i * 2 * LN + pos], b1 = b[i * 2 * LN + LN + pos];
+        u64* o = d + i * 3 * LN + pos;
+        o[0] = mulmod(a0, b0, lc);
+        o[LN] = addmod(mulmod(a0, b1, lc), mulmod(a1, b0, lc), lc.q);
+        o[2 * LN] = mulmod(a1, b1, lc);
     }
 }
 
@@ -539,8 +559,17 @@ int check_launch(hann_ctx* c, const char* what) {
 }
 
 // out = ma * a + mb * b + k (k on the c0 of every ciphertext); ma, mb, k signed integers below 2^62 in magnitude, reduced per limb
-// here; b may be null.  npoly polynomials of c->L limbs.
-int launch_linear(hann_ctx* c, const u64* a, long long ma, const u64* b, long long mb, long long k, int64_t npoly, u64* out) {
+// here; b may be null.  npoly polynomials of c->L limbs; b_period > 0: b is ONE ciphertext (b_period words) added to every one of a.
+int launch_mul_ct(hann_ctx* c, const u64* a, const u64* b, int64_t count, u64* d) {
+    {
+        KProf kp(c, KC_MAC);
+        k_mul_ct<<<grid_for(count * c->L * c->N), kThreads, 0, c->stream>>>(a, b, d, count, c->L, c->N, c->lt);
+    }
+    return check_launch(c, "mul_ct");
+}
+
+int launch_linear(hann_ctx* c, const u64* a, long long ma, const u64* b, long long mb, long long k, int64_t npoly, u64* out,
+                  int64_t b_period) {
     LinearArgs la = {};
     auto residue = [](long long v, u64 q) { return v >= 0 ? (u64)v % q : (q - ((u64)(-v) % q)) % q; };
     for (int l = 0; l < c->L; l++) {
@@ -550,7 +579,7 @@ int launch_linear(hann_ctx* c, const u64* a, long long ma, const u64* b, long lo
     }
     {
         KProf kp(c, KC_OTHER);
-        k_linear<<<grid_for(npoly * c->L * c->N), kThreads, 0, c->stream>>>(a, b, out, npoly, c->L, c->N, la, c->lt);
+        k_linear<<<grid_for(npoly * c->L * c->N), kThreads, 0, c->stream>>>(a, b, out, npoly, c->L, c->N, b_period, la, c->lt);
     }
     return check_launch(c, "linear");
 }

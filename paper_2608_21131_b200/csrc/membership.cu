@@ -20,10 +20,12 @@ namespace {
 
 inline int64_t align256(int64_t x) { return (x + 255) & ~(int64_t)255; }
 
+// n ciphertexts of one level and scale, stored one after the other: the circuit's operations act on all of them at once
 struct MCt {
     u64* p = nullptr;
     int level = 0;
     double scale = 0;
+    int64_t n = 1;
 };
 
 struct Circuit {
@@ -68,13 +70,16 @@ struct Circuit {
     // the first `level` primes of a: exact while the ciphertext's content is small against the shorter product
     MCt drop(const MCt& a, int level) {
         if (a.level == level || rc != HANN_OK) return a;
-        MCt o{take(level), level, a.scale};
-        if (o.p) ok(launch_copy2d(at(level), o.p, (int64_t)level * N, a.p, (int64_t)a.level * N, (int64_t)level * N, 2), at(level));
+        MCt o{take(level, a.n), level, a.scale, a.n};
+        if (o.p) ok(launch_copy2d(at(level), o.p, (int64_t)level * N, a.p, (int64_t)a.level * N, (int64_t)level * N, 2 * a.n), at(level));
         return o;
     }
+    // ma a + mb b + k; b is either as many ciphertexts as a or a single one that goes with every ciphertext of a
     MCt linear(const MCt& a, long long ma, const MCt* b, long long mb, long long k, double scale) {
-        MCt o{take(a.level), a.level, scale};
-        if (o.p) ok(launch_linear(at(a.level), a.p, ma, b ? b->p : nullptr, mb, k, 2, o.p), at(a.level));
+        MCt o{take(a.level, a.n), a.level, scale, a.n};
+        if (b && b->n != a.n && b->n != 1) fail(HANN_EINVAL, "hann_membership_decide: internal operand count mismatch");
+        const int64_t period = b && b->n == 1 && a.n > 1 ? 2LL * a.level * N : 0;
+        if (o.p && rc == HANN_OK) ok(launch_linear(at(a.level), a.p, ma, b ? b->p : nullptr, mb, k, 2 * a.n, o.p, period), at(a.level));
         return o;
     }
     MCt add(const MCt& a0, const MCt& b0, int sign) {
@@ -82,21 +87,22 @@ struct Circuit {
         const MCt a = drop(a0, l), b = drop(b0, l);
         return linear(a, 1, &b, sign, 0, a.scale);
     }
-    MCt neg(const MCt& a) { return linear(a, -1, nullptr, 0, 0, a.scale); }
+    // c - a
+    MCt const_minus(const MCt& a, double c) { return linear(a, -1, nullptr, 0, (long long)std::nearbyint(c * a.scale), a.scale); }
     MCt add_const(const MCt& a, double c) { return linear(a, 1, nullptr, 0, (long long)std::nearbyint(c * a.scale), a.scale); }
     MCt mul_int(const MCt& a, long long m) { return linear(a, m, nullptr, 0, 0, a.scale); }
     MCt rescale(const MCt& a) {
-        MCt o{take(a.level - 1), a.level - 1, a.scale / prime(a.level - 1)};
-        if (o.p) ok(hann_rescale(at(a.level), a.p, 1, o.p, sub, sub_bytes), at(a.level));
+        MCt o{take(a.level - 1, a.n), a.level - 1, a.scale / prime(a.level - 1), a.n};
+        if (o.p) ok(hann_rescale(at(a.level), a.p, a.n, o.p, sub, sub_bytes), at(a.level));
         return o;
     }
-    // ciphertext x ciphertext: the degree-2 product with one relinearisation (the multiply-accumulate of an encrypted block
-    // of one diagonal against a baby set of one ciphertext), then the rescale
+    // ciphertext x ciphertext, pair by pair: the degree-2 product with one relinearisation, then the rescale
     MCt mul(const MCt& a0, const MCt& b0) {
         const int l = a0.level < b0.level ? a0.level : b0.level;
         const MCt a = drop(a0, l), b = drop(b0, l);
-        MCt prod{take(l), l, a.scale * b.scale};
-        if (prod.p) ok(hann_score_level_ctdb(at(l), b.p, a.p, 1, prod.p, sub, sub_bytes), at(l));
+        if (a.n != b.n) fail(HANN_EINVAL, "hann_membership_decide: internal operand count mismatch");
+        MCt prod{take(l, a.n), l, a.scale * b.scale, a.n};
+        if (prod.p && rc == HANN_OK) ok(hann_multiply(at(l), a.p, b.p, a.n, prod.p, sub, sub_bytes), at(l));
         return rescale(prod);
     }
     MCt rotate(const MCt& a, int r) {
@@ -142,7 +148,7 @@ extern "C" int64_t hann_membership_bytes(hann_ctx* const* arith, int L, const ha
     while ((1 << folds) < prm->R) folds++;
     const int64_t cts = 16 + 12 * (int64_t)prm->deg + 2 * folds + n_blocks * (3 + 8 * (int64_t)prm->sign_iters);
     int64_t sub = 0;
-    for (int l = 1; l <= L; l++) sub = std::max<int64_t>(sub, hann_workspace_bytes(arith[l - 1], 1));
+    for (int l = 1; l <= L; l++) sub = std::max<int64_t>(sub, hann_workspace_bytes(arith[l - 1], l < scorer->L ? n_blocks : 1));
     sub = std::max<int64_t>(sub, hann_workspace_bytes(scorer, 8));
     const int64_t scoring = align256(hann_sizeof(scorer, HANN_SIZE_BABY)) + n_blocks * (align256(hann_sizeof(scorer, HANN_SIZE_INNER)) +
                                                                                       align256(hann_sizeof(scorer, HANN_SIZE_CT)));
@@ -182,7 +188,8 @@ extern "C" int hann_membership_decide(hann_ctx* const* arith, int L, hann_ctx* s
 
     const int N = top->N;
     int64_t sub = 0;
-    for (int l = 1; l <= L; l++) sub = std::max<int64_t>(sub, hann_workspace_bytes(arith[l - 1], 1));
+    // below the scorer's level the operations run over all blocks at once: room for several key switches side by side
+    for (int l = 1; l <= L; l++) sub = std::max<int64_t>(sub, hann_workspace_bytes(arith[l - 1], l < score_level ? n_blocks : 1));
     sub = align256(std::max<int64_t>(sub, hann_workspace_bytes(scorer, 8)));
     Circuit C;
     C.arith = arith; C.L = L; C.top = top; C.N = N;
@@ -242,18 +249,18 @@ extern "C" int hann_membership_decide(hann_ctx* const* arith, int L, hann_ctx* s
             C.ok(hann_score_level(scorer, baby, pt_dev, n_blocks, inner, C.sub, C.sub_bytes), scorer);
             C.ok(hann_rotate_sum(scorer, inner, n_blocks, score, C.sub, C.sub_bytes), scorer);
         }
-        const int64_t ctw = 2LL * score_level * N;
-        for (int64_t blk = 0; blk < n_blocks && C.rc == HANN_OK; blk++) {
-            const MCt s = C.rescale(MCt{score + blk * ctw, score_level, qs.scale * delta});
+        // all blocks advance together: every operation below is one (chunked) call over n_blocks ciphertexts
+        if (C.rc == HANN_OK) {
+            const MCt s = C.rescale(MCt{score, score_level, qs.scale * delta, n_blocks});
             MCt x = C.add(s, thr, -1);
             for (int it = 0; it < prm->sign_iters; it++) {
-                const MCt w = C.add_const(C.neg(C.mul(x, x)), 3.0);   // 3 - x^2 over a prime ~Delta
+                const MCt w = C.const_minus(C.mul(x, x), 3.0);         // 3 - x^2 over a prime ~Delta
                 x = C.mul(x, w);                                      // x (3 - x^2) over a prime ~2 Delta ...
                 x.scale *= 2.0;                                       // ... read at the same scale it is x (3 - x^2) / 2
             }
-            if (C.rc != HANN_OK) break;
+            if (C.rc != HANN_OK) return C.rc;
             if (x.level != 1) return bad(HANN_ESHAPE, "hann_membership_decide: internal level mismatch at the output");
-            C.ok(launch_copy2d(C.at(1), (u64*)out_dev + blk * 2LL * N, 2LL * N, x.p, 2LL * N, 2LL * N, 1), C.at(1));
+            C.ok(launch_copy2d(C.at(1), (u64*)out_dev, 2LL * N, x.p, 2LL * N, 2LL * N, n_blocks), C.at(1));
             *out_scale = x.scale;
         }
     }

@@ -11,7 +11,7 @@ from paper_2608_21131_b200 import synth
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("logN,R,B,deg,iters,n_rows", [(10, 16, 4, 7, 3, 900), (9, 8, 2, 3, 1, 200), (12, 32, 8, 7, 3, 2048)])
+@pytest.mark.parametrize("logN,R,B,deg,iters,n_rows", [(10, 16, 4, 7, 3, 900), (9, 8, 2, 3, 1, 200), (9, 8, 2, 3, 2, 2500), (12, 32, 8, 7, 3, 2048)])
 def test_membership_circuit_bit_exact(logN, R, B, deg, iters, n_rows):
     import torch
 
@@ -79,3 +79,41 @@ def test_membership_circuit_bit_exact(logN, R, B, deg, iters, n_rows):
     want = m.plain(rows, qR)["out"]
     assert np.abs(mine - want).max() < 1e-3
     assert mine[11] > 0
+
+
+@pytest.mark.parametrize("logN,L,count", [(10, 4, 1), (11, 3, 11), (12, 6, 3)])
+def test_multiply_bit_exact(logN, L, count):
+    """hann_multiply: `count` ciphertext pairs, degree-2 product and relinearisation, against the oracle's product of each
+    pair; then the rescale of all of them in one call."""
+    import torch
+
+    from oracle.oracle import Oracle, find_primes
+    from paper_2608_21131_b200 import binding as b
+
+    q, p = find_primes(45, logN + 1, L), find_primes(60, logN + 1, 1)[0]
+    ps = synth.ParamSet("mul", logN, tuple(q), p, 45, 1, 1, -10)
+    o = Oracle(logN, q, p, 45, 1, 1)
+    km = synth.key_material(ps, 5, rots=[])
+    rlk = o.rlk_gen(km.s, synth.uniform_residues(5, 50, list(q) + [p], ps.N, lead=(L,)), synth.rounded_gaussian(5, 51, (L, ps.N)))
+    c = b.Context(ps)
+    c.load_keys(rlk[None], [0])
+    mods = np.array(q, dtype=np.uint64)[None, None, :, None]
+    x = synth.uniform_residues(6, 1, list(q), ps.N, lead=(count, 2)) % mods
+    y = synth.uniform_residues(6, 2, list(q), ps.N, lead=(count, 2)) % mods
+    xd, yd = c.import_(b.KIND_CT, x, count), c.import_(b.KIND_CT, y, count)
+    ws = c.workspace(3)
+    prod = c.multiply(xd, yd, count, ws)
+    got = c.export(b.KIND_CT, prod, count)
+    want = np.stack([o.relin(o.mac_ct(x[i][None], y[i][None])[0], rlk) for i in range(count)])
+    assert np.array_equal(got, want)
+    low = b.Context(synth.ParamSet("mul1", logN, tuple(q[:-1]), p, 45, 1, 1, -10))
+    res = c.rescale(prod, count, ws)
+    c.sync()
+    got_r = low.export(b.KIND_CT, res, count)
+    assert np.array_equal(got_r, np.stack([o.compact(want[i], L - 1, rescale=True) for i in range(count)]))
+    # error paths
+    lib = b.load_library()
+    assert lib.hann_multiply(c.h, b._ptr(xd), b._ptr(yd), -1, b._ptr(prod), b._ptr(ws), ws.numel() * 8) == b.EINVAL
+    assert lib.hann_multiply(c.h, b._ptr(xd), b._ptr(yd), count, b._ptr(prod), b._ptr(ws), 1024) == b.EWORKSPACE
+    nokey = b.Context(ps)
+    assert lib.hann_multiply(nokey.h, b._ptr(xd), b._ptr(yd), count, b._ptr(prod), b._ptr(ws), ws.numel() * 8) == b.ENOKEY

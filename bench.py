@@ -110,6 +110,8 @@ def bench_keys(ctx, ps, args):
         ctx.set_tuning(binding.TUNE_GIANT_LAZY, 1)
     if args.lazy_lanes:
         ctx.set_tuning(binding.TUNE_LAZY_LANES, args.lazy_lanes)
+    if args.mac_f64 is not None:
+        ctx.set_tuning(binding.TUNE_MAC_F64, args.mac_f64)
     km = synth.key_material(ps, wl.KEY_SEED, rots=rots)
     ctx.load_keys(ctx.keygen_from_samples(km.s, km.rots, km.evk_a, km.evk_e), km.rots)
     return km
@@ -1054,6 +1056,7 @@ def main():
     ap.add_argument("--project-sweep", default="1,2,4,8,16,32", help="baby-step counts of --project")
     ap.add_argument("--giant", default="lazy", choices=["horner", "lazy"],
                     help="evaluation order of the giant steps of the rotate-and-sum (the library's own default is Horner)")
+    ap.add_argument("--mac-f64", type=int, default=None, help="tuning: 1 (default): the multiply-accumulate sums on the FP64 pipe, 0: on the integer multiplier")
     ap.add_argument("--lazy-lanes", type=int, default=None, help="tuning: block ranges the lazy rotate-and-sum runs side by side (1..4)")
     ap.add_argument("--baby", type=int, default=None, help="baby-step count B (default: the configuration's; must divide R)")
     ap.add_argument("--rows", type=int, default=None, help="override the row count (debugging, ncu captures)")

@@ -146,9 +146,11 @@ int hann_get_stats(hann_ctx *ctx, hann_stats *out);
  * HANN_TUNE_GIANT_LAZY (this one changes the result's BITS, not its meaning): 1 makes hann_rotate_sum, and with it
  * hann_query_level and hann_score_level_host, evaluate the giant steps in the order of hann_rotate_sum_lazy (the keys of
  * rotations 2B .. (G-1)B must then be loaded as well); 0 (default) is Horner with the single key of rotation B.
- * HANN_TUNE_LAZY_LANES: block ranges (1..4, default 2) hann_rotate_sum_lazy runs side by side on helper streams. */
+ * HANN_TUNE_LAZY_LANES: block ranges (1..4, default 2) hann_rotate_sum_lazy runs side by side on helper streams.
+ * HANN_TUNE_MAC_F64: 1 (default) lets the single-query multiply-accumulate of chains of primes below 2^50 sum its products
+ * exactly in pairs of binary64 words on the FP64 pipe, 0 on the integer multiplier; same residues either way. */
 enum { HANN_TUNE_ENCODE_GROUP = 1, HANN_TUNE_HOST_LIMBS = 2, HANN_TUNE_ENCODE_SYMMETRY = 3, HANN_TUNE_HOST_GROUPS = 4, HANN_TUNE_GIANT_LAZY = 5,
-       HANN_TUNE_LAZY_LANES = 6 };
+       HANN_TUNE_LAZY_LANES = 6, HANN_TUNE_MAC_F64 = 7 };
 int hann_set_tuning(hann_ctx *ctx, int what, int value);
 
 /* Per-launch profile: while enabled every kernel launch of the context is bracketed by a CUDA event pair (this

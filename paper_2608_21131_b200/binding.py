@@ -25,6 +25,7 @@ TUNE_ENCODE_SYMMETRY = 3
 TUNE_HOST_GROUPS = 4
 TUNE_GIANT_LAZY = 5
 TUNE_LAZY_LANES = 6
+TUNE_MAC_F64 = 7
 
 
 class HannError(RuntimeError):

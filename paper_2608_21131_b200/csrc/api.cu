@@ -575,6 +575,9 @@ extern "C" int hann_set_tuning(hann_ctx* c, int what, int value) {
             if (value < 1 || value > 4) return fail(c, HANN_EINVAL, "hann_set_tuning: lazy lanes must be 1..4");
             c->lazy_lanes = value;
             return HANN_OK;
+        case HANN_TUNE_MAC_F64:
+            c->mac_f64 = value ? 4 : 0;
+            return HANN_OK;
         default: return fail(c, HANN_EINVAL, "hann_set_tuning: unknown knob");
     }
 }

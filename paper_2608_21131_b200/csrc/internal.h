@@ -79,6 +79,7 @@ struct hann_ctx {
     // debugging aid: guards behind every workspace sub-buffer (see Arena in api.cu), filled when carved, checked on request
     int canaries = 0;
     std::vector<u64*> guards;
+    int mac_f64 = 4;     // how many of a thread's four sums the single-query multiply-accumulate keeps on the FP64 pipe
     int lazy_lanes = 2;  // block ranges hann_rotate_sum_lazy runs side by side
     int giant_lazy = 0;  // hann_rotate_sum (and the calls built on it) evaluates the giant steps in the lazy order
     int encode_sym = 1;  // encode_candidates computes half of every transform and mirrors it (real slot vectors)

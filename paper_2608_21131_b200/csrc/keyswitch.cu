@@ -94,10 +94,17 @@ __device__ __forceinline__ void ks_inner_body(const u64* __restrict__ digits, lo
         for (int k = 0; k < NST; k++) st[k] = key[(long long)k * L1N + pos];  // k = j*2 + comp
     }
     unsigned s0[NST], s1[NST];
+    double sd[NST];  // MODE 3: the stationary words as balanced binary64 integers
+    constexpr double kTwo52 = 4503599627370496.0, kBig = 0x1.8p103;
 #pragma unroll
     for (int k = 0; k < NST; k++) {
-        s0[k] = (unsigned)st[k] & MASK;
-        s1[k] = (unsigned)(st[k] >> SH);
+        if (MODE == 3) {
+            const double d = __dsub_rn(__longlong_as_double((long long)(st[k] | 0x4330000000000000ULL)), kTwo52);
+            sd[k] = d > (double)lc.half ? __dsub_rn(d, (double)lc.q) : d;
+        } else {
+            s0[k] = (unsigned)st[k] & MASK;
+            s1[k] = (unsigned)(st[k] >> SH);
+        }
     }
     u64 cur[NS], nxt[NS];
     auto load = [&](long long item, u64(&v)[NS]) {
@@ -115,7 +122,38 @@ __device__ __forceinline__ void ks_inner_body(const u64* __restrict__ digits, lo
     for (long long item = it0; item < it1; item++) {
         if (item + 1 < it1) load(item + 1, nxt);
         u64 out[2];
-        if (MODE != 2) {
+        if (MODE == 3) {
+            // moduli below 2^50, at most eight digits: the products summed exactly in two binary64 words per component on the
+            // FP64 pipe.  AH starts at 1.5 * 2^103 and so always rounds to a multiple of 2^51 (|stationary| < 2^49, streamed
+            // < 2^50: the sum stays below 2^102, inside the binade); what a rounding drops is an integer of at most 2^50,
+            // recovered exactly by a second multiply-add and summed in AL.
+            static_assert(MODE != 3 || LL <= 8, "the two-word binary64 sum holds eight products");
+            double ah[2] = {kBig, kBig}, al[2] = {0, 0};
+#pragma unroll
+            for (int j = 0; j < LL; j++)
+#pragma unroll
+                for (int c = 0; c < 2; c++) {
+                    const int ks = KEYS_STREAM ? j : 2 * j + c;
+                    const u64 sv = KEYS_STREAM ? cur[2 * j + c] : cur[j];
+                    const double b = __dsub_rn(__longlong_as_double((long long)(sv | 0x4330000000000000ULL)), kTwo52);
+                    const double nh = __fma_rn(b, sd[ks], ah[c]);
+                    al[c] = __dadd_rn(al[c], __fma_rn(b, sd[ks], __dsub_rn(ah[c], nh)));
+                    ah[c] = nh;
+                }
+#pragma unroll
+            for (int c = 0; c < 2; c++) {
+                // m 2^51 + sl + q 2^57 as an unsigned 128-bit integer (|sum| < 4 q^2 < q 2^57 for every q below 2^50)
+                const long long m = __double2ll_rn(__dmul_rn(__dsub_rn(ah[c], kBig), 0x1p-51)), sl = __double2ll_rn(al[c]);
+                u64 lo = (u64)m << 51, hi = (u64)(m >> 13);
+                const u64 s_lo = (u64)sl, s_hi = (u64)(sl >> 63);
+                lo += s_lo;
+                hi += s_hi + (lo < s_lo ? 1 : 0);
+                const u64 o_lo = lc.q << 57, o_hi = lc.q >> 7;
+                lo += o_lo;
+                hi += o_hi + (lo < o_lo ? 1 : 0);
+                out[c] = reduce128(hi, lo, lc);
+            }
+        } else if (MODE != 2) {
             u64 p00[2] = {0, 0}, p11[2] = {0, 0}, pm[2] = {0, 0};
 #pragma unroll
             for (int j = 0; j < LL; j++)
@@ -169,7 +207,7 @@ template <int LL, bool KEYS_STREAM>
 __global__ void __launch_bounds__(128) k_ks_inner_stream(const u64* __restrict__ digits, long long digit_stride,
                                                          const u64* const* __restrict__ keytab, int rot0, int rot_inc,
                                                          u64* __restrict__ u, int N, long long nitems, int items_per_cta,
-                                                         const LimbConst* __restrict__ lt, int rot_zinc) {
+                                                         const LimbConst* __restrict__ lt, int rot_zinc, int f64) {
     const long long L1N = (long long)(LL + 1) * N;
     const long long pos = (long long)blockIdx.x * 128 + threadIdx.x;  // i*N + x
     const LimbConst lc = lt[pos / N];
@@ -180,7 +218,8 @@ __global__ void __launch_bounds__(128) k_ks_inner_stream(const u64* __restrict__
     const long long it1 = it0 + items_per_cta < nitems ? it0 + items_per_cta : nitems;
     if (it0 >= it1) return;
     // a CTA lies inside one limb, so the choice is uniform
-    if (lc.q < (1ULL << 50)) ks_inner_body<LL, KEYS_STREAM, 0>(digits, digit_stride, keytab, rot0, rot_inc, u, L1N, pos, it0, it1, lc);
+    if (lc.q < (1ULL << 50) && f64) ks_inner_body<LL, KEYS_STREAM, 3>(digits, digit_stride, keytab, rot0, rot_inc, u, L1N, pos, it0, it1, lc);
+    else if (lc.q < (1ULL << 50)) ks_inner_body<LL, KEYS_STREAM, 0>(digits, digit_stride, keytab, rot0, rot_inc, u, L1N, pos, it0, it1, lc);
     else if (lc.q < (1ULL << 60)) ks_inner_body<LL, KEYS_STREAM, 1>(digits, digit_stride, keytab, rot0, rot_inc, u, L1N, pos, it0, it1, lc);
     else ks_inner_body<LL, KEYS_STREAM, 2>(digits, digit_stride, keytab, rot0, rot_inc, u, L1N, pos, it0, it1, lc);
 }
@@ -614,10 +653,10 @@ void launch_ks_inner_stream(hann_ctx* c, const u64* digits, int64_t digit_stride
     KProf kp(c, digit_stride == 0 && nitems > 1 ? KC_KS_INNER_KEYS : KC_KS_INNER);  // streamed keys timed on their own
     if (digit_stride == 0)
         k_ks_inner_stream<LL, true><<<dim3(tiles, split, nz), 128, 0, c->stream>>>(digits, 0, c->keytab_dev, rot0, rot_inc, u, c->N, nitems,
-                                                                                per, c->lt_dev, rot_zinc);
+                                                                                per, c->lt_dev, rot_zinc, c->mac_f64);
     else
         k_ks_inner_stream<LL, false><<<dim3(tiles, split, nz), 128, 0, c->stream>>>(digits, digit_stride, c->keytab_dev, rot0, rot_inc, u,
-                                                                                 c->N, nitems, per, c->lt_dev, rot_zinc);
+                                                                                 c->N, nitems, per, c->lt_dev, rot_zinc, c->mac_f64);
 }
 
 int launch_ks_inner(hann_ctx* c, const u64* digits, int64_t digit_stride, int rot0, int rot_inc, int64_t nitems, u64* u) {

@@ -247,20 +247,31 @@ __global__ void __launch_bounds__(32 * NG) k_mac_ct_stream(const u64* __restrict
 // context's kernel flag and lets the whole CTA leave at its next barrier.
 constexpr int kMacStages = 4;
 
-template <int NG, int BB>
+// partial sums per thread that cross the warps: four sums of three words (integer multiplier) or of two (FP64 pipe)
+template <int NG, int BB, int F64>
 constexpr size_t mac_bulk_smem() {
-    return (size_t)NG * kMacStages * BB * 256 + (size_t)2 * NG * 12 * 256 + (size_t)NG * kMacStages * 8 + 16;
+    return (size_t)NG * kMacStages * BB * 256 + (size_t)2 * NG * (F64 == 4 ? 8 : 12) * 256 + (size_t)NG * kMacStages * 8 + 16;
 }
 
-template <int NG, int BB>
+// Sums on the FP64 pipe instead of the integer multiplier: a baby-step word is lifted to a balanced
+// binary64 integer a (|a| < 2^49), a plaintext word to p in [0, 2^50); every product enters a two-word sum (AH, AL) exactly:
+//   AH starts at 1.5 * 2^103, so every AH = fma(p, a, AH) rounds to a multiple of 2^51 (the sum of at most eight products
+//   stays below 2^102 in magnitude: AH never leaves its binade); the part the rounding dropped, p a + (AH_old - AH_new), is
+//   an integer of at most 2^50 in magnitude that a second fma yields exactly; eight of them sum exactly in AL (<= 2^53).
+// Four FP64 operations per product against three wide integer multiply-adds and their additions, on a pipe with more than
+// twice the throughput; the result is the same integer, hence the same residue.
+// F64 = 1..4: that many of the four sums of a thread (side x component) run on the FP64 pipe, the rest on the integer
+// multiplier, so that both pipes work side by side; 0: all on the integer multiplier.
+template <int NG, int BB, int F64>
 __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ baby, const __grid_constant__ CUtensorMap pt_map,
                                                       u64* __restrict__ inner, int N, int L, long long n_bg, int bg_per_cta,
                                                       const LimbConst* __restrict__ lt, int* kflag) {
     constexpr int B = NG * BB;
     extern __shared__ __align__(128) u64 smem_mac[];
     u64(*ring)[kMacStages][BB][32] = (u64(*)[kMacStages][BB][32])smem_mac;                        // [NG]
-    u64(*part)[NG][12][32] = (u64(*)[NG][12][32])(smem_mac + (size_t)NG * kMacStages * BB * 32);  // [2]
-    u64(*bars)[kMacStages] = (u64(*)[kMacStages])(smem_mac + (size_t)NG * kMacStages * BB * 32 + (size_t)2 * NG * 12 * 32);  // [NG]
+    constexpr int PS = F64 == 4 ? 2 : 3, PW = 4 * PS;  // words per partial sum, per thread
+    u64(*part)[NG][PW][32] = (u64(*)[NG][PW][32])(smem_mac + (size_t)NG * kMacStages * BB * 32);  // [2]
+    u64(*bars)[kMacStages] = (u64(*)[kMacStages])(smem_mac + (size_t)NG * kMacStages * BB * 32 + (size_t)2 * NG * PW * 32);  // [NG]
     int& s_abort = *(int*)(&bars[NG][0]);
     const int n = N >> 1;
     const long long LN = (long long)L * N;
@@ -285,8 +296,13 @@ __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ ba
             tensor_load_2d(ring0 + i * BB * 256, &pt_map, (int)hpos0, row0 + i * B, bar0 + 8 * i);
         }
     }
-    // this warp's baby-step words of both sides, split into 25-bit halves
+    // this warp's baby-step words of both sides: split into 25-bit halves (sums on the integer multiplier), or as balanced
+    // binary64 integers (sums on the FP64 pipe); sum number v * 2 + c is of the second kind if it is below F64
+    static_assert(F64 == 0 || BB <= 8, "the two-word binary64 sum holds eight products");
+    constexpr double kTwo52 = 4503599627370496.0, kBig = 0x1.8p103;
     unsigned w0[2][BB][2], w1[2][BB][2];
+    double wd[2][BB][2];
+    const double qd = (double)lc->q, halfd = (double)lc->half;
 #pragma unroll
     for (int v = 0; v < 2; v++)
 #pragma unroll
@@ -294,8 +310,13 @@ __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ ba
 #pragma unroll
             for (int c = 0; c < 2; c++) {
                 const u64 x = baby[((long long)(wg * BB + k) * 2 + c) * LN + posv[v]];
-                w0[v][k][c] = (unsigned)x & kM25;
-                w1[v][k][c] = (unsigned)(x >> 25);
+                if (v * 2 + c < F64) {
+                    const double d = __dsub_rn(__longlong_as_double((long long)(x | 0x4330000000000000ULL)), kTwo52);
+                    wd[v][k][c] = d > halfd ? __dsub_rn(d, qd) : d;
+                } else {
+                    w0[v][k][c] = (unsigned)x & kM25;
+                    w1[v][k][c] = (unsigned)(x >> 25);
+                }
             }
     __syncthreads();  // s_abort and the barriers are initialised
     for (int i = 0; i < npairs; i++) {
@@ -315,27 +336,41 @@ __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ ba
             mbar_expect_tx(bar0 + 8 * st, BB * 256);
             tensor_load_2d(ring0 + st * BB * 256, &pt_map, (int)hpos0, row0 + (i + kMacStages) * B, bar0 + 8 * st);
         }
+        u64(*buf)[PW][32] = part[i & 1];
+        double ah[2][2] = {{kBig, kBig}, {kBig, kBig}}, al[2][2] = {{0, 0}, {0, 0}};
         u64 p00[2][2] = {{0, 0}, {0, 0}}, p11[2][2] = {{0, 0}, {0, 0}}, pm[2][2] = {{0, 0}, {0, 0}};
 #pragma unroll
         for (int k = 0; k < BB; k++) {
+            const double p = __dsub_rn(__longlong_as_double((long long)(cur[k] | 0x4330000000000000ULL)), kTwo52);
             const unsigned a0 = (unsigned)cur[k] & kM25, a1 = (unsigned)(cur[k] >> 25), as = a0 + a1;
 #pragma unroll
             for (int v = 0; v < 2; v++)
 #pragma unroll
                 for (int c = 0; c < 2; c++) {
-                    p00[v][c] += (u64)a0 * w0[v][k][c];
-                    p11[v][c] += (u64)a1 * w1[v][k][c];
-                    pm[v][c] += (u64)as * (w0[v][k][c] + w1[v][k][c]);
+                    if (v * 2 + c < F64) {
+                        const double nh = __fma_rn(p, wd[v][k][c], ah[v][c]);
+                        al[v][c] = __dadd_rn(al[v][c], __fma_rn(p, wd[v][k][c], __dsub_rn(ah[v][c], nh)));
+                        ah[v][c] = nh;
+                    } else {
+                        p00[v][c] += (u64)a0 * w0[v][k][c];
+                        p11[v][c] += (u64)a1 * w1[v][k][c];
+                        pm[v][c] += (u64)as * (w0[v][k][c] + w1[v][k][c]);
+                    }
                 }
         }
-        u64(*buf)[12][32] = part[i & 1];
 #pragma unroll
         for (int v = 0; v < 2; v++)
 #pragma unroll
             for (int c = 0; c < 2; c++) {
-                buf[wg][(v * 2 + c) * 3 + 0][lane] = p00[v][c];
-                buf[wg][(v * 2 + c) * 3 + 1][lane] = pm[v][c];
-                buf[wg][(v * 2 + c) * 3 + 2][lane] = p11[v][c];
+                if (v * 2 + c < F64) {
+                    // high word as a count of 2^51 (below 2^51 in magnitude), low word as it is
+                    buf[wg][(v * 2 + c) * PS + 0][lane] = (u64)__double2ll_rn(__dmul_rn(__dsub_rn(ah[v][c], kBig), 0x1p-51));
+                    buf[wg][(v * 2 + c) * PS + 1][lane] = (u64)__double2ll_rn(al[v][c]);
+                } else {
+                    buf[wg][(v * 2 + c) * PS + 0][lane] = p00[v][c];
+                    buf[wg][(v * 2 + c) * PS + 1][lane] = pm[v][c];
+                    buf[wg][(v * 2 + c) * PS + 2][lane] = p11[v][c];
+                }
             }
         __syncthreads();
         if (s_abort) {
@@ -344,21 +379,40 @@ __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ ba
             return;
         }
         for (int vc = wg; vc < 4; vc += NG) {
-            u64 s00 = 0, sm = 0, s11 = 0;
+            u64 lo, hi;
+            if (vc < F64) {
+                long long m = 0, sl = 0;
 #pragma unroll
-            for (int g = 0; g < NG; g++) {
-                s00 += buf[g][vc * 3 + 0][lane];
-                sm += buf[g][vc * 3 + 1][lane];
-                s11 += buf[g][vc * 3 + 2][lane];
+                for (int g = 0; g < NG; g++) {
+                    m += (long long)buf[g][vc * PS + 0][lane];
+                    sl += (long long)buf[g][vc * PS + 1][lane];
+                }
+                // m 2^51 + sl + q 2^57 as an unsigned 128-bit integer: |sum| < 32 q^2 (at most 64 products) < q 2^57
+                lo = (u64)m << 51;
+                hi = (u64)(m >> 13);
+                const u64 s_lo = (u64)sl, s_hi = (u64)(sl >> 63);
+                lo += s_lo;
+                hi += s_hi + (lo < s_lo ? 1 : 0);
+                const u64 o_lo = lc->q << 57, o_hi = lc->q >> 7;
+                lo += o_lo;
+                hi += o_hi + (lo < o_lo ? 1 : 0);
+            } else {
+                u64 s00 = 0, sm = 0, s11 = 0;
+#pragma unroll
+                for (int g = 0; g < NG; g++) {
+                    s00 += buf[g][vc * PS + 0][lane];
+                    sm += buf[g][vc * PS + 1][lane];
+                    s11 += buf[g][vc * PS + 2][lane];
+                }
+                const u64 cross = sm - s00 - s11;
+                lo = s00, hi = 0;
+                const u64 c_lo = cross << 25, c_hi = cross >> 39;
+                lo += c_lo;
+                hi += c_hi + (lo < c_lo ? 1 : 0);
+                const u64 d_lo = s11 << 50, d_hi = s11 >> 14;
+                lo += d_lo;
+                hi += d_hi + (lo < d_lo ? 1 : 0);
             }
-            const u64 cross = sm - s00 - s11;
-            u64 lo = s00, hi = 0;
-            const u64 c_lo = cross << 25, c_hi = cross >> 39;
-            lo += c_lo;
-            hi += c_hi + (lo < c_lo ? 1 : 0);
-            const u64 d_lo = s11 << 50, d_hi = s11 >> 14;
-            lo += d_lo;
-            hi += d_hi + (lo < d_lo ? 1 : 0);
             inner[((bg0 + i) * 2 + (vc & 1)) * LN + posv[vc >> 1]] = reduce128(hi, lo, *lc);
         }
         if (NG < 4) __syncthreads();
@@ -435,9 +489,14 @@ void launch_mac_stream(hann_ctx* c, const u64* baby, int64_t baby_stride, const 
     if constexpr (NQ == 1 && NG * BB <= 32) {
         CUtensorMap map;
         if (((uintptr_t)pt & 15) == 0 && n_bg * (NG * BB) < (1LL << 31) && plaintext_map(pt, Ln, n_bg * (NG * BB), BB, &map)) {
-            constexpr size_t smem = mac_bulk_smem<NG, BB>();
-            if (smem > 48 * 1024) cudaFuncSetAttribute(k_mac_bulk<NG, BB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-            k_mac_bulk<NG, BB><<<dim3(tiles, split), 32 * NG, smem, c->stream>>>(baby, map, inner, c->N, c->L, n_bg, per, c->lt_dev, c->kflag);
+            auto go = [&](auto kern, size_t smem) {
+                if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                kern<<<dim3(tiles, split), 32 * NG, smem, c->stream>>>(baby, map, inner, c->N, c->L, n_bg, per, c->lt_dev, c->kflag);
+            };
+            switch (c->mac_f64) {
+                case 0: go(k_mac_bulk<NG, BB, 0>, mac_bulk_smem<NG, BB, 0>()); break;
+                default: go(k_mac_bulk<NG, BB, 4>, mac_bulk_smem<NG, BB, 4>()); break;
+            }
             return;
         }
     }

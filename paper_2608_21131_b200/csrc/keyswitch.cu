@@ -95,12 +95,10 @@ __device__ __forceinline__ void ks_inner_body(const u64* __restrict__ digits, lo
     }
     unsigned s0[NST], s1[NST];
     double sd[NST];  // MODE 3: the stationary words as balanced binary64 integers
-    constexpr double kTwo52 = 4503599627370496.0, kBig = 0x1.8p103;
 #pragma unroll
     for (int k = 0; k < NST; k++) {
         if (MODE == 3) {
-            const double d = __dsub_rn(__longlong_as_double((long long)(st[k] | 0x4330000000000000ULL)), kTwo52);
-            sd[k] = d > (double)lc.half ? __dsub_rn(d, (double)lc.q) : d;
+            sd[k] = residue_to_balanced_f64(st[k], (double)lc.q, (double)lc.half);
         } else {
             s0[k] = (unsigned)st[k] & MASK;
             s1[k] = (unsigned)(st[k] >> SH);
@@ -124,35 +122,16 @@ __device__ __forceinline__ void ks_inner_body(const u64* __restrict__ digits, lo
         u64 out[2];
         if (MODE == 3) {
             // moduli below 2^50, at most eight digits: the products summed exactly in two binary64 words per component on the
-            // FP64 pipe.  AH starts at 1.5 * 2^103 and so always rounds to a multiple of 2^51 (|stationary| < 2^49, streamed
-            // < 2^50: the sum stays below 2^102, inside the binade); what a rounding drops is an integer of at most 2^50,
-            // recovered exactly by a second multiply-add and summed in AL.
+            // FP64 pipe (acc2_fma), the integer pipe keeps only the final reduction
             static_assert(MODE != 3 || LL <= 8, "the two-word binary64 sum holds eight products");
-            double ah[2] = {kBig, kBig}, al[2] = {0, 0};
+            double ah[2] = {kAcc2Start, kAcc2Start}, al[2] = {0, 0};
 #pragma unroll
             for (int j = 0; j < LL; j++)
 #pragma unroll
-                for (int c = 0; c < 2; c++) {
-                    const int ks = KEYS_STREAM ? j : 2 * j + c;
-                    const u64 sv = KEYS_STREAM ? cur[2 * j + c] : cur[j];
-                    const double b = __dsub_rn(__longlong_as_double((long long)(sv | 0x4330000000000000ULL)), kTwo52);
-                    const double nh = __fma_rn(b, sd[ks], ah[c]);
-                    al[c] = __dadd_rn(al[c], __fma_rn(b, sd[ks], __dsub_rn(ah[c], nh)));
-                    ah[c] = nh;
-                }
+                for (int c = 0; c < 2; c++)
+                    acc2_fma(ah[c], al[c], residue_to_f64(KEYS_STREAM ? cur[2 * j + c] : cur[j]), sd[KEYS_STREAM ? j : 2 * j + c]);
 #pragma unroll
-            for (int c = 0; c < 2; c++) {
-                // m 2^51 + sl + q 2^57 as an unsigned 128-bit integer (|sum| < 4 q^2 < q 2^57 for every q below 2^50)
-                const long long m = __double2ll_rn(__dmul_rn(__dsub_rn(ah[c], kBig), 0x1p-51)), sl = __double2ll_rn(al[c]);
-                u64 lo = (u64)m << 51, hi = (u64)(m >> 13);
-                const u64 s_lo = (u64)sl, s_hi = (u64)(sl >> 63);
-                lo += s_lo;
-                hi += s_hi + (lo < s_lo ? 1 : 0);
-                const u64 o_lo = lc.q << 57, o_hi = lc.q >> 7;
-                lo += o_lo;
-                hi += o_hi + (lo < o_lo ? 1 : 0);
-                out[c] = reduce128(hi, lo, lc);
-            }
+            for (int c = 0; c < 2; c++) out[c] = acc2_reduce(acc2_high(ah[c]), acc2_low(al[c]), lc);
         } else if (MODE != 2) {
             u64 p00[2] = {0, 0}, p11[2] = {0, 0}, pm[2] = {0, 0};
 #pragma unroll

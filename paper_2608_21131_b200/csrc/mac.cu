@@ -56,14 +56,16 @@ constexpr unsigned kM25 = (1u << 25) - 1;
 // NQ queries at once (cross-query batching against the same encoded candidates): the warp keeps the baby-step words of NQ
 // baby sets (query q at baby + q * baby_stride) and every plaintext word, still read once, feeds NQ times the products;
 // partial sums of query q go to inner + q * inner_stride.
-template <int NG, int BB, int NQ>
+template <int NG, int BB, int NQ, int F64>
 __global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ baby, long long baby_stride,
                                                         const u64* __restrict__ pt, u64* __restrict__ inner,
                                                         long long inner_stride, int N, int L, long long n_bg, int bg_per_cta,
                                                         const LimbConst* __restrict__ lt) {
     constexpr int B = NG * BB;
     constexpr int NV = 2 * NQ;  // (query, side): side 0 is position t, side 1 its mirror image N - 1 - t
-    __shared__ u64 part[2][NG][3 * 2 * NV][32];
+    constexpr int PS = F64 ? 2 : 3;  // words per partial sum: (high, low) of the binary64 sums, or the three Karatsuba sums
+    static_assert(F64 == 0 || BB <= 8, "the two-word binary64 sum holds eight products");
+    __shared__ u64 part[2][NG][PS * 2 * NV][32];
     const int n = N >> 1;
     const long long LN = (long long)L * N, Ln = (long long)L * n;
     const long long hpos0 = (long long)blockIdx.x * 32;  // in the stored plaintext layout [L][N/2]
@@ -71,8 +73,10 @@ __global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ 
     const int limb = (int)(hpos0 / n), t0 = (int)(hpos0 % n);
     const LimbConst* lc = lt + limb;
     const long long posv[2] = {(long long)limb * N + t0 + lane, (long long)limb * N + (N - 1 - t0 - lane)};
-    // this warp's baby-step words, split into 25-bit halves
+    // this warp's baby-step words, split into 25-bit halves or (F64) as balanced binary64 integers
     unsigned w0[NV][BB][2], w1[NV][BB][2];
+    double wd[NV][BB][2];
+    const double qd = (double)lc->q, halfd = (double)lc->half;
 #pragma unroll
     for (int v = 0; v < NV; v++)
 #pragma unroll
@@ -80,8 +84,12 @@ __global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ 
 #pragma unroll
             for (int c = 0; c < 2; c++) {
                 const u64 x = baby[(v >> 1) * baby_stride + ((long long)(wg * BB + k) * 2 + c) * LN + posv[v & 1]];
-                w0[v][k][c] = (unsigned)x & kM25;
-                w1[v][k][c] = (unsigned)(x >> 25);
+                if (F64) {
+                    wd[v][k][c] = residue_to_balanced_f64(x, qd, halfd);
+                } else {
+                    w0[v][k][c] = (unsigned)x & kM25;
+                    w1[v][k][c] = (unsigned)(x >> 25);
+                }
             }
     const long long bg0 = (long long)blockIdx.y * bg_per_cta;
     const long long bg1 = bg0 + bg_per_cta < n_bg ? bg0 + bg_per_cta : n_bg;
@@ -96,53 +104,88 @@ __global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ 
 #pragma unroll
             for (int k = 0; k < BB; k++) nxt[k] = __ldcs(pn + (long long)k * Ln);
         }
-        u64 p00[NV][2], p11[NV][2], pm[NV][2];
+        u64(*buf)[PS * 2 * NV][32] = part[bg & 1];
+        if (F64) {
+            double ah[NV][2], al[NV][2];
 #pragma unroll
-        for (int v = 0; v < NV; v++)
+            for (int v = 0; v < NV; v++)
 #pragma unroll
-            for (int c = 0; c < 2; c++) p00[v][c] = p11[v][c] = pm[v][c] = 0;
+                for (int c = 0; c < 2; c++) ah[v][c] = kAcc2Start, al[v][c] = 0;
 #pragma unroll
-        for (int k = 0; k < BB; k++) {
-            const unsigned a0 = (unsigned)cur[k] & kM25, a1 = (unsigned)(cur[k] >> 25), as = a0 + a1;
+            for (int k = 0; k < BB; k++) {
+                const double pd = residue_to_f64(cur[k]);
+#pragma unroll
+                for (int v = 0; v < NV; v++)
+#pragma unroll
+                    for (int c = 0; c < 2; c++) acc2_fma(ah[v][c], al[v][c], pd, wd[v][k][c]);
+            }
 #pragma unroll
             for (int v = 0; v < NV; v++)
 #pragma unroll
                 for (int c = 0; c < 2; c++) {
-                    p00[v][c] += (u64)a0 * w0[v][k][c];
-                    p11[v][c] += (u64)a1 * w1[v][k][c];
-                    pm[v][c] += (u64)as * (w0[v][k][c] + w1[v][k][c]);
+                    buf[wg][(v * 2 + c) * PS + 0][lane] = (u64)acc2_high(ah[v][c]);
+                    buf[wg][(v * 2 + c) * PS + 1][lane] = (u64)acc2_low(al[v][c]);
+                }
+        } else {
+            u64 p00[NV][2], p11[NV][2], pm[NV][2];
+#pragma unroll
+            for (int v = 0; v < NV; v++)
+#pragma unroll
+                for (int c = 0; c < 2; c++) p00[v][c] = p11[v][c] = pm[v][c] = 0;
+#pragma unroll
+            for (int k = 0; k < BB; k++) {
+                const unsigned a0 = (unsigned)cur[k] & kM25, a1 = (unsigned)(cur[k] >> 25), as = a0 + a1;
+#pragma unroll
+                for (int v = 0; v < NV; v++)
+#pragma unroll
+                    for (int c = 0; c < 2; c++) {
+                        p00[v][c] += (u64)a0 * w0[v][k][c];
+                        p11[v][c] += (u64)a1 * w1[v][k][c];
+                        pm[v][c] += (u64)as * (w0[v][k][c] + w1[v][k][c]);
+                    }
+            }
+#pragma unroll
+            for (int v = 0; v < NV; v++)
+#pragma unroll
+                for (int c = 0; c < 2; c++) {
+                    buf[wg][(v * 2 + c) * PS + 0][lane] = p00[v][c];
+                    buf[wg][(v * 2 + c) * PS + 1][lane] = pm[v][c];
+                    buf[wg][(v * 2 + c) * PS + 2][lane] = p11[v][c];
                 }
         }
-        u64(*buf)[3 * 2 * NV][32] = part[bg & 1];
-#pragma unroll
-        for (int v = 0; v < NV; v++)
-#pragma unroll
-            for (int c = 0; c < 2; c++) {
-                buf[wg][(v * 2 + c) * 3 + 0][lane] = p00[v][c];
-                buf[wg][(v * 2 + c) * 3 + 1][lane] = pm[v][c];
-                buf[wg][(v * 2 + c) * 3 + 2][lane] = p11[v][c];
-            }
         __syncthreads();
         // the warps share out the 2 * NV (query, side, component) sums
         for (int vc = wg; vc < 2 * NV; vc += NG) {
-            u64 s00 = 0, sm = 0, s11 = 0;
+            u64 r;
+            if (F64) {
+                long long m = 0, sl = 0;
 #pragma unroll
-            for (int g = 0; g < NG; g++) {
-                s00 += buf[g][vc * 3 + 0][lane];
-                sm += buf[g][vc * 3 + 1][lane];
-                s11 += buf[g][vc * 3 + 2][lane];
+                for (int g = 0; g < NG; g++) {
+                    m += (long long)buf[g][vc * PS + 0][lane];
+                    sl += (long long)buf[g][vc * PS + 1][lane];
+                }
+                r = acc2_reduce(m, sl, *lc);
+            } else {
+                u64 s00 = 0, sm = 0, s11 = 0;
+#pragma unroll
+                for (int g = 0; g < NG; g++) {
+                    s00 += buf[g][vc * PS + 0][lane];
+                    sm += buf[g][vc * PS + 1][lane];
+                    s11 += buf[g][vc * PS + 2][lane];
+                }
+                // value = s00 + cross * 2^25 + s11 * 2^50 with cross = sm - s00 - s11 < 2^59
+                const u64 cross = sm - s00 - s11;
+                u64 lo = s00, hi = 0;
+                const u64 c_lo = cross << 25, c_hi = cross >> 39;
+                lo += c_lo;
+                hi += c_hi + (lo < c_lo ? 1 : 0);
+                const u64 d_lo = s11 << 50, d_hi = s11 >> 14;
+                lo += d_lo;
+                hi += d_hi + (lo < d_lo ? 1 : 0);
+                r = reduce128(hi, lo, *lc);
             }
-            // value = s00 + cross * 2^25 + s11 * 2^50 with cross = sm - s00 - s11 < 2^59
-            const u64 cross = sm - s00 - s11;
-            u64 lo = s00, hi = 0;
-            const u64 c_lo = cross << 25, c_hi = cross >> 39;
-            lo += c_lo;
-            hi += c_hi + (lo < c_lo ? 1 : 0);
-            const u64 d_lo = s11 << 50, d_hi = s11 >> 14;
-            lo += d_lo;
-            hi += d_hi + (lo < d_lo ? 1 : 0);
             const int v = vc >> 1;
-            inner[(v >> 1) * inner_stride + (bg * 2 + (vc & 1)) * LN + posv[v & 1]] = reduce128(hi, lo, *lc);
+            inner[(v >> 1) * inner_stride + (bg * 2 + (vc & 1)) * LN + posv[v & 1]] = r;
         }
         if (NG < 2 * NV) __syncthreads();  // a warp that finishes several sums may still be reading while the next pair is written
 #pragma unroll
@@ -250,18 +293,12 @@ constexpr int kMacStages = 4;
 // partial sums per thread that cross the warps: four sums of three words (integer multiplier) or of two (FP64 pipe)
 template <int NG, int BB, int F64>
 constexpr size_t mac_bulk_smem() {
-    return (size_t)NG * kMacStages * BB * 256 + (size_t)2 * NG * (F64 == 4 ? 8 : 12) * 256 + (size_t)NG * kMacStages * 8 + 16;
+    return (size_t)NG * kMacStages * BB * 256 + (size_t)2 * NG * (F64 ? 8 : 12) * 256 + (size_t)NG * kMacStages * 8 + 16;
 }
 
-// Sums on the FP64 pipe instead of the integer multiplier: a baby-step word is lifted to a balanced
-// binary64 integer a (|a| < 2^49), a plaintext word to p in [0, 2^50); every product enters a two-word sum (AH, AL) exactly:
-//   AH starts at 1.5 * 2^103, so every AH = fma(p, a, AH) rounds to a multiple of 2^51 (the sum of at most eight products
-//   stays below 2^102 in magnitude: AH never leaves its binade); the part the rounding dropped, p a + (AH_old - AH_new), is
-//   an integer of at most 2^50 in magnitude that a second fma yields exactly; eight of them sum exactly in AL (<= 2^53).
-// Four FP64 operations per product against three wide integer multiply-adds and their additions, on a pipe with more than
-// twice the throughput; the result is the same integer, hence the same residue.
-// F64 = 1..4: that many of the four sums of a thread (side x component) run on the FP64 pipe, the rest on the integer
-// multiplier, so that both pipes work side by side; 0: all on the integer multiplier.
+// F64 != 0: the products are summed exactly in pairs of binary64 words on the FP64 pipe (acc2_fma: four operations per
+// product on a pipe of more than twice the multiplier's throughput, and two words of partial sum per thread instead of
+// three); 0: on the integer multiplier as in k_mac_stream.  Same integers either way, hence the same residues.
 template <int NG, int BB, int F64>
 __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ baby, const __grid_constant__ CUtensorMap pt_map,
                                                       u64* __restrict__ inner, int N, int L, long long n_bg, int bg_per_cta,
@@ -269,7 +306,7 @@ __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ ba
     constexpr int B = NG * BB;
     extern __shared__ __align__(128) u64 smem_mac[];
     u64(*ring)[kMacStages][BB][32] = (u64(*)[kMacStages][BB][32])smem_mac;                        // [NG]
-    constexpr int PS = F64 == 4 ? 2 : 3, PW = 4 * PS;  // words per partial sum, per thread
+    constexpr int PS = F64 ? 2 : 3, PW = 4 * PS;  // words per partial sum, per thread
     u64(*part)[NG][PW][32] = (u64(*)[NG][PW][32])(smem_mac + (size_t)NG * kMacStages * BB * 32);  // [2]
     u64(*bars)[kMacStages] = (u64(*)[kMacStages])(smem_mac + (size_t)NG * kMacStages * BB * 32 + (size_t)2 * NG * PW * 32);  // [NG]
     int& s_abort = *(int*)(&bars[NG][0]);
@@ -296,10 +333,8 @@ __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ ba
             tensor_load_2d(ring0 + i * BB * 256, &pt_map, (int)hpos0, row0 + i * B, bar0 + 8 * i);
         }
     }
-    // this warp's baby-step words of both sides: split into 25-bit halves (sums on the integer multiplier), or as balanced
-    // binary64 integers (sums on the FP64 pipe); sum number v * 2 + c is of the second kind if it is below F64
+    // this warp's baby-step words of both sides: split into 25-bit halves, or (F64) as balanced binary64 integers
     static_assert(F64 == 0 || BB <= 8, "the two-word binary64 sum holds eight products");
-    constexpr double kTwo52 = 4503599627370496.0, kBig = 0x1.8p103;
     unsigned w0[2][BB][2], w1[2][BB][2];
     double wd[2][BB][2];
     const double qd = (double)lc->q, halfd = (double)lc->half;
@@ -310,9 +345,8 @@ __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ ba
 #pragma unroll
             for (int c = 0; c < 2; c++) {
                 const u64 x = baby[((long long)(wg * BB + k) * 2 + c) * LN + posv[v]];
-                if (v * 2 + c < F64) {
-                    const double d = __dsub_rn(__longlong_as_double((long long)(x | 0x4330000000000000ULL)), kTwo52);
-                    wd[v][k][c] = d > halfd ? __dsub_rn(d, qd) : d;
+                if (F64) {
+                    wd[v][k][c] = residue_to_balanced_f64(x, qd, halfd);
                 } else {
                     w0[v][k][c] = (unsigned)x & kM25;
                     w1[v][k][c] = (unsigned)(x >> 25);
@@ -337,41 +371,46 @@ __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ ba
             tensor_load_2d(ring0 + st * BB * 256, &pt_map, (int)hpos0, row0 + (i + kMacStages) * B, bar0 + 8 * st);
         }
         u64(*buf)[PW][32] = part[i & 1];
-        double ah[2][2] = {{kBig, kBig}, {kBig, kBig}}, al[2][2] = {{0, 0}, {0, 0}};
-        u64 p00[2][2] = {{0, 0}, {0, 0}}, p11[2][2] = {{0, 0}, {0, 0}}, pm[2][2] = {{0, 0}, {0, 0}};
+        if (F64) {
+            double ah[2][2] = {{kAcc2Start, kAcc2Start}, {kAcc2Start, kAcc2Start}}, al[2][2] = {{0, 0}, {0, 0}};
 #pragma unroll
-        for (int k = 0; k < BB; k++) {
-            const double p = __dsub_rn(__longlong_as_double((long long)(cur[k] | 0x4330000000000000ULL)), kTwo52);
-            const unsigned a0 = (unsigned)cur[k] & kM25, a1 = (unsigned)(cur[k] >> 25), as = a0 + a1;
+            for (int k = 0; k < BB; k++) {
+                const double p = residue_to_f64(cur[k]);
+#pragma unroll
+                for (int v = 0; v < 2; v++)
+#pragma unroll
+                    for (int c = 0; c < 2; c++) acc2_fma(ah[v][c], al[v][c], p, wd[v][k][c]);
+            }
 #pragma unroll
             for (int v = 0; v < 2; v++)
 #pragma unroll
                 for (int c = 0; c < 2; c++) {
-                    if (v * 2 + c < F64) {
-                        const double nh = __fma_rn(p, wd[v][k][c], ah[v][c]);
-                        al[v][c] = __dadd_rn(al[v][c], __fma_rn(p, wd[v][k][c], __dsub_rn(ah[v][c], nh)));
-                        ah[v][c] = nh;
-                    } else {
+                    buf[wg][(v * 2 + c) * PS + 0][lane] = (u64)acc2_high(ah[v][c]);
+                    buf[wg][(v * 2 + c) * PS + 1][lane] = (u64)acc2_low(al[v][c]);
+                }
+        } else {
+            u64 p00[2][2] = {{0, 0}, {0, 0}}, p11[2][2] = {{0, 0}, {0, 0}}, pm[2][2] = {{0, 0}, {0, 0}};
+#pragma unroll
+            for (int k = 0; k < BB; k++) {
+                const unsigned a0 = (unsigned)cur[k] & kM25, a1 = (unsigned)(cur[k] >> 25), as = a0 + a1;
+#pragma unroll
+                for (int v = 0; v < 2; v++)
+#pragma unroll
+                    for (int c = 0; c < 2; c++) {
                         p00[v][c] += (u64)a0 * w0[v][k][c];
                         p11[v][c] += (u64)a1 * w1[v][k][c];
                         pm[v][c] += (u64)as * (w0[v][k][c] + w1[v][k][c]);
                     }
-                }
-        }
+            }
 #pragma unroll
-        for (int v = 0; v < 2; v++)
+            for (int v = 0; v < 2; v++)
 #pragma unroll
-            for (int c = 0; c < 2; c++) {
-                if (v * 2 + c < F64) {
-                    // high word as a count of 2^51 (below 2^51 in magnitude), low word as it is
-                    buf[wg][(v * 2 + c) * PS + 0][lane] = (u64)__double2ll_rn(__dmul_rn(__dsub_rn(ah[v][c], kBig), 0x1p-51));
-                    buf[wg][(v * 2 + c) * PS + 1][lane] = (u64)__double2ll_rn(al[v][c]);
-                } else {
+                for (int c = 0; c < 2; c++) {
                     buf[wg][(v * 2 + c) * PS + 0][lane] = p00[v][c];
                     buf[wg][(v * 2 + c) * PS + 1][lane] = pm[v][c];
                     buf[wg][(v * 2 + c) * PS + 2][lane] = p11[v][c];
                 }
-            }
+        }
         __syncthreads();
         if (s_abort) {
             // leave together; first give this warp's copies still in flight the same bounded time
@@ -379,23 +418,15 @@ __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ ba
             return;
         }
         for (int vc = wg; vc < 4; vc += NG) {
-            u64 lo, hi;
-            if (vc < F64) {
+            u64 r;
+            if (F64) {
                 long long m = 0, sl = 0;
 #pragma unroll
                 for (int g = 0; g < NG; g++) {
                     m += (long long)buf[g][vc * PS + 0][lane];
                     sl += (long long)buf[g][vc * PS + 1][lane];
                 }
-                // m 2^51 + sl + q 2^57 as an unsigned 128-bit integer: |sum| < 32 q^2 (at most 64 products) < q 2^57
-                lo = (u64)m << 51;
-                hi = (u64)(m >> 13);
-                const u64 s_lo = (u64)sl, s_hi = (u64)(sl >> 63);
-                lo += s_lo;
-                hi += s_hi + (lo < s_lo ? 1 : 0);
-                const u64 o_lo = lc->q << 57, o_hi = lc->q >> 7;
-                lo += o_lo;
-                hi += o_hi + (lo < o_lo ? 1 : 0);
+                r = acc2_reduce(m, sl, *lc);
             } else {
                 u64 s00 = 0, sm = 0, s11 = 0;
 #pragma unroll
@@ -405,15 +436,16 @@ __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ ba
                     s11 += buf[g][vc * PS + 2][lane];
                 }
                 const u64 cross = sm - s00 - s11;
-                lo = s00, hi = 0;
+                u64 lo = s00, hi = 0;
                 const u64 c_lo = cross << 25, c_hi = cross >> 39;
                 lo += c_lo;
                 hi += c_hi + (lo < c_lo ? 1 : 0);
                 const u64 d_lo = s11 << 50, d_hi = s11 >> 14;
                 lo += d_lo;
                 hi += d_hi + (lo < d_lo ? 1 : 0);
+                r = reduce128(hi, lo, *lc);
             }
-            inner[((bg0 + i) * 2 + (vc & 1)) * LN + posv[vc >> 1]] = reduce128(hi, lo, *lc);
+            inner[((bg0 + i) * 2 + (vc & 1)) * LN + posv[vc >> 1]] = r;
         }
         if (NG < 4) __syncthreads();
     }
@@ -495,14 +527,21 @@ void launch_mac_stream(hann_ctx* c, const u64* baby, int64_t baby_stride, const 
             };
             switch (c->mac_f64) {
                 case 0: go(k_mac_bulk<NG, BB, 0>, mac_bulk_smem<NG, BB, 0>()); break;
-                default: go(k_mac_bulk<NG, BB, 4>, mac_bulk_smem<NG, BB, 4>()); break;
+                default: go(k_mac_bulk<NG, BB, 1>, mac_bulk_smem<NG, BB, 1>()); break;
             }
             return;
         }
     }
 #endif
-    k_mac_stream<NG, BB, NQ><<<dim3(tiles, split), 32 * NG, 0, c->stream>>>(baby, baby_stride, pt, inner, inner_stride, c->N, c->L, n_bg,
-                                                                             per, c->lt_dev);
+    if constexpr (BB <= 8) {
+        if (c->mac_f64) {
+            k_mac_stream<NG, BB, NQ, 1><<<dim3(tiles, split), 32 * NG, 0, c->stream>>>(baby, baby_stride, pt, inner, inner_stride, c->N, c->L,
+                                                                                        n_bg, per, c->lt_dev);
+            return;
+        }
+    }
+    k_mac_stream<NG, BB, NQ, 0><<<dim3(tiles, split), 32 * NG, 0, c->stream>>>(baby, baby_stride, pt, inner, inner_stride, c->N, c->L, n_bg,
+                                                                                per, c->lt_dev);
 }
 
 // the baby-step words of NQ queries x 2 sides live in registers: 8 BB NQ of them per thread, hence BB <= 8 for one query

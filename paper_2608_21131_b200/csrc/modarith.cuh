@@ -85,6 +85,47 @@ __device__ __forceinline__ void mac128(u64& hi, u64& lo, u64 a, u64 b) {
     hi += ph + (lo < pl ? 1 : 0);
 }
 
+// ---- exact sums of products on the FP64 pipe (moduli below 2^50) --------------------------------------------------------------
+// The GPU has no native 64-bit integer multiplier (a product of two residues costs three or four 32 x 32 -> 64 multiply-adds
+// plus additions) but a full-rate binary64 multiply-add.  A sum of at most EIGHT products w * p, w a balanced residue
+// (|w| < 2^49) and p a residue in [0, 2^50), is kept exactly in two binary64 words:
+//   ah starts at 1.5 * 2^103, so every ah = fma(p, w, ah) is rounded to a multiple of 2^51 (the partial sums stay below 2^102
+//      in magnitude: ah never leaves its binade);
+//   what that rounding dropped, p w + (ah_old - ah_new), is an integer of magnitude at most 2^50, which a second fma yields
+//      exactly; eight of them sum exactly in al (|al| <= 2^53).
+// Four FP64 operations per product.  sum = (ah - 1.5 * 2^103) + al.
+constexpr double kAcc2Start = 0x1.8p103;
+
+// residue below 2^52 -> binary64 through the mantissa of 2^52 + x (one logic operation, one addition)
+__device__ __forceinline__ double residue_to_f64(u64 x) {
+    return __dsub_rn(__longlong_as_double((long long)(x | 0x4330000000000000ULL)), 4503599627370496.0);
+}
+__device__ __forceinline__ double residue_to_balanced_f64(u64 x, double q, double half) {
+    const double d = residue_to_f64(x);
+    return d > half ? __dsub_rn(d, q) : d;
+}
+__device__ __forceinline__ void acc2_fma(double& ah, double& al, double p, double w) {
+    const double nh = __fma_rn(p, w, ah);
+    al = __dadd_rn(al, __fma_rn(p, w, __dsub_rn(ah, nh)));
+    ah = nh;
+}
+// the two words as integers: high word as a count of 2^51 (below 2^51 in magnitude), low word as it is; both can be added up
+// over several partial sums in 64-bit integers
+__device__ __forceinline__ long long acc2_high(double ah) { return __double2ll_rn(__dmul_rn(__dsub_rn(ah, kAcc2Start), 0x1p-51)); }
+__device__ __forceinline__ long long acc2_low(double al) { return __double2ll_rn(al); }
+// (m 2^51 + sl) mod q for the integer sums of up to 64 products' words: |m 2^51 + sl| < 32 q^2 < q 2^57 (q < 2^50), so adding
+// q 2^57 makes it a non-negative 128-bit integer
+__device__ __forceinline__ u64 acc2_reduce(long long m, long long sl, const LimbConst& c) {
+    u64 lo = (u64)m << 51, hi = (u64)(m >> 13);
+    const u64 s_lo = (u64)sl, s_hi = (u64)(sl >> 63);
+    lo += s_lo;
+    hi += s_hi + (lo < s_lo ? 1 : 0);
+    const u64 o_lo = c.q << 57, o_hi = c.q >> 7;
+    lo += o_lo;
+    hi += o_hi + (lo < o_lo ? 1 : 0);
+    return reduce128(hi, lo, c);
+}
+
 // swap the two low nibbles of a position (an involution inside every aligned chunk of 256 positions)
 __device__ __forceinline__ int swap_nibbles(int t) { return (t & ~255) | ((t & 15) << 4) | ((t >> 4) & 15); }
 

@@ -741,3 +741,56 @@ def test_level_bit_exact_random_shapes(logN, R, B, q, p, log_scale, tol, dim, n_
     qv = np.zeros(R, dtype=np.float32)
     qv[:dim] = synth.toy_query(n_rows + 1, dim=dim)
     run_level(pair, rows, qv)
+
+
+@pytest.mark.parametrize("logN,R,B,L,nb", [(10, 128, 32, 4, 3), (10, 128, 64, 3, 2), (9, 64, 16, 2, 2), (8, 8, 8, 1, 1)])
+@pytest.mark.parametrize("f64", [1, 0])
+def test_multiply_accumulate_extreme_residues(logN, R, B, L, nb, f64):
+    """The multiply-accumulate on residues at the ends of their range (0, 1, q-1 and the two values around q/2, where the
+    balanced lift of the FP64 sums changes sign), written straight into the transform-domain buffers, against the
+    definition inner[g][c][l][t] = sum_b pt[g][b][l][t'] baby[b][c][l][t] mod q (t' = t or its mirror N-1-t in the
+    half-size stored plaintext) in exact integers; both arithmetic variants of the kernel."""
+    import torch
+
+    from paper_2608_21131_b200 import binding as b
+
+    ps = synth.small_params(logN, R, B, L=L, big=True)
+    g = b.Context(ps)
+    g.set_tuning(b.TUNE_MAC_F64, f64)
+    N, n, G = ps.N, ps.n, ps.G
+    q = np.array(ps.q, dtype=object)
+    t = np.arange(N)
+    ends = lambda ql: [0, 1, ql - 1, (ql - 1) // 2, (ql + 1) // 2]
+    tops = lambda ql: [ql - 1, ql - 2, (ql + 1) // 2]
+    baby = np.zeros((B, 2, L, N), dtype=np.uint64)
+    pt = np.zeros((nb, G, B, L, n), dtype=np.uint64)
+    for l in range(L):
+        e, f = np.array(ends(int(q[l])), dtype=np.uint64), np.array(tops(int(q[l])), dtype=np.uint64)
+        for bb in range(B):
+            for c in range(2):
+                baby[bb, c, l] = e[(bb + 2 * c + t) % 5]
+            for gg in range(G):
+                for blk in range(nb):
+                    pt[blk, gg, bb, l] = f[(gg + bb + blk + t[:n]) % 3]
+    # one position where every product is the largest possible on both sides of the balanced lift
+    for l in range(L):
+        ql = int(q[l])
+        baby[:, :, l, 5] = (ql + 1) // 2
+        baby[:, :, l, 6] = (ql - 1) // 2
+        pt[:, :, :, l, 5] = ql - 1
+        pt[:, :, :, l, 6] = ql - 1
+    assert g.sizeof(b.SIZE_BABY) == baby.nbytes and g.sizeof(b.SIZE_PT_BLOCK) * nb == pt.nbytes
+    dev = lambda a: torch.from_numpy(a.view(np.int64)).to(g.device)
+    inner = g.score_level(dev(baby), dev(pt), nb, g.workspace(nb))
+    g.sync()
+    got = inner.cpu().numpy().view(np.uint64)[: nb * G * 2 * L * N].reshape(nb, G, 2, L, N)
+    mirror = np.where(t < n, t, N - 1 - t)
+    for l in range(L):
+        ql = int(q[l])
+        bo = baby[:, :, l].astype(object)
+        for blk in range(nb):
+            for gg in range(G):
+                po = pt[blk, gg, :, l][:, mirror].astype(object)      # [B][N]
+                for c in range(2):
+                    want = (po * bo[:, c]).sum(axis=0) % ql
+                    assert np.array_equal(got[blk, gg, c, l].astype(object), want), (l, blk, gg, c)

@@ -112,6 +112,8 @@ def bench_keys(ctx, ps, args):
         ctx.set_tuning(binding.TUNE_LAZY_LANES, args.lazy_lanes)
     if args.mac_f64 is not None:
         ctx.set_tuning(binding.TUNE_MAC_F64, args.mac_f64)
+    if args.groups is not None:
+        ctx.set_tuning(binding.TUNE_HOST_GROUPS, args.groups)
     km = synth.key_material(ps, wl.KEY_SEED, rots=rots)
     ctx.load_keys(ctx.keygen_from_samples(km.s, km.rots, km.evk_a, km.evk_e), km.rots)
     return km
@@ -401,21 +403,31 @@ def run_ours(args):
                 "other_ceiling": other,
                 "traffic": traffic_step / dom_launches if traffic_step else None,
                 "traffic_source": "ncu dram bytes per polynomial on the 1-block case x polynomials per launch" if traffic_step else None}
-    # the streaming kernels against both of THEIR ceilings: bytes against the measured copy bandwidth, and residue
-    # products (three 32 x 32 -> 64 multiply-adds each) against the measured multiply-add rate
+    # the streaming kernels against THEIR ceilings: bytes against the measured copy bandwidth, and residue products against the
+    # pipe they run on.  By default (HANN_TUNE_MAC_F64) products of residues below 2^50 are summed in pairs of binary64 words,
+    # four FP64 operations each, against the FP64 rate the probe's butterflies reach (8 operations per butterfly); products
+    # modulo the 60-bit special prime (one limb in L + 1 of the key-switch inner products), and all of them with --mac-f64 0,
+    # are 32 x 32 -> 64 multiply-adds (three per product below 2^50, four above) against the measured multiply-add rate.
     L_, N_, B_, G_, R_ = ctx.L, ctx.N, ctx.B, ctx.G, ctx.R
-    products = {"mac": nb * R_ * L_ * N_ * 2,
-                "ks_inner_keys": (B_ - 1) * L_ * 2 * (L_ + 1) * N_,
-                "ks_inner": (G_ - 1) * nb * L_ * 2 * (L_ + 1) * N_}
+    f64_on = args.mac_f64 is None or args.mac_f64 != 0
+    f64_peak = 8.0 * bfly_peak
+    # (products on ciphertext-prime limbs, products on the special-prime limb)
+    products = {"mac": (nb * R_ * L_ * N_ * 2, 0),
+                "ks_inner_keys": ((B_ - 1) * L_ * 2 * L_ * N_, (B_ - 1) * L_ * 2 * N_),
+                "ks_inner": ((G_ - 1) * nb * L_ * 2 * L_ * N_, (G_ - 1) * nb * L_ * 2 * N_)}
     hbm_kernels = {}
     for k in ("mac", "ks_inner_keys", "ks_inner"):
         if k in kernels:
             sec = kernels[k]["ms_per_step"] * 1e-3
             gbs = work[k][1] / sec / 1e9
-            madds = 3.0 * products[k] / sec
+            small, special = products[k]
+            f64_ops = 4.0 * small / sec if f64_on else 0.0
+            madds = (4.0 * special + (0.0 if f64_on else 3.0 * small)) / sec
+            fracs = {"hbm": gbs / hbm_peak, "fp64": f64_ops / f64_peak, "multiply-add": madds / madd_peak}
             hbm_kernels[k] = {"GB/s": gbs, "frac_of_measured_copy": gbs / hbm_peak, "frac_of_8TBps_nominal": gbs / 8000.0,
+                              "T_f64_ops_per_s": f64_ops / 1e12, "frac_of_measured_f64_rate": f64_ops / f64_peak,
                               "T_madds_per_s": madds / 1e12, "frac_of_measured_madd_rate": madds / madd_peak,
-                              "tighter_ceiling": "hbm" if gbs / hbm_peak >= madds / madd_peak else "multiply-add"}
+                              "tighter_ceiling": max(fracs, key=fracs.get)}
 
     # end to end through the host-buffer entry point: pinned host inputs, copies inside the timed region
     rows_pin = torch.from_numpy(rows_np).pin_memory()
@@ -488,7 +500,7 @@ def run_ours(args):
             # candidates already encoded and resident (the paper's "warm" case): prepare + multiply-accumulate + rotate-and-sum
             "warm_value": world * n_rows / ((stage_ms["query_prepare"] + stage_ms["score_level"] + stage_ms["rotate_sum"]) * 1e-3),
             "kernels": kernels, "hbm_kernels": hbm_kernels, "roofline": roofline,
-            "measured_ceilings": {"f64_butterflies_per_s": bfly_peak, "int32_madds_per_s": madd_peak, "hbm_gbs": hbm_peak,
+            "measured_ceilings": {"f64_butterflies_per_s": bfly_peak, "f64_ops_per_s": 8.0 * bfly_peak, "int32_madds_per_s": madd_peak, "hbm_gbs": hbm_peak,
                                   "ntt_butterflies_per_s": {k: work[k][1] / 8.0 / (kernels[k]["ms_per_step"] * 1e-3)
                                                             for k in ("ntt_fwd_b", "ntt_inv_b", "lift_digits") if k in kernels}}, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": int(launches), "gpu_launches_per_step": launches / (n_timed_blocks * args.steps), "clocks": clocks, "compaction": compaction,
@@ -1056,6 +1068,7 @@ def main():
     ap.add_argument("--project-sweep", default="1,2,4,8,16,32", help="baby-step counts of --project")
     ap.add_argument("--giant", default="lazy", choices=["horner", "lazy"],
                     help="evaluation order of the giant steps of the rotate-and-sum (the library's own default is Horner)")
+    ap.add_argument("--groups", type=int, default=None, help="tuning: block groups a level is cut into (scored beside the encoding of the next group); default: plain order")
     ap.add_argument("--mac-f64", type=int, default=None, help="tuning: 1 (default): the multiply-accumulate sums on the FP64 pipe, 0: on the integer multiplier")
     ap.add_argument("--lazy-lanes", type=int, default=None, help="tuning: block ranges the lazy rotate-and-sum runs side by side (1..4)")
     ap.add_argument("--baby", type=int, default=None, help="baby-step count B (default: the configuration's; must divide R)")

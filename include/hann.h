@@ -141,8 +141,9 @@ int hann_get_stats(hann_ctx *ctx, hann_stats *out);
  * of that root): only half of every transform is computed and the other half is written as a mirror image; 0 computes
  * every transform in full.  Same bits either way.
  * HANN_TUNE_HOST_GROUPS: number of block groups hann_score_level_host cuts a level into (a group is scored and its scores
- * are downloaded while the rows of the following groups still travel); 0 (default) chooses from the level's size.  Ask
- * hann_level_host_bytes again after changing it.
+ * are downloaded while the rows of the following groups still travel); 0 (default) chooses from the level's size.  Values
+ * above 1 also make hann_query_level cut its level into that many groups (it keeps the plain order otherwise).  Ask
+ * hann_level_host_bytes / hann_workspace_bytes again after changing it.
  * HANN_TUNE_GIANT_LAZY (this one changes the result's BITS, not its meaning): 1 makes hann_rotate_sum, and with it
  * hann_query_level and hann_score_level_host, evaluate the giant steps in the order of hann_rotate_sum_lazy (the keys of
  * rotations 2B .. (G-1)B must then be loaded as well); 0 (default) is Horner with the single key of rotation B.
@@ -305,10 +306,13 @@ int hann_rotate_sum_lazy(hann_ctx *ctx, const void *inner_dev, int64_t n_blocks,
 
 /* One routing level for one query, device buffers in and out (Sec. 2 "Reproducing this": level + candidates +
  * encrypted query in, encrypted score vector out): hann_query_prepare, hann_encode_candidates,
- * hann_score_level and hann_rotate_sum in sequence, except that the query preparation runs on a helper stream beside
- * the candidate encoding (they are independent; both finish before the multiply-accumulate starts).  All buffers as in
- * the four calls; `ws` must hold hann_workspace_bytes(ctx, blocks).  On return everything is enqueued on the context's
- * stream again (the helper stream is joined). */
+ * hann_score_level and hann_rotate_sum, the same operations on the same data as the four calls in sequence (hence the same
+ * bits) but not one after the other: the query preparation runs on a helper stream beside the candidate encoding, and with
+ * HANN_TUNE_HOST_GROUPS above 1 the level is cut into groups of blocks, each scored (multiply-accumulate, rotate-and-sum)
+ * on one of two scoring streams as soon as it is encoded, beside the encoding of the next group.  All buffers as in the four
+ * calls; `ws` must hold hann_workspace_bytes(ctx, blocks) (with less, but enough for the four calls, the groups are given
+ * up and the level is scored after its encoding).  On return everything is enqueued on the context's stream again (the
+ * helper streams are joined). */
 int hann_query_level(hann_ctx *ctx, const void *ct_dev, const float *rows_dev, int64_t n_rows, int dim, void *baby_dev,
                      void *pt_dev, void *inner_dev, void *score_ct_dev, void *ws, size_t ws_bytes);
 

@@ -461,6 +461,18 @@ extern "C" int64_t hann_sizeof(const hann_ctx* c, int what) {
     }
 }
 
+// hann_query_level and hann_score_level_host cut a level into groups of blocks that are scored (multiply-accumulate,
+// rotate-and-sum) on two scoring streams while the following groups are still encoded: number of groups and the
+// rotate-and-sum workspace each scoring stream needs
+static void level_groups(const hann_ctx* c, int64_t nblk, int* ng_out, int64_t* ws_score_out) {
+    int64_t ng = c->host_groups;
+    if (ng <= 0) ng = nblk <= 24 ? (nblk + 2) / 3 : (nblk + 3) / 4;  // groups of three to four blocks
+    ng = std::max<int64_t>(1, std::min<int64_t>(ng, nblk));
+    const int64_t gmax = nblk - nblk * (ng - 1) / ng;
+    *ng_out = (int)ng;
+    *ws_score_out = ng > 1 ? align256(std::max(ks_item_words(c) * std::min<int64_t>(gmax, 8), lazy_block_words(c) * std::min<int64_t>(gmax, 4)) * 8 + kSlack) : 0;
+}
+
 extern "C" int64_t hann_workspace_bytes(const hann_ctx* c, int64_t max_blocks) {
     if (!c || max_blocks < 0) return HANN_EINVAL;
     const int64_t items = std::max<int64_t>(1, std::min<int64_t>(max_blocks, 8));
@@ -472,6 +484,11 @@ extern "C" int64_t hann_workspace_bytes(const hann_ctx* c, int64_t max_blocks) {
     w = std::max(w, encode_ws_bytes(c));
     // hann_query_level runs query_prepare and encode_candidates side by side, each in its own part
     w = std::max(w, align256(prepare_words(c) * 8 + kSlack) + encode_ws_bytes(c));
+    // ... and, with more than one group of blocks, the scoring of a group beside the encoding of the next
+    int ng = 1;
+    int64_t ws_score = 0;
+    if (c->host_groups > 1) level_groups(c, std::max<int64_t>(1, max_blocks), &ng, &ws_score);
+    w = std::max(w, align256(prepare_words(c) * 8 + kSlack) + align256(encode_ws_bytes(c)) + 2 * ws_score);
     return w + kSlack;
 }
 
@@ -1638,20 +1655,76 @@ extern "C" int hann_query_level(hann_ctx* c, const void* ct_dev, const float* ro
     const int64_t nblk = (n_rows + c->n - 1) / c->n;
     // fork: the baby rotations of the query on the helper stream, the candidate encoding on the context's stream
     cudaStream_t main_stream = c->stream;
+    // (measured on the face level: two groups gain 1.5 %, three and more lose, the device being limited by its FP64 pipe
+    // and its power cap in every stage: the groups are used only when asked for)
+    int ng = 1;
+    int64_t ws_score = 0;
+    if (c->host_groups > 1) level_groups(c, nblk, &ng, &ws_score);
+    const int64_t enc_bytes = align256(encode_ws_bytes(c));
+    // the groups need a workspace layout of their own; a smaller workspace, the per-launch profile (whose kernel times must
+    // not overlap) or a context that already runs on a helper stream take the plain order
+    if (ng > 1 && ((int64_t)ws_bytes < prep + enc_bytes + 2 * ws_score || c->kprof || main_stream == c->aux_stream)) ng = 1;
     CK(cudaEventRecord(c->ev_fork, main_stream));
     CK(cudaStreamWaitEvent(c->aux_stream, c->ev_fork, 0));
     c->stream = c->aux_stream;
     int rc = hann_query_prepare(c, ct_dev, baby_dev, ws, (size_t)prep);
     c->stream = main_stream;
-    cudaError_t e = cudaEventRecord(c->ev_join, c->aux_stream);
-    if (rc == HANN_OK) rc = hann_encode_candidates(c, rows_dev, n_rows, dim, pt_dev, (char*)ws + prep, ws_bytes - (size_t)prep);
-    // join before anything else is reported, so that the helper stream never runs past this call's buffers unobserved
-    cudaError_t e2 = cudaStreamWaitEvent(main_stream, c->ev_join, 0);
+    if (ng == 1) {
+        cudaError_t e = cudaEventRecord(c->ev_join, c->aux_stream);
+        if (rc == HANN_OK) rc = hann_encode_candidates(c, rows_dev, n_rows, dim, pt_dev, (char*)ws + prep, ws_bytes - (size_t)prep);
+        // join before anything else is reported, so that the helper stream never runs past this call's buffers unobserved
+        cudaError_t e2 = cudaStreamWaitEvent(main_stream, c->ev_join, 0);
+        RET(rc);
+        CK(e);
+        CK(e2);
+        RET(hann_score_level(c, baby_dev, pt_dev, nblk, inner_dev, ws, ws_bytes));
+        RET(hann_rotate_sum(c, inner_dev, nblk, score_ct_dev, ws, ws_bytes));
+        return HANN_OK;
+    }
+    // Groups of blocks: the context's stream encodes group after group; a group is scored (multiply-accumulate,
+    // rotate-and-sum) on one of two scoring streams as soon as it is encoded, beside the encoding of the next groups: the
+    // latency chains of a group's key switches fill the gaps of the encoding kernels.  Only the last group's scoring follows
+    // the last encoding.  Same operations on the same data as the plain order, hence the same bits.
+    cudaError_t ce = cudaEventRecord(c->prep_done, c->aux_stream);
+    for (int i = 0; i < 2 && ce == cudaSuccess; i++) ce = cudaStreamWaitEvent(c->score_stream[i], c->ev_fork, 0);
+    while ((int)c->enc_ev.size() < ng && ce == cudaSuccess) {
+        cudaEvent_t e;
+        ce = cudaEventCreateWithFlags(&e, cudaEventDisableTiming);
+        if (ce == cudaSuccess) c->enc_ev.push_back(e);
+    }
+    const int64_t ptw = hann_sizeof(c, HANN_SIZE_PT_BLOCK) / 8, ctw = hann_sizeof(c, HANN_SIZE_CT) / 8;
+    const int64_t innerw = hann_sizeof(c, HANN_SIZE_INNER) / 8;
+    char* ws_enc = (char*)ws + prep;
+    char* wss[2] = {ws_enc + enc_bytes, ws_enc + enc_bytes + ws_score};
+    const int saved_lanes = c->max_lanes;
+    for (int gi = 0; gi < ng && rc == HANN_OK && ce == cudaSuccess; gi++) {
+        const int64_t b0 = nblk - nblk * (ng - gi) / ng, b1 = nblk - nblk * (ng - gi - 1) / ng, nb = b1 - b0;
+        const int64_t r0 = b0 * c->n, rn = std::min<int64_t>(nb * c->n, n_rows - r0);
+        rc = hann_encode_candidates(c, rows_dev + r0 * dim, rn, dim, (u64*)pt_dev + b0 * ptw, ws_enc, (size_t)enc_bytes);
+        if (rc != HANN_OK) break;
+        cudaStream_t ss = c->score_stream[gi & 1];
+        ce = cudaEventRecord(c->enc_ev[gi], main_stream);
+        if (ce == cudaSuccess) ce = cudaStreamWaitEvent(ss, c->enc_ev[gi], 0);
+        if (ce == cudaSuccess && gi < 2) ce = cudaStreamWaitEvent(ss, c->prep_done, 0);  // the baby rotations are ready
+        if (ce != cudaSuccess) break;
+        c->stream = ss;
+        c->max_lanes = 1;  // the groups run side by side instead of the lanes
+        rc = hann_score_level(c, baby_dev, (const u64*)pt_dev + b0 * ptw, nb, (u64*)inner_dev + b0 * innerw, wss[gi & 1], (size_t)ws_score);
+        if (rc == HANN_OK)
+            rc = hann_rotate_sum(c, (const u64*)inner_dev + b0 * innerw, nb, (u64*)score_ct_dev + b0 * ctw, wss[gi & 1], (size_t)ws_score);
+        c->stream = main_stream;
+        c->max_lanes = saved_lanes;
+    }
+    // join every helper stream before reporting anything
+    cudaError_t ej[3];
+    ej[0] = cudaStreamWaitEvent(main_stream, c->prep_done, 0);
+    for (int i = 0; i < 2; i++) {
+        ej[1 + i] = cudaEventRecord(c->score_join[i], c->score_stream[i]);
+        if (ej[1 + i] == cudaSuccess) ej[1 + i] = cudaStreamWaitEvent(main_stream, c->score_join[i], 0);
+    }
     RET(rc);
-    CK(e);
-    CK(e2);
-    RET(hann_score_level(c, baby_dev, pt_dev, nblk, inner_dev, ws, ws_bytes));
-    RET(hann_rotate_sum(c, inner_dev, nblk, score_ct_dev, ws, ws_bytes));
+    CK(ce);
+    for (int i = 0; i < 3; i++) CK(ej[i]);
     return HANN_OK;
 }
 
@@ -1674,12 +1747,8 @@ LevelPlan plan_level(const hann_ctx* c, int64_t n_rows, int dim) {
     p.score = align256(p.nblk * ctb);
     p.stage = align256(p.nblk * ctb);
     p.ws = align256(hann_workspace_bytes(c, p.nblk));
-    p.ng = c->host_groups;
-    if (p.ng <= 0) p.ng = (int)(p.nblk <= 24 ? (p.nblk + 2) / 3 : (p.nblk + 3) / 4);  // groups of three to four blocks
-    p.ng = (int)std::max<int64_t>(1, std::min<int64_t>(p.ng, p.nblk));
     // with more than one group: a rotate-and-sum workspace for each of the two scoring streams
-    const int64_t gmax = p.nblk - p.nblk * (p.ng - 1) / p.ng;
-    p.ws_score = p.ng > 1 ? align256(std::max(ks_item_words(c) * std::min<int64_t>(gmax, 8), lazy_block_words(c) * std::min<int64_t>(gmax, 4)) * 8 + kSlack) : 0;
+    level_groups(c, p.nblk, &p.ng, &p.ws_score);
     p.total = p.ct + p.baby + p.rows + p.pt + p.inner + p.score + p.stage + p.ws + 2 * p.ws_score;
     return p;
 }

@@ -46,7 +46,7 @@ __global__ void __launch_bounds__(kThreads) k_lift_digits(const u64* __restrict_
 __global__ void __launch_bounds__(kThreads) k_ks_inner(const u64* __restrict__ digits, long long digit_stride,
                                                        const u64* const* __restrict__ keytab, int rot0, int rot_inc,
                                                        u64* __restrict__ u, int N, int L, long long nitems,
-                                                       LimbTable lt) {
+                                                       LimbTable lt, int f64) {
     const long long L1N = (long long)(L + 1) * N;
     const long long total = nitems * L1N;
     for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total; idx += (long long)gridDim.x * kThreads) {
@@ -55,15 +55,37 @@ __global__ void __launch_bounds__(kThreads) k_ks_inner(const u64* __restrict__ d
         const int i = (int)(pos / N);
         const u64* key = keytab[rot0 + (int)item * rot_inc];
         const u64* d = digits + item * digit_stride + pos;
+        const LimbConst& lc = lt.c[i];
+        u64* o = u + item * 2 * L1N + pos;
+        if (f64 && lc.q < (1ULL << 50)) {
+            // moduli below 2^50: exact two-word binary64 sums (acc2_fma) of eight digits at a time, their integer words added up
+            const double qd = (double)lc.q, halfd = (double)lc.half;
+            long long m0 = 0, s0 = 0, m1 = 0, s1 = 0;
+            for (int j0 = 0; j0 < L; j0 += 8) {
+                double ah0 = kAcc2Start, al0 = 0, ah1 = kAcc2Start, al1 = 0;
+                const int j1 = j0 + 8 < L ? j0 + 8 : L;
+#pragma unroll 4
+                for (int j = j0; j < j1; j++) {
+                    const double dv = residue_to_balanced_f64(d[(long long)j * L1N], qd, halfd);
+                    acc2_fma(ah0, al0, residue_to_f64(__ldcs(key + ((long long)j * 2 + 0) * L1N + pos)), dv);
+                    acc2_fma(ah1, al1, residue_to_f64(__ldcs(key + ((long long)j * 2 + 1) * L1N + pos)), dv);
+                }
+                m0 += acc2_high(ah0), s0 += acc2_low(al0);
+                m1 += acc2_high(ah1), s1 += acc2_low(al1);
+            }
+            o[0] = acc2_reduce(m0, s0, lc);
+            o[L1N] = acc2_reduce(m1, s1, lc);
+            continue;
+        }
         u64 h0 = 0, l0 = 0, h1 = 0, l1 = 0;
+#pragma unroll 4
         for (int j = 0; j < L; j++) {
             u64 dv = d[(long long)j * L1N];
             mac128(h0, l0, dv, __ldcs(key + ((long long)j * 2 + 0) * L1N + pos));
             mac128(h1, l1, dv, __ldcs(key + ((long long)j * 2 + 1) * L1N + pos));
         }
-        u64* o = u + item * 2 * L1N + pos;
-        o[0] = reduce128(h0, l0, lt.c[i]);
-        o[L1N] = reduce128(h1, l1, lt.c[i]);
+        o[0] = reduce128(h0, l0, lc);
+        o[L1N] = reduce128(h1, l1, lc);
     }
 }
 
@@ -653,7 +675,7 @@ int launch_ks_inner(hann_ctx* c, const u64* digits, int64_t digit_stride, int ro
     {
         KProf kp(c, KC_KS_INNER);
         k_ks_inner<<<grid_for(nitems * (c->L + 1) * c->N), kThreads, 0, c->stream>>>(digits, digit_stride, c->keytab_dev, rot0, rot_inc, u,
-                                                                                   c->N, c->L, nitems, c->lt);
+                                                                                   c->N, c->L, nitems, c->lt, c->mac_f64);
     }
     return check_launch(c, "ks_inner");
 }

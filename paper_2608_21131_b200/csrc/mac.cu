@@ -77,6 +77,7 @@ __global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ 
     unsigned w0[NV][BB][2], w1[NV][BB][2];
     double wd[NV][BB][2];
     const double qd = (double)lc->q, halfd = (double)lc->half;
+    const bool big = F64 == 2 && lc->q >= (1ULL << 50);  // see k_mac_bulk
 #pragma unroll
     for (int v = 0; v < NV; v++)
 #pragma unroll
@@ -85,7 +86,7 @@ __global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ 
             for (int c = 0; c < 2; c++) {
                 const u64 x = baby[(v >> 1) * baby_stride + ((long long)(wg * BB + k) * 2 + c) * LN + posv[v & 1]];
                 if (F64) {
-                    wd[v][k][c] = residue_to_balanced_f64(x, qd, halfd);
+                    wd[v][k][c] = big ? __longlong_as_double((long long)x) : residue_to_balanced_f64(x, qd, halfd);
                 } else {
                     w0[v][k][c] = (unsigned)x & kM25;
                     w1[v][k][c] = (unsigned)(x >> 25);
@@ -105,7 +106,26 @@ __global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ 
             for (int k = 0; k < BB; k++) nxt[k] = __ldcs(pn + (long long)k * Ln);
         }
         u64(*buf)[PS * 2 * NV][32] = part[bg & 1];
-        if (F64) {
+        if (F64 == 2 && big) {
+            u64 hi[NV][2], lo[NV][2];
+#pragma unroll
+            for (int v = 0; v < NV; v++)
+#pragma unroll
+                for (int c = 0; c < 2; c++) hi[v][c] = lo[v][c] = 0;
+#pragma unroll
+            for (int k = 0; k < BB; k++)
+#pragma unroll
+                for (int v = 0; v < NV; v++)
+#pragma unroll
+                    for (int c = 0; c < 2; c++) mac128(hi[v][c], lo[v][c], cur[k], (u64)__double_as_longlong(wd[v][k][c]));
+#pragma unroll
+            for (int v = 0; v < NV; v++)
+#pragma unroll
+                for (int c = 0; c < 2; c++) {
+                    buf[wg][(v * 2 + c) * PS + 0][lane] = hi[v][c];
+                    buf[wg][(v * 2 + c) * PS + 1][lane] = lo[v][c];
+                }
+        } else if (F64) {
             double ah[NV][2], al[NV][2];
 #pragma unroll
             for (int v = 0; v < NV; v++)
@@ -157,7 +177,16 @@ __global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ 
         // the warps share out the 2 * NV (query, side, component) sums
         for (int vc = wg; vc < 2 * NV; vc += NG) {
             u64 r;
-            if (F64) {
+            if (F64 == 2 && big) {
+                u64 hi = 0, lo = 0;  // at most 64 products below 2^120 each
+#pragma unroll
+                for (int g = 0; g < NG; g++) {
+                    const u64 l = buf[g][vc * PS + 1][lane];
+                    lo += l;
+                    hi += buf[g][vc * PS + 0][lane] + (lo < l ? 1 : 0);
+                }
+                r = reduce128(hi, lo, *lc);
+            } else if (F64) {
                 long long m = 0, sl = 0;
 #pragma unroll
                 for (int g = 0; g < NG; g++) {
@@ -338,6 +367,9 @@ __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ ba
     unsigned w0[2][BB][2], w1[2][BB][2];
     double wd[2][BB][2];
     const double qd = (double)lc->q, halfd = (double)lc->half;
+    // F64 == 2: the chain has primes in [2^50, 2^60); their limbs (uniform over a CTA) take 128-bit integer sums, the words
+    // kept as they are
+    const bool big = F64 == 2 && lc->q >= (1ULL << 50);
 #pragma unroll
     for (int v = 0; v < 2; v++)
 #pragma unroll
@@ -346,7 +378,7 @@ __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ ba
             for (int c = 0; c < 2; c++) {
                 const u64 x = baby[((long long)(wg * BB + k) * 2 + c) * LN + posv[v]];
                 if (F64) {
-                    wd[v][k][c] = residue_to_balanced_f64(x, qd, halfd);
+                    wd[v][k][c] = big ? __longlong_as_double((long long)x) : residue_to_balanced_f64(x, qd, halfd);
                 } else {
                     w0[v][k][c] = (unsigned)x & kM25;
                     w1[v][k][c] = (unsigned)(x >> 25);
@@ -371,7 +403,22 @@ __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ ba
             tensor_load_2d(ring0 + st * BB * 256, &pt_map, (int)hpos0, row0 + (i + kMacStages) * B, bar0 + 8 * st);
         }
         u64(*buf)[PW][32] = part[i & 1];
-        if (F64) {
+        if (F64 == 2 && big) {
+            u64 hi[2][2] = {{0, 0}, {0, 0}}, lo[2][2] = {{0, 0}, {0, 0}};
+#pragma unroll
+            for (int k = 0; k < BB; k++)
+#pragma unroll
+                for (int v = 0; v < 2; v++)
+#pragma unroll
+                    for (int c = 0; c < 2; c++) mac128(hi[v][c], lo[v][c], cur[k], (u64)__double_as_longlong(wd[v][k][c]));
+#pragma unroll
+            for (int v = 0; v < 2; v++)
+#pragma unroll
+                for (int c = 0; c < 2; c++) {
+                    buf[wg][(v * 2 + c) * PS + 0][lane] = hi[v][c];
+                    buf[wg][(v * 2 + c) * PS + 1][lane] = lo[v][c];
+                }
+        } else if (F64) {
             double ah[2][2] = {{kAcc2Start, kAcc2Start}, {kAcc2Start, kAcc2Start}}, al[2][2] = {{0, 0}, {0, 0}};
 #pragma unroll
             for (int k = 0; k < BB; k++) {
@@ -419,7 +466,16 @@ __global__ void __launch_bounds__(32 * NG) k_mac_bulk(const u64* __restrict__ ba
         }
         for (int vc = wg; vc < 4; vc += NG) {
             u64 r;
-            if (F64) {
+            if (F64 == 2 && big) {
+                u64 hi = 0, lo = 0;  // at most 64 products below 2^120 each
+#pragma unroll
+                for (int g = 0; g < NG; g++) {
+                    const u64 l = buf[g][vc * PS + 1][lane];
+                    lo += l;
+                    hi += buf[g][vc * PS + 0][lane] + (lo < l ? 1 : 0);
+                }
+                r = reduce128(hi, lo, *lc);
+            } else if (F64) {
                 long long m = 0, sl = 0;
 #pragma unroll
                 for (int g = 0; g < NG; g++) {
@@ -508,6 +564,8 @@ void launch_mac_stream(hann_ctx* c, const u64* baby, int64_t baby_stride, const 
                        int64_t inner_stride) {
     const long long Ln = (long long)c->L * c->n;
     const int tiles = (int)(Ln / 32);
+    bool big_primes = false;  // primes in [2^50, 2^60): the caller lets them through only with the FP64 variant and one query
+    for (int l = 0; l < c->L; l++) big_primes = big_primes || c->mod[l] >= (1ULL << 50);
     // split the (blk, g) range over grid.y only as far as needed to fill the machine: every extra split re-reads the
     // baby-step words
     int split = 1;
@@ -525,19 +583,25 @@ void launch_mac_stream(hann_ctx* c, const u64* baby, int64_t baby_stride, const 
                 if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
                 kern<<<dim3(tiles, split), 32 * NG, smem, c->stream>>>(baby, map, inner, c->N, c->L, n_bg, per, c->lt_dev, c->kflag);
             };
-            switch (c->mac_f64) {
-                case 0: go(k_mac_bulk<NG, BB, 0>, mac_bulk_smem<NG, BB, 0>()); break;
-                default: go(k_mac_bulk<NG, BB, 1>, mac_bulk_smem<NG, BB, 1>()); break;
-            }
+            if (!c->mac_f64) go(k_mac_bulk<NG, BB, 0>, mac_bulk_smem<NG, BB, 0>());
+            else if (big_primes) go(k_mac_bulk<NG, BB, 2>, mac_bulk_smem<NG, BB, 2>());
+            else go(k_mac_bulk<NG, BB, 1>, mac_bulk_smem<NG, BB, 1>());
             return;
         }
     }
 #endif
     if constexpr (BB <= 8) {
-        if (c->mac_f64) {
+        if (c->mac_f64 && !big_primes) {
             k_mac_stream<NG, BB, NQ, 1><<<dim3(tiles, split), 32 * NG, 0, c->stream>>>(baby, baby_stride, pt, inner, inner_stride, c->N, c->L,
                                                                                         n_bg, per, c->lt_dev);
             return;
+        }
+        if constexpr (NQ == 1) {
+            if (c->mac_f64) {
+                k_mac_stream<NG, BB, 1, 2><<<dim3(tiles, split), 32 * NG, 0, c->stream>>>(baby, baby_stride, pt, inner, inner_stride, c->N, c->L,
+                                                                                           n_bg, per, c->lt_dev);
+                return;
+            }
         }
     }
     k_mac_stream<NG, BB, NQ, 0><<<dim3(tiles, split), 32 * NG, 0, c->stream>>>(baby, baby_stride, pt, inner, inner_stride, c->N, c->L, n_bg,
@@ -570,14 +634,18 @@ int launch_mac_batch(hann_ctx* c, const u64* baby, int n_queries, const u64* pt,
     const long long LN = (long long)c->L * c->N;
     const long long n_bg = n_blocks * c->G;
     const int64_t baby_stride = (int64_t)c->B * 2 * LN, inner_stride = n_bg * 2 * LN;
+    // the streaming kernels: moduli below 2^50, or (their FP64 variant only) below 2^60 with the limbs of the larger primes
+    // summed in 128-bit integers
     bool small = c->N >= 64 && c->B <= 64 && (c->B & (c->B - 1)) == 0;
-    for (int l = 0; l < c->L; l++) small = small && c->mod[l] < (1ULL << 50);
+    for (int l = 0; l < c->L; l++) small = small && c->mod[l] < (c->mac_f64 ? (1ULL << 60) : (1ULL << 50));
     if (small) {
         // pairs of queries share one pass over the stored plaintexts where the baby-step words of two queries and both
         // sides fit the register file (B <= 16); a last odd query, and every query of wider baby sets, takes a pass of
         // its own
         int q = 0;
-        if (c->B <= 16)
+        bool pairs = c->B <= 16;
+        for (int l = 0; l < c->L; l++) pairs = pairs && c->mod[l] < (1ULL << 50);
+        if (pairs)
             for (; q + 2 <= n_queries; q += 2) launch_mac_stream_b<2>(c, baby + q * baby_stride, baby_stride, pt, n_bg, inner + q * inner_stride, inner_stride);
         for (; q < n_queries; q++) launch_mac_stream_b<1>(c, baby + q * baby_stride, baby_stride, pt, n_bg, inner + q * inner_stride, inner_stride);
         return check_launch(c, "mac_stream");

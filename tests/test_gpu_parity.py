@@ -224,6 +224,19 @@ def test_host_buffer_level_matches_device_path(n_rows):
         ws_g = p.g.alloc(p.g.level_host_bytes(rows.shape[0]))
         assert np.array_equal(p.g.score_level_host(ct_g, rows, ws_g), score_dev)
     p.g.set_tuning(p.b.TUNE_HOST_GROUPS, 0)
+    # the device-resident level call cuts the level the same way (a group scored beside the encoding of the next): same bits,
+    # also with both orders of the giant steps and with a workspace too small for the groups (plain order)
+    g, b = p.g, p.b
+    ct_dev = g.import_(b.KIND_CT, ct_g, 1)
+    for groups in (0, 1, 2, 3, 4):
+        g.set_tuning(b.TUNE_HOST_GROUPS, groups)
+        for ws in (g.workspace(nb), g.workspace(1)):
+            baby, pt, inner, score = (g.alloc(g.sizeof(b.SIZE_BABY)), g.alloc(nb * g.sizeof(b.SIZE_PT_BLOCK)),
+                                      g.alloc(nb * g.sizeof(b.SIZE_INNER)), g.alloc(nb * g.sizeof(b.SIZE_CT)))
+            g.query_level(ct_dev, torch_rows(p, rows), ws, baby, pt, inner, score)
+            g.sync()
+            assert np.array_equal(g.export(b.KIND_CT, score, nb), score_dev), groups
+    g.set_tuning(b.TUNE_HOST_GROUPS, 0)
 
 
 def test_full_ring_one_block():
@@ -743,7 +756,7 @@ def test_level_bit_exact_random_shapes(logN, R, B, q, p, log_scale, tol, dim, n_
     run_level(pair, rows, qv)
 
 
-@pytest.mark.parametrize("logN,R,B,L,nb", [(10, 128, 32, 4, 3), (10, 128, 64, 3, 2), (9, 64, 16, 2, 2), (8, 8, 8, 1, 1)])
+@pytest.mark.parametrize("logN,R,B,L,nb", [(10, 128, 32, 4, 3), (10, 128, 64, 3, 2), (9, 64, 16, 2, 2), (8, 8, 8, 1, 1), (10, 128, 32, -3, 2)])
 @pytest.mark.parametrize("f64", [1, 0])
 def test_multiply_accumulate_extreme_residues(logN, R, B, L, nb, f64):
     """The multiply-accumulate on residues at the ends of their range (0, 1, q-1 and the two values around q/2, where the
@@ -754,7 +767,15 @@ def test_multiply_accumulate_extreme_residues(logN, R, B, L, nb, f64):
 
     from paper_2608_21131_b200 import binding as b
 
-    ps = synth.small_params(logN, R, B, L=L, big=True)
+    if L < 0:
+        # a chain that starts with a 58-bit prime, as the membership circuit's does: that limb takes 128-bit integer sums inside
+        # the same kernel (FP64 variant) or the whole level goes through the generic kernel (integer variant)
+        from oracle.oracle import find_primes
+
+        L = -L
+        ps = synth.ParamSet("mixed", logN, tuple(find_primes(58, logN + 1, 1)) + tuple(synth.Q50[: L - 1]), synth.P60, 40, R, B, -18)
+    else:
+        ps = synth.small_params(logN, R, B, L=L, big=True)
     g = b.Context(ps)
     g.set_tuning(b.TUNE_MAC_F64, f64)
     N, n, G = ps.N, ps.n, ps.G

@@ -112,6 +112,8 @@ def bench_keys(ctx, ps, args):
         ctx.set_tuning(binding.TUNE_LAZY_LANES, args.lazy_lanes)
     if args.mac_f64 is not None:
         ctx.set_tuning(binding.TUNE_MAC_F64, args.mac_f64)
+    if args.pair_b32:
+        ctx.set_tuning(binding.TUNE_PAIR_B32, 1)
     if args.groups is not None:
         ctx.set_tuning(binding.TUNE_HOST_GROUPS, args.groups)
     km = synth.key_material(ps, wl.KEY_SEED, rots=rots)
@@ -524,6 +526,10 @@ def run_batch(args):
     ps, rows_np, qR, wname = build_workload(args.config, args.rows, args.logn)
     n_rows, Q = rows_np.shape[0], args.queries
     ctx = binding.Context(ps, device=0)
+    if args.pair_b32:
+        ctx.set_tuning(binding.TUNE_PAIR_B32, 1)
+    if args.mac_f64 is not None:
+        ctx.set_tuning(binding.TUNE_MAC_F64, args.mac_f64)
     km = synth.key_material(ps, wl.KEY_SEED)
     ctx.load_keys(ctx.keygen_from_samples(km.s, km.rots, km.evk_a, km.evk_e), km.rots)
     rng = np.random.default_rng(wl.KEY_SEED)
@@ -1069,6 +1075,7 @@ def main():
     ap.add_argument("--giant", default="lazy", choices=["horner", "lazy"],
                     help="evaluation order of the giant steps of the rotate-and-sum (the library's own default is Horner)")
     ap.add_argument("--groups", type=int, default=None, help="tuning: block groups a level is cut into (scored beside the encoding of the next group); default: plain order")
+    ap.add_argument("--pair-b32", action="store_true", help="tuning (--queries): two queries per pass over the plaintexts at B = 32 too")
     ap.add_argument("--mac-f64", type=int, default=None, help="tuning: 1 (default): the multiply-accumulate sums on the FP64 pipe, 0: on the integer multiplier")
     ap.add_argument("--lazy-lanes", type=int, default=None, help="tuning: block ranges the lazy rotate-and-sum runs side by side (1..4)")
     ap.add_argument("--baby", type=int, default=None, help="baby-step count B (default: the configuration's; must divide R)")

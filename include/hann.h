@@ -149,9 +149,11 @@ int hann_get_stats(hann_ctx *ctx, hann_stats *out);
  * rotations 2B .. (G-1)B must then be loaded as well); 0 (default) is Horner with the single key of rotation B.
  * HANN_TUNE_LAZY_LANES: block ranges (1..4, default 2) hann_rotate_sum_lazy runs side by side on helper streams.
  * HANN_TUNE_MAC_F64: 1 (default) lets the single-query multiply-accumulate of chains of primes below 2^50 sum its products
- * exactly in pairs of binary64 words on the FP64 pipe, 0 on the integer multiplier; same residues either way. */
+ * exactly in pairs of binary64 words on the FP64 pipe, 0 on the integer multiplier; same residues either way.
+ * HANN_TUNE_PAIR_B32: 1 lets hann_score_level_batch serve two queries per pass over the stored plaintexts at B = 32 as well
+ * (it does at B <= 16); 0 (default) gives every query its own pass there. */
 enum { HANN_TUNE_ENCODE_GROUP = 1, HANN_TUNE_HOST_LIMBS = 2, HANN_TUNE_ENCODE_SYMMETRY = 3, HANN_TUNE_HOST_GROUPS = 4, HANN_TUNE_GIANT_LAZY = 5,
-       HANN_TUNE_LAZY_LANES = 6, HANN_TUNE_MAC_F64 = 7 };
+       HANN_TUNE_LAZY_LANES = 6, HANN_TUNE_MAC_F64 = 7, HANN_TUNE_PAIR_B32 = 8 };
 int hann_set_tuning(hann_ctx *ctx, int what, int value);
 
 /* Per-launch profile: while enabled every kernel launch of the context is bracketed by a CUDA event pair (this

@@ -26,6 +26,7 @@ TUNE_HOST_GROUPS = 4
 TUNE_GIANT_LAZY = 5
 TUNE_LAZY_LANES = 6
 TUNE_MAC_F64 = 7
+TUNE_PAIR_B32 = 8
 
 
 class HannError(RuntimeError):

@@ -595,6 +595,9 @@ extern "C" int hann_set_tuning(hann_ctx* c, int what, int value) {
         case HANN_TUNE_MAC_F64:
             c->mac_f64 = value ? 4 : 0;
             return HANN_OK;
+        case HANN_TUNE_PAIR_B32:
+            c->pair_b32 = value ? 1 : 0;
+            return HANN_OK;
         default: return fail(c, HANN_EINVAL, "hann_set_tuning: unknown knob");
     }
 }

@@ -79,6 +79,7 @@ struct hann_ctx {
     // debugging aid: guards behind every workspace sub-buffer (see Arena in api.cu), filled when carved, checked on request
     int canaries = 0;
     std::vector<u64*> guards;
+    int pair_b32 = 0;    // hann_score_level_batch pairs queries at B = 32 too (eight warps of four baby steps, FP64 form)
     int mac_f64 = 4;     // how many of a thread's four sums the single-query multiply-accumulate keeps on the FP64 pipe
     int lazy_lanes = 2;  // block ranges hann_rotate_sum_lazy runs side by side
     int giant_lazy = 0;  // hann_rotate_sum (and the calls built on it) evaluates the giant steps in the lazy order

@@ -65,7 +65,10 @@ __global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ 
     constexpr int NV = 2 * NQ;  // (query, side): side 0 is position t, side 1 its mirror image N - 1 - t
     constexpr int PS = F64 ? 2 : 3;  // words per partial sum: (high, low) of the binary64 sums, or the three Karatsuba sums
     static_assert(F64 == 0 || BB <= 8, "the two-word binary64 sum holds eight products");
-    __shared__ u64 part[2][NG][PS * 2 * NV][32];
+    // two buffers (a warp may write the next pair's partial sums while others still add up this pair's) where they fit the
+    // static shared memory, one and a second barrier per pair otherwise
+    constexpr int NBUF = (size_t)2 * NG * PS * 2 * NV * 32 * 8 > 48 * 1024 ? 1 : 2;
+    __shared__ u64 part[NBUF][NG][PS * 2 * NV][32];
     const int n = N >> 1;
     const long long LN = (long long)L * N, Ln = (long long)L * n;
     const long long hpos0 = (long long)blockIdx.x * 32;  // in the stored plaintext layout [L][N/2]
@@ -105,7 +108,7 @@ __global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ 
 #pragma unroll
             for (int k = 0; k < BB; k++) nxt[k] = __ldcs(pn + (long long)k * Ln);
         }
-        u64(*buf)[PS * 2 * NV][32] = part[bg & 1];
+        u64(*buf)[PS * 2 * NV][32] = part[NBUF == 2 ? (bg & 1) : 0];
         if (F64 == 2 && big) {
             u64 hi[NV][2], lo[NV][2];
 #pragma unroll
@@ -216,7 +219,7 @@ __global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ 
             const int v = vc >> 1;
             inner[(v >> 1) * inner_stride + (bg * 2 + (vc & 1)) * LN + posv[v & 1]] = r;
         }
-        if (NG < 2 * NV) __syncthreads();  // a warp that finishes several sums may still be reading while the next pair is written
+        if (NBUF == 1 || NG < 2 * NV) __syncthreads();  // a warp that finishes several sums may still be reading while the next pair is written
 #pragma unroll
         for (int k = 0; k < BB; k++) cur[k] = nxt[k];
         p += (long long)B * Ln;
@@ -604,8 +607,11 @@ void launch_mac_stream(hann_ctx* c, const u64* baby, int64_t baby_stride, const 
             }
         }
     }
-    k_mac_stream<NG, BB, NQ, 0><<<dim3(tiles, split), 32 * NG, 0, c->stream>>>(baby, baby_stride, pt, inner, inner_stride, c->N, c->L, n_bg,
-                                                                                per, c->lt_dev);
+    // (two queries at more than 16 baby steps exist in the FP64 form only: the three-word partial sums of the integer form
+    // do not fit the static shared memory; the caller does not pair queries there)
+    if constexpr (!(NQ == 2 && NG * BB > 16))
+        k_mac_stream<NG, BB, NQ, 0><<<dim3(tiles, split), 32 * NG, 0, c->stream>>>(baby, baby_stride, pt, inner, inner_stride, c->N, c->L,
+                                                                                    n_bg, per, c->lt_dev);
 }
 
 // the baby-step words of NQ queries x 2 sides live in registers: 8 BB NQ of them per thread, hence BB <= 8 for one query
@@ -621,6 +627,7 @@ void launch_mac_stream_b(hann_ctx* c, const u64* baby, int64_t baby_stride, cons
         case 16: launch_mac_stream<4, 4, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride); break;
         case 32:
             if constexpr (NQ == 1) launch_mac_stream<4, 8, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride);
+            else launch_mac_stream<8, 4, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride);
             break;
         default:
             if constexpr (NQ == 1) launch_mac_stream<8, 8, NQ>(c, baby, baby_stride, pt, n_bg, inner, inner_stride);
@@ -643,7 +650,7 @@ int launch_mac_batch(hann_ctx* c, const u64* baby, int n_queries, const u64* pt,
         // sides fit the register file (B <= 16); a last odd query, and every query of wider baby sets, takes a pass of
         // its own
         int q = 0;
-        bool pairs = c->B <= 16;
+        bool pairs = c->B <= 16 || (c->B == 32 && c->mac_f64 && c->pair_b32);
         for (int l = 0; l < c->L; l++) pairs = pairs && c->mod[l] < (1ULL << 50);
         if (pairs)
             for (; q + 2 <= n_queries; q += 2) launch_mac_stream_b<2>(c, baby + q * baby_stride, baby_stride, pt, n_bg, inner + q * inner_stride, inner_stride);

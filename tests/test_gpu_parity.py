@@ -477,16 +477,21 @@ def test_compacted_scores_bit_exact_and_decrypt(logN, L, big, n_rows):
             assert np.abs(got - got_o).max() < 1e-9 * max(1.0, np.abs(got_o).max()) + 2 * sigma * 1e-6
 
 
-@pytest.mark.parametrize("logN,R,B,L,big,n_rows,nq", [(6, 8, 2, 2, False, 70, 3), (10, 64, 8, 2, False, 1200, 5), (11, 32, 32, 4, True, 1100, 2)])
+@pytest.mark.parametrize("logN,R,B,L,big,n_rows,nq", [(6, 8, 2, 2, False, 70, 3), (10, 64, 8, 2, False, 1200, 5), (11, 32, 32, 4, True, 1100, 2),
+                                                      (11, 32, -32, 4, True, 2100, 3)])
 def test_cross_query_batch_matches_single_queries(logN, R, B, L, big, n_rows, nq):
     """Several queries against the same encoded blocks in one call: every query's partial sums are bit-identical to the
     oracle's multiply-accumulate with that query's baby set (and hence to the single-query call), and the scores
     decrypt within tolerance."""
     import torch
 
+    pair_b32 = B < 0   # two queries per pass at B = 32 as well (off by default: it does not pay there)
+    B = abs(B)
     ps = synth.ParamSet("b%d" % logN, logN, synth.Q50, synth.P60, 40, R, B, -18) if big else synth.small_params(logN, R, B, L=L)
     p = Pair(ps, key_seed=logN + 7)
     g, o, b = p.g, p.o, p.b
+    if pair_b32:
+        g.set_tuning(b.TUNE_PAIR_B32, 1)
     rows = synth.toy_corpus(logN, rows=n_rows, dim=R)
     nb = g.n_blocks(n_rows)
     pt = g.encode_candidates(torch_rows(p, rows), p.ws)

@@ -31,6 +31,29 @@ def test_every_declared_symbol_is_exported_and_bound(lib):
         assert f.argtypes is not None or n in ("hann_kernel_classes",), n
 
 
+def test_binding_constants_match_the_header():
+    """Every enumerator and #define of the header that the binding mirrors has the header's value (status codes, size and
+    kind selectors, tuning knobs, the prime-count limit)."""
+    src = open(os.path.join(ROOT, "include", "hann.h")).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    header = {n: int(v) for n, v in re.findall(r"\b(HANN_[A-Z0-9_]+)\s*=\s*(-?\d+)", src)}
+    header.update({n: int(v) for n, v in re.findall(r"#define\s+(HANN_[A-Z0-9_]+)\s+\(?(-?\d+)\)?", src)})
+    assert len(header) >= 25
+    mirrored = 0
+    for name, value in header.items():
+        short = name[len("HANN_"):]
+        for cand in (name, short, short[1:] if short.startswith("E") and short[1:] in ("INVAL", "SHAPE", "NOKEY", "WORKSPACE", "CUDA", "NOMEM") else None):
+            if cand and hasattr(binding, cand):
+                assert getattr(binding, cand) == value, (name, value, getattr(binding, cand))
+                mirrored += 1
+                break
+    assert mirrored >= 20
+    # every tuning knob of the header is mirrored
+    for name in header:
+        if name.startswith("HANN_TUNE_"):
+            assert hasattr(binding, name[len("HANN_"):]), name
+
+
 def test_parameter_validation_without_a_device(lib):
     ps = synth.small_params(8, 8, 4, L=2)
 

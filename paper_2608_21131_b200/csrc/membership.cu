@@ -11,7 +11,9 @@
 // Every ciphertext carries (level, scale); the scale arithmetic below is written operation by operation in IEEE binary64 so
 // that any evaluation of the same circuit in the same order gets the same integer constants.
 #include <cmath>
+#include <algorithm>
 #include <string>
+#include <utility>
 #include <vector>
 
 #include "internal.h"
@@ -105,17 +107,37 @@ struct Circuit {
         if (prod.p && rc == HANN_OK) ok(hann_multiply(at(l), a.p, b.p, a.n, prod.p, sub, sub_bytes), at(l));
         return rescale(prod);
     }
+    // several independent products on one level in ONE multiply and ONE rescale call: pairs[i] = (a_i, b_i), every pair with
+    // the same lower level; the operands are gathered into two rows of ciphertexts first.  Item i comes back with its own scale
+    // (a_i.scale b_i.scale / q_last), as mul() would have given it; the bits are mul()'s too (the items do not interact).
+    std::vector<MCt> mul_many(const std::vector<std::pair<MCt, MCt>>& pairs) {
+        const int64_t k = (int64_t)pairs.size();
+        std::vector<MCt> out((size_t)k);
+        if (k == 0 || rc != HANN_OK) return out;
+        int l = pairs[0].first.level < pairs[0].second.level ? pairs[0].first.level : pairs[0].second.level;
+        for (const auto& pr : pairs) {
+            const int li = pr.first.level < pr.second.level ? pr.first.level : pr.second.level;
+            if (li != l || pr.first.n != 1 || pr.second.n != 1) fail(HANN_EINVAL, "hann_membership_decide: internal level mismatch in a batch of products");
+        }
+        const int64_t ctw = 2LL * l * N;
+        MCt a{take(l, k), l, 0, k}, b{take(l, k), l, 0, k}, prod{take(l, k), l, 0, k};
+        if (!a.p || !b.p || !prod.p || rc != HANN_OK) return out;
+        for (int64_t i = 0; i < k && rc == HANN_OK; i++) {
+            const MCt &x = pairs[(size_t)i].first, &y = pairs[(size_t)i].second;
+            ok(launch_copy2d(at(l), a.p + i * ctw, (int64_t)l * N, x.p, (int64_t)x.level * N, (int64_t)l * N, 2), at(l));
+            ok(launch_copy2d(at(l), b.p + i * ctw, (int64_t)l * N, y.p, (int64_t)y.level * N, (int64_t)l * N, 2), at(l));
+        }
+        if (rc == HANN_OK) ok(hann_multiply(at(l), a.p, b.p, k, prod.p, sub, sub_bytes), at(l));
+        const MCt low = rescale(prod);
+        if (!low.p || rc != HANN_OK) return out;
+        const int64_t ctw_low = 2LL * (l - 1) * N;
+        for (int64_t i = 0; i < k; i++)
+            out[(size_t)i] = MCt{low.p + i * ctw_low, l - 1, (pairs[(size_t)i].first.scale * pairs[(size_t)i].second.scale) / prime(l - 1), 1};
+        return out;
+    }
     MCt rotate(const MCt& a, int r) {
         MCt o{take(a.level), a.level, a.scale};
         if (o.p) ok(hann_rotate_hoisted(at(a.level), a.p, r, 1, o.p, sub, sub_bytes), at(a.level));
-        return o;
-    }
-    // factor * value at (very nearly) target_scale one level down: integer-constant multiply, then rescale
-    MCt to_scale(const MCt& a, double factor, double target_scale) {
-        const double q = prime(a.level - 1);
-        const double m = std::nearbyint(((factor * target_scale) * q) / a.scale);
-        MCt o = rescale(mul_int(a, (long long)m));
-        o.scale = ((a.scale * m) / q) / factor;
         return o;
     }
 };
@@ -148,7 +170,7 @@ extern "C" int64_t hann_membership_bytes(hann_ctx* const* arith, int L, const ha
     while ((1 << folds) < prm->R) folds++;
     const int64_t cts = 16 + 12 * (int64_t)prm->deg + 2 * folds + n_blocks * (3 + 8 * (int64_t)prm->sign_iters);
     int64_t sub = 0;
-    for (int l = 1; l <= L; l++) sub = std::max<int64_t>(sub, hann_workspace_bytes(arith[l - 1], l < scorer->L ? n_blocks : 1));
+    for (int l = 1; l <= L; l++) sub = std::max<int64_t>(sub, hann_workspace_bytes(arith[l - 1], l < scorer->L ? std::max<int64_t>(n_blocks, 4) : 4));
     sub = std::max<int64_t>(sub, hann_workspace_bytes(scorer, 8));
     const int64_t scoring = align256(hann_sizeof(scorer, HANN_SIZE_BABY)) + n_blocks * (align256(hann_sizeof(scorer, HANN_SIZE_INNER)) +
                                                                                       align256(hann_sizeof(scorer, HANN_SIZE_CT)));
@@ -188,8 +210,9 @@ extern "C" int hann_membership_decide(hann_ctx* const* arith, int L, hann_ctx* s
 
     const int N = top->N;
     int64_t sub = 0;
-    // below the scorer's level the operations run over all blocks at once: room for several key switches side by side
-    for (int l = 1; l <= L; l++) sub = std::max<int64_t>(sub, hann_workspace_bytes(arith[l - 1], l < score_level ? n_blocks : 1));
+    // below the scorer's level the operations run over all blocks at once, above it over the up to four products of one depth of
+    // the Chebyshev basis: room for several key switches side by side
+    for (int l = 1; l <= L; l++) sub = std::max<int64_t>(sub, hann_workspace_bytes(arith[l - 1], l < score_level ? std::max<int64_t>(n_blocks, 4) : 4));
     sub = align256(std::max<int64_t>(sub, hann_workspace_bytes(scorer, 8)));
     Circuit C;
     C.arith = arith; C.L = L; C.top = top; C.N = N;
@@ -207,21 +230,56 @@ extern "C" int hann_membership_decide(hann_ctx* const* arith, int L, hann_ctx* s
     t.scale = t.scale / (lam * lam) * a;
     const MCt u = C.add_const(t, -(prm->t_hi + prm->t_lo) / (prm->t_hi - prm->t_lo));
     // 3: Chebyshev basis by the product identity, then the combination at one common scale
+    // (the products of one depth do not depend on each other: T_3, T_4 need T_1, T_2 only, T_5 .. T_7 need T_2 .. T_4; each depth
+    // is one batched multiply and rescale)
     std::vector<MCt> T(prm->deg + 1);
     T[1] = u;
-    for (int k = 2; k <= prm->deg; k++) {
-        const int m = (k + 1) / 2, nn = k - m;
-        const MCt prod2 = C.mul_int(C.mul(T[m], T[nn]), 2);
-        T[k] = m == nn ? C.add_const(prod2, -1.0) : C.add(prod2, T[m - nn], -1);
+    for (int k0 = 2; k0 <= prm->deg;) {
+        // the run of k whose operands T_ceil(k/2), T_floor(k/2) exist already: k0 .. min(deg, 2 (k0 - 1))
+        const int k1 = std::min(prm->deg, 2 * (k0 - 1));
+        std::vector<std::pair<MCt, MCt>> pairs;
+        for (int k = k0; k <= k1; k++) pairs.emplace_back(T[(k + 1) / 2], T[k - (k + 1) / 2]);
+        // a batch needs one common level; it has one whenever the run starts at a power of two plus one .. (checked by mul_many:
+        // the lower operand of every pair of a run lies on the run's deepest level); single products go through mul()
+        bool same = true;
+        for (const auto& pr : pairs) same = same && std::min(pr.first.level, pr.second.level) == std::min(pairs[0].first.level, pairs[0].second.level);
+        std::vector<MCt> prods;
+        if (same && pairs.size() > 1) prods = C.mul_many(pairs);
+        else for (const auto& pr : pairs) prods.push_back(C.mul(pr.first, pr.second));
+        if (C.rc != HANN_OK) return C.rc;
+        for (int k = k0; k <= k1; k++) {
+            const int m = (k + 1) / 2, nn = k - m;
+            const MCt prod2 = C.mul_int(prods[(size_t)(k - k0)], 2);
+            T[k] = m == nn ? C.add_const(prod2, -1.0) : C.add(prod2, T[m - nn], -1);
+        }
+        k0 = k1 + 1;
     }
     int level = T[1].level;
     for (int k = 1; k <= prm->deg; k++) level = T[k].level < level ? T[k].level : level;
     level -= 1;
+    // every term's integer multiple (to_scale) lands in one row of ciphertexts, which takes ONE rescale call
+    std::vector<int> ks;
+    for (int k = 1; k <= prm->deg; k++)
+        if (std::fabs(prm->coef[k]) >= 1e-15) ks.push_back(k);
     MCt acc;
-    for (int k = 1; k <= prm->deg; k++) {
-        if (std::fabs(prm->coef[k]) < 1e-15) continue;
-        const MCt term = C.to_scale(C.drop(T[k], level + 1), prm->coef[k], delta);
-        acc = acc.p ? C.add(acc, term, 1) : term;
+    if (!ks.empty() && C.rc == HANN_OK) {
+        const int lv = level + 1;
+        const int64_t nt = (int64_t)ks.size(), ctw = 2LL * lv * N, ctw_low = 2LL * level * N;
+        const double ql = C.prime(lv - 1);
+        MCt row{C.take(lv, nt), lv, 0, nt};
+        std::vector<double> scales((size_t)nt);
+        for (int64_t i = 0; i < nt && row.p && C.rc == HANN_OK; i++) {
+            const MCt a = C.drop(T[ks[(size_t)i]], lv);
+            const double factor = prm->coef[ks[(size_t)i]];
+            const double m = std::nearbyint(((factor * delta) * ql) / a.scale);   // as to_scale()
+            if (a.p) C.ok(launch_linear(C.at(lv), a.p, (long long)m, nullptr, 0, 0, 2, row.p + i * ctw), C.at(lv));
+            scales[(size_t)i] = ((a.scale * m) / ql) / factor;
+        }
+        const MCt low = C.rescale(row);
+        for (int64_t i = 0; i < nt && low.p && C.rc == HANN_OK; i++) {
+            const MCt term{low.p + i * ctw_low, level, scales[(size_t)i], 1};
+            acc = acc.p ? C.add(acc, term, 1) : term;
+        }
     }
     if (C.rc == HANN_OK && !acc.p) return bad(HANN_EINVAL, "hann_membership_decide: all polynomial coefficients vanish");
     const MCt thr = C.add_const(acc, prm->coef[0]);

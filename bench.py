@@ -598,6 +598,8 @@ def run_encrypted_db(args):
     ps, rows_np, qR, wname = build_workload(args.config, args.rows, args.logn)
     n_rows = rows_np.shape[0]
     ctx = binding.Context(ps, device=0)
+    if args.mac_f64 is not None:
+        ctx.set_tuning(binding.TUNE_MAC_F64, args.mac_f64)
     km = synth.key_material(ps, wl.KEY_SEED)
     ctx.load_keys(ctx.keygen_from_samples(km.s, km.rots, km.evk_a, km.evk_e), km.rots)
     ka = synth.uniform_residues(wl.KEY_SEED, 50, list(ps.q) + [ps.p], ps.N, lead=(ps.L,))

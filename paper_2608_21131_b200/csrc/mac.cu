@@ -230,24 +230,33 @@ __global__ void __launch_bounds__(32 * NG) k_mac_stream(const u64* __restrict__ 
 // the 25-bit halves of its BB baby-step words, both components, in registers), with the two polynomials x0, x1 of every
 // database ciphertext streamed past them one after the other: x_h * y_c adds to d_{h+c}, so the three degree-2 sums share
 // one set of Karatsuba accumulators and every database word is read once.
-template <int NG, int BB>
+template <int NG, int BB, bool F64>
 __global__ void __launch_bounds__(32 * NG) k_mac_ct_stream(const u64* __restrict__ baby, const u64* __restrict__ ctdb,
                                                            u64* __restrict__ inner3, int N, int L, long long n_bg, int bg_per_cta,
                                                            const LimbConst* __restrict__ lt) {
     constexpr int B = NG * BB;
-    __shared__ u64 part[2][NG][9][32];
+    // partial sums per thread: three Karatsuba triples, or (F64) the two-word binary64 sums of the four products x_h y_c
+    constexpr int PW = F64 ? 8 : 9;
+    static_assert(!F64 || BB <= 8, "the two-word binary64 sum holds eight products");
+    __shared__ u64 part[2][NG][PW][32];
     const long long LN = (long long)L * N;
     const long long pos0 = (long long)blockIdx.x * 32;
     const int lane = threadIdx.x & 31, wg = threadIdx.x >> 5;
     const LimbConst* lc = lt + pos0 / N;
     unsigned w0[BB][2], w1[BB][2];
+    double wd[BB][2];
+    const double qd = (double)lc->q, halfd = (double)lc->half;
 #pragma unroll
     for (int k = 0; k < BB; k++)
 #pragma unroll
         for (int c = 0; c < 2; c++) {
             const u64 v = baby[((long long)(wg * BB + k) * 2 + c) * LN + pos0 + lane];
-            w0[k][c] = (unsigned)v & kM25;
-            w1[k][c] = (unsigned)(v >> 25);
+            if (F64) {
+                wd[k][c] = residue_to_balanced_f64(v, qd, halfd);
+            } else {
+                w0[k][c] = (unsigned)v & kM25;
+                w1[k][c] = (unsigned)(v >> 25);
+            }
         }
     const long long bg0 = (long long)blockIdx.y * bg_per_cta;
     const long long bg1 = bg0 + bg_per_cta < n_bg ? bg0 + bg_per_cta : n_bg;
@@ -259,6 +268,7 @@ __global__ void __launch_bounds__(32 * NG) k_mac_ct_stream(const u64* __restrict
     for (int k = 0; k < BB; k++) cur[k] = __ldcs(p + (long long)k * 2 * LN);
     for (long long bg = bg0; bg < bg1; bg++) {
         u64 p00[3] = {0, 0, 0}, p11[3] = {0, 0, 0}, pm[3] = {0, 0, 0};
+        double ah[2][2] = {{kAcc2Start, kAcc2Start}, {kAcc2Start, kAcc2Start}}, al[2][2] = {{0, 0}, {0, 0}};
 #pragma unroll
         for (int h = 0; h < 2; h++) {
             // next stream element: the other polynomial of this pair, or x0 of the next pair
@@ -270,44 +280,79 @@ __global__ void __launch_bounds__(32 * NG) k_mac_ct_stream(const u64* __restrict
             }
 #pragma unroll
             for (int k = 0; k < BB; k++) {
-                const unsigned a0 = (unsigned)cur[k] & kM25, a1 = (unsigned)(cur[k] >> 25), as = a0 + a1;
+                if (F64) {
+                    const double x = residue_to_f64(cur[k]);
 #pragma unroll
-                for (int c = 0; c < 2; c++) {
-                    p00[h + c] += (u64)a0 * w0[k][c];
-                    p11[h + c] += (u64)a1 * w1[k][c];
-                    pm[h + c] += (u64)as * (w0[k][c] + w1[k][c]);
+                    for (int c = 0; c < 2; c++) acc2_fma(ah[h][c], al[h][c], x, wd[k][c]);
+                } else {
+                    const unsigned a0 = (unsigned)cur[k] & kM25, a1 = (unsigned)(cur[k] >> 25), as = a0 + a1;
+#pragma unroll
+                    for (int c = 0; c < 2; c++) {
+                        p00[h + c] += (u64)a0 * w0[k][c];
+                        p11[h + c] += (u64)a1 * w1[k][c];
+                        pm[h + c] += (u64)as * (w0[k][c] + w1[k][c]);
+                    }
                 }
             }
 #pragma unroll
             for (int k = 0; k < BB; k++) cur[k] = nxt[k];
         }
         p += (long long)B * 2 * LN;
-        u64(*buf)[9][32] = part[bg & 1];
+        u64(*buf)[PW][32] = part[bg & 1];
+        if (F64) {
 #pragma unroll
-        for (int c = 0; c < 3; c++) {
-            buf[wg][c * 3 + 0][lane] = p00[c];
-            buf[wg][c * 3 + 1][lane] = pm[c];
-            buf[wg][c * 3 + 2][lane] = p11[c];
+            for (int h = 0; h < 2; h++)
+#pragma unroll
+                for (int c = 0; c < 2; c++) {
+                    buf[wg][(h * 2 + c) * 2 + 0][lane] = (u64)acc2_high(ah[h][c]);
+                    buf[wg][(h * 2 + c) * 2 + 1][lane] = (u64)acc2_low(al[h][c]);
+                }
+        } else {
+#pragma unroll
+            for (int c = 0; c < 3; c++) {
+                buf[wg][c * 3 + 0][lane] = p00[c];
+                buf[wg][c * 3 + 1][lane] = pm[c];
+                buf[wg][c * 3 + 2][lane] = p11[c];
+            }
         }
         __syncthreads();
         for (int c = wg; c < 3; c += NG) {
-            u64 s00 = 0, sm = 0, s11 = 0;
+            u64 r;
+            if (F64) {
+                // d_c = sum over the warps of the products x_h y_(c-h): (0,0) | (0,1) + (1,0) | (1,1)
+                long long m = 0, sl = 0;
 #pragma unroll
-            for (int g = 0; g < NG; g++) {
-                s00 += buf[g][c * 3 + 0][lane];
-                sm += buf[g][c * 3 + 1][lane];
-                s11 += buf[g][c * 3 + 2][lane];
+                for (int g = 0; g < NG; g++) {
+                    if (c != 2) {
+                        m += (long long)buf[g][c * 2 + 0][lane];
+                        sl += (long long)buf[g][c * 2 + 1][lane];
+                    }
+                    if (c != 0) {
+                        m += (long long)buf[g][(c + 1) * 2 + 0][lane];
+                        sl += (long long)buf[g][(c + 1) * 2 + 1][lane];
+                    }
+                }
+                r = acc2_reduce(m, sl, *lc);
+            } else {
+                u64 s00 = 0, sm = 0, s11 = 0;
+#pragma unroll
+                for (int g = 0; g < NG; g++) {
+                    s00 += buf[g][c * 3 + 0][lane];
+                    sm += buf[g][c * 3 + 1][lane];
+                    s11 += buf[g][c * 3 + 2][lane];
+                }
+                // d1 sums 2 B products: B <= 64 keeps the 25-bit-half sums below 2^57 and the half-sum products below 2^59
+                const u64 cross = sm - s00 - s11;
+                u64 lo = s00, hi = 0;
+                const u64 c_lo = cross << 25, c_hi = cross >> 39;
+                lo += c_lo;
+                hi += c_hi + (lo < c_lo ? 1 : 0);
+                const u64 d_lo = s11 << 50, d_hi = s11 >> 14;
+                lo += d_lo;
+                hi += d_hi + (lo < d_lo ? 1 : 0);
+                r = reduce128(hi, lo, *lc);
             }
-            // d1 sums 2 B products: B <= 64 keeps the 25-bit-half sums below 2^57 and the half-sum products below 2^59
-            const u64 cross = sm - s00 - s11;
-            u64 lo = s00, hi = 0;
-            const u64 c_lo = cross << 25, c_hi = cross >> 39;
-            lo += c_lo;
-            hi += c_hi + (lo < c_lo ? 1 : 0);
-            const u64 d_lo = s11 << 50, d_hi = s11 >> 14;
-            lo += d_lo;
-            hi += d_hi + (lo < d_lo ? 1 : 0);
-            inner3[(bg * 3 + c) * LN + pos0 + lane] = reduce128(hi, lo, *lc);
+            inner3[(bg * 3 + c) * LN + pos0 + lane] = r;
         }
         if (NG < 3) __syncthreads();
     }
@@ -689,13 +734,25 @@ int launch_mac_ct(hann_ctx* c, const u64* baby, const u64* ctdb, int64_t n_bg, u
         split = (int)((n_bg + per - 1) / per);
         KProf kp(c, KC_MAC);
         const dim3 grid(tiles, split);
-        switch (c->B) {
-            case 4: k_mac_ct_stream<4, 1><<<grid, 128, 0, c->stream>>>(baby, ctdb, inner3, c->N, c->L, n_bg, per, c->lt_dev); break;
-            case 8: k_mac_ct_stream<4, 2><<<grid, 128, 0, c->stream>>>(baby, ctdb, inner3, c->N, c->L, n_bg, per, c->lt_dev); break;
-            case 16: k_mac_ct_stream<4, 4><<<grid, 128, 0, c->stream>>>(baby, ctdb, inner3, c->N, c->L, n_bg, per, c->lt_dev); break;
-            case 32: k_mac_ct_stream<4, 8><<<grid, 128, 0, c->stream>>>(baby, ctdb, inner3, c->N, c->L, n_bg, per, c->lt_dev); break;
-            case 64: k_mac_ct_stream<8, 8><<<grid, 256, 0, c->stream>>>(baby, ctdb, inner3, c->N, c->L, n_bg, per, c->lt_dev); break;
-            default: small = false; break;
+        auto go = [&](auto kern, int threads) { kern<<<grid, threads, 0, c->stream>>>(baby, ctdb, inner3, c->N, c->L, n_bg, per, c->lt_dev); };
+        if (c->mac_f64) {
+            switch (c->B) {
+                case 4: go(k_mac_ct_stream<4, 1, true>, 128); break;
+                case 8: go(k_mac_ct_stream<4, 2, true>, 128); break;
+                case 16: go(k_mac_ct_stream<4, 4, true>, 128); break;
+                case 32: go(k_mac_ct_stream<4, 8, true>, 128); break;
+                case 64: go(k_mac_ct_stream<8, 8, true>, 256); break;
+                default: small = false; break;
+            }
+        } else {
+            switch (c->B) {
+                case 4: go(k_mac_ct_stream<4, 1, false>, 128); break;
+                case 8: go(k_mac_ct_stream<4, 2, false>, 128); break;
+                case 16: go(k_mac_ct_stream<4, 4, false>, 128); break;
+                case 32: go(k_mac_ct_stream<4, 8, false>, 128); break;
+                case 64: go(k_mac_ct_stream<8, 8, false>, 256); break;
+                default: small = false; break;
+            }
         }
         if (small) return check_launch(c, "mac_ct_stream");
     }

@@ -113,8 +113,8 @@ __device__ __forceinline__ void acc2_fma(double& ah, double& al, double p, doubl
 // over several partial sums in 64-bit integers
 __device__ __forceinline__ long long acc2_high(double ah) { return __double2ll_rn(__dmul_rn(__dsub_rn(ah, kAcc2Start), 0x1p-51)); }
 __device__ __forceinline__ long long acc2_low(double al) { return __double2ll_rn(al); }
-// (m 2^51 + sl) mod q for the integer sums of up to 64 products' words: |m 2^51 + sl| < 32 q^2 < q 2^57 (q < 2^50), so adding
-// q 2^57 makes it a non-negative 128-bit integer
+// (m 2^51 + sl) mod q for the integer sums of the words of n <= 128 products: |m 2^51 + sl| < n q^2 / 2 < q 2^57 (q < 2^50),
+// so adding q 2^57 makes it a non-negative 128-bit integer
 __device__ __forceinline__ u64 acc2_reduce(long long m, long long sl, const LimbConst& c) {
     u64 lo = (u64)m << 51, hi = (u64)(m >> 13);
     const u64 s_lo = (u64)sl, s_hi = (u64)(sl >> 63);

@@ -111,8 +111,9 @@ def test_multiply_bit_exact(logN, L, count):
     c.sync()
     got_r = low.export(b.KIND_CT, res, count)
     assert np.array_equal(got_r, np.stack([o.compact(want[i], L - 1, rescale=True) for i in range(count)]))
-    # error paths
+    # error paths; an empty batch is not an error
     lib = b.load_library()
+    assert lib.hann_multiply(c.h, None, None, 0, None, None, 0) == b.OK
     assert lib.hann_multiply(c.h, b._ptr(xd), b._ptr(yd), -1, b._ptr(prod), b._ptr(ws), ws.numel() * 8) == b.EINVAL
     assert lib.hann_multiply(c.h, b._ptr(xd), b._ptr(yd), count, b._ptr(prod), b._ptr(ws), 1024) == b.EWORKSPACE
     nokey = b.Context(ps)

@@ -11,7 +11,8 @@ from paper_2608_21131_b200 import synth
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("logN,R,B,deg,iters,n_rows", [(10, 16, 4, 7, 3, 900), (9, 8, 2, 3, 1, 200), (9, 8, 2, 3, 2, 2500), (12, 32, 8, 7, 3, 2048)])
+@pytest.mark.parametrize("logN,R,B,deg,iters,n_rows", [(10, 16, 4, 7, 3, 900), (9, 8, 2, 3, 1, 200), (9, 8, 2, 3, 2, 2500), (12, 32, 8, 7, 3, 2048),
+                          (15, 128, 32, 7, 3, 16000)])   # the last: the ring, rank and baby steps of the benchmark's scan, one ragged block
 def test_membership_circuit_bit_exact(logN, R, B, deg, iters, n_rows):
     import torch
 
@@ -48,7 +49,7 @@ def test_membership_circuit_bit_exact(logN, R, B, deg, iters, n_rows):
     # inputs: a query near a planted row, candidates enrolled times kappa / lam
     rows = synth.toy_corpus(3, rows=n_rows, dim=R)
     rng = np.random.default_rng(2)
-    qR = rows[11] + 0.25 * rng.standard_normal(R)
+    qR = rows[11] + rng.standard_normal(R) / np.sqrt(R)   # noise of norm ~1 beside the unit row: cosine ~0.7 at every R
     qR = (0.7 * qR / np.linalg.norm(qR)).astype(np.float32)
     ct = top_o.encrypt(km.s, top_o.encode(m.query_slots(qR), 45), km.ct_a, km.ct_e)
     ct_dev = arith[L - 1].import_(b.KIND_CT, ct, 1)

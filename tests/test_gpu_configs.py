@@ -383,8 +383,8 @@ def test_projection_with_encrypted_matrix():
     """Rank reduction as the paper deploys it (Sec. 3.1 "How": the server holds W as ENCRYPTED diagonals, so that it never
     learns the projection): the same diagonal scorer with the encrypted block of W^T (ct x ct multiply-accumulate, one
     relinearisation per giant step, rotate-and-sum).  Bit-identical to the oracle; the slots of the result hold the
-    projected query, tiled.  (Window packing of the chunks and the 0/1 masks of the paper's storage optimisation are
-    not built: W^T is stored as one 512-diagonal block.)"""
+    projected query, tiled.  (Here W^T is stored as one 512-diagonal block; the window-packed form with its 0/1 masks
+    and single fold, matrix in plaintext, is test_packed_projection_then_scoring.)"""
     import torch
 
     ps = synth.ParamSet("proj", 13, synth.Q50, synth.P60, 40, 512, 32, -18)

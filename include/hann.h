@@ -286,7 +286,11 @@ int hann_score_level_ctdb(hann_ctx *ctx, const void *baby_dev, const void *ctdb_
  * Sec. 2: the encrypted database and the membership path need it): out[i] = (d0 + ks0, d1 + ks1), (d0, d1, d2) =
  * (a0 b0, a0 b1 + a1 b0, a1 b1) of pair i, (ks0, ks1) the key switch of d2 under the relinearisation key (rotation 0).
  * The scale of out is the product of the scales; hann_rescale follows in a circuit.  a_dev, b_dev, out_dev: count
- * ciphertexts each (internal layout); out may not alias a or b. */
+ * ciphertexts each (internal layout, device memory, caller-owned); a and b may be the same buffer, out may not alias either.
+ * Workspace: hann_workspace_bytes(ctx, 1) serves any count (the pairs then go through one at a time); with room for k
+ * products (hann_workspace_bytes(ctx, k), k <= 8) k key switches run side by side.  Errors: HANN_EINVAL (null pointer,
+ * negative count; count = 0 is a no-op), HANN_ESHAPE (a ciphertext prime of 2^62 or more), HANN_ENOKEY (no relinearisation
+ * key loaded as rotation 0), HANN_EWORKSPACE. */
 int hann_multiply(hann_ctx *ctx, const void *a_dev, const void *b_dev, int64_t count, void *out_dev, void *ws, size_t ws_bytes);
 
 /* Rotate-and-sum (Sec. 3.1 Detail: the giant steps of the diagonal method): score_ct[blk] = sum_g rot_{g*B}(inner[blk][g]), evaluated by Horner with the single key of
